@@ -1,0 +1,67 @@
+/*
+ * CPU oracle for the execution-plan search -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, single-threaded restatement of the paper's performance model and of
+ * the exhaustive search over recovery plans.  It shares no code with the CUDA path and
+ * is used only by the tests, the smoke check and the bench's CPU-baseline leg.
+ *
+ * Every function cites the passage of the paper it follows (section / equation /
+ * algorithm).  Where the paper is silent, the reading taken is stated at the function.
+ *
+ * Two numeric builds of the model exist side by side: suffix _f64 (IEEE double, one
+ * rounding per written operation, no contraction) and suffix _i64 (integer nanoseconds,
+ * every division floors).  Bytes are always int64.
+ */
+#ifndef ORC_H
+#define ORC_H
+
+#include <stdint.h>
+
+#define ORC_MAX_PIPES 16
+#define ORC_MAX_STAGES 64
+#define ORC_MAX_LAYERS 128
+
+enum { ORC_REROUTE = 0, ORC_REDUNDANT = 1, ORC_DYNPAR = 2 };
+enum { ORC_LAYERS_FULL = 0, ORC_LAYERS_REMAINDER = 1, ORC_LAYERS_MINMAX = 2 };
+enum { ORC_BATCH_FULL = 0, ORC_BATCH_REMAINDER = 1 };
+
+typedef struct {
+    int32_t L, n_dp, n_pp, n_micro;
+    const double *fwd_ns, *bwd_ns;       /* [L] per micro-batch            */
+    const int64_t *fwd_ns_i, *bwd_ns_i;  /* [L] same, integer nanoseconds  */
+    const int64_t *act_bytes, *param_bytes, *opt_bytes, *p2p_bytes; /* [L] */
+    const int32_t *base_cuts;            /* [n_pp+1]                       */
+    int64_t mem_capacity_bytes;
+    int32_t devices_per_node;
+    int64_t bw_intra, bw_inter;          /* bytes per nanosecond           */
+} orc_profile;
+
+typedef struct {
+    int32_t dp_lo, dp_hi, pp_lo, pp_hi;
+    int32_t layer_mode, batch_mode;
+    uint64_t kappa_cap;
+} orc_opts;
+
+typedef struct {
+    int32_t policy, feasible;
+    double cost;      /* _f64 build; 0 in the _i64 build */
+    int64_t cost_ns;  /* _i64 build; 0 in the _f64 build */
+    uint32_t strategy, n_pipes;
+    uint64_t split_rank;
+    uint16_t stages[ORC_MAX_PIPES], micro[ORC_MAX_PIPES];
+    uint64_t kappa[ORC_MAX_PIPES];
+} orc_plan;
+
+/* ---- orc_enum.c: integer combinatorics (no cost arithmetic) ---- */
+uint64_t orc_binom(int n, int k);                       /* saturates at UINT64_MAX */
+void orc_unrank_subset(uint64_t rank, int t, int *c);   /* colex, c[0]<...<c[t-1]  */
+uint64_t orc_rank_subset(int t, const int *c);
+int orc_strategies(int n_surv, int dp_lo, int dp_hi, int pp_lo, int pp_hi, int L,
+                   int max_out, int32_t *dp_out, int32_t *stages_out /* [max_out][ORC_MAX_PIPES] */);
+uint64_t orc_split_count(int batch_mode, int G, int n_surv, int dp, const int32_t *stages);
+int orc_split_unrank(int batch_mode, int G, int n_surv, int dp, const int32_t *stages,
+                     uint64_t beta, int32_t *micro_out);
+uint64_t orc_layer_count(int layer_mode, int L, int S);  /* K of the enumerated part  */
+void orc_layer_unrank(int layer_mode, int L, int S, uint64_t kappa, int32_t *cuts_out /* [S+1] */);
+
+#endif
