@@ -1,0 +1,216 @@
+/*
+ * chameleon.h -- C ABI of the B200-native execution-plan search.
+ *
+ * The library answers the question the paper's decision center answers when a device
+ * fails (Chameleon, Section "Performance Modeling": given the current state, determine
+ * the next execution plan with the least step time; Section "Planner", Algorithm 1):
+ * enumerate the candidate recovery plans under each backup-free policy -- data
+ * rerouting, redundant computation, dynamic parallelism -- evaluate the unified
+ * performance model (Section "Estimator": step time and peak memory) on every
+ * candidate, and return the feasible plan with the least estimated iteration time.
+ *
+ * Everything is computed by hand-written CUDA kernels for sm_100a on the stream given
+ * to cm_create; the host side only builds small descriptor tables (strategies,
+ * segments) from the failure set.  There is no CPU fallback: without an sm_100 device
+ * cm_create fails with CM_ECUDA.
+ *
+ * Conventions
+ *  - Every call returns a cm_status and never throws, aborts or prints.  On error the
+ *    out-parameters are untouched; cm_last_error(ctx) holds a message.
+ *  - "HOST" / "DEVICE" at a pointer says where the memory lives.  The caller owns every
+ *    buffer it passes; the library owns cm_ctx and cm_space objects until they are
+ *    destroyed / freed.
+ *  - All device work is enqueued on the context's stream.  Calls that return results to
+ *    the host (cm_select, cm_search_batch, cm_decode_plan) synchronise that stream
+ *    before returning; cm_load_profile, cm_enumerate and cm_evaluate only enqueue.
+ *  - A cm_ctx is not thread-safe; distinct contexts are independent.
+ *  - Times are nanoseconds, sizes are bytes, bandwidths are bytes per nanosecond
+ *    (numerically GB/s).  Device d of the fault-free N_dp x N_pp grid is stage
+ *    d mod N_pp of pipeline d / N_pp and sits on node d / devices_per_node.
+ */
+#ifndef CHAMELEON_H
+#define CHAMELEON_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CM_MAX_PIPES 16    /* data-parallel pipelines of a plan            */
+#define CM_MAX_STAGES 64   /* stages of one pipeline                       */
+#define CM_MAX_LAYERS 128  /* model layers in a profile                    */
+#define CM_MAX_MICRO 4096  /* global micro-batches per iteration (N_dp*N_m) */
+
+typedef struct cm_ctx cm_ctx;     /* device buffers, profile copy, tables               */
+typedef struct cm_space cm_space; /* implicit candidate space of one (policy, failure set) */
+
+typedef enum {
+    CM_OK = 0,
+    CM_EINVAL = 1,      /* bad argument (message says which)                         */
+    CM_ENOPROFILE = 2,  /* cm_load_profile has not been called                       */
+    CM_EOVERFLOW = 3,   /* a candidate / split count does not fit the index type     */
+    CM_ENOFEASIBLE = 4, /* cm_select: no feasible plan in the given spaces           */
+    CM_ECUDA = 5,       /* CUDA runtime error or no sm_100 device                    */
+    CM_ENOMEM = 6,
+    CM_ETIMEOUT = 7     /* reserved: no kernel of this library waits on another      */
+} cm_status;
+
+/* Policies in ascending order of transition cost (Section "Performance Modeling":
+ * rerouting needs no reconstruction, dynamic parallelism moves weights and restarts),
+ * so that breaking a cost tie by the lowest id picks the cheapest transition. */
+typedef enum { CM_REROUTE = 0, CM_REDUNDANT = 1, CM_DYNPAR = 2 } cm_policy;
+
+/* Arithmetic of the time estimator: IEEE double with one rounding per operation of the
+ * model, or integer nanoseconds where every division floors (fully reproducible). */
+typedef enum { CM_COST_FP64 = 0, CM_COST_INT64NS = 1 } cm_cost_mode;
+
+/* Layer distribution (Section "Planner"): FULL = every composition of the L layers into
+ * S non-empty stages; REMAINDER = even split, then every placement of the L mod S
+ * leftover layers (C(S, L mod S) of them, the paper's rule); MINMAX = only the
+ * contiguous partition that minimises the largest stage time.  FULL and REMAINDER add
+ * that min-max partition as one more candidate per pipeline. */
+typedef enum { CM_LAYERS_FULL = 0, CM_LAYERS_REMAINDER = 1, CM_LAYERS_MINMAX = 2 } cm_layer_mode;
+
+/* Micro-batch distribution (Section "Planner"): REMAINDER = proportional to the nodes
+ * of each pipeline, every way of handing out the leftover micro-batches one each;
+ * FULL = every composition of the global micro-batch count into positive parts. */
+typedef enum { CM_BATCH_FULL = 0, CM_BATCH_REMAINDER = 1 } cm_batch_mode;
+
+/* The profile the paper's profiler delivers (Section "System Design", monitoring:
+ * execution time, HBM usage, parallel configuration) plus the link tiers.  All pointers
+ * are HOST memory and are copied by cm_load_profile. */
+typedef struct {
+    int32_t L, n_dp, n_pp, n_micro;     /* layers; fault-free grid; micro-batches per pipeline */
+    const double *fwd_ns, *bwd_ns;      /* [L] time per micro-batch (fp64 mode)                */
+    const int64_t *fwd_ns_i, *bwd_ns_i; /* [L] the same in whole nanoseconds (int64 mode)      */
+    const int64_t *act_bytes;           /* [L] activations stored per in-flight micro-batch    */
+    const int64_t *param_bytes;         /* [L] parameters; gradients take the same             */
+    const int64_t *opt_bytes;           /* [L] optimizer state                                 */
+    const int64_t *p2p_bytes;           /* [L] bytes crossing a stage boundary after layer l   */
+    const int32_t *base_cuts;           /* [n_pp+1] fault-free layer->stage cuts, 0 .. L       */
+    int64_t mem_capacity_bytes;         /* per device                                          */
+    int32_t devices_per_node;
+    int64_t bw_intra_Bpns, bw_inter_Bpns;
+} cm_profile;
+
+/* Search window (Algorithm 1 inputs R_dp, R_pp) and enumeration modes.  A pipeline whose
+ * enumerated layer compositions outnumber kappa_cap contributes only its min-max
+ * partition. */
+typedef struct {
+    int32_t dp_lo, dp_hi, pp_lo, pp_hi;
+    cm_layer_mode lm;
+    cm_batch_mode bm;
+    uint64_t kappa_cap;
+    cm_cost_mode cost;
+} cm_enum_opts;
+
+/* An execution plan (Definition 1: policy, parallel configuration, data distribution,
+ * layer distribution).  stages[p], micro[p], kappa[p] describe pipeline p: its stage
+ * count, its micro-batches per iteration and the rank of its layer composition (for
+ * CM_DYNPAR; kappa equal to the enumerated count means the min-max partition).
+ * cost is filled in fp64 mode, cost_ns in int64 mode; the other is 0. */
+typedef struct {
+    int32_t policy, feasible;
+    double cost;
+    int64_t cost_ns;
+    uint32_t strategy, n_pipes;
+    uint64_t split_rank;
+    uint16_t stages[CM_MAX_PIPES], micro[CM_MAX_PIPES];
+    uint64_t kappa[CM_MAX_PIPES];
+} cm_plan;
+
+/* Create a context on a CUDA device.  cuda_stream is a cudaStream_t owned by the caller
+ * (NULL = the default stream); all work of this context is enqueued on it.
+ * CM_ECUDA if the device is not compute capability 10.x. */
+cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream);
+cm_status cm_destroy(cm_ctx *ctx);
+
+/* Copy a profile to the device and build the per-layer prefix sums the estimators read
+ * (Section "Estimator": stage time and stage memory are sums over the stage's layers).
+ * Validates: 1 <= L <= CM_MAX_LAYERS, 1 <= n_pp <= min(L, CM_MAX_STAGES),
+ * 1 <= n_dp <= CM_MAX_PIPES, n_dp*n_micro <= CM_MAX_MICRO, finite non-negative times,
+ * non-negative bytes, positive bandwidths and capacity, base_cuts strictly increasing
+ * from 0 to L.  May be called again to replace the profile. */
+cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *profile);
+
+/* Describe the candidate space of one policy for one failure set (HOST failed_ids,
+ * distinct, each < n_dp*n_pp; n_failed may be 0).  For CM_DYNPAR the space is
+ * (Section "Planner"): every strategy (dp, S_1<=...<=S_dp) that uses all survivors
+ * within the window, every micro-batch split, every layer composition per pipeline;
+ * *n_candidates counts pipeline-plans (strategy, pipeline, micro-batch count, layer
+ * composition) in segment-major order.  CM_REROUTE and CM_REDUNDANT have one candidate.
+ * Nothing is stored per candidate: plans are unranked from their index on the device.
+ * opts may be NULL for the one-candidate policies (fp64 is then assumed). */
+cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids, int32_t n_failed,
+                       const cm_enum_opts *opts, cm_space **out, uint64_t *n_candidates);
+
+/* Evaluate candidates first .. first+count-1 of a space, or the count indices listed in
+ * DEVICE idx_dev (NULL = contiguous).  Writes, for each, the pipeline cost (pipeline
+ * time by the start/end recurrence of Section "Estimator" plus gradient-sync time) and
+ * the memory-feasibility flag (peak-memory formula of Section "Estimator") into the
+ * caller's DEVICE buffers; any of them may be NULL.  Infeasible candidates get
+ * +infinity / INT64_MAX and flag 0; that is not an error.  cost_dev is written in fp64
+ * mode, cost_ns_dev in int64 mode (the other buffer is left untouched).  Enqueues only. */
+cm_status cm_evaluate(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64_t count,
+                      const uint64_t *idx_dev, double *cost_dev, int64_t *cost_ns_dev,
+                      uint8_t *feasible_dev);
+
+/* Search the given spaces (Algorithm 1, get_execution_plan: keep the plan with the
+ * least estimated time; step time = slowest pipeline) and write the best plan to HOST
+ * *best: least cost, ties to the lexicographically smallest plan tuple within a policy
+ * and to the lowest policy id across policies.  CM_ENOFEASIBLE (best->feasible = 0) if
+ * nothing fits in memory.  All spaces must share one cost mode.  Synchronises. */
+cm_status cm_select(cm_ctx *ctx, cm_space *const *spaces, int32_t n_spaces, cm_plan *best);
+
+/* Layer cuts of every pipeline of a plan found in this space, concatenated into HOST
+ * cuts_out (sum over pipelines of stages[p]+1 entries, each pipeline 0 .. L). */
+cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan, int32_t *cuts_out);
+
+cm_status cm_space_free(cm_space *space);
+
+/* The whole search for B failure sets in one launch sequence (the paper pre-computes
+ * the plans for potential failure scenarios, Section "Planner"): scenario b fails
+ * failed_ids[offsets[b] .. offsets[b+1]-1] (HOST).  All three policies are searched for
+ * every scenario.  best_per_scenario: HOST [B]; best_per_policy: HOST [B*3] or NULL;
+ * a scenario without a feasible plan gets feasible = 0 and the call still returns
+ * CM_OK.  If latency_us (HOST [B]) is not NULL the scenarios are searched one at a
+ * time and latency_us[b] is the wall time of scenario b from descriptor build to its
+ * plan on the host; results are identical either way.  Synchronises. */
+cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                          const cm_enum_opts *opts, cm_plan *best_per_scenario,
+                          cm_plan *best_per_policy, float *latency_us);
+
+/* The same search split in two, for callers that search one set of scenarios repeatedly
+ * (and for timing the kernels with the descriptors already resident in device memory):
+ * cm_batch_prepare builds the descriptor tables of B failure sets, copies them to the
+ * device and computes the min-max partitions they need; cm_batch_search runs the launch
+ * sequence over a prepared batch and returns the plans as cm_search_batch does
+ * (synchronises); cm_batch_free releases it.  A batch belongs to the profile that was
+ * loaded when it was prepared. */
+typedef struct cm_batch cm_batch;
+cm_status cm_batch_prepare(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                           const cm_enum_opts *opts, cm_batch **out, uint64_t *n_candidates);
+cm_status cm_batch_search(cm_ctx *ctx, cm_batch *batch, cm_plan *best_per_scenario,
+                          cm_plan *best_per_policy);
+cm_status cm_batch_free(cm_batch *batch);
+
+/* Work counters of the last cm_select / cm_search_batch / cm_batch_search on this
+ * context (HOST out[16]):
+ *  [0] pipeline-plans evaluated by the search pass   [1] recurrence cells simulated by it
+ *      (2 * stages * micro-batches per memory-feasible plan, counted on the device)
+ *  [2] pipeline-plans re-evaluated by the tie-break pass   [3] kernels launched
+ *  [4] device time of the whole launch sequence, ns (CUDA events on the context's stream)
+ *  [5] segments  [6] strategies  [7] micro-batch splits reduced
+ *  [8] device time of the search-pass cost kernel(s) alone, ns   [9] bytes copied host->device
+ *  [10] bytes copied device->host   [11] device time of the tie-break kernel(s), ns
+ *  [12] launches of the search-pass cost kernel   [13..15] reserved (0). */
+cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]);
+
+const char *cm_strerror(cm_status status);
+const char *cm_last_error(const cm_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHAMELEON_H */

@@ -1,0 +1,853 @@
+// C ABI of the plan search: context, profile upload, host-side descriptor builder
+// (strategies, segments, survivor placement) and the launch sequences.
+//
+// The host never evaluates the cost model.  It only turns a failure set into small
+// integer tables -- which (dp, S_1<=...<=S_dp) strategies exist, which survivor sits
+// on which stage, how many layer compositions each pipeline has -- and the kernels in
+// cm_kernels.cu do the rest from plan indices.
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "cm_internal.h"
+
+using namespace cm;
+
+// ------------------------------------------------------------------ small utilities
+namespace {
+
+template <typename T> struct PinnedVec {   // host staging that async copies can read
+    T *p = nullptr;
+    size_t n = 0, cap = 0;
+    ~PinnedVec() { if (p) cudaFreeHost(p); }
+    bool reserve(size_t want) {
+        if (want <= cap) return true;
+        size_t nc = std::max(want, cap * 2 + 16);
+        T *q = nullptr;
+        if (cudaHostAlloc((void **)&q, nc * sizeof(T), cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (n) memcpy(q, p, n * sizeof(T));
+        if (p) cudaFreeHost(p);
+        p = q;
+        cap = nc;
+        return true;
+    }
+    bool push(const T &v) { if (n == cap && !reserve(n + 1)) return false; p[n++] = v; return true; }
+    bool resize(size_t m) { if (!reserve(m)) return false; n = m; return true; }
+    void clear() { n = 0; }
+    T &operator[](size_t i) { return p[i]; }
+    const T &operator[](size_t i) const { return p[i]; }
+    size_t size() const { return n; }
+    T &back() { return p[n - 1]; }
+};
+
+template <typename T> struct DevBuf {
+    T *p = nullptr;
+    size_t cap = 0;
+    ~DevBuf() { if (p) cudaFree(p); }
+    bool reserve(size_t want) {
+        if (want <= cap) return true;
+        size_t nc = std::max(want, cap + cap / 2 + 16);
+        T *q = nullptr;
+        if (cudaMalloc((void **)&q, nc * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (p) cudaFree(p);
+        p = q;
+        cap = nc;
+        return true;
+    }
+};
+
+inline uint64_t sat_add(uint64_t a, uint64_t b) { return a > kSat - b ? kSat : a + b; }
+
+}  // namespace
+
+// One batch of failure scenarios: host tables, device mirrors, result buffers.
+struct Batch {
+    PinnedVec<Scen> scen;
+    PinnedVec<Strat> strat;
+    PinnedVec<Seg> seg;
+    PinnedVec<uint32_t> failed, red_scen, keys;
+    PinnedVec<cm_plan> plans_host;
+    PinnedVec<unsigned long long> counters_host;
+    DevBuf<Scen> d_scen;
+    DevBuf<Strat> d_strat;
+    DevBuf<Seg> d_seg;
+    DevBuf<uint32_t> d_failed, d_red_scen, d_keys;
+    DevBuf<uint64_t> d_seg_best, d_kappa_sel, d_pol_cost;
+    DevBuf<Partial> d_partial;
+    DevBuf<Winner> d_winner;
+    DevBuf<uint16_t> d_rc_stages;
+    DevBuf<cm_plan> d_plans;
+    DevBuf<unsigned long long> d_counters;
+    cm_enum_opts opts{};
+    uint32_t policy_mask = 0;
+    uint64_t n_cand = 0, n_tiles = 0, n_split = 0;
+    uint32_t max_tiles_per_seg = 0, dp_max = 0;
+    int B = 0;
+    bool uploaded = false;
+};
+
+struct cm_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    bool has_profile = false;
+    DevProfile hp{};                  // host copy: scalars, raw inputs, base cuts
+    DevProfile *d_prof = nullptr;
+    std::vector<uint64_t> binom;      // [rows][kBinomCols+1]
+    int binom_rows = 0;
+    uint64_t *d_binom = nullptr;
+    uint8_t *d_mm[2] = {nullptr, nullptr};   // min-max cuts per cost mode
+    std::vector<uint8_t> mm_done[2];
+    int mm_stride_m = 0;
+    Batch batch;                      // reused by cm_search_batch
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    uint64_t stats[16] = {0};
+    std::string err;
+};
+
+struct cm_space {
+    cm_ctx *ctx = nullptr;
+    int policy = 0;
+    Batch batch;
+    std::vector<uint32_t> failed;
+    std::vector<int> strat_dp;                    // decode: pipelines per strategy
+};
+
+struct cm_batch {
+    cm_ctx *ctx = nullptr;
+    Batch batch;
+    int prep_launches = 0;
+};
+
+namespace {
+
+cm_status fail(cm_ctx *c, cm_status s, const std::string &msg) {
+    if (c) c->err = msg;
+    return s;
+}
+
+#define CM_CUDA(ctx, expr)                                                                       \
+    do {                                                                                         \
+        cudaError_t e_ = (expr);                                                                 \
+        if (e_ != cudaSuccess) {                                                                 \
+            cudaGetLastError();                                                                  \
+            return fail((ctx), CM_ECUDA, std::string(#expr) + ": " + cudaGetErrorString(e_));    \
+        }                                                                                        \
+    } while (0)
+
+uint64_t hbinom(const cm_ctx *c, int n, int k) {
+    if (k < 0 || n < 0 || k > n) return 0;
+    if (n >= c->binom_rows || k > kBinomCols) return kSat;
+    return c->binom[(size_t)n * (kBinomCols + 1) + k];
+}
+
+// Strategies (Algorithm 1, get_parallel_strategy): non-decreasing stage counts that use
+// every survivor, dp ascending, tuples in lexicographic order.
+void enum_strategies(int n_surv, int dp_lo, int dp_hi, int lo, int hi,
+                     std::vector<std::vector<uint16_t>> &out) {
+    std::vector<uint16_t> cur;
+    struct Rec {
+        static void go(int dp, int pos, int remaining, int min_part, int hi, std::vector<uint16_t> &cur,
+                       std::vector<std::vector<uint16_t>> &out) {
+            if (pos == dp) {
+                if (remaining == 0) out.push_back(cur);
+                return;
+            }
+            const int left = dp - pos - 1;
+            for (int s = min_part; s <= hi; ++s) {
+                if (remaining - s < left * s) break;            // later parts are >= s
+                if (remaining - s > left * hi) continue;        // later parts are <= hi
+                cur.push_back((uint16_t)s);
+                go(dp, pos + 1, remaining - s, s, hi, cur, out);
+                cur.pop_back();
+            }
+        }
+    };
+    for (int dp = dp_lo; dp <= dp_hi; ++dp) Rec::go(dp, 0, n_surv, lo, hi, cur, out);
+}
+
+cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
+    if (!o) return fail(ctx, CM_EINVAL, "opts is NULL");
+    if (o->dp_lo > o->dp_hi || o->pp_lo > o->pp_hi) return fail(ctx, CM_EINVAL, "empty dp/pp window");
+    if (o->dp_hi > CM_MAX_PIPES) return fail(ctx, CM_EINVAL, "dp_hi exceeds CM_MAX_PIPES");
+    if (o->pp_hi > CM_MAX_STAGES) return fail(ctx, CM_EINVAL, "pp_hi exceeds CM_MAX_STAGES");
+    if (o->lm < CM_LAYERS_FULL || o->lm > CM_LAYERS_MINMAX) return fail(ctx, CM_EINVAL, "bad layer mode");
+    if (o->bm < CM_BATCH_FULL || o->bm > CM_BATCH_REMAINDER) return fail(ctx, CM_EINVAL, "bad batch mode");
+    if (o->cost < CM_COST_FP64 || o->cost > CM_COST_INT64NS) return fail(ctx, CM_EINVAL, "bad cost mode");
+    return CM_OK;
+}
+
+// Build the descriptor tables of a batch on the host.
+cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const int32_t *offsets, int B,
+                      const cm_enum_opts &o, uint32_t policy_mask) {
+    const DevProfile &hp = ctx->hp;
+    const int N = hp.n_dp * hp.n_pp, L = hp.L, G = hp.G;
+    bt.scen.clear(); bt.strat.clear(); bt.seg.clear(); bt.failed.clear(); bt.red_scen.clear(); bt.keys.clear();
+    bt.opts = o;
+    bt.policy_mask = policy_mask;
+    bt.n_cand = bt.n_tiles = bt.n_split = 0;
+    bt.max_tiles_per_seg = 0;
+    bt.dp_max = 0;
+    bt.B = B;
+    bt.uploaded = false;
+    const int mode = o.cost;
+    std::vector<uint8_t> &mm_done = ctx->mm_done[mode];
+    std::vector<char> dead(N);
+    std::vector<int> surv;
+    std::vector<std::vector<uint16_t>> strategies;
+    const int dp_lo = std::max(1, (int)o.dp_lo), dp_hi = std::min((int)o.dp_hi, CM_MAX_PIPES);
+    const int pp_lo = std::max(1, (int)o.pp_lo), pp_hi = std::min(std::min((int)o.pp_hi, L), CM_MAX_STAGES);
+    uint32_t red_blocks = 0;
+
+    for (int b = 0; b < B; ++b) {
+        const int f0 = offsets[b], f1 = offsets[b + 1];
+        if (f1 < f0) return fail(ctx, CM_EINVAL, "offsets must be non-decreasing");
+        std::fill(dead.begin(), dead.end(), 0);
+        Scen sc{};
+        sc.failed_first = (uint32_t)bt.failed.size();
+        sc.n_failed = (uint32_t)(f1 - f0);
+        for (int f = f0; f < f1; ++f) {
+            const uint32_t d = failed_ids[f];
+            if (d >= (uint32_t)N) return fail(ctx, CM_EINVAL, "failed device id out of range");
+            if (dead[d]) return fail(ctx, CM_EINVAL, "failed device ids must be distinct");
+            dead[d] = 1;
+            if (!bt.failed.push(d)) return fail(ctx, CM_ENOMEM, "host memory");
+        }
+        sc.policy_mask = policy_mask;
+        sc.strat_first = (uint32_t)bt.strat.size();
+        sc.seg_first = (uint32_t)bt.seg.size();
+        sc.red_first = red_blocks;
+        if (policy_mask & (1u << CM_DYNPAR)) {
+            surv.clear();
+            for (int d = 0; d < N; ++d)
+                if (!dead[d]) surv.push_back(d);
+            const int n_surv = (int)surv.size();
+            strategies.clear();
+            if (n_surv > 0 && pp_lo <= pp_hi) enum_strategies(n_surv, dp_lo, dp_hi, pp_lo, pp_hi, strategies);
+            uint64_t split_first = 0;
+            for (const auto &tuple : strategies) {
+                Strat st{};
+                const int dp = (int)tuple.size();
+                st.dp = (uint16_t)dp;
+                st.seg_first = (uint32_t)bt.seg.size();
+                st.split_first = split_first;
+                bt.dp_max = std::max<uint32_t>(bt.dp_max, (uint32_t)dp);
+                int sum = 0;
+                for (int p = 0; p < dp; ++p) {
+                    st.S[p] = tuple[p];
+                    if (o.bm == CM_BATCH_REMAINDER) {
+                        st.m_lo[p] = (uint16_t)(((int64_t)G * tuple[p]) / n_surv);
+                        sum += st.m_lo[p];
+                    } else {
+                        st.m_lo[p] = 1;
+                    }
+                }
+                if (o.bm == CM_BATCH_REMAINDER) {
+                    st.R = (uint16_t)(G - sum);
+                    st.n_m = st.R > 0 ? 2 : 1;
+                    st.n_split = hbinom(ctx, dp, st.R);
+                } else {
+                    st.R = 0;
+                    st.n_m = (uint16_t)(G >= dp ? G - dp + 1 : 0);
+                    st.n_split = G >= dp ? hbinom(ctx, G - 1, dp - 1) : 0;
+                }
+                if (st.n_split == kSat) return fail(ctx, CM_EOVERFLOW, "micro-batch split count overflows 64 bits");
+                split_first = sat_add(split_first, st.n_split);
+                if (split_first >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "too many micro-batch splits");
+                int off = 0;
+                for (int p = 0; p < dp; ++p) {
+                    const int S = tuple[p];
+                    uint64_t tier = 0;
+                    for (int i = 0; i + 1 < S; ++i)
+                        if (surv[off + i] / hp.devices_per_node != surv[off + i + 1] / hp.devices_per_node)
+                            tier |= 1ull << i;
+                    uint64_t K = 0;
+                    if (o.lm == CM_LAYERS_REMAINDER) K = hbinom(ctx, S, L % S);
+                    else if (o.lm == CM_LAYERS_FULL) K = hbinom(ctx, L - 1, S - 1);
+                    if (o.lm == CM_LAYERS_MINMAX || K > o.kappa_cap) K = 0;
+                    if (K >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "layer composition count overflows");
+                    for (int mi = 0; mi < st.n_m; ++mi) {
+                        Seg g{};
+                        g.S = (uint16_t)S;
+                        g.m = (uint16_t)(st.m_lo[p] + mi);
+                        g.n_sync = (uint16_t)dp;
+                        g.pipe = (uint16_t)p;
+                        g.K = K;
+                        g.tier_mask = tier;
+                        g.strat = (uint32_t)bt.strat.size();
+                        g.scen = (uint32_t)b;
+                        g.row = (uint32_t)bt.seg.size();
+                        g.cand_first = bt.n_cand;
+                        g.tile_first = bt.n_tiles;
+                        g.mm_slot = (uint32_t)((S - 1) * ctx->mm_stride_m + g.m);
+                        const uint64_t count = K ? K + 1 : 1;
+                        const uint64_t tiles = (count + kTile - 1) / kTile;
+                        bt.n_cand = sat_add(bt.n_cand, count);
+                        bt.n_tiles += tiles;
+                        if (bt.n_cand >= (1ull << 62) || bt.n_tiles >= (1ull << 44))
+                            return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
+                        bt.max_tiles_per_seg = (uint32_t)std::max<uint64_t>(bt.max_tiles_per_seg, std::min<uint64_t>(tiles, 0x7fffffffu));
+                        if (tiles > 0x7fffffffu) return fail(ctx, CM_EOVERFLOW, "segment too large");
+                        if (g.m >= 1 && !mm_done[g.mm_slot]) {
+                            mm_done[g.mm_slot] = 1;
+                            if (!bt.keys.push(((uint32_t)S << 16) | g.m)) return fail(ctx, CM_ENOMEM, "host memory");
+                        }
+                        if (!bt.seg.push(g)) return fail(ctx, CM_ENOMEM, "host memory");
+                    }
+                    off += S;
+                }
+                if (!bt.strat.push(st)) return fail(ctx, CM_ENOMEM, "host memory");
+            }
+            sc.n_split_total = split_first;
+            bt.n_split += split_first;
+        }
+        sc.n_strat = (uint32_t)bt.strat.size() - sc.strat_first;
+        sc.n_seg = (uint32_t)bt.seg.size() - sc.seg_first;
+        sc.n_red = sc.n_split_total ? (uint32_t)std::min<uint64_t>((sc.n_split_total + 1023) / 1024, 64) : 0;
+        for (uint32_t r = 0; r < sc.n_red; ++r)
+            if (!bt.red_scen.push((uint32_t)b)) return fail(ctx, CM_ENOMEM, "host memory");
+        red_blocks += sc.n_red;
+        if (!bt.scen.push(sc)) return fail(ctx, CM_ENOMEM, "host memory");
+    }
+    return CM_OK;
+}
+
+template <typename T>
+cm_status upload(cm_ctx *ctx, DevBuf<T> &d, const PinnedVec<T> &h) {
+    if (!d.reserve(std::max<size_t>(h.size(), 1))) return fail(ctx, CM_ENOMEM, "device memory");
+    if (h.size()) CM_CUDA(ctx, cudaMemcpyAsync(d.p, h.p, h.size() * sizeof(T), cudaMemcpyHostToDevice, ctx->stream));
+    ctx->stats[9] += h.size() * sizeof(T);
+    return CM_OK;
+}
+
+BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
+    BatchDev v{};
+    v.scen = bt.d_scen.p; v.strat = bt.d_strat.p; v.seg = bt.d_seg.p; v.failed = bt.d_failed.p;
+    v.seg_best = bt.d_seg_best.p; v.red_scen = bt.d_red_scen.p; v.partial = bt.d_partial.p;
+    v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
+    v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p; v.counters = bt.d_counters.p;
+    v.B = bt.B; v.mode = bt.opts.cost;
+    v.n_seg = (uint32_t)bt.seg.size(); v.n_strat = (uint32_t)bt.strat.size();
+    v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
+    v.n_red_blocks = (uint32_t)bt.red_scen.size(); v.dp_max = bt.dp_max;
+    v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
+    (void)ctx;
+    return v;
+}
+
+Tables tables(const cm_ctx *ctx, int mode) {
+    Tables t{};
+    t.prof = ctx->d_prof; t.binom = ctx->d_binom; t.binom_rows = ctx->binom_rows;
+    t.mm_cuts = ctx->d_mm[mode]; t.mm_stride_m = ctx->mm_stride_m;
+    return t;
+}
+
+// Copy the tables of a batch to the device and run the min-max partitions it needs.
+cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
+    cm_status s;
+    if ((s = upload(ctx, bt.d_scen, bt.scen)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_strat, bt.strat)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_seg, bt.seg)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_failed, bt.failed)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_red_scen, bt.red_scen)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_keys, bt.keys)) != CM_OK) return s;
+    const size_t B = std::max(bt.B, 1);
+    bool ok = bt.d_seg_best.reserve(std::max<size_t>(bt.seg.size(), 1)) &&
+              bt.d_partial.reserve(std::max<size_t>(bt.red_scen.size(), 1)) && bt.d_winner.reserve(B) &&
+              bt.d_kappa_sel.reserve(B * kMaxP) && bt.d_pol_cost.reserve(B * 2) &&
+              bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4) && bt.d_counters.reserve(4);
+    if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
+    if (bt.keys.size()) {
+        CM_CUDA(ctx, launch_minmax(tables(ctx, bt.opts.cost), bt.d_keys.p, (int)bt.keys.size(), bt.opts.cost, ctx->stream));
+        if (launches) ++*launches;
+    }
+    bt.uploaded = true;
+    return CM_OK;
+}
+
+// The launch sequence of the search over an uploaded batch; results land in
+// bt.plans_host ([B][4]) after the stream is synchronised.
+cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
+    const Tables tb = tables(ctx, bt.opts.cost);
+    const BatchDev bd = dev_view(ctx, bt);
+    cudaStream_t st = ctx->stream;
+    int launches = launches_so_far, cost_launches = 0;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
+    if (bt.seg.size()) CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, bt.seg.size() * sizeof(uint64_t), st));
+    CM_CUDA(ctx, cudaMemsetAsync(bt.d_counters.p, 0, 4 * sizeof(unsigned long long), st));
+    if (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) {
+        CM_CUDA(ctx, launch_policies(tb, bd, st));
+        ++launches;
+    }
+    if (bt.policy_mask & (1u << CM_DYNPAR)) {
+        CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
+        if (bt.n_tiles) { CM_CUDA(ctx, launch_cost_pass1(tb, bd, st)); ++launches; ++cost_launches; }
+        CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
+        CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
+        launches += bd.n_red_blocks ? 2 : 1;
+        CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
+        if (bt.n_tiles) { CM_CUDA(ctx, launch_cost_pass2(tb, bd, st)); ++launches; }
+        CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
+    }
+    CM_CUDA(ctx, launch_finalize(tb, bd, st));
+    ++launches;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
+    if (!bt.plans_host.resize((size_t)bt.B * 4) || !bt.counters_host.resize(4)) return fail(ctx, CM_ENOMEM, "host memory");
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.plans_host.p, bt.d_plans.p, (size_t)bt.B * 4 * sizeof(cm_plan), cudaMemcpyDeviceToHost, st));
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.counters_host.p, bt.d_counters.p, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st));
+    CM_CUDA(ctx, cudaStreamSynchronize(st));
+    float ms = 0.f;
+    CM_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
+    if (bt.policy_mask & (1u << CM_DYNPAR)) {
+        float ms_cost = 0.f, ms_tie = 0.f;
+        CM_CUDA(ctx, cudaEventElapsedTime(&ms_cost, ctx->ev[2], ctx->ev[3]));
+        CM_CUDA(ctx, cudaEventElapsedTime(&ms_tie, ctx->ev[4], ctx->ev[5]));
+        ctx->stats[8] += (uint64_t)((double)ms_cost * 1e6);
+        ctx->stats[11] += (uint64_t)((double)ms_tie * 1e6);
+        ctx->stats[12] += (uint64_t)cost_launches;
+    }
+    ctx->stats[10] += (size_t)bt.B * 4 * sizeof(cm_plan) + 4 * sizeof(unsigned long long);
+    ctx->stats[0] += (bt.policy_mask & (1u << CM_DYNPAR)) ? bt.n_cand : 0;
+    ctx->stats[1] += bt.counters_host[0];
+    ctx->stats[2] += bt.counters_host[1];
+    ctx->stats[3] += (uint64_t)launches;
+    ctx->stats[4] += (uint64_t)((double)ms * 1e6);
+    ctx->stats[5] += bt.seg.size();
+    ctx->stats[6] += bt.strat.size();
+    ctx->stats[7] += bt.n_split;
+    return CM_OK;
+}
+
+// Keys of min-max partitions that were scheduled but never computed must be asked for
+// again by the next batch.
+void forget_keys(cm_ctx *ctx, Batch &bt) {
+    std::vector<uint8_t> &done = ctx->mm_done[bt.opts.cost];
+    for (size_t i = 0; i < bt.keys.size(); ++i) {
+        const uint32_t S = bt.keys[i] >> 16, m = bt.keys[i] & 0xffffu;
+        done[(size_t)(S - 1) * ctx->mm_stride_m + m] = 0;
+    }
+    bt.keys.clear();
+}
+
+// A pipeline-plan index that the winner kernel leaves untouched means "not found";
+// it cannot happen for a feasible winner, but never hand it to the caller as a rank.
+void scrub(cm_plan &pl) {
+    for (int p = 0; p < CM_MAX_PIPES; ++p)
+        if (pl.kappa[p] == ~0ull) { pl.kappa[p] = 0; pl.feasible = 0; }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------- C ABI
+extern "C" {
+
+const char *cm_strerror(cm_status s) {
+    switch (s) {
+    case CM_OK: return "ok";
+    case CM_EINVAL: return "invalid argument";
+    case CM_ENOPROFILE: return "no profile loaded";
+    case CM_EOVERFLOW: return "count overflows the index type";
+    case CM_ENOFEASIBLE: return "no feasible plan";
+    case CM_ECUDA: return "CUDA error";
+    case CM_ENOMEM: return "out of memory";
+    case CM_ETIMEOUT: return "timeout";
+    }
+    return "unknown status";
+}
+
+const char *cm_last_error(const cm_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
+    if (!out) return CM_EINVAL;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || cuda_device < 0 || cuda_device >= n) { cudaGetLastError(); return CM_ECUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess) { cudaGetLastError(); return CM_ECUDA; }
+    if (prop.major != 10) return CM_ECUDA;   // kernels are built for sm_100a only; no fallback
+    if (cudaSetDevice(cuda_device) != cudaSuccess) { cudaGetLastError(); return CM_ECUDA; }
+    cm_ctx *c = new (std::nothrow) cm_ctx();
+    if (!c) return CM_ENOMEM;
+    c->device = cuda_device;
+    c->stream = (cudaStream_t)cuda_stream;
+    bool ok = true;
+    for (int i = 0; i < 6; ++i) ok = ok && cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return CM_ECUDA;
+    }
+    *out = c;
+    return CM_OK;
+}
+
+cm_status cm_destroy(cm_ctx *c) {
+    if (!c) return CM_EINVAL;
+    cudaSetDevice(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (int i = 0; i < 6; ++i)
+        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    if (c->d_prof) cudaFree(c->d_prof);
+    if (c->d_binom) cudaFree(c->d_binom);
+    for (int i = 0; i < 2; ++i)
+        if (c->d_mm[i]) cudaFree(c->d_mm[i]);
+    delete c;
+    return CM_OK;
+}
+
+cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
+    if (!ctx) return CM_EINVAL;
+    if (!p) return fail(ctx, CM_EINVAL, "profile is NULL");
+    if (p->L < 1 || p->L > CM_MAX_LAYERS) return fail(ctx, CM_EINVAL, "L out of range");
+    if (p->n_pp < 1 || p->n_pp > std::min(p->L, CM_MAX_STAGES)) return fail(ctx, CM_EINVAL, "n_pp out of range");
+    if (p->n_dp < 1 || p->n_dp > CM_MAX_PIPES) return fail(ctx, CM_EINVAL, "n_dp out of range");
+    if (p->n_micro < 1 || (int64_t)p->n_dp * p->n_micro > CM_MAX_MICRO) return fail(ctx, CM_EINVAL, "n_micro out of range");
+    if (!p->fwd_ns || !p->bwd_ns || !p->fwd_ns_i || !p->bwd_ns_i || !p->act_bytes || !p->param_bytes ||
+        !p->opt_bytes || !p->p2p_bytes || !p->base_cuts)
+        return fail(ctx, CM_EINVAL, "profile array is NULL");
+    if (p->mem_capacity_bytes <= 0 || p->devices_per_node < 1 || p->bw_intra_Bpns <= 0 || p->bw_inter_Bpns <= 0)
+        return fail(ctx, CM_EINVAL, "capacity, devices_per_node and bandwidths must be positive");
+    for (int l = 0; l < p->L; ++l) {
+        if (!(p->fwd_ns[l] >= 0.0) || !(p->bwd_ns[l] >= 0.0) || !std::isfinite(p->fwd_ns[l]) || !std::isfinite(p->bwd_ns[l]))
+            return fail(ctx, CM_EINVAL, "layer times must be finite and non-negative");
+        if (p->fwd_ns_i[l] < 0 || p->bwd_ns_i[l] < 0 || p->fwd_ns_i[l] > (1ll << 40) || p->bwd_ns_i[l] > (1ll << 40))
+            return fail(ctx, CM_EINVAL, "integer layer times out of range");
+        if (p->act_bytes[l] < 0 || p->param_bytes[l] < 0 || p->opt_bytes[l] < 0 || p->p2p_bytes[l] < 0 ||
+            p->act_bytes[l] > (1ll << 44) || p->param_bytes[l] > (1ll << 44) || p->opt_bytes[l] > (1ll << 44))
+            return fail(ctx, CM_EINVAL, "layer bytes out of range");
+    }
+    if (p->base_cuts[0] != 0 || p->base_cuts[p->n_pp] != p->L) return fail(ctx, CM_EINVAL, "base_cuts must run from 0 to L");
+    for (int i = 0; i < p->n_pp; ++i)
+        if (p->base_cuts[i + 1] <= p->base_cuts[i]) return fail(ctx, CM_EINVAL, "base_cuts must be strictly increasing");
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // nothing may still read the old profile
+
+    DevProfile &h = ctx->hp;
+    memset(&h, 0, sizeof(h));
+    h.L = p->L; h.n_dp = p->n_dp; h.n_pp = p->n_pp; h.n_micro = p->n_micro;
+    h.devices_per_node = p->devices_per_node;
+    h.G = p->n_dp * p->n_micro;
+    h.cap = p->mem_capacity_bytes; h.bw_intra = p->bw_intra_Bpns; h.bw_inter = p->bw_inter_Bpns;
+    // gradient all-reduce runs over the inter-node tier as soon as the job spans nodes
+    h.bw_sync = (p->n_dp * p->n_pp > p->devices_per_node) ? p->bw_inter_Bpns : p->bw_intra_Bpns;
+    for (int l = 0; l < p->L; ++l) {
+        h.fwd[l] = p->fwd_ns[l]; h.bwd[l] = p->bwd_ns[l];
+        h.fwd_i[l] = p->fwd_ns_i[l]; h.bwd_i[l] = p->bwd_ns_i[l];
+        h.act[l] = p->act_bytes[l]; h.par[l] = p->param_bytes[l]; h.opt[l] = p->opt_bytes[l]; h.p2p[l] = p->p2p_bytes[l];
+    }
+    for (int i = 0; i <= p->n_pp; ++i) h.base_cuts[i] = p->base_cuts[i];
+    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
+    CM_CUDA(ctx, launch_prefix(ctx->d_prof, ctx->stream));
+
+    // saturating Pascal triangle: rows cover layers, stages, pipelines and micro-batches
+    const int rows = std::max(CM_MAX_LAYERS, h.G) + 1;
+    ctx->binom.assign((size_t)rows * (kBinomCols + 1), 0);
+    for (int n = 0; n < rows; ++n)
+        for (int k = 0; k <= kBinomCols; ++k) {
+            uint64_t v;
+            if (k == 0) v = 1;
+            else if (n == 0) v = 0;
+            else v = sat_add(ctx->binom[(size_t)(n - 1) * (kBinomCols + 1) + k - 1], ctx->binom[(size_t)(n - 1) * (kBinomCols + 1) + k]);
+            ctx->binom[(size_t)n * (kBinomCols + 1) + k] = v;
+        }
+    ctx->binom_rows = rows;
+    if (ctx->d_binom) { cudaFree(ctx->d_binom); ctx->d_binom = nullptr; }
+    CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_binom, ctx->binom.size() * sizeof(uint64_t)));
+    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_binom, ctx->binom.data(), ctx->binom.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
+
+    // min-max partition table, one row per (stages, micro-batches), per cost mode
+    ctx->mm_stride_m = h.G + 2;
+    const size_t slots = (size_t)CM_MAX_STAGES * ctx->mm_stride_m;
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->d_mm[i]) { cudaFree(ctx->d_mm[i]); ctx->d_mm[i] = nullptr; }
+        CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_mm[i], slots * (kMaxS + 1)));
+        CM_CUDA(ctx, cudaMemsetAsync(ctx->d_mm[i], 0xFF, slots * (kMaxS + 1), ctx->stream));
+        ctx->mm_done[i].assign(slots, 0);
+    }
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // ctx->hp / binom may change on the next load
+    ctx->has_profile = true;
+    return CM_OK;
+}
+
+cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids, int32_t n_failed,
+                       const cm_enum_opts *opts, cm_space **out, uint64_t *n_candidates) {
+    if (!ctx) return CM_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
+    if (!out) return fail(ctx, CM_EINVAL, "out is NULL");
+    if (policy < CM_REROUTE || policy > CM_DYNPAR) return fail(ctx, CM_EINVAL, "bad policy");
+    if (n_failed < 0 || (n_failed > 0 && !failed_ids)) return fail(ctx, CM_EINVAL, "bad failure set");
+    cm_enum_opts o{};
+    if (opts) o = *opts;
+    else if (policy == CM_DYNPAR) return fail(ctx, CM_EINVAL, "opts is NULL");
+    else { o.dp_lo = o.dp_hi = 1; o.pp_lo = o.pp_hi = 1; o.lm = CM_LAYERS_MINMAX; o.bm = CM_BATCH_REMAINDER; o.cost = CM_COST_FP64; }
+    cm_status s = check_opts(ctx, &o);
+    if (s != CM_OK) return s;
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    cm_space *sp = new (std::nothrow) cm_space();
+    if (!sp) return fail(ctx, CM_ENOMEM, "host memory");
+    sp->ctx = ctx;
+    sp->policy = policy;
+    sp->failed.assign(failed_ids, failed_ids + n_failed);
+    const int32_t offsets[2] = {0, n_failed};
+    s = build_batch(ctx, sp->batch, failed_ids, offsets, 1, o, 1u << policy);
+    if (s == CM_OK) s = upload_batch(ctx, sp->batch, nullptr);
+    if (s == CM_OK && policy != CM_DYNPAR) {
+        // the one candidate of these policies is evaluated right away so that
+        // cm_evaluate can hand its cost out
+        cudaError_t e = launch_policies(tables(ctx, o.cost), dev_view(ctx, sp->batch), ctx->stream);
+        if (e != cudaSuccess) s = fail(ctx, CM_ECUDA, cudaGetErrorString(e));
+    }
+    if (s != CM_OK) {
+        cudaStreamSynchronize(ctx->stream);
+        forget_keys(ctx, sp->batch);
+        delete sp;
+        return s;
+    }
+    for (size_t i = 0; i < sp->batch.strat.size(); ++i) sp->strat_dp.push_back(sp->batch.strat[i].dp);
+    *out = sp;
+    if (n_candidates) *n_candidates = policy == CM_DYNPAR ? sp->batch.n_cand : 1;
+    return CM_OK;
+}
+
+cm_status cm_space_free(cm_space *sp) {
+    if (!sp) return CM_EINVAL;
+    cudaSetDevice(sp->ctx->device);
+    cudaStreamSynchronize(sp->ctx->stream);   // queued copies still read its host tables
+    delete sp;
+    return CM_OK;
+}
+
+cm_status cm_evaluate(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64_t count,
+                      const uint64_t *idx_dev, double *cost_dev, int64_t *cost_ns_dev, uint8_t *feasible_dev) {
+    if (!ctx) return CM_EINVAL;
+    if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
+    if (count > (1ull << 40)) return fail(ctx, CM_EINVAL, "count too large");
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    Batch &bt = const_cast<Batch &>(space->batch);
+    const uint64_t n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
+    if (!idx_dev && (first > n_cand || count > n_cand - first)) return fail(ctx, CM_EINVAL, "candidate range out of bounds");
+    CM_CUDA(ctx, launch_evaluate(tables(ctx, bt.opts.cost), dev_view(ctx, bt), n_cand,
+                                 space->policy == CM_DYNPAR ? -1 : space->policy, first, count, idx_dev,
+                                 cost_dev, cost_ns_dev, feasible_dev, ctx->stream));
+    return CM_OK;
+}
+
+cm_status cm_select(cm_ctx *ctx, cm_space *const *spaces, int32_t n_spaces, cm_plan *best) {
+    if (!ctx) return CM_EINVAL;
+    if (!spaces || n_spaces < 1 || n_spaces > 64 || !best) return fail(ctx, CM_EINVAL, "bad arguments");
+    for (int i = 0; i < n_spaces; ++i) {
+        if (!spaces[i] || spaces[i]->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
+        if (spaces[i]->batch.opts.cost != spaces[0]->batch.opts.cost) return fail(ctx, CM_EINVAL, "spaces mix cost modes");
+    }
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    memset(ctx->stats, 0, sizeof(ctx->stats));
+    const int mode = spaces[0]->batch.opts.cost;
+    std::vector<const cm_plan *> ptrs(n_spaces);
+    for (int i = 0; i < n_spaces; ++i) {
+        cm_status s = run_batch(ctx, spaces[i]->batch, 0);
+        if (s != CM_OK) return s;
+        ptrs[i] = spaces[i]->batch.d_plans.p + spaces[i]->policy;
+    }
+    // best over the spaces, on the device as well
+    const cm_plan **d_ptrs = nullptr;
+    cm_plan *d_out = nullptr;
+    CM_CUDA(ctx, cudaMalloc((void **)&d_ptrs, sizeof(cm_plan *) * n_spaces + sizeof(cm_plan)));
+    d_out = (cm_plan *)(d_ptrs + n_spaces);
+    cm_plan result;
+    cudaError_t e = cudaMemcpyAsync(d_ptrs, ptrs.data(), sizeof(cm_plan *) * n_spaces, cudaMemcpyHostToDevice, ctx->stream);
+    if (e == cudaSuccess) e = launch_pick(d_ptrs, n_spaces, d_out, mode, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&result, d_out, sizeof(cm_plan), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    cudaFree(d_ptrs);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
+    ctx->stats[3] += 1;
+    scrub(result);
+    *best = result;
+    if (!result.feasible) return fail(ctx, CM_ENOFEASIBLE, "no feasible plan in the given spaces");
+    return CM_OK;
+}
+
+cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                          const cm_enum_opts *opts, cm_plan *best_per_scenario, cm_plan *best_per_policy,
+                          float *latency_us) {
+    if (!ctx) return CM_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
+    if (B < 0 || !offsets || !best_per_scenario || (offsets[B] > 0 && !failed_ids)) return fail(ctx, CM_EINVAL, "bad arguments");
+    cm_status s = check_opts(ctx, opts);
+    if (s != CM_OK) return s;
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    memset(ctx->stats, 0, sizeof(ctx->stats));
+    if (B == 0) return CM_OK;
+    const uint32_t mask = (1u << CM_REROUTE) | (1u << CM_REDUNDANT) | (1u << CM_DYNPAR);
+    Batch &bt = ctx->batch;
+    auto copy_out = [&](int b_dst, int b_src) {
+        for (int pol = 0; pol < 3; ++pol) {
+            cm_plan pl = bt.plans_host[(size_t)b_src * 4 + pol];
+            scrub(pl);
+            if (best_per_policy) best_per_policy[(size_t)b_dst * 3 + pol] = pl;
+        }
+        cm_plan pl = bt.plans_host[(size_t)b_src * 4 + 3];
+        scrub(pl);
+        best_per_scenario[b_dst] = pl;
+    };
+    if (!latency_us) {
+        int launches = 0;
+        if ((s = build_batch(ctx, bt, failed_ids, offsets, B, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
+        for (int b = 0; b < B; ++b) copy_out(b, b);
+        return CM_OK;
+    }
+    for (int b = 0; b < B; ++b) {
+        const auto t0 = std::chrono::steady_clock::now();
+        const int32_t off[2] = {0, offsets[b + 1] - offsets[b]};
+        int launches = 0;
+        if ((s = build_batch(ctx, bt, failed_ids + offsets[b], off, 1, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
+        copy_out(b, 0);
+        const auto t1 = std::chrono::steady_clock::now();
+        latency_us[b] = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
+    }
+    return CM_OK;
+}
+
+cm_status cm_batch_prepare(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                           const cm_enum_opts *opts, cm_batch **out, uint64_t *n_candidates) {
+    if (!ctx) return CM_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
+    if (B < 0 || !offsets || !out || (offsets[B] > 0 && !failed_ids)) return fail(ctx, CM_EINVAL, "bad arguments");
+    cm_status s = check_opts(ctx, opts);
+    if (s != CM_OK) return s;
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    cm_batch *bp = new (std::nothrow) cm_batch();
+    if (!bp) return fail(ctx, CM_ENOMEM, "host memory");
+    bp->ctx = ctx;
+    memset(ctx->stats, 0, sizeof(ctx->stats));
+    const uint32_t mask = (1u << CM_REROUTE) | (1u << CM_REDUNDANT) | (1u << CM_DYNPAR);
+    s = build_batch(ctx, bp->batch, failed_ids, offsets, B, *opts, mask);
+    if (s == CM_OK) s = upload_batch(ctx, bp->batch, &bp->prep_launches);
+    if (s != CM_OK) {
+        cudaStreamSynchronize(ctx->stream);
+        forget_keys(ctx, bp->batch);
+        delete bp;
+        return s;
+    }
+    *out = bp;
+    if (n_candidates) *n_candidates = bp->batch.n_cand;
+    return CM_OK;
+}
+
+cm_status cm_batch_search(cm_ctx *ctx, cm_batch *bp, cm_plan *best_per_scenario, cm_plan *best_per_policy) {
+    if (!ctx) return CM_EINVAL;
+    if (!bp || bp->ctx != ctx || !best_per_scenario) return fail(ctx, CM_EINVAL, "bad arguments");
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    memset(ctx->stats, 0, sizeof(ctx->stats));
+    Batch &bt = bp->batch;
+    if (bt.B == 0) return CM_OK;
+    cm_status s = run_batch(ctx, bt, 0);
+    if (s != CM_OK) return s;
+    for (int b = 0; b < bt.B; ++b) {
+        for (int pol = 0; pol < 3 && best_per_policy; ++pol) {
+            cm_plan pl = bt.plans_host[(size_t)b * 4 + pol];
+            scrub(pl);
+            best_per_policy[(size_t)b * 3 + pol] = pl;
+        }
+        cm_plan pl = bt.plans_host[(size_t)b * 4 + 3];
+        scrub(pl);
+        best_per_scenario[b] = pl;
+    }
+    return CM_OK;
+}
+
+cm_status cm_batch_free(cm_batch *bp) {
+    if (!bp) return CM_EINVAL;
+    cudaSetDevice(bp->ctx->device);
+    cudaStreamSynchronize(bp->ctx->stream);
+    delete bp;
+    return CM_OK;
+}
+
+cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]) {
+    if (!ctx || !out) return CM_EINVAL;
+    memcpy(out, ctx->stats, sizeof(ctx->stats));
+    return CM_OK;
+}
+
+cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan, int32_t *cuts_out) {
+    if (!ctx) return CM_EINVAL;
+    if (!space || space->ctx != ctx || !plan || !cuts_out) return fail(ctx, CM_EINVAL, "bad arguments");
+    if (plan->policy != space->policy) return fail(ctx, CM_EINVAL, "plan was not found in this space");
+    const DevProfile &hp = ctx->hp;
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    std::vector<int32_t> cuts;
+    if (space->policy != CM_DYNPAR) {
+        const int S0 = hp.n_pp;
+        for (int k = 0; k < hp.n_dp; ++k) {
+            std::vector<char> dead(S0, 0);
+            if (space->policy == CM_REDUNDANT)
+                for (uint32_t d : space->failed)
+                    if ((int)(d / S0) == k) dead[d % S0] = 1;
+            cuts.push_back(0);
+            for (int i = 0; i < S0; ++i) {
+                if (dead[i]) continue;
+                int hi = hp.base_cuts[i + 1];
+                if (i + 1 < S0 && dead[i + 1]) hi = hp.base_cuts[i + 2];
+                cuts.push_back(hi);
+            }
+        }
+    } else {
+        const Batch &bt = space->batch;
+        if (plan->strategy >= bt.strat.size()) return fail(ctx, CM_EINVAL, "strategy index out of range");
+        const Strat &st = bt.strat[plan->strategy];
+        if (plan->n_pipes != st.dp) return fail(ctx, CM_EINVAL, "plan does not match its strategy");
+        for (int p = 0; p < st.dp; ++p) {
+            const int S = st.S[p], L = hp.L;
+            const int off = (int)plan->micro[p] - (int)st.m_lo[p];
+            if (plan->stages[p] != S || off < 0 || off >= st.n_m) return fail(ctx, CM_EINVAL, "plan does not match its strategy");
+            const Seg &g = bt.seg[st.seg_first + p * st.n_m + off];
+            const uint64_t kappa = plan->kappa[p];
+            if (kappa > g.K) return fail(ctx, CM_EINVAL, "layer composition rank out of range");
+            if (kappa < g.K) {
+                // combinadic unranking, the same rule the kernels apply
+                auto unrank = [&](uint64_t rank, int n, int t, std::vector<int> &c) {
+                    c.assign(t, 0);
+                    int v = n;
+                    for (int u = t; u >= 1; --u) {
+                        uint64_t b;
+                        do { --v; b = hbinom(ctx, v, u); } while (b > rank);
+                        rank -= b;
+                        c[u - 1] = v;
+                    }
+                };
+                std::vector<int> c;
+                cuts.push_back(0);
+                if (bt.opts.lm == CM_LAYERS_REMAINDER) {
+                    unrank(kappa, S, L % S, c);
+                    std::vector<char> extra(S, 0);
+                    for (int v : c) extra[v] = 1;
+                    int acc = 0;
+                    for (int i = 0; i < S; ++i) { acc += L / S + extra[i]; cuts.push_back(acc); }
+                } else {
+                    unrank(kappa, L - 1, S - 1, c);
+                    for (int i = 0; i < S - 1; ++i) cuts.push_back(c[i] + 1);
+                    cuts.push_back(L);
+                }
+            } else {
+                uint8_t row[kMaxS + 1];
+                CM_CUDA(ctx, cudaMemcpyAsync(row, ctx->d_mm[bt.opts.cost] + (size_t)g.mm_slot * (kMaxS + 1), kMaxS + 1,
+                                             cudaMemcpyDeviceToHost, ctx->stream));
+                CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+                if (row[0] != 0) return fail(ctx, CM_EINVAL, "min-max partition of this pipeline is infeasible");
+                for (int i = 0; i <= S; ++i) cuts.push_back(row[i]);
+            }
+        }
+    }
+    memcpy(cuts_out, cuts.data(), cuts.size() * sizeof(int32_t));
+    return CM_OK;
+}
+
+}  // extern "C"

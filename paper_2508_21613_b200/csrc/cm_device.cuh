@@ -1,0 +1,248 @@
+// Device-side building blocks of the plan search: numeric traits for the two cost
+// modes, the shared-memory copy of the profile, combinadic unranking, the per-stage
+// sums with the memory check, and the 1F1B start/end recurrence.
+#pragma once
+
+#include "cm_internal.h"
+
+namespace cm {
+
+// ----------------------------------------------------------------------------------
+// Cost arithmetic.  T = double: IEEE, one rounding per written operation (compile with
+// --fmad=false).  T = long long: integer nanoseconds, divisions floor.  Costs are never
+// negative, so their 64-bit patterns order like the values and a plain unsigned
+// atomicMin implements "least cost"; infeasible is +inf / INT64_MAX.
+// ----------------------------------------------------------------------------------
+template <typename T> struct Num;
+
+template <> struct Num<double> {
+    static __device__ __forceinline__ double inf() { return __longlong_as_double(0x7FF0000000000000LL); }
+    static __device__ __forceinline__ uint64_t bits(double x) { return (uint64_t)__double_as_longlong(x); }
+    static __device__ __forceinline__ double from_bits(uint64_t b) { return __longlong_as_double((long long)b); }
+    static __device__ __forceinline__ const double *PF(const DevProfile *p) { return p->PFd; }
+    static __device__ __forceinline__ const double *PB(const DevProfile *p) { return p->PBd; }
+    static __device__ __forceinline__ const double *XT(const DevProfile *p, int tier) { return p->XTd[tier]; }
+    static __device__ __forceinline__ double sync(int64_t G, int n, int64_t bw) {
+        if (n <= 1) return 0.0;
+        return ((2.0 * (double)(n - 1)) * (double)G) / ((double)n * (double)bw);
+    }
+    static __device__ __forceinline__ double reroute_extra(int mF, double fb, int peers) {
+        return ((double)mF * fb) / (double)peers;
+    }
+};
+
+template <> struct Num<long long> {
+    static __device__ __forceinline__ long long inf() { return 0x7FFFFFFFFFFFFFFFLL; }
+    static __device__ __forceinline__ uint64_t bits(long long x) { return (uint64_t)x; }
+    static __device__ __forceinline__ long long from_bits(uint64_t b) { return (long long)b; }
+    static __device__ __forceinline__ const long long *PF(const DevProfile *p) { return (const long long *)p->PFi; }
+    static __device__ __forceinline__ const long long *PB(const DevProfile *p) { return (const long long *)p->PBi; }
+    static __device__ __forceinline__ const long long *XT(const DevProfile *p, int tier) { return (const long long *)p->XTi[tier]; }
+    static __device__ __forceinline__ long long sync(int64_t G, int n, int64_t bw) {
+        if (n <= 1) return 0;
+        return (2LL * (long long)(n - 1) * (long long)G) / ((long long)n * (long long)bw);
+    }
+    static __device__ __forceinline__ long long reroute_extra(int mF, long long fb, int peers) {
+        return ((long long)mF * fb) / (long long)peers;
+    }
+};
+
+constexpr uint64_t kInfBitsF64 = 0x7FF0000000000000ull;
+constexpr uint64_t kInfBitsI64 = 0x7FFFFFFFFFFFFFFFull;
+template <typename T> __device__ __forceinline__ uint64_t inf_bits() { return Num<T>::bits(Num<T>::inf()); }
+
+template <typename T> __device__ __forceinline__ T tmax(T a, T b) { return a > b ? a : b; }
+
+// ----------------------------------------------------------------------------------
+// Profile in shared memory: prefix sums over layers, so that any stage [lo,hi) costs a
+// subtraction per quantity (Section "Estimator": stage quantities are sums over layers).
+// ----------------------------------------------------------------------------------
+template <typename T> struct SProf {
+    T PF[kMaxL + 1], PB[kMaxL + 1];
+    long long PA[kMaxL + 1], PS[kMaxL + 1], PP[kMaxL + 1];
+    T XT[2][kMaxL];
+    long long cap, bw_sync;
+    int L, n_dp, n_pp, n_micro;
+};
+
+template <typename T>
+__device__ __forceinline__ void stage_profile(SProf<T> &s, const DevProfile *p) {
+    const int L = p->L;
+    for (int l = threadIdx.x; l <= L; l += blockDim.x) {
+        s.PF[l] = Num<T>::PF(p)[l];
+        s.PB[l] = Num<T>::PB(p)[l];
+        s.PA[l] = p->PA[l];
+        s.PS[l] = p->PS[l];
+        s.PP[l] = p->PP[l];
+        if (l < L) {
+            s.XT[0][l] = Num<T>::XT(p, 0)[l];
+            s.XT[1][l] = Num<T>::XT(p, 1)[l];
+        }
+    }
+    if (threadIdx.x == 0) {
+        s.cap = p->cap;
+        s.bw_sync = p->bw_sync;
+        s.L = L;
+        s.n_dp = p->n_dp;
+        s.n_pp = p->n_pp;
+        s.n_micro = p->n_micro;
+    }
+}
+
+// ----------------------------------------------------------------------------------
+// Combinatorial number system (colex): rank = sum_u C(c_u, u).  Greedy unranking from
+// the largest element; the scan position only moves down, so it costs O(n + t) lookups.
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t binom_at(const uint64_t *tab, int n, int k) {
+    return tab[n * (kBinomCols + 1) + k];
+}
+
+// Calls emit(u-1, v) for u = t..1 with v the u-th smallest element (0-based position u-1).
+template <typename Emit>
+__device__ __forceinline__ void unrank_subset(const uint64_t *tab, uint64_t rank, int n, int t, Emit emit) {
+    int v = n;
+    for (int u = t; u >= 1; --u) {
+        uint64_t c;
+        do {
+            --v;
+            c = binom_at(tab, v, u);
+        } while (c > rank);
+        rank -= c;
+        emit(u - 1, v);
+    }
+}
+
+// Layer cuts of composition kappa (Section "Planner", layer distribution).
+__device__ __forceinline__ void layer_cuts(const uint64_t *tab, int layer_mode, int L, int S,
+                                           uint64_t kappa, uint8_t *cuts /* [S+1] */) {
+    cuts[0] = 0;
+    if (layer_mode == CM_LAYERS_REMAINDER) {
+        const int q = L / S, r = L % S;
+        uint64_t extra = 0;
+        unrank_subset(tab, kappa, S, r, [&](int, int v) { extra |= 1ull << v; });
+        int c = 0;
+        for (int i = 0; i < S; ++i) {
+            c += q + (int)((extra >> i) & 1ull);
+            cuts[i + 1] = (uint8_t)c;
+        }
+    } else {
+        unrank_subset(tab, kappa, L - 1, S - 1, [&](int pos, int v) { cuts[pos + 1] = (uint8_t)(v + 1); });
+        cuts[S] = (uint8_t)L;
+    }
+}
+
+// ----------------------------------------------------------------------------------
+// Pipeline time by the start/end recurrence (Section "Estimator", the transition
+// equation) under the non-interleaved 1F1B order, thread-sequential with O(S) state.
+//
+// Evaluation order (any order that respects the dependencies gives the same values):
+//   phase 1  warm-up forwards, micro-batch by micro-batch, each running up the stages
+//            that still have a warm-up slot for it; the last one of a row is left
+//            pending for the stage above, whose first steady forward it feeds;
+//   phase 2  round k = 0..m-1, stages from last to first: the stage's next forward (if
+//            any is left) fed by the pending forward of the stage below, then its k-th
+//            backward fed by the k-th backward of the stage above (by its own forward at
+//            the last stage).
+// State per stage: clock (end of its latest computation) and pend (end of the forward
+// it has not consumed yet, transfer included).  xt[i] is the transfer time of the
+// boundary between stages i and i+1.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ T sim_pipe(int S, int m, const T *F, const T *B, const T *xt, T *clock, T *pend) {
+    for (int i = 0; i < S; ++i) clock[i] = (T)0;
+    const int n_rows = m < S - 1 ? m : S - 1;
+    for (int j = 0; j < n_rows; ++j) {
+        T chain = (T)0;
+        const int i_max = S - 2 - j;
+        for (int i = 0; i <= i_max; ++i) {
+            T start = i > 0 ? tmax(clock[i], chain) : clock[i];
+            T end = start + F[i];
+            clock[i] = end;
+            chain = end + xt[i];
+        }
+        pend[i_max + 1] = chain;
+    }
+    for (int k = 0; k < m; ++k) {
+        T chain_b = (T)0;
+        for (int i = S - 1; i >= 0; --i) {
+            int w = S - 1 - i;
+            if (w > m) w = m;
+            T c = clock[i];
+            T fend = (T)0;
+            if (w + k < m) {
+                T start = i > 0 ? tmax(c, pend[i]) : c;
+                fend = start + F[i];
+                c = fend;
+                if (i < S - 1) pend[i + 1] = fend + xt[i];
+            }
+            T dep = i < S - 1 ? chain_b + xt[i] : fend;
+            T start = tmax(c, dep);
+            T end = start + B[i];
+            clock[i] = end;
+            chain_b = end;
+        }
+    }
+    return clock[0];
+}
+
+// Peak memory of a stage at position i of S with m micro-batches (Section "Estimator",
+// memory estimator): static bytes + min(S - i, m) in-flight activations.
+__device__ __forceinline__ bool stage_fits(long long stat, long long act, int i, int S, int m, long long cap) {
+    int inflight = S - i;
+    if (m < inflight) inflight = m;
+    return stat + (long long)inflight * act <= cap;
+}
+
+// Cost of one pipeline given by its cuts: memory check, stage sums from the prefix
+// arrays, recurrence, gradient-sync lower bound.  Returns false if infeasible.
+template <typename T>
+__device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, int m, const uint8_t *cuts,
+                                                   uint64_t tier_mask, int n_sync, T &cost) {
+    if (m < 1) return false;
+    for (int i = 0; i < S; ++i) {
+        const int lo = cuts[i], hi = cuts[i + 1];
+        if (hi <= lo) return false;
+        if (!stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap)) return false;
+    }
+    T F[kMaxS], B[kMaxS], xt[kMaxS], clock[kMaxS], pend[kMaxS];
+    long long g_max = 0;
+    for (int i = 0; i < S; ++i) {
+        const int lo = cuts[i], hi = cuts[i + 1];
+        F[i] = sp.PF[hi] - sp.PF[lo];
+        B[i] = sp.PB[hi] - sp.PB[lo];
+        xt[i] = i < S - 1 ? sp.XT[(tier_mask >> i) & 1ull][hi - 1] : (T)0;
+        long long g = sp.PP[hi] - sp.PP[lo];
+        g_max = g > g_max ? g : g_max;
+    }
+    T t = sim_pipe<T>(S, m, F, B, xt, clock, pend);
+    // the sync time is monotone in the gradient bytes, so max over stages = sync of the max
+    cost = t + Num<T>::sync(g_max, n_sync, sp.bw_sync);
+    return true;
+}
+
+// Candidate kappa of a segment: an enumerated composition or the min-max partition.
+template <typename T>
+__device__ __forceinline__ bool segment_candidate_cost(const SProf<T> &sp, const Tables &tb, const Seg &g,
+                                                       int layer_mode, uint64_t kappa, T &cost) {
+    uint8_t cuts[kMaxS + 1];
+    const int S = g.S;
+    if (g.m < 1) return false;
+    if (kappa < g.K) {
+        layer_cuts(tb.binom, layer_mode, sp.L, S, kappa, cuts);
+    } else {
+        const uint8_t *mm = tb.mm_cuts + (size_t)g.mm_slot * (kMaxS + 1);
+        if (mm[0] != 0) return false;  // no memory-feasible partition exists
+        for (int i = 0; i <= S; ++i) cuts[i] = mm[i];
+    }
+    return pipe_cost_from_cuts<T>(sp, S, g.m, cuts, g.tier_mask, g.n_sync, cost);
+}
+
+__device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {
+    for (int o = 16; o > 0; o >>= 1) {
+        uint64_t w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w < v ? w : v;
+    }
+    return v;
+}
+
+}  // namespace cm

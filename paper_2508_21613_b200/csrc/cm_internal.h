@@ -1,0 +1,130 @@
+// Internal layout shared by the host-side descriptor builder and the kernels.
+// Nothing here is part of the C ABI.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "chameleon.h"
+
+namespace cm {
+
+constexpr int kMaxL = CM_MAX_LAYERS;
+constexpr int kMaxS = CM_MAX_STAGES;
+constexpr int kMaxP = CM_MAX_PIPES;
+constexpr int kBinomCols = 64;          // binomial table columns 0..64
+constexpr int kTile = 128;              // candidates per CTA in the generic cost kernel
+constexpr uint64_t kSat = ~0ull;        // saturated binomial
+
+// Per-layer prefix arrays, built on the device by cm_prefix_kernel and staged into shared
+// memory by every kernel that evaluates stages.  PS = 2*params + optimizer (static bytes).
+struct DevProfile {
+    int32_t L, n_dp, n_pp, n_micro;
+    int32_t devices_per_node, G;
+    int64_t cap, bw_intra, bw_inter, bw_sync;
+    double PFd[kMaxL + 1], PBd[kMaxL + 1];
+    int64_t PFi[kMaxL + 1], PBi[kMaxL + 1];
+    int64_t PA[kMaxL + 1], PS[kMaxL + 1], PP[kMaxL + 1];
+    double XTd[2][kMaxL];   // transfer time of the boundary after layer l: [0] intra, [1] inter
+    int64_t XTi[2][kMaxL];
+    int32_t base_cuts[kMaxS + 1];
+    // raw inputs (kept for the prefix kernel)
+    double fwd[kMaxL], bwd[kMaxL];
+    int64_t fwd_i[kMaxL], bwd_i[kMaxL], act[kMaxL], par[kMaxL], opt[kMaxL], p2p[kMaxL];
+};
+
+// One (strategy, pipeline, micro-batch count): its candidates are the layer compositions
+// kappa = 0..K-1 followed by the min-max partition, or the min-max partition alone (K = 0).
+struct Seg {
+    uint64_t cand_first;   // index of its first candidate within the space
+    uint64_t tile_first;   // index of its first tile in the cost kernel's grid
+    uint64_t tier_mask;    // bit i set: the boundary between stages i and i+1 crosses nodes
+    uint64_t K;            // enumerated compositions
+    uint32_t mm_slot;      // row of the min-max cuts table
+    uint32_t strat;        // global strategy row
+    uint16_t S, m, n_sync, pipe;
+    uint32_t scen;         // scenario of the batch
+    uint32_t row;          // its own row in the segment table
+};
+
+// One parallel strategy of one scenario.
+struct Strat {
+    uint64_t split_first;  // first split item of this strategy within its scenario
+    uint64_t n_split;      // micro-batch splits
+    uint32_t seg_first;    // its first segment (global row)
+    uint16_t dp, n_m;      // pipelines; micro-batch values per pipeline (segments per pipeline)
+    uint16_t R, pad;       // REMAINDER mode: pipelines that receive one more
+    uint16_t S[kMaxP], m_lo[kMaxP];
+};
+
+// One failure scenario of a batch.
+struct Scen {
+    uint64_t n_split_total;  // split items over all its strategies
+    uint32_t strat_first, n_strat;
+    uint32_t seg_first, n_seg;
+    uint32_t failed_first, n_failed;   // into the failed-id array
+    uint32_t red_first, n_red;         // blocks of the split reduction that belong to it
+    uint32_t policy_mask, pad;
+};
+
+// (cost, index) pair carried through the hierarchical argmin of the split reduction.
+struct Partial {
+    uint64_t cost_bits;     // cost as an order-preserving 64-bit pattern (inf = infeasible)
+    uint64_t item;          // split item index within the scenario
+};
+
+// Per-scenario winner of the split reduction, decoded for the tie-break pass.
+struct Winner {
+    uint64_t cost_bits;
+    uint64_t item;
+    uint32_t strat, dp;     // global strategy row; pipelines
+    uint32_t seg[kMaxP];    // global segment row of every pipeline
+    uint16_t micro[kMaxP];
+};
+
+struct BatchDev {
+    const Scen *scen;
+    const Strat *strat;
+    const Seg *seg;
+    const uint32_t *failed;
+    uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
+    const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
+    Partial *partial;       // [n_red_blocks]
+    Winner *winner;         // [B]
+    uint64_t *kappa_sel;    // [B][kMaxP] lowest kappa with cost <= T*
+    uint64_t *pol_cost;     // [B][2] rerouting / redundant cost bits
+    uint16_t *rc_stages;    // [B][kMaxP] stage counts of the redundant-computation plan
+    cm_plan *plans;         // [B][4]: per policy, then the overall best
+    unsigned long long *counters;  // [0] cells simulated in pass 1, [1] plans in pass 2
+    int32_t B, mode;
+    uint32_t n_seg, n_strat;
+    uint64_t n_tiles;
+    uint32_t max_tiles_per_seg, n_red_blocks;
+    uint32_t dp_max, pad;
+    int32_t layer_mode, batch_mode;
+};
+
+struct Tables {
+    const DevProfile *prof;
+    const uint64_t *binom;      // [rows][kBinomCols+1], saturating
+    int32_t binom_rows;
+    uint8_t *mm_cuts;           // [slots][kMaxS+1], min-max partitions; mm_cuts[slot][0]=255: infeasible
+    int32_t mm_stride_m;        // slot = (S-1)*mm_stride_m + m
+};
+
+// launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
+cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
+cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
+cudaError_t launch_policies(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st);
+// single_policy < 0: candidates of the dynamic-parallelism segments; otherwise the one
+// candidate of that policy (its cost must already be in pol_cost of scenario 0)
+cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand, int single_policy,
+                            uint64_t first, uint64_t count, const uint64_t *idx, double *cost,
+                            int64_t *cost_ns, uint8_t *feas, cudaStream_t st);
+cudaError_t launch_pick(const cm_plan *const *plans_dev, int n, cm_plan *out_dev, int mode, cudaStream_t st);
+
+}  // namespace cm

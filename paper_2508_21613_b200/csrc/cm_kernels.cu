@@ -1,0 +1,668 @@
+// Kernels of the plan search (sm_100a) and their launchers.
+//
+//   cm_prefix_kernel      per-layer prefix sums and per-boundary transfer times
+//   cm_minmax_kernel      min-max contiguous layer partition per (stages, micro-batches)
+//   cm_policy_kernel      data rerouting and redundant computation, one plan each
+//   cm_cost_kernel        pass 1: every pipeline-plan of every segment -> least cost per segment
+//   cm_split_kernel       (cost, index) argmin over (strategy, micro-batch split) per scenario
+//   cm_winner_kernel      finishes that argmin and decodes the winner
+//   cm_tiebreak_kernel    pass 2: lowest layer composition that meets the winning cost
+//   cm_finalize_kernel    assembles the plans and picks the best policy
+//   cm_evaluate_kernel    per-candidate cost / feasibility for cm_evaluate
+//   cm_pick_kernel        best of several spaces for cm_select
+#include "cm_device.cuh"
+
+namespace cm {
+
+// ----------------------------------------------------------------------------------
+// Prefix sums, accumulated left to right so that every consumer of a stage quantity
+// performs the same single subtraction (Section "Estimator": stage time / memory are
+// sums over the stage's layers).  One thread per array; the arrays are <= 129 long.
+// ----------------------------------------------------------------------------------
+__global__ void cm_prefix_kernel(DevProfile *p) {
+    const int L = p->L;
+    switch (threadIdx.x) {
+    case 0: { double a = 0.0; p->PFd[0] = a; for (int l = 0; l < L; ++l) { a = a + p->fwd[l]; p->PFd[l + 1] = a; } break; }
+    case 1: { double a = 0.0; p->PBd[0] = a; for (int l = 0; l < L; ++l) { a = a + p->bwd[l]; p->PBd[l + 1] = a; } break; }
+    case 2: { int64_t a = 0; p->PFi[0] = a; for (int l = 0; l < L; ++l) { a += p->fwd_i[l]; p->PFi[l + 1] = a; } break; }
+    case 3: { int64_t a = 0; p->PBi[0] = a; for (int l = 0; l < L; ++l) { a += p->bwd_i[l]; p->PBi[l + 1] = a; } break; }
+    case 4: { int64_t a = 0; p->PA[0] = a; for (int l = 0; l < L; ++l) { a += p->act[l]; p->PA[l + 1] = a; } break; }
+    case 5: { int64_t a = 0; p->PS[0] = a; for (int l = 0; l < L; ++l) { a += 2 * p->par[l] + p->opt[l]; p->PS[l + 1] = a; } break; }
+    case 6: { int64_t a = 0; p->PP[0] = a; for (int l = 0; l < L; ++l) { a += p->par[l]; p->PP[l + 1] = a; } break; }
+    default: break;
+    }
+    for (int l = threadIdx.x; l < L; l += blockDim.x) {
+        p->XTd[0][l] = (double)p->p2p[l] / (double)p->bw_intra;
+        p->XTd[1][l] = (double)p->p2p[l] / (double)p->bw_inter;
+        p->XTi[0][l] = p->p2p[l] / p->bw_intra;
+        p->XTi[1][l] = p->p2p[l] / p->bw_inter;
+    }
+}
+
+cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st) {
+    cm_prefix_kernel<<<1, 128, 0, st>>>(prof);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Min-max layer partition: D[l][s] = min_k max(D[k][s-1], W(k,l)), W = forward+backward
+// time of layers [k,l), only over stages that fit in memory at position s-1.  One CTA
+// per (S, m) key; stage columns are swept one after the other, the layers of a column
+// go to the warps, the split points k to the lanes, and a warp-shuffle argmin carrying
+// (value, k) with the lowest k on ties closes each cell.  Backtracking follows the
+// stored argmin, which is the smallest k that attains D[l][s].
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) cm_minmax_kernel(Tables tb, const uint32_t *keys, int n_keys) {
+    __shared__ T PF[kMaxL + 1], PB[kMaxL + 1];
+    __shared__ long long PA[kMaxL + 1], PS[kMaxL + 1];
+    __shared__ T D[2][kMaxL + 1];
+    __shared__ uint8_t argk[kMaxS + 1][kMaxL + 1];
+    const DevProfile *p = tb.prof;
+    const int L = p->L;
+    const uint32_t key = keys[blockIdx.x];
+    const int S = (int)(key >> 16), m = (int)(key & 0xffffu);
+    const long long cap = p->cap;
+    for (int l = threadIdx.x; l <= L; l += blockDim.x) {
+        PF[l] = Num<T>::PF(p)[l];
+        PB[l] = Num<T>::PB(p)[l];
+        PA[l] = p->PA[l];
+        PS[l] = p->PS[l];
+        D[0][l] = Num<T>::inf();
+        D[1][l] = Num<T>::inf();
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const T INF = Num<T>::inf();
+    for (int s = 1; s <= S; ++s) {
+        T *cur = D[s & 1];
+        const T *prev = D[(s - 1) & 1];
+        for (int l = s + warp; l <= L; l += n_warps) {
+            T best = INF;
+            int best_k = 0;
+            if (s == 1) {
+                if (lane == 0 && stage_fits(PS[l] - PS[0], PA[l] - PA[0], 0, S, m, cap))
+                    best = (PF[l] - PF[0]) + (PB[l] - PB[0]);
+            } else {
+                for (int k = s - 1 + lane; k <= l - 1; k += 32) {
+                    if (prev[k] == INF) continue;
+                    if (!stage_fits(PS[l] - PS[k], PA[l] - PA[k], s - 1, S, m, cap)) continue;
+                    T w = (PF[l] - PF[k]) + (PB[l] - PB[k]);
+                    T v = tmax(prev[k], w);
+                    if (v < best) { best = v; best_k = k; }
+                }
+            }
+            for (int o = 16; o > 0; o >>= 1) {
+                T ov = __shfl_xor_sync(0xffffffffu, best, o);
+                int ok = __shfl_xor_sync(0xffffffffu, best_k, o);
+                if (ov < best || (ov == best && ov != INF && ok < best_k)) { best = ov; best_k = ok; }
+            }
+            if (lane == 0) {
+                cur[l] = best;
+                argk[s][l] = (uint8_t)best_k;
+            }
+        }
+        // cells of this column below the first reachable layer stay infinite
+        for (int l = threadIdx.x; l < s; l += blockDim.x) cur[l] = INF;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint8_t *out = tb.mm_cuts + ((size_t)(S - 1) * tb.mm_stride_m + m) * (kMaxS + 1);
+        if (D[S & 1][L] == INF) {
+            out[0] = 255;
+        } else {
+            int l = L;
+            out[S] = (uint8_t)L;
+            for (int s = S; s >= 2; --s) {
+                l = argk[s][l];
+                out[s - 1] = (uint8_t)l;
+            }
+            out[0] = 0;
+        }
+    }
+}
+
+cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st) {
+    if (n_keys <= 0) return cudaSuccess;
+    if (mode == CM_COST_INT64NS) cm_minmax_kernel<long long><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
+    else cm_minmax_kernel<double><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Data rerouting and redundant computation: one plan per scenario each.
+//
+// Rerouting (Section "Estimator", single- and multi-failure step time): the failed
+// devices' micro-batches go to the data-parallel peers of the same stage; with F_i
+// failed devices in stage i the step grows by N_m F_i (F_i^st + B_i^st) / (N_dp - F_i) per
+// affected stage on top of the unchanged base pipeline; unrecoverable if F_i >= N_dp.
+//
+// Redundant computation (Section "Limitations of Backup-free Methods", prose): a failed
+// stage is taken over by its predecessor; every stage but the last also carries its
+// successor's work and state.  Infeasible if stage 0 failed or two neighbours failed.
+//
+// One warp per scenario: lane 0 evaluates rerouting, lane 1+k pipeline k of the
+// redundant plan; a shuffle max combines the pipelines.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(32) cm_policy_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ int base_cuts[kMaxS + 1];
+    const DevProfile *p = tb.prof;
+    stage_profile(sp, p);
+    for (int i = threadIdx.x; i <= p->n_pp; i += blockDim.x) base_cuts[i] = p->base_cuts[i];
+    __syncthreads();
+    const int b = blockIdx.x;
+    const Scen sc = bd.scen[b];
+    const uint32_t *failed = bd.failed + sc.failed_first;
+    const int S0 = sp.n_pp, m = sp.n_micro, n_dp = sp.n_dp;
+    const int lane = threadIdx.x;
+    const int dpn = p->devices_per_node;
+    T F[kMaxS], B[kMaxS], xt[kMaxS], clock[kMaxS], pend[kMaxS];
+
+    if (lane == 0) {
+        uint64_t out = inf_bits<T>();
+        if (sc.policy_mask & (1u << CM_REROUTE)) {
+            int fcnt[kMaxS];
+            for (int i = 0; i < S0; ++i) fcnt[i] = 0;
+            for (uint32_t f = 0; f < sc.n_failed; ++f) fcnt[failed[f] % S0]++;
+            bool ok = m >= 1;
+            for (int i = 0; i < S0; ++i) ok = ok && fcnt[i] < n_dp;
+            for (int i = 0; i < S0 && ok; ++i) {
+                const int lo = base_cuts[i], hi = base_cuts[i + 1];
+                ok = stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap);
+            }
+            if (ok) {
+                T extra = (T)0, t_sync = (T)0;
+                for (int i = 0; i < S0; ++i) {
+                    const int lo = base_cuts[i], hi = base_cuts[i + 1];
+                    F[i] = sp.PF[hi] - sp.PF[lo];
+                    B[i] = sp.PB[hi] - sp.PB[lo];
+                    // pipeline 0 sits on devices 0 .. S0-1
+                    const int tier = (i / dpn == (i + 1) / dpn) ? 0 : 1;
+                    xt[i] = i < S0 - 1 ? sp.XT[tier][hi - 1] : (T)0;
+                    if (fcnt[i] > 0) extra = extra + Num<T>::reroute_extra(m * fcnt[i], F[i] + B[i], n_dp - fcnt[i]);
+                    t_sync = tmax(t_sync, Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt[i], sp.bw_sync));
+                }
+                T base = sim_pipe<T>(S0, m, F, B, xt, clock, pend);
+                out = Num<T>::bits((base + extra) + t_sync);
+            }
+        }
+        bd.pol_cost[2 * b + 0] = out;
+    }
+
+    // redundant computation: lanes 1..n_dp
+    T my_cost = (T)0;
+    bool my_ok = true;
+    int my_S = 0;
+    const int k = lane - 1;
+    if (k >= 0 && k < n_dp) {
+        uint64_t dead = 0;
+        for (uint32_t f = 0; f < sc.n_failed; ++f)
+            if ((int)(failed[f] / S0) == k) dead |= 1ull << (failed[f] % S0);
+        if (dead & 1ull) my_ok = false;
+        if (dead & (dead >> 1)) my_ok = false;
+        if (m < 1) my_ok = false;
+        if (my_ok) {
+            int cuts[kMaxS + 1], devs[kMaxS];
+            int S = 0;
+            cuts[0] = 0;
+            for (int i = 0; i < S0; ++i) {
+                if ((dead >> i) & 1ull) continue;
+                int hi = base_cuts[i + 1];
+                if (i + 1 < S0 && ((dead >> (i + 1)) & 1ull)) hi = base_cuts[i + 2];
+                devs[S] = k * S0 + i;
+                cuts[S + 1] = hi;
+                ++S;
+            }
+            my_S = S;
+            long long g_max = 0;
+            for (int i = 0; i < S && my_ok; ++i) {
+                const int lo = cuts[i], hi = cuts[i + 1];
+                long long stat = sp.PS[hi] - sp.PS[lo], act = sp.PA[hi] - sp.PA[lo];
+                T f = sp.PF[hi] - sp.PF[lo], bw = sp.PB[hi] - sp.PB[lo];
+                if (i < S - 1) {
+                    const int hi2 = cuts[i + 2];
+                    f = f + (sp.PF[hi2] - sp.PF[hi]);
+                    bw = bw + (sp.PB[hi2] - sp.PB[hi]);
+                    stat = stat + (sp.PS[hi2] - sp.PS[hi]);
+                    act = act + (sp.PA[hi2] - sp.PA[hi]);
+                    const int tier = (devs[i] / dpn == devs[i + 1] / dpn) ? 0 : 1;
+                    xt[i] = sp.XT[tier][hi - 1];
+                } else {
+                    xt[i] = (T)0;
+                }
+                F[i] = f;
+                B[i] = bw;
+                if (!stage_fits(stat, act, i, S, m, sp.cap)) my_ok = false;
+                long long g = sp.PP[hi] - sp.PP[lo];
+                g_max = g > g_max ? g : g_max;
+            }
+            if (my_ok) my_cost = sim_pipe<T>(S, m, F, B, xt, clock, pend) + Num<T>::sync(g_max, n_dp, sp.bw_sync);
+        }
+    }
+    uint64_t bits = my_ok ? Num<T>::bits(my_cost) : inf_bits<T>();
+    // slowest pipeline sets the step; an infeasible pipeline (inf) wins the max
+    for (int o = 16; o > 0; o >>= 1) {
+        uint64_t w = __shfl_xor_sync(0xffffffffu, bits, o);
+        bits = w > bits ? w : bits;
+    }
+    if (k >= 0 && k < n_dp && k < kMaxP) bd.rc_stages[b * kMaxP + k] = (uint16_t)my_S;
+    if (lane == 0) bd.pol_cost[2 * b + 1] = (sc.policy_mask & (1u << CM_REDUNDANT)) ? bits : inf_bits<T>();
+}
+
+cudaError_t launch_policies(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    if (b.mode == CM_COST_INT64NS) cm_policy_kernel<long long><<<b.B, 32, 0, st>>>(t, b);
+    else cm_policy_kernel<double><<<b.B, 32, 0, st>>>(t, b);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Locate the segment that owns a tile / a candidate: the last row whose first index is
+// not above the query (rows are sorted and every segment owns at least one).
+// ----------------------------------------------------------------------------------
+template <typename Key>
+__device__ __forceinline__ uint32_t find_row(const Seg *seg, uint32_t n, uint64_t q, Key key) {
+    uint32_t lo = 0, hi = n - 1;
+    while (lo < hi) {
+        uint32_t mid = (lo + hi + 1) >> 1;
+        if (key(seg[mid]) <= q) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// ----------------------------------------------------------------------------------
+// Pass 1 (generic path): one CTA per tile of kTile consecutive layer compositions of one
+// segment, one thread per pipeline-plan: unrank -> stage sums -> memory check ->
+// recurrence -> sync -> cost; block min -> one atomicMin per CTA on the segment's best.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kTile) cm_cost_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ uint64_t red[kTile / 32];
+    __shared__ unsigned long long cells[kTile / 32];
+    __shared__ Seg g;
+    const uint64_t tile = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    if (tile >= bd.n_tiles) return;
+    stage_profile(sp, tb.prof);
+    if (threadIdx.x == 0) {
+        uint32_t s = find_row(bd.seg, bd.n_seg, tile, [](const Seg &x) { return x.tile_first; });
+        g = bd.seg[s];
+    }
+    __syncthreads();
+    const uint64_t count = g.K ? g.K + 1 : 1;
+    const uint64_t kappa = (tile - g.tile_first) * kTile + threadIdx.x;
+    uint64_t bits = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (kappa < count) {
+        T cost;
+        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * g.S * g.m;
+        }
+    }
+    bits = warp_min_u64(bits);
+    for (int o = 16; o > 0; o >>= 1) my_cells += __shfl_xor_sync(0xffffffffu, my_cells, o);
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = bits; cells[threadIdx.x >> 5] = my_cells; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long c = 0;
+        for (int w = 0; w < kTile / 32; ++w) { bits = red[w] < bits ? red[w] : bits; c += cells[w]; }
+        if (bits != inf_bits<T>()) atomicMin((unsigned long long *)&bd.seg_best[g.row], (unsigned long long)bits);
+        if (c) atomicAdd(&bd.counters[0], c);
+    }
+}
+
+static dim3 tile_grid(uint64_t n_tiles) {
+    const uint64_t maxx = 1u << 30;
+    if (n_tiles <= maxx) return dim3((unsigned)n_tiles, 1, 1);
+    return dim3((unsigned)maxx, (unsigned)((n_tiles + maxx - 1) / maxx), 1);
+}
+
+cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.n_tiles == 0) return cudaSuccess;
+    dim3 grid = tile_grid(b.n_tiles);
+    if (b.mode == CM_COST_INT64NS) cm_cost_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
+    else cm_cost_kernel<double><<<grid, kTile, 0, st>>>(t, b);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Micro-batch split of a strategy from its rank (Section "Planner", batch distribution).
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ void split_micro(const uint64_t *tab, int batch_mode, int G, const Strat &s,
+                                            uint64_t beta, uint16_t *micro) {
+    const int dp = s.dp;
+    if (batch_mode == CM_BATCH_REMAINDER) {
+        for (int p = 0; p < dp; ++p) micro[p] = s.m_lo[p];
+        unrank_subset(tab, beta, dp, s.R, [&](int, int v) { micro[v] = (uint16_t)(micro[v] + 1); });
+    } else {
+        int cutpos[kMaxP];
+        unrank_subset(tab, beta, G - 1, dp - 1, [&](int pos, int v) { cutpos[pos] = v + 1; });
+        int prev = 0;
+        for (int p = 0; p < dp - 1; ++p) { micro[p] = (uint16_t)(cutpos[p] - prev); prev = cutpos[p]; }
+        micro[dp - 1] = (uint16_t)(G - prev);
+    }
+}
+
+__device__ __forceinline__ bool pair_less(uint64_t c1, uint64_t i1, uint64_t c2, uint64_t i2) {
+    return c1 < c2 || (c1 == c2 && i1 < i2);
+}
+
+// ----------------------------------------------------------------------------------
+// Split reduction: item = (strategy, split rank) of one scenario; its step time is the
+// slowest pipeline's best cost (Section "Estimator": step time = max over pipelines).
+// Hierarchical argmin carrying (cost, item) with the lowest item on ties:
+// thread-serial over a strided range -> warp shuffle -> shared memory -> one partial
+// per block -> cm_winner_kernel over the scenario's partials.
+// ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) cm_split_kernel(Tables tb, BatchDev bd, uint64_t inf) {
+    __shared__ uint64_t rc[8], ri[8];
+    const uint32_t b = bd.red_scen[blockIdx.x];
+    const Scen sc = bd.scen[b];
+    const uint32_t local = blockIdx.x - sc.red_first;
+    const int G = tb.prof->G;
+    uint64_t best_c = inf, best_i = ~0ull;
+    for (uint64_t item = (uint64_t)local * blockDim.x + threadIdx.x; item < sc.n_split_total;
+         item += (uint64_t)sc.n_red * blockDim.x) {
+        // strategy that owns the item
+        uint32_t lo = 0, hi = sc.n_strat - 1;
+        while (lo < hi) {
+            uint32_t mid = (lo + hi + 1) >> 1;
+            if (bd.strat[sc.strat_first + mid].split_first <= item) lo = mid; else hi = mid - 1;
+        }
+        const Strat &s = bd.strat[sc.strat_first + lo];
+        uint16_t micro[kMaxP];
+        split_micro(tb.binom, bd.batch_mode, G, s, item - s.split_first, micro);
+        uint64_t T = 0;
+        for (int p = 0; p < s.dp; ++p) {
+            uint64_t c = inf;
+            const int off = (int)micro[p] - (int)s.m_lo[p];
+            if (micro[p] >= 1 && off >= 0 && off < s.n_m) c = bd.seg_best[s.seg_first + p * s.n_m + off];
+            c = c > inf ? inf : c;   // a segment nobody improved still holds its all-ones initial value
+            T = c > T ? c : T;
+        }
+        if (pair_less(T, item, best_c, best_i)) { best_c = T; best_i = item; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        uint64_t oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+        uint64_t oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { rc[threadIdx.x >> 5] = best_c; ri[threadIdx.x >> 5] = best_i; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w)
+            if (pair_less(rc[w], ri[w], best_c, best_i)) { best_c = rc[w]; best_i = ri[w]; }
+        bd.partial[blockIdx.x].cost_bits = best_c;
+        bd.partial[blockIdx.x].item = best_i;
+    }
+}
+
+// Grid level of the argmin: one warp per scenario over its block partials, then decode
+// the winner (strategy, split -> micro-batches, segment rows) for the tie-break pass.
+__global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, uint64_t inf) {
+    const uint32_t b = blockIdx.x;
+    const Scen sc = bd.scen[b];
+    uint64_t best_c = inf, best_i = ~0ull;
+    for (uint32_t r = threadIdx.x; r < sc.n_red; r += 32) {
+        const Partial q = bd.partial[sc.red_first + r];
+        if (pair_less(q.cost_bits, q.item, best_c, best_i)) { best_c = q.cost_bits; best_i = q.item; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        uint64_t oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+        uint64_t oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
+    }
+    if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
+    if (threadIdx.x == 0) {
+        Winner w;
+        w.cost_bits = best_c >= inf ? inf : best_c;
+        w.item = best_i;
+        w.strat = 0;
+        w.dp = 0;
+        for (int p = 0; p < kMaxP; ++p) { w.seg[p] = 0; w.micro[p] = 0; }
+        if (best_c < inf) {
+            uint32_t lo = 0, hi = sc.n_strat - 1;
+            while (lo < hi) {
+                uint32_t mid = (lo + hi + 1) >> 1;
+                if (bd.strat[sc.strat_first + mid].split_first <= best_i) lo = mid; else hi = mid - 1;
+            }
+            const Strat &s = bd.strat[sc.strat_first + lo];
+            w.strat = sc.strat_first + lo;
+            w.dp = s.dp;
+            split_micro(tb.binom, bd.batch_mode, tb.prof->G, s, best_i - s.split_first, w.micro);
+            for (int p = 0; p < s.dp; ++p) w.seg[p] = s.seg_first + p * s.n_m + (w.micro[p] - s.m_lo[p]);
+        }
+        bd.winner[b] = w;
+    }
+}
+
+cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    if (b.n_red_blocks) {
+        cm_split_kernel<<<b.n_red_blocks, 256, 0, st>>>(t, b, inf);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    cm_winner_kernel<<<b.B, 32, 0, st>>>(t, b, inf);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Pass 2 (tie-break): among optimal plans the lexicographically smallest tuple wins, so
+// each pipeline of the winning (strategy, split) takes the LOWEST layer composition
+// that is feasible with cost <= T* (not its own argmin).  grid.x = tiles of a segment,
+// grid.y = (scenario, pipeline).  Tiles above an already found index return at once.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ uint64_t red[kTile / 32];
+    __shared__ Seg g;
+    __shared__ uint64_t found_so_far;
+    stage_profile(sp, tb.prof);
+    for (uint32_t y = blockIdx.y; y < (uint32_t)bd.B * bd.dp_max; y += gridDim.y) {
+        const uint32_t b = y / bd.dp_max, p = y % bd.dp_max;
+        const Winner &w = bd.winner[b];
+        if (w.cost_bits >= inf_bits<T>() || p >= w.dp) continue;   // uniform over the CTA
+        uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            g = bd.seg[w.seg[p]];
+            found_so_far = *(volatile uint64_t *)slot;
+        }
+        __syncthreads();
+        const uint64_t count = g.K ? g.K + 1 : 1;
+        const uint64_t first = (uint64_t)blockIdx.x * kTile;
+        if (first >= count || found_so_far < first) continue;       // uniform: read from shared
+        const uint64_t kappa = first + threadIdx.x;
+        uint64_t hit = ~0ull;
+        if (kappa < count) {
+            T cost;
+            if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost) &&
+                Num<T>::bits(cost) <= w.cost_bits)
+                hit = kappa;
+        }
+        hit = warp_min_u64(hit);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = hit;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int q = 0; q < kTile / 32; ++q) hit = red[q] < hit ? red[q] : hit;
+            if (hit != ~0ull) atomicMin((unsigned long long *)slot, (unsigned long long)hit);
+            uint64_t n = count - first < kTile ? count - first : kTile;
+            atomicAdd(&bd.counters[1], (unsigned long long)n);
+        }
+    }
+}
+
+cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
+    uint64_t ny = (uint64_t)b.B * b.dp_max;
+    dim3 grid(b.max_tiles_per_seg, (unsigned)(ny < 65535 ? ny : 65535), 1);
+    if (b.mode == CM_COST_INT64NS) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
+    else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Assemble the per-policy plans and the overall best: least cost, ties to the lowest
+// policy id (Algorithm 1 keeps the plan with the least estimated time).
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ void plan_clear(cm_plan &pl, int policy) {
+    pl.policy = policy;
+    pl.feasible = 0;
+    pl.cost = 0.0;
+    pl.cost_ns = 0;
+    pl.strategy = 0;
+    pl.n_pipes = 0;
+    pl.split_rank = 0;
+    for (int p = 0; p < kMaxP; ++p) { pl.stages[p] = 0; pl.micro[p] = 0; pl.kappa[p] = 0; }
+}
+
+__device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mode) {
+    if (mode == CM_COST_INT64NS) pl.cost_ns = (int64_t)bits;
+    else pl.cost = __longlong_as_double((long long)bits);
+}
+
+__global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= bd.B) return;
+    const DevProfile *p = tb.prof;
+    const Scen sc = bd.scen[b];
+    cm_plan *out = bd.plans + (size_t)b * 4;
+    uint64_t cost[3] = {inf, inf, inf};
+    for (int pol = 0; pol < 2; ++pol) {
+        cm_plan pl;
+        plan_clear(pl, pol);
+        pl.n_pipes = (uint32_t)p->n_dp;
+        for (int k = 0; k < p->n_dp && k < kMaxP; ++k) {
+            pl.stages[k] = (uint16_t)p->n_pp;
+            pl.micro[k] = (uint16_t)p->n_micro;
+        }
+        uint64_t c = (sc.policy_mask & (1u << pol)) ? bd.pol_cost[2 * b + pol] : inf;
+        if (c < inf) {
+            pl.feasible = 1;
+            plan_set_cost(pl, c, bd.mode);
+            if (pol == CM_REDUNDANT)
+                for (int k = 0; k < p->n_dp && k < kMaxP; ++k) pl.stages[k] = bd.rc_stages[b * kMaxP + k];
+            cost[pol] = c;
+        }
+        out[pol] = pl;
+    }
+    {
+        cm_plan pl;
+        plan_clear(pl, CM_DYNPAR);
+        const Winner &w = bd.winner[b];
+        if ((sc.policy_mask & (1u << CM_DYNPAR)) && w.cost_bits < inf) {
+            const Strat &s = bd.strat[w.strat];
+            pl.feasible = 1;
+            plan_set_cost(pl, w.cost_bits, bd.mode);
+            pl.strategy = w.strat - sc.strat_first;
+            pl.n_pipes = w.dp;
+            pl.split_rank = w.item - s.split_first;
+            for (uint32_t q = 0; q < w.dp; ++q) {
+                pl.stages[q] = s.S[q];
+                pl.micro[q] = w.micro[q];
+                pl.kappa[q] = bd.kappa_sel[b * kMaxP + q];
+            }
+            cost[2] = w.cost_bits;
+        }
+        out[2] = pl;
+    }
+    int win = -1;
+    for (int pol = 0; pol < 3; ++pol)
+        if (cost[pol] < inf && (win < 0 || cost[pol] < cost[win])) win = pol;
+    if (win >= 0) out[3] = out[win];
+    else { cm_plan pl; plan_clear(pl, 0); out[3] = pl; }
+}
+
+cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    cm_finalize_kernel<<<(b.B + 127) / 128, 128, 0, st>>>(t, b, inf);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// cm_evaluate: one thread per requested candidate.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) cm_evaluate_kernel(Tables tb, BatchDev bd, uint64_t first, uint64_t count,
+                                                          const uint64_t *idx, uint64_t n_cand, double *cost,
+                                                          int64_t *cost_ns, uint8_t *feas) {
+    __shared__ SProf<T> sp;
+    stage_profile(sp, tb.prof);
+    __syncthreads();
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count) return;
+    const uint64_t e = idx ? idx[t] : first + t;
+    T c = Num<T>::inf();
+    bool ok = false;
+    if (e < n_cand) {
+        uint32_t s = find_row(bd.seg, bd.n_seg, e, [](const Seg &x) { return x.cand_first; });
+        const Seg g = bd.seg[s];
+        T v;
+        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, e - g.cand_first, v)) { c = v; ok = true; }
+    }
+    if (cost && bd.mode == CM_COST_FP64) cost[t] = __longlong_as_double((long long)Num<T>::bits(c));
+    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = (int64_t)Num<T>::bits(c);
+    if (feas) feas[t] = ok ? 1 : 0;
+}
+
+// One-candidate policies through cm_evaluate: the cost cm_policy_kernel left behind.
+__global__ void cm_evaluate_single_kernel(BatchDev bd, int policy, uint64_t inf, uint64_t first, uint64_t count,
+                                          const uint64_t *idx, double *cost, int64_t *cost_ns, uint8_t *feas) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count) return;
+    const uint64_t e = idx ? idx[t] : first + t;
+    uint64_t c = e == 0 ? bd.pol_cost[policy] : inf;
+    if (cost && bd.mode == CM_COST_FP64) cost[t] = __longlong_as_double((long long)c);
+    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = (int64_t)c;
+    if (feas) feas[t] = c < inf ? 1 : 0;
+}
+
+cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand, int single_policy,
+                            uint64_t first, uint64_t count, const uint64_t *idx, double *cost,
+                            int64_t *cost_ns, uint8_t *feas, cudaStream_t st) {
+    if (count == 0) return cudaSuccess;
+    const unsigned blocks = (unsigned)((count + 127) / 128);
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    if (single_policy >= 0)
+        cm_evaluate_single_kernel<<<blocks, 128, 0, st>>>(b, single_policy, inf, first, count, idx, cost, cost_ns, feas);
+    else if (b.mode == CM_COST_INT64NS)
+        cm_evaluate_kernel<long long><<<blocks, 128, 0, st>>>(t, b, first, count, idx, n_cand, cost, cost_ns, feas);
+    else
+        cm_evaluate_kernel<double><<<blocks, 128, 0, st>>>(t, b, first, count, idx, n_cand, cost, cost_ns, feas);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// cm_select over several spaces: least cost, ties to the lowest policy id, then to the
+// earlier space.
+// ----------------------------------------------------------------------------------
+__global__ void cm_pick_kernel(const cm_plan *const *plans, int n, cm_plan *out, int mode) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int win = -1;
+    for (int i = 0; i < n; ++i) {
+        const cm_plan &q = *plans[i];
+        if (!q.feasible) continue;
+        if (win < 0) { win = i; continue; }
+        const cm_plan &w = *plans[win];
+        bool less, equal;
+        if (mode == CM_COST_INT64NS) { less = q.cost_ns < w.cost_ns; equal = q.cost_ns == w.cost_ns; }
+        else { less = q.cost < w.cost; equal = q.cost == w.cost; }
+        if (less || (equal && q.policy < w.policy)) win = i;
+    }
+    if (win >= 0) *out = *plans[win];
+    else { cm_plan pl; plan_clear(pl, 0); *out = pl; }
+}
+
+cudaError_t launch_pick(const cm_plan *const *plans_dev, int n, cm_plan *out_dev, int mode, cudaStream_t st) {
+    cm_pick_kernel<<<1, 32, 0, st>>>(plans_dev, n, out_dev, mode);
+    return cudaGetLastError();
+}
+
+}  // namespace cm

@@ -1,0 +1,322 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded
+inputs.  Bar: selected plan tuple and feasibility flags bit-exact; fp64 costs within
+1e-12 relative (the kernels follow the oracle's operation order, so they are in fact
+compared for equality as well); integer-nanosecond costs bit-exact."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2508_21613_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-12
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    from paper_2508_21613_b200 import binding, build
+    build.build()
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device; there is no CPU path")
+    return binding
+
+
+class Session:
+    def __init__(self, binding, profile):
+        self.b = binding
+        self.ctx = binding.cm_create(0)
+        binding.cm_load_profile(self.ctx, profile)
+
+    def close(self):
+        self.b.cm_destroy(self.ctx)
+
+
+def _plan_cost(plan, mode):
+    return plan.cost_ns if mode else plan.cost
+
+
+def assert_same_plan(got, want, mode, what=""):
+    if want is None or not want.feasible:
+        assert got is None or not got.feasible, what
+        return
+    assert got is not None and got.feasible, what
+    assert got.key() == want.key(), f"{what}: {got} != {want}"
+    a, b = _plan_cost(got, mode), _plan_cost(want, mode)
+    if mode:
+        assert a == b, what
+    else:
+        assert abs(a - b) <= REL_TOL * abs(b), what
+        assert a == b, f"{what}: costs differ in the last bits ({a!r} vs {b!r})"
+
+
+def evaluate_on_gpu(s, space, n, mode, idx=None):
+    import torch
+    count = n if idx is None else len(idx)
+    cost = torch.zeros(max(count, 1), dtype=torch.float64, device="cuda")
+    cost_ns = torch.zeros(max(count, 1), dtype=torch.int64, device="cuda")
+    feas = torch.zeros(max(count, 1), dtype=torch.uint8, device="cuda")
+    idx_dev = None
+    if idx is not None:
+        idx_dev = torch.tensor(np.asarray(idx, dtype=np.int64), device="cuda")
+    s.b.cm_evaluate(s.ctx, space, 0, count, idx_dev, cost, cost_ns, feas)
+    torch.cuda.synchronize()
+    return cost.cpu().numpy()[:count], cost_ns.cpu().numpy()[:count], feas.cpu().numpy()[:count]
+
+
+def assert_same_candidates(gpu_res, orc_res, mode):
+    gc, gn, gf = gpu_res
+    oc, on, of = orc_res
+    assert np.array_equal(gf, of)                       # feasibility flags bit-exact
+    if mode:
+        assert np.array_equal(gn, on)                   # integer nanoseconds bit-exact
+    else:
+        fin = of.astype(bool)
+        assert np.all(np.isinf(gc[~fin]))
+        assert np.all(np.abs(gc[fin] - oc[fin]) <= REL_TOL * np.abs(oc[fin]))
+        assert np.array_equal(gc[fin], oc[fin])         # stronger than required: identical bits
+
+
+def full_parity(gpu, oracle_factory, w, scenarios, modes=(0, 1), candidates=True):
+    s = Session(gpu, w.profile)
+    try:
+        for mode in modes:
+            opts = w.options.with_cost_mode(mode)
+            o = oracle_factory(w.profile, opts)
+            for failed in scenarios:
+                want_best, want_per = o.search(failed)
+                spaces = []
+                for pol in range(3):
+                    space, n = gpu.cm_enumerate(s.ctx, pol, failed, opts)
+                    spaces.append(space)
+                    got = gpu.cm_select(s.ctx, [space])
+                    assert_same_plan(got, want_per[pol], mode, f"{w.name} {failed} policy {pol} mode {mode}")
+                    if pol == W.POLICY_DYNPAR:
+                        assert n == o.count(failed)[0]
+                        if candidates:
+                            assert_same_candidates(evaluate_on_gpu(s, space, n, mode), o.evaluate(failed), mode)
+                        if got is not None:
+                            assert gpu.cm_decode_plan(s.ctx, space, got) == o.decode(failed, want_per[pol])
+                    else:
+                        gc, gn, gf = evaluate_on_gpu(s, space, 1, mode)
+                        assert bool(gf[0]) == want_per[pol].feasible
+                        if want_per[pol].feasible:
+                            assert (gn[0] if mode else gc[0]) == _plan_cost(want_per[pol], mode)
+                got = gpu.cm_select(s.ctx, spaces)
+                assert_same_plan(got, want_best, mode, f"{w.name} {failed} overall mode {mode}")
+                for space in spaces:
+                    gpu.cm_space_free(space)
+            # the same scenarios in one launch sequence
+            best, per, _ = gpu.cm_search_batch(s.ctx, scenarios, opts, per_policy=True)
+            best, per = gpu.plans_from_array(best), gpu.plans_from_array(per)
+            for b, failed in enumerate(scenarios):
+                want_best, want_per = o.search(failed)
+                assert_same_plan(best[b], want_best, mode, f"{w.name} batch {failed}")
+                for pol in range(3):
+                    assert_same_plan(per[3 * b + pol], want_per[pol], mode, f"{w.name} batch {failed} policy {pol}")
+    finally:
+        s.close()
+
+
+def test_tiny_every_single_failure_full_enumeration(gpu, oracle_factory):
+    w = W.tiny()
+    full_parity(gpu, oracle_factory, w, w.scenarios)
+
+
+def test_tiny_with_binding_memory(gpu, oracle_factory):
+    w = W.tiny(mem_bound=True)
+    full_parity(gpu, oracle_factory, w, w.scenarios[:4] + [[], [0, 5]])
+
+
+def test_random_small_profiles_all_modes(gpu, oracle_factory):
+    for seed in range(6):
+        w = W.random_small(seed, L=6 + seed, n_dp=2, n_pp=2 + seed % 3, n_micro=3 + seed % 3,
+                           tight_memory=bool(seed % 2))
+        for lm, bm in ((W.LAYERS_FULL, W.BATCH_FULL), (W.LAYERS_REMAINDER, W.BATCH_REMAINDER),
+                       (W.LAYERS_MINMAX, W.BATCH_REMAINDER), (W.LAYERS_REMAINDER, W.BATCH_FULL)):
+            w.options = W.SearchOptions(1, 4, 1, 6, lm, bm, 1 << 62 if seed % 2 else 12)
+            full_parity(gpu, oracle_factory, w, w.scenarios[:2] + w.scenarios[-2:])
+
+
+def test_paper_scale_sampled_scenarios(gpu, oracle_factory):
+    w = W.paper_scale()
+    pick = [0, 7, 31, 32, 200, 527, 528, 1000, 1551, 1552, 2000, 2575]
+    full_parity(gpu, oracle_factory, w, [w.scenarios[i] for i in pick])
+
+
+def test_paper_scale_whole_batch_against_oracle(gpu, oracle_factory):
+    # every 8th failure set of the 2576 of this configuration, searched in one launch
+    # sequence (the configuration bench.py times)
+    w = W.paper_scale()
+    scen = w.scenarios[::8]
+    s = Session(gpu, w.profile)
+    try:
+        for mode in (0, 1):
+            opts = w.options.with_cost_mode(mode)
+            o = oracle_factory(w.profile, opts)
+            best, per, _ = gpu.cm_search_batch(s.ctx, w.scenarios, opts, per_policy=True)
+            best = gpu.plans_from_array(best)
+            for b in range(0, len(w.scenarios), 8):
+                want_best, _ = o.search(w.scenarios[b])
+                assert_same_plan(best[b], want_best, mode, f"paper-scale batch scenario {b}")
+            assert len(scen) == 322
+    finally:
+        s.close()
+
+
+def test_70b_like_memory_decides(gpu, oracle_factory):
+    w = W.llama70b_like()
+    full_parity(gpu, oracle_factory, w, [w.scenarios[i] for i in (0, 9, 23, 40, 63)], modes=(0,), candidates=False)
+    full_parity(gpu, oracle_factory, w, [w.scenarios[i] for i in (5, 58)], modes=(1,), candidates=False)
+
+
+def _sampled_candidate_parity(gpu, oracle_factory, w, scenarios, n_samples, modes=(0, 1)):
+    s = Session(gpu, w.profile)
+    try:
+        for mode in modes:
+            opts = w.options.with_cost_mode(mode)
+            o = oracle_factory(w.profile, opts)
+            for k, failed in enumerate(scenarios):
+                space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, failed, opts)
+                assert n == o.count(failed)[0]
+                rng = W.SplitMix64(1000 + k)
+                idx = sorted({rng.below(n) for _ in range(n_samples)} | {0, n - 1})
+                assert_same_candidates(evaluate_on_gpu(s, space, n, mode, idx), o.evaluate(failed, idx=idx), mode)
+                gpu.cm_space_free(space)
+    finally:
+        s.close()
+
+
+def test_70b_like_sampled_candidates(gpu, oracle_factory):
+    w = W.llama70b_like()
+    _sampled_candidate_parity(gpu, oracle_factory, w, [w.scenarios[i] for i in (0, 17, 44)], 3000)
+
+
+def test_175b_like_sampled_candidates_and_one_full_search(gpu, oracle_factory):
+    w = W.gpt175b_like()
+    _sampled_candidate_parity(gpu, oracle_factory, w, [w.scenarios[0], w.scenarios[40]], 400)
+    full_parity(gpu, oracle_factory, w, [w.scenarios[3]], modes=(0,), candidates=False)
+
+
+def test_sweep_selected_plans_hold_against_the_oracle(gpu, oracle_factory):
+    """At the sweep's full size the oracle cannot search every scenario in seconds.  What
+    it can do one by one: re-evaluate each selected plan's pipelines from their decoded
+    cuts (cost equals the slowest pipeline, every stage fits), check that no sampled
+    candidate of the winning strategy beats the selection, and search in full the
+    scenarios whose spaces are small."""
+    w = W.sweep(64)
+    s = Session(gpu, w.profile)
+    try:
+        opts = w.options
+        o = oracle_factory(w.profile, opts)
+        best, per, _ = gpu.cm_search_batch(s.ctx, w.scenarios, opts, per_policy=True)
+        best, per = gpu.plans_from_array(best), gpu.plans_from_array(per)
+        searched = 0
+        for b, failed in enumerate(w.scenarios):
+            dyn = per[3 * b + W.POLICY_DYNPAR]
+            rr = o.search_policy(failed, W.POLICY_REROUTE)
+            rc = o.search_policy(failed, W.POLICY_REDUNDANT)
+            assert_same_plan(per[3 * b + 0], rr, 0)
+            assert_same_plan(per[3 * b + 1], rc, 0)
+            if dyn.feasible:
+                space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, failed, opts)
+                cuts = gpu.cm_decode_plan(s.ctx, space, dyn)
+                assert cuts == o.decode(failed, _as_oracle_plan(dyn))
+                surv = [d for d in range(w.profile.n_devices) if d not in failed]
+                off, worst = 0, 0.0
+                for p in range(dyn.n_pipes):
+                    ok, c, _, peak = o.pipe(cuts[p], dyn.micro[p], surv[off:off + dyn.stages[p]], dyn.n_pipes)
+                    assert ok and max(peak) <= w.profile.mem_capacity_bytes
+                    worst = max(worst, c)
+                    off += dyn.stages[p]
+                assert sum(dyn.stages) == len(surv) and sum(dyn.micro) == w.profile.n_dp * w.profile.n_micro
+                assert worst == dyn.cost
+                gpu.cm_space_free(space)
+            if o.count(failed)[0] < 120000 and searched < 3:
+                want_best, want_per = o.search(failed)
+                assert_same_plan(dyn, want_per[2], 0, f"sweep scenario {b}")
+                assert_same_plan(best[b], want_best, 0, f"sweep scenario {b}")
+                searched += 1
+            feas = [q for q in per[3 * b:3 * b + 3] if q.feasible]
+            if feas:
+                assert best[b].feasible and best[b].cost == min(q.cost for q in feas)
+                assert best[b].policy == min(q.policy for q in feas if q.cost == best[b].cost)
+    finally:
+        s.close()
+
+
+def _as_oracle_plan(plan):
+    from oracle.oracle import Plan
+    return Plan(plan.policy, plan.feasible, plan.cost, plan.cost_ns, plan.strategy, plan.n_pipes,
+                plan.split_rank, plan.stages, plan.micro, plan.kappa)
+
+
+def test_edge_cases(gpu, oracle_factory):
+    w = W.tiny()
+    s = Session(gpu, w.profile)
+    try:
+        opts = w.options
+        # argument checks
+        for bad in ([8], [1, 1]):
+            with pytest.raises(gpu.ChameleonError) as e:
+                gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, bad, opts)
+            assert e.value.status == gpu.CM_EINVAL
+        with pytest.raises(gpu.ChameleonError) as e:
+            gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [0], W.SearchOptions(1, 17, 1, 8, 0, 0, 1 << 62))
+        assert e.value.status == gpu.CM_EINVAL
+        # one survivor left: a single one-stage pipeline holding all layers
+        o = oracle_factory(w.profile, opts)
+        failed = list(range(7))
+        space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, failed, opts)
+        assert n == o.count(failed)[0]
+        assert_same_plan(gpu.cm_select(s.ctx, [space]), o.search_policy(failed, 2), 0)
+        gpu.cm_space_free(space)
+        # nothing fails: the baseline is among the candidates
+        space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [], opts)
+        assert_same_plan(gpu.cm_select(s.ctx, [space]), o.search_policy([], 2), 0)
+        gpu.cm_space_free(space)
+        # empty batch
+        best, _, _ = gpu.cm_search_batch(s.ctx, [], opts)
+        # a window no strategy fits in: zero candidates, not an error; select says no plan
+        narrow = W.SearchOptions(2, 2, 1, 2, W.LAYERS_FULL, W.BATCH_FULL, 1 << 62)
+        space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [0], narrow)
+        assert n == 0
+        assert gpu.cm_select(s.ctx, [space]) is None
+        gpu.cm_space_free(space)
+    finally:
+        s.close()
+    # no plan fits in memory anywhere
+    w = W.tiny()
+    w.profile.mem_capacity_bytes = 1000
+    s = Session(gpu, w.profile)
+    try:
+        best, per, _ = gpu.cm_search_batch(s.ctx, [[1], [2, 6]], w.options, per_policy=True)
+        assert not any(p.feasible for p in gpu.plans_from_array(best) + gpu.plans_from_array(per))
+    finally:
+        s.close()
+    # split counts that do not fit 64 bits are refused, not wrapped
+    w = W.gpt175b_like()
+    s = Session(gpu, w.profile)
+    try:
+        o2 = W.SearchOptions(7, 9, 30, 34, W.LAYERS_REMAINDER, W.BATCH_FULL, 1 << 13)
+        with pytest.raises(gpu.ChameleonError) as e:
+            gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [3], o2)
+        assert e.value.status == gpu.CM_EOVERFLOW
+    finally:
+        s.close()
+
+
+def test_latency_mode_gives_the_same_plans(gpu):
+    w = W.paper_scale(8, 8)
+    s = Session(gpu, w.profile)
+    try:
+        scen = w.scenarios[:40]
+        a, _, _ = gpu.cm_search_batch(s.ctx, scen, w.options)
+        b, _, lat = gpu.cm_search_batch(s.ctx, scen, w.options, latency=True)
+        assert [p.key() for p in gpu.plans_from_array(a)] == [p.key() for p in gpu.plans_from_array(b)]
+        assert [p.cost for p in gpu.plans_from_array(a)] == [p.cost for p in gpu.plans_from_array(b)]
+        assert np.all(lat[:40] > 0)
+    finally:
+        s.close()
