@@ -1,0 +1,320 @@
+"""Benchmark of the execution-plan search: candidate plans evaluated per second and
+plan-search latency per failure on B200.
+
+A step is one pass of the whole hot path (descriptor tables -> min-max partitions ->
+rerouting / redundant-computation plans -> cost kernel over every pipeline-plan ->
+split reduction -> tie-break pass -> policy pick -> plans on the host) over one batch
+of synthetic failure scenarios.  Default workload: the paper-scale configuration
+(32 devices DP4 x PP8, L=32, 2576 failure sets of 1-4 devices, every policy).
+
+  python bench.py --gpus 1 --steps K --warmup W            # this library
+  python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidate_plans_evaluated_per_sec"
+UNIT = "plans/s"
+N_SM = 148
+SM_MAX_MHZ_FALLBACK = 1965.0
+# issue cycles per recurrence cell (2 adds + 1 max of 64-bit values) on sm_100a, where an
+# FP64 instruction holds a scheduler for 2 cycles (16 FP64 lanes per scheduler) and the
+# 64-bit integer max costs 4 half-rate integer instructions:
+#   fp64:  2 DADD (4) + DSETP (2) + 2 SEL (2) = 8       int64: measured 12.3 by a probe kernel
+ISSUE_SLOTS_PER_CELL = {0: 8.0, 1: 12.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": SM_MAX_MHZ_FALLBACK}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def rank_workload(name: str, rank: int):
+    """The workload of one rank.  Ranks beyond 0 draw their random failure sets from their
+    own seeds, so that N GPUs search N different batches of the same shape (weak scaling;
+    no data-path collective: the scenarios are independent)."""
+    from paper_2508_21613_b200 import workloads as W
+    w = W.ALL_WORKLOADS[name]()
+    if rank > 0:
+        rng = W.SplitMix64(0xBEEF + 7919 * rank)
+        n = w.profile.n_devices
+        w.scenarios = [rng.sample_distinct(n, max(1, len(s))) for s in w.scenarios]
+    return w
+
+
+def aggregate(per_rank):
+    """Whole-job numbers from per-rank (plans, seconds) pairs: units summed, time = max."""
+    plans = sum(p for p, _ in per_rank)
+    seconds = max(s for _, s in per_rank)
+    return plans, seconds
+
+
+def oracle_sample(w, mode: int, budget_s: float, max_scenarios: int):
+    """Time the CPU oracle, as it stands, on the first scenarios of the workload until the
+    budget is used.  -> (plans, seconds, scenarios)."""
+    from oracle.oracle import Oracle
+    opts = w.options.with_cost_mode(mode)
+    orc = Oracle(w.profile, opts)
+    plans, t_total, n = 0, 0.0, 0
+    for failed in w.scenarios[:max_scenarios]:
+        t0 = time.perf_counter()
+        orc.search(failed)
+        t_total += time.perf_counter() - t0
+        plans += orc.count(failed)[0] + 2
+        n += 1
+        if t_total >= budget_s:
+            break
+    return plans, t_total, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2508_21613_b200 import workloads as W
+    w = W.ALL_WORKLOADS[args.workload]()
+    per_step = max(1, args.ref_scenarios)
+    for _ in range(args.warmup):
+        oracle_sample(w, args.cost_mode, 1e9, min(2, per_step))
+    plans, seconds = 0, 0.0
+    for k in range(args.steps):
+        sub = W.Workload(w.name, w.profile, w.options, w.scenarios[k * per_step:(k + 1) * per_step] or w.scenarios[:per_step])
+        p, s, _ = oracle_sample(sub, args.cost_mode, 1e9, per_step)
+        plans += p
+        seconds += s
+    value = plans / seconds
+    sample = f"{per_step} failure scenarios of '{w.name}' per step, single thread, all three policies"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * seconds / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "i64" if args.cost_mode else "f64", "data": "synthetic",
+            "config": {"workload": w.name, "scenarios_per_step": per_step, "cost_mode": args.cost_mode},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="paper-scale")
+    ap.add_argument("--cost-mode", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--ref-scenarios", type=int, default=16, help="oracle scenarios per step (--impl reference)")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--latency-scenarios", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scenarios", type=int, default=0, help="use only the first N scenarios (profiling runs)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2508_21613_b200 import binding, build
+    build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the plan search has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    w = rank_workload(args.workload, rank)
+    if args.scenarios > 0:
+        w.scenarios = w.scenarios[:args.scenarios]
+    opts = w.options.with_cost_mode(args.cost_mode)
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    packed = binding.PackedScenarios(w.scenarios)
+    flush = torch.empty(256 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")  # > 126 MB L2
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident arm: descriptors already in HBM when the timed region starts
+    batch, n_cand = packed.prepare(ctx, opts)
+    for _ in range(args.warmup):
+        packed.search_prepared(ctx, batch)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    stats_sum = {}
+    for k in range(args.steps):
+        flush.fill_(float(k))                       # evict L2 between timed iterations (untimed)
+        ev[k][0].record()
+        packed.search_prepared(ctx, batch)          # kernels + plans back on the host
+        ev[k][1].record()
+        st = binding.cm_last_stats(ctx)
+        for key, v in st.items():
+            stats_sum[key] = stats_sum.get(key, 0) + v
+    barrier()
+    clocks = sampler.stop()
+    dev_seconds = sum(a.elapsed_time(b) for a, b in ev) * 1e-3
+    plans_per_step = n_cand + 2 * len(w.scenarios)   # + one rerouting and one redundant plan each
+    binding.cm_batch_free(batch)
+
+    # ---- end-to-end arm: host failure sets in, host plans out, every step
+    for _ in range(args.warmup):
+        packed.search(ctx, opts)
+    barrier()
+    e2e_seconds = 0.0
+    h2d = d2h = 0
+    for k in range(args.steps):
+        flush.fill_(float(k))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        packed.search(ctx, opts)                    # cm_search_batch: build, H2D, kernels, D2H, sync
+        e2e_seconds += time.perf_counter() - t0
+        st = binding.cm_last_stats(ctx)
+        h2d, d2h = st["h2d_bytes"] + packed.ids.nbytes + packed.offsets.nbytes, st["d2h_bytes"]
+    barrier()
+
+    # ---- search latency per failure: scenarios searched one at a time
+    n_lat = min(args.latency_scenarios, len(w.scenarios))
+    lat_pack = binding.PackedScenarios(w.scenarios[:: max(1, len(w.scenarios) // n_lat)][:n_lat])
+    lat_pack.search(ctx, opts, latency=True)
+    lat_pack.search(ctx, opts, latency=True)
+    lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
+
+    if world > 1:
+        t = torch.tensor([float(plans_per_step * args.steps), dev_seconds, e2e_seconds], dtype=torch.float64, device="cuda")
+        gathered = [torch.zeros_like(t) for _ in range(world)]
+        dist.all_gather(gathered, t)
+        rows = [g.cpu().tolist() for g in gathered]
+    else:
+        rows = [[float(plans_per_step * args.steps), dev_seconds, e2e_seconds]]
+    total_plans, max_dev = aggregate([(r[0], r[1]) for r in rows])
+    _, max_e2e = aggregate([(r[0], r[2]) for r in rows])
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        sm_max = float(peaks.get("sm_max_mhz") or SM_MAX_MHZ_FALLBACK)
+        slots = ISSUE_SLOTS_PER_CELL[args.cost_mode]
+        peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
+        cost_s = stats_sum["cost_kernel_ns"] * 1e-9
+        achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
+        line = {
+            "metric": METRIC, "value": total_plans / max_dev, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * max_dev / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "i64" if args.cost_mode else "f64", "data": "synthetic",
+            "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": plans_per_step,
+                       "policies": 3, "cost_mode": "int64ns" if args.cost_mode else "fp64",
+                       "l2": "flushed between timed iterations (256 MB write)",
+                       "parallelism": "replicas, scenarios independent" if world > 1 else "1 gpu"},
+            "e2e": {"value": total_plans / max_e2e, "unit": UNIT, "ms_per_step": 1e3 * max_e2e / args.steps,
+                    "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "timing": "wall clock around cm_search_batch (host descriptor build inside)"},
+            "latency_us": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
+                           "max": float(lat[-1]), "scenarios": int(lat_pack.B),
+                           "what": "one failure set, all policies, descriptor build to plan on host"},
+            "gpu_launches": int(stats_sum["launches"]),
+            "clocks": clocks,
+            "roofline": {
+                "bound": "alu", "kernel": "cm_cost_kernel", "achieved": achieved / 1e9, "peak": peak_cells / 1e9,
+                "unit": "Gcell/s", "frac": achieved / peak_cells if peak_cells else None,
+                "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {sm_max:.0f} MHz ({peak_kind} max clock) / "
+                             f"{slots:.0f} issue slots per cell",
+                "cells_per_launch": stats_sum["cells"] / max(1, stats_sum["cost_kernel_launches"]),
+                "ms_per_launch": 1e3 * cost_s / max(1, stats_sum["cost_kernel_launches"]),
+                "share_of_step": cost_s / dev_seconds if dev_seconds else None,
+                "traffic": None,
+            },
+        }
+        if not args.no_cpu_baseline:
+            p, s, n = oracle_sample(w, args.cost_mode, args.cpu_budget, len(w.scenarios))
+            line["cpu_baseline"] = {"value": p / s, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": f"first {n} failure scenarios of '{w.name}', all three policies, "
+                                              f"{s:.1f} s single-threaded",
+                                    "latency_us_per_failure": 1e6 * s / n}
+        print(json.dumps(line))
+    binding.cm_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
