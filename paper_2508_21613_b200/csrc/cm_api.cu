@@ -70,13 +70,17 @@ struct Batch {
     PinnedVec<Scen> scen;
     PinnedVec<Strat> strat;
     PinnedVec<Seg> seg;
-    PinnedVec<uint32_t> failed, red_scen, keys;
+    PinnedVec<uint32_t> failed, red_scen, keys, order;
+    PinnedVec<Bucket> bucket;
+    std::vector<LaunchClass> classes;
+    std::vector<uint32_t> bin_count;   // scratch of the bucket sort
     PinnedVec<cm_plan> plans_host;
     PinnedVec<unsigned long long> counters_host;
     DevBuf<Scen> d_scen;
     DevBuf<Strat> d_strat;
     DevBuf<Seg> d_seg;
-    DevBuf<uint32_t> d_failed, d_red_scen, d_keys;
+    DevBuf<uint32_t> d_failed, d_red_scen, d_keys, d_order;
+    DevBuf<Bucket> d_bucket;
     DevBuf<uint64_t> d_seg_best, d_kappa_sel, d_pol_cost;
     DevBuf<Partial> d_partial;
     DevBuf<Winner> d_winner;
@@ -178,6 +182,58 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
     if (o->lm < CM_LAYERS_FULL || o->lm > CM_LAYERS_MINMAX) return fail(ctx, CM_EINVAL, "bad layer mode");
     if (o->bm < CM_BATCH_FULL || o->bm > CM_BATCH_REMAINDER) return fail(ctx, CM_EINVAL, "bad batch mode");
     if (o->cost < CM_COST_FP64 || o->cost > CM_COST_INT64NS) return fail(ctx, CM_EINVAL, "bad cost mode");
+    return CM_OK;
+}
+
+// Work layout of the search pass: counting sort of the segments by (stages, micro-batches)
+// into buckets, buckets grouped into launch classes (one per stage count the
+// register-resident kernel covers, one for everything else).
+cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
+    const int G = ctx->hp.G;
+    const size_t stride = (size_t)G + 2, n_bins = (size_t)(CM_MAX_STAGES + 1) * stride;
+    const size_t n_seg = bt.seg.size();
+    bt.bucket.clear();
+    bt.classes.clear();
+    bt.order.clear();
+    if (!bt.order.resize(n_seg)) return fail(ctx, CM_ENOMEM, "host memory");
+    bt.bin_count.assign(n_bins + 1, 0);
+    for (size_t i = 0; i < n_seg; ++i) bt.bin_count[(size_t)bt.seg[i].S * stride + bt.seg[i].m + 1]++;
+    for (size_t b = 0; b < n_bins; ++b) bt.bin_count[b + 1] += bt.bin_count[b];
+    {
+        std::vector<uint32_t> cursor(bt.bin_count.begin(), bt.bin_count.end() - 1);
+        for (size_t i = 0; i < n_seg; ++i) bt.order[cursor[(size_t)bt.seg[i].S * stride + bt.seg[i].m]++] = (uint32_t)i;
+    }
+    // pass 0: register-resident classes, stage count ascending; pass 1: the generic rest
+    for (int pass = 0; pass < 2; ++pass) {
+        LaunchClass generic{0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+        for (int S = 1; S <= CM_MAX_STAGES; ++S) {
+            LaunchClass cls{S, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+            LaunchClass &c = pass == 0 ? cls : generic;
+            for (int m = 0; m <= G + 1; ++m) {
+                const size_t bin = (size_t)S * stride + m;
+                const uint32_t begin = bt.bin_count[bin], end = bt.bin_count[bin + 1];
+                if (begin == end) continue;
+                const bool regs = S <= kRegStagesMax && m >= S - 1 && m >= 1;
+                if (regs != (pass == 0)) continue;
+                const Seg &g = bt.seg[bt.order[begin]];
+                Bucket bk{};
+                bk.count = g.K ? g.K + 1 : 1;
+                bk.chunk_first = c.n_chunks;
+                bk.seg_begin = begin;
+                bk.n_seg = end - begin;
+                bk.S = (uint16_t)S;
+                bk.m = (uint16_t)m;
+                const uint64_t plans = bk.count * bk.n_seg;
+                c.n_chunks += (plans + kChunk - 1) / kChunk;
+                if (!bt.bucket.push(bk)) return fail(ctx, CM_ENOMEM, "host memory");
+                c.bucket_end = (uint32_t)bt.bucket.size();
+            }
+            if (pass == 0 && cls.n_chunks) bt.classes.push_back(cls);
+        }
+        if (pass == 1 && generic.n_chunks) bt.classes.push_back(generic);
+    }
+    for (const LaunchClass &c : bt.classes)
+        if (c.n_chunks >= (1ull << 44)) return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
     return CM_OK;
 }
 
@@ -313,7 +369,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
         red_blocks += sc.n_red;
         if (!bt.scen.push(sc)) return fail(ctx, CM_ENOMEM, "host memory");
     }
-    return CM_OK;
+    return build_buckets(ctx, bt);
 }
 
 template <typename T>
@@ -327,6 +383,7 @@ cm_status upload(cm_ctx *ctx, DevBuf<T> &d, const PinnedVec<T> &h) {
 BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     BatchDev v{};
     v.scen = bt.d_scen.p; v.strat = bt.d_strat.p; v.seg = bt.d_seg.p; v.failed = bt.d_failed.p;
+    v.bucket = bt.d_bucket.p; v.order = bt.d_order.p;
     v.seg_best = bt.d_seg_best.p; v.red_scen = bt.d_red_scen.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p; v.counters = bt.d_counters.p;
@@ -355,6 +412,8 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     if ((s = upload(ctx, bt.d_failed, bt.failed)) != CM_OK) return s;
     if ((s = upload(ctx, bt.d_red_scen, bt.red_scen)) != CM_OK) return s;
     if ((s = upload(ctx, bt.d_keys, bt.keys)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_order, bt.order)) != CM_OK) return s;
+    if ((s = upload(ctx, bt.d_bucket, bt.bucket)) != CM_OK) return s;
     const size_t B = std::max(bt.B, 1);
     bool ok = bt.d_seg_best.reserve(std::max<size_t>(bt.seg.size(), 1)) &&
               bt.d_partial.reserve(std::max<size_t>(bt.red_scen.size(), 1)) && bt.d_winner.reserve(B) &&
@@ -385,7 +444,8 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     }
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
-        if (bt.n_tiles) { CM_CUDA(ctx, launch_cost_pass1(tb, bd, st)); ++launches; ++cost_launches; }
+        CM_CUDA(ctx, launch_cost_pass1(tb, bd, bt.classes.data(), (int)bt.classes.size(), st, &cost_launches));
+        launches += cost_launches;
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
         CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
         launches += bd.n_red_blocks ? 2 : 1;

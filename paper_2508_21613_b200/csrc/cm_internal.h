@@ -67,6 +67,28 @@ struct Scen {
     uint32_t policy_mask, pad;
 };
 
+// Work layout of the search pass: all segments of a batch that share (stages,
+// micro-batches) form a bucket; its pipeline-plans are flattened segment-major
+// (index = segment-in-bucket * count + kappa) and cut into chunks of kChunk plans, one CTA
+// each.  Lanes of a warp therefore run recurrences of identical shape.
+constexpr int kChunk = 128;
+constexpr int kRegStagesMax = 16;   // deepest pipeline the register-resident kernel is built for
+struct Bucket {
+    uint64_t count;        // candidates per segment (K+1 or 1)
+    uint64_t chunk_first;  // first chunk of the bucket within its launch class
+    uint32_t seg_begin;    // first entry of the bucket in the sorted segment order
+    uint32_t n_seg;
+    uint16_t S, m;
+    uint32_t pad;
+};
+
+// Buckets that one kernel instantiation handles: stages == 0 is the generic kernel.
+struct LaunchClass {
+    int stages;
+    uint32_t bucket_begin, bucket_end;
+    uint64_t n_chunks;
+};
+
 // (cost, index) pair carried through the hierarchical argmin of the split reduction.
 struct Partial {
     uint64_t cost_bits;     // cost as an order-preserving 64-bit pattern (inf = infeasible)
@@ -87,6 +109,8 @@ struct BatchDev {
     const Strat *strat;
     const Seg *seg;
     const uint32_t *failed;
+    const Bucket *bucket;   // search-pass work layout
+    const uint32_t *order;  // segment rows sorted by bucket
     uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
     const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
     Partial *partial;       // [n_red_blocks]
@@ -116,7 +140,8 @@ struct Tables {
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, cudaStream_t st);
-cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
+                              cudaStream_t st, int *launches);
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);
 cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st);
 cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st);

@@ -3,7 +3,7 @@
 //   cm_prefix_kernel      per-layer prefix sums and per-boundary transfer times
 //   cm_minmax_kernel      min-max contiguous layer partition per (stages, micro-batches)
 //   cm_policy_kernel      data rerouting and redundant computation, one plan each
-//   cm_cost_kernel        pass 1: every pipeline-plan of every segment -> least cost per segment
+//   (the search pass over every pipeline-plan lives in cm_cost.cu)
 //   cm_split_kernel       (cost, index) argmin over (strategy, micro-batch split) per scenario
 //   cm_winner_kernel      finishes that argmin and decodes the winner
 //   cm_tiebreak_kernel    pass 2: lowest layer composition that meets the winning cost
@@ -270,62 +270,6 @@ __device__ __forceinline__ uint32_t find_row(const Seg *seg, uint32_t n, uint64_
         if (key(seg[mid]) <= q) lo = mid; else hi = mid - 1;
     }
     return lo;
-}
-
-// ----------------------------------------------------------------------------------
-// Pass 1 (generic path): one CTA per tile of kTile consecutive layer compositions of one
-// segment, one thread per pipeline-plan: unrank -> stage sums -> memory check ->
-// recurrence -> sync -> cost; block min -> one atomicMin per CTA on the segment's best.
-// ----------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(kTile) cm_cost_kernel(Tables tb, BatchDev bd) {
-    __shared__ SProf<T> sp;
-    __shared__ uint64_t red[kTile / 32];
-    __shared__ unsigned long long cells[kTile / 32];
-    __shared__ Seg g;
-    const uint64_t tile = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
-    if (tile >= bd.n_tiles) return;
-    stage_profile(sp, tb.prof);
-    if (threadIdx.x == 0) {
-        uint32_t s = find_row(bd.seg, bd.n_seg, tile, [](const Seg &x) { return x.tile_first; });
-        g = bd.seg[s];
-    }
-    __syncthreads();
-    const uint64_t count = g.K ? g.K + 1 : 1;
-    const uint64_t kappa = (tile - g.tile_first) * kTile + threadIdx.x;
-    uint64_t bits = inf_bits<T>();
-    unsigned long long my_cells = 0;
-    if (kappa < count) {
-        T cost;
-        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
-            bits = Num<T>::bits(cost);
-            my_cells = 2ull * g.S * g.m;
-        }
-    }
-    bits = warp_min_u64(bits);
-    for (int o = 16; o > 0; o >>= 1) my_cells += __shfl_xor_sync(0xffffffffu, my_cells, o);
-    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = bits; cells[threadIdx.x >> 5] = my_cells; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned long long c = 0;
-        for (int w = 0; w < kTile / 32; ++w) { bits = red[w] < bits ? red[w] : bits; c += cells[w]; }
-        if (bits != inf_bits<T>()) atomicMin((unsigned long long *)&bd.seg_best[g.row], (unsigned long long)bits);
-        if (c) atomicAdd(&bd.counters[0], c);
-    }
-}
-
-static dim3 tile_grid(uint64_t n_tiles) {
-    const uint64_t maxx = 1u << 30;
-    if (n_tiles <= maxx) return dim3((unsigned)n_tiles, 1, 1);
-    return dim3((unsigned)maxx, (unsigned)((n_tiles + maxx - 1) / maxx), 1);
-}
-
-cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, cudaStream_t st) {
-    if (b.n_tiles == 0) return cudaSuccess;
-    dim3 grid = tile_grid(b.n_tiles);
-    if (b.mode == CM_COST_INT64NS) cm_cost_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
-    else cm_cost_kernel<double><<<grid, kTile, 0, st>>>(t, b);
-    return cudaGetLastError();
 }
 
 // ----------------------------------------------------------------------------------
