@@ -203,18 +203,21 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
         std::vector<uint32_t> cursor(bt.bin_count.begin(), bt.bin_count.end() - 1);
         for (size_t i = 0; i < n_seg; ++i) bt.order[cursor[(size_t)bt.seg[i].S * stride + bt.seg[i].m]++] = (uint32_t)i;
     }
-    // pass 0: register-resident classes, stage count ascending; pass 1: the generic rest
-    for (int pass = 0; pass < 2; ++pass) {
-        LaunchClass generic{0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+    // one class per (kernel kind, stage count); the generic kernel takes the rest in one class
+    auto kind_of = [](int S, int m, uint32_t n_seg) {
+        if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_GENERIC;
+        if (S <= kWideStagesMax) return n_seg >= (uint32_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
+        return (int)CM_CLASS_GENERIC;
+    };
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_GENERIC; ++kind) {
+        LaunchClass generic{CM_CLASS_GENERIC, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
-            LaunchClass cls{S, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
-            LaunchClass &c = pass == 0 ? cls : generic;
-            for (int m = 0; m <= G + 1; ++m) {
+            LaunchClass cls{kind, S, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+            LaunchClass &c = kind == CM_CLASS_GENERIC ? generic : cls;
+            for (int m = 1; m <= G + 1; ++m) {   // m = 0 cannot be feasible: no work is scheduled
                 const size_t bin = (size_t)S * stride + m;
                 const uint32_t begin = bt.bin_count[bin], end = bt.bin_count[bin + 1];
-                if (begin == end) continue;
-                const bool regs = S <= kRegStagesMax && m >= S - 1 && m >= 1;
-                if (regs != (pass == 0)) continue;
+                if (begin == end || kind_of(S, m, end - begin) != kind) continue;
                 const Seg &g = bt.seg[bt.order[begin]];
                 Bucket bk{};
                 bk.count = g.K ? g.K + 1 : 1;
@@ -223,14 +226,19 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 bk.n_seg = end - begin;
                 bk.S = (uint16_t)S;
                 bk.m = (uint16_t)m;
-                const uint64_t plans = bk.count * bk.n_seg;
-                c.n_chunks += (plans + kChunk - 1) / kChunk;
+                if (kind == CM_CLASS_WIDE_UNI) {
+                    const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
+                    c.n_chunks += (items + kChunk / 32 - 1) / (kChunk / 32);
+                } else {
+                    const uint64_t plans = bk.count * bk.n_seg;
+                    c.n_chunks += (plans + kChunk - 1) / kChunk;
+                }
                 if (!bt.bucket.push(bk)) return fail(ctx, CM_ENOMEM, "host memory");
                 c.bucket_end = (uint32_t)bt.bucket.size();
             }
-            if (pass == 0 && cls.n_chunks) bt.classes.push_back(cls);
+            if (kind != CM_CLASS_GENERIC && cls.n_chunks) bt.classes.push_back(cls);
         }
-        if (pass == 1 && generic.n_chunks) bt.classes.push_back(generic);
+        if (kind == CM_CLASS_GENERIC && generic.n_chunks) bt.classes.push_back(generic);
     }
     for (const LaunchClass &c : bt.classes)
         if (c.n_chunks >= (1ull << 44)) return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
@@ -439,7 +447,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     if (bt.seg.size()) CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, bt.seg.size() * sizeof(uint64_t), st));
     CM_CUDA(ctx, cudaMemsetAsync(bt.d_counters.p, 0, 4 * sizeof(unsigned long long), st));
     if (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) {
-        CM_CUDA(ctx, launch_policies(tb, bd, st));
+        CM_CUDA(ctx, launch_policies(tb, bd, ctx->hp.n_dp, st));
         ++launches;
     }
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
@@ -657,7 +665,7 @@ cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids
     if (s == CM_OK && policy != CM_DYNPAR) {
         // the one candidate of these policies is evaluated right away so that
         // cm_evaluate can hand its cost out
-        cudaError_t e = launch_policies(tables(ctx, o.cost), dev_view(ctx, sp->batch), ctx->stream);
+        cudaError_t e = launch_policies(tables(ctx, o.cost), dev_view(ctx, sp->batch), ctx->hp.n_dp, ctx->stream);
         if (e != cudaSuccess) s = fail(ctx, CM_ECUDA, cudaGetErrorString(e));
     }
     if (s != CM_OK) {

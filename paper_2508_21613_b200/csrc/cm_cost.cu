@@ -3,20 +3,23 @@
 // recurrence cells per plan (Section "Estimator", the start/end transition equation;
 // the paper puts the estimator at O(N_pp x N_m) per asymmetric pipeline).
 //
-// Work layout: segments with the same (stages S, micro-batches m) are bucketed, a CTA
-// takes kChunk consecutive pipeline-plans of one bucket, one thread per plan, so all
-// lanes of a warp run recurrences of the same shape.
+// Work layout: segments with the same (stages S, micro-batches m) are bucketed, so all
+// lanes of a warp run recurrences of the same shape.  Three kernels share one evaluation
+// order (sim_rounds below):
 //
-//   cm_cost_regs_kernel<T, S>   S compile-time (1..kRegStagesMax), m >= S-1: the whole
-//       per-plan state -- stage forward/backward/transfer times, per-stage clock and
-//       pending forward -- lives in registers and every loop over stages is unrolled,
-//       so a cell costs its two adds and one max and nothing else.
-//   cm_cost_generic_kernel<T>   any S <= CM_MAX_STAGES and any m: same arithmetic with
-//       the per-stage state in local memory.
-//
-// The recurrence is latency-bound along the backward chain of one plan (each cell needs
-// the previous cell's end) but the forwards of a round are independent of it, and warps
-// of other plans fill the remaining issue slots.
+//   cm_cost_regs_kernel<T, S>       S = 1..16, m >= S-1.  One thread per plan, everything in
+//       registers: stage forward/backward/transfer times, per-stage clock and pending
+//       forward; every loop over stages is unrolled, so a cell costs its two adds and one
+//       max and nothing else.
+//   cm_cost_wide_kernel<T, S, UNI>  S = 17..48.  Clock and pending forward stay in
+//       registers (4 S of them), the stage times move to shared memory.
+//       UNI = true ("transposed"): the 32 lanes of a warp take the SAME layer composition
+//       in 32 DIFFERENT segments of the bucket (they differ in link tiers and sync
+//       peers only), so stage times are warp-uniform -- one broadcast 16-byte load per
+//       stage and round -- and memory feasibility is decided once per warp.
+//       UNI = false: one plan per lane as in the register kernel, stage times in a
+//       per-lane shared-memory column; for buckets with too few segments to transpose.
+//   cm_cost_generic_kernel<T>       any S <= CM_MAX_STAGES: per-stage state in local memory.
 #include "cm_device.cuh"
 
 namespace cm {
@@ -31,7 +34,8 @@ __device__ __forceinline__ uint32_t find_bucket(const Bucket *bk, uint32_t b0, u
     return lo;
 }
 
-// (segment-in-bucket, kappa) of plan `tid` of a chunk whose first plan is `base`.
+// (segment-in-bucket, kappa) of plan `tid` of a chunk whose first plan is `base`
+// (plan-major buckets: index = segment-in-bucket * count + kappa).
 __device__ __forceinline__ void plan_of_thread(uint64_t base, uint64_t count, uint32_t tid,
                                                uint64_t &seg_local, uint64_t &kappa) {
     const uint64_t seg0 = base / count, rem0 = base - seg0 * count;
@@ -128,60 +132,93 @@ __device__ __forceinline__ bool make_walker(CutWalker &w, const Tables &tb, int 
 }
 
 // ----------------------------------------------------------------------------------
-// Register-resident recurrence, S compile-time, m >= S-1 (every stage has its full
-// warm-up).  Same dependency order as sim_pipe; the steady rounds k = 0..m-S need no
-// predicate at all, warm-up and cool-down are unrolled triangles.
+// The recurrence in "rounds", S compile-time, clock and pending forward in registers.
+//
+// Round t = 0 .. S-2+m; stages are visited from last to first.  In round t stage i runs
+//   its forward of micro-batch t-i      if 0 <= t-i < m   (fed by the forward that stage
+//                                        i-1 ran in round t-1 and left pending), then
+//   its backward of micro-batch t-S+1   if t >= S-1       (fed by the backward stage i+1
+//                                        ran just before in the same round; by its own
+//                                        forward at the last stage).
+// Per stage this is exactly the 1F1B order -- min(S-1-i, m) forwards, forward/backward
+// pairs, the remaining backwards -- for every m >= 1, and every dependency is either one
+// round or one stage old, so two values per stage are all the state there is.
+// Rounds S-1 .. m-1 have every stage fully active and carry no predicate at all; the
+// ramp-up and ramp-down rounds skip inactive stages with warp-uniform branches.
+//
+// stage(i) returns the stage's forward and backward time, xt(i) the transfer time of the
+// boundary above stage i; both are called with compile-time i only.
 // ----------------------------------------------------------------------------------
-template <typename T, int S>
-__device__ __forceinline__ T sim_regs(int m, const T (&F)[S], const T (&B)[S], const T (&xt)[S]) {
+template <typename T> struct alignas(16) FB { T f, b; };
+
+// Shared-memory loads the compiler must issue where they stand: the stage times are loop
+// invariants, and hoisting ~100 of them into registers would push the per-stage state out.
+template <typename T>
+__device__ __forceinline__ FB<T> lds_fb(const FB<T> *p) {
+    unsigned long long a, b;
+    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"((unsigned)__cvta_generic_to_shared(p)));
+    FB<T> d;
+    d.f = Num<T>::from_bits(a);
+    d.b = Num<T>::from_bits(b);
+    return d;
+}
+template <typename T>
+__device__ __forceinline__ T lds_t(const T *p) {
+    unsigned long long a;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(a) : "r"((unsigned)__cvta_generic_to_shared(p)));
+    return Num<T>::from_bits(a);
+}
+
+template <typename T, int S, typename StageFn, typename XtFn>
+__device__ __forceinline__ T sim_rounds(int m, StageFn stage, XtFn xt) {
     T clock[S], pend[S];
 #pragma unroll
     for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
-    // warm-up forwards: micro-batch j runs up stages 0 .. S-2-j
+    // ramp-up: forwards only
+    for (int t = 0; t < S - 1; ++t) {
 #pragma unroll
-    for (int j = 0; j < S - 1; ++j) {
-        T chain = (T)0;
-#pragma unroll
-        for (int i = 0; i <= S - 2 - j; ++i) {
-            const T start = i > 0 ? tmax(clock[i], chain) : clock[i];
-            const T end = start + F[i];
-            clock[i] = end;
-            chain = end + xt[i];
+        for (int i = S - 2; i >= 0; --i) {
+            if (i <= t && t < i + m) {
+                const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
+                const T fend = fstart + stage(i).f;
+                clock[i] = fend;
+                pend[i + 1] = fend + xt(i);
+            }
         }
-        pend[S - 1 - j] = chain;
     }
     // steady rounds: every stage does one forward and one backward
-    for (int k = 0; k <= m - S; ++k) {
+    for (int t = S - 1; t < m; ++t) {
         T chain_b = (T)0;
 #pragma unroll
         for (int i = S - 1; i >= 0; --i) {
+            const FB<T> d = stage(i);
+            const T x = i < S - 1 ? xt(i) : (T)0;
             const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-            const T fend = fstart + F[i];
-            if (i < S - 1) pend[i + 1] = fend + xt[i];
-            const T dep = i < S - 1 ? chain_b + xt[i] : fend;
+            const T fend = fstart + d.f;
+            if (i < S - 1) pend[i + 1] = fend + x;
+            const T dep = i < S - 1 ? chain_b + x : fend;
             const T bstart = tmax(fend, dep);
-            const T bend = bstart + B[i];
+            const T bend = bstart + d.b;
             clock[i] = bend;
             chain_b = bend;
         }
     }
-    // cool-down rounds r = 0..S-2: only stages above r still have a forward left
-#pragma unroll
-    for (int r = 0; r < S - 1; ++r) {
+    // ramp-down: every stage still has a backward, the upper ones a forward too
+    for (int t = (m > S - 1 ? m : S - 1); t < S - 1 + m; ++t) {
         T chain_b = (T)0;
 #pragma unroll
         for (int i = S - 1; i >= 0; --i) {
+            const FB<T> d = stage(i);
+            const T x = i < S - 1 ? xt(i) : (T)0;
             T c = clock[i];
-            T fend = (T)0;
-            if (i > r) {
+            if (t < i + m) {
                 const T fstart = i > 0 ? tmax(c, pend[i]) : c;
-                fend = fstart + F[i];
-                c = fend;
-                if (i < S - 1) pend[i + 1] = fend + xt[i];
+                c = fstart + d.f;
+                if (i < S - 1) pend[i + 1] = c + x;
             }
-            const T dep = i < S - 1 ? chain_b + xt[i] : fend;
+            const T dep = i < S - 1 ? chain_b + x : c;
             const T bstart = tmax(c, dep);
-            const T bend = bstart + B[i];
+            const T bend = bstart + d.b;
             clock[i] = bend;
             chain_b = bend;
         }
@@ -189,6 +226,69 @@ __device__ __forceinline__ T sim_regs(int m, const T (&F)[S], const T (&B)[S], c
     return clock[0];
 }
 
+// ----------------------------------------------------------------------------------
+// The same recurrence for shallow pipelines (S <= 16) with m >= S-1, where every stage
+// has its full warm-up: warm-up and cool-down are unrolled triangles without a single
+// branch (S^2 cells of code, affordable at this depth), the steady rounds as above.
+// Order: warm-up forwards micro-batch by micro-batch up the stages, the last forward of
+// a row left pending for the stage above; then rounds k = 0..m-1 from the last stage to
+// the first, forward (while one is left) then backward.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__device__ __forceinline__ T sim_regs(int m, const FB<T> (&st)[S], const T (&xt)[S]) {
+    T clock[S], pend[S];
+#pragma unroll
+    for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
+#pragma unroll
+    for (int j = 0; j < S - 1; ++j) {
+        T chain = (T)0;
+#pragma unroll
+        for (int i = 0; i <= S - 2 - j; ++i) {
+            const T start = i > 0 ? tmax(clock[i], chain) : clock[i];
+            const T end = start + st[i].f;
+            clock[i] = end;
+            chain = end + xt[i];
+        }
+        pend[S - 1 - j] = chain;
+    }
+    for (int k = 0; k <= m - S; ++k) {
+        T chain_b = (T)0;
+#pragma unroll
+        for (int i = S - 1; i >= 0; --i) {
+            const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
+            const T fend = fstart + st[i].f;
+            if (i < S - 1) pend[i + 1] = fend + xt[i];
+            const T dep = i < S - 1 ? chain_b + xt[i] : fend;
+            const T bstart = tmax(fend, dep);
+            const T bend = bstart + st[i].b;
+            clock[i] = bend;
+            chain_b = bend;
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < S - 1; ++r) {
+        T chain_b = (T)0;
+#pragma unroll
+        for (int i = S - 1; i >= 0; --i) {
+            T c = clock[i];
+            if (i > r) {
+                const T fstart = i > 0 ? tmax(c, pend[i]) : c;
+                c = fstart + st[i].f;
+                if (i < S - 1) pend[i + 1] = c + xt[i];
+            }
+            const T dep = i < S - 1 ? chain_b + xt[i] : c;
+            const T bstart = tmax(c, dep);
+            const T bend = bstart + st[i].b;
+            clock[i] = bend;
+            chain_b = bend;
+        }
+    }
+    return clock[0];
+}
+
+// ----------------------------------------------------------------------------------
+// S <= 16: one thread per plan, all in registers.
+// ----------------------------------------------------------------------------------
 template <typename T, int S>
 __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
     __shared__ SProf<T> sp;
@@ -204,34 +304,160 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
     uint32_t row = 0xffffffffu;
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
-    if (seg_local < bk.n_seg) {
+    if (seg_local < bk.n_seg && m >= 1) {
         row = bd.order[bk.seg_begin + seg_local];
         const Seg *g = bd.seg + row;
         const uint64_t tier = g->tier_mask, K = g->K;
         const int n_sync = g->n_sync;
         CutWalker cw;
         bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, K, g->mm_slot);
-        T F[S], B[S], xt[S];
+        FB<T> st[S];
+        T xts[S];
         long long g_max = 0;
         int lo = 0;
 #pragma unroll
         for (int i = 0; i < S; ++i) {
             const int hi = ok ? cw.next() : lo + 1;
             ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-            F[i] = sp.PF[hi] - sp.PF[lo];
-            B[i] = sp.PB[hi] - sp.PB[lo];
-            xt[i] = i < S - 1 ? sp.XT[(tier >> i) & 1ull][hi - 1] : (T)0;
+            st[i].f = sp.PF[hi] - sp.PF[lo];
+            st[i].b = sp.PB[hi] - sp.PB[lo];
+            xts[i] = i < S - 1 ? sp.XT[(tier >> i) & 1ull][hi - 1] : (T)0;
             const long long gb = sp.PP[hi] - sp.PP[lo];
             g_max = gb > g_max ? gb : g_max;
             lo = hi;
         }
         if (ok) {
-            const T t = sim_regs<T, S>(m, F, B, xt);
+            const T t = sim_regs<T, S>(m, st, xts);
             bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync));
             my_cells = 2ull * S * m;
         }
     }
     segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+// ----------------------------------------------------------------------------------
+// 16 < S <= 48: stage times in shared memory.
+// Dynamic shared memory:  UNI:  FB<T> fb[4 warps][S] | T xt[S][128] | uint8 cuts[4][S+1]
+//                         !UNI: FB<T> fb[S][128]     | T xt[S][128]
+// ----------------------------------------------------------------------------------
+#ifndef CM_WIDE3
+#define CM_WIDE3 34   // deepest pipeline compiled for three resident CTAs per SM (<= 168 registers)
+#endif
+template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
+    return UNI ? sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8)
+               : sizeof(FB<T>) * S * kChunk + sizeof(T) * S * kChunk;
+}
+
+template <typename T, int S, bool UNI>
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint64_t chunk = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const int m = bk.m, L = sp.L;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    unsigned long long my_cells = 0;
+
+    if (UNI) {
+        FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+        uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
+        // warp item = (kappa, group of 32 segments), group minor
+        const uint64_t item = (chunk - bk.chunk_first) * (kChunk / 32) + warp;
+        const uint32_t n_groups = (bk.n_seg + 31) / 32;
+        const uint64_t kappa = item / n_groups;
+        const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
+        if (kappa < bk.count && m >= 1) {           // warp-uniform
+            const bool active = seg_local < bk.n_seg;
+            const uint32_t row = bd.order[bk.seg_begin + (active ? seg_local : 0)];
+            const Seg *g = bd.seg + row;
+            const uint64_t tier = g->tier_mask;
+            const int n_sync = g->n_sync;
+            // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
+            CutWalker cw;
+            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g->K, g->mm_slot);
+            if (ok) {
+                int lo = 0;
+                for (int i = 0; i < S; ++i) {
+                    const int hi = cw.next();
+                    ok = ok && hi > lo;
+                    if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+                    lo = hi;
+                }
+                if (lane == 0) cuts[0] = 0;
+            }
+            __syncwarp();
+            long long g_max = 0;
+            if (ok) {
+                // stage sums and the memory check, one stage per lane
+                for (int i = lane; i < S; i += 32) {
+                    const int lo = cuts[i], hi = cuts[i + 1];
+                    ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                    FB<T> d;
+                    d.f = sp.PF[hi] - sp.PF[lo];
+                    d.b = sp.PB[hi] - sp.PB[lo];
+                    fb[i] = d;
+                    const long long gb = sp.PP[hi] - sp.PP[lo];
+                    g_max = gb > g_max ? gb : g_max;
+                }
+                for (int o = 16; o > 0; o >>= 1) {
+                    const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+                    g_max = og > g_max ? og : g_max;
+                }
+                // transfer times of this lane's segment (its own link tiers)
+                for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(tier >> i) & 1ull][cuts[i + 1] - 1];
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            __syncwarp();
+            if (ok) {
+                const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+                if (active) {
+                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync));
+                    if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
+                    my_cells = 2ull * S * m;
+                }
+            }
+        }
+    } else {
+        FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + tid;                               // [i * kChunk]
+        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + tid;           // [i * kChunk]
+        const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+        uint64_t seg_local, kappa;
+        plan_of_thread(base, bk.count, tid, seg_local, kappa);
+        uint32_t row = 0xffffffffu;
+        uint64_t bits = inf_bits<T>();
+        if (seg_local < bk.n_seg && m >= 1) {
+            row = bd.order[bk.seg_begin + seg_local];
+            const Seg *g = bd.seg + row;
+            const uint64_t tier = g->tier_mask;
+            CutWalker cw;
+            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g->K, g->mm_slot);
+            long long g_max = 0;
+            int lo = 0;
+            for (int i = 0; i < S && ok; ++i) {
+                const int hi = cw.next();
+                ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                FB<T> d;
+                d.f = sp.PF[hi] - sp.PF[lo];
+                d.b = sp.PB[hi] - sp.PB[lo];
+                fcol[i * kChunk] = d;
+                xcol[i * kChunk] = i < S - 1 ? sp.XT[(tier >> i) & 1ull][hi - 1] : (T)0;
+                const long long gb = sp.PP[hi] - sp.PP[lo];
+                g_max = gb > g_max ? gb : g_max;
+                lo = hi;
+            }
+            if (ok) {
+                const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+                bits = Num<T>::bits(t + Num<T>::sync(g_max, g->n_sync, sp.bw_sync));
+                my_cells = 2ull * S * m;
+            }
+        }
+        segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    }
     count_cells(&bd.counters[0], my_cells, cells_w);
 }
 
@@ -269,45 +495,64 @@ static dim3 chunk_grid(uint64_t n) {
 }
 
 template <typename T, int S>
-static void launch_regs(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+static cudaError_t launch_regs(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
     cm_cost_regs_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    return cudaGetLastError();
+}
+
+template <typename T, int S, bool UNI>
+static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, UNI, T>();
+    static bool configured[16] = {false};   // per device; the attribute sticks to the function
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 16 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(cm_cost_wide_kernel<T, S, UNI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    return cudaGetLastError();
+}
+
+template <typename T, int S>
+static cudaError_t launch_wide(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : launch_wide_one<T, S, false>(t, b, c, st);
 }
 
 template <typename T>
-static void launch_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    switch (c.stages) {
-    case 1: launch_regs<T, 1>(t, b, c, st); break;
-    case 2: launch_regs<T, 2>(t, b, c, st); break;
-    case 3: launch_regs<T, 3>(t, b, c, st); break;
-    case 4: launch_regs<T, 4>(t, b, c, st); break;
-    case 5: launch_regs<T, 5>(t, b, c, st); break;
-    case 6: launch_regs<T, 6>(t, b, c, st); break;
-    case 7: launch_regs<T, 7>(t, b, c, st); break;
-    case 8: launch_regs<T, 8>(t, b, c, st); break;
-    case 9: launch_regs<T, 9>(t, b, c, st); break;
-    case 10: launch_regs<T, 10>(t, b, c, st); break;
-    case 11: launch_regs<T, 11>(t, b, c, st); break;
-    case 12: launch_regs<T, 12>(t, b, c, st); break;
-    case 13: launch_regs<T, 13>(t, b, c, st); break;
-    case 14: launch_regs<T, 14>(t, b, c, st); break;
-    case 15: launch_regs<T, 15>(t, b, c, st); break;
-    case 16: launch_regs<T, 16>(t, b, c, st); break;
-    default:
-        cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end);
-        break;
+static cudaError_t launch_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    if (c.kind == CM_CLASS_REGS) {
+        switch (c.stages) {
+#define CM_CASE(S) case S: return launch_regs<T, S>(t, b, c, st);
+            CM_CASE(1) CM_CASE(2) CM_CASE(3) CM_CASE(4) CM_CASE(5) CM_CASE(6) CM_CASE(7) CM_CASE(8)
+            CM_CASE(9) CM_CASE(10) CM_CASE(11) CM_CASE(12) CM_CASE(13) CM_CASE(14) CM_CASE(15) CM_CASE(16)
+#undef CM_CASE
+        default: break;
+        }
+    } else if (c.kind == CM_CLASS_WIDE_UNI || c.kind == CM_CLASS_WIDE_LANE) {
+        switch (c.stages) {
+#define CM_CASE(S) case S: return launch_wide<T, S>(t, b, c, st);
+            CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
+            CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
+            CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
+            CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
+#undef CM_CASE
+        default: break;
+        }
     }
+    cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    return cudaGetLastError();
 }
 
-// The chunks of a class beyond its last bucket's plans are empty lanes; a chunk index
-// past n_chunks cannot occur because the grid is exactly n_chunks (x * y may overshoot
-// only in the 2-D case, where the surplus CTAs find the last bucket and idle).
+// A 2-D grid may overshoot the class's chunk count; surplus CTAs find the last bucket,
+// see indices past its plans and idle.
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
                               cudaStream_t st, int *launches) {
     for (int i = 0; i < n_classes; ++i) {
         if (classes[i].n_chunks == 0) continue;
-        if (b.mode == CM_COST_INT64NS) launch_class<long long>(t, b, classes[i], st);
-        else launch_class<double>(t, b, classes[i], st);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = b.mode == CM_COST_INT64NS ? launch_class<long long>(t, b, classes[i], st)
+                                                  : launch_class<double>(t, b, classes[i], st);
         if (e != cudaSuccess) return e;
         if (launches) ++*launches;
     }

@@ -82,9 +82,14 @@ struct Bucket {
     uint32_t pad;
 };
 
-// Buckets that one kernel instantiation handles: stages == 0 is the generic kernel.
+// Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
+// flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
+// transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
+enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_GENERIC = 3 };
+constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
+constexpr int kUniMinSegments = 16; // fewer segments in a bucket: not worth transposing
 struct LaunchClass {
-    int stages;
+    int kind, stages;
     uint32_t bucket_begin, bucket_end;
     uint64_t n_chunks;
 };
@@ -139,7 +144,7 @@ struct Tables {
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
-cudaError_t launch_policies(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st);
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
                               cudaStream_t st, int *launches);
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);

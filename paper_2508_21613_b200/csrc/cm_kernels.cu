@@ -2,7 +2,7 @@
 //
 //   cm_prefix_kernel      per-layer prefix sums and per-boundary transfer times
 //   cm_minmax_kernel      min-max contiguous layer partition per (stages, micro-batches)
-//   cm_policy_kernel      data rerouting and redundant computation, one plan each
+//   (data rerouting / redundant computation: cm_policy.cu)
 //   (the search pass over every pipeline-plan lives in cm_cost.cu)
 //   cm_split_kernel       (cost, index) argmin over (strategy, micro-batch split) per scenario
 //   cm_winner_kernel      finishes that argmin and decodes the winner
@@ -126,135 +126,6 @@ cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys,
     if (n_keys <= 0) return cudaSuccess;
     if (mode == CM_COST_INT64NS) cm_minmax_kernel<long long><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
     else cm_minmax_kernel<double><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
-    return cudaGetLastError();
-}
-
-// ----------------------------------------------------------------------------------
-// Data rerouting and redundant computation: one plan per scenario each.
-//
-// Rerouting (Section "Estimator", single- and multi-failure step time): the failed
-// devices' micro-batches go to the data-parallel peers of the same stage; with F_i
-// failed devices in stage i the step grows by N_m F_i (F_i^st + B_i^st) / (N_dp - F_i) per
-// affected stage on top of the unchanged base pipeline; unrecoverable if F_i >= N_dp.
-//
-// Redundant computation (Section "Limitations of Backup-free Methods", prose): a failed
-// stage is taken over by its predecessor; every stage but the last also carries its
-// successor's work and state.  Infeasible if stage 0 failed or two neighbours failed.
-//
-// One warp per scenario: lane 0 evaluates rerouting, lane 1+k pipeline k of the
-// redundant plan; a shuffle max combines the pipelines.
-// ----------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(32) cm_policy_kernel(Tables tb, BatchDev bd) {
-    __shared__ SProf<T> sp;
-    __shared__ int base_cuts[kMaxS + 1];
-    const DevProfile *p = tb.prof;
-    stage_profile(sp, p);
-    for (int i = threadIdx.x; i <= p->n_pp; i += blockDim.x) base_cuts[i] = p->base_cuts[i];
-    __syncthreads();
-    const int b = blockIdx.x;
-    const Scen sc = bd.scen[b];
-    const uint32_t *failed = bd.failed + sc.failed_first;
-    const int S0 = sp.n_pp, m = sp.n_micro, n_dp = sp.n_dp;
-    const int lane = threadIdx.x;
-    const int dpn = p->devices_per_node;
-    T F[kMaxS], B[kMaxS], xt[kMaxS], clock[kMaxS], pend[kMaxS];
-
-    if (lane == 0) {
-        uint64_t out = inf_bits<T>();
-        if (sc.policy_mask & (1u << CM_REROUTE)) {
-            int fcnt[kMaxS];
-            for (int i = 0; i < S0; ++i) fcnt[i] = 0;
-            for (uint32_t f = 0; f < sc.n_failed; ++f) fcnt[failed[f] % S0]++;
-            bool ok = m >= 1;
-            for (int i = 0; i < S0; ++i) ok = ok && fcnt[i] < n_dp;
-            for (int i = 0; i < S0 && ok; ++i) {
-                const int lo = base_cuts[i], hi = base_cuts[i + 1];
-                ok = stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap);
-            }
-            if (ok) {
-                T extra = (T)0, t_sync = (T)0;
-                for (int i = 0; i < S0; ++i) {
-                    const int lo = base_cuts[i], hi = base_cuts[i + 1];
-                    F[i] = sp.PF[hi] - sp.PF[lo];
-                    B[i] = sp.PB[hi] - sp.PB[lo];
-                    // pipeline 0 sits on devices 0 .. S0-1
-                    const int tier = (i / dpn == (i + 1) / dpn) ? 0 : 1;
-                    xt[i] = i < S0 - 1 ? sp.XT[tier][hi - 1] : (T)0;
-                    if (fcnt[i] > 0) extra = extra + Num<T>::reroute_extra(m * fcnt[i], F[i] + B[i], n_dp - fcnt[i]);
-                    t_sync = tmax(t_sync, Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt[i], sp.bw_sync));
-                }
-                T base = sim_pipe<T>(S0, m, F, B, xt, clock, pend);
-                out = Num<T>::bits((base + extra) + t_sync);
-            }
-        }
-        bd.pol_cost[2 * b + 0] = out;
-    }
-
-    // redundant computation: lanes 1..n_dp
-    T my_cost = (T)0;
-    bool my_ok = true;
-    int my_S = 0;
-    const int k = lane - 1;
-    if (k >= 0 && k < n_dp) {
-        uint64_t dead = 0;
-        for (uint32_t f = 0; f < sc.n_failed; ++f)
-            if ((int)(failed[f] / S0) == k) dead |= 1ull << (failed[f] % S0);
-        if (dead & 1ull) my_ok = false;
-        if (dead & (dead >> 1)) my_ok = false;
-        if (m < 1) my_ok = false;
-        if (my_ok) {
-            int cuts[kMaxS + 1], devs[kMaxS];
-            int S = 0;
-            cuts[0] = 0;
-            for (int i = 0; i < S0; ++i) {
-                if ((dead >> i) & 1ull) continue;
-                int hi = base_cuts[i + 1];
-                if (i + 1 < S0 && ((dead >> (i + 1)) & 1ull)) hi = base_cuts[i + 2];
-                devs[S] = k * S0 + i;
-                cuts[S + 1] = hi;
-                ++S;
-            }
-            my_S = S;
-            long long g_max = 0;
-            for (int i = 0; i < S && my_ok; ++i) {
-                const int lo = cuts[i], hi = cuts[i + 1];
-                long long stat = sp.PS[hi] - sp.PS[lo], act = sp.PA[hi] - sp.PA[lo];
-                T f = sp.PF[hi] - sp.PF[lo], bw = sp.PB[hi] - sp.PB[lo];
-                if (i < S - 1) {
-                    const int hi2 = cuts[i + 2];
-                    f = f + (sp.PF[hi2] - sp.PF[hi]);
-                    bw = bw + (sp.PB[hi2] - sp.PB[hi]);
-                    stat = stat + (sp.PS[hi2] - sp.PS[hi]);
-                    act = act + (sp.PA[hi2] - sp.PA[hi]);
-                    const int tier = (devs[i] / dpn == devs[i + 1] / dpn) ? 0 : 1;
-                    xt[i] = sp.XT[tier][hi - 1];
-                } else {
-                    xt[i] = (T)0;
-                }
-                F[i] = f;
-                B[i] = bw;
-                if (!stage_fits(stat, act, i, S, m, sp.cap)) my_ok = false;
-                long long g = sp.PP[hi] - sp.PP[lo];
-                g_max = g > g_max ? g : g_max;
-            }
-            if (my_ok) my_cost = sim_pipe<T>(S, m, F, B, xt, clock, pend) + Num<T>::sync(g_max, n_dp, sp.bw_sync);
-        }
-    }
-    uint64_t bits = my_ok ? Num<T>::bits(my_cost) : inf_bits<T>();
-    // slowest pipeline sets the step; an infeasible pipeline (inf) wins the max
-    for (int o = 16; o > 0; o >>= 1) {
-        uint64_t w = __shfl_xor_sync(0xffffffffu, bits, o);
-        bits = w > bits ? w : bits;
-    }
-    if (k >= 0 && k < n_dp && k < kMaxP) bd.rc_stages[b * kMaxP + k] = (uint16_t)my_S;
-    if (lane == 0) bd.pol_cost[2 * b + 1] = (sc.policy_mask & (1u << CM_REDUNDANT)) ? bits : inf_bits<T>();
-}
-
-cudaError_t launch_policies(const Tables &t, const BatchDev &b, cudaStream_t st) {
-    if (b.B <= 0) return cudaSuccess;
-    if (b.mode == CM_COST_INT64NS) cm_policy_kernel<long long><<<b.B, 32, 0, st>>>(t, b);
-    else cm_policy_kernel<double><<<b.B, 32, 0, st>>>(t, b);
     return cudaGetLastError();
 }
 
