@@ -66,21 +66,25 @@ inline uint64_t sat_add(uint64_t a, uint64_t b) { return a > kSat - b ? kSat : a
 }  // namespace
 
 // One batch of failure scenarios: host tables, device mirrors, result buffers.
+// All descriptor tables are small (templates per survivor count plus ~100 bytes per
+// scenario), so they are packed into one pinned arena and reach the device in one copy.
 struct Batch {
-    PinnedVec<Scen> scen;
-    PinnedVec<Strat> strat;
-    PinnedVec<Seg> seg;
-    PinnedVec<uint32_t> failed, red_scen, keys, order;
-    PinnedVec<Bucket> bucket;
+    std::vector<Scen> scen;
+    std::vector<Tmpl> tmpl;
+    std::vector<Strat> strat;
+    std::vector<TSeg> tseg;
+    std::vector<uint32_t> failed, red_scen, keys, tmpl_scen, bucket_tseg;
+    std::vector<uint64_t> cross;
+    std::vector<Bucket> bucket;
     std::vector<LaunchClass> classes;
-    std::vector<uint32_t> bin_count;   // scratch of the bucket sort
+    std::vector<int> tmpl_of_nsurv;        // survivor count -> template, -1 = not built
+    std::vector<uint16_t> strategies;      // scratch: flattened stage-count tuples
+    PinnedVec<unsigned char> arena;        // host image of the tables
+    DevBuf<unsigned char> d_arena;
+    size_t off_scen = 0, off_tmpl = 0, off_strat = 0, off_tseg = 0, off_failed = 0, off_red = 0, off_keys = 0,
+           off_tmpl_scen = 0, off_bucket_tseg = 0, off_cross = 0, off_bucket = 0;
     PinnedVec<cm_plan> plans_host;
     PinnedVec<unsigned long long> counters_host;
-    DevBuf<Scen> d_scen;
-    DevBuf<Strat> d_strat;
-    DevBuf<Seg> d_seg;
-    DevBuf<uint32_t> d_failed, d_red_scen, d_keys, d_order;
-    DevBuf<Bucket> d_bucket;
     DevBuf<uint64_t> d_seg_best, d_kappa_sel, d_pol_cost;
     DevBuf<Partial> d_partial;
     DevBuf<Winner> d_winner;
@@ -90,6 +94,7 @@ struct Batch {
     cm_enum_opts opts{};
     uint32_t policy_mask = 0;
     uint64_t n_cand = 0, n_tiles = 0, n_split = 0;
+    uint64_t n_rows = 0;                   // rows of seg_best over all scenarios
     uint32_t max_tiles_per_seg = 0, dp_max = 0;
     int B = 0;
     bool uploaded = false;
@@ -118,7 +123,6 @@ struct cm_space {
     int policy = 0;
     Batch batch;
     std::vector<uint32_t> failed;
-    std::vector<int> strat_dp;                    // decode: pipelines per strategy
 };
 
 struct cm_batch {
@@ -185,55 +189,69 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
     return CM_OK;
 }
 
-// Work layout of the search pass: counting sort of the segments by (stages, micro-batches)
-// into buckets, buckets grouped into launch classes (one per stage count the
-// register-resident kernel covers, one for everything else).
+// Work layout of the search pass: the template segments of every template are grouped by
+// (stages, micro-batches) into buckets (a bucket's segments are its template segments
+// times the template's scenarios), buckets grouped into launch classes: one per
+// (kernel kind, stage count), the generic kernel takes the rest in one class.
 cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
-    const int G = ctx->hp.G;
-    const size_t stride = (size_t)G + 2, n_bins = (size_t)(CM_MAX_STAGES + 1) * stride;
-    const size_t n_seg = bt.seg.size();
     bt.bucket.clear();
     bt.classes.clear();
-    bt.order.clear();
-    if (!bt.order.resize(n_seg)) return fail(ctx, CM_ENOMEM, "host memory");
-    bt.bin_count.assign(n_bins + 1, 0);
-    for (size_t i = 0; i < n_seg; ++i) bt.bin_count[(size_t)bt.seg[i].S * stride + bt.seg[i].m + 1]++;
-    for (size_t b = 0; b < n_bins; ++b) bt.bin_count[b + 1] += bt.bin_count[b];
-    {
-        std::vector<uint32_t> cursor(bt.bin_count.begin(), bt.bin_count.end() - 1);
-        for (size_t i = 0; i < n_seg; ++i) bt.order[cursor[(size_t)bt.seg[i].S * stride + bt.seg[i].m]++] = (uint32_t)i;
-    }
-    // one class per (kernel kind, stage count); the generic kernel takes the rest in one class
-    auto kind_of = [](int S, int m, uint32_t n_seg) {
+    bt.bucket_tseg.clear();
+    struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; };
+    std::vector<Pre> pre;
+    auto kind_of = [](int S, int m, uint64_t n_seg) {
         if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_GENERIC;
-        if (S <= kWideStagesMax) return n_seg >= (uint32_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
+        if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
         return (int)CM_CLASS_GENERIC;
     };
+    std::vector<uint32_t> idx;
+    for (size_t t = 0; t < bt.tmpl.size(); ++t) {
+        const Tmpl &tp = bt.tmpl[t];
+        if (tp.n_scen == 0 || tp.n_tseg == 0) continue;
+        idx.resize(tp.n_tseg);
+        for (uint32_t i = 0; i < tp.n_tseg; ++i) idx[i] = tp.tseg_first + i;
+        std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
+            const TSeg &x = bt.tseg[a], &y = bt.tseg[b];
+            return x.S != y.S ? x.S < y.S : x.m < y.m;
+        });
+        for (size_t i = 0; i < idx.size();) {
+            size_t j = i;
+            const TSeg &g = bt.tseg[idx[i]];
+            while (j < idx.size() && bt.tseg[idx[j]].S == g.S && bt.tseg[idx[j]].m == g.m) ++j;
+            if (g.m >= 1) {   // m = 0 cannot be feasible: no work is scheduled
+                const uint64_t n_seg = (uint64_t)(j - i) * tp.n_scen;
+                if (n_seg >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "too many segments in one bucket");
+                Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(j - i), g.S, g.m,
+                      g.K ? g.K + 1 : 1, (uint32_t)n_seg, kind_of(g.S, g.m, n_seg)};
+                for (size_t k = i; k < j; ++k) bt.bucket_tseg.push_back(idx[k]);
+                pre.push_back(q);
+            }
+            i = j;
+        }
+    }
     for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_GENERIC; ++kind) {
         LaunchClass generic{CM_CLASS_GENERIC, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
             LaunchClass cls{kind, S, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
             LaunchClass &c = kind == CM_CLASS_GENERIC ? generic : cls;
-            for (int m = 1; m <= G + 1; ++m) {   // m = 0 cannot be feasible: no work is scheduled
-                const size_t bin = (size_t)S * stride + m;
-                const uint32_t begin = bt.bin_count[bin], end = bt.bin_count[bin + 1];
-                if (begin == end || kind_of(S, m, end - begin) != kind) continue;
-                const Seg &g = bt.seg[bt.order[begin]];
+            for (const Pre &q : pre) {
+                if (q.kind != kind || q.S != S) continue;
                 Bucket bk{};
-                bk.count = g.K ? g.K + 1 : 1;
+                bk.count = q.count;
                 bk.chunk_first = c.n_chunks;
-                bk.seg_begin = begin;
-                bk.n_seg = end - begin;
-                bk.S = (uint16_t)S;
-                bk.m = (uint16_t)m;
+                bk.list_first = q.list_first;
+                bk.n_tseg = q.n_tseg;
+                bk.tmpl = q.tmpl;
+                bk.n_seg = q.n_seg;
+                bk.S = q.S;
+                bk.m = q.m;
                 if (kind == CM_CLASS_WIDE_UNI) {
                     const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
                     c.n_chunks += (items + kChunk / 32 - 1) / (kChunk / 32);
                 } else {
-                    const uint64_t plans = bk.count * bk.n_seg;
-                    c.n_chunks += (plans + kChunk - 1) / kChunk;
+                    c.n_chunks += (bk.count * bk.n_seg + kChunk - 1) / kChunk;
                 }
-                if (!bt.bucket.push(bk)) return fail(ctx, CM_ENOMEM, "host memory");
+                bt.bucket.push_back(bk);
                 c.bucket_end = (uint32_t)bt.bucket.size();
             }
             if (kind != CM_CLASS_GENERIC && cls.n_chunks) bt.classes.push_back(cls);
@@ -245,158 +263,208 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     return CM_OK;
 }
 
-// Build the descriptor tables of a batch on the host.
+// The template of a survivor count (Algorithm 1, get_parallel_strategy, plus the batch
+// and layer distribution rules of Section "Planner"): strategies, their micro-batch split
+// ranges and one template segment per (strategy, pipeline, micro-batch count).
+cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
+    const DevProfile &hp = ctx->hp;
+    const cm_enum_opts &o = bt.opts;
+    const int L = hp.L, G = hp.G;
+    const int dp_lo = std::max(1, (int)o.dp_lo), dp_hi = std::min((int)o.dp_hi, CM_MAX_PIPES);
+    const int pp_lo = std::max(1, (int)o.pp_lo), pp_hi = std::min(std::min((int)o.pp_hi, L), CM_MAX_STAGES);
+    std::vector<uint8_t> &mm_done = ctx->mm_done[o.cost];
+    Tmpl tp{};
+    tp.strat_first = (uint32_t)bt.strat.size();
+    tp.tseg_first = (uint32_t)bt.tseg.size();
+    std::vector<std::vector<uint16_t>> strategies;
+    if (n_surv > 0 && pp_lo <= pp_hi) enum_strategies(n_surv, dp_lo, dp_hi, pp_lo, pp_hi, strategies);
+    uint64_t split_first = 0, cand = 0;
+    for (const auto &tuple : strategies) {
+        Strat st{};
+        const int dp = (int)tuple.size();
+        st.dp = (uint16_t)dp;
+        st.seg_first = (uint32_t)bt.tseg.size();
+        st.split_first = split_first;
+        bt.dp_max = std::max<uint32_t>(bt.dp_max, (uint32_t)dp);
+        int sum = 0;
+        for (int p = 0; p < dp; ++p) {
+            st.S[p] = tuple[p];
+            if (o.bm == CM_BATCH_REMAINDER) {
+                st.m_lo[p] = (uint16_t)(((int64_t)G * tuple[p]) / n_surv);
+                sum += st.m_lo[p];
+            } else {
+                st.m_lo[p] = 1;
+            }
+        }
+        if (o.bm == CM_BATCH_REMAINDER) {
+            st.R = (uint16_t)(G - sum);
+            st.n_m = st.R > 0 ? 2 : 1;
+            st.n_split = hbinom(ctx, dp, st.R);
+        } else {
+            st.R = 0;
+            st.n_m = (uint16_t)(G >= dp ? G - dp + 1 : 0);
+            st.n_split = G >= dp ? hbinom(ctx, G - 1, dp - 1) : 0;
+        }
+        if (st.n_split == kSat) return fail(ctx, CM_EOVERFLOW, "micro-batch split count overflows 64 bits");
+        split_first = sat_add(split_first, st.n_split);
+        if (split_first >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "too many micro-batch splits");
+        int off = 0;
+        for (int p = 0; p < dp; ++p) {
+            const int S = tuple[p];
+            uint64_t K = 0;
+            if (o.lm == CM_LAYERS_REMAINDER) K = hbinom(ctx, S, L % S);
+            else if (o.lm == CM_LAYERS_FULL) K = hbinom(ctx, L - 1, S - 1);
+            if (o.lm == CM_LAYERS_MINMAX || K > o.kappa_cap) K = 0;
+            if (K >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "layer composition count overflows");
+            for (int mi = 0; mi < st.n_m; ++mi) {
+                TSeg g{};
+                g.S = (uint16_t)S;
+                g.m = (uint16_t)(st.m_lo[p] + mi);
+                g.n_sync = (uint16_t)dp;
+                g.off = (uint16_t)off;
+                g.K = K;
+                g.cand_first = cand;
+                const uint64_t count = K ? K + 1 : 1;
+                const uint64_t tiles = (count + kTile - 1) / kTile;
+                cand = sat_add(cand, count);
+                if (cand >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
+                if (tiles > 0x7fffffffu) return fail(ctx, CM_EOVERFLOW, "segment too large");
+                bt.max_tiles_per_seg = std::max(bt.max_tiles_per_seg, (uint32_t)tiles);
+                const uint32_t slot = (uint32_t)((S - 1) * ctx->mm_stride_m + g.m);
+                if (g.m >= 1 && !mm_done[slot]) {
+                    mm_done[slot] = 1;
+                    bt.keys.push_back(((uint32_t)S << 16) | g.m);
+                }
+                bt.tseg.push_back(g);
+            }
+            off += S;
+        }
+        bt.strat.push_back(st);
+    }
+    tp.n_strat = (uint32_t)bt.strat.size() - tp.strat_first;
+    tp.n_tseg = (uint32_t)bt.tseg.size() - tp.tseg_first;
+    tp.n_split_total = split_first;
+    tp.n_cand = cand;
+    tp.n_red = split_first ? (uint32_t)std::min<uint64_t>((split_first + 1023) / 1024, 64) : 0;
+    *out = (uint32_t)bt.tmpl.size();
+    bt.tmpl.push_back(tp);
+    return CM_OK;
+}
+
+// Build the descriptor tables of a batch on the host: integers only, no cost arithmetic.
 cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const int32_t *offsets, int B,
                       const cm_enum_opts &o, uint32_t policy_mask) {
     const DevProfile &hp = ctx->hp;
-    const int N = hp.n_dp * hp.n_pp, L = hp.L, G = hp.G;
-    bt.scen.clear(); bt.strat.clear(); bt.seg.clear(); bt.failed.clear(); bt.red_scen.clear(); bt.keys.clear();
+    const int N = hp.n_dp * hp.n_pp;
+    bt.scen.clear(); bt.tmpl.clear(); bt.strat.clear(); bt.tseg.clear(); bt.failed.clear(); bt.red_scen.clear();
+    bt.keys.clear(); bt.tmpl_scen.clear(); bt.cross.clear();
     bt.opts = o;
     bt.policy_mask = policy_mask;
-    bt.n_cand = bt.n_tiles = bt.n_split = 0;
+    bt.n_cand = bt.n_tiles = bt.n_split = bt.n_rows = 0;
     bt.max_tiles_per_seg = 0;
     bt.dp_max = 0;
     bt.B = B;
     bt.uploaded = false;
-    const int mode = o.cost;
-    std::vector<uint8_t> &mm_done = ctx->mm_done[mode];
+    bt.tmpl_of_nsurv.assign((size_t)N + 1, -1);
+    bt.tmpl.push_back(Tmpl{});   // template 0: no strategies (scenarios without a dynamic-parallelism search)
+    const int cross_words = (N + 63) / 64 + 1;
     std::vector<char> dead(N);
-    std::vector<int> surv;
-    std::vector<std::vector<uint16_t>> strategies;
-    const int dp_lo = std::max(1, (int)o.dp_lo), dp_hi = std::min((int)o.dp_hi, CM_MAX_PIPES);
-    const int pp_lo = std::max(1, (int)o.pp_lo), pp_hi = std::min(std::min((int)o.pp_hi, L), CM_MAX_STAGES);
-    uint32_t red_blocks = 0;
+    bt.scen.reserve(B);
+    bt.cross.reserve((size_t)B * cross_words);
 
     for (int b = 0; b < B; ++b) {
         const int f0 = offsets[b], f1 = offsets[b + 1];
         if (f1 < f0) return fail(ctx, CM_EINVAL, "offsets must be non-decreasing");
-        std::fill(dead.begin(), dead.end(), 0);
         Scen sc{};
         sc.failed_first = (uint32_t)bt.failed.size();
         sc.n_failed = (uint32_t)(f1 - f0);
+        sc.policy_mask = policy_mask;
+        bool bad = false;
         for (int f = f0; f < f1; ++f) {
             const uint32_t d = failed_ids[f];
-            if (d >= (uint32_t)N) return fail(ctx, CM_EINVAL, "failed device id out of range");
-            if (dead[d]) return fail(ctx, CM_EINVAL, "failed device ids must be distinct");
+            if (d >= (uint32_t)N || dead[d]) { bad = true; break; }
             dead[d] = 1;
-            if (!bt.failed.push(d)) return fail(ctx, CM_ENOMEM, "host memory");
+            bt.failed.push_back(d);
         }
-        sc.policy_mask = policy_mask;
-        sc.strat_first = (uint32_t)bt.strat.size();
-        sc.seg_first = (uint32_t)bt.seg.size();
-        sc.red_first = red_blocks;
+        if (bad) {
+            const bool range = std::any_of(failed_ids + f0, failed_ids + f1, [&](uint32_t d) { return d >= (uint32_t)N; });
+            for (int f = f0; f < f1; ++f) if (failed_ids[f] < (uint32_t)N) dead[failed_ids[f]] = 0;
+            return fail(ctx, CM_EINVAL, range ? "failed device id out of range" : "failed device ids must be distinct");
+        }
+        // survivors ascending; bit j: survivors j and j+1 sit on different nodes
+        sc.cross_first = (uint32_t)bt.cross.size();
+        bt.cross.resize(bt.cross.size() + cross_words, 0);
+        uint64_t *cw = bt.cross.data() + sc.cross_first;
+        int n_surv = 0, prev_node = -1;
+        for (int d = 0; d < N; ++d) {
+            if (dead[d]) continue;
+            const int node = d / hp.devices_per_node;
+            if (n_surv > 0 && node != prev_node) cw[(n_surv - 1) >> 6] |= 1ull << ((n_surv - 1) & 63);
+            prev_node = node;
+            ++n_surv;
+        }
+        for (int f = f0; f < f1; ++f) dead[failed_ids[f]] = 0;
         if (policy_mask & (1u << CM_DYNPAR)) {
-            surv.clear();
-            for (int d = 0; d < N; ++d)
-                if (!dead[d]) surv.push_back(d);
-            const int n_surv = (int)surv.size();
-            strategies.clear();
-            if (n_surv > 0 && pp_lo <= pp_hi) enum_strategies(n_surv, dp_lo, dp_hi, pp_lo, pp_hi, strategies);
-            uint64_t split_first = 0;
-            for (const auto &tuple : strategies) {
-                Strat st{};
-                const int dp = (int)tuple.size();
-                st.dp = (uint16_t)dp;
-                st.seg_first = (uint32_t)bt.seg.size();
-                st.split_first = split_first;
-                bt.dp_max = std::max<uint32_t>(bt.dp_max, (uint32_t)dp);
-                int sum = 0;
-                for (int p = 0; p < dp; ++p) {
-                    st.S[p] = tuple[p];
-                    if (o.bm == CM_BATCH_REMAINDER) {
-                        st.m_lo[p] = (uint16_t)(((int64_t)G * tuple[p]) / n_surv);
-                        sum += st.m_lo[p];
-                    } else {
-                        st.m_lo[p] = 1;
-                    }
-                }
-                if (o.bm == CM_BATCH_REMAINDER) {
-                    st.R = (uint16_t)(G - sum);
-                    st.n_m = st.R > 0 ? 2 : 1;
-                    st.n_split = hbinom(ctx, dp, st.R);
-                } else {
-                    st.R = 0;
-                    st.n_m = (uint16_t)(G >= dp ? G - dp + 1 : 0);
-                    st.n_split = G >= dp ? hbinom(ctx, G - 1, dp - 1) : 0;
-                }
-                if (st.n_split == kSat) return fail(ctx, CM_EOVERFLOW, "micro-batch split count overflows 64 bits");
-                split_first = sat_add(split_first, st.n_split);
-                if (split_first >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "too many micro-batch splits");
-                int off = 0;
-                for (int p = 0; p < dp; ++p) {
-                    const int S = tuple[p];
-                    uint64_t tier = 0;
-                    for (int i = 0; i + 1 < S; ++i)
-                        if (surv[off + i] / hp.devices_per_node != surv[off + i + 1] / hp.devices_per_node)
-                            tier |= 1ull << i;
-                    uint64_t K = 0;
-                    if (o.lm == CM_LAYERS_REMAINDER) K = hbinom(ctx, S, L % S);
-                    else if (o.lm == CM_LAYERS_FULL) K = hbinom(ctx, L - 1, S - 1);
-                    if (o.lm == CM_LAYERS_MINMAX || K > o.kappa_cap) K = 0;
-                    if (K >= (1ull << 62)) return fail(ctx, CM_EOVERFLOW, "layer composition count overflows");
-                    for (int mi = 0; mi < st.n_m; ++mi) {
-                        Seg g{};
-                        g.S = (uint16_t)S;
-                        g.m = (uint16_t)(st.m_lo[p] + mi);
-                        g.n_sync = (uint16_t)dp;
-                        g.pipe = (uint16_t)p;
-                        g.K = K;
-                        g.tier_mask = tier;
-                        g.strat = (uint32_t)bt.strat.size();
-                        g.scen = (uint32_t)b;
-                        g.row = (uint32_t)bt.seg.size();
-                        g.cand_first = bt.n_cand;
-                        g.tile_first = bt.n_tiles;
-                        g.mm_slot = (uint32_t)((S - 1) * ctx->mm_stride_m + g.m);
-                        const uint64_t count = K ? K + 1 : 1;
-                        const uint64_t tiles = (count + kTile - 1) / kTile;
-                        bt.n_cand = sat_add(bt.n_cand, count);
-                        bt.n_tiles += tiles;
-                        if (bt.n_cand >= (1ull << 62) || bt.n_tiles >= (1ull << 44))
-                            return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
-                        bt.max_tiles_per_seg = (uint32_t)std::max<uint64_t>(bt.max_tiles_per_seg, std::min<uint64_t>(tiles, 0x7fffffffu));
-                        if (tiles > 0x7fffffffu) return fail(ctx, CM_EOVERFLOW, "segment too large");
-                        if (g.m >= 1 && !mm_done[g.mm_slot]) {
-                            mm_done[g.mm_slot] = 1;
-                            if (!bt.keys.push(((uint32_t)S << 16) | g.m)) return fail(ctx, CM_ENOMEM, "host memory");
-                        }
-                        if (!bt.seg.push(g)) return fail(ctx, CM_ENOMEM, "host memory");
-                    }
-                    off += S;
-                }
-                if (!bt.strat.push(st)) return fail(ctx, CM_ENOMEM, "host memory");
+            int t = bt.tmpl_of_nsurv[n_surv];
+            if (t < 0) {
+                uint32_t nt = 0;
+                cm_status s = build_template(ctx, bt, n_surv, &nt);
+                if (s != CM_OK) return s;
+                t = (int)nt;
+                bt.tmpl_of_nsurv[n_surv] = t;
             }
-            sc.n_split_total = split_first;
-            bt.n_split += split_first;
+            sc.tmpl = (uint32_t)t;
         }
-        sc.n_strat = (uint32_t)bt.strat.size() - sc.strat_first;
-        sc.n_seg = (uint32_t)bt.seg.size() - sc.seg_first;
-        sc.n_red = sc.n_split_total ? (uint32_t)std::min<uint64_t>((sc.n_split_total + 1023) / 1024, 64) : 0;
-        for (uint32_t r = 0; r < sc.n_red; ++r)
-            if (!bt.red_scen.push((uint32_t)b)) return fail(ctx, CM_ENOMEM, "host memory");
-        red_blocks += sc.n_red;
-        if (!bt.scen.push(sc)) return fail(ctx, CM_ENOMEM, "host memory");
+        bt.tmpl[sc.tmpl].n_scen++;
+        bt.scen.push_back(sc);
     }
+    // scenarios grouped by template; result rows and reduction blocks per scenario
+    uint32_t first = 0;
+    for (Tmpl &tp : bt.tmpl) { tp.scen_first = first; first += tp.n_scen; tp.n_scen = 0; }
+    bt.tmpl_scen.resize(B);
+    uint64_t rows = 0, red = 0;
+    for (int b = 0; b < B; ++b) {
+        Scen &sc = bt.scen[b];
+        Tmpl &tp = bt.tmpl[sc.tmpl];
+        bt.tmpl_scen[tp.scen_first + tp.n_scen++] = (uint32_t)b;
+        sc.seg_base = (uint32_t)rows;
+        sc.red_first = (uint32_t)red;
+        rows += tp.n_tseg;
+        red += tp.n_red;
+        for (uint32_t r = 0; r < tp.n_red; ++r) bt.red_scen.push_back((uint32_t)b);
+        bt.n_cand = sat_add(bt.n_cand, tp.n_cand);
+        bt.n_split = sat_add(bt.n_split, tp.n_split_total);
+        if (rows >= (1ull << 31) || red >= (1ull << 31) || bt.n_cand >= (1ull << 62))
+            return fail(ctx, CM_EOVERFLOW, "batch too large for the index type");
+    }
+    bt.n_rows = rows;
+    bt.n_tiles = bt.max_tiles_per_seg ? 1 : 0;   // only "is there anything to tie-break" matters
     return build_buckets(ctx, bt);
 }
 
+// Pack the host tables into the pinned arena (16-byte aligned sections).
 template <typename T>
-cm_status upload(cm_ctx *ctx, DevBuf<T> &d, const PinnedVec<T> &h) {
-    if (!d.reserve(std::max<size_t>(h.size(), 1))) return fail(ctx, CM_ENOMEM, "device memory");
-    if (h.size()) CM_CUDA(ctx, cudaMemcpyAsync(d.p, h.p, h.size() * sizeof(T), cudaMemcpyHostToDevice, ctx->stream));
-    ctx->stats[9] += h.size() * sizeof(T);
-    return CM_OK;
+size_t arena_put(PinnedVec<unsigned char> &arena, const std::vector<T> &v, bool &ok) {
+    const size_t off = (arena.size() + 15) & ~(size_t)15;
+    const size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(T);
+    if (!arena.resize(off + bytes)) { ok = false; return off; }
+    if (!v.empty()) memcpy(arena.p + off, v.data(), v.size() * sizeof(T));
+    return off;
 }
 
 BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     BatchDev v{};
-    v.scen = bt.d_scen.p; v.strat = bt.d_strat.p; v.seg = bt.d_seg.p; v.failed = bt.d_failed.p;
-    v.bucket = bt.d_bucket.p; v.order = bt.d_order.p;
-    v.seg_best = bt.d_seg_best.p; v.red_scen = bt.d_red_scen.p; v.partial = bt.d_partial.p;
+    const unsigned char *a = bt.d_arena.p;
+    v.scen = (const Scen *)(a + bt.off_scen); v.tmpl = (const Tmpl *)(a + bt.off_tmpl);
+    v.strat = (const Strat *)(a + bt.off_strat); v.tseg = (const TSeg *)(a + bt.off_tseg);
+    v.failed = (const uint32_t *)(a + bt.off_failed); v.cross = (const uint64_t *)(a + bt.off_cross);
+    v.tmpl_scen = (const uint32_t *)(a + bt.off_tmpl_scen); v.bucket = (const Bucket *)(a + bt.off_bucket);
+    v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
+    v.seg_best = bt.d_seg_best.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p; v.counters = bt.d_counters.p;
     v.B = bt.B; v.mode = bt.opts.cost;
-    v.n_seg = (uint32_t)bt.seg.size(); v.n_strat = (uint32_t)bt.strat.size();
+    v.n_rows = (uint32_t)bt.n_rows; v.n_strat = (uint32_t)bt.strat.size();
     v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
     v.n_red_blocks = (uint32_t)bt.red_scen.size(); v.dp_max = bt.dp_max;
     v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
@@ -411,25 +479,34 @@ Tables tables(const cm_ctx *ctx, int mode) {
     return t;
 }
 
-// Copy the tables of a batch to the device and run the min-max partitions it needs.
+// Copy the tables of a batch to the device (one copy) and run the min-max partitions it needs.
 cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
-    cm_status s;
-    if ((s = upload(ctx, bt.d_scen, bt.scen)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_strat, bt.strat)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_seg, bt.seg)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_failed, bt.failed)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_red_scen, bt.red_scen)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_keys, bt.keys)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_order, bt.order)) != CM_OK) return s;
-    if ((s = upload(ctx, bt.d_bucket, bt.bucket)) != CM_OK) return s;
+    bool ok = true;
+    bt.arena.clear();
+    bt.off_scen = arena_put(bt.arena, bt.scen, ok);
+    bt.off_tmpl = arena_put(bt.arena, bt.tmpl, ok);
+    bt.off_strat = arena_put(bt.arena, bt.strat, ok);
+    bt.off_tseg = arena_put(bt.arena, bt.tseg, ok);
+    bt.off_failed = arena_put(bt.arena, bt.failed, ok);
+    bt.off_red = arena_put(bt.arena, bt.red_scen, ok);
+    bt.off_keys = arena_put(bt.arena, bt.keys, ok);
+    bt.off_tmpl_scen = arena_put(bt.arena, bt.tmpl_scen, ok);
+    bt.off_bucket_tseg = arena_put(bt.arena, bt.bucket_tseg, ok);
+    bt.off_cross = arena_put(bt.arena, bt.cross, ok);
+    bt.off_bucket = arena_put(bt.arena, bt.bucket, ok);
+    if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
+    if (!bt.d_arena.reserve(bt.arena.size())) return fail(ctx, CM_ENOMEM, "device memory");
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.d_arena.p, bt.arena.p, bt.arena.size(), cudaMemcpyHostToDevice, ctx->stream));
+    ctx->stats[9] += bt.arena.size();
     const size_t B = std::max(bt.B, 1);
-    bool ok = bt.d_seg_best.reserve(std::max<size_t>(bt.seg.size(), 1)) &&
-              bt.d_partial.reserve(std::max<size_t>(bt.red_scen.size(), 1)) && bt.d_winner.reserve(B) &&
-              bt.d_kappa_sel.reserve(B * kMaxP) && bt.d_pol_cost.reserve(B * 2) &&
-              bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4) && bt.d_counters.reserve(4);
+    ok = bt.d_seg_best.reserve(std::max<size_t>(bt.n_rows, 1)) &&
+         bt.d_partial.reserve(std::max<size_t>(bt.red_scen.size(), 1)) && bt.d_winner.reserve(B) &&
+         bt.d_kappa_sel.reserve(B * kMaxP) && bt.d_pol_cost.reserve(B * 2) &&
+         bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4) && bt.d_counters.reserve(4);
     if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
     if (bt.keys.size()) {
-        CM_CUDA(ctx, launch_minmax(tables(ctx, bt.opts.cost), bt.d_keys.p, (int)bt.keys.size(), bt.opts.cost, ctx->stream));
+        CM_CUDA(ctx, launch_minmax(tables(ctx, bt.opts.cost), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
+                                   (int)bt.keys.size(), bt.opts.cost, ctx->stream));
         if (launches) ++*launches;
     }
     bt.uploaded = true;
@@ -444,7 +521,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     cudaStream_t st = ctx->stream;
     int launches = launches_so_far, cost_launches = 0;
     CM_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
-    if (bt.seg.size()) CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, bt.seg.size() * sizeof(uint64_t), st));
+    if (bt.n_rows) CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, bt.n_rows * sizeof(uint64_t), st));
     CM_CUDA(ctx, cudaMemsetAsync(bt.d_counters.p, 0, 4 * sizeof(unsigned long long), st));
     if (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) {
         CM_CUDA(ctx, launch_policies(tb, bd, ctx->hp.n_dp, st));
@@ -484,7 +561,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     ctx->stats[2] += bt.counters_host[1];
     ctx->stats[3] += (uint64_t)launches;
     ctx->stats[4] += (uint64_t)((double)ms * 1e6);
-    ctx->stats[5] += bt.seg.size();
+    ctx->stats[5] += bt.n_rows;
     ctx->stats[6] += bt.strat.size();
     ctx->stats[7] += bt.n_split;
     return CM_OK;
@@ -674,7 +751,6 @@ cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids
         delete sp;
         return s;
     }
-    for (size_t i = 0; i < sp->batch.strat.size(); ++i) sp->strat_dp.push_back(sp->batch.strat[i].dp);
     *out = sp;
     if (n_candidates) *n_candidates = policy == CM_DYNPAR ? sp->batch.n_cand : 1;
     return CM_OK;
@@ -869,14 +945,15 @@ cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan
         }
     } else {
         const Batch &bt = space->batch;
-        if (plan->strategy >= bt.strat.size()) return fail(ctx, CM_EINVAL, "strategy index out of range");
-        const Strat &st = bt.strat[plan->strategy];
+        const Tmpl &tp = bt.tmpl[bt.scen[0].tmpl];
+        if (plan->strategy >= tp.n_strat) return fail(ctx, CM_EINVAL, "strategy index out of range");
+        const Strat &st = bt.strat[tp.strat_first + plan->strategy];
         if (plan->n_pipes != st.dp) return fail(ctx, CM_EINVAL, "plan does not match its strategy");
         for (int p = 0; p < st.dp; ++p) {
             const int S = st.S[p], L = hp.L;
             const int off = (int)plan->micro[p] - (int)st.m_lo[p];
             if (plan->stages[p] != S || off < 0 || off >= st.n_m) return fail(ctx, CM_EINVAL, "plan does not match its strategy");
-            const Seg &g = bt.seg[st.seg_first + p * st.n_m + off];
+            const TSeg &g = bt.tseg[st.seg_first + p * st.n_m + off];
             const uint64_t kappa = plan->kappa[p];
             if (kappa > g.K) return fail(ctx, CM_EINVAL, "layer composition rank out of range");
             if (kappa < g.K) {
@@ -906,7 +983,7 @@ cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan
                 }
             } else {
                 uint8_t row[kMaxS + 1];
-                CM_CUDA(ctx, cudaMemcpyAsync(row, ctx->d_mm[bt.opts.cost] + (size_t)g.mm_slot * (kMaxS + 1), kMaxS + 1,
+                CM_CUDA(ctx, cudaMemcpyAsync(row, ctx->d_mm[bt.opts.cost] + ((size_t)(S - 1) * ctx->mm_stride_m + g.m) * (kMaxS + 1), kMaxS + 1,
                                              cudaMemcpyDeviceToHost, ctx->stream));
                 CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
                 if (row[0] != 0) return fail(ctx, CM_EINVAL, "min-max partition of this pipeline is infeasible");

@@ -52,6 +52,14 @@ __device__ __forceinline__ void plan_of_thread(uint64_t base, uint64_t count, ui
     }
 }
 
+// Segment number `seg_local` of a bucket = (template segment of the bucket, scenario of the
+// template), scenario minor.
+__device__ __forceinline__ SegView bucket_segment(const BatchDev &bd, const Bucket &bk, uint32_t seg_local) {
+    const Tmpl &tp = bd.tmpl[bk.tmpl];
+    const uint32_t ti = seg_local / tp.n_scen, si = seg_local - ti * tp.n_scen;
+    return seg_view(bd, bd.tmpl_scen[tp.scen_first + si], bd.bucket_tseg[bk.list_first + ti]);
+}
+
 // Least cost per segment from per-lane (segment row, cost bits): lanes of one segment
 // are contiguous, so a segmented shuffle scan leaves each run's minimum in its last lane,
 // which issues the one atomicMin.
@@ -305,12 +313,12 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
     if (seg_local < bk.n_seg && m >= 1) {
-        row = bd.order[bk.seg_begin + seg_local];
-        const Seg *g = bd.seg + row;
-        const uint64_t tier = g->tier_mask, K = g->K;
-        const int n_sync = g->n_sync;
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        const uint64_t tier = g.tier, K = g.K;
+        const int n_sync = g.n_sync;
         CutWalker cw;
-        bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, K, g->mm_slot);
+        bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, K, tb.mm_slot(S, m));
         FB<T> st[S];
         T xts[S];
         long long g_max = 0;
@@ -373,13 +381,13 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
         const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
         if (kappa < bk.count && m >= 1) {           // warp-uniform
             const bool active = seg_local < bk.n_seg;
-            const uint32_t row = bd.order[bk.seg_begin + (active ? seg_local : 0)];
-            const Seg *g = bd.seg + row;
-            const uint64_t tier = g->tier_mask;
-            const int n_sync = g->n_sync;
+            const SegView g = bucket_segment(bd, bk, active ? seg_local : 0);
+            const uint32_t row = g.row;
+            const uint64_t tier = g.tier;
+            const int n_sync = g.n_sync;
             // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
             CutWalker cw;
-            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g->K, g->mm_slot);
+            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
             if (ok) {
                 int lo = 0;
                 for (int i = 0; i < S; ++i) {
@@ -431,11 +439,11 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
         uint32_t row = 0xffffffffu;
         uint64_t bits = inf_bits<T>();
         if (seg_local < bk.n_seg && m >= 1) {
-            row = bd.order[bk.seg_begin + seg_local];
-            const Seg *g = bd.seg + row;
-            const uint64_t tier = g->tier_mask;
+            const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+            row = g.row;
+            const uint64_t tier = g.tier;
             CutWalker cw;
-            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g->K, g->mm_slot);
+            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
             long long g_max = 0;
             int lo = 0;
             for (int i = 0; i < S && ok; ++i) {
@@ -452,7 +460,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
             }
             if (ok) {
                 const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-                bits = Num<T>::bits(t + Num<T>::sync(g_max, g->n_sync, sp.bw_sync));
+                bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync));
                 my_cells = 2ull * S * m;
             }
         }
@@ -476,8 +484,8 @@ __global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, Batc
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
     if (seg_local < bk.n_seg) {
-        row = bd.order[bk.seg_begin + seg_local];
-        const Seg g = bd.seg[row];
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
         T cost;
         if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
             bits = Num<T>::bits(cost);

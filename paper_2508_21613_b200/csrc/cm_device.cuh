@@ -220,9 +220,40 @@ __device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, i
     return true;
 }
 
+// ----------------------------------------------------------------------------------
+// A segment of one scenario, resolved from the template tables: the template gives the
+// shape (stages, micro-batches, peers, compositions), the scenario gives the link tiers
+// -- n bits cut out of its node-crossing bit string at the pipeline's survivor offset.
+// ----------------------------------------------------------------------------------
+struct SegView {
+    uint64_t tier, K;
+    uint32_t row;          // row of seg_best
+    int S, m, n_sync;
+};
+
+__device__ __forceinline__ uint64_t cut_bits(const uint64_t *words, int off, int n /* <= 63 */) {
+    const int w = off >> 6, sh = off & 63;
+    uint64_t v = words[w] >> sh;
+    if (sh) v |= words[w + 1] << (64 - sh);
+    return v & ((1ull << n) - 1ull);
+}
+
+__device__ __forceinline__ SegView seg_view(const BatchDev &bd, uint32_t scen_id, uint32_t tseg_row) {
+    const Scen &sc = bd.scen[scen_id];
+    const TSeg g = bd.tseg[tseg_row];
+    SegView v;
+    v.S = g.S;
+    v.m = g.m;
+    v.n_sync = g.n_sync;
+    v.K = g.K;
+    v.row = sc.seg_base + (tseg_row - bd.tmpl[sc.tmpl].tseg_first);
+    v.tier = cut_bits(bd.cross + sc.cross_first, g.off, g.S - 1);
+    return v;
+}
+
 // Candidate kappa of a segment: an enumerated composition or the min-max partition.
 template <typename T>
-__device__ __forceinline__ bool segment_candidate_cost(const SProf<T> &sp, const Tables &tb, const Seg &g,
+__device__ __forceinline__ bool segment_candidate_cost(const SProf<T> &sp, const Tables &tb, const SegView &g,
                                                        int layer_mode, uint64_t kappa, T &cost) {
     uint8_t cuts[kMaxS + 1];
     const int S = g.S;
@@ -230,11 +261,11 @@ __device__ __forceinline__ bool segment_candidate_cost(const SProf<T> &sp, const
     if (kappa < g.K) {
         layer_cuts(tb.binom, layer_mode, sp.L, S, kappa, cuts);
     } else {
-        const uint8_t *mm = tb.mm_cuts + (size_t)g.mm_slot * (kMaxS + 1);
+        const uint8_t *mm = tb.mm_cuts + (size_t)tb.mm_slot(S, g.m) * (kMaxS + 1);
         if (mm[0] != 0) return false;  // no memory-feasible partition exists
         for (int i = 0; i <= S; ++i) cuts[i] = mm[i];
     }
-    return pipe_cost_from_cuts<T>(sp, S, g.m, cuts, g.tier_mask, g.n_sync, cost);
+    return pipe_cost_from_cuts<T>(sp, S, g.m, cuts, g.tier, g.n_sync, cost);
 }
 
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {

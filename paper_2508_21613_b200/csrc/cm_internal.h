@@ -33,37 +33,47 @@ struct DevProfile {
     int64_t fwd_i[kMaxL], bwd_i[kMaxL], act[kMaxL], par[kMaxL], opt[kMaxL], p2p[kMaxL];
 };
 
-// One (strategy, pipeline, micro-batch count): its candidates are the layer compositions
-// kappa = 0..K-1 followed by the min-max partition, or the min-max partition alone (K = 0).
-struct Seg {
-    uint64_t cand_first;   // index of its first candidate within the space
-    uint64_t tile_first;   // index of its first tile in the cost kernel's grid
-    uint64_t tier_mask;    // bit i set: the boundary between stages i and i+1 crosses nodes
+// The descriptor tables are TEMPLATES keyed by the survivor count: which strategies exist,
+// how micro-batches split and how many layer compositions a pipeline has depend only on
+// how many devices survive, not on which.  A failure scenario adds just its failed ids
+// and one bit per pair of neighbouring survivors ("do they sit on different nodes?"),
+// from which a pipeline's link tiers are cut out on the device.
+//
+// One template segment = (strategy, pipeline, micro-batch count): its candidates are the
+// layer compositions kappa = 0..K-1 followed by the min-max partition, or the min-max
+// partition alone (K = 0).
+struct TSeg {              // 24 bytes
+    uint64_t cand_first;   // index of its first candidate within one scenario's space
     uint64_t K;            // enumerated compositions
-    uint32_t mm_slot;      // row of the min-max cuts table
-    uint32_t strat;        // global strategy row
-    uint16_t S, m, n_sync, pipe;
-    uint32_t scen;         // scenario of the batch
-    uint32_t row;          // its own row in the segment table
+    uint16_t S, m, n_sync; // stages, micro-batches, data-parallel peers of the strategy
+    uint16_t off;          // survivor index of the pipeline's first stage
 };
 
-// One parallel strategy of one scenario.
+// One parallel strategy of a template.
 struct Strat {
-    uint64_t split_first;  // first split item of this strategy within its scenario
+    uint64_t split_first;  // first split item of this strategy within its template
     uint64_t n_split;      // micro-batch splits
-    uint32_t seg_first;    // its first segment (global row)
+    uint32_t seg_first;    // its first template segment (global row of the TSeg table)
     uint16_t dp, n_m;      // pipelines; micro-batch values per pipeline (segments per pipeline)
     uint16_t R, pad;       // REMAINDER mode: pipelines that receive one more
     uint16_t S[kMaxP], m_lo[kMaxP];
 };
 
-// One failure scenario of a batch.
-struct Scen {
+struct Tmpl {
     uint64_t n_split_total;  // split items over all its strategies
+    uint64_t n_cand;         // candidates of one scenario
     uint32_t strat_first, n_strat;
-    uint32_t seg_first, n_seg;
+    uint32_t tseg_first, n_tseg;
+    uint32_t scen_first, n_scen;   // its scenarios, as a range of the tmpl_scen list
+    uint32_t n_red, pad;           // blocks of the split reduction per scenario
+};
+
+// One failure scenario of a batch.  Its segments own rows seg_base .. seg_base+n_tseg-1 of
+// the per-segment result array, in template order.
+struct Scen {              // 32 bytes
+    uint32_t tmpl, seg_base;
     uint32_t failed_first, n_failed;   // into the failed-id array
-    uint32_t red_first, n_red;         // blocks of the split reduction that belong to it
+    uint32_t cross_first, red_first;   // into the node-crossing bit words; first reduction block
     uint32_t policy_mask, pad;
 };
 
@@ -76,8 +86,9 @@ constexpr int kRegStagesMax = 16;   // deepest pipeline the register-resident ke
 struct Bucket {
     uint64_t count;        // candidates per segment (K+1 or 1)
     uint64_t chunk_first;  // first chunk of the bucket within its launch class
-    uint32_t seg_begin;    // first entry of the bucket in the sorted segment order
-    uint32_t n_seg;
+    uint32_t list_first;   // its template segments, as a range of the bucket_tseg list
+    uint32_t n_tseg;
+    uint32_t tmpl, n_seg;  // n_seg = n_tseg * scenarios of the template
     uint16_t S, m;
     uint32_t pad;
 };
@@ -111,11 +122,14 @@ struct Winner {
 
 struct BatchDev {
     const Scen *scen;
+    const Tmpl *tmpl;
     const Strat *strat;
-    const Seg *seg;
+    const TSeg *tseg;
     const uint32_t *failed;
-    const Bucket *bucket;   // search-pass work layout
-    const uint32_t *order;  // segment rows sorted by bucket
+    const uint64_t *cross;        // per scenario: bit j = survivors j and j+1 sit on different nodes
+    const uint32_t *tmpl_scen;    // scenario ids grouped by template
+    const Bucket *bucket;         // search-pass work layout
+    const uint32_t *bucket_tseg;  // template segment rows grouped by bucket
     uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
     const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
     Partial *partial;       // [n_red_blocks]
@@ -126,7 +140,7 @@ struct BatchDev {
     cm_plan *plans;         // [B][4]: per policy, then the overall best
     unsigned long long *counters;  // [0] cells simulated in pass 1, [1] plans in pass 2
     int32_t B, mode;
-    uint32_t n_seg, n_strat;
+    uint32_t n_rows, n_strat;    // rows of seg_best over all scenarios
     uint64_t n_tiles;
     uint32_t max_tiles_per_seg, n_red_blocks;
     uint32_t dp_max, pad;
@@ -139,6 +153,7 @@ struct Tables {
     int32_t binom_rows;
     uint8_t *mm_cuts;           // [slots][kMaxS+1], min-max partitions; mm_cuts[slot][0]=255: infeasible
     int32_t mm_stride_m;        // slot = (S-1)*mm_stride_m + m
+    __host__ __device__ uint32_t mm_slot(int S, int m) const { return (uint32_t)((S - 1) * mm_stride_m + m); }
 };
 
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error

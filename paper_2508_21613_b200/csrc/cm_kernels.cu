@@ -133,12 +133,11 @@ cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys,
 // Locate the segment that owns a tile / a candidate: the last row whose first index is
 // not above the query (rows are sorted and every segment owns at least one).
 // ----------------------------------------------------------------------------------
-template <typename Key>
-__device__ __forceinline__ uint32_t find_row(const Seg *seg, uint32_t n, uint64_t q, Key key) {
+__device__ __forceinline__ uint32_t find_row(const TSeg *seg, uint32_t n, uint64_t q) {
     uint32_t lo = 0, hi = n - 1;
     while (lo < hi) {
         uint32_t mid = (lo + hi + 1) >> 1;
-        if (key(seg[mid]) <= q) lo = mid; else hi = mid - 1;
+        if (seg[mid].cand_first <= q) lo = mid; else hi = mid - 1;
     }
     return lo;
 }
@@ -176,25 +175,27 @@ __global__ void __launch_bounds__(256) cm_split_kernel(Tables tb, BatchDev bd, u
     __shared__ uint64_t rc[8], ri[8];
     const uint32_t b = bd.red_scen[blockIdx.x];
     const Scen sc = bd.scen[b];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
     const uint32_t local = blockIdx.x - sc.red_first;
     const int G = tb.prof->G;
+    const uint64_t *best = bd.seg_best + sc.seg_base;   // this scenario's rows, in template order
     uint64_t best_c = inf, best_i = ~0ull;
-    for (uint64_t item = (uint64_t)local * blockDim.x + threadIdx.x; item < sc.n_split_total;
-         item += (uint64_t)sc.n_red * blockDim.x) {
+    for (uint64_t item = (uint64_t)local * blockDim.x + threadIdx.x; item < tp.n_split_total;
+         item += (uint64_t)tp.n_red * blockDim.x) {
         // strategy that owns the item
-        uint32_t lo = 0, hi = sc.n_strat - 1;
+        uint32_t lo = 0, hi = tp.n_strat - 1;
         while (lo < hi) {
             uint32_t mid = (lo + hi + 1) >> 1;
-            if (bd.strat[sc.strat_first + mid].split_first <= item) lo = mid; else hi = mid - 1;
+            if (bd.strat[tp.strat_first + mid].split_first <= item) lo = mid; else hi = mid - 1;
         }
-        const Strat &s = bd.strat[sc.strat_first + lo];
+        const Strat &s = bd.strat[tp.strat_first + lo];
         uint16_t micro[kMaxP];
         split_micro(tb.binom, bd.batch_mode, G, s, item - s.split_first, micro);
         uint64_t T = 0;
         for (int p = 0; p < s.dp; ++p) {
             uint64_t c = inf;
             const int off = (int)micro[p] - (int)s.m_lo[p];
-            if (micro[p] >= 1 && off >= 0 && off < s.n_m) c = bd.seg_best[s.seg_first + p * s.n_m + off];
+            if (micro[p] >= 1 && off >= 0 && off < s.n_m) c = best[s.seg_first - tp.tseg_first + p * s.n_m + off];
             c = c > inf ? inf : c;   // a segment nobody improved still holds its all-ones initial value
             T = c > T ? c : T;
         }
@@ -220,8 +221,9 @@ __global__ void __launch_bounds__(256) cm_split_kernel(Tables tb, BatchDev bd, u
 __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, uint64_t inf) {
     const uint32_t b = blockIdx.x;
     const Scen sc = bd.scen[b];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
     uint64_t best_c = inf, best_i = ~0ull;
-    for (uint32_t r = threadIdx.x; r < sc.n_red; r += 32) {
+    for (uint32_t r = threadIdx.x; r < tp.n_red; r += 32) {
         const Partial q = bd.partial[sc.red_first + r];
         if (pair_less(q.cost_bits, q.item, best_c, best_i)) { best_c = q.cost_bits; best_i = q.item; }
     }
@@ -239,15 +241,16 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
         w.dp = 0;
         for (int p = 0; p < kMaxP; ++p) { w.seg[p] = 0; w.micro[p] = 0; }
         if (best_c < inf) {
-            uint32_t lo = 0, hi = sc.n_strat - 1;
+            uint32_t lo = 0, hi = tp.n_strat - 1;
             while (lo < hi) {
                 uint32_t mid = (lo + hi + 1) >> 1;
-                if (bd.strat[sc.strat_first + mid].split_first <= best_i) lo = mid; else hi = mid - 1;
+                if (bd.strat[tp.strat_first + mid].split_first <= best_i) lo = mid; else hi = mid - 1;
             }
-            const Strat &s = bd.strat[sc.strat_first + lo];
-            w.strat = sc.strat_first + lo;
+            const Strat &s = bd.strat[tp.strat_first + lo];
+            w.strat = tp.strat_first + lo;
             w.dp = s.dp;
             split_micro(tb.binom, bd.batch_mode, tb.prof->G, s, best_i - s.split_first, w.micro);
+            // template segment rows of the winner's pipelines
             for (int p = 0; p < s.dp; ++p) w.seg[p] = s.seg_first + p * s.n_m + (w.micro[p] - s.m_lo[p]);
         }
         bd.winner[b] = w;
@@ -276,7 +279,7 @@ template <typename T>
 __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev bd) {
     __shared__ SProf<T> sp;
     __shared__ uint64_t red[kTile / 32];
-    __shared__ Seg g;
+    __shared__ SegView g;
     __shared__ uint64_t found_so_far;
     stage_profile(sp, tb.prof);
     for (uint32_t y = blockIdx.y; y < (uint32_t)bd.B * bd.dp_max; y += gridDim.y) {
@@ -286,7 +289,7 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
         __syncthreads();
         if (threadIdx.x == 0) {
-            g = bd.seg[w.seg[p]];
+            g = seg_view(bd, b, w.seg[p]);
             found_so_far = *(volatile uint64_t *)slot;
         }
         __syncthreads();
@@ -375,7 +378,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
             const Strat &s = bd.strat[w.strat];
             pl.feasible = 1;
             plan_set_cost(pl, w.cost_bits, bd.mode);
-            pl.strategy = w.strat - sc.strat_first;
+            pl.strategy = w.strat - bd.tmpl[sc.tmpl].strat_first;
             pl.n_pipes = w.dp;
             pl.split_rank = w.item - s.split_first;
             for (uint32_t q = 0; q < w.dp; ++q) {
@@ -417,10 +420,12 @@ __global__ void __launch_bounds__(128) cm_evaluate_kernel(Tables tb, BatchDev bd
     T c = Num<T>::inf();
     bool ok = false;
     if (e < n_cand) {
-        uint32_t s = find_row(bd.seg, bd.n_seg, e, [](const Seg &x) { return x.cand_first; });
-        const Seg g = bd.seg[s];
+        // spaces hold one scenario: its template's segments are sorted by first candidate
+        const Tmpl tp = bd.tmpl[bd.scen[0].tmpl];
+        const uint32_t s = tp.tseg_first + find_row(bd.tseg + tp.tseg_first, tp.n_tseg, e);
+        const SegView g = seg_view(bd, 0, s);
         T v;
-        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, e - g.cand_first, v)) { c = v; ok = true; }
+        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, e - bd.tseg[s].cand_first, v)) { c = v; ok = true; }
     }
     if (cost && bd.mode == CM_COST_FP64) cost[t] = __longlong_as_double((long long)Num<T>::bits(c));
     if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = (int64_t)Num<T>::bits(c);
