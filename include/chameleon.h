@@ -195,6 +195,31 @@ cm_status cm_batch_search(cm_ctx *ctx, cm_batch *batch, cm_plan *best_per_scenar
                           cm_plan *best_per_policy);
 cm_status cm_batch_free(cm_batch *batch);
 
+/* The paper has no counterpart to this call: it exists for callers that must not allocate.
+ * A failure handler may run while the training framework's caching allocator holds all
+ * free device memory, on a path where the device-wide synchronisation of an allocation
+ * is unaffordable, or in a process whose memory budget was fixed at start-up.  Such a
+ * caller builds its candidate space beforehand with cm_enumerate (that does allocate)
+ * and later calls this function, which allocates nothing on host or device.
+ *
+ * Evaluates candidates first .. first+count-1 of a CM_DYNPAR space exactly as cm_evaluate
+ * does and reduces them on the device to the least cost and the lowest candidate index
+ * that attains it, written to the caller's DEVICE buffers: best_cost_dev in fp64 mode,
+ * best_cost_ns_dev in int64 mode (the other is left untouched; any pointer may be NULL),
+ * best_index_dev = UINT64_MAX and cost = +infinity / INT64_MAX if no candidate of the
+ * range is memory-feasible.  Enqueues on the context's stream and returns.
+ *
+ * Limits and rules: count must be 1 .. CM_NOALLOC_MAX_CANDIDATES (larger ranges are
+ * rejected with CM_EINVAL; split them).  The block partials of the reduction live in a
+ * fixed 64 KB array inside the library, one per GPU, shared by every call on that GPU:
+ * two calls that overlap on the device (different streams or contexts) race on it, so
+ * serialise them.  The first call on a device looks up the array's address; make that
+ * call before starting any stream capture. */
+#define CM_NOALLOC_MAX_CANDIDATES 524288
+cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64_t count,
+                                     double *best_cost_dev, int64_t *best_cost_ns_dev,
+                                     uint64_t *best_index_dev);
+
 /* Work counters of the last cm_select / cm_search_batch / cm_batch_search on this
  * context (HOST out[16]):
  *  [0] pipeline-plans evaluated by the search pass   [1] recurrence cells simulated by it

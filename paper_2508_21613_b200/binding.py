@@ -28,8 +28,9 @@ CM_COST_FP64, CM_COST_INT64NS = 0, 1
 
 EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_evaluate", "cm_select",
            "cm_decode_plan", "cm_space_free", "cm_search_batch", "cm_batch_prepare", "cm_batch_search",
-           "cm_batch_free", "cm_last_stats", "cm_strerror", "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:13]
+           "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:14]
+NOALLOC_MAX_CANDIDATES = 524288
 
 
 class ChameleonError(RuntimeError):
@@ -124,6 +125,7 @@ def load_library() -> C.CDLL:
                                      C.POINTER(cm_enum_opts), C.POINTER(vp), u64p]
     lib.cm_batch_search.argtypes = [vp, vp, C.POINTER(cm_plan), C.POINTER(cm_plan)]
     lib.cm_batch_free.argtypes = [vp]
+    lib.cm_evaluate_argmin_noalloc.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp, vp, vp]
     for name in _STATUS_CALLS:
         getattr(lib, name).restype = C.c_int
     _lib = lib
@@ -247,6 +249,16 @@ def cm_search_batch(ctx, scenarios: Sequence[Sequence[int]], opts, per_policy: b
         ctx, ids.ctypes.data_as(C.POINTER(C.c_uint32)), offsets.ctypes.data_as(C.POINTER(C.c_int32)), B,
         C.byref(o), best, pol, lat.ctypes.data_as(C.POINTER(C.c_float)) if latency else None))
     return best, pol, lat
+
+
+def cm_evaluate_argmin_noalloc(ctx, space, first: int, count: int, best_cost_dev=None, best_cost_ns_dev=None,
+                               best_index_dev=None) -> None:
+    """Best (cost, index) of a candidate range, for callers that must not allocate: the
+    three outputs are caller-owned device buffers (torch tensors or raw pointers) and the
+    call itself allocates nothing.  At most NOALLOC_MAX_CANDIDATES candidates per call."""
+    ptr = lambda t: None if t is None else C.c_void_p(t.data_ptr() if hasattr(t, "data_ptr") else int(t))
+    _check(ctx, load_library().cm_evaluate_argmin_noalloc(ctx, space, first, count, ptr(best_cost_dev),
+                                                          ptr(best_cost_ns_dev), ptr(best_index_dev)))
 
 
 def cm_batch_free(batch) -> None:

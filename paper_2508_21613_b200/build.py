@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libchameleon.so")
-SOURCES = ["cm_api.cu", "cm_kernels.cu", "cm_policy.cu", "cm_cost.cu"]
+SOURCES = ["cm_api.cu", "cm_kernels.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu"]
 HEADERS = ["cm_internal.h", "cm_device.cuh"]
 
 NVCC_FLAGS = [

@@ -587,6 +587,21 @@ void scrub(cm_plan &pl) {
 
 }  // namespace
 
+// Accessors for entry points that live in other translation units.
+cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message) { return fail(ctx, status, message); }
+
+cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, SpaceView *out) {
+    if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
+    Batch &bt = const_cast<Batch &>(space->batch);
+    out->tb = tables(ctx, bt.opts.cost);
+    out->bd = dev_view(ctx, bt);
+    out->n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
+    out->stream = ctx->stream;
+    out->device = ctx->device;
+    out->policy = space->policy;
+    return CM_OK;
+}
+
 // ------------------------------------------------------------------------- C ABI
 extern "C" {
 

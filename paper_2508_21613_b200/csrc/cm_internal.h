@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cstdint>
+#include <string>
 #include <cuda_runtime.h>
 
 #include "chameleon.h"
@@ -172,4 +173,18 @@ cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand,
                             int64_t *cost_ns, uint8_t *feas, cudaStream_t st);
 cudaError_t launch_pick(const cm_plan *const *plans_dev, int n, cm_plan *out_dev, int mode, cudaStream_t st);
 
+// What an entry point implemented outside cm_api.cu needs to know about a space.
+struct SpaceView {
+    Tables tb;
+    BatchDev bd;
+    uint64_t n_cand;
+    cudaStream_t stream;
+    int device, policy;
+};
+
 }  // namespace cm
+
+struct cm_ctx;
+struct cm_space;
+cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, cm::SpaceView *out);
+cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message);
