@@ -272,8 +272,8 @@ cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t
 // ----------------------------------------------------------------------------------
 // Pass 2 (tie-break): among optimal plans the lexicographically smallest tuple wins, so
 // each pipeline of the winning (strategy, split) takes the LOWEST layer composition
-// that is feasible with cost <= T* (not its own argmin).  grid.x = tiles of a segment,
-// grid.y = (scenario, pipeline).  Tiles above an already found index return at once.
+// that is feasible with cost <= T* (not its own argmin).  grid.x = (scenario, pipeline),
+// grid.y = tiles of a segment.  Tiles above an already found index return at once.
 // ----------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev bd) {
@@ -282,10 +282,14 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
     __shared__ SegView g;
     __shared__ uint64_t found_so_far;
     stage_profile(sp, tb.prof);
-    for (uint32_t y = blockIdx.y; y < (uint32_t)bd.B * bd.dp_max; y += gridDim.y) {
-        const uint32_t b = y / bd.dp_max, p = y % bd.dp_max;
-        const Winner &w = bd.winner[b];
-        if (w.cost_bits >= inf_bits<T>() || p >= w.dp) continue;   // uniform over the CTA
+    // grid.x runs over (scenario, pipeline), grid.y over tiles: CTAs are dispatched x-fastest,
+    // so every segment's first tile is evaluated before anybody's second one and most later
+    // tiles find their answer already there.
+    const uint32_t y = blockIdx.x;
+    const uint32_t b = y / bd.dp_max, p = y % bd.dp_max;
+    const Winner &w = bd.winner[b];
+    if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;          // uniform over the CTA
+    for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
         uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -294,8 +298,8 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         }
         __syncthreads();
         const uint64_t count = g.K ? g.K + 1 : 1;
-        const uint64_t first = (uint64_t)blockIdx.x * kTile;
-        if (first >= count || found_so_far < first) continue;       // uniform: read from shared
+        const uint64_t first = tile * kTile;
+        if (first >= count || found_so_far < first) break;          // uniform: later tiles cannot win either
         const uint64_t kappa = first + threadIdx.x;
         uint64_t hit = ~0ull;
         if (kappa < count) {
@@ -318,8 +322,9 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
 
 cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st) {
     if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
-    uint64_t ny = (uint64_t)b.B * b.dp_max;
-    dim3 grid(b.max_tiles_per_seg, (unsigned)(ny < 65535 ? ny : 65535), 1);
+    const uint64_t nx = (uint64_t)b.B * b.dp_max;
+    if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)nx, b.max_tiles_per_seg < 65535u ? b.max_tiles_per_seg : 65535u, 1);
     if (b.mode == CM_COST_INT64NS) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
     else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b);
     return cudaGetLastError();
