@@ -119,6 +119,20 @@ def aggregate(per_rank):
     return plans, seconds
 
 
+def gather_rows(values, world: int, device: str):
+    """Every rank's list of numbers on every rank (one all_gather; a list of one row when
+    there is a single rank).  The only collective of the benchmark: the search itself
+    exchanges nothing between GPUs."""
+    if world <= 1:
+        return [list(values)]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    gathered = [torch.zeros_like(t) for _ in range(world)]
+    dist.all_gather(gathered, t)
+    return [g.cpu().tolist() for g in gathered]
+
+
 def oracle_sample(w, mode: int, budget_s: float, max_scenarios: int):
     """Time the CPU oracle, as it stands, on the first scenarios of the workload until the
     budget is used.  -> (plans, seconds, scenarios)."""
@@ -259,13 +273,7 @@ def main():
     lat_pack.search(ctx, opts, latency=True)
     lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
 
-    if world > 1:
-        t = torch.tensor([float(plans_per_step * args.steps), dev_seconds, e2e_seconds], dtype=torch.float64, device="cuda")
-        gathered = [torch.zeros_like(t) for _ in range(world)]
-        dist.all_gather(gathered, t)
-        rows = [g.cpu().tolist() for g in gathered]
-    else:
-        rows = [[float(plans_per_step * args.steps), dev_seconds, e2e_seconds]]
+    rows = gather_rows([float(plans_per_step * args.steps), dev_seconds, e2e_seconds], world, "cuda")
     total_plans, max_dev = aggregate([(r[0], r[1]) for r in rows])
     _, max_e2e = aggregate([(r[0], r[2]) for r in rows])
 

@@ -294,3 +294,25 @@ ALL_WORKLOADS = {
     "175b-like": gpt175b_like,
     "sweep": sweep,
 }
+
+
+def deep_pipeline(seed: int = 0) -> Workload:
+    """A deliberately deep, narrow job (DP2 x PP40, L=70) whose search window reaches
+    pipelines of up to 64 stages: exercises the code paths for pipelines deeper than a
+    warp (40 stages fault-free) and deeper than the register-resident kernels cover."""
+    rng = SplitMix64(0xDEE9 + seed)
+    L, n_dp, n_pp, n_micro = 70, 2, 40, 48
+    fwd = [rng.uniform(2.0, 6.0) for _ in range(L)]
+    bwd = [f * rng.uniform(1.8, 2.2) for f in fwd]
+    act = [int(rng.uniform(2e6, 6e6)) for _ in range(L)]
+    par = [int(rng.uniform(4e7, 9e7)) for _ in range(L)]
+    p2p = [int(rng.uniform(1e6, 4e7)) for _ in range(L)]
+    base = [0]
+    for s in range(n_pp):
+        base.append(base[-1] + (2 if s < L - n_pp else 1))
+    prof = _make_profile(L, n_dp, n_pp, n_micro, fwd, bwd, act, par, [6 * v for v in par], p2p, base,
+                         cap=4_000_000_000, dev_per_node=8, bw_intra=300, bw_inter=20)
+    opts = SearchOptions(1, 3, 18, 64, LAYERS_REMAINDER, BATCH_REMAINDER, 40)
+    n = n_dp * n_pp
+    scen = [[7], [0], [41, 42], rng.sample_distinct(n, 3), rng.sample_distinct(n, 6), [39, 79]]
+    return Workload(f"deep-pipeline-{seed}", prof, opts, scen)

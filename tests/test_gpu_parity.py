@@ -172,6 +172,13 @@ def test_70b_like_memory_decides(gpu, oracle_factory):
     full_parity(gpu, oracle_factory, w, [w.scenarios[i] for i in (5, 58)], modes=(1,), candidates=False)
 
 
+def test_deep_pipelines_beyond_a_warp_and_beyond_the_register_kernels(gpu, oracle_factory):
+    # fault-free pipelines of 40 stages (policy kernel's serial path) and candidates of up to
+    # 61 stages (generic cost kernel), next to 18..48-stage ones with few segments per bucket
+    w = W.deep_pipeline()
+    full_parity(gpu, oracle_factory, w, w.scenarios)
+
+
 def _sampled_candidate_parity(gpu, oracle_factory, w, scenarios, n_samples, modes=(0, 1)):
     s = Session(gpu, w.profile)
     try:
