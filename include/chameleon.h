@@ -229,7 +229,8 @@ cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *space, uint64_
  *  [5] segments  [6] strategies  [7] micro-batch splits reduced
  *  [8] device time of the search-pass cost kernel(s) alone, ns   [9] bytes copied host->device
  *  [10] bytes copied device->host   [11] device time of the tie-break kernel(s), ns
- *  [12] launches of the search-pass cost kernel   [13..15] reserved (0). */
+ *  [12] launches of the search-pass cost kernel   [13] host time building descriptor tables, ns
+ *  [14] host time enqueueing the launch sequence, ns   [15] host time waiting for the stream, ns. */
 cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]);
 
 const char *cm_strerror(cm_status status);

@@ -63,6 +63,10 @@ template <typename T> struct DevBuf {
 
 inline uint64_t sat_add(uint64_t a, uint64_t b) { return a > kSat - b ? kSat : a + b; }
 
+inline uint64_t now_ns() {
+    return (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
 }  // namespace
 
 // One batch of failure scenarios: host tables, device mirrors, result buffers.
@@ -84,13 +88,11 @@ struct Batch {
     size_t off_scen = 0, off_tmpl = 0, off_strat = 0, off_tseg = 0, off_failed = 0, off_red = 0, off_keys = 0,
            off_tmpl_scen = 0, off_bucket_tseg = 0, off_cross = 0, off_bucket = 0;
     PinnedVec<cm_plan> plans_host;
-    PinnedVec<unsigned long long> counters_host;
     DevBuf<uint64_t> d_seg_best, d_kappa_sel, d_pol_cost;
     DevBuf<Partial> d_partial;
     DevBuf<Winner> d_winner;
     DevBuf<uint16_t> d_rc_stages;
     DevBuf<cm_plan> d_plans;
-    DevBuf<unsigned long long> d_counters;
     cm_enum_opts opts{};
     uint32_t policy_mask = 0;
     uint64_t n_cand = 0, n_tiles = 0, n_split = 0;
@@ -230,15 +232,16 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
         }
     }
     for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_GENERIC; ++kind) {
-        LaunchClass generic{CM_CLASS_GENERIC, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+        uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
+        LaunchClass generic{CM_CLASS_GENERIC, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
-            LaunchClass cls{kind, S, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+            LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
             LaunchClass &c = kind == CM_CLASS_GENERIC ? generic : cls;
             for (const Pre &q : pre) {
                 if (q.kind != kind || q.S != S) continue;
                 Bucket bk{};
                 bk.count = q.count;
-                bk.chunk_first = c.n_chunks;
+                bk.chunk_first = c.chunk_begin + c.n_chunks;
                 bk.list_first = q.list_first;
                 bk.n_tseg = q.n_tseg;
                 bk.tmpl = q.tmpl;
@@ -254,7 +257,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 bt.bucket.push_back(bk);
                 c.bucket_end = (uint32_t)bt.bucket.size();
             }
-            if (kind != CM_CLASS_GENERIC && cls.n_chunks) bt.classes.push_back(cls);
+            if (kind != CM_CLASS_GENERIC && cls.n_chunks) { bt.classes.push_back(cls); kind_chunks += cls.n_chunks; }
         }
         if (kind == CM_CLASS_GENERIC && generic.n_chunks) bt.classes.push_back(generic);
     }
@@ -462,7 +465,8 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
     v.seg_best = bt.d_seg_best.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
-    v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p; v.counters = bt.d_counters.p;
+    v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
+    v.counters = reinterpret_cast<unsigned long long *>(bt.d_seg_best.p + bt.n_rows);
     v.B = bt.B; v.mode = bt.opts.cost;
     v.n_rows = (uint32_t)bt.n_rows; v.n_strat = (uint32_t)bt.strat.size();
     v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
@@ -499,10 +503,10 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     CM_CUDA(ctx, cudaMemcpyAsync(bt.d_arena.p, bt.arena.p, bt.arena.size(), cudaMemcpyHostToDevice, ctx->stream));
     ctx->stats[9] += bt.arena.size();
     const size_t B = std::max(bt.B, 1);
-    ok = bt.d_seg_best.reserve(std::max<size_t>(bt.n_rows, 1)) &&
+    ok = bt.d_seg_best.reserve(bt.n_rows + 4) &&   // + the four work counters, cleared by the same memset
          bt.d_partial.reserve(std::max<size_t>(bt.red_scen.size(), 1)) && bt.d_winner.reserve(B) &&
          bt.d_kappa_sel.reserve(B * kMaxP) && bt.d_pol_cost.reserve(B * 2) &&
-         bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4) && bt.d_counters.reserve(4);
+         bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4 + 1);   // + room for the counters
     if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
     if (bt.keys.size()) {
         CM_CUDA(ctx, launch_minmax(tables(ctx, bt.opts.cost), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
@@ -520,9 +524,11 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     const BatchDev bd = dev_view(ctx, bt);
     cudaStream_t st = ctx->stream;
     int launches = launches_so_far, cost_launches = 0;
+    const uint64_t h_enqueue = now_ns();
     CM_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
-    if (bt.n_rows) CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, bt.n_rows * sizeof(uint64_t), st));
-    CM_CUDA(ctx, cudaMemsetAsync(bt.d_counters.p, 0, 4 * sizeof(unsigned long long), st));
+    // per-segment minima start at all-ones (above every cost); so do the work counters, which
+    // therefore read "value - 1" until cm_finalize_kernel adds the one back
+    CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, (bt.n_rows + 4) * sizeof(uint64_t), st));
     if (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) {
         CM_CUDA(ctx, launch_policies(tb, bd, ctx->hp.n_dp, st));
         ++launches;
@@ -541,10 +547,13 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     CM_CUDA(ctx, launch_finalize(tb, bd, st));
     ++launches;
     CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
-    if (!bt.plans_host.resize((size_t)bt.B * 4) || !bt.counters_host.resize(4)) return fail(ctx, CM_ENOMEM, "host memory");
-    CM_CUDA(ctx, cudaMemcpyAsync(bt.plans_host.p, bt.d_plans.p, (size_t)bt.B * 4 * sizeof(cm_plan), cudaMemcpyDeviceToHost, st));
-    CM_CUDA(ctx, cudaMemcpyAsync(bt.counters_host.p, bt.d_counters.p, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st));
+    const size_t plan_bytes = (size_t)bt.B * 4 * sizeof(cm_plan), back_bytes = plan_bytes + 4 * sizeof(unsigned long long);
+    if (!bt.plans_host.resize((size_t)bt.B * 4 + 1)) return fail(ctx, CM_ENOMEM, "host memory");
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.plans_host.p, bt.d_plans.p, back_bytes, cudaMemcpyDeviceToHost, st));
+    const uint64_t h_wait = now_ns();
     CM_CUDA(ctx, cudaStreamSynchronize(st));
+    ctx->stats[14] += h_wait - h_enqueue;
+    ctx->stats[15] += now_ns() - h_wait;
     float ms = 0.f;
     CM_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
@@ -555,10 +564,11 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
         ctx->stats[11] += (uint64_t)((double)ms_tie * 1e6);
         ctx->stats[12] += (uint64_t)cost_launches;
     }
-    ctx->stats[10] += (size_t)bt.B * 4 * sizeof(cm_plan) + 4 * sizeof(unsigned long long);
+    ctx->stats[10] += back_bytes;
+    const unsigned long long *counters_host = reinterpret_cast<const unsigned long long *>(bt.plans_host.p + (size_t)bt.B * 4);
     ctx->stats[0] += (bt.policy_mask & (1u << CM_DYNPAR)) ? bt.n_cand : 0;
-    ctx->stats[1] += bt.counters_host[0];
-    ctx->stats[2] += bt.counters_host[1];
+    ctx->stats[1] += counters_host[0];
+    ctx->stats[2] += counters_host[1];
     ctx->stats[3] += (uint64_t)launches;
     ctx->stats[4] += (uint64_t)((double)ms * 1e6);
     ctx->stats[5] += bt.n_rows;
@@ -854,7 +864,9 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
     };
     if (!latency_us) {
         int launches = 0;
+        const uint64_t h0 = now_ns();
         if ((s = build_batch(ctx, bt, failed_ids, offsets, B, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        ctx->stats[13] += now_ns() - h0;
         if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
         if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
         for (int b = 0; b < B; ++b) copy_out(b, b);
@@ -864,7 +876,9 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         const auto t0 = std::chrono::steady_clock::now();
         const int32_t off[2] = {0, offsets[b + 1] - offsets[b]};
         int launches = 0;
+        const uint64_t h0 = now_ns();
         if ((s = build_batch(ctx, bt, failed_ids + offsets[b], off, 1, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        ctx->stats[13] += now_ns() - h0;
         if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
         if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
         copy_out(b, 0);

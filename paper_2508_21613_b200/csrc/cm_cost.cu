@@ -20,7 +20,7 @@
 //       UNI = false: one plan per lane as in the register kernel, stage times in a
 //       per-lane shared-memory column; for buckets with too few segments to transpose.
 //   cm_cost_generic_kernel<T>       any S <= CM_MAX_STAGES: per-stage state in local memory.
-#include "cm_device.cuh"
+#include "cm_plan_eval.cuh"
 
 namespace cm {
 
@@ -88,256 +88,59 @@ __device__ __forceinline__ void count_cells(unsigned long long *counter, unsigne
 }
 
 // ----------------------------------------------------------------------------------
-// Layer cuts of a plan, stage after stage (no array: the caller consumes them in order).
-//   kind 0  REMAINDER: n_i = q + bit i of a           (a = subset mask from the rank)
-//   kind 1  FULL:      cut positions are the set bits of the 128-bit mask (a, b)
-//   kind 2  min-max partition row
-// ----------------------------------------------------------------------------------
-struct CutWalker {
-    uint64_t a, b;
-    const uint8_t *row;
-    int kind, q, L, S, i, pos;
-    __device__ __forceinline__ int next() {   // upper cut of stage i, then advance
-        int hi;
-        if (kind == 0) {
-            hi = pos + q + (int)((a >> i) & 1ull);
-        } else if (kind == 1) {
-            if (i == S - 1) hi = L;
-            else if (a) { hi = __ffsll((long long)a); a &= a - 1; }
-            else { hi = 64 + __ffsll((long long)b); b &= b - 1; }
-        } else {
-            hi = row[i + 1];
-        }
-        pos = hi;
-        ++i;
-        return hi;
-    }
-};
-
-__device__ __forceinline__ bool make_walker(CutWalker &w, const Tables &tb, int layer_mode, int L, int S,
-                                            uint64_t kappa, uint64_t K, uint32_t mm_slot) {
-    w.a = 0; w.b = 0; w.row = nullptr; w.q = 0; w.L = L; w.S = S; w.i = 0; w.pos = 0;
-    if (kappa < K) {
-        if (layer_mode == CM_LAYERS_REMAINDER) {
-            w.kind = 0;
-            w.q = L / S;
-            uint64_t mask = 0;
-            unrank_subset(tb.binom, kappa, S, L % S, [&](int, int v) { mask |= 1ull << v; });
-            w.a = mask;
-        } else {
-            w.kind = 1;
-            uint64_t m0 = 0, m1 = 0;
-            unrank_subset(tb.binom, kappa, L - 1, S - 1, [&](int, int v) {
-                if (v < 64) m0 |= 1ull << v; else m1 |= 1ull << (v - 64);
-            });
-            w.a = m0; w.b = m1;
-        }
-        return true;
-    }
-    w.kind = 2;
-    w.row = tb.mm_cuts + (size_t)mm_slot * (kMaxS + 1);
-    return w.row[0] == 0;   // 255 marks "no memory-feasible partition"
-}
-
-// ----------------------------------------------------------------------------------
-// The recurrence in "rounds", S compile-time, clock and pending forward in registers.
-//
-// Round t = 0 .. S-2+m; stages are visited from last to first.  In round t stage i runs
-//   its forward of micro-batch t-i      if 0 <= t-i < m   (fed by the forward that stage
-//                                        i-1 ran in round t-1 and left pending), then
-//   its backward of micro-batch t-S+1   if t >= S-1       (fed by the backward stage i+1
-//                                        ran just before in the same round; by its own
-//                                        forward at the last stage).
-// Per stage this is exactly the 1F1B order -- min(S-1-i, m) forwards, forward/backward
-// pairs, the remaining backwards -- for every m >= 1, and every dependency is either one
-// round or one stage old, so two values per stage are all the state there is.
-// Rounds S-1 .. m-1 have every stage fully active and carry no predicate at all; the
-// ramp-up and ramp-down rounds skip inactive stages with warp-uniform branches.
-//
-// stage(i) returns the stage's forward and backward time, xt(i) the transfer time of the
-// boundary above stage i; both are called with compile-time i only.
-// ----------------------------------------------------------------------------------
-template <typename T> struct alignas(16) FB { T f, b; };
-
-// Shared-memory loads the compiler must issue where they stand: the stage times are loop
-// invariants, and hoisting ~100 of them into registers would push the per-stage state out.
-template <typename T>
-__device__ __forceinline__ FB<T> lds_fb(const FB<T> *p) {
-    unsigned long long a, b;
-    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"((unsigned)__cvta_generic_to_shared(p)));
-    FB<T> d;
-    d.f = Num<T>::from_bits(a);
-    d.b = Num<T>::from_bits(b);
-    return d;
-}
-template <typename T>
-__device__ __forceinline__ T lds_t(const T *p) {
-    unsigned long long a;
-    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(a) : "r"((unsigned)__cvta_generic_to_shared(p)));
-    return Num<T>::from_bits(a);
-}
-
-template <typename T, int S, typename StageFn, typename XtFn>
-__device__ __forceinline__ T sim_rounds(int m, StageFn stage, XtFn xt) {
-    T clock[S], pend[S];
-#pragma unroll
-    for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
-    // ramp-up: forwards only
-    for (int t = 0; t < S - 1; ++t) {
-#pragma unroll
-        for (int i = S - 2; i >= 0; --i) {
-            if (i <= t && t < i + m) {
-                const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-                const T fend = fstart + stage(i).f;
-                clock[i] = fend;
-                pend[i + 1] = fend + xt(i);
-            }
-        }
-    }
-    // steady rounds: every stage does one forward and one backward
-    for (int t = S - 1; t < m; ++t) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            const FB<T> d = stage(i);
-            const T x = i < S - 1 ? xt(i) : (T)0;
-            const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-            const T fend = fstart + d.f;
-            if (i < S - 1) pend[i + 1] = fend + x;
-            const T dep = i < S - 1 ? chain_b + x : fend;
-            const T bstart = tmax(fend, dep);
-            const T bend = bstart + d.b;
-            clock[i] = bend;
-            chain_b = bend;
-        }
-    }
-    // ramp-down: every stage still has a backward, the upper ones a forward too
-    for (int t = (m > S - 1 ? m : S - 1); t < S - 1 + m; ++t) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            const FB<T> d = stage(i);
-            const T x = i < S - 1 ? xt(i) : (T)0;
-            T c = clock[i];
-            if (t < i + m) {
-                const T fstart = i > 0 ? tmax(c, pend[i]) : c;
-                c = fstart + d.f;
-                if (i < S - 1) pend[i + 1] = c + x;
-            }
-            const T dep = i < S - 1 ? chain_b + x : c;
-            const T bstart = tmax(c, dep);
-            const T bend = bstart + d.b;
-            clock[i] = bend;
-            chain_b = bend;
-        }
-    }
-    return clock[0];
-}
-
-// ----------------------------------------------------------------------------------
-// The same recurrence for shallow pipelines (S <= 16) with m >= S-1, where every stage
-// has its full warm-up: warm-up and cool-down are unrolled triangles without a single
-// branch (S^2 cells of code, affordable at this depth), the steady rounds as above.
-// Order: warm-up forwards micro-batch by micro-batch up the stages, the last forward of
-// a row left pending for the stage above; then rounds k = 0..m-1 from the last stage to
-// the first, forward (while one is left) then backward.
-// ----------------------------------------------------------------------------------
-template <typename T, int S>
-__device__ __forceinline__ T sim_regs(int m, const FB<T> (&st)[S], const T (&xt)[S]) {
-    T clock[S], pend[S];
-#pragma unroll
-    for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
-#pragma unroll
-    for (int j = 0; j < S - 1; ++j) {
-        T chain = (T)0;
-#pragma unroll
-        for (int i = 0; i <= S - 2 - j; ++i) {
-            const T start = i > 0 ? tmax(clock[i], chain) : clock[i];
-            const T end = start + st[i].f;
-            clock[i] = end;
-            chain = end + xt[i];
-        }
-        pend[S - 1 - j] = chain;
-    }
-    for (int k = 0; k <= m - S; ++k) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-            const T fend = fstart + st[i].f;
-            if (i < S - 1) pend[i + 1] = fend + xt[i];
-            const T dep = i < S - 1 ? chain_b + xt[i] : fend;
-            const T bstart = tmax(fend, dep);
-            const T bend = bstart + st[i].b;
-            clock[i] = bend;
-            chain_b = bend;
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < S - 1; ++r) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            T c = clock[i];
-            if (i > r) {
-                const T fstart = i > 0 ? tmax(c, pend[i]) : c;
-                c = fstart + st[i].f;
-                if (i < S - 1) pend[i + 1] = c + xt[i];
-            }
-            const T dep = i < S - 1 ? chain_b + xt[i] : c;
-            const T bstart = tmax(c, dep);
-            const T bend = bstart + st[i].b;
-            clock[i] = bend;
-            chain_b = bend;
-        }
-    }
-    return clock[0];
-}
-
-// ----------------------------------------------------------------------------------
 // S <= 16: one thread per plan, all in registers.
 // ----------------------------------------------------------------------------------
 template <typename T, int S>
-__global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+__global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1,
+                                                              uint64_t chunk_offset) {
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
-    const uint64_t chunk = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
     stage_profile(sp, tb.prof);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
-    const int m = bk.m, L = sp.L;
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
     uint64_t seg_local, kappa;
     plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
     uint32_t row = 0xffffffffu;
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
-    if (seg_local < bk.n_seg && m >= 1) {
+    if (seg_local < bk.n_seg) {
         const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
         row = g.row;
-        const uint64_t tier = g.tier, K = g.K;
-        const int n_sync = g.n_sync;
-        CutWalker cw;
-        bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, K, tb.mm_slot(S, m));
-        FB<T> st[S];
-        T xts[S];
-        long long g_max = 0;
-        int lo = 0;
-#pragma unroll
-        for (int i = 0; i < S; ++i) {
-            const int hi = ok ? cw.next() : lo + 1;
-            ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-            st[i].f = sp.PF[hi] - sp.PF[lo];
-            st[i].b = sp.PB[hi] - sp.PB[lo];
-            xts[i] = i < S - 1 ? sp.XT[(tier >> i) & 1ull][hi - 1] : (T)0;
-            const long long gb = sp.PP[hi] - sp.PP[lo];
-            g_max = gb > g_max ? gb : g_max;
-            lo = hi;
+        T cost;
+        if (plan_cost_regs<T, S>(sp, tb, bd.layer_mode, g, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * S * g.m;
         }
-        if (ok) {
-            const T t = sim_regs<T, S>(m, st, xts);
-            bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync));
-            my_cells = 2ull * S * m;
+    }
+    segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+// Every shallow depth in one launch: for batches so small that a launch per depth would
+// cost more than the work (a single failure scenario of a 32-device job is ~250 CTAs).
+template <typename T>
+__global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    const uint64_t chunk = (uint64_t)blockIdx.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T cost;
+        if (plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * g.S * g.m;
         }
     }
     segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
@@ -358,11 +161,11 @@ template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
 }
 
 template <typename T, int S, bool UNI>
-__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     extern __shared__ __align__(16) unsigned char dyn[];
-    const uint64_t chunk = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
     stage_profile(sp, tb.prof);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
@@ -470,10 +273,10 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+__global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
-    const uint64_t chunk = (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
     stage_profile(sp, tb.prof);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
@@ -504,7 +307,7 @@ static dim3 chunk_grid(uint64_t n) {
 
 template <typename T, int S>
 static cudaError_t launch_regs(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    cm_cost_regs_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    cm_cost_regs_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
     return cudaGetLastError();
 }
 
@@ -519,7 +322,7 @@ static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const Lau
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
     return cudaGetLastError();
 }
 
@@ -549,7 +352,7 @@ static cudaError_t launch_class(const Tables &t, const BatchDev &b, const Launch
         default: break;
         }
     }
-    cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end);
+    cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
     return cudaGetLastError();
 }
 
@@ -557,7 +360,21 @@ static cudaError_t launch_class(const Tables &t, const BatchDev &b, const Launch
 // see indices past its plans and idle.
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
                               cudaStream_t st, int *launches) {
-    for (int i = 0; i < n_classes; ++i) {
+    // the register-resident classes come first and share one chunk numbering
+    int n_regs = 0;
+    uint64_t regs_chunks = 0;
+    while (n_regs < n_classes && classes[n_regs].kind == CM_CLASS_REGS) regs_chunks += classes[n_regs++].n_chunks;
+    int first = 0;
+    if (n_regs > 1 && regs_chunks > 0 && regs_chunks <= (uint64_t)kAnyMaxChunks) {
+        const uint32_t b0 = classes[0].bucket_begin, b1 = classes[n_regs - 1].bucket_end;
+        if (b.mode == CM_COST_INT64NS) cm_cost_regs_any_kernel<long long><<<(unsigned)regs_chunks, kChunk, 0, st>>>(t, b, b0, b1);
+        else cm_cost_regs_any_kernel<double><<<(unsigned)regs_chunks, kChunk, 0, st>>>(t, b, b0, b1);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        if (launches) ++*launches;
+        first = n_regs;
+    }
+    for (int i = first; i < n_classes; ++i) {
         if (classes[i].n_chunks == 0) continue;
         cudaError_t e = b.mode == CM_COST_INT64NS ? launch_class<long long>(t, b, classes[i], st)
                                                   : launch_class<double>(t, b, classes[i], st);

@@ -100,8 +100,10 @@ struct Bucket {
 enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_GENERIC = 3 };
 constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
 constexpr int kUniMinSegments = 16; // fewer segments in a bucket: not worth transposing
+constexpr int kAnyMaxChunks = 4096; // shallow classes smaller than this together: one launch for all depths
 struct LaunchClass {
     int kind, stages;
+    uint64_t chunk_begin;  // first chunk of the class in its kind's chunk numbering
     uint32_t bucket_begin, bucket_end;
     uint64_t n_chunks;
 };

@@ -10,7 +10,7 @@
 //   cm_finalize_kernel    assembles the plans and picks the best policy
 //   cm_evaluate_kernel    per-candidate cost / feasibility for cm_evaluate
 //   cm_pick_kernel        best of several spaces for cm_select
-#include "cm_device.cuh"
+#include "cm_plan_eval.cuh"
 
 namespace cm {
 
@@ -304,9 +304,11 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         uint64_t hit = ~0ull;
         if (kappa < count) {
             T cost;
-            if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost) &&
-                Num<T>::bits(cost) <= w.cost_bits)
-                hit = kappa;
+            // shallow pipelines take the register-resident evaluation, the rest the generic one
+            const bool ok = (g.S <= kRegStagesMax && g.m >= g.S - 1)
+                                ? plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost)
+                                : segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost);
+            if (ok && Num<T>::bits(cost) <= w.cost_bits) hit = kappa;
         }
         hit = warp_min_u64(hit);
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = hit;
@@ -352,6 +354,11 @@ __device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mo
 
 __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b == 0) {
+        // work counters ride home behind the plans (they start at all-ones, i.e. -1)
+        unsigned long long *tail = reinterpret_cast<unsigned long long *>(bd.plans + (size_t)bd.B * 4);
+        for (int i = 0; i < 4; ++i) tail[i] = bd.counters[i] + 1ull;
+    }
     if (b >= bd.B) return;
     const DevProfile *p = tb.prof;
     const Scen sc = bd.scen[b];
