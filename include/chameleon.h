@@ -20,7 +20,9 @@
  *  - "HOST" / "DEVICE" at a pointer says where the memory lives.  The caller owns every
  *    buffer it passes; the library owns cm_ctx and cm_space objects until they are
  *    destroyed / freed.
- *  - All device work is enqueued on the context's stream.  Calls that return results to
+ *  - All device work is enqueued on the context's stream (independent kernels of the search
+ *    pass may run on streams the library owns, forked from and joined back into the
+ *    context's stream, so ordering as seen from that stream is unchanged).  Calls that return results to
  *    the host (cm_select, cm_search_batch, cm_decode_plan) synchronise that stream
  *    before returning; cm_load_profile, cm_enumerate and cm_evaluate only enqueue.
  *  - A cm_ctx is not thread-safe; distinct contexts are independent.

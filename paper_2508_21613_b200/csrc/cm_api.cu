@@ -116,6 +116,7 @@ struct cm_ctx {
     int mm_stride_m = 0;
     Batch batch;                      // reused by cm_search_batch
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
 };
@@ -535,13 +536,19 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
     }
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
-        CM_CUDA(ctx, launch_cost_pass1(tb, bd, bt.classes.data(), (int)bt.classes.size(), st, &cost_launches));
+        CM_CUDA(ctx, launch_cost_pass1(tb, bd, bt.classes.data(), (int)bt.classes.size(), st, &ctx->side, &cost_launches));
         launches += cost_launches;
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
         CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
         launches += bd.n_red_blocks ? 2 : 1;
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
-        if (bt.n_tiles) { CM_CUDA(ctx, launch_cost_pass2(tb, bd, st)); ++launches; }
+        if (bt.n_tiles) {
+            CM_CUDA(ctx, launch_cost_pass2(tb, bd, st));
+            ++launches;
+            uint64_t stage_mask = 0;
+            for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
+            CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &launches));
+        }
         CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
     }
     CM_CUDA(ctx, launch_finalize(tb, bd, st));
@@ -645,6 +652,12 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
     c->stream = (cudaStream_t)cuda_stream;
     bool ok = true;
     for (int i = 0; i < 6; ++i) ok = ok && cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->side.fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 3 && ok; ++i) {
+        ok = cudaStreamCreateWithFlags(&c->side.stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->side.join[i], cudaEventDisableTiming) == cudaSuccess;
+        if (ok) c->side.n = i + 1;
+    }
     if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess) {
         cudaGetLastError();
         delete c;
@@ -660,6 +673,11 @@ cm_status cm_destroy(cm_ctx *c) {
     cudaStreamSynchronize(c->stream);
     for (int i = 0; i < 6; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (int i = 0; i < 3; ++i) {
+        if (c->side.stream[i]) { cudaStreamSynchronize(c->side.stream[i]); cudaStreamDestroy(c->side.stream[i]); }
+        if (c->side.join[i]) cudaEventDestroy(c->side.join[i]);
+    }
+    if (c->side.fork) cudaEventDestroy(c->side.fork);
     if (c->d_prof) cudaFree(c->d_prof);
     if (c->d_binom) cudaFree(c->d_binom);
     for (int i = 0; i < 2; ++i)

@@ -244,26 +244,9 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
         if (seg_local < bk.n_seg && m >= 1) {
             const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
             row = g.row;
-            const uint64_t tier = g.tier;
-            CutWalker cw;
-            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
-            long long g_max = 0;
-            int lo = 0;
-            for (int i = 0; i < S && ok; ++i) {
-                const int hi = cw.next();
-                ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-                FB<T> d;
-                d.f = sp.PF[hi] - sp.PF[lo];
-                d.b = sp.PB[hi] - sp.PB[lo];
-                fcol[i * kChunk] = d;
-                xcol[i * kChunk] = i < S - 1 ? sp.XT[(tier >> i) & 1ull][hi - 1] : (T)0;
-                const long long gb = sp.PP[hi] - sp.PP[lo];
-                g_max = gb > g_max ? gb : g_max;
-                lo = hi;
-            }
-            if (ok) {
-                const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-                bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync));
+            T cost;
+            if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost)) {
+                bits = Num<T>::bits(cost);
                 my_cells = 2ull * S * m;
             }
         }
@@ -356,10 +339,105 @@ static cudaError_t launch_class(const Tables &t, const BatchDev &b, const Launch
     return cudaGetLastError();
 }
 
+// ----------------------------------------------------------------------------------
+// Tie-break pass for the winners' deep pipelines (17..48 stages): the lowest layer
+// composition that is feasible with cost <= T*.  Same grid as the generic tie-break
+// kernel -- x = (scenario, pipeline), y = tiles of kChunk compositions -- one launch per
+// stage count; CTAs whose winner segment has another depth leave at once.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_wide_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ uint64_t red[kChunk / 32];
+    __shared__ SegView g;
+    __shared__ uint64_t found_so_far;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint32_t b = blockIdx.x / bd.dp_max, p = blockIdx.x % bd.dp_max;
+    const Winner &w = bd.winner[b];
+    if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;            // uniform over the CTA
+    if (bd.tseg[w.seg[p]].S != S) return;
+    stage_profile(sp, tb.prof);
+    FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + threadIdx.x;
+    T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + threadIdx.x;
+    uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
+    for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            g = seg_view(bd, b, w.seg[p]);
+            found_so_far = *(volatile uint64_t *)slot;
+        }
+        __syncthreads();
+        const uint64_t count = g.K ? g.K + 1 : 1;
+        const uint64_t first = tile * kChunk;
+        if (first >= count || found_so_far < first) break;              // uniform: later tiles cannot win either
+        const uint64_t kappa = first + threadIdx.x;
+        uint64_t hit = ~0ull;
+        if (kappa < count) {
+            T cost;
+            if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost) &&
+                Num<T>::bits(cost) <= w.cost_bits)
+                hit = kappa;
+        }
+        hit = warp_min_u64(hit);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = hit;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int q = 0; q < kChunk / 32; ++q) hit = red[q] < hit ? red[q] : hit;
+            if (hit != ~0ull) atomicMin((unsigned long long *)slot, (unsigned long long)hit);
+            const uint64_t n = count - first < (uint64_t)kChunk ? count - first : (uint64_t)kChunk;
+            atomicAdd(&bd.counters[1], (unsigned long long)n);
+        }
+    }
+}
+
+template <typename T, int S>
+static cudaError_t launch_tiebreak_wide_one(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, false, T>();
+    static bool configured[16] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 16 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(cm_tiebreak_wide_kernel<T, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const uint64_t nx = (uint64_t)b.B * b.dp_max;
+    if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)nx, tiebreak_grid_y(nx, b.max_tiles_per_seg), 1);
+    cm_tiebreak_wide_kernel<T, S><<<grid, kChunk, smem, st>>>(t, b);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t launch_tiebreak_wide_S(const Tables &t, const BatchDev &b, int S, cudaStream_t st) {
+    switch (S) {
+#define CM_CASE(S) case S: return launch_tiebreak_wide_one<T, S>(t, b, st);
+        CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
+        CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
+        CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
+        CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
+#undef CM_CASE
+    default: return cudaSuccess;
+    }
+}
+
+// stage_mask: bit S set = some template segment of the batch has S stages (17 <= S <= 48)
+cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st, int *launches) {
+    if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
+    for (int S = kRegStagesMax + 1; S <= kWideStagesMax; ++S) {
+        if (!((stage_mask >> S) & 1ull)) continue;
+        cudaError_t e = b.mode == CM_COST_INT64NS ? launch_tiebreak_wide_S<long long>(t, b, S, st)
+                                                  : launch_tiebreak_wide_S<double>(t, b, S, st);
+        if (e != cudaSuccess) return e;
+        if (launches) ++*launches;
+    }
+    return cudaSuccess;
+}
+
 // A 2-D grid may overshoot the class's chunk count; surplus CTAs find the last bucket,
 // see indices past its plans and idle.
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
-                              cudaStream_t st, int *launches) {
+                              cudaStream_t st, const SideStreams *side, int *launches) {
     // the register-resident classes come first and share one chunk numbering
     int n_regs = 0;
     uint64_t regs_chunks = 0;
@@ -374,14 +452,31 @@ cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchCl
         if (launches) ++*launches;
         first = n_regs;
     }
-    for (int i = first; i < n_classes; ++i) {
-        if (classes[i].n_chunks == 0) continue;
-        cudaError_t e = b.mode == CM_COST_INT64NS ? launch_class<long long>(t, b, classes[i], st)
-                                                  : launch_class<double>(t, b, classes[i], st);
+    int n_launch = 0;
+    for (int i = first; i < n_classes; ++i) n_launch += classes[i].n_chunks ? 1 : 0;
+    // classes only share the per-segment minima they atomically lower: run them side by side
+    const int n_side = (side && n_launch > 1) ? side->n : 0;
+    if (n_side) {
+        cudaError_t e = cudaEventRecord(side->fork, st);
+        for (int k = 0; k < n_side && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(side->stream[k], side->fork, 0);
         if (e != cudaSuccess) return e;
-        if (launches) ++*launches;
     }
-    return cudaSuccess;
+    cudaError_t err = cudaSuccess;
+    int slot = 0;
+    for (int i = first; i < n_classes && err == cudaSuccess; ++i) {
+        if (classes[i].n_chunks == 0) continue;
+        cudaStream_t s = (n_side && slot % (n_side + 1)) ? side->stream[slot % (n_side + 1) - 1] : st;
+        ++slot;
+        err = b.mode == CM_COST_INT64NS ? launch_class<long long>(t, b, classes[i], s) : launch_class<double>(t, b, classes[i], s);
+        if (err == cudaSuccess && launches) ++*launches;
+    }
+    // always join, even after a failed launch, so that the side streams never run ahead unobserved
+    for (int k = 0; k < n_side; ++k) {
+        cudaError_t e = cudaEventRecord(side->join[k], side->stream[k]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join[k], 0);
+        if (err == cudaSuccess) err = e;
+    }
+    return err;
 }
 
 }  // namespace cm

@@ -163,10 +163,30 @@ struct Tables {
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st);
+// Tiles of a segment that the tie-break kernels take side by side (grid.y); the rest is
+// walked serially inside the CTA.  A single scenario gets every tile its own CTA (lowest
+// latency), a large batch about one CTA per (scenario, pipeline): most of those stop after
+// their first tile anyway, and an idle CTA per tile would cost more than the work.
+inline unsigned tiebreak_grid_y(uint64_t nx, uint32_t max_tiles) {
+    const uint64_t target = 2048;   // CTAs worth launching
+    uint64_t y = nx ? (target + nx - 1) / nx : 1;
+    if (y > max_tiles) y = max_tiles;
+    if (y > 65535) y = 65535;
+    return (unsigned)(y ? y : 1);
+}
+
+// side streams (may be NULL / 0): launch classes are independent of one another, so they are
+// spread over the caller's stream and the side streams and joined again before returning
+struct SideStreams {
+    cudaStream_t stream[3];
+    cudaEvent_t fork, join[3];
+    int n;
+};
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
-                              cudaStream_t st, int *launches);
+                              cudaStream_t st, const SideStreams *side, int *launches);
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);
 cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st);
+cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st, int *launches);
 cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st);
 // single_policy < 0: candidates of the dynamic-parallelism segments; otherwise the one
 // candidate of that policy (its cost must already be in pol_cost of scenario 0)

@@ -289,6 +289,10 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
     const uint32_t b = y / bd.dp_max, p = y % bd.dp_max;
     const Winner &w = bd.winner[b];
     if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;          // uniform over the CTA
+    {
+        const int S = bd.tseg[w.seg[p]].S;   // 17..48 stages: cm_tiebreak_wide_kernel's job
+        if (S > kRegStagesMax && S <= kWideStagesMax) return;
+    }
     for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
         uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
         __syncthreads();
@@ -326,7 +330,7 @@ cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t s
     if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
     const uint64_t nx = (uint64_t)b.B * b.dp_max;
     if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
-    dim3 grid((unsigned)nx, b.max_tiles_per_seg < 65535u ? b.max_tiles_per_seg : 65535u, 1);
+    dim3 grid((unsigned)nx, tiebreak_grid_y(nx, b.max_tiles_per_seg), 1);
     if (b.mode == CM_COST_INT64NS) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
     else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b);
     return cudaGetLastError();

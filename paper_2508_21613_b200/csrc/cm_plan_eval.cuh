@@ -244,6 +244,39 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
     return true;
 }
 
+// ----------------------------------------------------------------------------------
+// Cost of one pipeline-plan of a deep pipeline (S compile-time, any m >= 1): clock and
+// pending forward in registers, the stage times in this lane's shared-memory columns
+// fcol / xcol (element i at index i * kChunk).  Returns false if the plan is infeasible.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Tables &tb, int layer_mode,
+                                                    const SegView &g, uint64_t kappa, FB<T> *fcol, T *xcol, T &cost) {
+    const int m = g.m;
+    if (m < 1) return false;
+    CutWalker cw;
+    bool ok = make_walker(cw, tb, layer_mode, sp.L, S, kappa, g.K, tb.mm_slot(S, m));
+    long long g_max = 0;
+    int lo = 0;
+    for (int i = 0; i < S && ok; ++i) {
+        const int hi = cw.next();
+        ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+        FB<T> d;
+        d.f = sp.PF[hi] - sp.PF[lo];
+        d.b = sp.PB[hi] - sp.PB[lo];
+        fcol[i * kChunk] = d;
+        xcol[i * kChunk] = i < S - 1 ? sp.XT[(g.tier >> i) & 1ull][hi - 1] : (T)0;
+        const long long gb = sp.PP[hi] - sp.PP[lo];
+        g_max = gb > g_max ? gb : g_max;
+        lo = hi;
+    }
+    if (!ok) return false;
+    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); },
+                                 [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+    cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync);
+    return true;
+}
+
 // The same with S chosen at run time (one kernel for every shallow depth; used where the
 // work is too small to be worth one launch per depth).  Caller guarantees 1 <= S <= 16, m >= S-1.
 template <typename T>
