@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libchameleon.so")
 SOURCES = ["cm_api.cu", "cm_kernels.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu"]
-HEADERS = ["cm_internal.h", "cm_device.cuh"]
+HEADERS = ["cm_internal.h", "cm_device.cuh", "cm_plan_eval.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

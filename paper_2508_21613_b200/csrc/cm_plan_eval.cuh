@@ -115,6 +115,9 @@ __device__ __forceinline__ T sim_rounds(int m, StageFn stage, XtFn xt) {
         }
     }
     // steady rounds: every stage does one forward and one backward
+    // four rounds per trip: the backward chain of one round overlaps the forwards of the
+    // next ones in the instruction stream, which hides its fixed latencies
+#pragma unroll 4
     for (int t = S - 1; t < m; ++t) {
         T chain_b = (T)0;
 #pragma unroll
@@ -179,6 +182,7 @@ __device__ __forceinline__ T sim_regs(int m, const FB<T> (&st)[S], const T (&xt)
         }
         pend[S - 1 - j] = chain;
     }
+#pragma unroll 4
     for (int k = 0; k <= m - S; ++k) {
         T chain_b = (T)0;
 #pragma unroll
