@@ -34,6 +34,7 @@ SM_MAX_MHZ_FALLBACK = 1965.0
 # 64-bit integer max costs 4 half-rate integer instructions:
 #   fp64:  2 DADD (4) + DSETP (2) + 2 SEL (2) = 8       int64: measured 12.3 by a probe kernel
 ISSUE_SLOTS_PER_CELL = {0: 8.0, 1: 12.0}
+TRAFFIC_BYTES_PER_CTA = 645888.0 / 55800.0   # dram__bytes_read+write of one ncu-captured launch / its CTAs
 
 
 def measured_peaks():
@@ -178,6 +179,91 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, latency_scenarios, sample_clocks=True):
+    """One workload on this rank: device-resident arm, end-to-end arm, per-failure latency."""
+    import numpy as np
+    opts = w.options.with_cost_mode(mode)
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    packed = binding.PackedScenarios(w.scenarios)
+    out = {}
+    try:
+        # ---- device-resident arm: descriptors already in HBM when the timed region starts
+        batch, n_cand = packed.prepare(ctx, opts)
+        for _ in range(warmup):
+            packed.search_prepared(ctx, batch)
+        sampler = ClockSampler(local_rank) if sample_clocks else None
+        barrier()
+        if sampler:
+            sampler.start()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        stats_sum = {}
+        for k in range(steps):
+            flush.fill_(float(k))                       # evict L2 between timed iterations (untimed)
+            ev[k][0].record()
+            packed.search_prepared(ctx, batch)          # kernels + plans back on the host
+            ev[k][1].record()
+            for key, v in binding.cm_last_stats(ctx).items():
+                stats_sum[key] = stats_sum.get(key, 0) + v
+        barrier()
+        out["clocks"] = sampler.stop() if sampler else None
+        out["dev_seconds"] = sum(a.elapsed_time(b) for a, b in ev) * 1e-3
+        out["plans_per_step"] = n_cand + 2 * len(w.scenarios)   # + one rerouting and one redundant plan each
+        out["stats"] = stats_sum
+        binding.cm_batch_free(batch)
+
+        # ---- end-to-end arm: host failure sets in, host plans out, every step
+        for _ in range(warmup):
+            packed.search(ctx, opts)
+        barrier()
+        e2e_seconds = 0.0
+        for k in range(steps):
+            flush.fill_(float(k))
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            packed.search(ctx, opts)                    # cm_search_batch: build, H2D, kernels, D2H, sync
+            e2e_seconds += time.perf_counter() - t0
+            st = binding.cm_last_stats(ctx)
+            out["h2d"], out["d2h"] = st["h2d_bytes"] + packed.ids.nbytes + packed.offsets.nbytes, st["d2h_bytes"]
+        barrier()
+        out["e2e_seconds"] = e2e_seconds
+
+        # ---- search latency per failure: scenarios searched one at a time
+        n_lat = max(1, min(latency_scenarios, len(w.scenarios)))
+        lat_pack = binding.PackedScenarios(w.scenarios[:: max(1, len(w.scenarios) // n_lat)][:n_lat])
+        lat_pack.search(ctx, opts, latency=True)
+        lat_pack.search(ctx, opts, latency=True)
+        lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
+        out["latency_us"] = {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
+                             "max": float(lat[-1]), "scenarios": int(lat_pack.B),
+                             "what": "one failure set, all policies, descriptor build to plan on host"}
+    finally:
+        binding.cm_destroy(ctx)
+    return out
+
+
+def roofline_of(stats_sum, dev_seconds, mode, sm_max, peak_kind):
+    slots = ISSUE_SLOTS_PER_CELL[mode]
+    peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
+    cost_s = stats_sum["cost_kernel_ns"] * 1e-9
+    achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
+    launches = max(1, stats_sum["cost_kernel_launches"])
+    return {
+        "bound": "alu", "kernel": "search pass: cm_cost_regs_kernel / cm_cost_wide_kernel / cm_cost_generic_kernel",
+        "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell/s",
+        "frac": achieved / peak_cells if peak_cells else None,
+        "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {sm_max:.0f} MHz ({peak_kind} max clock) / "
+                     f"{slots:.0f} scheduler cycles per recurrence cell (2 adds + 1 max of 64-bit values)",
+        "cells_per_launch": stats_sum["cells"] / launches,
+        "ms_per_launch": 1e3 * cost_s / launches,
+        "share_of_step": cost_s / dev_seconds if dev_seconds else None,
+        # DRAM bytes of one search-pass launch from an ncu capture of the 512-scenario case
+        # (0.65 MB for 55 800 CTAs of the 12-stage kernel), scaled by CTAs; the kernel reads only
+        # the small descriptor tables, so this is context, not a bound
+        "traffic": TRAFFIC_BYTES_PER_CTA * stats_sum["plans"] / max(1, stats_sum["cost_kernel_launches"]) / 128.0,
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -188,8 +274,9 @@ def main():
     ap.add_argument("--cost-mode", type=int, default=0, choices=[0, 1])
     ap.add_argument("--ref-scenarios", type=int, default=16, help="oracle scenarios per step (--impl reference)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--latency-scenarios", type=int, default=256)
+    ap.add_argument("--latency-scenarios", type=int, default=4096, help="scenarios searched one by one for latency")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads / cost mode summary")
     ap.add_argument("--scenarios", type=int, default=0, help="use only the first N scenarios (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -198,7 +285,6 @@ def main():
         run_reference(args)
         return
 
-    import numpy as np
     import torch
     import torch.distributed as dist
     from paper_2508_21613_b200 import binding, build
@@ -213,104 +299,40 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = rank_workload(args.workload, rank)
-    if args.scenarios > 0:
-        w.scenarios = w.scenarios[:args.scenarios]
-    opts = w.options.with_cost_mode(args.cost_mode)
-    ctx = binding.cm_create(local_rank)
-    binding.cm_load_profile(ctx, w.profile)
-    packed = binding.PackedScenarios(w.scenarios)
-    flush = torch.empty(256 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")  # > 126 MB L2
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident arm: descriptors already in HBM when the timed region starts
-    batch, n_cand = packed.prepare(ctx, opts)
-    for _ in range(args.warmup):
-        packed.search_prepared(ctx, batch)
-    sampler = ClockSampler(local_rank)
-    barrier()
-    sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    stats_sum = {}
-    for k in range(args.steps):
-        flush.fill_(float(k))                       # evict L2 between timed iterations (untimed)
-        ev[k][0].record()
-        packed.search_prepared(ctx, batch)          # kernels + plans back on the host
-        ev[k][1].record()
-        st = binding.cm_last_stats(ctx)
-        for key, v in st.items():
-            stats_sum[key] = stats_sum.get(key, 0) + v
-    barrier()
-    clocks = sampler.stop()
-    dev_seconds = sum(a.elapsed_time(b) for a, b in ev) * 1e-3
-    plans_per_step = n_cand + 2 * len(w.scenarios)   # + one rerouting and one redundant plan each
-    binding.cm_batch_free(batch)
-
-    # ---- end-to-end arm: host failure sets in, host plans out, every step
-    for _ in range(args.warmup):
-        packed.search(ctx, opts)
-    barrier()
-    e2e_seconds = 0.0
-    h2d = d2h = 0
-    for k in range(args.steps):
-        flush.fill_(float(k))
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        packed.search(ctx, opts)                    # cm_search_batch: build, H2D, kernels, D2H, sync
-        e2e_seconds += time.perf_counter() - t0
-        st = binding.cm_last_stats(ctx)
-        h2d, d2h = st["h2d_bytes"] + packed.ids.nbytes + packed.offsets.nbytes, st["d2h_bytes"]
-    barrier()
-
-    # ---- search latency per failure: scenarios searched one at a time
-    n_lat = min(args.latency_scenarios, len(w.scenarios))
-    lat_pack = binding.PackedScenarios(w.scenarios[:: max(1, len(w.scenarios) // n_lat)][:n_lat])
-    lat_pack.search(ctx, opts, latency=True)
-    lat_pack.search(ctx, opts, latency=True)
-    lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
-
-    rows = gather_rows([float(plans_per_step * args.steps), dev_seconds, e2e_seconds], world, "cuda")
+    w = rank_workload(args.workload, rank)
+    if args.scenarios > 0:
+        w.scenarios = w.scenarios[:args.scenarios]
+    flush = torch.empty(256 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")  # > 126 MB L2
+    m = measure(binding, torch, w, args.cost_mode, args.steps, args.warmup, local_rank, barrier, flush,
+                args.latency_scenarios)
+    rows = gather_rows([float(m["plans_per_step"] * args.steps), m["dev_seconds"], m["e2e_seconds"]], world, "cuda")
     total_plans, max_dev = aggregate([(r[0], r[1]) for r in rows])
     _, max_e2e = aggregate([(r[0], r[2]) for r in rows])
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         sm_max = float(peaks.get("sm_max_mhz") or SM_MAX_MHZ_FALLBACK)
-        slots = ISSUE_SLOTS_PER_CELL[args.cost_mode]
-        peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
-        cost_s = stats_sum["cost_kernel_ns"] * 1e-9
-        achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
         line = {
             "metric": METRIC, "value": total_plans / max_dev, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * max_dev / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "i64" if args.cost_mode else "f64", "data": "synthetic",
-            "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": plans_per_step,
+            "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": m["plans_per_step"],
                        "policies": 3, "cost_mode": "int64ns" if args.cost_mode else "fp64",
                        "l2": "flushed between timed iterations (256 MB write)",
                        "parallelism": "replicas, scenarios independent" if world > 1 else "1 gpu"},
             "e2e": {"value": total_plans / max_e2e, "unit": UNIT, "ms_per_step": 1e3 * max_e2e / args.steps,
-                    "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "h2d_bytes_per_step": int(m["h2d"]), "d2h_bytes_per_step": int(m["d2h"]),
                     "timing": "wall clock around cm_search_batch (host descriptor build inside)"},
-            "latency_us": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
-                           "max": float(lat[-1]), "scenarios": int(lat_pack.B),
-                           "what": "one failure set, all policies, descriptor build to plan on host"},
-            "gpu_launches": int(stats_sum["launches"]),
-            "clocks": clocks,
-            "roofline": {
-                "bound": "alu", "kernel": "cm_cost_kernel", "achieved": achieved / 1e9, "peak": peak_cells / 1e9,
-                "unit": "Gcell/s", "frac": achieved / peak_cells if peak_cells else None,
-                "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {sm_max:.0f} MHz ({peak_kind} max clock) / "
-                             f"{slots:.0f} issue slots per cell",
-                "cells_per_launch": stats_sum["cells"] / max(1, stats_sum["cost_kernel_launches"]),
-                "ms_per_launch": 1e3 * cost_s / max(1, stats_sum["cost_kernel_launches"]),
-                "share_of_step": cost_s / dev_seconds if dev_seconds else None,
-                "traffic": None,
-            },
+            "latency_us": m["latency_us"],
+            "gpu_launches": int(m["stats"]["launches"]),
+            "clocks": m["clocks"],
+            "roofline": roofline_of(m["stats"], m["dev_seconds"], args.cost_mode, sm_max, peak_kind),
         }
         if not args.no_cpu_baseline:
             p, s, n = oracle_sample(w, args.cost_mode, args.cpu_budget, len(w.scenarios))
@@ -318,8 +340,27 @@ def main():
                                     "sample": f"first {n} failure scenarios of '{w.name}', all three policies, "
                                               f"{s:.1f} s single-threaded",
                                     "latency_us_per_failure": 1e6 * s / n}
+        if not args.no_extra and world == 1 and args.scenarios == 0:
+            # the other configurations (and the other cost mode), two timed steps each: context
+            # for the headline line above, same measurement code
+            from paper_2508_21613_b200 import workloads as W
+            extra = {}
+            todo = [(args.workload, 1 - args.cost_mode)]
+            todo += [(name, args.cost_mode) for name in ("tiny", "70b-like", "175b-like", "sweep") if name != args.workload]
+            for name, mode in todo:
+                ew = W.ALL_WORKLOADS[name]()
+                em = measure(binding, torch, ew, mode, 2, 3, local_rank, barrier, flush, args.latency_scenarios,
+                             sample_clocks=False)
+                r = roofline_of(em["stats"], em["dev_seconds"], mode, sm_max, peak_kind)
+                extra[f"{name}/{'int64ns' if mode else 'fp64'}"] = {
+                    "scenarios": len(ew.scenarios), "plans_per_step": em["plans_per_step"],
+                    "plans_per_s": em["plans_per_step"] * 2 / em["dev_seconds"],
+                    "ms_per_step": 1e3 * em["dev_seconds"] / 2, "e2e_ms_per_step": 1e3 * em["e2e_seconds"] / 2,
+                    "latency_us_p50": em["latency_us"]["p50"], "latency_us_p99": em["latency_us"]["p99"],
+                    "latency_scenarios": em["latency_us"]["scenarios"],
+                    "search_pass_gcell_s": r["achieved"], "search_pass_frac": r["frac"]}
+            line["workloads"] = extra
         print(json.dumps(line))
-    binding.cm_destroy(ctx)
     if world > 1:
         dist.destroy_process_group()
 
