@@ -9,8 +9,9 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libchameleon.so")
-SOURCES = ["cm_api.cu", "cm_kernels.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu"]
-HEADERS = ["cm_internal.h", "cm_device.cuh", "cm_plan_eval.cuh"]
+SOURCES = ["cm_cost_deep_f64.cu", "cm_cost_deep_i64.cu", "cm_cost_shallow_f64.cu", "cm_cost_shallow_i64.cu",
+           "cm_kernels.cu", "cm_api.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu"]
+HEADERS = ["cm_internal.h", "cm_device.cuh", "cm_plan_eval.cuh", "cm_cost_impl.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
@@ -32,8 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objs = []
-    for src in SOURCES:
+
+    def compile_one(src: str) -> str:
         obj = os.path.join(_CSRC, src.replace(".cu", ".o"))
         cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"), "-I", _CSRC,
                "-c", os.path.join(_CSRC, src), "-o", obj]
@@ -41,7 +42,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
         subprocess.check_call(cmd)
-        objs.append(obj)
+        return obj
+
+    # the translation units are independent: compile them side by side (the four
+    # cm_cost_* units hold the hundred-odd kernel instantiations and take longest)
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=max(1, min(len(SOURCES), os.cpu_count() or 1))) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
     tmp = LIB_PATH + f".tmp{os.getpid()}"
     subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
                            "-o", tmp, *objs])

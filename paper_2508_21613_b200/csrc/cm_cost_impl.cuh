@@ -1,0 +1,444 @@
+// Search pass of the plan search (sm_100a): every pipeline-plan of every segment ->
+// least cost per segment.  This is the hot kernel: 2 * stages * micro-batches
+// recurrence cells per plan (Section "Estimator", the start/end transition equation;
+// the paper puts the estimator at O(N_pp x N_m) per asymmetric pipeline).
+//
+// Work layout: segments with the same (stages S, micro-batches m) are bucketed, so all
+// lanes of a warp run recurrences of the same shape.  Three kernels share one evaluation
+// order (sim_rounds below):
+//
+//   cm_cost_regs_kernel<T, S>       S = 1..16, m >= S-1.  One thread per plan, everything in
+//       registers: stage forward/backward/transfer times, per-stage clock and pending
+//       forward; every loop over stages is unrolled, so a cell costs its two adds and one
+//       max and nothing else.
+//   cm_cost_wide_kernel<T, S, UNI>  S = 17..48.  Clock and pending forward stay in
+//       registers (4 S of them), the stage times move to shared memory.
+//       UNI = true ("transposed"): the 32 lanes of a warp take the SAME layer composition
+//       in 32 DIFFERENT segments of the bucket (they differ in link tiers and sync
+//       peers only), so stage times are warp-uniform -- one broadcast 16-byte load per
+//       stage and round -- and memory feasibility is decided once per warp.
+//       UNI = false: one plan per lane as in the register kernel, stage times in a
+//       per-lane shared-memory column; for buckets with too few segments to transpose.
+//   cm_cost_generic_kernel<T>       any S <= CM_MAX_STAGES: per-stage state in local memory.
+#pragma once
+
+#include "cm_plan_eval.cuh"
+
+namespace cm {
+
+
+// Bucket that owns a chunk: the last bucket of the class whose first chunk is not above it.
+__device__ __forceinline__ uint32_t find_bucket(const Bucket *bk, uint32_t b0, uint32_t b1, uint64_t chunk) {
+    uint32_t lo = b0, hi = b1 - 1;
+    while (lo < hi) {
+        uint32_t mid = (lo + hi + 1) >> 1;
+        if (bk[mid].chunk_first <= chunk) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// (segment-in-bucket, kappa) of plan `tid` of a chunk whose first plan is `base`
+// (plan-major buckets: index = segment-in-bucket * count + kappa).
+__device__ __forceinline__ void plan_of_thread(uint64_t base, uint64_t count, uint32_t tid,
+                                               uint64_t &seg_local, uint64_t &kappa) {
+    const uint64_t seg0 = base / count, rem0 = base - seg0 * count;
+    if (count > (uint64_t)kChunk) {
+        const uint64_t x = rem0 + tid;
+        const bool wrap = x >= count;
+        seg_local = seg0 + (wrap ? 1 : 0);
+        kappa = wrap ? x - count : x;
+    } else {
+        const uint32_t x = (uint32_t)rem0 + tid, c = (uint32_t)count;
+        const uint32_t q = x / c;
+        seg_local = seg0 + q;
+        kappa = x - q * c;
+    }
+}
+
+// Segment number `seg_local` of a bucket = (template segment of the bucket, scenario of the
+// template), scenario minor.
+__device__ __forceinline__ SegView bucket_segment(const BatchDev &bd, const Bucket &bk, uint32_t seg_local) {
+    const Tmpl &tp = bd.tmpl[bk.tmpl];
+    const uint32_t ti = seg_local / tp.n_scen, si = seg_local - ti * tp.n_scen;
+    return seg_view(bd, bd.tmpl_scen[tp.scen_first + si], bd.bucket_tseg[bk.list_first + ti]);
+}
+
+// Least cost per segment from per-lane (segment row, cost bits): lanes of one segment
+// are contiguous, so a segmented shuffle scan leaves each run's minimum in its last lane,
+// which issues the one atomicMin.
+__device__ __forceinline__ void segmented_min_commit(uint64_t *seg_best, uint32_t row, uint64_t bits, uint64_t inf) {
+    const uint32_t lane = threadIdx.x & 31;
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint64_t ov = __shfl_up_sync(0xffffffffu, bits, o);
+        const uint32_t orow = __shfl_up_sync(0xffffffffu, row, o);
+        if (lane >= (uint32_t)o && orow == row && ov < bits) bits = ov;
+    }
+    const uint32_t next_row = __shfl_down_sync(0xffffffffu, row, 1);
+    const bool last = lane == 31 || next_row != row;
+    if (last && row != 0xffffffffu && bits < inf) atomicMin((unsigned long long *)&seg_best[row], (unsigned long long)bits);
+}
+
+__device__ __forceinline__ void count_cells(unsigned long long *counter, unsigned long long my_cells,
+                                            unsigned long long *smem /* [kChunk/32] */) {
+    for (int o = 16; o > 0; o >>= 1) my_cells += __shfl_xor_sync(0xffffffffu, my_cells, o);
+    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = my_cells;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long c = 0;
+        for (int w = 0; w < kChunk / 32; ++w) c += smem[w];
+        if (c) atomicAdd(counter, c);
+    }
+}
+
+// ----------------------------------------------------------------------------------
+// S <= 16: one thread per plan, all in registers.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1,
+                                                              uint64_t chunk_offset) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T cost;
+        if (plan_cost_regs<T, S>(sp, tb, bd.layer_mode, g, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * S * g.m;
+        }
+    }
+    segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+// Every shallow depth in one launch: for batches so small that a launch per depth would
+// cost more than the work (a single failure scenario of a 32-device job is ~250 CTAs).
+template <typename T>
+__global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    const uint64_t chunk = (uint64_t)blockIdx.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T cost;
+        if (plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * g.S * g.m;
+        }
+    }
+    segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+// ----------------------------------------------------------------------------------
+// 16 < S <= 48: stage times in shared memory.
+// Dynamic shared memory:  UNI:  FB<T> fb[4 warps][S] | T xt[S][128] | uint8 cuts[4][S+1]
+//                         !UNI: FB<T> fb[S][128]     | T xt[S][128]
+// ----------------------------------------------------------------------------------
+#ifndef CM_WIDE3
+#define CM_WIDE3 34   // deepest pipeline compiled for three resident CTAs per SM (<= 168 registers)
+#endif
+template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
+    return UNI ? sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8)
+               : sizeof(FB<T>) * S * kChunk + sizeof(T) * S * kChunk;
+}
+
+template <typename T, int S, bool UNI>
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const int m = bk.m, L = sp.L;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    unsigned long long my_cells = 0;
+
+    if (UNI) {
+        FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+        uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
+        // warp item = (kappa, group of 32 segments), group minor
+        const uint64_t item = (chunk - bk.chunk_first) * (kChunk / 32) + warp;
+        const uint32_t n_groups = (bk.n_seg + 31) / 32;
+        const uint64_t kappa = item / n_groups;
+        const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
+        if (kappa < bk.count && m >= 1) {           // warp-uniform
+            const bool active = seg_local < bk.n_seg;
+            const SegView g = bucket_segment(bd, bk, active ? seg_local : 0);
+            const uint32_t row = g.row;
+            const uint64_t tier = g.tier;
+            const int n_sync = g.n_sync;
+            // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
+            CutWalker cw;
+            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
+            if (ok) {
+                int lo = 0;
+                for (int i = 0; i < S; ++i) {
+                    const int hi = cw.next();
+                    ok = ok && hi > lo;
+                    if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+                    lo = hi;
+                }
+                if (lane == 0) cuts[0] = 0;
+            }
+            __syncwarp();
+            long long g_max = 0;
+            if (ok) {
+                // stage sums and the memory check, one stage per lane
+                for (int i = lane; i < S; i += 32) {
+                    const int lo = cuts[i], hi = cuts[i + 1];
+                    ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                    FB<T> d;
+                    d.f = sp.PF[hi] - sp.PF[lo];
+                    d.b = sp.PB[hi] - sp.PB[lo];
+                    fb[i] = d;
+                    const long long gb = sp.PP[hi] - sp.PP[lo];
+                    g_max = gb > g_max ? gb : g_max;
+                }
+                for (int o = 16; o > 0; o >>= 1) {
+                    const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+                    g_max = og > g_max ? og : g_max;
+                }
+                // transfer times of this lane's segment (its own link tiers)
+                for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(tier >> i) & 1ull][cuts[i + 1] - 1];
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            __syncwarp();
+            if (ok) {
+                const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+                if (active) {
+                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync));
+                    if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
+                    my_cells = 2ull * S * m;
+                }
+            }
+        }
+    } else {
+        FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + tid;                               // [i * kChunk]
+        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + tid;           // [i * kChunk]
+        const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+        uint64_t seg_local, kappa;
+        plan_of_thread(base, bk.count, tid, seg_local, kappa);
+        uint32_t row = 0xffffffffu;
+        uint64_t bits = inf_bits<T>();
+        if (seg_local < bk.n_seg && m >= 1) {
+            const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+            row = g.row;
+            T cost;
+            if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost)) {
+                bits = Num<T>::bits(cost);
+                my_cells = 2ull * S * m;
+            }
+        }
+        segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    }
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb.prof);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T cost;
+        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
+            bits = Num<T>::bits(cost);
+            my_cells = 2ull * g.S * g.m;
+        }
+    }
+    segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
+static dim3 chunk_grid(uint64_t n) {
+    const uint64_t maxx = 1u << 30;
+    if (n <= maxx) return dim3((unsigned)n, 1, 1);
+    return dim3((unsigned)maxx, (unsigned)((n + maxx - 1) / maxx), 1);
+}
+
+template <typename T, int S>
+static cudaError_t launch_regs(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    cm_cost_regs_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    return cudaGetLastError();
+}
+
+template <typename T, int S, bool UNI>
+static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, UNI, T>();
+    static bool configured[16] = {false};   // per device; the attribute sticks to the function
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 16 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(cm_cost_wide_kernel<T, S, UNI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    return cudaGetLastError();
+}
+
+template <typename T, int S>
+static cudaError_t launch_wide(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : launch_wide_one<T, S, false>(t, b, c, st);
+}
+
+
+// ---------------------------------------------------------------------------------
+// Launchers per cost type.  They are explicitly instantiated in four translation units
+// (shallow / deep x fp64 / int64) so that the hundred-odd kernel instantiations compile
+// side by side; cm_cost.cu only dispatches.
+// ---------------------------------------------------------------------------------
+template <typename T>
+cudaError_t launch_shallow_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    switch (c.stages) {
+#define CM_CASE(S) case S: return launch_regs<T, S>(t, b, c, st);
+        CM_CASE(1) CM_CASE(2) CM_CASE(3) CM_CASE(4) CM_CASE(5) CM_CASE(6) CM_CASE(7) CM_CASE(8)
+        CM_CASE(9) CM_CASE(10) CM_CASE(11) CM_CASE(12) CM_CASE(13) CM_CASE(14) CM_CASE(15) CM_CASE(16)
+#undef CM_CASE
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+template <typename T>
+cudaError_t launch_shallow_any(const Tables &t, const BatchDev &b, uint32_t b0, uint32_t b1, uint64_t chunks, cudaStream_t st) {
+    cm_cost_regs_any_kernel<T><<<(unsigned)chunks, kChunk, 0, st>>>(t, b, b0, b1);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_generic_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_deep_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    switch (c.stages) {
+#define CM_CASE(S) case S: return launch_wide<T, S>(t, b, c, st);
+        CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
+        CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
+        CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
+        CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
+#undef CM_CASE
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+// ----------------------------------------------------------------------------------
+// Tie-break pass for the winners' deep pipelines (17..48 stages): the lowest layer
+// composition that is feasible with cost <= T*.  Same grid as the generic tie-break
+// kernel -- x = (scenario, pipeline), y = tiles of kChunk compositions -- one launch per
+// stage count; CTAs whose winner segment has another depth leave at once.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_wide_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ uint64_t red[kChunk / 32];
+    __shared__ SegView g;
+    __shared__ uint64_t found_so_far;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint32_t b = blockIdx.x / bd.dp_max, p = blockIdx.x % bd.dp_max;
+    const Winner &w = bd.winner[b];
+    if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;            // uniform over the CTA
+    if (bd.tseg[w.seg[p]].S != S) return;
+    stage_profile(sp, tb.prof);
+    FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + threadIdx.x;
+    T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + threadIdx.x;
+    uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
+    for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            g = seg_view(bd, b, w.seg[p]);
+            found_so_far = *(volatile uint64_t *)slot;
+        }
+        __syncthreads();
+        const uint64_t count = g.K ? g.K + 1 : 1;
+        const uint64_t first = tile * kChunk;
+        if (first >= count || found_so_far < first) break;              // uniform: later tiles cannot win either
+        const uint64_t kappa = first + threadIdx.x;
+        uint64_t hit = ~0ull;
+        if (kappa < count) {
+            T cost;
+            if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost) &&
+                Num<T>::bits(cost) <= w.cost_bits)
+                hit = kappa;
+        }
+        hit = warp_min_u64(hit);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = hit;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int q = 0; q < kChunk / 32; ++q) hit = red[q] < hit ? red[q] : hit;
+            if (hit != ~0ull) atomicMin((unsigned long long *)slot, (unsigned long long)hit);
+            const uint64_t n = count - first < (uint64_t)kChunk ? count - first : (uint64_t)kChunk;
+            atomicAdd(&bd.counters[1], (unsigned long long)n);
+        }
+    }
+}
+
+template <typename T, int S>
+static cudaError_t launch_tiebreak_wide_one(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, false, T>();
+    static bool configured[16] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 16 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(cm_tiebreak_wide_kernel<T, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const uint64_t nx = (uint64_t)b.B * b.dp_max;
+    if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)nx, tiebreak_grid_y(nx, b.max_tiles_per_seg), 1);
+    cm_tiebreak_wide_kernel<T, S><<<grid, kChunk, smem, st>>>(t, b);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_tiebreak_deep(const Tables &t, const BatchDev &b, int S, cudaStream_t st) {
+    switch (S) {
+#define CM_CASE(S) case S: return launch_tiebreak_wide_one<T, S>(t, b, st);
+        CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
+        CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
+        CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
+        CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
+#undef CM_CASE
+    default: return cudaSuccess;
+    }
+}
+
+}  // namespace cm
