@@ -198,3 +198,37 @@ def test_integer_and_double_builds_agree_on_integer_inputs(oracle_factory):
             b = oracle_factory(prof, None).pipe(cuts, n_m, devs, n_sync, 1)
             assert a[0] and b[0]
             assert a[1] == float(b[2])
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_transfer_and_sync_terms_on_a_two_stage_pipeline(oracle_factory, mode):
+    """S=2, m=1 has a single path: F0, transfer, F1, B1, transfer, B0 -- so the pipeline
+    time is their plain sum, and the step adds the slower stage's gradient all-reduce
+    (ring lower bound 2(n-1)/n * bytes / bandwidth, a textbook figure).  Pins that the
+    transfer is paid in both directions, that the link tier follows the two devices'
+    nodes, and which bandwidth the synchronisation uses."""
+    L, dpn = 4, 4
+    fwd = [1000.0, 3000.0, 5000.0, 7000.0]
+    bwd = [2000.0, 6000.0, 10000.0, 14000.0]
+    par = [4 * 3 * 5 * 1000, 8 * 3 * 5 * 1000, 1000 * 3 * 5, 1000 * 3 * 5]
+    p2p = [0, 600 * 20 * 7, 0, 0]                      # the cut sits after layer 1
+    prof = W.make_profile_ns(L, 3, 2, 1, fwd, bwd, 0, par, [6 * v for v in par], p2p, [0, 2, 4],
+                             10**15, dpn, 600, 20)
+    o = oracle_factory(prof, None)
+    F0, F1, B0, B1 = 4000.0, 12000.0, 8000.0, 24000.0
+    g0 = par[0] + par[1]                               # stage 0 holds the larger gradients
+    for devs, bw in (([0, 1], 600), ([3, 4], 20), ([4, 3], 20), ([5, 6], 600)):
+        xt = p2p[1] / bw                               # exact: 600*20*7 divides by both tiers
+        for n_sync in (1, 3):
+            # 6 devices > 4 per node: the job spans nodes, sync runs on the inter-node tier
+            sync = 0.0 if n_sync == 1 else 2 * (n_sync - 1) * g0 / (n_sync * 20)
+            assert sync == int(sync)
+            ok, cost, cost_ns, _ = o.pipe([0, 2, 4], 1, devs, n_sync, mode)
+            want = F0 + xt + F1 + B1 + xt + B0 + sync
+            assert ok and (cost_ns == int(want) if mode else cost == want)
+    # a job inside one node synchronises over the intra-node tier
+    prof1 = W.make_profile_ns(L, 2, 2, 1, fwd, bwd, 0, par, [6 * v for v in par], p2p, [0, 2, 4],
+                              10**15, dpn, 600, 20)
+    ok, cost, cost_ns, _ = oracle_factory(prof1, None).pipe([0, 2, 4], 1, [0, 1], 2, mode)
+    want = F0 + F1 + B1 + B0 + 2 * p2p[1] / 600 + 2 * 1 * g0 / (2 * 600)
+    assert ok and (cost_ns == int(want) if mode else cost == want)
