@@ -82,7 +82,6 @@ struct Batch {
     std::vector<Bucket> bucket;
     std::vector<LaunchClass> classes;
     std::vector<int> tmpl_of_nsurv;        // survivor count -> template, -1 = not built
-    std::vector<uint16_t> strategies;      // scratch: flattened stage-count tuples
     PinnedVec<unsigned char> arena;        // host image of the tables
     DevBuf<unsigned char> d_arena;
     size_t off_scen = 0, off_tmpl = 0, off_strat = 0, off_tseg = 0, off_failed = 0, off_red = 0, off_keys = 0,
@@ -99,7 +98,6 @@ struct Batch {
     uint64_t n_rows = 0;                   // rows of seg_best over all scenarios
     uint32_t max_tiles_per_seg = 0, dp_max = 0;
     int B = 0;
-    bool uploaded = false;
 };
 
 struct cm_ctx {
@@ -368,7 +366,6 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.max_tiles_per_seg = 0;
     bt.dp_max = 0;
     bt.B = B;
-    bt.uploaded = false;
     bt.tmpl_of_nsurv.assign((size_t)N + 1, -1);
     bt.tmpl.push_back(Tmpl{});   // template 0: no strategies (scenarios without a dynamic-parallelism search)
     const int cross_words = (N + 63) / 64 + 1;
@@ -469,7 +466,7 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
     v.counters = reinterpret_cast<unsigned long long *>(bt.d_seg_best.p + bt.n_rows);
     v.B = bt.B; v.mode = bt.opts.cost;
-    v.n_rows = (uint32_t)bt.n_rows; v.n_strat = (uint32_t)bt.strat.size();
+    v.n_rows = (uint32_t)bt.n_rows;
     v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
     v.n_red_blocks = (uint32_t)bt.red_scen.size(); v.dp_max = bt.dp_max;
     v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
@@ -514,7 +511,6 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
                                    (int)bt.keys.size(), bt.opts.cost, ctx->stream));
         if (launches) ++*launches;
     }
-    bt.uploaded = true;
     return CM_OK;
 }
 

@@ -14,7 +14,7 @@ constexpr int kMaxL = CM_MAX_LAYERS;
 constexpr int kMaxS = CM_MAX_STAGES;
 constexpr int kMaxP = CM_MAX_PIPES;
 constexpr int kBinomCols = 64;          // binomial table columns 0..64
-constexpr int kTile = 128;              // candidates per CTA in the generic cost kernel
+constexpr int kTile = 128;              // layer compositions per CTA in the tie-break kernels
 constexpr uint64_t kSat = ~0ull;        // saturated binomial
 
 // Per-layer prefix arrays, built on the device by cm_prefix_kernel and staged into shared
@@ -143,7 +143,7 @@ struct BatchDev {
     cm_plan *plans;         // [B][4]: per policy, then the overall best
     unsigned long long *counters;  // [0] cells simulated in pass 1, [1] plans in pass 2
     int32_t B, mode;
-    uint32_t n_rows, n_strat;    // rows of seg_best over all scenarios
+    uint32_t n_rows, pad0;       // rows of seg_best over all scenarios
     uint64_t n_tiles;
     uint32_t max_tiles_per_seg, n_red_blocks;
     uint32_t dp_max, pad;
