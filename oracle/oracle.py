@@ -1,7 +1,7 @@
 """ctypes front end of the CPU oracle -- TEST INFRASTRUCTURE, not the product.
 
 Only ``tests/``, the smoke check and the bench's CPU-baseline leg may import this
-module.  It compiles ``orc_enum.c`` and ``orc_model.c`` (the latter twice: double and
+module.  It compiles ``orc_enum.c``, ``orc_restore.c`` and ``orc_model.c`` (the latter twice: double and
 integer-nanosecond arithmetic) with gcc into ``liborc.so`` next to the sources and
 exposes the entry points.  Nothing here touches CUDA and nothing in the CUDA path
 imports this.
@@ -18,7 +18,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liborc.so")
-_SOURCES = ["orc_enum.c", "orc_model.c", "orc.h"]
+_SOURCES = ["orc_enum.c", "orc_restore.c", "orc_model.c", "orc.h"]
 
 MAX_PIPES = 16
 MAX_STAGES = 64
@@ -35,9 +35,9 @@ def build(force: bool = False) -> str:
     flags = ["-O2", "-fPIC", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-Wall",
              "-Wno-maybe-uninitialized"]
     objs = []
-    for name, defs in (("orc_enum", []), ("orc_model_f64", ["-DORC_INT=0"]),
+    for name, defs in (("orc_enum", []), ("orc_restore", []), ("orc_model_f64", ["-DORC_INT=0"]),
                        ("orc_model_i64", ["-DORC_INT=1"])):
-        src = os.path.join(_HERE, "orc_enum.c" if name == "orc_enum" else "orc_model.c")
+        src = os.path.join(_HERE, name + ".c" if not defs else "orc_model.c")
         obj = os.path.join(_HERE, name + ".o")
         subprocess.check_call(["gcc", *flags, *defs, "-c", src, "-o", obj])
         objs.append(obj)
@@ -68,6 +68,32 @@ class _Plan(C.Structure):
                 ("cost_ns", C.c_int64), ("strategy", C.c_uint32), ("n_pipes", C.c_uint32),
                 ("split_rank", C.c_uint64), ("stages", C.c_uint16 * MAX_PIPES),
                 ("micro", C.c_uint16 * MAX_PIPES), ("kappa", C.c_uint64 * MAX_PIPES)]
+
+
+class _Objective(C.Structure):
+    _fields_ = [("topk", C.c_int32), ("pad", C.c_int32), ("t_gap", C.c_double), ("t_restart", C.c_double),
+                ("t_gap_ns", C.c_int64), ("t_restart_ns", C.c_int64), ("bw_xfer", C.c_int64)]
+
+
+class _Transition(C.Structure):
+    _fields_ = [("policy", C.c_int32), ("feasible", C.c_int32), ("rank", C.c_int32), ("n_surv", C.c_int32),
+                ("xfer_bytes", C.c_int64), ("t_trans", C.c_double), ("t_trans_ns", C.c_int64),
+                ("objective", C.c_double)]
+
+
+@dataclass
+class Transition:
+    policy: int
+    feasible: bool
+    rank: int
+    n_surv: int
+    xfer_bytes: int
+    t_trans: float
+    t_trans_ns: int
+    objective: float
+    assign: Tuple[int, ...] = ()
+    shortlist: Tuple = ()
+    shortlist_bytes: Tuple[int, ...] = ()
 
 
 @dataclass
@@ -108,9 +134,12 @@ class Oracle:
         self._lib.orc_rank_subset.restype = C.c_uint64
         self._lib.orc_split_count.restype = C.c_uint64
         self._lib.orc_layer_count.restype = C.c_uint64
+        self._lib.orc_assign.restype = C.c_int64
+        self._lib.orc_assign_brute.restype = C.c_int64
         for sfx in ("_f64", "_i64"):
             getattr(self._lib, "orc_pipe_time" + sfx).restype = C.c_double
             getattr(self._lib, "orc_count" + sfx).restype = C.c_uint64
+            getattr(self._lib, "orc_plan_transfer" + sfx).restype = C.c_int64
         self.profile = profile
         self.options = options
         p = profile
@@ -273,13 +302,86 @@ class Oracle:
         ok = self._fn("orc_search", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(best), per)
         return (_plan_from(best) if ok else None), [_plan_from(per[i]) for i in range(3)]
 
-    def decode(self, failed: Sequence[int], plan: Plan, options=None) -> List[List[int]]:
-        o, sfx = self._opts(options)
-        _, fp, nf = self._failed(failed)
+    @staticmethod
+    def _cplan(plan: Plan) -> _Plan:
         c = _Plan(plan.policy, int(plan.feasible), plan.cost, plan.cost_ns, plan.strategy, plan.n_pipes,
                   plan.split_rank)
         for i in range(plan.n_pipes):
             c.stages[i], c.micro[i], c.kappa[i] = plan.stages[i], plan.micro[i], plan.kappa[i]
+        return c
+
+    # -- weight transfer, full objective ------------------------------------------
+    def state_bytes(self) -> np.ndarray:
+        """Bytes of model state per layer that a migration moves (parameters + optimizer)."""
+        return np.asarray(self.profile.param_bytes, dtype=np.int64) + np.asarray(self.profile.opt_bytes, dtype=np.int64)
+
+    def transfer_cost_matrix(self, old: Sequence[Tuple[int, int]], new: Sequence[Tuple[int, int]],
+                             weights: Optional[Sequence[int]] = None) -> np.ndarray:
+        """Cost[i][j] of device i (old layer range) serving position j (new layer range)."""
+        n = len(old)
+        w = np.ascontiguousarray(self.state_bytes() if weights is None else weights, dtype=np.int64)
+        olo = np.ascontiguousarray([a for a, _ in old], dtype=np.int32)
+        ohi = np.ascontiguousarray([b for _, b in old], dtype=np.int32)
+        nlo = np.ascontiguousarray([a for a, _ in new], dtype=np.int32)
+        nhi = np.ascontiguousarray([b for _, b in new], dtype=np.int32)
+        cost = np.zeros((n, n), dtype=np.int64)
+        self._lib.orc_transfer_cost_matrix(len(w), _ptr(w, C.c_int64), n, _ptr(olo, C.c_int32), _ptr(ohi, C.c_int32),
+                                           _ptr(nlo, C.c_int32), _ptr(nhi, C.c_int32), _ptr(cost, C.c_int64))
+        return cost
+
+    def assign(self, cost: np.ndarray) -> Tuple[int, List[int]]:
+        """Minimum-cost perfect matching -> (total, row matched to every column)."""
+        c = np.ascontiguousarray(cost, dtype=np.int64)
+        n = c.shape[0]
+        out = np.zeros(max(n, 1), dtype=np.int32)
+        total = self._lib.orc_assign(n, _ptr(c, C.c_int64), _ptr(out, C.c_int32))
+        return int(total), [int(x) for x in out[:n]]
+
+    def assign_brute(self, cost: np.ndarray) -> int:
+        c = np.ascontiguousarray(cost, dtype=np.int64)
+        return int(self._lib.orc_assign_brute(c.shape[0], _ptr(c, C.c_int64)))
+
+    def plan_transfer(self, failed: Sequence[int], plan: Plan, options=None) -> Tuple[int, List[int]]:
+        """Bytes moved by the cheapest migration into ``plan`` and its matching."""
+        o, sfx = self._opts(options)
+        _, fp, nf = self._failed(failed)
+        n_surv = self.profile.n_dp * self.profile.n_pp - nf
+        out = np.zeros(max(n_surv, 1), dtype=np.int32)
+        c = self._cplan(plan)
+        b = self._fn("orc_plan_transfer", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(c), _ptr(out, C.c_int32))
+        return int(b), [int(x) for x in out[:n_surv]]
+
+    def search_objective(self, failed: Sequence[int], objective, options=None):
+        """Full-objective search -> (best plan or None, Transition).
+
+        ``objective`` carries topk, t_gap_ns, t_restart_ns (floats; rounded for the integer
+        build) and bw_xfer_Bpns."""
+        o, sfx = self._opts(options)
+        _, fp, nf = self._failed(failed)
+        k = max(1, int(objective.topk))
+        q = _Objective(k, 0, float(objective.t_gap_ns), float(objective.t_restart_ns),
+                       int(round(objective.t_gap_ns)), int(round(objective.t_restart_ns)),
+                       int(objective.bw_xfer_Bpns))
+        n_surv = self.profile.n_dp * self.profile.n_pp - nf
+        best, tr = _Plan(), _Transition()
+        asg = np.zeros(max(n_surv, 1), dtype=np.int32)
+        sp = (_Plan * k)()
+        sb = np.zeros(k, dtype=np.int64)
+        ns = C.c_int32()
+        ok = self._fn("orc_search_objective", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(q),
+                                                   C.byref(best), C.byref(tr), _ptr(asg, C.c_int32), sp,
+                                                   _ptr(sb, C.c_int64), C.byref(ns))
+        t = Transition(tr.policy, bool(tr.feasible), tr.rank, tr.n_surv, tr.xfer_bytes, tr.t_trans, tr.t_trans_ns,
+                       tr.objective,
+                       tuple(int(x) for x in asg[:n_surv]) if (ok and tr.policy == DYNPAR) else (),
+                       tuple(_plan_from(sp[i]) for i in range(ns.value)),
+                       tuple(int(x) for x in sb[:ns.value]))
+        return (_plan_from(best) if ok else None), t
+
+    def decode(self, failed: Sequence[int], plan: Plan, options=None) -> List[List[int]]:
+        o, sfx = self._opts(options)
+        _, fp, nf = self._failed(failed)
+        c = self._cplan(plan)
         out = np.zeros(MAX_PIPES * (MAX_STAGES + 1), dtype=np.int32)
         n = self._fn("orc_decode", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(c), _ptr(out, C.c_int32))
         if n < 0:

@@ -52,6 +52,32 @@ typedef struct {
     uint64_t kappa[ORC_MAX_PIPES];
 } orc_plan;
 
+/* The paper's full objective (Section "Problem Formulation"): throughput of the next state
+ * times the share of the time until the next fault that is spent training.  */
+typedef struct {
+    int32_t topk;                    /* dynamic-parallelism plans that are re-scored, >= 1   */
+    int32_t pad;
+    double t_gap, t_restart;         /* ns between two faults / restart overhead (_f64)     */
+    int64_t t_gap_ns, t_restart_ns;  /* the same as integers (_i64)                         */
+    int64_t bw_xfer;                 /* bytes per ns available to the weight transfer       */
+} orc_objective;
+
+typedef struct {
+    int32_t policy, feasible;
+    int32_t rank;                    /* position of the chosen plan in the shortlist, -1 for the other policies */
+    int32_t n_surv;
+    int64_t xfer_bytes;              /* bytes moved by the cheapest migration scheme        */
+    double t_trans;                  /* transition time, _f64                               */
+    int64_t t_trans_ns;              /* transition time, _i64                               */
+    double objective;                /* steps completed before the next fault               */
+} orc_transition;
+
+/* ---- orc_restore.c: weight-transfer matching (integer) ---- */
+void orc_transfer_cost_matrix(int L, const int64_t *w, int n, const int32_t *old_lo, const int32_t *old_hi,
+                              const int32_t *new_lo, const int32_t *new_hi, int64_t *cost /* [n][n] */);
+int64_t orc_assign(int n, const int64_t *cost, int32_t *row_of_col);
+int64_t orc_assign_brute(int n, const int64_t *cost);
+
 /* ---- orc_enum.c: integer combinatorics (no cost arithmetic) ---- */
 uint64_t orc_binom(int n, int k);                       /* saturates at UINT64_MAX */
 void orc_unrank_subset(uint64_t rank, int t, int *c);   /* colex, c[0]<...<c[t-1]  */

@@ -561,17 +561,8 @@ static const segment *find_segment(const space *sp, int si, int p, int m) {
     return NULL;
 }
 
-/*
- * Search over dynamic-parallelism plans (Algorithm 1, get_execution_plan: keep the plan
- * with the least estimated time; step time = slowest pipeline).  A plan is the tuple
- * (strategy, split rank beta, kappa_1..kappa_dp).  Selected: the feasible plan of least
- * cost, ties to the lexicographically smallest tuple.  Because feasibility and
- * "cost <= T" are per-pipeline conditions this is found in three plain steps:
- *   1. best[segment] = min over feasible kappa of the pipeline cost;
- *   2. T(strategy, beta) = max over pipelines of best[...]; T* = min, first on ties;
- *   3. for the winner, kappa_p = the lowest kappa that is feasible with cost <= T*.
- */
-static void dynpar_search(const space *sp, orc_plan *out) {
+/* Step 1 of the search: the least feasible cost of every segment (malloc'ed, n_seg entries). */
+static num_t *segment_minima(const space *sp) {
     num_t *best = (num_t *)malloc(sizeof(num_t) * (size_t)(sp->n_seg + 1));
     for (int s = 0; s < sp->n_seg; s++) {
         const segment *g = &sp->seg[s];
@@ -583,6 +574,21 @@ static void dynpar_search(const space *sp, orc_plan *out) {
         }
         best[s] = b;
     }
+    return best;
+}
+
+/*
+ * Search over dynamic-parallelism plans (Algorithm 1, get_execution_plan: keep the plan
+ * with the least estimated time; step time = slowest pipeline).  A plan is the tuple
+ * (strategy, split rank beta, kappa_1..kappa_dp).  Selected: the feasible plan of least
+ * cost, ties to the lexicographically smallest tuple.  Because feasibility and
+ * "cost <= T" are per-pipeline conditions this is found in three plain steps:
+ *   1. best[segment] = min over feasible kappa of the pipeline cost;
+ *   2. T(strategy, beta) = max over pipelines of best[...]; T* = min, first on ties;
+ *   3. for the winner, kappa_p = the lowest kappa that is feasible with cost <= T*.
+ */
+static void dynpar_search(const space *sp, orc_plan *out) {
+    num_t *best = segment_minima(sp);
     num_t Tstar = NUM_INF;
     int win_si = -1;
     uint64_t win_beta = 0;
@@ -879,3 +885,216 @@ int NAME(orc_decode)(const orc_profile *prof, const orc_opts *o, const uint32_t 
     }
     return n;
 }
+
+/* ------------------------------------------------- transition time, full objective */
+
+/*
+ * Shortlist of dynamic-parallelism plans for the full objective.  The pairs (strategy,
+ * split) are ordered by their step time T(strategy, split), ties by position in the
+ * enumeration; the first k feasible ones are kept.  Each is completed the same way the
+ * search completes its winner: kappa_p = the lowest kappa that is feasible with pipeline
+ * cost <= T of that pair.  (Reading: the paper ranks plans by the product of throughput
+ * and effective-time ratio but gives no procedure for the coupled problem; the transfer
+ * cost couples the pipelines, so only a shortlist by step time is re-scored.)
+ */
+typedef struct { num_t T; int si; uint64_t beta; uint64_t order; } pair_t;
+
+static int pair_cmp(const void *a, const void *b) {
+    const pair_t *x = (const pair_t *)a, *y = (const pair_t *)b;
+    if (x->T < y->T) return -1;
+    if (x->T > y->T) return 1;
+    return x->order < y->order ? -1 : (x->order > y->order ? 1 : 0);
+}
+
+static int dynpar_shortlist(const space *sp, int k, orc_plan *plans) {
+    num_t *best = segment_minima(sp);
+    size_t cap = 1024, n = 0;
+    pair_t *pairs = (pair_t *)malloc(cap * sizeof(pair_t));
+    uint64_t order = 0;
+    for (int si = 0; si < sp->n_strat; si++) {
+        int dp = sp->dp[si];
+        const int32_t *st = &sp->stages[(size_t)si * ORC_MAX_PIPES];
+        uint64_t n_split = orc_split_count(sp->o.batch_mode, sp->G, sp->n_surv, dp, st);
+        for (uint64_t beta = 0; beta < n_split; beta++, order++) {
+            int32_t micro[ORC_MAX_PIPES];
+            if (!orc_split_unrank(sp->o.batch_mode, sp->G, sp->n_surv, dp, st, beta, micro)) continue;
+            num_t T = 0;
+            for (int p = 0; p < dp; p++) {
+                const segment *g = find_segment(sp, si, p, micro[p]);
+                num_t b = g ? best[g - sp->seg] : NUM_INF;
+                T = nmax(T, b);
+            }
+            if (!(T < NUM_INF)) continue;
+            if (n == cap) { cap *= 2; pairs = (pair_t *)realloc(pairs, cap * sizeof(pair_t)); }
+            pairs[n].T = T; pairs[n].si = si; pairs[n].beta = beta; pairs[n].order = order;
+            n++;
+        }
+    }
+    qsort(pairs, n, sizeof(pair_t), pair_cmp);
+    int kept = 0;
+    for (size_t t = 0; t < n && kept < k; t++, kept++) {
+        orc_plan *out = &plans[kept];
+        int si = pairs[t].si;
+        int dp = sp->dp[si];
+        int32_t micro[ORC_MAX_PIPES];
+        memset(out, 0, sizeof(*out));
+        orc_split_unrank(sp->o.batch_mode, sp->G, sp->n_surv, dp, &sp->stages[(size_t)si * ORC_MAX_PIPES],
+                         pairs[t].beta, micro);
+        out->policy = ORC_DYNPAR;
+        out->feasible = 1;
+#if ORC_INT
+        out->cost_ns = pairs[t].T;
+#else
+        out->cost = pairs[t].T;
+#endif
+        out->strategy = (uint32_t)si;
+        out->n_pipes = (uint32_t)dp;
+        out->split_rank = pairs[t].beta;
+        for (int p = 0; p < dp; p++) {
+            const segment *g = find_segment(sp, si, p, micro[p]);
+            out->stages[p] = (uint16_t)g->S;
+            out->micro[p] = (uint16_t)micro[p];
+            for (uint64_t kappa = 0; kappa < g->count; kappa++) {
+                num_t c; int ok;
+                segment_eval(sp, g, kappa, &c, &ok);
+                if (ok && c <= pairs[t].T) { out->kappa[p] = kappa; break; }
+            }
+        }
+    }
+    free(pairs);
+    free(best);
+    return kept;
+}
+
+/*
+ * Bytes moved by the cheapest migration into a dynamic-parallelism plan (Section
+ * "Restorer", Weight Transfer).  Survivor u (ascending device id, device = pipeline *
+ * n_pp + stage) still holds the layers of its old stage; position j = off_p + i of the
+ * plan needs the layers of stage i of pipeline p.  assign[j] = index of the survivor that
+ * takes position j.
+ */
+static int64_t plan_transfer_bytes(const space *sp, const orc_plan *pl, int32_t *assign) {
+    const orc_profile *pr = sp->M.p;
+    int n = sp->n_surv;
+    int32_t *olo = (int32_t *)malloc(sizeof(int32_t) * 4 * (size_t)n);
+    int32_t *ohi = olo + n, *nlo = ohi + n, *nhi = nlo + n;
+    int64_t *w = (int64_t *)malloc(sizeof(int64_t) * (size_t)pr->L);
+    for (int l = 0; l < pr->L; l++) w[l] = pr->param_bytes[l] + pr->opt_bytes[l];
+    for (int u = 0; u < n; u++) {
+        int stage = sp->surv[u] % pr->n_pp;
+        olo[u] = pr->base_cuts[stage];
+        ohi[u] = pr->base_cuts[stage + 1];
+    }
+    int j = 0;
+    for (uint32_t p = 0; p < pl->n_pipes; p++) {
+        int32_t cuts[ORC_MAX_STAGES + 1];
+        const segment *g = find_segment(sp, (int)pl->strategy, (int)p, pl->micro[p]);
+        segment_cuts(sp, g, pl->kappa[p], cuts);
+        for (int i = 0; i < g->S; i++, j++) { nlo[j] = cuts[i]; nhi[j] = cuts[i + 1]; }
+    }
+    int64_t *cost = (int64_t *)malloc(sizeof(int64_t) * (size_t)n * (size_t)n);
+    int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+    orc_transfer_cost_matrix(pr->L, w, n, olo, ohi, nlo, nhi, cost);
+    int64_t total = orc_assign(n, cost, tmp);
+    if (assign) memcpy(assign, tmp, sizeof(int32_t) * (size_t)n);
+    free(cost); free(tmp); free(w); free(olo);
+    return total;
+}
+
+/*
+ * Objective of one candidate next state (Section "Problem Formulation", the arg max over
+ * the next state): throughput B / t_step times the effective-time ratio
+ * t_state / (t_trans + t_state), where t_trans + t_state = t_gap is the same for every
+ * plan.  B and t_gap are constants of the arg max, so plans are ranked by
+ *     (t_gap - t_trans) / t_step  =  training steps completed before the next fault.
+ * Transition time (Section "Estimator"): search cost is overlapped with training and not
+ * charged; restart overhead is a constant of the training scale; the weight transfer is
+ * the matched bytes over the transfer bandwidth (reading: the paper gives no formula for
+ * the time of the transfer, only that its amount is minimised).  Rerouting and redundant
+ * computation need no reconstruction: transition time 0.
+ * _f64: one IEEE operation per written operation.  _i64: the quotient bytes / bandwidth
+ * floors and two objectives are compared exactly as fractions.
+ */
+typedef struct { num_t numer, denom; } frac_t;
+
+static int frac_greater(frac_t a, frac_t b) {   /* a > b, both denominators > 0 */
+#if ORC_INT
+    return (__int128)a.numer * (__int128)b.denom > (__int128)b.numer * (__int128)a.denom;
+#else
+    return a.numer / a.denom > b.numer / b.denom;
+#endif
+}
+
+int NAME(orc_search_objective)(const orc_profile *prof, const orc_opts *o, const uint32_t *failed, int n_failed,
+                               const orc_objective *q, orc_plan *best, orc_transition *tr,
+                               int32_t *assign /* [n_surv] or NULL */,
+                               orc_plan *short_plans /* [topk] or NULL */, int64_t *short_bytes /* [topk] or NULL */,
+                               int32_t *n_short /* or NULL */) {
+#if ORC_INT
+    const num_t t_gap = q->t_gap_ns, t_restart = q->t_restart_ns;
+#else
+    const num_t t_gap = q->t_gap, t_restart = q->t_restart;
+#endif
+    int k = q->topk < 1 ? 1 : q->topk;
+    orc_plan *plans = (orc_plan *)calloc((size_t)k + 2, sizeof(orc_plan));
+    space sp;
+    space_build(&sp, prof, o, failed, n_failed);
+    int32_t *asg = (int32_t *)malloc(sizeof(int32_t) * (size_t)(sp.n_surv + 1));
+    int have = 0;
+    frac_t best_j = {0, 1};
+    memset(best, 0, sizeof(*best));
+    memset(tr, 0, sizeof(*tr));
+    tr->n_surv = sp.n_surv;
+    tr->rank = -1;
+    /* policies without reconstruction, in policy order */
+    for (int pol = 0; pol < 2; pol++) {
+        orc_plan pl;
+        NAME(orc_search_policy)(prof, o, failed, n_failed, pol, 0, &pl, NULL);
+        if (!pl.feasible) continue;
+        frac_t j = {t_gap, get_cost(&pl)};
+        if (!have || frac_greater(j, best_j)) {
+            have = 1; best_j = j; *best = pl;
+            tr->policy = pol; tr->feasible = 1; tr->rank = -1; tr->xfer_bytes = 0;
+            tr->t_trans = 0; tr->t_trans_ns = 0;
+        }
+    }
+    int ns = dynpar_shortlist(&sp, k, plans);
+    if (n_short) *n_short = ns;
+    for (int r = 0; r < ns; r++) {
+        int64_t bytes = plan_transfer_bytes(&sp, &plans[r], asg);
+        if (short_plans) short_plans[r] = plans[r];
+        if (short_bytes) short_bytes[r] = bytes;
+#if ORC_INT
+        num_t t_trans = t_restart + bytes / q->bw_xfer;
+#else
+        num_t t_trans = t_restart + (double)bytes / (double)q->bw_xfer;
+#endif
+        frac_t j = {t_gap - t_trans, get_cost(&plans[r])};
+        if (!have || frac_greater(j, best_j)) {
+            have = 1; best_j = j; *best = plans[r];
+            tr->policy = ORC_DYNPAR; tr->feasible = 1; tr->rank = r; tr->xfer_bytes = bytes;
+#if ORC_INT
+            tr->t_trans_ns = t_trans; tr->t_trans = 0;
+#else
+            tr->t_trans = t_trans; tr->t_trans_ns = 0;
+#endif
+            if (assign) memcpy(assign, asg, sizeof(int32_t) * (size_t)sp.n_surv);
+        }
+    }
+    if (have) tr->objective = (double)best_j.numer / (double)best_j.denom;
+    free(asg);
+    free(plans);
+    space_free(&sp);
+    return have;
+}
+
+/* Transfer bytes and matching of one given dynamic-parallelism plan. */
+int64_t NAME(orc_plan_transfer)(const orc_profile *prof, const orc_opts *o, const uint32_t *failed, int n_failed,
+                                const orc_plan *pl, int32_t *assign /* [n_surv] or NULL */) {
+    space sp;
+    space_build(&sp, prof, o, failed, n_failed);
+    int64_t b = plan_transfer_bytes(&sp, pl, assign);
+    space_free(&sp);
+    return b;
+}
+

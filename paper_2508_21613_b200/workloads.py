@@ -111,6 +111,21 @@ class SearchOptions:
 
 
 @dataclass
+class ObjectiveOptions:
+    """Inputs of the full objective: how many dynamic-parallelism plans are re-scored with
+    their transition time, the time between two faults, the restart overhead of a
+    reconfiguration and the bandwidth the weight transfer gets (bytes per ns).
+
+    Defaults at the scale of the paper's evaluation: its simulated trace fails each of 32
+    devices at 10 % per hour (one fault every 1125 s on average) and its measured recoveries
+    take around ten seconds, transfer included."""
+    topk: int = 8
+    t_gap_ns: float = 1125e9
+    t_restart_ns: float = 5e9
+    bw_xfer_Bpns: int = 25
+
+
+@dataclass
 class Workload:
     name: str
     profile: Profile
