@@ -43,6 +43,8 @@ extern "C" {
 #define CM_MAX_STAGES 64   /* stages of one pipeline                       */
 #define CM_MAX_LAYERS 128  /* model layers in a profile                    */
 #define CM_MAX_MICRO 4096  /* global micro-batches per iteration (N_dp*N_m) */
+#define CM_MAX_SHORTLIST 16 /* dynamic-parallelism plans re-scored by the full objective */
+#define CM_MAX_MATCH 256   /* devices in one weight-transfer matching      */
 
 typedef struct cm_ctx cm_ctx;     /* device buffers, profile copy, tables               */
 typedef struct cm_space cm_space; /* implicit candidate space of one (policy, failure set) */
@@ -221,6 +223,87 @@ cm_status cm_batch_free(cm_batch *batch);
 cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64_t count,
                                      double *best_cost_dev, int64_t *best_cost_ns_dev,
                                      uint64_t *best_index_dev);
+
+/* ---------------------------------------------------------------------------------
+ * Full objective: transition time included.
+ *
+ * Section "Problem Formulation" ranks a candidate next state by
+ *     throughput * effective-time ratio = (B / t_step) * t_state / (t_trans + t_state),
+ * where t_trans + t_state (the time between two faults, t_gap) does not depend on the plan.
+ * B and t_gap being constants of the arg max, plans are ranked by
+ *     (t_gap - t_trans) / t_step,   the training steps completed before the next fault.
+ * Section "Estimator": rerouting (and redundant computation) need no reconstruction,
+ * t_trans = 0; for dynamic parallelism t_trans = restart overhead + weight transfer (the
+ * search itself is overlapped with training).  Section "Restorer", Weight Transfer: the
+ * survivors are matched to the positions of the new plan by a minimum-cost perfect
+ * matching over Cost[i][j] = model state (parameters + optimizer bytes per layer, from the
+ * loaded profile) of the layers position j holds and device i does not hold yet; the
+ * transfer takes (matched bytes) / bw_xfer.
+ *
+ * The transfer couples the pipelines of a plan, so it is applied to a shortlist: the
+ * `topk` (strategy, split) pairs of least step time (ties: enumeration order), each
+ * completed with the lowest layer compositions that meet its own step time.  The winner
+ * is the candidate of greatest objective among rerouting, redundant computation and the
+ * shortlist, ties to the lower policy id, then to the earlier shortlist rank.  fp64 mode
+ * computes t_trans = t_restart + bytes / bw and the objective with one IEEE operation each;
+ * int64 mode floors bytes / bw and compares objectives exactly as fractions.
+ * --------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t topk;              /* 1 .. CM_MAX_SHORTLIST                                   */
+    int32_t reserved;
+    double t_gap_ns;           /* time between two faults (fp64 mode), finite, > 0          */
+    double t_restart_ns;       /* restart overhead of a reconstruction (fp64 mode), >= 0     */
+    int64_t t_gap_ns_i;        /* the same, integer nanoseconds (int64 mode)                */
+    int64_t t_restart_ns_i;
+    int64_t bw_xfer_Bpns;      /* bandwidth of the weight transfer, bytes per ns, > 0       */
+} cm_objective_opts;
+
+typedef struct {
+    int32_t policy, feasible;
+    int32_t rank;              /* shortlist rank of the chosen plan, -1 for the other policies */
+    int32_t n_survivors;
+    int64_t xfer_bytes;        /* bytes moved by the cheapest migration (0 without one)     */
+    double t_trans;            /* transition time, ns (fp64 mode; 0 in int64 mode)          */
+    int64_t t_trans_ns;        /* transition time, ns (int64 mode; 0 in fp64 mode)          */
+    double objective;          /* steps before the next fault (int64 mode: numerator / denominator rounded once) */
+    uint16_t assign[CM_MAX_MATCH]; /* dynamic parallelism: position j (pipeline-major, stage-minor) ->
+                                      index, among the survivors in ascending id order, of the device
+                                      that takes it; zeros otherwise                         */
+} cm_transition;
+
+/* The search of cm_search_batch followed by the re-scoring above, for B failure sets.
+ * failed_ids / offsets / opts as for cm_search_batch (HOST).  best[B] and trans[B] (HOST,
+ * caller-owned) receive the chosen plan (plan.cost / cost_ns = its step time) and its
+ * transition.  shortlist (HOST [B * topk], may be NULL) receives the shortlisted plans in
+ * rank order, shortlist_bytes (HOST [B * topk], may be NULL) their matched bytes; unused
+ * slots have feasible = 0 and bytes = -1.  Several matchings of one plan can be optimal:
+ * assign[] is one of them, xfer_bytes is unique.
+ * Errors: CM_EINVAL (bad options; more than CM_MAX_MATCH devices in the profile's grid),
+ * CM_ENOPROFILE, CM_EOVERFLOW, CM_ENOMEM, CM_ECUDA.  A scenario without any feasible plan
+ * has best[b].feasible = 0 and is not an error of the batch.  Synchronises the stream. */
+cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                              const cm_enum_opts *opts, const cm_objective_opts *objective,
+                              cm_plan *best, cm_transition *trans, cm_plan *shortlist,
+                              int64_t *shortlist_bytes);
+
+/* Device time and work of the objective pass of the last cm_search_objective (HOST out[8]):
+ * [0] shortlist kernel, ns  [1] completing the shortlisted plans (tie-break kernels), ns
+ * [2] matching kernel, ns  [3] objective kernel, ns  [4] matchings solved (only counted when
+ * shortlist_bytes was asked for)  [5] kernels launched  [6] bytes copied device->host
+ * [7] sum of [0..3].  cm_last_stats describes the search that ran before it. */
+cm_status cm_objective_stats(const cm_ctx *ctx, uint64_t out[8]);
+
+/* Weight-transfer matchings over explicit layer ranges (Section "Restorer", Weight
+ * Transfer), using the per-layer model state of the loaded profile.  Problem q has
+ * sizes[q] devices (1 .. CM_MAX_MATCH); device i holds layers [old_lo[q][i], old_hi[q][i]),
+ * position j needs [new_lo[q][j], new_hi[q][j]) (all HOST, row stride CM_MAX_MATCH, values
+ * 0 .. L, empty ranges allowed).  total[q] (HOST) = bytes of the cheapest perfect matching;
+ * assign (HOST [n_problems][CM_MAX_MATCH], may be NULL): device index matched to position j.
+ * Errors: CM_EINVAL, CM_ENOPROFILE, CM_ENOMEM, CM_ECUDA.  Synchronises the stream. */
+cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *sizes,
+                               const uint8_t *old_lo, const uint8_t *old_hi,
+                               const uint8_t *new_lo, const uint8_t *new_hi,
+                               int64_t *total, uint16_t *assign);
 
 /* Work counters of the last cm_select / cm_search_batch / cm_batch_search on this
  * context (HOST out[16]):

@@ -28,9 +28,11 @@ CM_COST_FP64, CM_COST_INT64NS = 0, 1
 
 EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_evaluate", "cm_select",
            "cm_decode_plan", "cm_space_free", "cm_search_batch", "cm_batch_prepare", "cm_batch_search",
-           "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_strerror", "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:14]
+           "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
+           "cm_objective_stats", "cm_transfer_matching", "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:17]
 NOALLOC_MAX_CANDIDATES = 524288
+MAX_SHORTLIST, MAX_MATCH = 16, 256
 
 
 class ChameleonError(RuntimeError):
@@ -60,6 +62,18 @@ class cm_plan(C.Structure):
                 ("cost_ns", C.c_int64), ("strategy", C.c_uint32), ("n_pipes", C.c_uint32),
                 ("split_rank", C.c_uint64), ("stages", C.c_uint16 * MAX_PIPES),
                 ("micro", C.c_uint16 * MAX_PIPES), ("kappa", C.c_uint64 * MAX_PIPES)]
+
+
+class cm_objective_opts(C.Structure):
+    _fields_ = [("topk", C.c_int32), ("reserved", C.c_int32), ("t_gap_ns", C.c_double),
+                ("t_restart_ns", C.c_double), ("t_gap_ns_i", C.c_int64), ("t_restart_ns_i", C.c_int64),
+                ("bw_xfer_Bpns", C.c_int64)]
+
+
+class cm_transition(C.Structure):
+    _fields_ = [("policy", C.c_int32), ("feasible", C.c_int32), ("rank", C.c_int32), ("n_survivors", C.c_int32),
+                ("xfer_bytes", C.c_int64), ("t_trans", C.c_double), ("t_trans_ns", C.c_int64),
+                ("objective", C.c_double), ("assign", C.c_uint16 * 256)]
 
 
 @dataclass
@@ -126,6 +140,12 @@ def load_library() -> C.CDLL:
     lib.cm_batch_search.argtypes = [vp, vp, C.POINTER(cm_plan), C.POINTER(cm_plan)]
     lib.cm_batch_free.argtypes = [vp]
     lib.cm_evaluate_argmin_noalloc.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp, vp, vp]
+    lib.cm_search_objective.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_int32), C.c_int32,
+                                        C.POINTER(cm_enum_opts), C.POINTER(cm_objective_opts), C.POINTER(cm_plan),
+                                        C.POINTER(cm_transition), C.POINTER(cm_plan), C.POINTER(C.c_int64)]
+    lib.cm_objective_stats.argtypes = [vp, u64p]
+    lib.cm_transfer_matching.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), vp, vp, vp, vp,
+                                         C.POINTER(C.c_int64), C.POINTER(C.c_uint16)]
     for name in _STATUS_CALLS:
         getattr(lib, name).restype = C.c_int
     _lib = lib
@@ -261,6 +281,51 @@ def cm_evaluate_argmin_noalloc(ctx, space, first: int, count: int, best_cost_dev
                                                           ptr(best_cost_ns_dev), ptr(best_index_dev)))
 
 
+def _objective(obj) -> cm_objective_opts:
+    return cm_objective_opts(int(obj.topk), 0, float(obj.t_gap_ns), float(obj.t_restart_ns),
+                             int(round(obj.t_gap_ns)), int(round(obj.t_restart_ns)), int(obj.bw_xfer_Bpns))
+
+
+def cm_search_objective(ctx, scenarios: Sequence[Sequence[int]], opts, objective, shortlist: bool = False):
+    """Search plus re-scoring with the transition time.  -> (best plans, transitions,
+    shortlisted plans or None, their matched bytes as numpy int64 [B, topk] or None); the
+    first three are ctypes arrays (cm_plan / cm_transition), shortlist slots scenario-major."""
+    packed = PackedScenarios(scenarios)
+    return packed.search_objective(ctx, opts, objective, shortlist)
+
+
+def cm_objective_stats(ctx) -> dict:
+    out = (C.c_uint64 * 8)()
+    _check(ctx, load_library().cm_objective_stats(ctx, out))
+    keys = ["shortlist_ns", "complete_ns", "matching_ns", "objective_ns", "matchings", "launches", "d2h_bytes",
+            "device_ns"]
+    return dict(zip(keys, [int(v) for v in out]))
+
+
+def cm_transfer_matching(ctx, problems: Sequence[Tuple[Sequence[Tuple[int, int]], Sequence[Tuple[int, int]]]]):
+    """Weight-transfer matchings over explicit layer ranges.  ``problems`` = [(old ranges,
+    new ranges)], ranges as (lo, hi) pairs.  -> (total bytes int64 [n], assignments: list of lists)."""
+    n = len(problems)
+    sizes = np.zeros(max(n, 1), dtype=np.int32)
+    arr = np.zeros((4, max(n, 1), MAX_MATCH), dtype=np.uint8)
+    for q, (old, new) in enumerate(problems):
+        if len(old) != len(new):
+            raise ValueError("a matching needs as many devices as positions")
+        sizes[q] = len(old)
+        if len(old) <= MAX_MATCH:
+            for j, (a, b) in enumerate(old):
+                arr[0, q, j], arr[1, q, j] = a, b
+            for j, (a, b) in enumerate(new):
+                arr[2, q, j], arr[3, q, j] = a, b
+    total = np.zeros(max(n, 1), dtype=np.int64)
+    assign = np.zeros((max(n, 1), MAX_MATCH), dtype=np.uint16)
+    ptr = lambda a: C.c_void_p(a.ctypes.data)
+    _check(ctx, load_library().cm_transfer_matching(
+        ctx, n, sizes.ctypes.data_as(C.POINTER(C.c_int32)), ptr(arr[0]), ptr(arr[1]), ptr(arr[2]), ptr(arr[3]),
+        total.ctypes.data_as(C.POINTER(C.c_int64)), assign.ctypes.data_as(C.POINTER(C.c_uint16))))
+    return total[:n], [[int(x) for x in assign[q, :sizes[q]]] for q in range(n)]
+
+
 def cm_batch_free(batch) -> None:
     _check(None, load_library().cm_batch_free(batch))
 
@@ -308,3 +373,17 @@ class PackedScenarios:
             ctx, self.ids.ctypes.data_as(C.POINTER(C.c_uint32)), self.offsets.ctypes.data_as(C.POINTER(C.c_int32)),
             self.B, C.byref(o), self.best, self.per_policy,
             self.latency.ctypes.data_as(C.POINTER(C.c_float)) if latency else None))
+
+    def search_objective(self, ctx, opts, objective, shortlist: bool = False):
+        """cm_search_objective into freshly made host arrays (see the module function)."""
+        o, q = _opts(opts), _objective(objective)
+        B, k = self.B, int(objective.topk)
+        best = (cm_plan * max(B, 1))()
+        trans = (cm_transition * max(B, 1))()
+        sl = (cm_plan * max(B * k, 1))() if shortlist else None
+        sb = np.full((max(B, 1), max(k, 1)), -1, dtype=np.int64) if shortlist else None
+        _check(ctx, load_library().cm_search_objective(
+            ctx, self.ids.ctypes.data_as(C.POINTER(C.c_uint32)), self.offsets.ctypes.data_as(C.POINTER(C.c_int32)),
+            B, C.byref(o), C.byref(q), best, trans, sl,
+            sb.ctypes.data_as(C.POINTER(C.c_int64)) if shortlist else None))
+        return best, trans, sl, sb

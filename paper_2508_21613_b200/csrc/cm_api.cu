@@ -92,6 +92,16 @@ struct Batch {
     DevBuf<Winner> d_winner;
     DevBuf<uint16_t> d_rc_stages;
     DevBuf<cm_plan> d_plans;
+    // full objective: shortlist slots (scenario-major) and per-scenario results
+    DevBuf<Winner> d_short_win;
+    DevBuf<uint64_t> d_short_kappa;
+    DevBuf<int64_t> d_short_bytes;
+    DevBuf<uint16_t> d_short_assign;
+    DevBuf<cm_plan> d_short_plans, d_obj_best;
+    DevBuf<cm_transition> d_trans;
+    PinnedVec<cm_plan> obj_best_host, short_plans_host;
+    PinnedVec<cm_transition> trans_host;
+    PinnedVec<int64_t> short_bytes_host;
     cm_enum_opts opts{};
     uint32_t policy_mask = 0;
     uint64_t n_cand = 0, n_tiles = 0, n_split = 0;
@@ -114,6 +124,8 @@ struct cm_ctx {
     int mm_stride_m = 0;
     Batch batch;                      // reused by cm_search_batch
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_obj[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // phases of the objective pass
+    uint64_t obj_stats[8] = {0};
     SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
@@ -648,6 +660,7 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
     c->stream = (cudaStream_t)cuda_stream;
     bool ok = true;
     for (int i = 0; i < 6; ++i) ok = ok && cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    for (int i = 0; i < 5; ++i) ok = ok && cudaEventCreate(&c->ev_obj[i]) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->side.fork, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 3 && ok; ++i) {
         ok = cudaStreamCreateWithFlags(&c->side.stream[i], cudaStreamNonBlocking) == cudaSuccess &&
@@ -669,6 +682,8 @@ cm_status cm_destroy(cm_ctx *c) {
     cudaStreamSynchronize(c->stream);
     for (int i = 0; i < 6; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (int i = 0; i < 5; ++i)
+        if (c->ev_obj[i]) cudaEventDestroy(c->ev_obj[i]);
     for (int i = 0; i < 3; ++i) {
         if (c->side.stream[i]) { cudaStreamSynchronize(c->side.stream[i]); cudaStreamDestroy(c->side.stream[i]); }
         if (c->side.join[i]) cudaEventDestroy(c->side.join[i]);
@@ -899,6 +914,163 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         const auto t1 = std::chrono::steady_clock::now();
         latency_us[b] = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
     }
+    return CM_OK;
+}
+
+cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
+                              const cm_enum_opts *opts, const cm_objective_opts *objective,
+                              cm_plan *best, cm_transition *trans, cm_plan *shortlist, int64_t *shortlist_bytes) {
+    if (!ctx) return CM_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
+    if (B < 0 || !offsets || !best || !trans || !objective || (offsets[B] > 0 && !failed_ids))
+        return fail(ctx, CM_EINVAL, "bad arguments");
+    cm_status s = check_opts(ctx, opts);
+    if (s != CM_OK) return s;
+    const cm_objective_opts &q = *objective;
+    if (q.topk < 1 || q.topk > CM_MAX_SHORTLIST) return fail(ctx, CM_EINVAL, "topk must be 1 .. CM_MAX_SHORTLIST");
+    if (q.bw_xfer_Bpns <= 0) return fail(ctx, CM_EINVAL, "transfer bandwidth must be positive");
+    if (!(q.t_gap_ns > 0.0) || !std::isfinite(q.t_gap_ns) || !(q.t_restart_ns >= 0.0) || !std::isfinite(q.t_restart_ns) ||
+        q.t_gap_ns_i <= 0 || q.t_restart_ns_i < 0 || q.t_gap_ns_i > (1ll << 60) || q.t_restart_ns_i > (1ll << 60))
+        return fail(ctx, CM_EINVAL, "fault gap must be positive and finite, restart overhead non-negative");
+    if (ctx->hp.n_dp * ctx->hp.n_pp > CM_MAX_MATCH) return fail(ctx, CM_EINVAL, "more than CM_MAX_MATCH devices");
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    memset(ctx->stats, 0, sizeof(ctx->stats));
+    memset(ctx->obj_stats, 0, sizeof(ctx->obj_stats));
+    if (B == 0) return CM_OK;
+    const uint32_t mask = (1u << CM_REROUTE) | (1u << CM_REDUNDANT) | (1u << CM_DYNPAR);
+    Batch &bt = ctx->batch;
+    int launches = 0;
+    const uint64_t h0 = now_ns();
+    if ((s = build_batch(ctx, bt, failed_ids, offsets, B, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+    ctx->stats[13] += now_ns() - h0;
+    if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
+    if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
+
+    // the objective pass works on what the search left on the device
+    const size_t slots = (size_t)B * q.topk;
+    bool ok = bt.d_short_win.reserve(slots) && bt.d_short_kappa.reserve(slots * kMaxP) && bt.d_short_bytes.reserve(slots) &&
+              bt.d_short_assign.reserve(slots * kMaxMatch) && bt.d_short_plans.reserve(slots) &&
+              bt.d_obj_best.reserve(B) && bt.d_trans.reserve(B);
+    if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
+    ok = bt.obj_best_host.resize(B) && bt.trans_host.resize(B) && bt.short_plans_host.resize(slots) &&
+         bt.short_bytes_host.resize(slots);
+    if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
+    const Tables tb = tables(ctx, bt.opts.cost);
+    const BatchDev bd = dev_view(ctx, bt);
+    ObjDev od{};
+    od.topk = q.topk;
+    od.t_gap = q.t_gap_ns; od.t_restart = q.t_restart_ns;
+    od.t_gap_i = q.t_gap_ns_i; od.t_restart_i = q.t_restart_ns_i; od.bw_xfer = q.bw_xfer_Bpns;
+    od.short_win = bt.d_short_win.p; od.short_kappa = bt.d_short_kappa.p; od.short_bytes = bt.d_short_bytes.p;
+    od.short_assign = bt.d_short_assign.p; od.short_plans = shortlist ? bt.d_short_plans.p : nullptr;
+    od.best = bt.d_obj_best.p; od.trans = bt.d_trans.p;
+    cudaStream_t st = ctx->stream;
+    int obj_launches = 0;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[0], st));
+    CM_CUDA(ctx, launch_shortlist(tb, bd, od, st));
+    ++obj_launches;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[1], st));
+    if (bt.n_tiles) {
+        // the tie-break kernels complete every shortlisted pair exactly as they complete the winner
+        BatchDev sd = bd;
+        sd.winner = od.short_win;
+        sd.kappa_sel = od.short_kappa;
+        sd.B = (int32_t)slots;
+        CM_CUDA(ctx, launch_cost_pass2(tb, sd, st));
+        ++obj_launches;
+        uint64_t stage_mask = 0;
+        for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
+        CM_CUDA(ctx, launch_tiebreak_wide(tb, sd, stage_mask, st, &obj_launches));
+    }
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[2], st));
+    CM_CUDA(ctx, launch_plan_matching(tb, bd, od, st));
+    ++obj_launches;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[3], st));
+    CM_CUDA(ctx, launch_objective(tb, bd, od, st));
+    ++obj_launches;
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[4], st));
+    size_t back = 0;
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.obj_best_host.p, bt.d_obj_best.p, sizeof(cm_plan) * B, cudaMemcpyDeviceToHost, st));
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.trans_host.p, bt.d_trans.p, sizeof(cm_transition) * B, cudaMemcpyDeviceToHost, st));
+    back += (sizeof(cm_plan) + sizeof(cm_transition)) * (size_t)B;
+    if (shortlist) {
+        CM_CUDA(ctx, cudaMemcpyAsync(bt.short_plans_host.p, bt.d_short_plans.p, sizeof(cm_plan) * slots, cudaMemcpyDeviceToHost, st));
+        back += sizeof(cm_plan) * slots;
+    }
+    if (shortlist_bytes) {
+        CM_CUDA(ctx, cudaMemcpyAsync(bt.short_bytes_host.p, bt.d_short_bytes.p, sizeof(int64_t) * slots, cudaMemcpyDeviceToHost, st));
+        back += sizeof(int64_t) * slots;
+    }
+    CM_CUDA(ctx, cudaStreamSynchronize(st));
+    for (int i = 0; i < 4; ++i) {
+        float ms = 0.f;
+        CM_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev_obj[i], ctx->ev_obj[i + 1]));
+        ctx->obj_stats[i] = (uint64_t)((double)ms * 1e6);
+        ctx->obj_stats[7] += ctx->obj_stats[i];
+    }
+    ctx->obj_stats[5] = (uint64_t)obj_launches;
+    ctx->obj_stats[6] = back;
+    for (int b = 0; b < B; ++b) {
+        cm_plan pl = bt.obj_best_host[b];
+        scrub(pl);
+        best[b] = pl;
+        trans[b] = bt.trans_host[b];
+        if (!pl.feasible) trans[b].feasible = 0;
+    }
+    uint64_t solved = 0;
+    for (size_t i = 0; i < slots; ++i) {
+        if (shortlist) { cm_plan pl = bt.short_plans_host[i]; scrub(pl); shortlist[i] = pl; }
+        if (shortlist_bytes) { shortlist_bytes[i] = bt.short_bytes_host[i]; solved += bt.short_bytes_host[i] >= 0; }
+    }
+    ctx->obj_stats[4] = solved;
+    return CM_OK;
+}
+
+cm_status cm_objective_stats(const cm_ctx *ctx, uint64_t out[8]) {
+    if (!ctx || !out) return CM_EINVAL;
+    memcpy(out, ctx->obj_stats, sizeof(ctx->obj_stats));
+    return CM_OK;
+}
+
+cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *sizes, const uint8_t *old_lo,
+                               const uint8_t *old_hi, const uint8_t *new_lo, const uint8_t *new_hi,
+                               int64_t *total, uint16_t *assign) {
+    if (!ctx) return CM_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
+    if (n_problems < 0 || (n_problems > 0 && (!sizes || !old_lo || !old_hi || !new_lo || !new_hi || !total)))
+        return fail(ctx, CM_EINVAL, "bad arguments");
+    if (n_problems == 0) return CM_OK;
+    const int L = ctx->hp.L;
+    for (int q = 0; q < n_problems; ++q) {
+        if (sizes[q] < 1 || sizes[q] > CM_MAX_MATCH) return fail(ctx, CM_EINVAL, "problem size must be 1 .. CM_MAX_MATCH");
+        for (int j = 0; j < sizes[q]; ++j) {
+            const size_t i = (size_t)q * CM_MAX_MATCH + j;
+            if (old_lo[i] > L || old_hi[i] > L || new_lo[i] > L || new_hi[i] > L) return fail(ctx, CM_EINVAL, "layer index above L");
+        }
+    }
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    const size_t rows = (size_t)n_problems * CM_MAX_MATCH;
+    const size_t off_sizes = 0, off_rng = ((size_t)n_problems * sizeof(int32_t) + 15) & ~(size_t)15;
+    const size_t off_total = (off_rng + 4 * rows + 15) & ~(size_t)15, off_assign = off_total + (size_t)n_problems * sizeof(int64_t);
+    const size_t bytes = off_assign + rows * sizeof(uint16_t);
+    unsigned char *d = nullptr;
+    CM_CUDA(ctx, cudaMalloc((void **)&d, bytes));
+    cudaStream_t st = ctx->stream;
+    cudaError_t e = cudaMemcpyAsync(d + off_sizes, sizes, (size_t)n_problems * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+    const uint8_t *src[4] = {old_lo, old_hi, new_lo, new_hi};
+    for (int a = 0; a < 4 && e == cudaSuccess; ++a)
+        e = cudaMemcpyAsync(d + off_rng + a * rows, src[a], rows, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = launch_range_matching(tables(ctx, CM_COST_FP64), n_problems, (const int32_t *)(d + off_sizes), d + off_rng,
+                                  d + off_rng + rows, d + off_rng + 2 * rows, d + off_rng + 3 * rows,
+                                  (int64_t *)(d + off_total), (uint16_t *)(d + off_assign), st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(total, d + off_total, (size_t)n_problems * sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && assign) e = cudaMemcpyAsync(assign, d + off_assign, rows * sizeof(uint16_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(d);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
+    for (int q = 0; q < n_problems; ++q)
+        if (total[q] < 0) return fail(ctx, CM_ECUDA, "matching iteration did not terminate");
     return CM_OK;
 }
 

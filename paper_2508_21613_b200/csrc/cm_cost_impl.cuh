@@ -383,7 +383,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_w
     for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
         __syncthreads();
         if (threadIdx.x == 0) {
-            g = seg_view(bd, b, w.seg[p]);
+            g = seg_view(bd, w.scen, w.seg[p]);
             found_so_far = *(volatile uint64_t *)slot;
         }
         __syncthreads();

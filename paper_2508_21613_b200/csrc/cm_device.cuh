@@ -268,6 +268,92 @@ __device__ __forceinline__ bool segment_candidate_cost(const SProf<T> &sp, const
     return pipe_cost_from_cuts<T>(sp, S, g.m, cuts, g.tier, g.n_sync, cost);
 }
 
+// ----------------------------------------------------------------------------------
+// Micro-batch split of a strategy from its rank (Section "Planner", batch distribution).
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ void split_micro(const uint64_t *tab, int batch_mode, int G, const Strat &s,
+                                            uint64_t beta, uint16_t *micro) {
+    const int dp = s.dp;
+    if (batch_mode == CM_BATCH_REMAINDER) {
+        for (int p = 0; p < dp; ++p) micro[p] = s.m_lo[p];
+        unrank_subset(tab, beta, dp, s.R, [&](int, int v) { micro[v] = (uint16_t)(micro[v] + 1); });
+    } else {
+        int cutpos[kMaxP];
+        unrank_subset(tab, beta, G - 1, dp - 1, [&](int pos, int v) { cutpos[pos] = v + 1; });
+        int prev = 0;
+        for (int p = 0; p < dp - 1; ++p) { micro[p] = (uint16_t)(cutpos[p] - prev); prev = cutpos[p]; }
+        micro[dp - 1] = (uint16_t)(G - prev);
+    }
+}
+
+__device__ __forceinline__ bool pair_less(uint64_t c1, uint64_t i1, uint64_t c2, uint64_t i2) {
+    return c1 < c2 || (c1 == c2 && i1 < i2);
+}
+
+// Step time of one (strategy, split) item of a scenario from its per-segment minima `best`
+// (rows in template order): the slowest pipeline's best cost (Section "Estimator": step
+// time = max over pipelines).  inf if a pipeline has no feasible plan.
+__device__ __forceinline__ uint32_t strat_of_item(const BatchDev &bd, const Tmpl &tp, uint64_t item) {
+    uint32_t lo = 0, hi = tp.n_strat - 1;
+    while (lo < hi) {
+        uint32_t mid = (lo + hi + 1) >> 1;
+        if (bd.strat[tp.strat_first + mid].split_first <= item) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ uint64_t item_step_time(const Tables &tb, const BatchDev &bd, const Tmpl &tp,
+                                                   const uint64_t *best, uint64_t item, uint64_t inf) {
+    const Strat &s = bd.strat[tp.strat_first + strat_of_item(bd, tp, item)];
+    uint16_t micro[kMaxP];
+    split_micro(tb.binom, bd.batch_mode, tb.prof->G, s, item - s.split_first, micro);
+    uint64_t T = 0;
+    for (int p = 0; p < s.dp; ++p) {
+        uint64_t c = inf;
+        const int off = (int)micro[p] - (int)s.m_lo[p];
+        if (micro[p] >= 1 && off >= 0 && off < s.n_m) c = best[s.seg_first - tp.tseg_first + p * s.n_m + off];
+        c = c > inf ? inf : c;   // a segment nobody improved still holds its all-ones initial value
+        T = c > T ? c : T;
+    }
+    return T;
+}
+
+// The winner record of an item: strategy, micro-batches and segment rows of its pipelines.
+__device__ __forceinline__ void decode_winner(const Tables &tb, const BatchDev &bd, const Tmpl &tp, uint32_t scen,
+                                              uint64_t cost_bits, uint64_t item, uint64_t inf, Winner &w) {
+    w.cost_bits = cost_bits >= inf ? inf : cost_bits;
+    w.item = item;
+    w.strat = 0;
+    w.dp = 0;
+    w.scen = scen;
+    w.pad = 0;
+    for (int p = 0; p < kMaxP; ++p) { w.seg[p] = 0; w.micro[p] = 0; }
+    if (cost_bits < inf) {
+        const uint32_t si = strat_of_item(bd, tp, item);
+        const Strat &s = bd.strat[tp.strat_first + si];
+        w.strat = tp.strat_first + si;
+        w.dp = s.dp;
+        split_micro(tb.binom, bd.batch_mode, tb.prof->G, s, item - s.split_first, w.micro);
+        for (int p = 0; p < s.dp; ++p) w.seg[p] = s.seg_first + p * s.n_m + (w.micro[p] - s.m_lo[p]);
+    }
+}
+
+__device__ __forceinline__ void plan_clear(cm_plan &pl, int policy) {
+    pl.policy = policy;
+    pl.feasible = 0;
+    pl.cost = 0.0;
+    pl.cost_ns = 0;
+    pl.strategy = 0;
+    pl.n_pipes = 0;
+    pl.split_rank = 0;
+    for (int p = 0; p < kMaxP; ++p) { pl.stages[p] = 0; pl.micro[p] = 0; pl.kappa[p] = 0; }
+}
+
+__device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mode) {
+    if (mode == CM_COST_INT64NS) pl.cost_ns = (int64_t)bits;
+    else pl.cost = __longlong_as_double((long long)bits);
+}
+
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {
     for (int o = 16; o > 0; o >>= 1) {
         uint64_t w = __shfl_xor_sync(0xffffffffu, v, o);

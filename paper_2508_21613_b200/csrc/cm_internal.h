@@ -26,6 +26,7 @@ struct DevProfile {
     double PFd[kMaxL + 1], PBd[kMaxL + 1];
     int64_t PFi[kMaxL + 1], PBi[kMaxL + 1];
     int64_t PA[kMaxL + 1], PS[kMaxL + 1], PP[kMaxL + 1];
+    int64_t PW[kMaxL + 1];  // parameters + optimizer state: what a migration moves per layer
     double XTd[2][kMaxL];   // transfer time of the boundary after layer l: [0] intra, [1] inter
     int64_t XTi[2][kMaxL];
     int32_t base_cuts[kMaxS + 1];
@@ -121,6 +122,7 @@ struct Winner {
     uint32_t strat, dp;     // global strategy row; pipelines
     uint32_t seg[kMaxP];    // global segment row of every pipeline
     uint16_t micro[kMaxP];
+    uint32_t scen, pad;     // scenario it belongs to (a shortlist holds several records per scenario)
 };
 
 struct BatchDev {
@@ -159,6 +161,24 @@ struct Tables {
     __host__ __device__ uint32_t mm_slot(int S, int m) const { return (uint32_t)((S - 1) * mm_stride_m + m); }
 };
 
+// Full objective (transition time included): per scenario a shortlist of the `topk` best
+// (strategy, split) pairs by step time, each completed to a plan and matched against the old
+// placement.  Slot = scenario * topk + rank.
+constexpr int kMaxShort = CM_MAX_SHORTLIST;
+constexpr int kMaxMatch = CM_MAX_MATCH;
+struct ObjDev {
+    int32_t topk, pad;
+    double t_gap, t_restart;
+    int64_t t_gap_i, t_restart_i, bw_xfer;
+    Winner *short_win;        // [B*topk]
+    uint64_t *short_kappa;    // [B*topk][kMaxP]
+    int64_t *short_bytes;     // [B*topk] bytes moved by the cheapest migration, -1 = empty slot
+    uint16_t *short_assign;   // [B*topk][kMaxMatch] position -> survivor index
+    cm_plan *short_plans;     // [B*topk] or NULL
+    cm_plan *best;            // [B]
+    cm_transition *trans;     // [B]
+};
+
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
@@ -193,6 +213,14 @@ cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st)
 cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand, int single_policy,
                             uint64_t first, uint64_t count, const uint64_t *idx, double *cost,
                             int64_t *cost_ns, uint8_t *feas, cudaStream_t st);
+// cm_restore.cu
+cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
+cudaError_t launch_plan_matching(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
+cudaError_t launch_objective(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
+// stand-alone matchings over explicit layer ranges ([n_problems][kMaxMatch] each)
+cudaError_t launch_range_matching(const Tables &t, int n_problems, const int32_t *sizes, const uint8_t *old_lo,
+                                  const uint8_t *old_hi, const uint8_t *new_lo, const uint8_t *new_hi,
+                                  int64_t *total, uint16_t *assign, cudaStream_t st);
 cudaError_t launch_pick(const cm_plan *const *plans_dev, int n, cm_plan *out_dev, int mode, cudaStream_t st);
 
 // What an entry point implemented outside cm_api.cu needs to know about a space.

@@ -29,6 +29,7 @@ __global__ void cm_prefix_kernel(DevProfile *p) {
     case 4: { int64_t a = 0; p->PA[0] = a; for (int l = 0; l < L; ++l) { a += p->act[l]; p->PA[l + 1] = a; } break; }
     case 5: { int64_t a = 0; p->PS[0] = a; for (int l = 0; l < L; ++l) { a += 2 * p->par[l] + p->opt[l]; p->PS[l + 1] = a; } break; }
     case 6: { int64_t a = 0; p->PP[0] = a; for (int l = 0; l < L; ++l) { a += p->par[l]; p->PP[l + 1] = a; } break; }
+    case 7: { int64_t a = 0; p->PW[0] = a; for (int l = 0; l < L; ++l) { a += p->par[l] + p->opt[l]; p->PW[l + 1] = a; } break; }
     default: break;
     }
     for (int l = threadIdx.x; l < L; l += blockDim.x) {
@@ -143,28 +144,6 @@ __device__ __forceinline__ uint32_t find_row(const TSeg *seg, uint32_t n, uint64
 }
 
 // ----------------------------------------------------------------------------------
-// Micro-batch split of a strategy from its rank (Section "Planner", batch distribution).
-// ----------------------------------------------------------------------------------
-__device__ __forceinline__ void split_micro(const uint64_t *tab, int batch_mode, int G, const Strat &s,
-                                            uint64_t beta, uint16_t *micro) {
-    const int dp = s.dp;
-    if (batch_mode == CM_BATCH_REMAINDER) {
-        for (int p = 0; p < dp; ++p) micro[p] = s.m_lo[p];
-        unrank_subset(tab, beta, dp, s.R, [&](int, int v) { micro[v] = (uint16_t)(micro[v] + 1); });
-    } else {
-        int cutpos[kMaxP];
-        unrank_subset(tab, beta, G - 1, dp - 1, [&](int pos, int v) { cutpos[pos] = v + 1; });
-        int prev = 0;
-        for (int p = 0; p < dp - 1; ++p) { micro[p] = (uint16_t)(cutpos[p] - prev); prev = cutpos[p]; }
-        micro[dp - 1] = (uint16_t)(G - prev);
-    }
-}
-
-__device__ __forceinline__ bool pair_less(uint64_t c1, uint64_t i1, uint64_t c2, uint64_t i2) {
-    return c1 < c2 || (c1 == c2 && i1 < i2);
-}
-
-// ----------------------------------------------------------------------------------
 // Split reduction: item = (strategy, split rank) of one scenario; its step time is the
 // slowest pipeline's best cost (Section "Estimator": step time = max over pipelines).
 // Hierarchical argmin carrying (cost, item) with the lowest item on ties:
@@ -177,28 +156,11 @@ __global__ void __launch_bounds__(256) cm_split_kernel(Tables tb, BatchDev bd, u
     const Scen sc = bd.scen[b];
     const Tmpl tp = bd.tmpl[sc.tmpl];
     const uint32_t local = blockIdx.x - sc.red_first;
-    const int G = tb.prof->G;
     const uint64_t *best = bd.seg_best + sc.seg_base;   // this scenario's rows, in template order
     uint64_t best_c = inf, best_i = ~0ull;
     for (uint64_t item = (uint64_t)local * blockDim.x + threadIdx.x; item < tp.n_split_total;
          item += (uint64_t)tp.n_red * blockDim.x) {
-        // strategy that owns the item
-        uint32_t lo = 0, hi = tp.n_strat - 1;
-        while (lo < hi) {
-            uint32_t mid = (lo + hi + 1) >> 1;
-            if (bd.strat[tp.strat_first + mid].split_first <= item) lo = mid; else hi = mid - 1;
-        }
-        const Strat &s = bd.strat[tp.strat_first + lo];
-        uint16_t micro[kMaxP];
-        split_micro(tb.binom, bd.batch_mode, G, s, item - s.split_first, micro);
-        uint64_t T = 0;
-        for (int p = 0; p < s.dp; ++p) {
-            uint64_t c = inf;
-            const int off = (int)micro[p] - (int)s.m_lo[p];
-            if (micro[p] >= 1 && off >= 0 && off < s.n_m) c = best[s.seg_first - tp.tseg_first + p * s.n_m + off];
-            c = c > inf ? inf : c;   // a segment nobody improved still holds its all-ones initial value
-            T = c > T ? c : T;
-        }
+        const uint64_t T = item_step_time(tb, bd, tp, best, item, inf);
         if (pair_less(T, item, best_c, best_i)) { best_c = T; best_i = item; }
     }
     for (int o = 16; o > 0; o >>= 1) {
@@ -235,24 +197,7 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
     if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
     if (threadIdx.x == 0) {
         Winner w;
-        w.cost_bits = best_c >= inf ? inf : best_c;
-        w.item = best_i;
-        w.strat = 0;
-        w.dp = 0;
-        for (int p = 0; p < kMaxP; ++p) { w.seg[p] = 0; w.micro[p] = 0; }
-        if (best_c < inf) {
-            uint32_t lo = 0, hi = tp.n_strat - 1;
-            while (lo < hi) {
-                uint32_t mid = (lo + hi + 1) >> 1;
-                if (bd.strat[tp.strat_first + mid].split_first <= best_i) lo = mid; else hi = mid - 1;
-            }
-            const Strat &s = bd.strat[tp.strat_first + lo];
-            w.strat = tp.strat_first + lo;
-            w.dp = s.dp;
-            split_micro(tb.binom, bd.batch_mode, tb.prof->G, s, best_i - s.split_first, w.micro);
-            // template segment rows of the winner's pipelines
-            for (int p = 0; p < s.dp; ++p) w.seg[p] = s.seg_first + p * s.n_m + (w.micro[p] - s.m_lo[p]);
-        }
+        decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
     }
 }
@@ -297,7 +242,7 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
         __syncthreads();
         if (threadIdx.x == 0) {
-            g = seg_view(bd, b, w.seg[p]);
+            g = seg_view(bd, w.scen, w.seg[p]);
             found_so_far = *(volatile uint64_t *)slot;
         }
         __syncthreads();
@@ -340,22 +285,6 @@ cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t s
 // Assemble the per-policy plans and the overall best: least cost, ties to the lowest
 // policy id (Algorithm 1 keeps the plan with the least estimated time).
 // ----------------------------------------------------------------------------------
-__device__ __forceinline__ void plan_clear(cm_plan &pl, int policy) {
-    pl.policy = policy;
-    pl.feasible = 0;
-    pl.cost = 0.0;
-    pl.cost_ns = 0;
-    pl.strategy = 0;
-    pl.n_pipes = 0;
-    pl.split_rank = 0;
-    for (int p = 0; p < kMaxP; ++p) { pl.stages[p] = 0; pl.micro[p] = 0; pl.kappa[p] = 0; }
-}
-
-__device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mode) {
-    if (mode == CM_COST_INT64NS) pl.cost_ns = (int64_t)bits;
-    else pl.cost = __longlong_as_double((long long)bits);
-}
-
 __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b == 0) {

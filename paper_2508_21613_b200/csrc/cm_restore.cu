@@ -1,0 +1,385 @@
+// Transition time and the full objective (sm_100a).
+//
+//   cm_shortlist_kernel       per scenario: the topk (strategy, split) pairs of least step time
+//   (the tie-break kernels then complete every shortlisted pair to a plan)
+//   cm_plan_matching_kernel   one warp per shortlisted plan: layer ranges of the survivors
+//                             before and after, minimum-cost perfect matching
+//   cm_range_matching_kernel  the same matching over caller-given layer ranges
+//   cm_objective_kernel       per scenario: steps before the next fault of every candidate,
+//                             the best one, its plan and its migration scheme
+//
+// Section "Restorer", Weight Transfer: the N x N cost matrix is never stored.  Old and new
+// holdings are contiguous layer ranges, so Cost[i][j] = W(new_j) - W(new_j ∩ old_i) is two
+// prefix differences; a warp keeps the potentials of the Kuhn-Munkres iteration in shared
+// memory, its lanes share the columns, and the argmin over the columns is a shuffle
+// reduction carrying (slack, column) with the lowest column on ties.
+#include <climits>
+
+#include "cm_device.cuh"
+
+namespace cm {
+
+// ----------------------------------------------------------------------------------
+// Shortlist: topk rounds of a block-wide argmin over the scenario's (strategy, split)
+// items; round r takes the least (step time, item) pair that comes after round r-1's.
+// ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) cm_shortlist_kernel(Tables tb, BatchDev bd, ObjDev od, uint64_t inf) {
+    __shared__ uint64_t rc[8], ri[8];
+    __shared__ uint64_t last_c, last_i;
+    const uint32_t b = blockIdx.x;
+    const Scen sc = bd.scen[b];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
+    const uint64_t *best = bd.seg_best + sc.seg_base;
+    const bool searched = (sc.policy_mask & (1u << CM_DYNPAR)) != 0;
+    bool exhausted = !searched || tp.n_split_total == 0;
+    for (int r = 0; r < od.topk; ++r) {
+        uint64_t best_c = inf, best_i = ~0ull;
+        if (!exhausted) {
+            const uint64_t lc = r ? last_c : 0, li = r ? last_i : 0;
+            for (uint64_t item = threadIdx.x; item < tp.n_split_total; item += blockDim.x) {
+                const uint64_t T = item_step_time(tb, bd, tp, best, item, inf);
+                if (T >= inf) continue;
+                if (r && !pair_less(lc, li, T, item)) continue;     // taken by an earlier round
+                if (pair_less(T, item, best_c, best_i)) { best_c = T; best_i = item; }
+            }
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            uint64_t oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+            uint64_t oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+            if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
+        }
+        __syncthreads();   // everybody has read last_c / last_i of the previous round
+        if ((threadIdx.x & 31) == 0) { rc[threadIdx.x >> 5] = best_c; ri[threadIdx.x >> 5] = best_i; }
+        __syncthreads();
+        const size_t slot = (size_t)b * od.topk + r;
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < 8; ++w)
+                if (pair_less(rc[w], ri[w], best_c, best_i)) { best_c = rc[w]; best_i = ri[w]; }
+            last_c = best_c;
+            last_i = best_i;
+            Winner w;
+            decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
+            od.short_win[slot] = w;
+            od.short_bytes[slot] = -1;
+        }
+        if (threadIdx.x < kMaxP) od.short_kappa[slot * kMaxP + threadIdx.x] = ~0ull;
+        __syncthreads();
+        if (last_c >= inf) exhausted = true;   // uniform: nothing is left for later rounds either
+    }
+}
+
+cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    cm_shortlist_kernel<<<b.B, 256, 0, st>>>(t, b, o, inf);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Minimum-cost perfect matching, one warp per problem (Kuhn-Munkres in its potentials /
+// shortest-augmenting-path form).  Rows = devices with their old layer range, columns =
+// positions with their new range.  Rows enter one at a time; for the new row an
+// alternating tree is grown column by column over the reduced costs
+// cost(i,j) - u[i] - v[j], potentials are shifted so that tree edges stay tight, and the
+// matching is flipped along the path to the first free column.  Every loop is bounded by
+// the problem size: the tree gains a column per step and a free column always exists.
+// ----------------------------------------------------------------------------------
+constexpr int kMatchWarps = 4;
+
+struct MatchWork {
+    long long u[kMaxMatch], v[kMaxMatch], slack[kMaxMatch], need[kMaxMatch];
+    short match[kMaxMatch], prev[kMaxMatch];
+    uint8_t olo[kMaxMatch], ohi[kMaxMatch], nlo[kMaxMatch], nhi[kMaxMatch];
+};
+
+__device__ __forceinline__ long long match_cost(const MatchWork &w, const long long *PW, int row, int j) {
+    const int lo = max((int)w.olo[row], (int)w.nlo[j]), hi = min((int)w.ohi[row], (int)w.nhi[j]);
+    return w.need[j] - (hi > lo ? PW[hi] - PW[lo] : 0ll);
+}
+
+// Returns the total of the matching (same value in every lane), -1 if the iteration broke
+// down (cannot happen for n >= 1; guards the loops).  w.match[j] = row of column j.
+__device__ long long warp_match(MatchWork &w, const long long *PW, int n, int lane) {
+    const long long INF = LLONG_MAX / 4;
+    for (int j = lane; j < n; j += 32) {
+        w.u[j] = 0;
+        w.v[j] = 0;
+        w.match[j] = -1;
+        const int x = w.nlo[j], y = w.nhi[j];
+        w.need[j] = y > x ? PW[y] - PW[x] : 0ll;
+    }
+    __syncwarp();
+    bool broken = false;
+    for (int r = 0; r < n && !broken; ++r) {
+        for (int j = lane; j < n; j += 32) { w.slack[j] = INF; w.prev[j] = (short)n; }
+        uint32_t tree = 0;            // bit c: column c*32+lane belongs to the tree
+        int col = n, row = r;         // column n is the root and holds the new row
+        for (int step = 0; step <= n; ++step) {
+            const int a = w.olo[row], b = w.ohi[row];
+            const long long ur = w.u[row];
+            long long delta = INF;
+            int next = n;
+            for (int c = 0, j = lane; j < n; ++c, j += 32) {
+                if ((tree >> c) & 1u) continue;
+                const int lo = max(a, (int)w.nlo[j]), hi = min(b, (int)w.nhi[j]);
+                const long long cost = w.need[j] - (hi > lo ? PW[hi] - PW[lo] : 0ll);
+                const long long red = cost - ur - w.v[j];
+                long long s = w.slack[j];
+                if (red < s) { s = red; w.slack[j] = s; w.prev[j] = (short)col; }
+                if (s < delta) { delta = s; next = j; }
+            }
+            for (int o = 16; o > 0; o >>= 1) {
+                const long long od = __shfl_xor_sync(0xffffffffu, delta, o);
+                const int on = __shfl_xor_sync(0xffffffffu, next, o);
+                if (od < delta || (od == delta && on < next)) { delta = od; next = on; }
+            }
+            if (next >= n) { broken = true; break; }
+            for (int c = 0, j = lane; j < n; ++c, j += 32) {
+                if ((tree >> c) & 1u) { w.u[w.match[j]] += delta; w.v[j] -= delta; }
+                else w.slack[j] -= delta;
+            }
+            if (lane == 0) w.u[r] += delta;
+            __syncwarp();
+            col = next;
+            if ((col & 31) == lane) tree |= 1u << (col >> 5);
+            row = w.match[col];
+            if (row < 0) break;
+        }
+        if (row >= 0) broken = true;   // step bound hit without reaching a free column
+        if (!broken && lane == 0) {
+            int c = col;
+            for (int step = 0; step <= n && c != n; ++step) {
+                const int p = w.prev[c];
+                w.match[c] = p == n ? (short)r : w.match[p];
+                c = p;
+            }
+        }
+        __syncwarp();
+    }
+    if (broken) return -1;
+    long long total = 0;
+    for (int j = lane; j < n; j += 32) total += match_cost(w, PW, w.match[j], j);
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    return total;
+}
+
+__device__ __forceinline__ void stage_state_bytes(long long *PW, const DevProfile *p) {
+    for (int l = threadIdx.x; l <= p->L; l += blockDim.x) PW[l] = p->PW[l];
+    __syncthreads();
+}
+
+// One warp per shortlist slot: survivors keep the layers of their old stage (device =
+// pipeline * n_pp + stage); position off_p + i of the plan holds stage i of pipeline p.
+__global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_matching_kernel(Tables tb, BatchDev bd, ObjDev od, uint64_t inf) {
+    __shared__ MatchWork work[kMatchWarps];
+    __shared__ long long PW[kMaxL + 1];
+    const DevProfile *p = tb.prof;
+    stage_state_bytes(PW, p);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t slot = (size_t)blockIdx.x * kMatchWarps + warp;
+    if (slot >= (size_t)bd.B * od.topk) return;
+    const Winner &w = od.short_win[slot];
+    if (w.cost_bits >= inf || w.dp == 0) return;            // empty slot: bytes stay -1
+    MatchWork &mw = work[warp];
+    const Scen sc = bd.scen[w.scen];
+    const int N = p->n_dp * p->n_pp, n_pp = p->n_pp;
+    int n = 0;
+    for (int base = 0; base < N; base += 32) {
+        const int d = base + lane;
+        bool alive = d < N;
+        for (uint32_t f = 0; f < sc.n_failed; ++f) alive = alive && bd.failed[sc.failed_first + f] != (uint32_t)d;
+        const uint32_t mask = __ballot_sync(0xffffffffu, alive);
+        const int idx = n + __popc(mask & ((1u << lane) - 1u));
+        if (alive && idx < kMaxMatch) {
+            mw.olo[idx] = (uint8_t)p->base_cuts[d % n_pp];
+            mw.ohi[idx] = (uint8_t)p->base_cuts[d % n_pp + 1];
+        }
+        n += __popc(mask);
+    }
+    bool ok = n >= 1 && n <= kMaxMatch;
+    int covered = 0;
+    if (ok && lane < (int)w.dp) {
+        const Strat &s = bd.strat[w.strat];
+        int off = 0;
+        for (int q = 0; q < lane; ++q) off += s.S[q];
+        const TSeg g = bd.tseg[w.seg[lane]];
+        const uint64_t kappa = od.short_kappa[slot * kMaxP + lane];
+        const int S = g.S;
+        uint8_t cuts[kMaxS + 1];
+        if (off + S > n) ok = false;
+        else if (kappa < g.K) layer_cuts(tb.binom, bd.layer_mode, p->L, S, kappa, cuts);
+        else if (kappa == g.K) {
+            const uint8_t *mm = tb.mm_cuts + (size_t)tb.mm_slot(S, g.m) * (kMaxS + 1);
+            if (mm[0] != 0) ok = false;
+            else for (int i = 0; i <= S; ++i) cuts[i] = mm[i];
+        } else ok = false;                                   // no composition met the step time
+        if (ok) {
+            for (int i = 0; i < S; ++i) { mw.nlo[off + i] = cuts[i]; mw.nhi[off + i] = cuts[i + 1]; }
+            covered = S;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) covered += __shfl_xor_sync(0xffffffffu, covered, o);
+    ok = __all_sync(0xffffffffu, ok) && covered == n;       // a strategy uses every survivor
+    __syncwarp();
+    if (!ok) return;
+    const long long total = warp_match(mw, PW, n, lane);
+    if (total < 0) return;
+    uint16_t *asg = od.short_assign + slot * kMaxMatch;
+    for (int j = lane; j < kMaxMatch; j += 32) asg[j] = j < n ? (uint16_t)mw.match[j] : (uint16_t)0;
+    if (lane == 0) od.short_bytes[slot] = total;
+}
+
+cudaError_t launch_plan_matching(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const size_t slots = (size_t)b.B * o.topk;
+    cm_plan_matching_kernel<<<(unsigned)((slots + kMatchWarps - 1) / kMatchWarps), kMatchWarps * 32, 0, st>>>(t, b, o, inf);
+    return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(kMatchWarps * 32) cm_range_matching_kernel(Tables tb, int n_problems, const int32_t *sizes,
+                                                                             const uint8_t *old_lo, const uint8_t *old_hi,
+                                                                             const uint8_t *new_lo, const uint8_t *new_hi,
+                                                                             int64_t *total, uint16_t *assign) {
+    __shared__ MatchWork work[kMatchWarps];
+    __shared__ long long PW[kMaxL + 1];
+    stage_state_bytes(PW, tb.prof);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int q = blockIdx.x * kMatchWarps + warp;
+    if (q >= n_problems) return;
+    MatchWork &mw = work[warp];
+    const int n = sizes[q], L = tb.prof->L;
+    const size_t base = (size_t)q * kMaxMatch;
+    for (int j = lane; j < n; j += 32) {
+        mw.olo[j] = (uint8_t)min((int)old_lo[base + j], L); mw.ohi[j] = (uint8_t)min((int)old_hi[base + j], L);
+        mw.nlo[j] = (uint8_t)min((int)new_lo[base + j], L); mw.nhi[j] = (uint8_t)min((int)new_hi[base + j], L);
+    }
+    __syncwarp();
+    const long long t = warp_match(mw, PW, n, lane);
+    if (lane == 0) total[q] = t;
+    if (assign)
+        for (int j = lane; j < kMaxMatch; j += 32) assign[base + j] = (j < n && t >= 0) ? (uint16_t)mw.match[j] : (uint16_t)0;
+}
+
+cudaError_t launch_range_matching(const Tables &t, int n_problems, const int32_t *sizes, const uint8_t *old_lo,
+                                  const uint8_t *old_hi, const uint8_t *new_lo, const uint8_t *new_hi,
+                                  int64_t *total, uint16_t *assign, cudaStream_t st) {
+    if (n_problems <= 0) return cudaSuccess;
+    cm_range_matching_kernel<<<(n_problems + kMatchWarps - 1) / kMatchWarps, kMatchWarps * 32, 0, st>>>(
+        t, n_problems, sizes, old_lo, old_hi, new_lo, new_hi, total, assign);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Objective (Section "Problem Formulation"): steps before the next fault,
+// (t_gap - t_trans) / t_step, of rerouting, redundant computation (t_trans = 0) and every
+// shortlisted plan (t_trans = restart + matched bytes / bandwidth).  The greatest wins,
+// ties to the lower policy id, then to the earlier rank.  fp64: the quotients are compared
+// as rounded; int64: fractions are compared exactly by cross-multiplication.
+// ----------------------------------------------------------------------------------
+struct Frac {
+    double nd, dd;          // fp64 mode
+    long long ni, di;       // int64 mode
+};
+
+__device__ __forceinline__ bool frac_greater(const Frac &a, const Frac &b, int mode) {
+    if (mode == CM_COST_INT64NS) return (__int128)a.ni * (__int128)b.di > (__int128)b.ni * (__int128)a.di;
+    return a.nd / a.dd > b.nd / b.dd;
+}
+
+__device__ __forceinline__ void plan_from_winner(const BatchDev &bd, const Winner &w, const uint64_t *kappa, cm_plan &pl) {
+    plan_clear(pl, CM_DYNPAR);
+    const Strat &s = bd.strat[w.strat];
+    pl.feasible = 1;
+    plan_set_cost(pl, w.cost_bits, bd.mode);
+    pl.strategy = w.strat - bd.tmpl[bd.scen[w.scen].tmpl].strat_first;
+    pl.n_pipes = w.dp;
+    pl.split_rank = w.item - s.split_first;
+    for (uint32_t q = 0; q < w.dp; ++q) {
+        pl.stages[q] = s.S[q];
+        pl.micro[q] = w.micro[q];
+        pl.kappa[q] = kappa[q];
+    }
+}
+
+__global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd, ObjDev od, uint64_t inf) {
+    __shared__ int win_slot;
+    const uint32_t b = blockIdx.x;
+    const int mode = bd.mode;
+    const cm_plan *pol = bd.plans + (size_t)b * 4;
+    if (threadIdx.x == 0) {
+        cm_transition tr;
+        tr.policy = 0; tr.feasible = 0; tr.rank = -1;
+        tr.n_survivors = tb.prof->n_dp * tb.prof->n_pp - (int)bd.scen[b].n_failed;
+        tr.xfer_bytes = 0; tr.t_trans = 0.0; tr.t_trans_ns = 0; tr.objective = 0.0;
+        Frac best{0.0, 1.0, 0, 1};
+        bool have = false;
+        int slot_sel = -1;
+        for (int q = 0; q < 2; ++q) {
+            if (!pol[q].feasible) continue;
+            Frac j{od.t_gap, pol[q].cost, od.t_gap_i, pol[q].cost_ns};
+            if (!have || frac_greater(j, best, mode)) { have = true; best = j; tr.policy = q; }
+        }
+        for (int r = 0; r < od.topk; ++r) {
+            const size_t slot = (size_t)b * od.topk + r;
+            const long long bytes = od.short_bytes[slot];
+            if (bytes < 0) continue;
+            const Winner &w = od.short_win[slot];
+            Frac j{0.0, 1.0, 0, 1};
+            double tt = 0.0;
+            long long tti = 0;
+            if (mode == CM_COST_INT64NS) {
+                tti = od.t_restart_i + bytes / od.bw_xfer;
+                j.ni = od.t_gap_i - tti;
+                j.di = (long long)w.cost_bits;
+            } else {
+                tt = od.t_restart + (double)bytes / (double)od.bw_xfer;
+                j.nd = od.t_gap - tt;
+                j.dd = __longlong_as_double((long long)w.cost_bits);
+            }
+            if (!have || frac_greater(j, best, mode)) {
+                have = true; best = j; slot_sel = (int)r;
+                tr.policy = CM_DYNPAR; tr.rank = r; tr.xfer_bytes = bytes; tr.t_trans = tt; tr.t_trans_ns = tti;
+            }
+        }
+        cm_plan pl;
+        if (!have) plan_clear(pl, 0);
+        else if (tr.policy != CM_DYNPAR) {
+            pl = pol[tr.policy];
+            tr.rank = -1; tr.xfer_bytes = 0; tr.t_trans = 0.0; tr.t_trans_ns = 0;
+        } else {
+            const size_t slot = (size_t)b * od.topk + slot_sel;
+            plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, pl);
+        }
+        if (have) {
+            tr.feasible = 1;
+            tr.objective = mode == CM_COST_INT64NS ? (double)best.ni / (double)best.di : best.nd / best.dd;
+        }
+        od.best[b] = pl;
+        // header of the transition record; the matching follows from all lanes
+        cm_transition *out = od.trans + b;
+        out->policy = tr.policy; out->feasible = tr.feasible; out->rank = tr.rank; out->n_survivors = tr.n_survivors;
+        out->xfer_bytes = tr.xfer_bytes; out->t_trans = tr.t_trans; out->t_trans_ns = tr.t_trans_ns;
+        out->objective = tr.objective;
+        win_slot = (have && tr.policy == CM_DYNPAR) ? slot_sel : -1;
+    }
+    __syncthreads();
+    const uint16_t *src = win_slot >= 0 ? od.short_assign + ((size_t)b * od.topk + win_slot) * kMaxMatch : nullptr;
+    for (int j = threadIdx.x; j < kMaxMatch; j += 32) od.trans[b].assign[j] = src ? src[j] : (uint16_t)0;
+    if (od.short_plans && (int)threadIdx.x < od.topk) {
+        const size_t slot = (size_t)b * od.topk + threadIdx.x;
+        cm_plan pl;
+        if (od.short_bytes[slot] >= 0) plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, pl);
+        else plan_clear(pl, CM_DYNPAR);
+        od.short_plans[slot] = pl;
+    }
+}
+
+cudaError_t launch_objective(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    cm_objective_kernel<<<b.B, 32, 0, st>>>(t, b, o, inf);
+    return cudaGetLastError();
+}
+
+}  // namespace cm
