@@ -242,6 +242,57 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
     return out
 
 
+def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush):
+    """The full-objective search (search + shortlist + weight-transfer matchings + ranking by
+    steps before the next fault) through cm_search_objective, host buffers in and out."""
+    from paper_2508_21613_b200 import workloads as W
+    opts = w.options.with_cost_mode(mode)
+    obj = W.ObjectiveOptions()
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    packed = binding.PackedScenarios(w.scenarios)
+    try:
+        for _ in range(warmup):
+            res = packed.search_objective(ctx, opts, obj, shortlist=True)
+        wall, phases = 0.0, {}
+        search_ns = 0
+        for k in range(steps):
+            flush.fill_(float(k))
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            res = packed.search_objective(ctx, opts, obj, shortlist=True)
+            wall += time.perf_counter() - t0
+            for key, v in binding.cm_objective_stats(ctx).items():
+                phases[key] = phases.get(key, 0) + v
+            search_ns += binding.cm_last_stats(ctx)["device_ns"]
+        best, trans, _, sb = res
+        packed.search(ctx, opts)
+        plain = packed.best
+        policies = [0, 0, 0]
+        changed = 0
+        for b in range(packed.B):
+            policies[trans[b].policy] += 1
+            changed += int(plain[b].policy != best[b].policy or plain[b].strategy != best[b].strategy
+                           or plain[b].split_rank != best[b].split_rank)
+        matchings = int((sb >= 0).sum())
+        return {
+            "topk": obj.topk, "t_gap_s": obj.t_gap_ns * 1e-9, "t_restart_s": obj.t_restart_ns * 1e-9,
+            "bw_xfer_GBps": obj.bw_xfer_Bpns, "scenarios": packed.B,
+            "e2e_ms_per_call": 1e3 * wall / steps,
+            "search_device_ms": 1e-6 * search_ns / steps,
+            "objective_pass_device_ms": 1e-6 * phases["device_ns"] / steps,
+            "phase_ms": {k[:-3]: 1e-6 * phases[k] / steps for k in ("shortlist_ns", "complete_ns", "matching_ns", "objective_ns")},
+            "matchings_per_call": matchings,
+            "matchings_per_s": matchings / (1e-9 * phases["matching_ns"] / steps) if phases["matching_ns"] else None,
+            "devices_per_matching": int(trans[0].n_survivors),
+            "chosen_policy_counts": {"reroute": policies[0], "redundant": policies[1], "dynpar": policies[2]},
+            "choices_changed_by_transition_time": changed,
+            "gpu_launches": int(phases["launches"] / steps),
+        }
+    finally:
+        binding.cm_destroy(ctx)
+
+
 def roofline_of(stats_sum, dev_seconds, mode, sm_max, peak_kind):
     slots = ISSUE_SLOTS_PER_CELL[mode]
     peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
@@ -360,6 +411,10 @@ def main():
                     "latency_scenarios": em["latency_us"]["scenarios"],
                     "search_pass_gcell_s": r["achieved"], "search_pass_frac": r["frac"]}
             line["workloads"] = extra
+            # widening beyond the plan search: transition time in the objective
+            line["full_objective"] = {
+                name: measure_objective(binding, torch, W.ALL_WORKLOADS[name](), args.cost_mode, 3, 3, local_rank, flush)
+                for name in dict.fromkeys((args.workload, "175b-like", "sweep"))}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -224,6 +224,21 @@ def test_objective_parity_deep_pipelines_sampled(gpu, oracle_factory):
         s.close()
 
 
+def test_objective_parity_255_device_matchings(gpu, oracle_factory):
+    # 175B-like grid: 256 devices, matchings of 248 and 255 survivors inside the search
+    w = W.gpt175b_like()
+    opts = w.options
+    o = oracle_factory(w.profile, opts)
+    s = Session(gpu, w.profile)
+    try:
+        obj = W.ObjectiveOptions(topk=3)
+        scen = [w.scenarios[0], w.scenarios[40]]
+        res = gpu.cm_search_objective(s.ctx, scen, opts, obj, shortlist=True)
+        _check_objective(gpu, o, w, scen, opts, obj, 0, res)
+    finally:
+        s.close()
+
+
 def test_objective_limits_and_errors(gpu):
     w = W.paper_scale(2, 2)
     s = Session(gpu, w.profile)
