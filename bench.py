@@ -329,6 +329,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads / cost mode summary")
     ap.add_argument("--scenarios", type=int, default=0, help="use only the first N scenarios (profiling runs)")
+    ap.add_argument("--objective", action="store_true",
+                    help="also time the full-objective search on the selected workload (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -415,6 +417,9 @@ def main():
             line["full_objective"] = {
                 name: measure_objective(binding, torch, W.ALL_WORKLOADS[name](), args.cost_mode, 3, 3, local_rank, flush)
                 for name in dict.fromkeys((args.workload, "175b-like", "sweep"))}
+        if args.objective and "full_objective" not in line:
+            line["full_objective"] = {w.name: measure_objective(binding, torch, w, args.cost_mode, args.steps,
+                                                                args.warmup, local_rank, flush)}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -11,8 +11,9 @@
 // Section "Restorer", Weight Transfer: the N x N cost matrix is never stored.  Old and new
 // holdings are contiguous layer ranges, so Cost[i][j] = W(new_j) - W(new_j ∩ old_i) is two
 // prefix differences; a warp keeps the potentials of the Kuhn-Munkres iteration in shared
-// memory, its lanes share the columns, and the argmin over the columns is a shuffle
-// reduction carrying (slack, column) with the lowest column on ties.
+// memory, its lanes share the columns (their potentials and slacks stay in registers), and
+// the argmin over the columns is a shuffle reduction carrying (slack, column) with the
+// lowest column on ties.
 #include <climits>
 
 #include "cm_device.cuh"
@@ -87,31 +88,66 @@ cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o
 constexpr int kMatchWarps = 4;
 
 struct MatchWork {
-    long long u[kMaxMatch], v[kMaxMatch], slack[kMaxMatch], need[kMaxMatch];
-    short match[kMaxMatch], prev[kMaxMatch];
+    long long u[kMaxMatch];                       // row potentials
+    short match[kMaxMatch], prev[kMaxMatch];      // row of a column (-1 = free); previous column on the path
+    int row_col[kMaxMatch];                       // column of a row (-1 = free); claimed with atomicCAS
     uint8_t olo[kMaxMatch], ohi[kMaxMatch], nlo[kMaxMatch], nhi[kMaxMatch];
 };
 
-__device__ __forceinline__ long long match_cost(const MatchWork &w, const long long *PW, int row, int j) {
-    const int lo = max((int)w.olo[row], (int)w.nlo[j]), hi = min((int)w.ohi[row], (int)w.nhi[j]);
-    return w.need[j] - (hi > lo ? PW[hi] - PW[lo] : 0ll);
+__device__ __forceinline__ long long range_cost(const long long *PW, long long need, int a, int b, int x, int y) {
+    const int lo = max(a, x), hi = min(b, y);
+    return need - (hi > lo ? PW[hi] - PW[lo] : 0ll);
 }
 
 // Returns the total of the matching (same value in every lane), -1 if the iteration broke
 // down (cannot happen for n >= 1; guards the loops).  w.match[j] = row of column j.
+// Lane `lane` owns the columns c*32+lane, c < NC, and keeps their range, column potential
+// and slack in registers; rows are read from shared memory (same address in every lane).
+template <int NC>
 __device__ long long warp_match(MatchWork &w, const long long *PW, int n, int lane) {
     const long long INF = LLONG_MAX / 4;
-    for (int j = lane; j < n; j += 32) {
-        w.u[j] = 0;
-        w.v[j] = 0;
-        w.match[j] = -1;
-        const int x = w.nlo[j], y = w.nhi[j];
-        w.need[j] = y > x ? PW[y] - PW[x] : 0ll;
+    long long v[NC], slack[NC], need[NC];
+    int nlo[NC], nhi[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int j = c * 32 + lane;
+        nlo[c] = j < n ? (int)w.nlo[j] : 0;
+        nhi[c] = j < n ? (int)w.nhi[j] : 0;
+        need[c] = nhi[c] > nlo[c] ? PW[nhi[c]] - PW[nlo[c]] : 0ll;
+        v[c] = INF;
+        if (j < n) { w.u[j] = 0; w.match[j] = -1; w.row_col[j] = -1; }
+    }
+    __syncwarp();
+    // Start from feasible potentials instead of zeros: v[j] = the cheapest row of column j
+    // (u = 0), then every column claims a free row that attains it, scanning rows upwards.
+    // Most positions find a device that already holds most of their layers, so few rows are
+    // left for the augmenting phase.
+    for (int i = 0; i < n; ++i) {
+        const int a = w.olo[i], b = w.ohi[i];
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const long long cost = range_cost(PW, need[c], a, b, nlo[c], nhi[c]);
+            v[c] = cost < v[c] ? cost : v[c];
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int j = c * 32 + lane;
+        if (j >= n) continue;
+        for (int i = 0; i < n; ++i) {
+            if (range_cost(PW, need[c], w.olo[i], w.ohi[i], nlo[c], nhi[c]) != v[c]) continue;
+            if (atomicCAS(&w.row_col[i], -1, j) == -1) { w.match[j] = (short)i; break; }
+        }
     }
     __syncwarp();
     bool broken = false;
     for (int r = 0; r < n && !broken; ++r) {
-        for (int j = lane; j < n; j += 32) { w.slack[j] = INF; w.prev[j] = (short)n; }
+        if (w.row_col[r] >= 0) continue;           // uniform: already matched by the start-up pass
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            slack[c] = INF;
+            if (c * 32 + lane < n) w.prev[c * 32 + lane] = (short)n;
+        }
         uint32_t tree = 0;            // bit c: column c*32+lane belongs to the tree
         int col = n, row = r;         // column n is the root and holds the new row
         for (int step = 0; step <= n; ++step) {
@@ -119,24 +155,32 @@ __device__ long long warp_match(MatchWork &w, const long long *PW, int n, int la
             const long long ur = w.u[row];
             long long delta = INF;
             int next = n;
-            for (int c = 0, j = lane; j < n; ++c, j += 32) {
-                if ((tree >> c) & 1u) continue;
-                const int lo = max(a, (int)w.nlo[j]), hi = min(b, (int)w.nhi[j]);
-                const long long cost = w.need[j] - (hi > lo ? PW[hi] - PW[lo] : 0ll);
-                const long long red = cost - ur - w.v[j];
-                long long s = w.slack[j];
-                if (red < s) { s = red; w.slack[j] = s; w.prev[j] = (short)col; }
-                if (s < delta) { delta = s; next = j; }
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int j = c * 32 + lane;
+                if (j >= n || ((tree >> c) & 1u)) continue;
+                const long long red = range_cost(PW, need[c], a, b, nlo[c], nhi[c]) - ur - v[c];
+                if (red < slack[c]) { slack[c] = red; w.prev[j] = (short)col; }
+                if (slack[c] < delta) { delta = slack[c]; next = j; }
             }
-            for (int o = 16; o > 0; o >>= 1) {
-                const long long od = __shfl_xor_sync(0xffffffffu, delta, o);
-                const int on = __shfl_xor_sync(0xffffffffu, next, o);
-                if (od < delta || (od == delta && on < next)) { delta = od; next = on; }
+            // warp argmin of (slack, column), lowest column on ties: three hardware min-reductions
+            // (high word, low word among the lanes that hold the least high word, column among
+            // the lanes that hold the least slack); slacks are never negative
+            {
+                const uint32_t hi = (uint32_t)((unsigned long long)delta >> 32), lo = (uint32_t)delta;
+                const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+                const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+                const bool least = hi == mhi && lo == mlo;
+                next = (int)__reduce_min_sync(0xffffffffu, least ? (uint32_t)next : 0xffffffffu);
+                delta = (long long)(((unsigned long long)mhi << 32) | mlo);
             }
             if (next >= n) { broken = true; break; }
-            for (int c = 0, j = lane; j < n; ++c, j += 32) {
-                if ((tree >> c) & 1u) { w.u[w.match[j]] += delta; w.v[j] -= delta; }
-                else w.slack[j] -= delta;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int j = c * 32 + lane;
+                if (j >= n) continue;
+                if ((tree >> c) & 1u) { w.u[w.match[j]] += delta; v[c] -= delta; }
+                else slack[c] -= delta;
             }
             if (lane == 0) w.u[r] += delta;
             __syncwarp();
@@ -146,6 +190,9 @@ __device__ long long warp_match(MatchWork &w, const long long *PW, int n, int la
             if (row < 0) break;
         }
         if (row >= 0) broken = true;   // step bound hit without reaching a free column
+        // every lane must have read match[col] above before lane 0 rewrites the matching:
+        // a lane that sees the flipped entry would take the free column for a matched one
+        __syncwarp();
         if (!broken && lane == 0) {
             int c = col;
             for (int step = 0; step <= n && c != n; ++step) {
@@ -158,9 +205,20 @@ __device__ long long warp_match(MatchWork &w, const long long *PW, int n, int la
     }
     if (broken) return -1;
     long long total = 0;
-    for (int j = lane; j < n; j += 32) total += match_cost(w, PW, w.match[j], j);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int j = c * 32 + lane;
+        if (j < n) { const int i = w.match[j]; total += range_cost(PW, need[c], w.olo[i], w.ohi[i], nlo[c], nhi[c]); }
+    }
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     return total;
+}
+
+__device__ __forceinline__ long long warp_match_any(MatchWork &w, const long long *PW, int n, int lane) {
+    if (n <= 32) return warp_match<1>(w, PW, n, lane);
+    if (n <= 64) return warp_match<2>(w, PW, n, lane);
+    if (n <= 128) return warp_match<4>(w, PW, n, lane);
+    return warp_match<8>(w, PW, n, lane);
 }
 
 __device__ __forceinline__ void stage_state_bytes(long long *PW, const DevProfile *p) {
@@ -222,7 +280,7 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_matching_kernel(Tabl
     ok = __all_sync(0xffffffffu, ok) && covered == n;       // a strategy uses every survivor
     __syncwarp();
     if (!ok) return;
-    const long long total = warp_match(mw, PW, n, lane);
+    const long long total = warp_match_any(mw, PW, n, lane);
     if (total < 0) return;
     uint16_t *asg = od.short_assign + slot * kMaxMatch;
     for (int j = lane; j < kMaxMatch; j += 32) asg[j] = j < n ? (uint16_t)mw.match[j] : (uint16_t)0;
@@ -255,7 +313,7 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_range_matching_kernel(Tab
         mw.nlo[j] = (uint8_t)min((int)new_lo[base + j], L); mw.nhi[j] = (uint8_t)min((int)new_hi[base + j], L);
     }
     __syncwarp();
-    const long long t = warp_match(mw, PW, n, lane);
+    const long long t = warp_match_any(mw, PW, n, lane);
     if (lane == 0) total[q] = t;
     if (assign)
         for (int j = lane; j < kMaxMatch; j += 32) assign[base + j] = (j < n && t >= 0) ? (uint16_t)mw.match[j] : (uint16_t)0;
