@@ -71,14 +71,15 @@ class _Plan(C.Structure):
 
 
 class _Objective(C.Structure):
-    _fields_ = [("topk", C.c_int32), ("pad", C.c_int32), ("t_gap", C.c_double), ("t_restart", C.c_double),
+    _fields_ = [("topk", C.c_int32), ("sync_rounds", C.c_int32), ("t_gap", C.c_double), ("t_restart", C.c_double),
                 ("t_gap_ns", C.c_int64), ("t_restart_ns", C.c_int64), ("bw_xfer", C.c_int64)]
 
 
 class _Transition(C.Structure):
     _fields_ = [("policy", C.c_int32), ("feasible", C.c_int32), ("rank", C.c_int32), ("n_surv", C.c_int32),
                 ("xfer_bytes", C.c_int64), ("t_trans", C.c_double), ("t_trans_ns", C.c_int64),
-                ("objective", C.c_double)]
+                ("objective", C.c_double), ("rounds", C.c_int32), ("domains", C.c_int32),
+                ("t_sync", C.c_double), ("t_sync_ns", C.c_int64)]
 
 
 @dataclass
@@ -94,6 +95,11 @@ class Transition:
     assign: Tuple[int, ...] = ()
     shortlist: Tuple = ()
     shortlist_bytes: Tuple[int, ...] = ()
+    rounds: int = 0
+    domains: int = 0
+    t_sync: float = 0.0
+    t_sync_ns: int = 0
+    shortlist_rounds: Tuple[int, ...] = ()
 
 
 @dataclass
@@ -140,6 +146,7 @@ class Oracle:
             getattr(self._lib, "orc_pipe_time" + sfx).restype = C.c_double
             getattr(self._lib, "orc_count" + sfx).restype = C.c_uint64
             getattr(self._lib, "orc_plan_transfer" + sfx).restype = C.c_int64
+            getattr(self._lib, "orc_plan_async_step" + sfx).restype = C.c_double
         self.profile = profile
         self.options = options
         p = profile
@@ -351,6 +358,27 @@ class Oracle:
         b = self._fn("orc_plan_transfer", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(c), _ptr(out, C.c_int32))
         return int(b), [int(x) for x in out[:n_surv]]
 
+    def comm_rounds(self, stage_of: Sequence[Sequence[int]]) -> Tuple[int, List[int], int]:
+        """Greedy communication rounds of a layer placement: stage_of[p][l] = stage of pipeline p
+        holding layer l.  -> (rounds, colour per layer, communication domains)."""
+        a = np.ascontiguousarray(stage_of, dtype=np.int32)
+        dp, L = a.shape
+        colour = np.zeros(L, dtype=np.int32)
+        r = self._lib.orc_comm_rounds(L, dp, _ptr(a, C.c_int32), _ptr(colour, C.c_int32))
+        d = self._lib.orc_comm_domains(L, dp, _ptr(a, C.c_int32))
+        return int(r), [int(x) for x in colour], int(d)
+
+    def plan_async_step(self, failed: Sequence[int], plan: Plan, options=None):
+        """Step time of a plan under asymmetric synchronisation -> (step, rounds, domains, t_sync);
+        times as floats (exact for the integer build below 2^53)."""
+        o, sfx = self._opts(options)
+        _, fp, nf = self._failed(failed)
+        c = self._cplan(plan)
+        r, d, ts = C.c_int32(), C.c_int32(), C.c_double()
+        t = self._fn("orc_plan_async_step", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(c),
+                                                 C.byref(r), C.byref(d), C.byref(ts))
+        return t, r.value, d.value, ts.value
+
     def search_objective(self, failed: Sequence[int], objective, options=None):
         """Full-objective search -> (best plan or None, Transition).
 
@@ -359,7 +387,7 @@ class Oracle:
         o, sfx = self._opts(options)
         _, fp, nf = self._failed(failed)
         k = max(1, int(objective.topk))
-        q = _Objective(k, 0, float(objective.t_gap_ns), float(objective.t_restart_ns),
+        q = _Objective(k, int(getattr(objective, "sync_rounds", 0)), float(objective.t_gap_ns), float(objective.t_restart_ns),
                        int(round(objective.t_gap_ns)), int(round(objective.t_restart_ns)),
                        int(objective.bw_xfer_Bpns))
         n_surv = self.profile.n_dp * self.profile.n_pp - nf
@@ -367,15 +395,17 @@ class Oracle:
         asg = np.zeros(max(n_surv, 1), dtype=np.int32)
         sp = (_Plan * k)()
         sb = np.zeros(k, dtype=np.int64)
+        sr = np.zeros(k, dtype=np.int32)
         ns = C.c_int32()
         ok = self._fn("orc_search_objective", sfx)(C.byref(self._cp), C.byref(o), fp, nf, C.byref(q),
                                                    C.byref(best), C.byref(tr), _ptr(asg, C.c_int32), sp,
-                                                   _ptr(sb, C.c_int64), C.byref(ns))
+                                                   _ptr(sb, C.c_int64), _ptr(sr, C.c_int32), C.byref(ns))
         t = Transition(tr.policy, bool(tr.feasible), tr.rank, tr.n_surv, tr.xfer_bytes, tr.t_trans, tr.t_trans_ns,
                        tr.objective,
                        tuple(int(x) for x in asg[:n_surv]) if (ok and tr.policy == DYNPAR) else (),
                        tuple(_plan_from(sp[i]) for i in range(ns.value)),
-                       tuple(int(x) for x in sb[:ns.value]))
+                       tuple(int(x) for x in sb[:ns.value]),
+                       tr.rounds, tr.domains, tr.t_sync, tr.t_sync_ns, tuple(int(x) for x in sr[:ns.value]))
         return (_plan_from(best) if ok else None), t
 
     def decode(self, failed: Sequence[int], plan: Plan, options=None) -> List[List[int]]:

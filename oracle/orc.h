@@ -56,7 +56,8 @@ typedef struct {
  * times the share of the time until the next fault that is spent training.  */
 typedef struct {
     int32_t topk;                    /* dynamic-parallelism plans that are re-scored, >= 1   */
-    int32_t pad;
+    int32_t sync_rounds;             /* 1: step time of a shortlisted plan = slowest pipeline +
+                                        all-reduce rounds of the coloured layer graph         */
     double t_gap, t_restart;         /* ns between two faults / restart overhead (_f64)     */
     int64_t t_gap_ns, t_restart_ns;  /* the same as integers (_i64)                         */
     int64_t bw_xfer;                 /* bytes per ns available to the weight transfer       */
@@ -70,6 +71,9 @@ typedef struct {
     double t_trans;                  /* transition time, _f64                               */
     int64_t t_trans_ns;              /* transition time, _i64                               */
     double objective;                /* steps completed before the next fault               */
+    int32_t rounds, domains;         /* communication rounds / domains of the chosen plan (sync_rounds = 1) */
+    double t_sync;                   /* time of those rounds, _f64                          */
+    int64_t t_sync_ns;               /* _i64                                                */
 } orc_transition;
 
 /* ---- orc_restore.c: weight-transfer matching (integer) ---- */
@@ -77,6 +81,8 @@ void orc_transfer_cost_matrix(int L, const int64_t *w, int n, const int32_t *old
                               const int32_t *new_lo, const int32_t *new_hi, int64_t *cost /* [n][n] */);
 int64_t orc_assign(int n, const int64_t *cost, int32_t *row_of_col);
 int64_t orc_assign_brute(int n, const int64_t *cost);
+int orc_comm_rounds(int L, int dp, const int32_t *stage_of /* [dp][L] */, int32_t *colour /* [L] */);
+int orc_comm_domains(int L, int dp, const int32_t *stage_of);
 
 /* ---- orc_enum.c: integer combinatorics (no cost arithmetic) ---- */
 uint64_t orc_binom(int n, int k);                       /* saturates at UINT64_MAX */

@@ -1015,6 +1015,48 @@ static int64_t plan_transfer_bytes(const space *sp, const orc_plan *pl, int32_t 
  * _f64: one IEEE operation per written operation.  _i64: the quotient bytes / bandwidth
  * floors and two objectives are compared exactly as fractions.
  */
+/*
+ * Step time of a dynamic-parallelism plan with the asymmetric synchronisation of Section
+ * "Restorer" (Asymmetric Communication): the slowest pipeline (without a synchronisation
+ * term of its own) plus the all-reduce rounds of the coloured layer graph.  Reading (the
+ * paper gives the rounds, not their time): the all-reduce of layer l over the dp pipelines
+ * takes the ring lower bound 2(n-1) * params(l) / (n * bw_sync), a round lasts as long as
+ * its largest layer, rounds run one after the other (summed in colour order).
+ */
+static num_t plan_async_step(const space *sp, const orc_plan *pl, int *rounds_out, int *domains_out, num_t *t_sync_out) {
+    const orc_profile *pr = sp->M.p;
+    int L = pr->L, dp = (int)pl->n_pipes;
+    int32_t *stage_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)dp * (size_t)L);
+    int32_t colour[ORC_MAX_LAYERS];
+    num_t t_pipe = 0;
+    for (int p = 0; p < dp; p++) {
+        int32_t cuts[ORC_MAX_STAGES + 1];
+        int devs[ORC_MAX_STAGES];
+        const segment *g = find_segment(sp, (int)pl->strategy, p, pl->micro[p]);
+        segment_cuts(sp, g, pl->kappa[p], cuts);
+        for (int i = 0; i < g->S; i++) {
+            devs[i] = sp->surv[g->off + i];
+            for (int l = cuts[i]; l < cuts[i + 1]; l++) stage_of[(size_t)p * L + l] = i;
+        }
+        num_t c; int ok;
+        pipe_from_cuts(&sp->M, g->S, cuts, g->m, devs, 1 /* no peers: bare pipeline time */, &c, &ok);
+        t_pipe = nmax(t_pipe, c);
+    }
+    int rounds = orc_comm_rounds(L, dp, stage_of, colour);
+    num_t t_sync = 0;
+    for (int c = 0; c < rounds; c++) {
+        num_t longest = 0;
+        for (int l = 0; l < L; l++)
+            if (colour[l] == c) longest = nmax(longest, sync_time(pr, pr->param_bytes[l], dp));
+        t_sync = t_sync + longest;
+    }
+    if (rounds_out) *rounds_out = rounds;
+    if (domains_out) *domains_out = orc_comm_domains(L, dp, stage_of);
+    if (t_sync_out) *t_sync_out = t_sync;
+    free(stage_of);
+    return t_pipe + t_sync;
+}
+
 typedef struct { num_t numer, denom; } frac_t;
 
 static int frac_greater(frac_t a, frac_t b) {   /* a > b, both denominators > 0 */
@@ -1029,7 +1071,7 @@ int NAME(orc_search_objective)(const orc_profile *prof, const orc_opts *o, const
                                const orc_objective *q, orc_plan *best, orc_transition *tr,
                                int32_t *assign /* [n_surv] or NULL */,
                                orc_plan *short_plans /* [topk] or NULL */, int64_t *short_bytes /* [topk] or NULL */,
-                               int32_t *n_short /* or NULL */) {
+                               int32_t *short_rounds /* [topk] or NULL */, int32_t *n_short /* or NULL */) {
 #if ORC_INT
     const num_t t_gap = q->t_gap_ns, t_restart = q->t_restart_ns;
 #else
@@ -1062,8 +1104,12 @@ int NAME(orc_search_objective)(const orc_profile *prof, const orc_opts *o, const
     if (n_short) *n_short = ns;
     for (int r = 0; r < ns; r++) {
         int64_t bytes = plan_transfer_bytes(&sp, &plans[r], asg);
+        int rounds = 0, domains = 0;
+        num_t t_sync = 0;
+        if (q->sync_rounds) set_cost(&plans[r], plan_async_step(&sp, &plans[r], &rounds, &domains, &t_sync));
         if (short_plans) short_plans[r] = plans[r];
         if (short_bytes) short_bytes[r] = bytes;
+        if (short_rounds) short_rounds[r] = rounds;
 #if ORC_INT
         num_t t_trans = t_restart + bytes / q->bw_xfer;
 #else
@@ -1073,10 +1119,13 @@ int NAME(orc_search_objective)(const orc_profile *prof, const orc_opts *o, const
         if (!have || frac_greater(j, best_j)) {
             have = 1; best_j = j; *best = plans[r];
             tr->policy = ORC_DYNPAR; tr->feasible = 1; tr->rank = r; tr->xfer_bytes = bytes;
+            tr->rounds = rounds; tr->domains = domains;
 #if ORC_INT
             tr->t_trans_ns = t_trans; tr->t_trans = 0;
+            tr->t_sync_ns = t_sync; tr->t_sync = 0;
 #else
             tr->t_trans = t_trans; tr->t_trans_ns = 0;
+            tr->t_sync = t_sync; tr->t_sync_ns = 0;
 #endif
             if (assign) memcpy(assign, asg, sizeof(int32_t) * (size_t)sp.n_surv);
         }
@@ -1098,3 +1147,17 @@ int64_t NAME(orc_plan_transfer)(const orc_profile *prof, const orc_opts *o, cons
     return b;
 }
 
+/* Asymmetric-synchronisation step time of one given dynamic-parallelism plan. */
+double NAME(orc_plan_async_step)(const orc_profile *prof, const orc_opts *o, const uint32_t *failed, int n_failed,
+                                 const orc_plan *pl, int32_t *rounds, int32_t *domains, double *t_sync) {
+    space sp;
+    space_build(&sp, prof, o, failed, n_failed);
+    int r = 0, d = 0;
+    num_t ts = 0;
+    num_t t = plan_async_step(&sp, pl, &r, &d, &ts);
+    if (rounds) *rounds = r;
+    if (domains) *domains = d;
+    if (t_sync) *t_sync = (double)ts;
+    space_free(&sp);
+    return (double)t;
+}

@@ -114,3 +114,48 @@ int64_t orc_assign_brute(int n, const int64_t *cost) {
     }
     return best;
 }
+
+/*
+ * Section "Restorer", Asymmetric Communication: every model layer is a vertex; two layers
+ * are joined when some device holds both (then their data-parallel all-reduces cannot run
+ * at the same time); a greedy colouring gives the communication rounds, layers of one
+ * colour synchronise in parallel.  stage_of[p * L + l] = stage of pipeline p that holds
+ * layer l (device = (pipeline, stage)).  Greedy in layer order: a layer takes the least
+ * colour that none of its already coloured neighbours has.  Returns the number of colours;
+ * colour[l] in 0..rounds-1.  O(L^2 * dp).
+ */
+int orc_comm_rounds(int L, int dp, const int32_t *stage_of, int32_t *colour) {
+    int rounds = 0;
+    for (int l = 0; l < L; l++) {
+        char used[ORC_MAX_LAYERS + 1];
+        memset(used, 0, sizeof(used));
+        for (int k = 0; k < l; k++) {
+            int adjacent = 0;
+            for (int p = 0; p < dp; p++)
+                if (stage_of[(size_t)p * L + l] == stage_of[(size_t)p * L + k]) adjacent = 1;
+            if (adjacent) used[colour[k]] = 1;
+        }
+        int c = 0;
+        while (used[c]) c++;
+        colour[l] = c;
+        if (c + 1 > rounds) rounds = c + 1;
+    }
+    return rounds;
+}
+
+/*
+ * Communication domains of a plan: maximal runs of layers that sit on the same device in
+ * every pipeline, i.e. the distinct tuples (stage in pipeline 1, ..., stage in pipeline dp).
+ * One all-reduce group is set up per domain (the paper's example counts 4 of them in the
+ * symmetric and 6 in the asymmetric layout of its figure).
+ */
+int orc_comm_domains(int L, int dp, const int32_t *stage_of) {
+    int n = 0;
+    for (int l = 0; l < L; l++) {
+        int fresh = l == 0;
+        for (int p = 0; p < dp && !fresh; p++)
+            if (stage_of[(size_t)p * L + l] != stage_of[(size_t)p * L + l - 1]) fresh = 1;
+        n += fresh;
+    }
+    return n;
+}

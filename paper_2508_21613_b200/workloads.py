@@ -123,6 +123,7 @@ class ObjectiveOptions:
     t_gap_ns: float = 1125e9
     t_restart_ns: float = 5e9
     bw_xfer_Bpns: int = 25
+    sync_rounds: int = 0     # 1: shortlisted plans are timed with the coloured all-reduce rounds
 
 
 @dataclass

@@ -10,7 +10,13 @@ feasible, strategy, pipelines, split rank, stages, micro-batches, layer-composit
 and the cost bits -- everything the parity bar requires to be bit-exact.  The GPU tests
 recompute the fingerprint from the library's plan and compare.
 
-    python tests/golden/make_search_goldens.py [workload ...] [--procs N]
+    python tests/golden/make_search_goldens.py [workload ...] [--procs N] [--objective]
+
+With --objective the full-objective search (default ObjectiveOptions) is stored instead, in
+objective_<workload>_<mode>.txt:
+
+    <policy> <rank> <matched bytes> <transition time: double as hex / integer ns> <objective as hex>
+    <fingerprint of the chosen plan> <fingerprint of the shortlist: every plan tuple, cost and matched bytes>
 
 The sweep costs about four core-hours per cost mode.
 """
@@ -70,6 +76,31 @@ def _one(b):
     return b, line_of(best, _state["mode"])
 
 
+def objective_line(best, tr, mode: int) -> str:
+    """One stored line of the full-objective search (works for oracle and library results:
+    `tr` needs policy, rank, xfer_bytes, t_trans, t_trans_ns, objective, shortlist, shortlist_bytes)."""
+    if best is None or not best.feasible:
+        return "-1 -1 0 - - ffffffffffffffff ffffffffffffffff"
+    h = 0xCBF29CE484222325
+    for plan, nbytes in zip(tr.shortlist, tr.shortlist_bytes):
+        for w in (fingerprint(plan, mode), nbytes):
+            for byte in struct.pack("<Q", int(w) & 0xFFFFFFFFFFFFFFFF):
+                h = ((h ^ byte) * 0x100000001B3) & 0xFFFFFFFFFFFFFFFF
+    t_trans = str(tr.t_trans_ns) if mode else float(tr.t_trans).hex()
+    return (f"{tr.policy} {tr.rank} {tr.xfer_bytes} {t_trans} {float(tr.objective).hex()} "
+            f"{fingerprint(best, mode):016x} {h:016x}")
+
+
+def _one_objective(b):
+    from paper_2508_21613_b200 import workloads as W
+    best, tr = _state["o"].search_objective(_state["w"].scenarios[b], W.ObjectiveOptions())
+    return b, objective_line(best, tr, _state["mode"])
+
+
+def objective_path(name: str, mode: int) -> str:
+    return os.path.join(HERE, f"objective_{name}_{'i64' if mode else 'f64'}.txt")
+
+
 def golden_path(name: str, mode: int) -> str:
     return os.path.join(HERE, f"search_{name}_{'i64' if mode else 'f64'}.txt")
 
@@ -79,6 +110,7 @@ def main():
     ap.add_argument("workloads", nargs="*", default=WORKLOADS)
     ap.add_argument("--procs", type=int, default=os.cpu_count())
     ap.add_argument("--modes", type=int, nargs="*", default=[0, 1])
+    ap.add_argument("--objective", action="store_true", help="store the full-objective search instead")
     args = ap.parse_args()
     from oracle.oracle import build
     build()
@@ -89,8 +121,16 @@ def main():
             t0 = time.time()
             with mp.Pool(args.procs, initializer=_init, initargs=(name, mode)) as pool:
                 lines = [None] * n
-                for b, line in pool.imap_unordered(_one, range(n), chunksize=1):
+                for b, line in pool.imap_unordered(_one_objective if args.objective else _one, range(n), chunksize=1):
                     lines[b] = line
+            if args.objective:
+                with open(objective_path(name, mode), "w") as f:
+                    f.write(f"# {name}, cost mode {'int64 ns' if mode else 'fp64'}: full-objective search per failure scenario "
+                            f"from the CPU oracle (tests/golden/make_search_goldens.py --objective)\n"
+                            f"# policy rank matched_bytes transition_time objective plan_fingerprint shortlist_fingerprint\n")
+                    f.write("\n".join(lines) + "\n")
+                print(f"{name} mode {mode} (objective): {n} scenarios in {time.time() - t0:.0f} s", flush=True)
+                continue
             with open(golden_path(name, mode), "w") as f:
                 f.write(f"# {name}, cost mode {'int64 ns' if mode else 'fp64'}: best plan per failure scenario from the CPU "
                         f"oracle (tests/golden/make_search_goldens.py)\n# policy feasible cost fingerprint\n")

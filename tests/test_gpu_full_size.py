@@ -50,3 +50,45 @@ def test_every_scenario_matches_the_stored_oracle_result(gpu, name, mode):
                            f"{w.scenarios[wrong[0]]}: got {got[wrong[0]]} want {want[wrong[0]]}")
     finally:
         gpu.cm_destroy(ctx)
+
+
+def _stored_objective(name, mode):
+    path = goldens.objective_path(name, mode)
+    assert os.path.exists(path), f"{path} is missing: run tests/golden/make_search_goldens.py {name} --objective"
+    return [l.strip() for l in open(path) if l.strip() and not l.startswith("#")]
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("name", ["paper-scale", "70b-like", "175b-like"])
+def test_full_objective_of_every_scenario_matches_the_stored_oracle_result(gpu, name, mode):
+    """cm_search_objective with the default options over the whole workload: chosen policy,
+    shortlist rank, matched bytes, transition time, objective, the chosen plan and the whole
+    shortlist (plan tuples, costs, matched bytes) of every scenario against the oracle's."""
+    from types import SimpleNamespace
+    w = W.ALL_WORKLOADS[name]()
+    want = _stored_objective(name, mode)
+    assert len(want) == len(w.scenarios)
+    obj = W.ObjectiveOptions()
+    k = obj.topk
+    ctx = gpu.cm_create(0)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        best, trans, sl, sb = gpu.cm_search_objective(ctx, w.scenarios, w.options.with_cost_mode(mode), obj,
+                                                      shortlist=True)
+        plans = gpu.plans_from_array(best)
+        short = gpu.plans_from_array(sl)
+        wrong = []
+        for b in range(len(want)):
+            used = [r for r in range(k) if sb[b, r] >= 0]
+            tr = SimpleNamespace(policy=trans[b].policy, rank=trans[b].rank, xfer_bytes=trans[b].xfer_bytes,
+                                 t_trans=trans[b].t_trans, t_trans_ns=trans[b].t_trans_ns,
+                                 objective=trans[b].objective,
+                                 shortlist=[short[b * k + r] for r in used],
+                                 shortlist_bytes=[int(sb[b, r]) for r in used])
+            got = goldens.objective_line(plans[b] if trans[b].feasible else None, tr, mode)
+            if got != want[b]:
+                wrong.append((b, got))
+        assert not wrong, (f"{len(wrong)} of {len(want)} scenarios differ, first: scenario {wrong[0][0]} "
+                           f"{w.scenarios[wrong[0][0]]}: got {wrong[0][1]} want {want[wrong[0][0]]}")
+    finally:
+        gpu.cm_destroy(ctx)

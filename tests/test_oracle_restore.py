@@ -275,3 +275,132 @@ def test_objective_limits(oracle_factory):
         k = [o.search_objective(failed, W.ObjectiveOptions(topk=4, t_gap_ns=60e9, bw_xfer_Bpns=b))[1].objective
              for b in (400, 25, 1)]
         assert k[0] >= k[1] >= k[2]
+
+
+# ---- asymmetric communication: rounds by greedy colouring (Section "Restorer") ----
+
+def _stage_of(cuts_per_pipeline, L):
+    out = []
+    for cuts in cuts_per_pipeline:
+        row = [0] * L
+        for i in range(len(cuts) - 1):
+            for l in range(cuts[i], cuts[i + 1]):
+                row[l] = i
+        out.append(row)
+    return out
+
+
+def test_rounds_equal_library_greedy_colouring_in_layer_order(oracle_factory):
+    import networkx as nx
+    _, o = _tiny_oracle(oracle_factory)
+    rng = np.random.default_rng(21)
+    for trial in range(60):
+        L = int(rng.integers(2, 25))
+        dp = int(rng.integers(1, 5))
+        pipes = []
+        for _ in range(dp):
+            S = int(rng.integers(1, L + 1))
+            inner = sorted(rng.choice(np.arange(1, L), size=S - 1, replace=False).tolist()) if S > 1 else []
+            pipes.append([0] + inner + [L])
+        st = _stage_of(pipes, L)
+        rounds, colour, domains = o.comm_rounds(st)
+        g = nx.Graph()
+        g.add_nodes_from(range(L))
+        for a in range(L):
+            for b in range(a + 1, L):
+                if any(st[p][a] == st[p][b] for p in range(dp)):
+                    g.add_edge(a, b)
+        ref = nx.coloring.greedy_color(g, strategy=lambda graph, colors: list(range(L)))
+        assert colour == [ref[l] for l in range(L)]
+        assert rounds == max(colour) + 1
+        # a proper colouring, at least as many colours as the fullest device holds layers
+        assert all(colour[a] != colour[b] for a, b in g.edges)
+        fullest = max(max(c[i + 1] - c[i] for i in range(len(c) - 1)) for c in pipes)
+        assert fullest <= rounds <= max(dict(g.degree).values(), default=0) + 1
+        # domains: one per distinct cut position of any pipeline
+        assert domains == len(set().union(*[set(c) for c in pipes])) - 1
+
+
+def test_rounds_of_symmetric_and_shifted_layouts(oracle_factory):
+    _, o = _tiny_oracle(oracle_factory)
+    # symmetric: every pipeline cuts alike -> rounds = layers of the fullest stage, domains = stages
+    st = _stage_of([[0, 2, 4, 6, 9]] * 3, 9)
+    rounds, colour, domains = o.comm_rounds(st)
+    assert (rounds, domains) == (3, 4)
+    assert colour == [0, 1, 0, 1, 0, 1, 0, 1, 2]
+    # by hand: 4 stages (2,2,2,2) next to 3 stages (3,3,2) over 8 layers.  Layer 2 shares a
+    # device with layers 0,1 (second pipeline) and 3 (first), layer 3 with 2 and 4,5, ...
+    st = _stage_of([[0, 2, 4, 6, 8], [0, 3, 6, 8]], 8)
+    rounds, colour, domains = o.comm_rounds(st)
+    assert colour == [0, 1, 2, 0, 1, 2, 0, 1]
+    assert (rounds, domains) == (3, 5)      # domains: cut positions {0,2,3,4,6,8} -> 5 runs
+    # one pipeline alone: its stages are disjoint cliques
+    rounds, colour, domains = o.comm_rounds(_stage_of([[0, 1, 5, 7]], 7))
+    assert (rounds, domains) == (4, 3) and colour == [0, 0, 1, 2, 3, 0, 1]
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_async_step_time_by_hand_composition(oracle_factory, mode):
+    w = W.paper_scale(2, 2)
+    opts = w.options.with_cost_mode(mode)
+    o = oracle_factory(w.profile, opts)
+    p = w.profile
+    for failed in (w.scenarios[3], w.scenarios[-1]):
+        plan = o.search_policy(failed, W.POLICY_DYNPAR)
+        step, rounds, domains, t_sync = o.plan_async_step(failed, plan)
+        cuts = o.decode(failed, plan)
+        surv = [d for d in range(p.n_dp * p.n_pp) if d not in failed]
+        # slowest bare pipeline (one participant: no synchronisation term)
+        off, t_pipe = 0, 0
+        for q in range(plan.n_pipes):
+            ok, c, c_ns, _ = o.pipe(cuts[q], plan.micro[q], surv[off:off + plan.stages[q]], 1, mode)
+            assert ok
+            t_pipe = max(t_pipe, c_ns if mode else c)
+            off += plan.stages[q]
+        r2, colour, d2 = o.comm_rounds(_stage_of(cuts, p.L))
+        assert (rounds, domains) == (r2, d2)
+        n = plan.n_pipes
+        bw = p.bw_inter_Bpns if p.n_dp * p.n_pp > p.devices_per_node else p.bw_intra_Bpns
+        total = 0
+        for c in range(r2):
+            sizes = [int(p.param_bytes[l]) for l in range(p.L) if colour[l] == c]
+            big = max(sizes)
+            total = total + ((2 * (n - 1) * big) // (n * bw) if mode else ((2.0 * (n - 1)) * big) / (float(n) * bw))
+        assert t_sync == total
+        assert step == t_pipe + total
+        if mode:   # uniform layers: the rounds cost exactly rounds x one layer's all-reduce
+            one = (2 * (n - 1) * int(p.param_bytes[0])) // (n * bw)
+            assert len(set(int(x) for x in p.param_bytes)) == 1 and t_sync == rounds * one
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_objective_with_sync_rounds_ranks_by_the_async_step(oracle_factory, mode):
+    w = W.paper_scale(2, 2)
+    opts = w.options.with_cost_mode(mode)
+    o = oracle_factory(w.profile, opts)
+    obj0 = W.ObjectiveOptions(topk=6)
+    obj1 = W.ObjectiveOptions(topk=6, sync_rounds=1)
+    for failed in (w.scenarios[0], w.scenarios[7], w.scenarios[-2]):
+        _, t0 = o.search_objective(failed, obj0)
+        best, t1 = o.search_objective(failed, obj1)
+        _, per = o.search(failed)
+        assert [p.key() for p in t0.shortlist] == [p.key() for p in t1.shortlist]     # same shortlist
+        assert t0.shortlist_bytes == t1.shortlist_bytes
+        cands = []
+        for pol in (W.POLICY_REROUTE, W.POLICY_REDUNDANT):
+            if per[pol].feasible:
+                cands.append((Fraction(int(obj1.t_gap_ns)) / Fraction(per[pol].cost_ns if mode else per[pol].cost), pol, -1))
+        for r, (plan, b) in enumerate(zip(t1.shortlist, t1.shortlist_bytes)):
+            step, rounds, _, _ = o.plan_async_step(failed, t0.shortlist[r])
+            assert (plan.cost_ns if mode else plan.cost) == step and t1.shortlist_rounds[r] == rounds
+            if mode:
+                j = Fraction(int(obj1.t_gap_ns) - (int(obj1.t_restart_ns) + b // obj1.bw_xfer_Bpns), plan.cost_ns)
+            else:
+                j = Fraction((obj1.t_gap_ns - (obj1.t_restart_ns + float(b) / float(obj1.bw_xfer_Bpns))) / plan.cost)
+            cands.append((j, W.POLICY_DYNPAR, r))
+        top = max(c[0] for c in cands)
+        first = next(c for c in cands if c[0] == top)
+        assert (t1.policy, t1.rank) == (first[1], first[2])
+        if t1.policy == W.POLICY_DYNPAR:
+            assert best.key() == t1.shortlist[t1.rank].key()
+            assert t1.rounds == t1.shortlist_rounds[t1.rank] and t1.rounds >= 1
