@@ -265,7 +265,7 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
             for key, v in binding.cm_objective_stats(ctx).items():
                 phases[key] = phases.get(key, 0) + v
             search_ns += binding.cm_last_stats(ctx)["device_ns"]
-        best, trans, _, sb = res
+        best, trans, _, sb, _ = res
         packed.search(ctx, opts)
         plain = packed.best
         policies = [0, 0, 0]

@@ -247,10 +247,22 @@ cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *space, uint64_
  * shortlist, ties to the lower policy id, then to the earlier shortlist rank.  fp64 mode
  * computes t_trans = t_restart + bytes / bw and the objective with one IEEE operation each;
  * int64 mode floors bytes / bw and compares objectives exactly as fractions.
+ *
+ * sync_rounds = 1 (Section "Restorer", Asymmetric Communication): when pipelines cut the
+ * model differently, the all-reduce of a layer spans different stages in different
+ * pipelines and two layers that share a device in any pipeline cannot synchronise at the
+ * same time.  Layers are vertices, such pairs edges; a greedy colouring in layer order
+ * (least colour no coloured neighbour has) gives the communication rounds.  A shortlisted
+ * plan is then timed as  slowest pipeline (without a synchronisation term of its own)
+ * + sum over rounds of the longest all-reduce of the round, the all-reduce of layer l over
+ * the dp pipelines taking 2 (dp-1) params(l) / (dp * bw_sync) as in the search's model;
+ * that step time replaces the search's in plan.cost / cost_ns and in the objective.
+ * Communication domains = maximal runs of layers held by the same device in every pipeline.
  * --------------------------------------------------------------------------------- */
 typedef struct {
     int32_t topk;              /* 1 .. CM_MAX_SHORTLIST                                   */
-    int32_t reserved;
+    int32_t sync_rounds;       /* 0: step time as the search computes it; 1: asymmetric
+                                  synchronisation rounds (below)                           */
     double t_gap_ns;           /* time between two faults (fp64 mode), finite, > 0          */
     double t_restart_ns;       /* restart overhead of a reconstruction (fp64 mode), >= 0     */
     int64_t t_gap_ns_i;        /* the same, integer nanoseconds (int64 mode)                */
@@ -266,6 +278,10 @@ typedef struct {
     double t_trans;            /* transition time, ns (fp64 mode; 0 in int64 mode)          */
     int64_t t_trans_ns;        /* transition time, ns (int64 mode; 0 in fp64 mode)          */
     double objective;          /* steps before the next fault (int64 mode: numerator / denominator rounded once) */
+    int32_t rounds, domains;   /* sync_rounds = 1, dynamic parallelism: communication rounds and
+                                  communication domains of the chosen plan; 0 otherwise     */
+    double t_sync;             /* time of those rounds, ns (fp64 mode)                      */
+    int64_t t_sync_ns;         /* time of those rounds, ns (int64 mode)                     */
     uint16_t assign[CM_MAX_MATCH]; /* dynamic parallelism: position j (pipeline-major, stage-minor) ->
                                       index, among the survivors in ascending id order, of the device
                                       that takes it; zeros otherwise                         */
@@ -275,8 +291,9 @@ typedef struct {
  * failed_ids / offsets / opts as for cm_search_batch (HOST).  best[B] and trans[B] (HOST,
  * caller-owned) receive the chosen plan (plan.cost / cost_ns = its step time) and its
  * transition.  shortlist (HOST [B * topk], may be NULL) receives the shortlisted plans in
- * rank order, shortlist_bytes (HOST [B * topk], may be NULL) their matched bytes; unused
- * slots have feasible = 0 and bytes = -1.  Several matchings of one plan can be optimal:
+ * rank order, shortlist_bytes (HOST [B * topk], may be NULL) their matched bytes,
+ * shortlist_rounds (HOST [B * topk], may be NULL) their communication rounds (0 unless
+ * sync_rounds = 1); unused slots have feasible = 0, bytes = -1, rounds = 0.  Several matchings of one plan can be optimal:
  * assign[] is one of them, xfer_bytes is unique.
  * Errors: CM_EINVAL (bad options; more than CM_MAX_MATCH devices in the profile's grid),
  * CM_ENOPROFILE, CM_EOVERFLOW, CM_ENOMEM, CM_ECUDA.  A scenario without any feasible plan
@@ -284,11 +301,11 @@ typedef struct {
 cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
                               const cm_enum_opts *opts, const cm_objective_opts *objective,
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist,
-                              int64_t *shortlist_bytes);
+                              int64_t *shortlist_bytes, int32_t *shortlist_rounds);
 
 /* Device time and work of the objective pass of the last cm_search_objective (HOST out[8]):
  * [0] shortlist kernel, ns  [1] completing the shortlisted plans (tie-break kernels), ns
- * [2] matching kernel, ns  [3] objective kernel, ns  [4] matchings solved (only counted when
+ * [2] matching kernel (and, with sync_rounds, the rounds kernel), ns  [3] objective kernel, ns  [4] matchings solved (only counted when
  * shortlist_bytes was asked for)  [5] kernels launched  [6] bytes copied device->host
  * [7] sum of [0..3].  cm_last_stats describes the search that ran before it. */
 cm_status cm_objective_stats(const cm_ctx *ctx, uint64_t out[8]);

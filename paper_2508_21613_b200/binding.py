@@ -65,7 +65,7 @@ class cm_plan(C.Structure):
 
 
 class cm_objective_opts(C.Structure):
-    _fields_ = [("topk", C.c_int32), ("reserved", C.c_int32), ("t_gap_ns", C.c_double),
+    _fields_ = [("topk", C.c_int32), ("sync_rounds", C.c_int32), ("t_gap_ns", C.c_double),
                 ("t_restart_ns", C.c_double), ("t_gap_ns_i", C.c_int64), ("t_restart_ns_i", C.c_int64),
                 ("bw_xfer_Bpns", C.c_int64)]
 
@@ -73,7 +73,8 @@ class cm_objective_opts(C.Structure):
 class cm_transition(C.Structure):
     _fields_ = [("policy", C.c_int32), ("feasible", C.c_int32), ("rank", C.c_int32), ("n_survivors", C.c_int32),
                 ("xfer_bytes", C.c_int64), ("t_trans", C.c_double), ("t_trans_ns", C.c_int64),
-                ("objective", C.c_double), ("assign", C.c_uint16 * 256)]
+                ("objective", C.c_double), ("rounds", C.c_int32), ("domains", C.c_int32),
+                ("t_sync", C.c_double), ("t_sync_ns", C.c_int64), ("assign", C.c_uint16 * 256)]
 
 
 @dataclass
@@ -142,7 +143,8 @@ def load_library() -> C.CDLL:
     lib.cm_evaluate_argmin_noalloc.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp, vp, vp]
     lib.cm_search_objective.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_int32), C.c_int32,
                                         C.POINTER(cm_enum_opts), C.POINTER(cm_objective_opts), C.POINTER(cm_plan),
-                                        C.POINTER(cm_transition), C.POINTER(cm_plan), C.POINTER(C.c_int64)]
+                                        C.POINTER(cm_transition), C.POINTER(cm_plan), C.POINTER(C.c_int64),
+                                        C.POINTER(C.c_int32)]
     lib.cm_objective_stats.argtypes = [vp, u64p]
     lib.cm_transfer_matching.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), vp, vp, vp, vp,
                                          C.POINTER(C.c_int64), C.POINTER(C.c_uint16)]
@@ -282,14 +284,15 @@ def cm_evaluate_argmin_noalloc(ctx, space, first: int, count: int, best_cost_dev
 
 
 def _objective(obj) -> cm_objective_opts:
-    return cm_objective_opts(int(obj.topk), 0, float(obj.t_gap_ns), float(obj.t_restart_ns),
+    return cm_objective_opts(int(obj.topk), int(getattr(obj, "sync_rounds", 0)), float(obj.t_gap_ns), float(obj.t_restart_ns),
                              int(round(obj.t_gap_ns)), int(round(obj.t_restart_ns)), int(obj.bw_xfer_Bpns))
 
 
 def cm_search_objective(ctx, scenarios: Sequence[Sequence[int]], opts, objective, shortlist: bool = False):
     """Search plus re-scoring with the transition time.  -> (best plans, transitions,
-    shortlisted plans or None, their matched bytes as numpy int64 [B, topk] or None); the
-    first three are ctypes arrays (cm_plan / cm_transition), shortlist slots scenario-major."""
+    shortlisted plans or None, their matched bytes as numpy int64 [B, topk] or None, their
+    communication rounds as numpy int32 [B, topk] or None); the first three are ctypes arrays
+    (cm_plan / cm_transition), shortlist slots scenario-major."""
     packed = PackedScenarios(scenarios)
     return packed.search_objective(ctx, opts, objective, shortlist)
 
@@ -382,8 +385,10 @@ class PackedScenarios:
         trans = (cm_transition * max(B, 1))()
         sl = (cm_plan * max(B * k, 1))() if shortlist else None
         sb = np.full((max(B, 1), max(k, 1)), -1, dtype=np.int64) if shortlist else None
+        sr = np.zeros((max(B, 1), max(k, 1)), dtype=np.int32) if shortlist else None
         _check(ctx, load_library().cm_search_objective(
             ctx, self.ids.ctypes.data_as(C.POINTER(C.c_uint32)), self.offsets.ctypes.data_as(C.POINTER(C.c_int32)),
             B, C.byref(o), C.byref(q), best, trans, sl,
-            sb.ctypes.data_as(C.POINTER(C.c_int64)) if shortlist else None))
-        return best, trans, sl, sb
+            sb.ctypes.data_as(C.POINTER(C.c_int64)) if shortlist else None,
+            sr.ctypes.data_as(C.POINTER(C.c_int32)) if shortlist else None))
+        return best, trans, sl, sb, sr

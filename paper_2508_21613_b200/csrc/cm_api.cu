@@ -97,6 +97,9 @@ struct Batch {
     DevBuf<uint64_t> d_short_kappa;
     DevBuf<int64_t> d_short_bytes;
     DevBuf<uint16_t> d_short_assign;
+    DevBuf<uint64_t> d_short_step;
+    DevBuf<int32_t> d_short_rounds;
+    PinnedVec<int32_t> short_rounds_host;
     DevBuf<cm_plan> d_short_plans, d_obj_best;
     DevBuf<cm_transition> d_trans;
     PinnedVec<cm_plan> obj_best_host, short_plans_host;
@@ -919,7 +922,8 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
 
 cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
                               const cm_enum_opts *opts, const cm_objective_opts *objective,
-                              cm_plan *best, cm_transition *trans, cm_plan *shortlist, int64_t *shortlist_bytes) {
+                              cm_plan *best, cm_transition *trans, cm_plan *shortlist, int64_t *shortlist_bytes,
+                              int32_t *shortlist_rounds) {
     if (!ctx) return CM_EINVAL;
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (B < 0 || !offsets || !best || !trans || !objective || (offsets[B] > 0 && !failed_ids))
@@ -929,6 +933,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     const cm_objective_opts &q = *objective;
     if (q.topk < 1 || q.topk > CM_MAX_SHORTLIST) return fail(ctx, CM_EINVAL, "topk must be 1 .. CM_MAX_SHORTLIST");
     if (q.bw_xfer_Bpns <= 0) return fail(ctx, CM_EINVAL, "transfer bandwidth must be positive");
+    if (q.sync_rounds != 0 && q.sync_rounds != 1) return fail(ctx, CM_EINVAL, "sync_rounds must be 0 or 1");
     if (!(q.t_gap_ns > 0.0) || !std::isfinite(q.t_gap_ns) || !(q.t_restart_ns >= 0.0) || !std::isfinite(q.t_restart_ns) ||
         q.t_gap_ns_i <= 0 || q.t_restart_ns_i < 0 || q.t_gap_ns_i > (1ll << 60) || q.t_restart_ns_i > (1ll << 60))
         return fail(ctx, CM_EINVAL, "fault gap must be positive and finite, restart overhead non-negative");
@@ -950,15 +955,18 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     const size_t slots = (size_t)B * q.topk;
     bool ok = bt.d_short_win.reserve(slots) && bt.d_short_kappa.reserve(slots * kMaxP) && bt.d_short_bytes.reserve(slots) &&
               bt.d_short_assign.reserve(slots * kMaxMatch) && bt.d_short_plans.reserve(slots) &&
+              bt.d_short_step.reserve(slots * 2) && bt.d_short_rounds.reserve(slots * 2) &&
               bt.d_obj_best.reserve(B) && bt.d_trans.reserve(B);
     if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
     ok = bt.obj_best_host.resize(B) && bt.trans_host.resize(B) && bt.short_plans_host.resize(slots) &&
-         bt.short_bytes_host.resize(slots);
+         bt.short_bytes_host.resize(slots) && bt.short_rounds_host.resize(slots * 2);
     if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
     const Tables tb = tables(ctx, bt.opts.cost);
     const BatchDev bd = dev_view(ctx, bt);
     ObjDev od{};
     od.topk = q.topk;
+    od.sync_rounds = q.sync_rounds;
+    od.short_step = bt.d_short_step.p; od.short_rounds = bt.d_short_rounds.p;
     od.t_gap = q.t_gap_ns; od.t_restart = q.t_restart_ns;
     od.t_gap_i = q.t_gap_ns_i; od.t_restart_i = q.t_restart_ns_i; od.bw_xfer = q.bw_xfer_Bpns;
     od.short_win = bt.d_short_win.p; od.short_kappa = bt.d_short_kappa.p; od.short_bytes = bt.d_short_bytes.p;
@@ -985,6 +993,10 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[2], st));
     CM_CUDA(ctx, launch_plan_matching(tb, bd, od, st));
     ++obj_launches;
+    if (q.sync_rounds) {
+        CM_CUDA(ctx, launch_plan_rounds(tb, bd, od, st));
+        ++obj_launches;
+    }
     CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[3], st));
     CM_CUDA(ctx, launch_objective(tb, bd, od, st));
     ++obj_launches;
@@ -1000,6 +1012,10 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     if (shortlist_bytes) {
         CM_CUDA(ctx, cudaMemcpyAsync(bt.short_bytes_host.p, bt.d_short_bytes.p, sizeof(int64_t) * slots, cudaMemcpyDeviceToHost, st));
         back += sizeof(int64_t) * slots;
+    }
+    if (shortlist_rounds && q.sync_rounds) {
+        CM_CUDA(ctx, cudaMemcpyAsync(bt.short_rounds_host.p, bt.d_short_rounds.p, sizeof(int32_t) * 2 * slots, cudaMemcpyDeviceToHost, st));
+        back += sizeof(int32_t) * 2 * slots;
     }
     CM_CUDA(ctx, cudaStreamSynchronize(st));
     for (int i = 0; i < 4; ++i) {
@@ -1021,6 +1037,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     for (size_t i = 0; i < slots; ++i) {
         if (shortlist) { cm_plan pl = bt.short_plans_host[i]; scrub(pl); shortlist[i] = pl; }
         if (shortlist_bytes) { shortlist_bytes[i] = bt.short_bytes_host[i]; solved += bt.short_bytes_host[i] >= 0; }
+        if (shortlist_rounds) shortlist_rounds[i] = q.sync_rounds ? bt.short_rounds_host[i * 2] : 0;
     }
     ctx->obj_stats[4] = solved;
     return CM_OK;

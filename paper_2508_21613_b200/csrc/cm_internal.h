@@ -167,13 +167,15 @@ struct Tables {
 constexpr int kMaxShort = CM_MAX_SHORTLIST;
 constexpr int kMaxMatch = CM_MAX_MATCH;
 struct ObjDev {
-    int32_t topk, pad;
+    int32_t topk, sync_rounds;
     double t_gap, t_restart;
     int64_t t_gap_i, t_restart_i, bw_xfer;
     Winner *short_win;        // [B*topk]
     uint64_t *short_kappa;    // [B*topk][kMaxP]
     int64_t *short_bytes;     // [B*topk] bytes moved by the cheapest migration, -1 = empty slot
     uint16_t *short_assign;   // [B*topk][kMaxMatch] position -> survivor index
+    uint64_t *short_step;     // [B*topk][2] step time / time of the rounds under asymmetric synchronisation (cost bits)
+    int32_t *short_rounds;    // [B*topk][2] communication rounds, communication domains
     cm_plan *short_plans;     // [B*topk] or NULL
     cm_plan *best;            // [B]
     cm_transition *trans;     // [B]
@@ -216,6 +218,7 @@ cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand,
 // cm_restore.cu
 cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
 cudaError_t launch_plan_matching(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
+cudaError_t launch_plan_rounds(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
 cudaError_t launch_objective(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st);
 // stand-alone matchings over explicit layer ranges ([n_problems][kMaxMatch] each)
 cudaError_t launch_range_matching(const Tables &t, int n_problems, const int32_t *sizes, const uint8_t *old_lo,

@@ -5,6 +5,8 @@
 //   cm_plan_matching_kernel   one warp per shortlisted plan: layer ranges of the survivors
 //                             before and after, minimum-cost perfect matching
 //   cm_range_matching_kernel  the same matching over caller-given layer ranges
+//   cm_plan_rounds_kernel     one warp per shortlisted plan: communication rounds of the
+//                             asymmetric synchronisation and the step time they give
 //   cm_objective_kernel       per scenario: steps before the next fault of every candidate,
 //                             the best one, its plan and its migration scheme
 //
@@ -226,6 +228,25 @@ __device__ __forceinline__ void stage_state_bytes(long long *PW, const DevProfil
     __syncthreads();
 }
 
+// Layer cuts of pipeline q of a shortlisted plan: its completed layer composition, or the
+// min-max partition; false if the completion found no composition (cannot happen for a
+// feasible pair) or the partition does not exist.
+__device__ __forceinline__ bool pipeline_cuts(const Tables &tb, const BatchDev &bd, const ObjDev &od, size_t slot,
+                                              const Winner &w, int q, uint8_t *cuts /* [S+1] */) {
+    const TSeg g = bd.tseg[w.seg[q]];
+    const uint64_t kappa = od.short_kappa[slot * kMaxP + q];
+    const int S = g.S;
+    if (kappa < g.K) {
+        layer_cuts(tb.binom, bd.layer_mode, tb.prof->L, S, kappa, cuts);
+        return true;
+    }
+    if (kappa != g.K) return false;
+    const uint8_t *mm = tb.mm_cuts + (size_t)tb.mm_slot(S, g.m) * (kMaxS + 1);
+    if (mm[0] != 0) return false;
+    for (int i = 0; i <= S; ++i) cuts[i] = mm[i];
+    return true;
+}
+
 // One warp per shortlist slot: survivors keep the layers of their old stage (device =
 // pipeline * n_pp + stage); position off_p + i of the plan holds stage i of pipeline p.
 __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_matching_kernel(Tables tb, BatchDev bd, ObjDev od, uint64_t inf) {
@@ -260,17 +281,10 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_matching_kernel(Tabl
         const Strat &s = bd.strat[w.strat];
         int off = 0;
         for (int q = 0; q < lane; ++q) off += s.S[q];
-        const TSeg g = bd.tseg[w.seg[lane]];
-        const uint64_t kappa = od.short_kappa[slot * kMaxP + lane];
-        const int S = g.S;
+        const int S = s.S[lane];
         uint8_t cuts[kMaxS + 1];
         if (off + S > n) ok = false;
-        else if (kappa < g.K) layer_cuts(tb.binom, bd.layer_mode, p->L, S, kappa, cuts);
-        else if (kappa == g.K) {
-            const uint8_t *mm = tb.mm_cuts + (size_t)tb.mm_slot(S, g.m) * (kMaxS + 1);
-            if (mm[0] != 0) ok = false;
-            else for (int i = 0; i <= S; ++i) cuts[i] = mm[i];
-        } else ok = false;                                   // no composition met the step time
+        else ok = pipeline_cuts(tb, bd, od, slot, w, lane, cuts);
         if (ok) {
             for (int i = 0; i < S; ++i) { mw.nlo[off + i] = cuts[i]; mw.nhi[off + i] = cuts[i + 1]; }
             covered = S;
@@ -329,6 +343,106 @@ cudaError_t launch_range_matching(const Tables &t, int n_problems, const int32_t
 }
 
 // ----------------------------------------------------------------------------------
+// Asymmetric synchronisation (Section "Restorer", Asymmetric Communication).  One warp per
+// shortlisted plan: lane q evaluates the bare time of pipeline q (one participant: no
+// synchronisation term) and writes the stage of every layer; the layer graph (edge = some
+// pipeline keeps both layers on one device) is coloured greedily in layer order, lanes
+// sharing the earlier layers and OR-reducing the colours their neighbours took; a round
+// lasts as long as its largest all-reduce, rounds add up in colour order.
+// ----------------------------------------------------------------------------------
+struct RoundsWork {
+    uint8_t stage_of[kMaxP][kMaxL];
+    uint8_t colour[kMaxL];
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables tb, BatchDev bd, ObjDev od) {
+    __shared__ SProf<T> sp;
+    __shared__ RoundsWork work[kMatchWarps];
+    stage_profile(sp, tb.prof);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t slot = (size_t)blockIdx.x * kMatchWarps + warp;
+    if (slot >= (size_t)bd.B * od.topk) return;
+    if (lane < 2) { od.short_step[slot * 2 + lane] = inf_bits<T>(); od.short_rounds[slot * 2 + lane] = 0; }
+    const Winner &w = od.short_win[slot];
+    if (w.cost_bits >= inf_bits<T>() || w.dp == 0) return;
+    RoundsWork &rw = work[warp];
+    const int L = sp.L, dp = (int)w.dp;
+    T t_pipe = (T)0;
+    bool ok = true;
+    if (lane < dp) {
+        uint8_t cuts[kMaxS + 1];
+        ok = pipeline_cuts(tb, bd, od, slot, w, lane, cuts);
+        if (ok) {
+            const SegView g = seg_view(bd, w.scen, w.seg[lane]);
+            for (int i = 0; i < g.S; ++i)
+                for (int l = cuts[i]; l < cuts[i + 1]; ++l) rw.stage_of[lane][l] = (uint8_t)i;
+            ok = pipe_cost_from_cuts<T>(sp, g.S, g.m, cuts, g.tier, 1, t_pipe);
+        }
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) return;
+    for (int o = 16; o > 0; o >>= 1) {
+        const uint64_t other = __shfl_xor_sync(0xffffffffu, Num<T>::bits(t_pipe), o);
+        t_pipe = tmax(t_pipe, Num<T>::from_bits(other));     // times are non-negative: bit order = value order
+    }
+    __syncwarp();
+    int rounds = 0;
+    for (int l = 0; l < L; ++l) {
+        uint32_t used[4] = {0u, 0u, 0u, 0u};
+        for (int k = lane; k < l; k += 32) {
+            bool adjacent = false;
+            for (int q = 0; q < dp; ++q) adjacent = adjacent || rw.stage_of[q][l] == rw.stage_of[q][k];
+            if (adjacent) { const int c = rw.colour[k]; used[c >> 5] |= 1u << (c & 31); }
+        }
+        int c = -1;
+#pragma unroll
+        for (int word = 0; word < 4; ++word) {
+            const uint32_t all = __reduce_or_sync(0xffffffffu, used[word]);
+            if (c < 0 && all != 0xffffffffu) c = word * 32 + __ffs((int)~all) - 1;
+        }
+        if (lane == 0) rw.colour[l] = (uint8_t)c;
+        rounds = c + 1 > rounds ? c + 1 : rounds;
+        __syncwarp();
+    }
+    T t_sync = (T)0;
+    for (int c = 0; c < rounds; ++c) {
+        T longest = (T)0;
+        for (int l = lane; l < L; l += 32)
+            if (rw.colour[l] == c) longest = tmax(longest, Num<T>::sync(sp.PP[l + 1] - sp.PP[l], dp, sp.bw_sync));
+        for (int o = 16; o > 0; o >>= 1) {
+            const uint64_t other = __shfl_xor_sync(0xffffffffu, Num<T>::bits(longest), o);
+            longest = tmax(longest, Num<T>::from_bits(other));
+        }
+        t_sync = t_sync + longest;
+    }
+    int domains = 0;
+    for (int base = 0; base < L; base += 32) {
+        const int l = base + lane;
+        bool fresh = l == 0;
+        if (l > 0 && l < L)
+            for (int q = 0; q < dp; ++q) fresh = fresh || rw.stage_of[q][l] != rw.stage_of[q][l - 1];
+        domains += __popc(__ballot_sync(0xffffffffu, fresh && l < L));
+    }
+    if (lane == 0) {
+        od.short_step[slot * 2] = Num<T>::bits(t_pipe + t_sync);
+        od.short_step[slot * 2 + 1] = Num<T>::bits(t_sync);
+        od.short_rounds[slot * 2] = rounds;
+        od.short_rounds[slot * 2 + 1] = domains;
+    }
+}
+
+cudaError_t launch_plan_rounds(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
+    if (b.B <= 0) return cudaSuccess;
+    const size_t slots = (size_t)b.B * o.topk;
+    const unsigned grid = (unsigned)((slots + kMatchWarps - 1) / kMatchWarps);
+    if (b.mode == CM_COST_INT64NS) cm_plan_rounds_kernel<long long><<<grid, kMatchWarps * 32, 0, st>>>(t, b, o);
+    else cm_plan_rounds_kernel<double><<<grid, kMatchWarps * 32, 0, st>>>(t, b, o);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
 // Objective (Section "Problem Formulation"): steps before the next fault,
 // (t_gap - t_trans) / t_step, of rerouting, redundant computation (t_trans = 0) and every
 // shortlisted plan (t_trans = restart + matched bytes / bandwidth).  The greatest wins,
@@ -345,11 +459,12 @@ __device__ __forceinline__ bool frac_greater(const Frac &a, const Frac &b, int m
     return a.nd / a.dd > b.nd / b.dd;
 }
 
-__device__ __forceinline__ void plan_from_winner(const BatchDev &bd, const Winner &w, const uint64_t *kappa, cm_plan &pl) {
+__device__ __forceinline__ void plan_from_winner(const BatchDev &bd, const Winner &w, const uint64_t *kappa,
+                                                 uint64_t step_bits, cm_plan &pl) {
     plan_clear(pl, CM_DYNPAR);
     const Strat &s = bd.strat[w.strat];
     pl.feasible = 1;
-    plan_set_cost(pl, w.cost_bits, bd.mode);
+    plan_set_cost(pl, step_bits, bd.mode);
     pl.strategy = w.strat - bd.tmpl[bd.scen[w.scen].tmpl].strat_first;
     pl.n_pipes = w.dp;
     pl.split_rank = w.item - s.split_first;
@@ -367,6 +482,7 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
     const cm_plan *pol = bd.plans + (size_t)b * 4;
     if (threadIdx.x == 0) {
         cm_transition tr;
+        tr.rounds = 0; tr.domains = 0; tr.t_sync = 0.0; tr.t_sync_ns = 0;
         tr.policy = 0; tr.feasible = 0; tr.rank = -1;
         tr.n_survivors = tb.prof->n_dp * tb.prof->n_pp - (int)bd.scen[b].n_failed;
         tr.xfer_bytes = 0; tr.t_trans = 0.0; tr.t_trans_ns = 0; tr.objective = 0.0;
@@ -382,18 +498,19 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
             const size_t slot = (size_t)b * od.topk + r;
             const long long bytes = od.short_bytes[slot];
             if (bytes < 0) continue;
-            const Winner &w = od.short_win[slot];
+            const uint64_t step = od.sync_rounds ? od.short_step[slot * 2] : od.short_win[slot].cost_bits;
+            if (step >= inf) continue;
             Frac j{0.0, 1.0, 0, 1};
             double tt = 0.0;
             long long tti = 0;
             if (mode == CM_COST_INT64NS) {
                 tti = od.t_restart_i + bytes / od.bw_xfer;
                 j.ni = od.t_gap_i - tti;
-                j.di = (long long)w.cost_bits;
+                j.di = (long long)step;
             } else {
                 tt = od.t_restart + (double)bytes / (double)od.bw_xfer;
                 j.nd = od.t_gap - tt;
-                j.dd = __longlong_as_double((long long)w.cost_bits);
+                j.dd = __longlong_as_double((long long)step);
             }
             if (!have || frac_greater(j, best, mode)) {
                 have = true; best = j; slot_sel = (int)r;
@@ -407,7 +524,14 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
             tr.rank = -1; tr.xfer_bytes = 0; tr.t_trans = 0.0; tr.t_trans_ns = 0;
         } else {
             const size_t slot = (size_t)b * od.topk + slot_sel;
-            plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, pl);
+            plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP,
+                             od.sync_rounds ? od.short_step[slot * 2] : od.short_win[slot].cost_bits, pl);
+            if (od.sync_rounds) {
+                tr.rounds = od.short_rounds[slot * 2];
+                tr.domains = od.short_rounds[slot * 2 + 1];
+                if (mode == CM_COST_INT64NS) tr.t_sync_ns = (long long)od.short_step[slot * 2 + 1];
+                else tr.t_sync = __longlong_as_double((long long)od.short_step[slot * 2 + 1]);
+            }
         }
         if (have) {
             tr.feasible = 1;
@@ -419,6 +543,7 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
         out->policy = tr.policy; out->feasible = tr.feasible; out->rank = tr.rank; out->n_survivors = tr.n_survivors;
         out->xfer_bytes = tr.xfer_bytes; out->t_trans = tr.t_trans; out->t_trans_ns = tr.t_trans_ns;
         out->objective = tr.objective;
+        out->rounds = tr.rounds; out->domains = tr.domains; out->t_sync = tr.t_sync; out->t_sync_ns = tr.t_sync_ns;
         win_slot = (have && tr.policy == CM_DYNPAR) ? slot_sel : -1;
     }
     __syncthreads();
@@ -427,7 +552,8 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
     if (od.short_plans && (int)threadIdx.x < od.topk) {
         const size_t slot = (size_t)b * od.topk + threadIdx.x;
         cm_plan pl;
-        if (od.short_bytes[slot] >= 0) plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, pl);
+        const uint64_t step = od.sync_rounds ? od.short_step[slot * 2] : od.short_win[slot].cost_bits;
+        if (od.short_bytes[slot] >= 0 && step < inf) plan_from_winner(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, step, pl);
         else plan_clear(pl, CM_DYNPAR);
         od.short_plans[slot] = pl;
     }

@@ -73,7 +73,7 @@ def test_full_objective_of_every_scenario_matches_the_stored_oracle_result(gpu, 
     ctx = gpu.cm_create(0)
     try:
         gpu.cm_load_profile(ctx, w.profile)
-        best, trans, sl, sb = gpu.cm_search_objective(ctx, w.scenarios, w.options.with_cost_mode(mode), obj,
+        best, trans, sl, sb, _ = gpu.cm_search_objective(ctx, w.scenarios, w.options.with_cost_mode(mode), obj,
                                                       shortlist=True)
         plans = gpu.plans_from_array(best)
         short = gpu.plans_from_array(sl)

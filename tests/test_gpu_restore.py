@@ -101,7 +101,7 @@ def test_matching_rejects_bad_problems(gpu):
 
 
 def _check_objective(gpu, o, w, scenarios, opts, obj, mode, res):
-    best, trans, sl, sb = res
+    best, trans, sl, sb, sr = res
     p = w.profile
     wts = o.state_bytes()
     for b, failed in enumerate(scenarios):
@@ -123,6 +123,8 @@ def _check_objective(gpu, o, w, scenarios, opts, obj, mode, res):
             assert tr.t_trans == wt.t_trans, what
         assert abs(tr.objective - wt.objective) <= REL_TOL * abs(wt.objective), what
         assert tr.objective == wt.objective, what
+        assert (tr.rounds, tr.domains, tr.t_sync_ns) == (wt.rounds, wt.domains, wt.t_sync_ns), what
+        assert tr.t_sync == wt.t_sync, what
         # the shortlist, slot by slot
         k = obj.topk
         plans = gpu.plans_from_array([sl[b * k + r] for r in range(k)])
@@ -130,6 +132,9 @@ def _check_objective(gpu, o, w, scenarios, opts, obj, mode, res):
             if r < len(wt.shortlist):
                 assert plans[r].feasible and plans[r].key() == wt.shortlist[r].key(), f"{what} rank {r}"
                 assert int(sb[b, r]) == wt.shortlist_bytes[r], f"{what} rank {r}"
+                assert int(sr[b, r]) == wt.shortlist_rounds[r], f"{what} rank {r}"
+                a, c = (plans[r].cost_ns, wt.shortlist[r].cost_ns) if mode else (plans[r].cost, wt.shortlist[r].cost)
+                assert a == c, f"{what} rank {r}: step time {a!r} != {c!r}"
             else:
                 assert not plans[r].feasible and int(sb[b, r]) == -1, f"{what} rank {r}"
         # the migration scheme: a permutation of the survivors whose cost is the matched bytes
@@ -155,7 +160,8 @@ def test_objective_parity_tiny(gpu, oracle_factory, mode):
         s = Session(gpu, w.profile)
         try:
             for obj in (W.ObjectiveOptions(topk=1), W.ObjectiveOptions(topk=6, t_gap_ns=40e9, bw_xfer_Bpns=1),
-                        W.ObjectiveOptions(topk=16, t_gap_ns=1e14, t_restart_ns=0.0)):
+                        W.ObjectiveOptions(topk=16, t_gap_ns=1e14, t_restart_ns=0.0),
+                        W.ObjectiveOptions(topk=7, sync_rounds=1)):
                 res = gpu.cm_search_objective(s.ctx, w.scenarios, opts, obj, shortlist=True)
                 _check_objective(gpu, o, w, w.scenarios, opts, obj, mode, res)
         finally:
@@ -173,28 +179,30 @@ def test_objective_parity_random_small(gpu, oracle_factory, mode):
         s = Session(gpu, w.profile)
         try:
             obj = W.ObjectiveOptions(topk=1 + seed % 5, t_gap_ns=[1e9, 30e9, 1125e9][seed % 3],
-                                     t_restart_ns=[0.0, 2e9][seed % 2], bw_xfer_Bpns=1 + seed)
+                                     t_restart_ns=[0.0, 2e9][seed % 2], bw_xfer_Bpns=1 + seed,
+                                     sync_rounds=(seed // 2) % 2)
             res = gpu.cm_search_objective(s.ctx, w.scenarios, opts, obj, shortlist=True)
             _check_objective(gpu, o, w, w.scenarios, opts, obj, mode, res)
         finally:
             s.close()
 
 
+@pytest.mark.parametrize("rounds", [0, 1])
 @pytest.mark.parametrize("mode", [0, 1])
-def test_objective_parity_paper_scale_sampled(gpu, oracle_factory, mode):
+def test_objective_parity_paper_scale_sampled(gpu, oracle_factory, mode, rounds):
     w = W.paper_scale()
     opts = w.options.with_cost_mode(mode)
     o = oracle_factory(w.profile, opts)
     s = Session(gpu, w.profile)
     try:
-        obj = W.ObjectiveOptions()
+        obj = W.ObjectiveOptions(sync_rounds=rounds)
         # the whole batch runs in the launch configuration the bench times; a sample is checked one by one
         res = gpu.cm_search_objective(s.ctx, w.scenarios, opts, obj, shortlist=True)
         pick = list(range(0, len(w.scenarios), 97))[:28]
-        best, trans, sl, sb = res
+        best, trans, sl, sb, sr = res
         k = obj.topk
         sub = ([best[b] for b in pick], [trans[b] for b in pick],
-               [sl[b * k + r] for b in pick for r in range(k)], sb[pick])
+               [sl[b * k + r] for b in pick for r in range(k)], sb[pick], sr[pick])
         _check_objective(gpu, o, w, [w.scenarios[b] for b in pick], opts, obj, mode, sub)
         # properties that hold for every scenario of the batch
         for b in range(len(w.scenarios)):
@@ -231,7 +239,7 @@ def test_objective_parity_255_device_matchings(gpu, oracle_factory):
     o = oracle_factory(w.profile, opts)
     s = Session(gpu, w.profile)
     try:
-        obj = W.ObjectiveOptions(topk=3)
+        obj = W.ObjectiveOptions(topk=3, sync_rounds=1)
         scen = [w.scenarios[0], w.scenarios[40]]
         res = gpu.cm_search_objective(s.ctx, scen, opts, obj, shortlist=True)
         _check_objective(gpu, o, w, scen, opts, obj, 0, res)
@@ -246,17 +254,18 @@ def test_objective_limits_and_errors(gpu):
         scen = w.scenarios[:16]
         plain, _, _ = gpu.cm_search_batch(s.ctx, scen, w.options)
         # faults far apart: the plain search's choice stands
-        best, trans, _, _ = gpu.cm_search_objective(s.ctx, scen, w.options, W.ObjectiveOptions(topk=4, t_gap_ns=1e18))
+        best, trans, _, _, _ = gpu.cm_search_objective(s.ctx, scen, w.options, W.ObjectiveOptions(topk=4, t_gap_ns=1e18))
         assert [p.key() for p in gpu.plans_from_array(best)] == [p.key() for p in gpu.plans_from_array(plain)]
         # faults closer together than a restart: no reconstruction
-        best, trans, _, _ = gpu.cm_search_objective(s.ctx, scen, w.options,
+        best, trans, _, _, _ = gpu.cm_search_objective(s.ctx, scen, w.options,
                                                     W.ObjectiveOptions(topk=4, t_gap_ns=4e9, t_restart_ns=5e9))
         assert all(trans[b].policy != W.POLICY_DYNPAR and trans[b].xfer_bytes == 0 for b in range(len(scen)))
         for bad in (W.ObjectiveOptions(topk=0), W.ObjectiveOptions(topk=17), W.ObjectiveOptions(bw_xfer_Bpns=0),
+                    W.ObjectiveOptions(sync_rounds=2),
                     W.ObjectiveOptions(t_gap_ns=0.0), W.ObjectiveOptions(t_restart_ns=-1.0)):
             with pytest.raises(gpu.ChameleonError):
                 gpu.cm_search_objective(s.ctx, scen, w.options, bad)
-        best, trans, _, _ = gpu.cm_search_objective(s.ctx, [], w.options, W.ObjectiveOptions())
+        best, trans, _, _, _ = gpu.cm_search_objective(s.ctx, [], w.options, W.ObjectiveOptions())
         st = gpu.cm_objective_stats(s.ctx)
         assert st["launches"] == 0
     finally:
