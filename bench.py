@@ -245,6 +245,7 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
 def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush):
     """The full-objective search (search + shortlist + weight-transfer matchings + ranking by
     steps before the next fault) through cm_search_objective, host buffers in and out."""
+    import numpy as np
     from paper_2508_21613_b200 import workloads as W
     opts = w.options.with_cost_mode(mode)
     obj = W.ObjectiveOptions()
@@ -275,7 +276,7 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
             changed += int(plain[b].policy != best[b].policy or plain[b].strategy != best[b].strategy
                            or plain[b].split_rank != best[b].split_rank)
         matchings = int((sb >= 0).sum())
-        return {
+        out = {
             "topk": obj.topk, "t_gap_s": obj.t_gap_ns * 1e-9, "t_restart_s": obj.t_restart_ns * 1e-9,
             "bw_xfer_GBps": obj.bw_xfer_Bpns, "scenarios": packed.B,
             "e2e_ms_per_call": 1e3 * wall / steps,
@@ -289,6 +290,31 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
             "choices_changed_by_transition_time": changed,
             "gpu_launches": int(phases["launches"] / steps),
         }
+        # the same with the asymmetric-synchronisation rounds in the step time
+        obj_r = W.ObjectiveOptions(sync_rounds=1)
+        packed.search_objective(ctx, opts, obj_r, shortlist=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        best_r, trans_r, _, _, sr = packed.search_objective(ctx, opts, obj_r, shortlist=True)
+        wall_r = time.perf_counter() - t0
+        ph = binding.cm_objective_stats(ctx)
+        dyn = [b for b in range(packed.B) if trans_r[b].policy == 2]
+        out["sync_rounds"] = {
+            "e2e_ms_per_call": 1e3 * wall_r,
+            "matching_plus_rounds_kernel_ms": 1e-6 * ph["matching_ns"],
+            "plans_coloured": int((sr > 0).sum()),
+            "rounds_mean": float(sr[sr > 0].mean()) if (sr > 0).any() else None,
+            "rounds_max": int(sr.max()),
+            "layers": int(w.profile.L),
+            "domains_mean_of_chosen": float(np.mean([trans_r[b].domains for b in dyn])) if dyn else None,
+            "chosen_policy_counts": {"reroute": sum(trans_r[b].policy == 0 for b in range(packed.B)),
+                                     "redundant": sum(trans_r[b].policy == 1 for b in range(packed.B)),
+                                     "dynpar": len(dyn)},
+            "choices_changed_vs_without_rounds": sum(
+                int(best[b].policy != best_r[b].policy or best[b].strategy != best_r[b].strategy
+                    or best[b].split_rank != best_r[b].split_rank) for b in range(packed.B)),
+        }
+        return out
     finally:
         binding.cm_destroy(ctx)
 

@@ -354,6 +354,61 @@ __device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mo
     else pl.cost = __longlong_as_double((long long)bits);
 }
 
+// ----------------------------------------------------------------------------------
+// The pipeline-time recurrence of ONE pipeline spread over a warp: PER consecutive stages
+// per lane (S <= 32 * PER), walked in lock step over time slots.  With unit durations the
+// 1F1B schedule puts forward (i,j) at slot i+j while j <= S-1-i and at slot i+2j afterwards,
+// and backward (i,j) at slot 2S-1-i+2j; taking those slots as the evaluation order is a
+// valid topological order for arbitrary durations and every m >= 1.  Every stage keeps
+// its clock, its latest forward end (transfer added) and its latest backward end; inputs
+// of a slot are gathered from the neighbours' state before any stage of the slot updates.
+// F, B, xt: the lane's own stages.  Returns the pipeline time in every lane.
+// ----------------------------------------------------------------------------------
+template <typename T, int PER>
+__device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B, const T *xt) {
+    const int lane = threadIdx.x & 31;
+    T clock[PER], last_f[PER], last_b[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) { clock[k] = (T)0; last_f[k] = (T)0; last_b[k] = (T)0; }
+    const int n_slots = 2 * (S + m) - 2;
+    for (int s = 0; s < n_slots; ++s) {
+        T f_in[PER], b_in[PER];
+        const T up = __shfl_up_sync(0xffffffffu, last_f[PER - 1], 1);
+        const T down = __shfl_down_sync(0xffffffffu, last_b[0], 1);
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            f_in[k] = k == 0 ? up : last_f[k > 0 ? k - 1 : 0];
+            b_in[k] = k == PER - 1 ? down : last_b[k < PER - 1 ? k + 1 : 0];
+        }
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            const int i = lane * PER + k;
+            if (i >= S) continue;
+            bool is_f = false, is_b = false;
+            const int d = s - i;
+            if (s <= S - 1) {
+                is_f = d >= 0 && d < m;
+            } else if ((d & 1) == 0) {
+                const int j = d >> 1;
+                is_f = j > S - 1 - i && j < m;
+            }
+            const int e = s - (2 * S - 1 - i);
+            if (e >= 0 && (e & 1) == 0) is_b = (e >> 1) < m;
+            if (is_f) {
+                const T start = i > 0 ? tmax(clock[k], f_in[k]) : clock[k];
+                clock[k] = start + F[k];
+                last_f[k] = clock[k] + xt[k];
+            } else if (is_b) {
+                const T dep = i < S - 1 ? b_in[k] + xt[k] : clock[k];   // last stage: its own forward just ended
+                const T start = tmax(clock[k], dep);
+                clock[k] = start + B[k];
+                last_b[k] = clock[k];
+            }
+        }
+    }
+    return __shfl_sync(0xffffffffu, clock[0], 0);
+}
+
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {
     for (int o = 16; o > 0; o >>= 1) {
         uint64_t w = __shfl_xor_sync(0xffffffffu, v, o);

@@ -352,8 +352,27 @@ cudaError_t launch_range_matching(const Tables &t, int n_problems, const int32_t
 // ----------------------------------------------------------------------------------
 struct RoundsWork {
     uint8_t stage_of[kMaxP][kMaxL];
+    uint8_t cuts[kMaxP][kMaxS + 4];
     uint8_t colour[kMaxL];
 };
+
+// Bare time of one pipeline (no synchronisation term), its stages spread over the warp.
+template <typename T, int PER>
+__device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *cuts, int S, int m, uint64_t tier, int lane) {
+    T F[PER], B[PER], xt[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        const int i = lane * PER + k;
+        F[k] = (T)0; B[k] = (T)0; xt[k] = (T)0;
+        if (i < S) {
+            const int lo = cuts[i], hi = cuts[i + 1];
+            F[k] = sp.PF[hi] - sp.PF[lo];
+            B[k] = sp.PB[hi] - sp.PB[lo];
+            if (i < S - 1) xt[k] = sp.XT[(tier >> i) & 1ull][hi - 1];
+        }
+    }
+    return sim_lockstep_n<T, PER>(S, m, F, B, xt);
+}
 
 template <typename T>
 __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables tb, BatchDev bd, ObjDev od) {
@@ -369,25 +388,28 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables
     if (w.cost_bits >= inf_bits<T>() || w.dp == 0) return;
     RoundsWork &rw = work[warp];
     const int L = sp.L, dp = (int)w.dp;
-    T t_pipe = (T)0;
     bool ok = true;
     if (lane < dp) {
         uint8_t cuts[kMaxS + 1];
         ok = pipeline_cuts(tb, bd, od, slot, w, lane, cuts);
         if (ok) {
-            const SegView g = seg_view(bd, w.scen, w.seg[lane]);
-            for (int i = 0; i < g.S; ++i)
+            const int S = bd.tseg[w.seg[lane]].S;
+            for (int i = 0; i <= S; ++i) rw.cuts[lane][i] = cuts[i];
+            for (int i = 0; i < S; ++i)
                 for (int l = cuts[i]; l < cuts[i + 1]; ++l) rw.stage_of[lane][l] = (uint8_t)i;
-            ok = pipe_cost_from_cuts<T>(sp, g.S, g.m, cuts, g.tier, 1, t_pipe);
         }
     }
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) return;
-    for (int o = 16; o > 0; o >>= 1) {
-        const uint64_t other = __shfl_xor_sync(0xffffffffu, Num<T>::bits(t_pipe), o);
-        t_pipe = tmax(t_pipe, Num<T>::from_bits(other));     // times are non-negative: bit order = value order
-    }
     __syncwarp();
+    T t_pipe = (T)0;
+    for (int q = 0; q < dp; ++q) {            // one pipeline after the other, each over the whole warp
+        const SegView g = seg_view(bd, w.scen, w.seg[q]);
+        T t;
+        if (g.S <= 32) t = warp_pipe_time<T, 1>(sp, rw.cuts[q], g.S, g.m, g.tier, lane);
+        else t = warp_pipe_time<T, 2>(sp, rw.cuts[q], g.S, g.m, g.tier, lane);
+        t_pipe = tmax(t_pipe, t);
+    }
     int rounds = 0;
     for (int l = 0; l < L; ++l) {
         uint32_t used[4] = {0u, 0u, 0u, 0u};
