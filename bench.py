@@ -319,6 +319,34 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
         binding.cm_destroy(ctx)
 
 
+def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
+    """Plan cache: every failure set of at most k devices searched ahead of time; lookups."""
+    from paper_2508_21613_b200 import workloads as W
+    opts = w.options.with_cost_mode(mode)
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    out = {}
+    try:
+        binding.cm_cache_free(binding.cm_cache_build(ctx, 1, opts)[0])           # warm-up
+        rng = W.SplitMix64(99)
+        n_dev = w.profile.n_dp * w.profile.n_pp
+        for k in sizes:
+            t0 = time.perf_counter()
+            cache, n = binding.cm_cache_build(ctx, k, opts)
+            dt = time.perf_counter() - t0
+            sets = [rng.sample_distinct(n_dev, 1 + rng.below(k)) for _ in range(2000)]
+            t0 = time.perf_counter()
+            for f in sets:
+                binding.cm_cache_lookup(cache, f)
+            lk = (time.perf_counter() - t0) / len(sets)
+            binding.cm_cache_free(cache)
+            out[f"up_to_{k}_failures"] = {"failure_sets": n, "build_ms": 1e3 * dt, "sets_per_s": n / dt,
+                                          "lookup_us_through_ctypes": 1e6 * lk}
+    finally:
+        binding.cm_destroy(ctx)
+    return out
+
+
 def roofline_of(stats_sum, dev_seconds, mode, sm_max, peak_kind):
     slots = ISSUE_SLOTS_PER_CELL[mode]
     peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
@@ -443,6 +471,8 @@ def main():
             line["full_objective"] = {
                 name: measure_objective(binding, torch, W.ALL_WORKLOADS[name](), args.cost_mode, 3, 3, local_rank, flush)
                 for name in dict.fromkeys((args.workload, "175b-like", "sweep"))}
+        if not args.no_extra and world == 1 and args.scenarios == 0 and w.profile.n_dp * w.profile.n_pp <= 64:
+            line["plan_cache"] = measure_cache(binding, w, args.cost_mode, local_rank)
         if args.objective and "full_objective" not in line:
             line["full_objective"] = {w.name: measure_objective(binding, torch, w, args.cost_mode, args.steps,
                                                                 args.warmup, local_rank, flush)}

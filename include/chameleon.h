@@ -322,6 +322,30 @@ cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *s
                                const uint8_t *new_lo, const uint8_t *new_hi,
                                int64_t *total, uint16_t *assign);
 
+/* ---------------------------------------------------------------------------------
+ * Plan cache (Section "Planner", last paragraph: the best plans for the loss of 1 to k
+ * devices are computed and cached during fault-free training, so that the decision at
+ * failure time is a lookup).  The cache holds the result of the search for EVERY failure
+ * set of at most max_failures devices (the empty set included) of the loaded profile's
+ * grid; entries are addressed by the set's size and combinatorial rank.
+ *
+ * cm_cache_build: max_failures 0 .. 16; the number of sets may not exceed 2^20
+ * (CM_EOVERFLOW).  Runs cm_search_batch over all
+ * sets, 4096 at a time, on the context's stream (synchronises).  The cache is a HOST object
+ * owned by the caller until cm_cache_free; it keeps no reference to device memory and stays
+ * valid when the profile is reloaded (its plans then describe the old profile).
+ * cm_cache_lookup: failed_ids in any order (HOST); best and per_policy[3] (may be NULL) are
+ * HOST out-parameters; exactly what cm_search_batch returns for that set.  Errors:
+ * CM_EINVAL (id out of range, duplicate ids), CM_ENOFEASIBLE if the set is larger than the
+ * cache covers (the caller searches it instead).  Thread-safe for concurrent lookups.
+ * --------------------------------------------------------------------------------- */
+typedef struct cm_cache cm_cache;
+cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *opts, cm_cache **out,
+                         uint64_t *n_scenarios);
+cm_status cm_cache_lookup(const cm_cache *cache, const uint32_t *failed_ids, int32_t n_failed,
+                          cm_plan *best, cm_plan *per_policy);
+cm_status cm_cache_free(cm_cache *cache);
+
 /* Work counters of the last cm_select / cm_search_batch / cm_batch_search on this
  * context (HOST out[16]):
  *  [0] pipeline-plans evaluated by the search pass   [1] recurrence cells simulated by it

@@ -29,8 +29,9 @@ CM_COST_FP64, CM_COST_INT64NS = 0, 1
 EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_evaluate", "cm_select",
            "cm_decode_plan", "cm_space_free", "cm_search_batch", "cm_batch_prepare", "cm_batch_search",
            "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
-           "cm_objective_stats", "cm_transfer_matching", "cm_strerror", "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:17]
+           "cm_objective_stats", "cm_transfer_matching", "cm_cache_build", "cm_cache_lookup", "cm_cache_free",
+           "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:20]
 NOALLOC_MAX_CANDIDATES = 524288
 MAX_SHORTLIST, MAX_MATCH = 16, 256
 
@@ -148,6 +149,9 @@ def load_library() -> C.CDLL:
     lib.cm_objective_stats.argtypes = [vp, u64p]
     lib.cm_transfer_matching.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), vp, vp, vp, vp,
                                          C.POINTER(C.c_int64), C.POINTER(C.c_uint16)]
+    lib.cm_cache_build.argtypes = [vp, C.c_int32, C.POINTER(cm_enum_opts), C.POINTER(vp), u64p]
+    lib.cm_cache_lookup.argtypes = [vp, C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_plan), C.POINTER(cm_plan)]
+    lib.cm_cache_free.argtypes = [vp]
     for name in _STATUS_CALLS:
         getattr(lib, name).restype = C.c_int
     _lib = lib
@@ -327,6 +331,31 @@ def cm_transfer_matching(ctx, problems: Sequence[Tuple[Sequence[Tuple[int, int]]
         ctx, n, sizes.ctypes.data_as(C.POINTER(C.c_int32)), ptr(arr[0]), ptr(arr[1]), ptr(arr[2]), ptr(arr[3]),
         total.ctypes.data_as(C.POINTER(C.c_int64)), assign.ctypes.data_as(C.POINTER(C.c_uint16))))
     return total[:n], [[int(x) for x in assign[q, :sizes[q]]] for q in range(n)]
+
+
+def cm_cache_build(ctx, max_failures: int, opts) -> Tuple[C.c_void_p, int]:
+    """Plans for every failure set of at most ``max_failures`` devices -> (cache handle, entries)."""
+    o = _opts(opts)
+    cache, n = C.c_void_p(), C.c_uint64()
+    _check(ctx, load_library().cm_cache_build(ctx, max_failures, C.byref(o), C.byref(cache), C.byref(n)))
+    return cache, n.value
+
+
+def cm_cache_lookup(cache, failed: Sequence[int], per_policy: bool = False):
+    """-> best Plan (and the three per-policy Plans) of a cached failure set, or None if the set
+    is larger than the cache covers."""
+    ids = (C.c_uint32 * max(len(failed), 1))(*failed)
+    best = cm_plan()
+    pol = (cm_plan * 3)() if per_policy else None
+    st = load_library().cm_cache_lookup(cache, ids, len(failed), C.byref(best), pol)
+    if st == CM_ENOFEASIBLE:
+        return (None, None) if per_policy else None
+    _check(None, st)
+    return (_plan_from(best), plans_from_array(pol)) if per_policy else _plan_from(best)
+
+
+def cm_cache_free(cache) -> None:
+    _check(None, load_library().cm_cache_free(cache))
 
 
 def cm_batch_free(batch) -> None:

@@ -618,6 +618,8 @@ void scrub(cm_plan &pl) {
 // Accessors for entry points that live in other translation units.
 cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message) { return fail(ctx, status, message); }
 
+int cm_internal_grid_devices(const cm_ctx *ctx) { return ctx && ctx->has_profile ? ctx->hp.n_dp * ctx->hp.n_pp : 0; }
+
 cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, SpaceView *out) {
     if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
     Batch &bt = const_cast<Batch &>(space->batch);

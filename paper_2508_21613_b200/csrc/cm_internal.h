@@ -241,3 +241,4 @@ struct cm_ctx;
 struct cm_space;
 cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, cm::SpaceView *out);
 cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message);
+int cm_internal_grid_devices(const cm_ctx *ctx);   // n_dp * n_pp of the loaded profile, 0 without one
