@@ -319,6 +319,32 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
         binding.cm_destroy(ctx)
 
 
+def measure_shared(binding, torch, w, mode, local_rank, flush, steps=5):
+    """The same batch with sharing on: failure sets that leave the same survivor count and node
+    boundaries have identical dynamic-parallelism searches and are searched once.  Not the
+    headline: `value` above evaluates every scenario's plans."""
+    opts = w.options.with_cost_mode(mode)
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    packed = binding.PackedScenarios(w.scenarios)
+    try:
+        binding.cm_set_sharing(ctx, True)
+        for _ in range(3):
+            packed.search(ctx, opts)
+        wall = 0.0
+        for k in range(steps):
+            flush.fill_(float(k))
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            packed.search(ctx, opts)
+            wall += time.perf_counter() - t0
+        st = binding.cm_last_stats(ctx)
+        return {"scenarios": packed.B, "e2e_ms_per_step": 1e3 * wall / steps, "device_ms_per_step": 1e-6 * st["device_ns"],
+                "plans_evaluated_per_step": st["plans"], "scenarios_per_s": packed.B / (wall / steps)}
+    finally:
+        binding.cm_destroy(ctx)
+
+
 def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
     """Plan cache: every failure set of at most k devices searched ahead of time; lookups."""
     from paper_2508_21613_b200 import workloads as W
@@ -471,6 +497,8 @@ def main():
             line["full_objective"] = {
                 name: measure_objective(binding, torch, W.ALL_WORKLOADS[name](), args.cost_mode, 3, 3, local_rank, flush)
                 for name in dict.fromkeys((args.workload, "175b-like", "sweep"))}
+        if not args.no_extra and world == 1 and args.scenarios == 0:
+            line["shared_search"] = measure_shared(binding, torch, w, args.cost_mode, local_rank, flush)
         if not args.no_extra and world == 1 and args.scenarios == 0 and w.profile.n_dp * w.profile.n_pp <= 64:
             line["plan_cache"] = measure_cache(binding, w, args.cost_mode, local_rank)
         if args.objective and "full_objective" not in line:

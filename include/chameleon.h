@@ -303,6 +303,15 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist,
                               int64_t *shortlist_bytes, int32_t *shortlist_rounds);
 
+/* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
+ * with node boundaries at the same places among them have identical dynamic-parallelism
+ * searches -- survivors are placed in consecutive blocks and nothing else of the failure set
+ * enters that policy's model.  With sharing on, cm_search_batch / cm_batch_prepare search
+ * such scenarios once and copy the result; rerouting and redundant computation are always
+ * evaluated per scenario.  Results are identical either way; cm_last_stats then counts only
+ * the plans that were actually evaluated.  cm_cache_build always shares. */
+cm_status cm_set_sharing(cm_ctx *ctx, int on);
+
 /* Device time and work of the objective pass of the last cm_search_objective (HOST out[8]):
  * [0] shortlist kernel, ns  [1] completing the shortlisted plans (tie-break kernels), ns
  * [2] matching kernel (and, with sync_rounds, the rounds kernel), ns  [3] objective kernel, ns  [4] matchings solved (only counted when

@@ -7,6 +7,7 @@
 // cm_kernels.cu do the rest from plan indices.
 #include <algorithm>
 #include <chrono>
+#include <map>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -129,6 +130,7 @@ struct cm_ctx {
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_obj[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // phases of the objective pass
     uint64_t obj_stats[8] = {0};
+    bool share = false;               // search scenarios with identical dynamic-parallelism spaces once
     SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
@@ -385,6 +387,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.tmpl.push_back(Tmpl{});   // template 0: no strategies (scenarios without a dynamic-parallelism search)
     const int cross_words = (N + 63) / 64 + 1;
     std::vector<char> dead(N);
+    std::map<std::string, uint32_t> seen;   // sharing: (node-crossing string, survivor count) -> first scenario
     bt.scen.reserve(B);
     bt.cross.reserve((size_t)B * cross_words);
 
@@ -420,7 +423,27 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
             ++n_surv;
         }
         for (int f = f0; f < f1; ++f) dead[failed_ids[f]] = 0;
+        sc.rep = (uint32_t)b;
         if (policy_mask & (1u << CM_DYNPAR)) {
+            // The dynamic-parallelism space of a scenario is a function of how many devices survive
+            // and of where node boundaries fall among them (survivors are placed in consecutive
+            // blocks; which device failed enters nowhere else).  With sharing on, scenarios that
+            // agree in both are searched once and the others point at that result.
+            if (ctx->share) {
+                std::string key((const char *)cw, sizeof(uint64_t) * cross_words);
+                key.append((const char *)&n_surv, sizeof(n_surv));
+                auto it = seen.find(key);
+                if (it != seen.end()) {
+                    const Scen &r = bt.scen[it->second];
+                    sc.rep = it->second;
+                    sc.tmpl = r.tmpl;
+                    sc.cross_first = r.cross_first;
+                    bt.cross.resize(bt.cross.size() - cross_words);
+                    bt.scen.push_back(sc);
+                    continue;
+                }
+                seen.emplace(std::move(key), (uint32_t)b);
+            }
             int t = bt.tmpl_of_nsurv[n_surv];
             if (t < 0) {
                 uint32_t nt = 0;
@@ -442,6 +465,11 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     for (int b = 0; b < B; ++b) {
         Scen &sc = bt.scen[b];
         Tmpl &tp = bt.tmpl[sc.tmpl];
+        if (sc.rep != (uint32_t)b) {   // shares the rows of an earlier scenario; nothing of its own to search
+            sc.seg_base = bt.scen[sc.rep].seg_base;
+            sc.red_first = 0;
+            continue;
+        }
         bt.tmpl_scen[tp.scen_first + tp.n_scen++] = (uint32_t)b;
         sc.seg_base = (uint32_t)rows;
         sc.red_first = (uint32_t)red;
@@ -617,6 +645,12 @@ void scrub(cm_plan &pl) {
 
 // Accessors for entry points that live in other translation units.
 cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message) { return fail(ctx, status, message); }
+
+int cm_internal_set_sharing(cm_ctx *ctx, int on) {
+    const int before = ctx->share ? 1 : 0;
+    ctx->share = on != 0;
+    return before;
+}
 
 int cm_internal_grid_devices(const cm_ctx *ctx) { return ctx && ctx->has_profile ? ctx->hp.n_dp * ctx->hp.n_pp : 0; }
 
@@ -1042,6 +1076,12 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
         if (shortlist_rounds) shortlist_rounds[i] = q.sync_rounds ? bt.short_rounds_host[i * 2] : 0;
     }
     ctx->obj_stats[4] = solved;
+    return CM_OK;
+}
+
+cm_status cm_set_sharing(cm_ctx *ctx, int on) {
+    if (!ctx) return CM_EINVAL;
+    cm_internal_set_sharing(ctx, on);
     return CM_OK;
 }
 

@@ -87,6 +87,9 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
     std::vector<uint32_t> ids;
     std::vector<int32_t> offsets;
     std::vector<cm_plan> best(kBatch), pol((size_t)kBatch * 3);
+    // failure sets that leave the same number of survivors with the same node boundaries have
+    // the same dynamic-parallelism search: let the batches share it
+    const int sharing_before = cm_internal_set_sharing(ctx, 1);
     for (int s = 0; s <= K; ++s) {
         const uint64_t cnt = c->choose(n_devices, s);
         for (uint64_t first = 0; first < cnt; first += kBatch) {
@@ -98,7 +101,7 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
                 offsets[b + 1] = (b + 1) * s;
             }
             cm_status st = cm_search_batch(ctx, ids.data(), offsets.data(), B, opts, best.data(), pol.data(), nullptr);
-            if (st != CM_OK) { delete c; return st; }
+            if (st != CM_OK) { cm_internal_set_sharing(ctx, sharing_before); delete c; return st; }
             for (int b = 0; b < B; ++b) {
                 cm_plan *dst = c->plans.data() + (size_t)(c->offset[s] + first + b) * 4;
                 for (int q = 0; q < 3; ++q) dst[q] = pol[(size_t)b * 3 + q];
@@ -106,6 +109,7 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
             }
         }
     }
+    cm_internal_set_sharing(ctx, sharing_before);
     *out = c;
     if (n_scenarios) *n_scenarios = total;
     return CM_OK;

@@ -76,7 +76,8 @@ struct Scen {              // 32 bytes
     uint32_t tmpl, seg_base;
     uint32_t failed_first, n_failed;   // into the failed-id array
     uint32_t cross_first, red_first;   // into the node-crossing bit words; first reduction block
-    uint32_t policy_mask, pad;
+    uint32_t policy_mask;
+    uint32_t rep;                      // scenario whose dynamic-parallelism search this one shares (itself if none)
 };
 
 // Work layout of the search pass: all segments of a batch that share (stages,
@@ -241,4 +242,5 @@ struct cm_ctx;
 struct cm_space;
 cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, cm::SpaceView *out);
 cm_status cm_internal_fail(cm_ctx *ctx, cm_status status, const std::string &message);
+int cm_internal_set_sharing(cm_ctx *ctx, int on);   // returns the previous setting
 int cm_internal_grid_devices(const cm_ctx *ctx);   // n_dp * n_pp of the loaded profile, 0 without one

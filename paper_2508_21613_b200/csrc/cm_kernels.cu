@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
     const Scen sc = bd.scen[b];
     const Tmpl tp = bd.tmpl[sc.tmpl];
     uint64_t best_c = inf, best_i = ~0ull;
-    for (uint32_t r = threadIdx.x; r < tp.n_red; r += 32) {
+    for (uint32_t r = threadIdx.x; r < (sc.rep == b ? tp.n_red : 0u); r += 32) {
         const Partial q = bd.partial[sc.red_first + r];
         if (pair_less(q.cost_bits, q.item, best_c, best_i)) { best_c = q.cost_bits; best_i = q.item; }
     }
@@ -197,6 +197,7 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
     if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
     if (threadIdx.x == 0) {
         Winner w;
+        if (sc.rep != b) { best_c = inf; best_i = ~0ull; }   // shares another scenario's search: nothing to tie-break here
         decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
     }
@@ -318,7 +319,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
     {
         cm_plan pl;
         plan_clear(pl, CM_DYNPAR);
-        const Winner &w = bd.winner[b];
+        const Winner &w = bd.winner[sc.rep];   // its own search, or the one it shares
         if ((sc.policy_mask & (1u << CM_DYNPAR)) && w.cost_bits < inf) {
             const Strat &s = bd.strat[w.strat];
             pl.feasible = 1;
@@ -329,7 +330,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
             for (uint32_t q = 0; q < w.dp; ++q) {
                 pl.stages[q] = s.S[q];
                 pl.micro[q] = w.micro[q];
-                pl.kappa[q] = bd.kappa_sel[b * kMaxP + q];
+                pl.kappa[q] = bd.kappa_sel[sc.rep * kMaxP + q];
             }
             cost[2] = w.cost_bits;
         }

@@ -92,3 +92,43 @@ def test_full_objective_of_every_scenario_matches_the_stored_oracle_result(gpu, 
                            f"{w.scenarios[wrong[0][0]]}: got {wrong[0][1]} want {want[wrong[0][0]]}")
     finally:
         gpu.cm_destroy(ctx)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("name", ["paper-scale", "175b-like"])
+def test_shared_search_matches_the_stored_oracle_results(gpu, name, mode):
+    """With sharing on, scenarios whose dynamic-parallelism spaces coincide are searched once;
+    every scenario must still come out exactly as the oracle has it, in the plain search and
+    in the full-objective search."""
+    from types import SimpleNamespace
+    w = W.ALL_WORKLOADS[name]()
+    want = _stored(name, mode)
+    want_obj = _stored_objective(name, mode)
+    obj = W.ObjectiveOptions()
+    k = obj.topk
+    ctx = gpu.cm_create(0)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        opts = w.options.with_cost_mode(mode)
+        gpu.cm_search_batch(ctx, w.scenarios, opts)
+        plain_plans = gpu.cm_last_stats(ctx)["plans"]
+        gpu.cm_set_sharing(ctx, True)
+        best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, opts)
+        shared_plans = gpu.cm_last_stats(ctx)["plans"]
+        got = [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)]
+        assert got == want
+        assert shared_plans <= plain_plans
+        if name == "paper-scale":
+            assert shared_plans * 20 < plain_plans        # 2576 failure sets fall into a few dozen classes
+        best, trans, sl, sb, _ = gpu.cm_search_objective(ctx, w.scenarios, opts, obj, shortlist=True)
+        plans = gpu.plans_from_array(best)
+        short = gpu.plans_from_array(sl)
+        for b in range(len(want_obj)):
+            used = [r for r in range(k) if sb[b, r] >= 0]
+            tr = SimpleNamespace(policy=trans[b].policy, rank=trans[b].rank, xfer_bytes=trans[b].xfer_bytes,
+                                 t_trans=trans[b].t_trans, t_trans_ns=trans[b].t_trans_ns, objective=trans[b].objective,
+                                 shortlist=[short[b * k + r] for r in used], shortlist_bytes=[int(sb[b, r]) for r in used])
+            assert goldens.objective_line(plans[b] if trans[b].feasible else None, tr, mode) == want_obj[b], f"scenario {b}"
+        gpu.cm_set_sharing(ctx, False)
+    finally:
+        gpu.cm_destroy(ctx)
