@@ -218,6 +218,23 @@ def test_objective_parity_paper_scale_sampled(gpu, oracle_factory, mode, rounds)
         s.close()
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_objective_parity_minmax_only_and_capped_segments(gpu, oracle_factory, mode):
+    # segments whose only candidate is the min-max partition (layer mode MINMAX, or more
+    # compositions than kappa_cap): the completed plan carries kappa = 0 = that partition
+    w = W.tiny()
+    for lm, cap in ((W.LAYERS_MINMAX, 1 << 62), (W.LAYERS_FULL, 20), (W.LAYERS_REMAINDER, 3)):
+        opts = W.SearchOptions(1, 4, 1, 6, lm, W.BATCH_REMAINDER, cap, mode)
+        o = oracle_factory(w.profile, opts)
+        s = Session(gpu, w.profile)
+        try:
+            for obj in (W.ObjectiveOptions(topk=5), W.ObjectiveOptions(topk=5, sync_rounds=1)):
+                res = gpu.cm_search_objective(s.ctx, w.scenarios, opts, obj, shortlist=True)
+                _check_objective(gpu, o, w, w.scenarios, opts, obj, mode, res)
+        finally:
+            s.close()
+
+
 def test_objective_parity_deep_pipelines_sampled(gpu, oracle_factory):
     w = W.llama70b_like()
     opts = w.options
