@@ -172,7 +172,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * seconds / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "i64" if args.cost_mode else "f64", "data": "synthetic",
+            "dtype": ("f64 (integer-valued, exact)" if m["arith"] == 0 else "i64") if args.cost_mode else "f64",
+            "data": "synthetic",
             "config": {"workload": w.name, "scenarios_per_step": per_step, "cost_mode": args.cost_mode},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -210,6 +211,8 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
         out["dev_seconds"] = sum(a.elapsed_time(b) for a, b in ev) * 1e-3
         out["plans_per_step"] = n_cand + 2 * len(w.scenarios)   # + one rerouting and one redundant plan each
         out["stats"] = stats_sum
+        # the arithmetic the recurrence ran in: the integer mode runs in fp64 whenever that is exact
+        out["arith"] = 0 if (mode == 0 or binding.cm_int64_runs_in_fp64(ctx)) else 1
         binding.cm_batch_free(batch)
 
         # ---- end-to-end arm: host failure sets in, host plans out, every step
@@ -373,8 +376,8 @@ def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
     return out
 
 
-def roofline_of(stats_sum, dev_seconds, mode, sm_max, peak_kind):
-    slots = ISSUE_SLOTS_PER_CELL[mode]
+def roofline_of(stats_sum, dev_seconds, arith, sm_max, peak_kind):
+    slots = ISSUE_SLOTS_PER_CELL[arith]
     peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
     cost_s = stats_sum["cost_kernel_ns"] * 1e-9
     achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
@@ -454,7 +457,8 @@ def main():
             "metric": METRIC, "value": total_plans / max_dev, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * max_dev / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "i64" if args.cost_mode else "f64", "data": "synthetic",
+            "dtype": ("f64 (integer-valued, exact)" if m["arith"] == 0 else "i64") if args.cost_mode else "f64",
+            "data": "synthetic",
             "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": m["plans_per_step"],
                        "policies": 3, "cost_mode": "int64ns" if args.cost_mode else "fp64",
                        "l2": "flushed between timed iterations (256 MB write)",
@@ -465,7 +469,7 @@ def main():
             "latency_us": m["latency_us"],
             "gpu_launches": int(m["stats"]["launches"]),
             "clocks": m["clocks"],
-            "roofline": roofline_of(m["stats"], m["dev_seconds"], args.cost_mode, sm_max, peak_kind),
+            "roofline": roofline_of(m["stats"], m["dev_seconds"], m["arith"], sm_max, peak_kind),
         }
         if not args.no_cpu_baseline:
             p, s, n = oracle_sample(w, args.cost_mode, args.cpu_budget, len(w.scenarios))
@@ -484,7 +488,7 @@ def main():
                 ew = W.ALL_WORKLOADS[name]()
                 em = measure(binding, torch, ew, mode, 2, 3, local_rank, barrier, flush, args.latency_scenarios,
                              sample_clocks=False)
-                r = roofline_of(em["stats"], em["dev_seconds"], mode, sm_max, peak_kind)
+                r = roofline_of(em["stats"], em["dev_seconds"], em["arith"], sm_max, peak_kind)
                 extra[f"{name}/{'int64ns' if mode else 'fp64'}"] = {
                     "scenarios": len(ew.scenarios), "plans_per_step": em["plans_per_step"],
                     "plans_per_s": em["plans_per_step"] * 2 / em["dev_seconds"],

@@ -303,6 +303,20 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist,
                               int64_t *shortlist_bytes, int32_t *shortlist_rounds);
 
+/* Arithmetic of the integer-nanosecond mode.  Its inputs are integers and the model only adds,
+ * takes maxima and floors quotients, so every value is an integer; as long as all of them
+ * stay below 2^53 a double holds them exactly, and 64-bit floating-point adds issue faster
+ * on this GPU than 64-bit integer adds.  cm_load_profile bounds the largest value the loaded
+ * profile can produce (all work of all micro-batches, rerouted and redundant load included,
+ * plus every transfer in sequence plus the longest synchronisation); below 2^52 the integer
+ * mode is evaluated in double arithmetic with floored quotients, bit-identical to the integer
+ * kernels, otherwise in 64-bit integer arithmetic.  cm_set_int64_arithmetic(ctx, 1) forces the
+ * integer kernels for batches and spaces built afterwards, (ctx, 0) restores the default;
+ * cm_int64_runs_in_fp64 returns 1 if the integer mode of the loaded profile currently runs in
+ * double arithmetic. */
+cm_status cm_set_int64_arithmetic(cm_ctx *ctx, int native);
+int cm_int64_runs_in_fp64(const cm_ctx *ctx);
+
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
  * with node boundaries at the same places among them have identical dynamic-parallelism
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set

@@ -112,6 +112,7 @@ struct Batch {
     uint64_t n_rows = 0;                   // rows of seg_best over all scenarios
     uint32_t max_tiles_per_seg = 0, dp_max = 0;
     int B = 0;
+    bool intval = false;                   // integer mode evaluated in double arithmetic (fixed when the batch is built)
 };
 
 struct cm_ctx {
@@ -120,6 +121,15 @@ struct cm_ctx {
     bool has_profile = false;
     DevProfile hp{};                  // host copy: scalars, raw inputs, base cuts
     DevProfile *d_prof = nullptr;
+    // The integer-nanosecond mode normally runs in double arithmetic: its inputs are integers,
+    // the recurrence only adds and takes maxima, so every value is an integer that a double
+    // holds exactly as long as it stays below 2^53 -- and 64-bit floating-point adds issue
+    // faster on this GPU than 64-bit integer adds, which are pairs of 32-bit operations.
+    // d_prof53 is the profile with integer-valued double arrays; exact53 says whether the
+    // loaded profile keeps every intermediate below 2^52 (otherwise, or when the caller asks
+    // for it, the long long kernels run).
+    DevProfile *d_prof53 = nullptr;
+    bool exact53 = false, force_native_i64 = false;
     std::vector<uint64_t> binom;      // [rows][kBinomCols+1]
     int binom_rows = 0;
     uint64_t *d_binom = nullptr;
@@ -378,6 +388,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.scen.clear(); bt.tmpl.clear(); bt.strat.clear(); bt.tseg.clear(); bt.failed.clear(); bt.red_scen.clear();
     bt.keys.clear(); bt.tmpl_scen.clear(); bt.cross.clear();
     bt.opts = o;
+    bt.intval = o.cost == CM_COST_INT64NS && ctx->exact53 && !ctx->force_native_i64;
     bt.policy_mask = policy_mask;
     bt.n_cand = bt.n_tiles = bt.n_split = bt.n_rows = 0;
     bt.max_tiles_per_seg = 0;
@@ -508,7 +519,7 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
     v.counters = reinterpret_cast<unsigned long long *>(bt.d_seg_best.p + bt.n_rows);
-    v.B = bt.B; v.mode = bt.opts.cost;
+    v.B = bt.B; v.mode = bt.opts.cost; v.intval = bt.intval ? 1u : 0u;
     v.n_rows = (uint32_t)bt.n_rows;
     v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
     v.n_red_blocks = (uint32_t)bt.red_scen.size(); v.dp_max = bt.dp_max;
@@ -517,10 +528,17 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     return v;
 }
 
-Tables tables(const cm_ctx *ctx, int mode) {
+Tables tables(const cm_ctx *ctx, const Batch &bt) {
+    Tables t{};
+    t.prof = bt.intval ? ctx->d_prof53 : ctx->d_prof; t.binom = ctx->d_binom; t.binom_rows = ctx->binom_rows;
+    t.mm_cuts = ctx->d_mm[bt.opts.cost]; t.mm_stride_m = ctx->mm_stride_m;
+    return t;
+}
+
+Tables tables_plain(const cm_ctx *ctx) {   // for kernels that only read the byte prefix sums
     Tables t{};
     t.prof = ctx->d_prof; t.binom = ctx->d_binom; t.binom_rows = ctx->binom_rows;
-    t.mm_cuts = ctx->d_mm[mode]; t.mm_stride_m = ctx->mm_stride_m;
+    t.mm_cuts = ctx->d_mm[0]; t.mm_stride_m = ctx->mm_stride_m;
     return t;
 }
 
@@ -550,8 +568,8 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
          bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4 + 1);   // + room for the counters
     if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
     if (bt.keys.size()) {
-        CM_CUDA(ctx, launch_minmax(tables(ctx, bt.opts.cost), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
-                                   (int)bt.keys.size(), bt.opts.cost, ctx->stream));
+        CM_CUDA(ctx, launch_minmax(tables(ctx, bt), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
+                                   (int)bt.keys.size(), bt.intval ? CM_COST_FP64 : bt.opts.cost, ctx->stream));
         if (launches) ++*launches;
     }
     return CM_OK;
@@ -560,7 +578,7 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
 // The launch sequence of the search over an uploaded batch; results land in
 // bt.plans_host ([B][4]) after the stream is synchronised.
 cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
-    const Tables tb = tables(ctx, bt.opts.cost);
+    const Tables tb = tables(ctx, bt);
     const BatchDev bd = dev_view(ctx, bt);
     cudaStream_t st = ctx->stream;
     int launches = launches_so_far, cost_launches = 0;
@@ -657,7 +675,7 @@ int cm_internal_grid_devices(const cm_ctx *ctx) { return ctx && ctx->has_profile
 cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, SpaceView *out) {
     if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
     Batch &bt = const_cast<Batch &>(space->batch);
-    out->tb = tables(ctx, bt.opts.cost);
+    out->tb = tables(ctx, bt);
     out->bd = dev_view(ctx, bt);
     out->n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
     out->stream = ctx->stream;
@@ -706,7 +724,9 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
              cudaEventCreateWithFlags(&c->side.join[i], cudaEventDisableTiming) == cudaSuccess;
         if (ok) c->side.n = i + 1;
     }
-    if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess) {
+    if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess ||
+        cudaMalloc((void **)&c->d_prof53, sizeof(DevProfile)) != cudaSuccess) {
+        if (c->d_prof) cudaFree(c->d_prof);
         cudaGetLastError();
         delete c;
         return CM_ECUDA;
@@ -729,6 +749,7 @@ cm_status cm_destroy(cm_ctx *c) {
     }
     if (c->side.fork) cudaEventDestroy(c->side.fork);
     if (c->d_prof) cudaFree(c->d_prof);
+    if (c->d_prof53) cudaFree(c->d_prof53);
     if (c->d_binom) cudaFree(c->d_binom);
     for (int i = 0; i < 2; ++i)
         if (c->d_mm[i]) cudaFree(c->d_mm[i]);
@@ -777,8 +798,27 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
         h.act[l] = p->act_bytes[l]; h.par[l] = p->param_bytes[l]; h.opt[l] = p->opt_bytes[l]; h.p2p[l] = p->p2p_bytes[l];
     }
     for (int i = 0; i <= p->n_pp; ++i) h.base_cuts[i] = p->base_cuts[i];
+    h.intval = 1;
+    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof53, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
+    CM_CUDA(ctx, launch_prefix(ctx->d_prof53, ctx->stream));
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // the next copy reuses the host image
+    h.intval = 0;
     CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
     CM_CUDA(ctx, launch_prefix(ctx->d_prof, ctx->stream));
+    {
+        // Largest value the integer mode can form: all work of all micro-batches in sequence
+        // (rerouted and redundant load included: at most three times that), every transfer of
+        // every micro-batch in sequence, the longest synchronisation.
+        double work = 0.0, xfer = 0.0, params = 0.0;
+        const double bw_min = (double)std::min(h.bw_intra, h.bw_inter);
+        for (int l = 0; l < h.L; ++l) {
+            work += (double)h.fwd_i[l] + (double)h.bwd_i[l];
+            xfer = std::max(xfer, (double)h.p2p[l] / bw_min);
+            params += (double)h.par[l];
+        }
+        const double bound = 3.0 * h.G * work + 2.0 * h.G * CM_MAX_STAGES * xfer + 2.0 * params / bw_min;
+        ctx->exact53 = bound < 4503599627370496.0;   // 2^52
+    }
 
     // saturating Pascal triangle: rows cover layers, stages, pipelines and micro-batches
     const int rows = std::max(CM_MAX_LAYERS, h.G) + 1;
@@ -835,7 +875,7 @@ cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids
     if (s == CM_OK && policy != CM_DYNPAR) {
         // the one candidate of these policies is evaluated right away so that
         // cm_evaluate can hand its cost out
-        cudaError_t e = launch_policies(tables(ctx, o.cost), dev_view(ctx, sp->batch), ctx->hp.n_dp, ctx->stream);
+        cudaError_t e = launch_policies(tables(ctx, sp->batch), dev_view(ctx, sp->batch), ctx->hp.n_dp, ctx->stream);
         if (e != cudaSuccess) s = fail(ctx, CM_ECUDA, cudaGetErrorString(e));
     }
     if (s != CM_OK) {
@@ -866,7 +906,7 @@ cm_status cm_evaluate(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64
     Batch &bt = const_cast<Batch &>(space->batch);
     const uint64_t n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
     if (!idx_dev && (first > n_cand || count > n_cand - first)) return fail(ctx, CM_EINVAL, "candidate range out of bounds");
-    CM_CUDA(ctx, launch_evaluate(tables(ctx, bt.opts.cost), dev_view(ctx, bt), n_cand,
+    CM_CUDA(ctx, launch_evaluate(tables(ctx, bt), dev_view(ctx, bt), n_cand,
                                  space->policy == CM_DYNPAR ? -1 : space->policy, first, count, idx_dev,
                                  cost_dev, cost_ns_dev, feasible_dev, ctx->stream));
     return CM_OK;
@@ -997,7 +1037,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     ok = bt.obj_best_host.resize(B) && bt.trans_host.resize(B) && bt.short_plans_host.resize(slots) &&
          bt.short_bytes_host.resize(slots) && bt.short_rounds_host.resize(slots * 2);
     if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
-    const Tables tb = tables(ctx, bt.opts.cost);
+    const Tables tb = tables(ctx, bt);
     const BatchDev bd = dev_view(ctx, bt);
     ObjDev od{};
     od.topk = q.topk;
@@ -1079,6 +1119,16 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     return CM_OK;
 }
 
+cm_status cm_set_int64_arithmetic(cm_ctx *ctx, int native) {
+    if (!ctx) return CM_EINVAL;
+    ctx->force_native_i64 = native != 0;
+    return CM_OK;
+}
+
+int cm_int64_runs_in_fp64(const cm_ctx *ctx) {
+    return ctx && ctx->has_profile && ctx->exact53 && !ctx->force_native_i64 ? 1 : 0;
+}
+
 cm_status cm_set_sharing(cm_ctx *ctx, int on) {
     if (!ctx) return CM_EINVAL;
     cm_internal_set_sharing(ctx, on);
@@ -1120,7 +1170,7 @@ cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *s
     for (int a = 0; a < 4 && e == cudaSuccess; ++a)
         e = cudaMemcpyAsync(d + off_rng + a * rows, src[a], rows, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess)
-        e = launch_range_matching(tables(ctx, CM_COST_FP64), n_problems, (const int32_t *)(d + off_sizes), d + off_rng,
+        e = launch_range_matching(tables_plain(ctx), n_problems, (const int32_t *)(d + off_sizes), d + off_rng,
                                   d + off_rng + rows, d + off_rng + 2 * rows, d + off_rng + 3 * rows,
                                   (int64_t *)(d + off_total), (uint16_t *)(d + off_assign), st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(total, d + off_total, (size_t)n_problems * sizeof(int64_t), cudaMemcpyDeviceToHost, st);

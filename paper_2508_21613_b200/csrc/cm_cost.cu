@@ -32,7 +32,7 @@ cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t st
     if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
     for (int S = kRegStagesMax + 1; S <= kWideStagesMax; ++S) {
         if (!((stage_mask >> S) & 1ull)) continue;
-        cudaError_t e = b.mode == CM_COST_INT64NS ? launch_tiebreak_deep<long long>(t, b, S, st)
+        cudaError_t e = native_i64(b) ? launch_tiebreak_deep<long long>(t, b, S, st)
                                                   : launch_tiebreak_deep<double>(t, b, S, st);
         if (e != cudaSuccess) return e;
         if (launches) ++*launches;
@@ -51,7 +51,7 @@ cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchCl
     int first = 0;
     if (n_regs > 1 && regs_chunks > 0 && regs_chunks <= (uint64_t)kAnyMaxChunks) {
         const uint32_t b0 = classes[0].bucket_begin, b1 = classes[n_regs - 1].bucket_end;
-        cudaError_t e = b.mode == CM_COST_INT64NS ? launch_shallow_any<long long>(t, b, b0, b1, regs_chunks, st)
+        cudaError_t e = native_i64(b) ? launch_shallow_any<long long>(t, b, b0, b1, regs_chunks, st)
                                                   : launch_shallow_any<double>(t, b, b0, b1, regs_chunks, st);
         if (e != cudaSuccess) return e;
         if (launches) ++*launches;
@@ -72,7 +72,7 @@ cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchCl
         if (classes[i].n_chunks == 0) continue;
         cudaStream_t s = (n_side && slot % (n_side + 1)) ? side->stream[slot % (n_side + 1) - 1] : st;
         ++slot;
-        err = b.mode == CM_COST_INT64NS ? launch_class<long long>(t, b, classes[i], s) : launch_class<double>(t, b, classes[i], s);
+        err = native_i64(b) ? launch_class<long long>(t, b, classes[i], s) : launch_class<double>(t, b, classes[i], s);
         if (err == cudaSuccess && launches) ++*launches;
     }
     // always join, even after a failed launch, so that the side streams never run ahead unobserved

@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
             if (ok) {
                 const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
                 if (active) {
-                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync));
+                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval));
                     if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
                     my_cells = 2ull * S * m;
                 }

@@ -22,11 +22,15 @@ template <> struct Num<double> {
     static __device__ __forceinline__ const double *PF(const DevProfile *p) { return p->PFd; }
     static __device__ __forceinline__ const double *PB(const DevProfile *p) { return p->PBd; }
     static __device__ __forceinline__ const double *XT(const DevProfile *p, int tier) { return p->XTd[tier]; }
-    static __device__ __forceinline__ double sync(int64_t G, int n, int64_t bw) {
+    // intval: the values are integer nanoseconds held in doubles; quotients floor as in the
+    // integer mode (sums and maxima of such values are exact below 2^53)
+    static __device__ __forceinline__ double sync(int64_t G, int n, int64_t bw, int intval) {
         if (n <= 1) return 0.0;
+        if (intval) return (double)((2LL * (long long)(n - 1) * (long long)G) / ((long long)n * (long long)bw));
         return ((2.0 * (double)(n - 1)) * (double)G) / ((double)n * (double)bw);
     }
-    static __device__ __forceinline__ double reroute_extra(int mF, double fb, int peers) {
+    static __device__ __forceinline__ double reroute_extra(int mF, double fb, int peers, int intval) {
+        if (intval) return (double)(((long long)mF * (long long)fb) / (long long)peers);
         return ((double)mF * fb) / (double)peers;
     }
 };
@@ -38,17 +42,26 @@ template <> struct Num<long long> {
     static __device__ __forceinline__ const long long *PF(const DevProfile *p) { return (const long long *)p->PFi; }
     static __device__ __forceinline__ const long long *PB(const DevProfile *p) { return (const long long *)p->PBi; }
     static __device__ __forceinline__ const long long *XT(const DevProfile *p, int tier) { return (const long long *)p->XTi[tier]; }
-    static __device__ __forceinline__ long long sync(int64_t G, int n, int64_t bw) {
+    static __device__ __forceinline__ long long sync(int64_t G, int n, int64_t bw, int) {
         if (n <= 1) return 0;
         return (2LL * (long long)(n - 1) * (long long)G) / ((long long)n * (long long)bw);
     }
-    static __device__ __forceinline__ long long reroute_extra(int mF, long long fb, int peers) {
+    static __device__ __forceinline__ long long reroute_extra(int mF, long long fb, int peers, int) {
         return ((long long)mF * fb) / (long long)peers;
     }
 };
 
 constexpr uint64_t kInfBitsF64 = 0x7FF0000000000000ull;
 constexpr uint64_t kInfBitsI64 = 0x7FFFFFFFFFFFFFFFull;
+// "infeasible" in the bit patterns a batch carries on the device
+__host__ __device__ __forceinline__ uint64_t batch_inf_bits(const BatchDev &b) {
+    return (b.mode == CM_COST_INT64NS && !b.intval) ? kInfBitsI64 : kInfBitsF64;
+}
+// integer nanoseconds of a cost bit pattern of a batch in integer mode
+__device__ __forceinline__ int64_t batch_cost_ns(const BatchDev &b, uint64_t bits) {
+    if (!b.intval) return (int64_t)bits;
+    return bits >= kInfBitsF64 ? (int64_t)kInfBitsI64 : (int64_t)__longlong_as_double((long long)bits);
+}
 template <typename T> __device__ __forceinline__ uint64_t inf_bits() { return Num<T>::bits(Num<T>::inf()); }
 
 template <typename T> __device__ __forceinline__ T tmax(T a, T b) { return a > b ? a : b; }
@@ -63,6 +76,7 @@ template <typename T> struct SProf {
     T XT[2][kMaxL];
     long long cap, bw_sync;
     int L, n_dp, n_pp, n_micro;
+    int intval, pad;
 };
 
 template <typename T>
@@ -86,6 +100,7 @@ __device__ __forceinline__ void stage_profile(SProf<T> &s, const DevProfile *p) 
         s.n_dp = p->n_dp;
         s.n_pp = p->n_pp;
         s.n_micro = p->n_micro;
+        s.intval = p->intval;
     }
 }
 
@@ -216,7 +231,7 @@ __device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, i
     }
     T t = sim_pipe<T>(S, m, F, B, xt, clock, pend);
     // the sync time is monotone in the gradient bytes, so max over stages = sync of the max
-    cost = t + Num<T>::sync(g_max, n_sync, sp.bw_sync);
+    cost = t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval);
     return true;
 }
 
@@ -349,8 +364,8 @@ __device__ __forceinline__ void plan_clear(cm_plan &pl, int policy) {
     for (int p = 0; p < kMaxP; ++p) { pl.stages[p] = 0; pl.micro[p] = 0; pl.kappa[p] = 0; }
 }
 
-__device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, int mode) {
-    if (mode == CM_COST_INT64NS) pl.cost_ns = (int64_t)bits;
+__device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, const BatchDev &bd) {
+    if (bd.mode == CM_COST_INT64NS) pl.cost_ns = batch_cost_ns(bd, bits);
     else pl.cost = __longlong_as_double((long long)bits);
 }
 

@@ -22,6 +22,7 @@ constexpr uint64_t kSat = ~0ull;        // saturated binomial
 struct DevProfile {
     int32_t L, n_dp, n_pp, n_micro;
     int32_t devices_per_node, G;
+    int32_t intval, pad;   // 1: the double arrays hold the integer-nanosecond values (see cm_load_profile)
     int64_t cap, bw_intra, bw_inter, bw_sync;
     double PFd[kMaxL + 1], PBd[kMaxL + 1];
     int64_t PFi[kMaxL + 1], PBi[kMaxL + 1];
@@ -146,7 +147,10 @@ struct BatchDev {
     cm_plan *plans;         // [B][4]: per policy, then the overall best
     unsigned long long *counters;  // [0] cells simulated in pass 1, [1] plans in pass 2
     int32_t B, mode;
-    uint32_t n_rows, pad0;       // rows of seg_best over all scenarios
+    uint32_t n_rows;             // rows of seg_best over all scenarios
+    // 1: integer-nanosecond mode evaluated in double arithmetic on integer-valued inputs; every
+    // cost on the device is then a double bit pattern and becomes an integer only on the way out
+    uint32_t intval;
     uint64_t n_tiles;
     uint32_t max_tiles_per_seg, n_red_blocks;
     uint32_t dp_max, pad;
@@ -181,6 +185,10 @@ struct ObjDev {
     cm_plan *best;            // [B]
     cm_transition *trans;     // [B]
 };
+
+// Integer-nanosecond mode runs the long long instantiations unless the batch evaluates it in
+// double arithmetic on integer-valued inputs (BatchDev::intval).
+inline bool native_i64(const BatchDev &b) { return b.mode == CM_COST_INT64NS && !b.intval; }
 
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);

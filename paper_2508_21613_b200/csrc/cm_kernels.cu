@@ -22,8 +22,9 @@ namespace cm {
 __global__ void cm_prefix_kernel(DevProfile *p) {
     const int L = p->L;
     switch (threadIdx.x) {
-    case 0: { double a = 0.0; p->PFd[0] = a; for (int l = 0; l < L; ++l) { a = a + p->fwd[l]; p->PFd[l + 1] = a; } break; }
-    case 1: { double a = 0.0; p->PBd[0] = a; for (int l = 0; l < L; ++l) { a = a + p->bwd[l]; p->PBd[l + 1] = a; } break; }
+    // intval: the double arrays carry the integer-nanosecond inputs (sums exact below 2^53)
+    case 0: { double a = 0.0; p->PFd[0] = a; for (int l = 0; l < L; ++l) { a = a + (p->intval ? (double)p->fwd_i[l] : p->fwd[l]); p->PFd[l + 1] = a; } break; }
+    case 1: { double a = 0.0; p->PBd[0] = a; for (int l = 0; l < L; ++l) { a = a + (p->intval ? (double)p->bwd_i[l] : p->bwd[l]); p->PBd[l + 1] = a; } break; }
     case 2: { int64_t a = 0; p->PFi[0] = a; for (int l = 0; l < L; ++l) { a += p->fwd_i[l]; p->PFi[l + 1] = a; } break; }
     case 3: { int64_t a = 0; p->PBi[0] = a; for (int l = 0; l < L; ++l) { a += p->bwd_i[l]; p->PBi[l + 1] = a; } break; }
     case 4: { int64_t a = 0; p->PA[0] = a; for (int l = 0; l < L; ++l) { a += p->act[l]; p->PA[l + 1] = a; } break; }
@@ -33,8 +34,8 @@ __global__ void cm_prefix_kernel(DevProfile *p) {
     default: break;
     }
     for (int l = threadIdx.x; l < L; l += blockDim.x) {
-        p->XTd[0][l] = (double)p->p2p[l] / (double)p->bw_intra;
-        p->XTd[1][l] = (double)p->p2p[l] / (double)p->bw_inter;
+        p->XTd[0][l] = p->intval ? (double)(p->p2p[l] / p->bw_intra) : (double)p->p2p[l] / (double)p->bw_intra;
+        p->XTd[1][l] = p->intval ? (double)(p->p2p[l] / p->bw_inter) : (double)p->p2p[l] / (double)p->bw_inter;
         p->XTi[0][l] = p->p2p[l] / p->bw_intra;
         p->XTi[1][l] = p->p2p[l] / p->bw_inter;
     }
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
 
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     if (b.n_red_blocks) {
         cm_split_kernel<<<b.n_red_blocks, 256, 0, st>>>(t, b, inf);
         cudaError_t e = cudaGetLastError();
@@ -277,7 +278,7 @@ cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t s
     const uint64_t nx = (uint64_t)b.B * b.dp_max;
     if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
     dim3 grid((unsigned)nx, tiebreak_grid_y(nx, b.max_tiles_per_seg), 1);
-    if (b.mode == CM_COST_INT64NS) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
+    if (native_i64(b)) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
     else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b);
     return cudaGetLastError();
 }
@@ -309,7 +310,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
         uint64_t c = (sc.policy_mask & (1u << pol)) ? bd.pol_cost[2 * b + pol] : inf;
         if (c < inf) {
             pl.feasible = 1;
-            plan_set_cost(pl, c, bd.mode);
+            plan_set_cost(pl, c, bd);
             if (pol == CM_REDUNDANT)
                 for (int k = 0; k < p->n_dp && k < kMaxP; ++k) pl.stages[k] = bd.rc_stages[b * kMaxP + k];
             cost[pol] = c;
@@ -323,7 +324,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
         if ((sc.policy_mask & (1u << CM_DYNPAR)) && w.cost_bits < inf) {
             const Strat &s = bd.strat[w.strat];
             pl.feasible = 1;
-            plan_set_cost(pl, w.cost_bits, bd.mode);
+            plan_set_cost(pl, w.cost_bits, bd);
             pl.strategy = w.strat - bd.tmpl[sc.tmpl].strat_first;
             pl.n_pipes = w.dp;
             pl.split_rank = w.item - s.split_first;
@@ -345,7 +346,7 @@ __global__ void cm_finalize_kernel(Tables tb, BatchDev bd, uint64_t inf) {
 
 cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     cm_finalize_kernel<<<(b.B + 127) / 128, 128, 0, st>>>(t, b, inf);
     return cudaGetLastError();
 }
@@ -374,7 +375,7 @@ __global__ void __launch_bounds__(128) cm_evaluate_kernel(Tables tb, BatchDev bd
         if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, e - bd.tseg[s].cand_first, v)) { c = v; ok = true; }
     }
     if (cost && bd.mode == CM_COST_FP64) cost[t] = __longlong_as_double((long long)Num<T>::bits(c));
-    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = (int64_t)Num<T>::bits(c);
+    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = batch_cost_ns(bd, Num<T>::bits(c));
     if (feas) feas[t] = ok ? 1 : 0;
 }
 
@@ -386,7 +387,7 @@ __global__ void cm_evaluate_single_kernel(BatchDev bd, int policy, uint64_t inf,
     const uint64_t e = idx ? idx[t] : first + t;
     uint64_t c = e == 0 ? bd.pol_cost[policy] : inf;
     if (cost && bd.mode == CM_COST_FP64) cost[t] = __longlong_as_double((long long)c);
-    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = (int64_t)c;
+    if (cost_ns && bd.mode == CM_COST_INT64NS) cost_ns[t] = batch_cost_ns(bd, c);
     if (feas) feas[t] = c < inf ? 1 : 0;
 }
 
@@ -395,10 +396,10 @@ cudaError_t launch_evaluate(const Tables &t, const BatchDev &b, uint64_t n_cand,
                             int64_t *cost_ns, uint8_t *feas, cudaStream_t st) {
     if (count == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((count + 127) / 128);
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     if (single_policy >= 0)
         cm_evaluate_single_kernel<<<blocks, 128, 0, st>>>(b, single_policy, inf, first, count, idx, cost, cost_ns, feas);
-    else if (b.mode == CM_COST_INT64NS)
+    else if (native_i64(b))
         cm_evaluate_kernel<long long><<<blocks, 128, 0, st>>>(t, b, first, count, idx, n_cand, cost, cost_ns, feas);
     else
         cm_evaluate_kernel<double><<<blocks, 128, 0, st>>>(t, b, first, count, idx, n_cand, cost, cost_ns, feas);

@@ -95,7 +95,7 @@ cm_evaluate_argmin_kernel(Tables tb, BatchDev bd, uint64_t first, uint64_t count
     if (threadIdx.x == 0) {
         for (int w = 1; w < kNoAllocThreads / 32; ++w)
             if (pair_before(wc[w], wi[w], c, idx)) { c = wc[w]; idx = wi[w]; }
-        if (bd.mode == CM_COST_INT64NS) { if (best_cost_ns) *best_cost_ns = (int64_t)c; }
+        if (bd.mode == CM_COST_INT64NS) { if (best_cost_ns) *best_cost_ns = batch_cost_ns(bd, c); }
         else if (best_cost) *best_cost = __longlong_as_double((long long)c);
         if (best_index) *best_index = c < inf_bits<T>() ? idx : ~0ull;
         *arrived = 0;   // leave the counter clean for the next call
@@ -146,7 +146,7 @@ extern "C" cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *spa
     e = cudaMemsetAsync(scratch + 2 * kNoAllocMaxBlocks, 0, sizeof(unsigned long long), v.stream);
     if (e != cudaSuccess) { cudaGetLastError(); return cm_internal_fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
     const unsigned blocks = (unsigned)((count + kNoAllocThreads - 1) / kNoAllocThreads);
-    if (v.bd.mode == CM_COST_INT64NS)
+    if (native_i64(v.bd))
         cm_evaluate_argmin_kernel<long long><<<blocks, kNoAllocThreads, 0, v.stream>>>(v.tb, v.bd, first, count, scratch, best_cost_dev, best_cost_ns_dev, best_index_dev);
     else
         cm_evaluate_argmin_kernel<double><<<blocks, kNoAllocThreads, 0, v.stream>>>(v.tb, v.bd, first, count, scratch, best_cost_dev, best_cost_ns_dev, best_index_dev);

@@ -244,7 +244,7 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
         lo = hi;
     }
     if (!ok) return false;
-    cost = sim_regs<T, S>(m, st, xts) + Num<T>::sync(g_max, g.n_sync, sp.bw_sync);
+    cost = sim_regs<T, S>(m, st, xts) + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
     return true;
 }
 
@@ -277,7 +277,7 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
     if (!ok) return false;
     const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); },
                                  [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-    cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync);
+    cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
     return true;
 }
 

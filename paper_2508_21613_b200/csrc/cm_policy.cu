@@ -109,8 +109,8 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                     B = sp.PB[hi] - sp.PB[lo];
                     const int tier = (i / dpn == (i + 1) / dpn) ? 0 : 1;   // pipeline 0 sits on devices 0 .. S0-1
                     xt = i < S0 - 1 ? sp.XT[tier][hi - 1] : (T)0;
-                    if (ok && fcnt > 0) extra_i = Num<T>::reroute_extra(m * fcnt, F + B, n_dp - fcnt);
-                    if (ok) sync_i = Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt, sp.bw_sync);
+                    if (ok && fcnt > 0) extra_i = Num<T>::reroute_extra(m * fcnt, F + B, n_dp - fcnt, sp.intval);
+                    if (ok) sync_i = Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt, sp.bw_sync, sp.intval);
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
@@ -142,8 +142,8 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                         Bs[i] = sp.PB[hi] - sp.PB[lo];
                         const int tier = (i / dpn == (i + 1) / dpn) ? 0 : 1;
                         xts[i] = i < S0 - 1 ? sp.XT[tier][hi - 1] : (T)0;
-                        if (fcnt[i] > 0) extra = extra + Num<T>::reroute_extra(m * fcnt[i], Fs[i] + Bs[i], n_dp - fcnt[i]);
-                        t_sync = tmax(t_sync, Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt[i], sp.bw_sync));
+                        if (fcnt[i] > 0) extra = extra + Num<T>::reroute_extra(m * fcnt[i], Fs[i] + Bs[i], n_dp - fcnt[i], sp.intval);
+                        t_sync = tmax(t_sync, Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt[i], sp.bw_sync, sp.intval));
                     }
                     const T base = sim_pipe<T>(S0, m, Fs, Bs, xts, clk, pnd);
                     out = Num<T>::bits((base + extra) + t_sync);
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
             if (ok) {
                 const T t = sim_lockstep<T>(S, m, f, bw, xt);
                 const long long g_max = warp_max<long long>(g);
-                bits = Num<T>::bits(t + Num<T>::sync(g_max, n_dp, sp.bw_sync));
+                bits = Num<T>::bits(t + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
             }
         } else if (ok && lane == 0) {
             int cuts[kMaxS + 1], devs[kMaxS];
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 const long long gb = sp.PP[hi] - sp.PP[lo];
                 g_max = gb > g_max ? gb : g_max;
             }
-            if (fits) bits = Num<T>::bits(sim_pipe<T>(n, m, Fs, Bs, xts, clk, pnd) + Num<T>::sync(g_max, n_dp, sp.bw_sync));
+            if (fits) bits = Num<T>::bits(sim_pipe<T>(n, m, Fs, Bs, xts, clk, pnd) + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
         }
         if (wide) bits = __shfl_sync(0xffffffffu, bits, 0);
         if (lane == 0 && k < kMaxP) { rc_bits[k] = bits; rc_S[k] = (uint16_t)S; }
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
     const int threads = 32 * (1 + (n_dp < kMaxP ? n_dp : kMaxP));
-    if (b.mode == CM_COST_INT64NS) cm_policy_kernel<long long><<<b.B, threads, 0, st>>>(t, b);
+    if (native_i64(b)) cm_policy_kernel<long long><<<b.B, threads, 0, st>>>(t, b);
     else cm_policy_kernel<double><<<b.B, threads, 0, st>>>(t, b);
     return cudaGetLastError();
 }

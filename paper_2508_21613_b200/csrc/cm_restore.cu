@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256) cm_shortlist_kernel(Tables tb, BatchDev b
 
 cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     cm_shortlist_kernel<<<b.B, 256, 0, st>>>(t, b, o, inf);
     return cudaGetLastError();
 }
@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_matching_kernel(Tabl
 
 cudaError_t launch_plan_matching(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     const size_t slots = (size_t)b.B * o.topk;
     cm_plan_matching_kernel<<<(unsigned)((slots + kMatchWarps - 1) / kMatchWarps), kMatchWarps * 32, 0, st>>>(t, b, o, inf);
     return cudaGetLastError();
@@ -432,7 +432,7 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables
     for (int c = 0; c < rounds; ++c) {
         T longest = (T)0;
         for (int l = lane; l < L; l += 32)
-            if (rw.colour[l] == c) longest = tmax(longest, Num<T>::sync(sp.PP[l + 1] - sp.PP[l], dp, sp.bw_sync));
+            if (rw.colour[l] == c) longest = tmax(longest, Num<T>::sync(sp.PP[l + 1] - sp.PP[l], dp, sp.bw_sync, sp.intval));
         for (int o = 16; o > 0; o >>= 1) {
             const uint64_t other = __shfl_xor_sync(0xffffffffu, Num<T>::bits(longest), o);
             longest = tmax(longest, Num<T>::from_bits(other));
@@ -459,7 +459,7 @@ cudaError_t launch_plan_rounds(const Tables &t, const BatchDev &b, const ObjDev 
     if (b.B <= 0) return cudaSuccess;
     const size_t slots = (size_t)b.B * o.topk;
     const unsigned grid = (unsigned)((slots + kMatchWarps - 1) / kMatchWarps);
-    if (b.mode == CM_COST_INT64NS) cm_plan_rounds_kernel<long long><<<grid, kMatchWarps * 32, 0, st>>>(t, b, o);
+    if (native_i64(b)) cm_plan_rounds_kernel<long long><<<grid, kMatchWarps * 32, 0, st>>>(t, b, o);
     else cm_plan_rounds_kernel<double><<<grid, kMatchWarps * 32, 0, st>>>(t, b, o);
     return cudaGetLastError();
 }
@@ -486,7 +486,7 @@ __device__ __forceinline__ void plan_from_winner(const BatchDev &bd, const Winne
     plan_clear(pl, CM_DYNPAR);
     const Strat &s = bd.strat[w.strat];
     pl.feasible = 1;
-    plan_set_cost(pl, step_bits, bd.mode);
+    plan_set_cost(pl, step_bits, bd);
     pl.strategy = w.strat - bd.tmpl[bd.scen[w.scen].tmpl].strat_first;
     pl.n_pipes = w.dp;
     pl.split_rank = w.item - s.split_first;
@@ -528,7 +528,7 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
             if (mode == CM_COST_INT64NS) {
                 tti = od.t_restart_i + bytes / od.bw_xfer;
                 j.ni = od.t_gap_i - tti;
-                j.di = (long long)step;
+                j.di = batch_cost_ns(bd, step);
             } else {
                 tt = od.t_restart + (double)bytes / (double)od.bw_xfer;
                 j.nd = od.t_gap - tt;
@@ -551,7 +551,7 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
             if (od.sync_rounds) {
                 tr.rounds = od.short_rounds[slot * 2];
                 tr.domains = od.short_rounds[slot * 2 + 1];
-                if (mode == CM_COST_INT64NS) tr.t_sync_ns = (long long)od.short_step[slot * 2 + 1];
+                if (mode == CM_COST_INT64NS) tr.t_sync_ns = batch_cost_ns(bd, od.short_step[slot * 2 + 1]);
                 else tr.t_sync = __longlong_as_double((long long)od.short_step[slot * 2 + 1]);
             }
         }
@@ -583,7 +583,7 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
 
 cudaError_t launch_objective(const Tables &t, const BatchDev &b, const ObjDev &o, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
-    const uint64_t inf = b.mode == CM_COST_INT64NS ? kInfBitsI64 : kInfBitsF64;
+    const uint64_t inf = batch_inf_bits(b);
     cm_objective_kernel<<<b.B, 32, 0, st>>>(t, b, o, inf);
     return cudaGetLastError();
 }

@@ -132,3 +132,22 @@ def test_shared_search_matches_the_stored_oracle_results(gpu, name, mode):
         gpu.cm_set_sharing(ctx, False)
     finally:
         gpu.cm_destroy(ctx)
+
+
+@pytest.mark.parametrize("name", ["paper-scale", "175b-like"])
+def test_forced_integer_kernels_match_the_stored_oracle_results(gpu, name):
+    """The integer mode normally runs in double arithmetic (exact for these profiles); the
+    64-bit integer kernels stay covered by forcing them."""
+    w = W.ALL_WORKLOADS[name]()
+    want = _stored(name, 1)
+    ctx = gpu.cm_create(0)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        assert gpu.cm_int64_runs_in_fp64(ctx)
+        gpu.cm_set_int64_arithmetic(ctx, True)
+        assert not gpu.cm_int64_runs_in_fp64(ctx)
+        best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, w.options.with_cost_mode(1))
+        got = [goldens.line_of(p, 1) for p in gpu.plans_from_array(best)]
+        assert got == want
+    finally:
+        gpu.cm_destroy(ctx)

@@ -327,3 +327,61 @@ def test_latency_mode_gives_the_same_plans(gpu):
         assert np.all(lat[:40] > 0)
     finally:
         s.close()
+
+
+# ---- arithmetic of the integer-nanosecond mode ----
+
+def test_integer_mode_runs_in_double_arithmetic_when_exact_and_both_paths_agree(gpu, oracle_factory):
+    """By default the integer mode is evaluated in double arithmetic on the integer-valued
+    inputs; the 64-bit integer kernels can be forced.  Both must reproduce the oracle."""
+    for w in (W.tiny(), W.tiny(mem_bound=True), W.random_small(3, L=9, n_dp=3, n_pp=3, n_micro=6)):
+        opts = w.options.with_cost_mode(1)
+        o = oracle_factory(w.profile, opts)
+        s = Session(gpu, w.profile)
+        try:
+            assert gpu.cm_int64_runs_in_fp64(s.ctx)
+            for native in (False, True):
+                gpu.cm_set_int64_arithmetic(s.ctx, native)
+                assert gpu.cm_int64_runs_in_fp64(s.ctx) == (not native)
+                best, pol, _ = gpu.cm_search_batch(s.ctx, w.scenarios, opts, per_policy=True)
+                plans = gpu.plans_from_array(best)
+                per = gpu.plans_from_array(pol)
+                for b, failed in enumerate(w.scenarios):
+                    want, want_per = o.search(failed)
+                    assert_same_plan(plans[b], want, 1, f"{w.name} {failed} native={native}")
+                    for q in range(3):
+                        assert_same_plan(per[3 * b + q], want_per[q] if want_per[q].feasible else None, 1,
+                                         f"{w.name} {failed} policy {q} native={native}")
+                # per-candidate costs through cm_evaluate as well
+                failed = w.scenarios[1]
+                space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, failed, opts)
+                assert_same_candidates(evaluate_on_gpu(s, space, n, 1), o.evaluate(failed), 1)
+                gpu.cm_space_free(space)
+        finally:
+            s.close()
+
+
+def test_integer_mode_falls_back_to_integer_kernels_when_values_exceed_2_pow_52(gpu, oracle_factory):
+    # layer times near 2^39 ns, 24 layers, 1600 global micro-batches: pipeline times pass 2^52,
+    # where doubles no longer hold every integer
+    L, n_dp, n_pp, n_micro = 24, 2, 3, 800
+    rng = W.SplitMix64(77)
+    fwd = [float(int(rng.uniform(0.5, 1.0) * (1 << 39))) for _ in range(L)]
+    bwd = [float(int(f * rng.uniform(1.5, 2.0))) for f in fwd]
+    prof = W.make_profile_ns(L, n_dp, n_pp, n_micro, fwd, bwd, act=1_000_000, param=50_000_000, opt=300_000_000,
+                             p2p=[int(rng.uniform(1e6, 6e7)) for _ in range(L)], base_cuts=[0, 8, 16, 24],
+                             cap=80_000_000_000, dev_per_node=4, bw_intra=300, bw_inter=20)
+    opts = W.SearchOptions(1, 3, 1, 4, W.LAYERS_REMAINDER, W.BATCH_REMAINDER, 1 << 62, 1)
+    o = oracle_factory(prof, opts)
+    s = Session(gpu, prof)
+    try:
+        assert not gpu.cm_int64_runs_in_fp64(s.ctx)
+        scen = [[0], [4], [1, 5]]
+        best, _, _ = gpu.cm_search_batch(s.ctx, scen, opts)
+        plans = gpu.plans_from_array(best)
+        for b, failed in enumerate(scen):
+            want, _ = o.search(failed)
+            assert want.cost_ns > (1 << 52)
+            assert_same_plan(plans[b], want, 1, f"big values {failed}")
+    finally:
+        s.close()
