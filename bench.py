@@ -180,12 +180,15 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, latency_scenarios, sample_clocks=True):
+def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, latency_scenarios, sample_clocks=True,
+            native_i64=False):
     """One workload on this rank: device-resident arm, end-to-end arm, per-failure latency."""
     import numpy as np
     opts = w.options.with_cost_mode(mode)
     ctx = binding.cm_create(local_rank)
     binding.cm_load_profile(ctx, w.profile)
+    if native_i64:
+        binding.cm_set_int64_arithmetic(ctx, True)
     packed = binding.PackedScenarios(w.scenarios)
     out = {}
     try:
@@ -412,6 +415,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads / cost mode summary")
     ap.add_argument("--scenarios", type=int, default=0, help="use only the first N scenarios (profiling runs)")
+    ap.add_argument("--native-int64", action="store_true",
+                    help="with --cost-mode 1: force the 64-bit integer kernels (default: exact double arithmetic)")
     ap.add_argument("--objective", action="store_true",
                     help="also time the full-objective search on the selected workload (profiling runs)")
     args = ap.parse_args()
@@ -445,7 +450,7 @@ def main():
         w.scenarios = w.scenarios[:args.scenarios]
     flush = torch.empty(256 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")  # > 126 MB L2
     m = measure(binding, torch, w, args.cost_mode, args.steps, args.warmup, local_rank, barrier, flush,
-                args.latency_scenarios)
+                args.latency_scenarios, native_i64=args.native_int64)
     rows = gather_rows([float(m["plans_per_step"] * args.steps), m["dev_seconds"], m["e2e_seconds"]], world, "cuda")
     total_plans, max_dev = aggregate([(r[0], r[1]) for r in rows])
     _, max_e2e = aggregate([(r[0], r[2]) for r in rows])
