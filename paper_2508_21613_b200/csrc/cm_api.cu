@@ -259,10 +259,19 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     }
     for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_GENERIC; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
-        LaunchClass generic{CM_CLASS_GENERIC, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+        LaunchClass generic{CM_CLASS_GENERIC, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
-            LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0};
+            LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
             LaunchClass &c = kind == CM_CLASS_GENERIC ? generic : cls;
+            if (kind == CM_CLASS_WIDE_UNI) {
+                // a warp of the transposed kernel takes several consecutive items once the class
+                // is large enough to fill the GPU anyway
+                uint64_t items = 0;
+                for (const Pre &q : pre)
+                    if (q.kind == kind && q.S == S) items += q.count * ((q.n_seg + 31) / 32);
+                const uint64_t per = items / ((uint64_t)(kChunk / 32) * kUniMinChunks);
+                c.uni_items = S <= kUniBatchStagesMax ? (uint32_t)std::min<uint64_t>(std::max<uint64_t>(per, 1), kUniItemsMax) : 1u;
+            }
             for (const Pre &q : pre) {
                 if (q.kind != kind || q.S != S) continue;
                 Bucket bk{};
@@ -276,7 +285,8 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 bk.m = q.m;
                 if (kind == CM_CLASS_WIDE_UNI) {
                     const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
-                    c.n_chunks += (items + kChunk / 32 - 1) / (kChunk / 32);
+                    const uint64_t per_cta = (uint64_t)(kChunk / 32) * c.uni_items;
+                    c.n_chunks += (items + per_cta - 1) / per_cta;
                 } else {
                     c.n_chunks += (bk.count * bk.n_seg + kChunk - 1) / kChunk;
                 }

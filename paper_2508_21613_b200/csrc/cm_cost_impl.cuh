@@ -158,13 +158,17 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, Bat
 #ifndef CM_WIDE3
 #define CM_WIDE3 34   // deepest pipeline compiled for three resident CTAs per SM (<= 168 registers)
 #endif
+// Transposed kernel: up to this depth a warp takes several items per CTA (see the kernel);
+// deeper pipelines keep one item per warp -- their items are long enough to hide the CTA's
+// fixed cost, and their recurrence leaves no register for anything carried across it.
+#define CM_UNI_BATCH_STAGES kUniBatchStagesMax
 template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
     return UNI ? sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8)
                : sizeof(FB<T>) * S * kChunk + sizeof(T) * S * kChunk;
 }
 
 template <typename T, int S, bool UNI>
-__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
+__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset, int uni_items) {
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -177,62 +181,149 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
     unsigned long long my_cells = 0;
 
     if (UNI) {
-        FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
-        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
-        uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
-        // warp item = (kappa, group of 32 segments), group minor
-        const uint64_t item = (chunk - bk.chunk_first) * (kChunk / 32) + warp;
-        const uint32_t n_groups = (bk.n_seg + 31) / 32;
-        const uint64_t kappa = item / n_groups;
-        const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
-        if (kappa < bk.count && m >= 1) {           // warp-uniform
-            const bool active = seg_local < bk.n_seg;
-            const SegView g = bucket_segment(bd, bk, active ? seg_local : 0);
-            const uint32_t row = g.row;
-            const uint64_t tier = g.tier;
-            const int n_sync = g.n_sync;
-            // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
-            CutWalker cw;
-            bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
-            if (ok) {
-                int lo = 0;
-                for (int i = 0; i < S; ++i) {
-                    const int hi = cw.next();
-                    ok = ok && hi > lo;
-                    if (lane == 0) cuts[i + 1] = (uint8_t)hi;
-                    lo = hi;
+        if (S <= CM_UNI_BATCH_STAGES) {
+            // warp item = (kappa, group of 32 segments), group minor; a warp takes uni_items
+            // consecutive items, so that the CTA's fixed cost (staging the profile) is spread over
+            // more work and a composition shared by consecutive groups is unranked, summed and
+            // checked against memory only once.  Everything an item needs from the previous one
+            // lives in shared memory: nothing but the loop counter stays in registers across the
+            // recurrence, whose per-stage state needs nearly all of them.
+            __shared__ Bucket bks;
+            __shared__ unsigned long long st_kappa[kChunk / 32];
+            __shared__ long long st_gmax[kChunk / 32];
+            __shared__ int st_ok[kChunk / 32];
+            if (tid == 0) bks = bk;
+            if (lane == 0) { st_kappa[warp] = ~0ull; st_ok[warp] = 0; st_gmax[warp] = 0; cells_w[warp] = 0; }
+            __syncthreads();
+            for (int r = 0; r < uni_items; ++r) {
+                FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+                T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+                uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
+                const uint64_t item = ((chunk - bks.chunk_first) * (kChunk / 32) + warp) * (uint64_t)uni_items + r;
+                const uint32_t n_groups = (bks.n_seg + 31) / 32;
+                const uint64_t kappa = item / n_groups;
+                if (kappa >= bks.count || m < 1) break;            // warp-uniform; items ascend
+                const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
+                const bool active = seg_local < bks.n_seg;
+                const SegView g = bucket_segment(bd, bks, active ? seg_local : 0);
+                if (kappa != st_kappa[warp]) {
+                    // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
+                    CutWalker cw;
+                    bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
+                    if (ok) {
+                        int lo = 0;
+                        for (int i = 0; i < S; ++i) {
+                            const int hi = cw.next();
+                            ok = ok && hi > lo;
+                            if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+                            lo = hi;
+                        }
+                        if (lane == 0) cuts[0] = 0;
+                    }
+                    __syncwarp();
+                    long long g_max = 0;
+                    if (ok) {
+                        // stage sums and the memory check, one stage per lane
+                        for (int i = lane; i < S; i += 32) {
+                            const int lo = cuts[i], hi = cuts[i + 1];
+                            ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                            FB<T> d;
+                            d.f = sp.PF[hi] - sp.PF[lo];
+                            d.b = sp.PB[hi] - sp.PB[lo];
+                            fb[i] = d;
+                            const long long gb = sp.PP[hi] - sp.PP[lo];
+                            g_max = gb > g_max ? gb : g_max;
+                        }
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+                            g_max = og > g_max ? og : g_max;
+                        }
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (lane == 0) { st_kappa[warp] = kappa; st_ok[warp] = ok ? 1 : 0; st_gmax[warp] = g_max; }
+                    __syncwarp();
                 }
-                if (lane == 0) cuts[0] = 0;
+                if (st_ok[warp]) {
+                    // transfer times of this lane's segment (its own link tiers)
+                    for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(g.tier >> i) & 1ull][cuts[i + 1] - 1];
+                    const uint32_t row = g.row;
+                    const int n_sync = g.n_sync;
+                    __syncwarp();
+                    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+                    if (active) {
+                        const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], n_sync, sp.bw_sync, sp.intval));
+                        if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
+                    }
+                    const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, active));
+                    if (lane == 0) cells_w[warp] += 2ull * S * m * n_active;
+                    __syncwarp();   // the next item overwrites the stage times and cuts
+                }
             }
-            __syncwarp();
-            long long g_max = 0;
-            if (ok) {
-                // stage sums and the memory check, one stage per lane
-                for (int i = lane; i < S; i += 32) {
-                    const int lo = cuts[i], hi = cuts[i + 1];
-                    ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-                    FB<T> d;
-                    d.f = sp.PF[hi] - sp.PF[lo];
-                    d.b = sp.PB[hi] - sp.PB[lo];
-                    fb[i] = d;
-                    const long long gb = sp.PP[hi] - sp.PP[lo];
-                    g_max = gb > g_max ? gb : g_max;
-                }
-                for (int o = 16; o > 0; o >>= 1) {
-                    const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
-                    g_max = og > g_max ? og : g_max;
-                }
-                // transfer times of this lane's segment (its own link tiers)
-                for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(tier >> i) & 1ull][cuts[i + 1] - 1];
+            __syncthreads();
+            if (tid == 0) {
+                unsigned long long c = 0;
+                for (int w = 0; w < kChunk / 32; ++w) c += cells_w[w];
+                if (c) atomicAdd(&bd.counters[0], c);
             }
-            ok = __all_sync(0xffffffffu, ok);
-            __syncwarp();
-            if (ok) {
-                const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-                if (active) {
-                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval));
-                    if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
-                    my_cells = 2ull * S * m;
+            return;
+        } else {
+            FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+            T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+            uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
+            // warp item = (kappa, group of 32 segments), group minor
+            const uint64_t item = (chunk - bk.chunk_first) * (kChunk / 32) + warp;
+            const uint32_t n_groups = (bk.n_seg + 31) / 32;
+            const uint64_t kappa = item / n_groups;
+            const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
+            if (kappa < bk.count && m >= 1) {           // warp-uniform
+                const bool active = seg_local < bk.n_seg;
+                const SegView g = bucket_segment(bd, bk, active ? seg_local : 0);
+                const uint32_t row = g.row;
+                const uint64_t tier = g.tier;
+                const int n_sync = g.n_sync;
+                // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
+                CutWalker cw;
+                bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
+                if (ok) {
+                    int lo = 0;
+                    for (int i = 0; i < S; ++i) {
+                        const int hi = cw.next();
+                        ok = ok && hi > lo;
+                        if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+                        lo = hi;
+                    }
+                    if (lane == 0) cuts[0] = 0;
+                }
+                __syncwarp();
+                long long g_max = 0;
+                if (ok) {
+                    // stage sums and the memory check, one stage per lane
+                    for (int i = lane; i < S; i += 32) {
+                        const int lo = cuts[i], hi = cuts[i + 1];
+                        ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                        FB<T> d;
+                        d.f = sp.PF[hi] - sp.PF[lo];
+                        d.b = sp.PB[hi] - sp.PB[lo];
+                        fb[i] = d;
+                        const long long gb = sp.PP[hi] - sp.PP[lo];
+                        g_max = gb > g_max ? gb : g_max;
+                    }
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+                        g_max = og > g_max ? og : g_max;
+                    }
+                    // transfer times of this lane's segment (its own link tiers)
+                    for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(tier >> i) & 1ull][cuts[i + 1] - 1];
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                __syncwarp();
+                if (ok) {
+                    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+                    if (active) {
+                        const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval));
+                        if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
+                        my_cells = 2ull * S * m;
+                    }
                 }
             }
         }
@@ -308,7 +399,7 @@ static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const Lau
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin, (int)c.uni_items);
     return cudaGetLastError();
 }
 

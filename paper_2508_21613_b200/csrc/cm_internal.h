@@ -109,7 +109,11 @@ struct LaunchClass {
     uint64_t chunk_begin;  // first chunk of the class in its kind's chunk numbering
     uint32_t bucket_begin, bucket_end;
     uint64_t n_chunks;
+    uint32_t uni_items, pad;   // transposed class: consecutive warp items one warp takes (1..kUniItemsMax)
 };
+constexpr int kUniItemsMax = 8;
+constexpr int kUniBatchStagesMax = 28;     // deeper transposed classes keep one item per warp
+constexpr uint64_t kUniMinChunks = 4096;   // keep at least this many CTAs (about ten waves) in a class before batching items
 
 // (cost, index) pair carried through the hierarchical argmin of the split reduction.
 struct Partial {
