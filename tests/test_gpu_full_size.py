@@ -58,8 +58,8 @@ def _stored_objective(name, mode):
     return [l.strip() for l in open(path) if l.strip() and not l.startswith("#")]
 
 
-@pytest.mark.parametrize("mode", [0, 1])
-@pytest.mark.parametrize("name", ["paper-scale", "70b-like", "175b-like"])
+@pytest.mark.parametrize("name,mode", [("paper-scale", 0), ("paper-scale", 1), ("70b-like", 0), ("70b-like", 1),
+                                       ("175b-like", 0), ("175b-like", 1), ("sweep", 0)])
 def test_full_objective_of_every_scenario_matches_the_stored_oracle_result(gpu, name, mode):
     """cm_search_objective with the default options over the whole workload: chosen policy,
     shortlist rank, matched bytes, transition time, objective, the chosen plan and the whole
