@@ -303,6 +303,16 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist,
                               int64_t *shortlist_bytes, int32_t *shortlist_rounds);
 
+/* The host-side descriptor builder alone, for one failure set and the dynamic-parallelism
+ * policy (Algorithm 1, get_parallel_strategy; Section "Planner", batch and layer
+ * distribution): no CUDA call is made, so it also runs on a machine without a GPU.
+ * HOST out[8]: [0] candidates (pipeline-plans)  [1] strategies  [2] segments
+ * [3] (strategy, split) pairs  [4] surviving devices  [5] launch classes  [6] buckets
+ * [7] node boundaries between neighbouring survivors.  Errors as cm_load_profile /
+ * cm_enumerate (CM_EINVAL, CM_EOVERFLOW). */
+cm_status cm_host_describe(const cm_profile *profile, const uint32_t *failed_ids, int32_t n_failed,
+                           const cm_enum_opts *opts, uint64_t out[8]);
+
 /* Arithmetic of the integer-nanosecond mode.  Its inputs are integers and the model only adds,
  * takes maxima and floors quotients, so every value is an integer; as long as all of them
  * stay below 2^53 a double holds them exactly, and 64-bit floating-point adds issue faster

@@ -30,8 +30,9 @@ EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_eva
            "cm_decode_plan", "cm_space_free", "cm_search_batch", "cm_batch_prepare", "cm_batch_search",
            "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
            "cm_objective_stats", "cm_transfer_matching", "cm_cache_build", "cm_cache_lookup", "cm_cache_free",
-           "cm_set_sharing", "cm_set_int64_arithmetic", "cm_int64_runs_in_fp64", "cm_strerror", "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:22]
+           "cm_set_sharing", "cm_set_int64_arithmetic", "cm_host_describe", "cm_int64_runs_in_fp64", "cm_strerror",
+           "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:23]
 NOALLOC_MAX_CANDIDATES = 524288
 MAX_SHORTLIST, MAX_MATCH = 16, 256
 
@@ -153,6 +154,7 @@ def load_library() -> C.CDLL:
     lib.cm_cache_lookup.argtypes = [vp, C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_plan), C.POINTER(cm_plan)]
     lib.cm_cache_free.argtypes = [vp]
     lib.cm_set_sharing.argtypes = [vp, C.c_int]
+    lib.cm_host_describe.argtypes = [C.POINTER(cm_profile), C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_enum_opts), u64p]
     lib.cm_set_int64_arithmetic.argtypes = [vp, C.c_int]
     lib.cm_int64_runs_in_fp64.argtypes = [vp]
     lib.cm_int64_runs_in_fp64.restype = C.c_int
@@ -199,8 +201,8 @@ def cm_destroy(ctx) -> None:
     _check(None, load_library().cm_destroy(ctx))
 
 
-def cm_load_profile(ctx, profile) -> None:
-    """``profile``: an object with the fields of ``workloads.Profile`` (host numpy arrays)."""
+def _profile_struct(profile):
+    """cm_profile over host arrays; returns (struct, arrays to keep alive)."""
     f64 = lambda a: np.ascontiguousarray(a, dtype=np.float64)
     i64 = lambda a: np.ascontiguousarray(a, dtype=np.int64)
     keep = [f64(profile.fwd_ns), f64(profile.bwd_ns), i64(profile.fwd_ns_i), i64(profile.bwd_ns_i),
@@ -212,7 +214,25 @@ def cm_load_profile(ctx, profile) -> None:
                     ip(keep[2]), ip(keep[3]), ip(keep[4]), ip(keep[5]), ip(keep[6]), ip(keep[7]),
                     keep[8].ctypes.data_as(C.POINTER(C.c_int32)), profile.mem_capacity_bytes,
                     profile.devices_per_node, profile.bw_intra_Bpns, profile.bw_inter_Bpns)
+    return cp, keep
+
+
+def cm_load_profile(ctx, profile) -> None:
+    """``profile``: an object with the fields of ``workloads.Profile`` (host numpy arrays)."""
+    cp, keep = _profile_struct(profile)
     _check(ctx, load_library().cm_load_profile(ctx, C.byref(cp)))
+
+
+def cm_host_describe(profile, failed: Sequence[int], opts) -> dict:
+    """The host-side descriptor builder alone (no GPU needed): counts of the dynamic-parallelism
+    space of one failure set."""
+    cp, keep = _profile_struct(profile)
+    ids = (C.c_uint32 * max(len(failed), 1))(*failed)
+    o = _opts(opts)
+    out = (C.c_uint64 * 8)()
+    _check(None, load_library().cm_host_describe(C.byref(cp), ids, len(failed), C.byref(o), out))
+    keys = ["candidates", "strategies", "segments", "splits", "survivors", "launch_classes", "buckets", "node_crossings"]
+    return dict(zip(keys, [int(v) for v in out]))
 
 
 def cm_enumerate(ctx, policy: int, failed: Sequence[int], opts) -> Tuple[C.c_void_p, int]:

@@ -767,8 +767,9 @@ cm_status cm_destroy(cm_ctx *c) {
     return CM_OK;
 }
 
-cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
-    if (!ctx) return CM_EINVAL;
+// Host half of cm_load_profile: validation, the host copy of the profile, the binomial table,
+// the bound that decides the arithmetic of the integer mode.  No CUDA call.
+static cm_status load_profile_host(cm_ctx *ctx, const cm_profile *p) {
     if (!p) return fail(ctx, CM_EINVAL, "profile is NULL");
     if (p->L < 1 || p->L > CM_MAX_LAYERS) return fail(ctx, CM_EINVAL, "L out of range");
     if (p->n_pp < 1 || p->n_pp > std::min(p->L, CM_MAX_STAGES)) return fail(ctx, CM_EINVAL, "n_pp out of range");
@@ -791,8 +792,6 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     if (p->base_cuts[0] != 0 || p->base_cuts[p->n_pp] != p->L) return fail(ctx, CM_EINVAL, "base_cuts must run from 0 to L");
     for (int i = 0; i < p->n_pp; ++i)
         if (p->base_cuts[i + 1] <= p->base_cuts[i]) return fail(ctx, CM_EINVAL, "base_cuts must be strictly increasing");
-    CM_CUDA(ctx, cudaSetDevice(ctx->device));
-    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // nothing may still read the old profile
 
     DevProfile &h = ctx->hp;
     memset(&h, 0, sizeof(h));
@@ -808,13 +807,6 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
         h.act[l] = p->act_bytes[l]; h.par[l] = p->param_bytes[l]; h.opt[l] = p->opt_bytes[l]; h.p2p[l] = p->p2p_bytes[l];
     }
     for (int i = 0; i <= p->n_pp; ++i) h.base_cuts[i] = p->base_cuts[i];
-    h.intval = 1;
-    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof53, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
-    CM_CUDA(ctx, launch_prefix(ctx->d_prof53, ctx->stream));
-    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // the next copy reuses the host image
-    h.intval = 0;
-    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
-    CM_CUDA(ctx, launch_prefix(ctx->d_prof, ctx->stream));
     {
         // Largest value the integer mode can form: all work of all micro-batches in sequence
         // (rerouted and redundant load included: at most three times that), every transfer of
@@ -829,7 +821,6 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
         const double bound = 3.0 * h.G * work + 2.0 * h.G * CM_MAX_STAGES * xfer + 2.0 * params / bw_min;
         ctx->exact53 = bound < 4503599627370496.0;   // 2^52
     }
-
     // saturating Pascal triangle: rows cover layers, stages, pipelines and micro-batches
     const int rows = std::max(CM_MAX_LAYERS, h.G) + 1;
     ctx->binom.assign((size_t)rows * (kBinomCols + 1), 0);
@@ -842,21 +833,65 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
             ctx->binom[(size_t)n * (kBinomCols + 1) + k] = v;
         }
     ctx->binom_rows = rows;
+    // min-max partition table, one row per (stages, micro-batches), per cost mode
+    ctx->mm_stride_m = h.G + 2;
+    const size_t slots = (size_t)CM_MAX_STAGES * ctx->mm_stride_m;
+    for (int i = 0; i < 2; ++i) ctx->mm_done[i].assign(slots, 0);
+    return CM_OK;
+}
+
+cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
+    if (!ctx) return CM_EINVAL;
+    CM_CUDA(ctx, cudaSetDevice(ctx->device));
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // nothing may still read the old profile
+    ctx->has_profile = false;
+    cm_status s = load_profile_host(ctx, p);
+    if (s != CM_OK) return s;
+    DevProfile &h = ctx->hp;
+    h.intval = 1;
+    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof53, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
+    CM_CUDA(ctx, launch_prefix(ctx->d_prof53, ctx->stream));
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // the next copy reuses the host image
+    h.intval = 0;
+    CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_prof, &h, sizeof(h), cudaMemcpyHostToDevice, ctx->stream));
+    CM_CUDA(ctx, launch_prefix(ctx->d_prof, ctx->stream));
     if (ctx->d_binom) { cudaFree(ctx->d_binom); ctx->d_binom = nullptr; }
     CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_binom, ctx->binom.size() * sizeof(uint64_t)));
     CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_binom, ctx->binom.data(), ctx->binom.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
-
-    // min-max partition table, one row per (stages, micro-batches), per cost mode
-    ctx->mm_stride_m = h.G + 2;
     const size_t slots = (size_t)CM_MAX_STAGES * ctx->mm_stride_m;
     for (int i = 0; i < 2; ++i) {
         if (ctx->d_mm[i]) { cudaFree(ctx->d_mm[i]); ctx->d_mm[i] = nullptr; }
         CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_mm[i], slots * (kMaxS + 1)));
         CM_CUDA(ctx, cudaMemsetAsync(ctx->d_mm[i], 0xFF, slots * (kMaxS + 1), ctx->stream));
-        ctx->mm_done[i].assign(slots, 0);
     }
     CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // ctx->hp / binom may change on the next load
     ctx->has_profile = true;
+    return CM_OK;
+}
+
+// The descriptor builder alone, for one failure set, without a GPU (no CUDA call is made).
+cm_status cm_host_describe(const cm_profile *p, const uint32_t *failed_ids, int32_t n_failed,
+                           const cm_enum_opts *opts, uint64_t out[8]) {
+    if (!p || !opts || !out || n_failed < 0 || (n_failed > 0 && !failed_ids)) return CM_EINVAL;
+    cm_ctx ctx;   // plain host object: nothing here touches the device
+    cm_status s = load_profile_host(&ctx, p);
+    if (s == CM_OK) s = check_opts(&ctx, opts);
+    if (s != CM_OK) return s;
+    Batch bt;
+    const int32_t offsets[2] = {0, n_failed};
+    s = build_batch(&ctx, bt, failed_ids, offsets, 1, *opts, 1u << CM_DYNPAR);
+    if (s != CM_OK) return s;
+    const Tmpl &tp = bt.tmpl[bt.scen[0].tmpl];
+    uint64_t crossings = 0;
+    for (uint64_t w : bt.cross) crossings += (uint64_t)__builtin_popcountll(w);
+    out[0] = bt.n_cand;
+    out[1] = tp.n_strat;
+    out[2] = tp.n_tseg;
+    out[3] = tp.n_split_total;
+    out[4] = (uint64_t)(ctx.hp.n_dp * ctx.hp.n_pp - n_failed);
+    out[5] = bt.classes.size();
+    out[6] = bt.bucket.size();
+    out[7] = crossings;
     return CM_OK;
 }
 

@@ -18,7 +18,7 @@ def lib_path():
 def test_every_declared_entry_point_is_exported(lib_path):
     header = open(os.path.join(ROOT, "include", "chameleon.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(cm_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(cm_[a-z0-9_]+)\s*\(", header))
     assert {"cm_create", "cm_load_profile", "cm_enumerate", "cm_evaluate", "cm_select",
             "cm_search_batch", "cm_decode_plan"} <= declared
     lib = ctypes.CDLL(lib_path)
