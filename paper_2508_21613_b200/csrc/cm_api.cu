@@ -8,6 +8,7 @@
 #include <algorithm>
 #include <chrono>
 #include <map>
+#include <memory>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -141,6 +142,16 @@ struct cm_ctx {
     cudaEvent_t ev_obj[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // phases of the objective pass
     uint64_t obj_stats[8] = {0};
     bool share = false;               // search scenarios with identical dynamic-parallelism spaces once
+    // One-scenario searches (per-failure latency): everything but the failed ids and the
+    // node-crossing bits depends only on the survivor count and the options, so a prepared
+    // batch per (survivor count, options) stays resident and a search patches those few bytes.
+    struct Single {
+        int n_surv = 0;
+        cm_enum_opts opts{};
+        bool intval = false;
+        std::unique_ptr<Batch> batch;
+    };
+    std::vector<Single> single;
     SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
@@ -669,6 +680,65 @@ void scrub(cm_plan &pl) {
         if (pl.kappa[p] == ~0ull) { pl.kappa[p] = 0; pl.feasible = 0; }
 }
 
+// A prepared one-scenario batch for this failure set: found among the context's resident ones
+// (same survivor count, same options, same arithmetic) and patched, or built and uploaded.
+cm_status single_batch(cm_ctx *ctx, const uint32_t *ids, int n, const cm_enum_opts &o, uint32_t mask, Batch **out,
+                       int *launches) {
+    const DevProfile &hp = ctx->hp;
+    const int N = hp.n_dp * hp.n_pp;
+    const int32_t off[2] = {0, n};
+    const bool intval = o.cost == CM_COST_INT64NS && ctx->exact53 && !ctx->force_native_i64;
+    // distinct ids in range (the builder checks the same; here it decides the survivor count)
+    bool ok = n <= N;
+    for (int i = 0; i < n && ok; ++i) {
+        ok = ids[i] < (uint32_t)N;
+        for (int j = 0; j < i && ok; ++j) ok = ids[j] != ids[i];
+    }
+    cm_ctx::Single *hit = nullptr;
+    if (ok)
+        for (cm_ctx::Single &e : ctx->single)
+            if (e.n_surv == N - n && e.intval == intval && memcmp(&e.opts, &o, sizeof(o)) == 0) { hit = &e; break; }
+    if (!hit) {
+        // (also the path of malformed sets: the builder produces the error)
+        std::unique_ptr<Batch> b(new (std::nothrow) Batch());
+        if (!b) return fail(ctx, CM_ENOMEM, "host memory");
+        cm_status s = build_batch(ctx, *b, ids, off, 1, o, mask);
+        if (s == CM_OK) s = upload_batch(ctx, *b, launches);
+        if (s != CM_OK) { cudaStreamSynchronize(ctx->stream); forget_keys(ctx, *b); return s; }
+        if (ctx->single.size() >= 64) {   // bounded: start over rather than grow without limit
+            cudaStreamSynchronize(ctx->stream);
+            ctx->single.clear();
+        }
+        ctx->single.emplace_back();
+        cm_ctx::Single &e = ctx->single.back();
+        e.n_surv = N - n; e.opts = o; e.intval = intval; e.batch = std::move(b);
+        *out = e.batch.get();
+        return CM_OK;
+    }
+    Batch &bt = *hit->batch;
+    // patch what depends on WHICH devices failed: the ids and the node-crossing bits
+    const size_t cross_words = bt.cross.size();
+    std::fill(bt.cross.begin(), bt.cross.end(), 0ull);
+    int n_surv = 0, prev_node = -1, f = 0;
+    uint32_t sorted[CM_MAX_PIPES * CM_MAX_STAGES];
+    for (int i = 0; i < n; ++i) { bt.failed[i] = ids[i]; sorted[i] = ids[i]; }
+    std::sort(sorted, sorted + n);
+    for (int d = 0; d < N; ++d) {
+        if (f < n && sorted[f] == (uint32_t)d) { ++f; continue; }
+        const int node = d / hp.devices_per_node;
+        if (n_surv > 0 && node != prev_node) bt.cross[(n_surv - 1) >> 6] |= 1ull << ((n_surv - 1) & 63);
+        prev_node = node;
+        ++n_surv;
+    }
+    if (n) memcpy(bt.arena.p + bt.off_failed, bt.failed.data(), sizeof(uint32_t) * n);
+    memcpy(bt.arena.p + bt.off_cross, bt.cross.data(), sizeof(uint64_t) * cross_words);
+    if (n) CM_CUDA(ctx, cudaMemcpyAsync(bt.d_arena.p + bt.off_failed, bt.arena.p + bt.off_failed, sizeof(uint32_t) * n, cudaMemcpyHostToDevice, ctx->stream));
+    CM_CUDA(ctx, cudaMemcpyAsync(bt.d_arena.p + bt.off_cross, bt.arena.p + bt.off_cross, sizeof(uint64_t) * cross_words, cudaMemcpyHostToDevice, ctx->stream));
+    ctx->stats[9] += sizeof(uint32_t) * n + sizeof(uint64_t) * cross_words;
+    *out = &bt;
+    return CM_OK;
+}
+
 }  // namespace
 
 // Accessors for entry points that live in other translation units.
@@ -845,6 +915,7 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
     CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // nothing may still read the old profile
     ctx->has_profile = false;
+    ctx->single.clear();                                 // prepared one-scenario batches describe the old profile
     cm_status s = load_profile_host(ctx, p);
     if (s != CM_OK) return s;
     DevProfile &h = ctx->hp;
@@ -1027,14 +1098,20 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
     }
     for (int b = 0; b < B; ++b) {
         const auto t0 = std::chrono::steady_clock::now();
-        const int32_t off[2] = {0, offsets[b + 1] - offsets[b]};
         int launches = 0;
         const uint64_t h0 = now_ns();
-        if ((s = build_batch(ctx, bt, failed_ids + offsets[b], off, 1, *opts, mask)) != CM_OK) { forget_keys(ctx, bt); return s; }
+        Batch *sb = nullptr;
+        if ((s = single_batch(ctx, failed_ids + offsets[b], offsets[b + 1] - offsets[b], *opts, mask, &sb, &launches)) != CM_OK) return s;
         ctx->stats[13] += now_ns() - h0;
-        if ((s = upload_batch(ctx, bt, &launches)) != CM_OK) { forget_keys(ctx, bt); return s; }
-        if ((s = run_batch(ctx, bt, launches)) != CM_OK) return s;
-        copy_out(b, 0);
+        if ((s = run_batch(ctx, *sb, launches)) != CM_OK) return s;
+        for (int pol = 0; pol < 3; ++pol) {
+            cm_plan pl = sb->plans_host[pol];
+            scrub(pl);
+            if (best_per_policy) best_per_policy[(size_t)b * 3 + pol] = pl;
+        }
+        cm_plan pl = sb->plans_host[3];
+        scrub(pl);
+        best_per_scenario[b] = pl;
         const auto t1 = std::chrono::steady_clock::now();
         latency_us[b] = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
     }
