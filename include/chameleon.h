@@ -327,6 +327,16 @@ cm_status cm_host_describe(const cm_profile *profile, const uint32_t *failed_ids
 cm_status cm_set_int64_arithmetic(cm_ctx *ctx, int native);
 int cm_int64_runs_in_fp64(const cm_ctx *ctx);
 
+/* Per-failure searches (cm_search_batch with latency_us): everything but the failed ids and the
+ * node-crossing bits of a one-scenario search depends only on the survivor count and the
+ * options, so the context keeps a prepared batch per (survivor count, options) resident (at most
+ * 64; dropped by cm_load_profile) and a search patches those few bytes.  From its second use on,
+ * such a batch replays its launch sequence as a CUDA graph, captured on a library-owned stream
+ * and launched on the context's stream; cm_last_stats then reports the whole device time but
+ * not the per-phase times ([8], [11], [12] stay 0).  cm_set_latency_graphs(ctx, 0) keeps the
+ * plain launches (default 1).  Results are identical either way. */
+cm_status cm_set_latency_graphs(cm_ctx *ctx, int on);
+
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
  * with node boundaries at the same places among them have identical dynamic-parallelism
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set

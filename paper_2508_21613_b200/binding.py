@@ -30,9 +30,9 @@ EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_eva
            "cm_decode_plan", "cm_space_free", "cm_search_batch", "cm_batch_prepare", "cm_batch_search",
            "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
            "cm_objective_stats", "cm_transfer_matching", "cm_cache_build", "cm_cache_lookup", "cm_cache_free",
-           "cm_set_sharing", "cm_set_int64_arithmetic", "cm_host_describe", "cm_int64_runs_in_fp64", "cm_strerror",
-           "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:23]
+           "cm_set_sharing", "cm_set_int64_arithmetic", "cm_host_describe", "cm_set_latency_graphs",
+           "cm_int64_runs_in_fp64", "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:24]
 NOALLOC_MAX_CANDIDATES = 524288
 MAX_SHORTLIST, MAX_MATCH = 16, 256
 
@@ -154,6 +154,7 @@ def load_library() -> C.CDLL:
     lib.cm_cache_lookup.argtypes = [vp, C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_plan), C.POINTER(cm_plan)]
     lib.cm_cache_free.argtypes = [vp]
     lib.cm_set_sharing.argtypes = [vp, C.c_int]
+    lib.cm_set_latency_graphs.argtypes = [vp, C.c_int]
     lib.cm_host_describe.argtypes = [C.POINTER(cm_profile), C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_enum_opts), u64p]
     lib.cm_set_int64_arithmetic.argtypes = [vp, C.c_int]
     lib.cm_int64_runs_in_fp64.argtypes = [vp]
@@ -381,6 +382,11 @@ def cm_cache_lookup(cache, failed: Sequence[int], per_policy: bool = False):
 def cm_set_sharing(ctx, on: bool) -> None:
     """Search scenarios of a batch with identical dynamic-parallelism spaces once (default off)."""
     _check(ctx, load_library().cm_set_sharing(ctx, int(bool(on))))
+
+
+def cm_set_latency_graphs(ctx, on: bool) -> None:
+    """Replay resident one-scenario searches as CUDA graphs (default on)."""
+    _check(ctx, load_library().cm_set_latency_graphs(ctx, int(bool(on))))
 
 
 def cm_set_int64_arithmetic(ctx, native: bool) -> None:

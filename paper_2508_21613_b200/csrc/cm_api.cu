@@ -145,13 +145,22 @@ struct cm_ctx {
     // One-scenario searches (per-failure latency): everything but the failed ids and the
     // node-crossing bits depends only on the survivor count and the options, so a prepared
     // batch per (survivor count, options) stays resident and a search patches those few bytes.
+    // From its second use on, such a batch replays its launch sequence as a CUDA graph (captured
+    // on a library-owned stream, launched on the caller's): same kernels, same arguments, one
+    // submission instead of a dozen.
     struct Single {
         int n_surv = 0;
         cm_enum_opts opts{};
         bool intval = false;
         std::unique_ptr<Batch> batch;
+        cudaGraphExec_t exec = nullptr;
+        bool graph_failed = false;
+        int launches = 0;
+        ~Single() { if (exec) cudaGraphExecDestroy(exec); }
     };
-    std::vector<Single> single;
+    std::vector<std::unique_ptr<Single>> single;
+    cudaStream_t graph_stream = nullptr;
+    bool use_graphs = true;
     SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
@@ -596,15 +605,13 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     return CM_OK;
 }
 
-// The launch sequence of the search over an uploaded batch; results land in
-// bt.plans_host ([B][4]) after the stream is synchronised.
-cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
+// Enqueue the launch sequence of a search on `st`: clear, the two one-plan policies, search
+// pass, split reduction, tie-break pass, finalize, plans back to the host.  phase_events: record
+// the events between the phases (not while the sequence is being captured into a graph).
+cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_events, int *launches_out, int *cost_launches_out) {
     const Tables tb = tables(ctx, bt);
     const BatchDev bd = dev_view(ctx, bt);
-    cudaStream_t st = ctx->stream;
-    int launches = launches_so_far, cost_launches = 0;
-    const uint64_t h_enqueue = now_ns();
-    CM_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
+    int launches = 0, cost_launches = 0;
     // per-segment minima start at all-ones (above every cost); so do the work counters, which
     // therefore read "value - 1" until cm_finalize_kernel adds the one back
     CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, (bt.n_rows + 4) * sizeof(uint64_t), st));
@@ -613,13 +620,13 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
         ++launches;
     }
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
-        CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
+        if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
         CM_CUDA(ctx, launch_cost_pass1(tb, bd, bt.classes.data(), (int)bt.classes.size(), st, &ctx->side, &cost_launches));
         launches += cost_launches;
-        CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
+        if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
         CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
         launches += bd.n_red_blocks ? 2 : 1;
-        CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
+        if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
         if (bt.n_tiles) {
             CM_CUDA(ctx, launch_cost_pass2(tb, bd, st));
             ++launches;
@@ -627,21 +634,60 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far) {
             for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
             CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &launches));
         }
-        CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
+        if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
     }
     CM_CUDA(ctx, launch_finalize(tb, bd, st));
     ++launches;
-    CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
-    const size_t plan_bytes = (size_t)bt.B * 4 * sizeof(cm_plan), back_bytes = plan_bytes + 4 * sizeof(unsigned long long);
-    if (!bt.plans_host.resize((size_t)bt.B * 4 + 1)) return fail(ctx, CM_ENOMEM, "host memory");
+    if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
+    const size_t back_bytes = (size_t)bt.B * 4 * sizeof(cm_plan) + 4 * sizeof(unsigned long long);
     CM_CUDA(ctx, cudaMemcpyAsync(bt.plans_host.p, bt.d_plans.p, back_bytes, cudaMemcpyDeviceToHost, st));
+    *launches_out = launches;
+    *cost_launches_out = cost_launches;
+    return CM_OK;
+}
+
+// The search over an uploaded batch; results land in bt.plans_host ([B][4]) after the stream is
+// synchronised.  `single`: a resident one-scenario entry whose sequence may replay as a graph.
+cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far, cm_ctx::Single *single = nullptr) {
+    cudaStream_t st = ctx->stream;
+    int launches = 0, cost_launches = 0;
+    const size_t back_bytes = (size_t)bt.B * 4 * sizeof(cm_plan) + 4 * sizeof(unsigned long long);
+    if (!bt.plans_host.resize((size_t)bt.B * 4 + 1)) return fail(ctx, CM_ENOMEM, "host memory");
+    const uint64_t h_enqueue = now_ns();
+    bool replay = false;
+    if (single && ctx->use_graphs && ctx->graph_stream && !single->graph_failed) {
+        if (!single->exec) {
+            // capture the sequence once; any failure leaves the entry on the plain path for good
+            cudaGraph_t graph = nullptr;
+            bool ok = cudaStreamBeginCapture(ctx->graph_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+            if (ok) {
+                const cm_status cs = enqueue_search(ctx, bt, ctx->graph_stream, false, &single->launches, &cost_launches);
+                const cudaError_t ce = cudaStreamEndCapture(ctx->graph_stream, &graph);
+                ok = cs == CM_OK && ce == cudaSuccess && graph;
+            }
+            if (ok) ok = cudaGraphInstantiate(&single->exec, graph, 0) == cudaSuccess;
+            if (graph) cudaGraphDestroy(graph);
+            if (!ok) { cudaGetLastError(); single->exec = nullptr; single->graph_failed = true; ctx->err.clear(); }
+        }
+        replay = single->exec != nullptr;
+    }
+    CM_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
+    if (replay) {
+        CM_CUDA(ctx, cudaGraphLaunch(single->exec, st));
+        CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
+        launches = single->launches;
+    } else {
+        cm_status s = enqueue_search(ctx, bt, st, true, &launches, &cost_launches);
+        if (s != CM_OK) return s;
+    }
+    launches += launches_so_far;
     const uint64_t h_wait = now_ns();
     CM_CUDA(ctx, cudaStreamSynchronize(st));
     ctx->stats[14] += h_wait - h_enqueue;
     ctx->stats[15] += now_ns() - h_wait;
     float ms = 0.f;
     CM_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
-    if (bt.policy_mask & (1u << CM_DYNPAR)) {
+    if (!replay && (bt.policy_mask & (1u << CM_DYNPAR))) {
         float ms_cost = 0.f, ms_tie = 0.f;
         CM_CUDA(ctx, cudaEventElapsedTime(&ms_cost, ctx->ev[2], ctx->ev[3]));
         CM_CUDA(ctx, cudaEventElapsedTime(&ms_tie, ctx->ev[4], ctx->ev[5]));
@@ -682,8 +728,10 @@ void scrub(cm_plan &pl) {
 
 // A prepared one-scenario batch for this failure set: found among the context's resident ones
 // (same survivor count, same options, same arithmetic) and patched, or built and uploaded.
+// *entry: the resident entry that was reused (its launch sequence may replay as a graph), NULL
+// if the batch was just built.
 cm_status single_batch(cm_ctx *ctx, const uint32_t *ids, int n, const cm_enum_opts &o, uint32_t mask, Batch **out,
-                       int *launches) {
+                       int *launches, cm_ctx::Single **entry) {
     const DevProfile &hp = ctx->hp;
     const int N = hp.n_dp * hp.n_pp;
     const int32_t off[2] = {0, n};
@@ -696,8 +744,9 @@ cm_status single_batch(cm_ctx *ctx, const uint32_t *ids, int n, const cm_enum_op
     }
     cm_ctx::Single *hit = nullptr;
     if (ok)
-        for (cm_ctx::Single &e : ctx->single)
-            if (e.n_surv == N - n && e.intval == intval && memcmp(&e.opts, &o, sizeof(o)) == 0) { hit = &e; break; }
+        for (auto &e : ctx->single)
+            if (e->n_surv == N - n && e->intval == intval && memcmp(&e->opts, &o, sizeof(o)) == 0) { hit = e.get(); break; }
+    *entry = hit;
     if (!hit) {
         // (also the path of malformed sets: the builder produces the error)
         std::unique_ptr<Batch> b(new (std::nothrow) Batch());
@@ -709,10 +758,11 @@ cm_status single_batch(cm_ctx *ctx, const uint32_t *ids, int n, const cm_enum_op
             cudaStreamSynchronize(ctx->stream);
             ctx->single.clear();
         }
-        ctx->single.emplace_back();
-        cm_ctx::Single &e = ctx->single.back();
-        e.n_surv = N - n; e.opts = o; e.intval = intval; e.batch = std::move(b);
-        *out = e.batch.get();
+        std::unique_ptr<cm_ctx::Single> e(new (std::nothrow) cm_ctx::Single());
+        if (!e) return fail(ctx, CM_ENOMEM, "host memory");
+        e->n_surv = N - n; e->opts = o; e->intval = intval; e->batch = std::move(b);
+        *out = e->batch.get();
+        ctx->single.push_back(std::move(e));
         return CM_OK;
     }
     Batch &bt = *hit->batch;
@@ -798,6 +848,7 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
     bool ok = true;
     for (int i = 0; i < 6; ++i) ok = ok && cudaEventCreate(&c->ev[i]) == cudaSuccess;
     for (int i = 0; i < 5; ++i) ok = ok && cudaEventCreate(&c->ev_obj[i]) == cudaSuccess;
+    if (cudaStreamCreateWithFlags(&c->graph_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->graph_stream = nullptr; }
     ok = ok && cudaEventCreateWithFlags(&c->side.fork, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 3 && ok; ++i) {
         ok = cudaStreamCreateWithFlags(&c->side.stream[i], cudaStreamNonBlocking) == cudaSuccess &&
@@ -823,6 +874,8 @@ cm_status cm_destroy(cm_ctx *c) {
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     for (int i = 0; i < 5; ++i)
         if (c->ev_obj[i]) cudaEventDestroy(c->ev_obj[i]);
+    c->single.clear();
+    if (c->graph_stream) cudaStreamDestroy(c->graph_stream);
     for (int i = 0; i < 3; ++i) {
         if (c->side.stream[i]) { cudaStreamSynchronize(c->side.stream[i]); cudaStreamDestroy(c->side.stream[i]); }
         if (c->side.join[i]) cudaEventDestroy(c->side.join[i]);
@@ -1101,9 +1154,10 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         int launches = 0;
         const uint64_t h0 = now_ns();
         Batch *sb = nullptr;
-        if ((s = single_batch(ctx, failed_ids + offsets[b], offsets[b + 1] - offsets[b], *opts, mask, &sb, &launches)) != CM_OK) return s;
+        cm_ctx::Single *entry = nullptr;
+        if ((s = single_batch(ctx, failed_ids + offsets[b], offsets[b + 1] - offsets[b], *opts, mask, &sb, &launches, &entry)) != CM_OK) return s;
         ctx->stats[13] += now_ns() - h0;
-        if ((s = run_batch(ctx, *sb, launches)) != CM_OK) return s;
+        if ((s = run_batch(ctx, *sb, launches, entry)) != CM_OK) return s;
         for (int pol = 0; pol < 3; ++pol) {
             cm_plan pl = sb->plans_host[pol];
             scrub(pl);
@@ -1249,6 +1303,12 @@ cm_status cm_set_int64_arithmetic(cm_ctx *ctx, int native) {
 
 int cm_int64_runs_in_fp64(const cm_ctx *ctx) {
     return ctx && ctx->has_profile && ctx->exact53 && !ctx->force_native_i64 ? 1 : 0;
+}
+
+cm_status cm_set_latency_graphs(cm_ctx *ctx, int on) {
+    if (!ctx) return CM_EINVAL;
+    ctx->use_graphs = on != 0;
+    return CM_OK;
 }
 
 cm_status cm_set_sharing(cm_ctx *ctx, int on) {

@@ -385,3 +385,43 @@ def test_integer_mode_falls_back_to_integer_kernels_when_values_exceed_2_pow_52(
             assert_same_plan(plans[b], want, 1, f"big values {failed}")
     finally:
         s.close()
+
+
+@pytest.mark.parametrize("graphs", [True, False])
+def test_per_failure_searches_reuse_resident_batches_and_match_the_batched_search(gpu, oracle_factory, graphs):
+    """Latency mode keeps one prepared batch per survivor count and, with graphs on, replays its
+    launch sequence; interleaved survivor counts, repeated sets, both cost modes and a profile
+    reload in between must all give what the batched search and the oracle give."""
+    w = W.paper_scale(6, 6)
+    scen = [w.scenarios[i] for i in (0, 5, 31, 40, 41, 300, 527, 528, 529, 533, 534, 539, 5, 300)]
+    scen += [[], [7, 3], [3, 7]]                                 # nothing failed; ids in either order
+    s = Session(gpu, w.profile)
+    try:
+        gpu.cm_set_latency_graphs(s.ctx, graphs)
+        for mode in (0, 1, 0):
+            opts = w.options.with_cost_mode(mode)
+            batched, _, _ = gpu.cm_search_batch(s.ctx, scen, opts)
+            single, pol, lat = gpu.cm_search_batch(s.ctx, scen, opts, per_policy=True, latency=True)
+            a, b = gpu.plans_from_array(batched), gpu.plans_from_array(single)
+            for i in range(len(scen)):
+                assert a[i].key() == b[i].key() and a[i].cost == b[i].cost and a[i].cost_ns == b[i].cost_ns, (mode, scen[i])
+            assert np.all(lat[:len(scen)] > 0)
+        o = oracle_factory(w.profile, w.options)
+        for i in (3, 9, 16):
+            want, _ = o.search(scen[i])
+            assert_same_plan(b[i], want, 0, f"latency mode {scen[i]}")
+        # another profile on the same context: resident batches of the old one must not survive
+        t = W.tiny()
+        gpu.cm_load_profile(s.ctx, t.profile)
+        ot = oracle_factory(t.profile, t.options)
+        for rep in range(2):
+            got, _, _ = gpu.cm_search_batch(s.ctx, t.scenarios, t.options, latency=True)
+            for i, failed in enumerate(t.scenarios):
+                want, _ = ot.search(failed)
+                assert_same_plan(gpu.plans_from_array(got)[i], want, 0, f"after reload {failed}")
+        with pytest.raises(gpu.ChameleonError):
+            gpu.cm_search_batch(s.ctx, [[1, 1]], t.options, latency=True)
+        with pytest.raises(gpu.ChameleonError):
+            gpu.cm_search_batch(s.ctx, [[99]], t.options, latency=True)
+    finally:
+        s.close()
