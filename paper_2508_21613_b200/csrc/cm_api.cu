@@ -161,6 +161,9 @@ struct cm_ctx {
     std::vector<std::unique_ptr<Single>> single;
     cudaStream_t graph_stream = nullptr;
     bool use_graphs = true;
+    // the two one-plan policies do not depend on the dynamic-parallelism search: they run beside it
+    cudaStream_t pol_stream = nullptr;
+    cudaEvent_t pol_fork = nullptr, pol_join = nullptr;
     SideStreams side{};               // library-owned streams for independent launch classes
     uint64_t stats[16] = {0};
     std::string err;
@@ -615,8 +618,15 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
     // per-segment minima start at all-ones (above every cost); so do the work counters, which
     // therefore read "value - 1" until cm_finalize_kernel adds the one back
     CM_CUDA(ctx, cudaMemsetAsync(bt.d_seg_best.p, 0xFF, (bt.n_rows + 4) * sizeof(uint64_t), st));
-    if (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) {
-        CM_CUDA(ctx, launch_policies(tb, bd, ctx->hp.n_dp, st));
+    const bool policies = (bt.policy_mask & ((1u << CM_REROUTE) | (1u << CM_REDUNDANT))) != 0;
+    const bool beside = policies && (bt.policy_mask & (1u << CM_DYNPAR)) && ctx->pol_stream;
+    if (policies) {
+        if (beside) {
+            CM_CUDA(ctx, cudaEventRecord(ctx->pol_fork, st));
+            CM_CUDA(ctx, cudaStreamWaitEvent(ctx->pol_stream, ctx->pol_fork, 0));
+        }
+        CM_CUDA(ctx, launch_policies(tb, bd, ctx->hp.n_dp, beside ? ctx->pol_stream : st));
+        if (beside) CM_CUDA(ctx, cudaEventRecord(ctx->pol_join, ctx->pol_stream));
         ++launches;
     }
     if (bt.policy_mask & (1u << CM_DYNPAR)) {
@@ -636,6 +646,7 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
         }
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
     }
+    if (beside) CM_CUDA(ctx, cudaStreamWaitEvent(st, ctx->pol_join, 0));
     CM_CUDA(ctx, launch_finalize(tb, bd, st));
     ++launches;
     if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
@@ -849,6 +860,13 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
     for (int i = 0; i < 6; ++i) ok = ok && cudaEventCreate(&c->ev[i]) == cudaSuccess;
     for (int i = 0; i < 5; ++i) ok = ok && cudaEventCreate(&c->ev_obj[i]) == cudaSuccess;
     if (cudaStreamCreateWithFlags(&c->graph_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->graph_stream = nullptr; }
+    if (cudaStreamCreateWithFlags(&c->pol_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->pol_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->pol_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        if (c->pol_stream) cudaStreamDestroy(c->pol_stream);
+        c->pol_stream = nullptr;
+    }
     ok = ok && cudaEventCreateWithFlags(&c->side.fork, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 3 && ok; ++i) {
         ok = cudaStreamCreateWithFlags(&c->side.stream[i], cudaStreamNonBlocking) == cudaSuccess &&
@@ -876,6 +894,9 @@ cm_status cm_destroy(cm_ctx *c) {
         if (c->ev_obj[i]) cudaEventDestroy(c->ev_obj[i]);
     c->single.clear();
     if (c->graph_stream) cudaStreamDestroy(c->graph_stream);
+    if (c->pol_stream) { cudaStreamSynchronize(c->pol_stream); cudaStreamDestroy(c->pol_stream); }
+    if (c->pol_fork) cudaEventDestroy(c->pol_fork);
+    if (c->pol_join) cudaEventDestroy(c->pol_join);
     for (int i = 0; i < 3; ++i) {
         if (c->side.stream[i]) { cudaStreamSynchronize(c->side.stream[i]); cudaStreamDestroy(c->side.stream[i]); }
         if (c->side.join[i]) cudaEventDestroy(c->side.join[i]);
