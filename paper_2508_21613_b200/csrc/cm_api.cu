@@ -556,6 +556,8 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.n_rows = (uint32_t)bt.n_rows;
     v.n_tiles = bt.n_tiles; v.max_tiles_per_seg = bt.max_tiles_per_seg;
     v.n_red_blocks = (uint32_t)bt.red_scen.size(); v.dp_max = bt.dp_max;
+    v.max_red_per_scen = 0;
+    for (const Tmpl &tp : bt.tmpl) v.max_red_per_scen = std::max(v.max_red_per_scen, tp.n_scen ? tp.n_red : 0u);
     v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
     (void)ctx;
     return v;
@@ -635,7 +637,7 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
         launches += cost_launches;
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
         CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
-        launches += bd.n_red_blocks ? 2 : 1;
+        launches += (bd.n_red_blocks && bd.max_red_per_scen > 1) ? 2 : 1;
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
         if (bt.n_tiles) {
             CM_CUDA(ctx, launch_cost_pass2(tb, bd, st));

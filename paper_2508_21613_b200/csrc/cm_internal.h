@@ -157,7 +157,8 @@ struct BatchDev {
     uint32_t intval;
     uint64_t n_tiles;
     uint32_t max_tiles_per_seg, n_red_blocks;
-    uint32_t dp_max, pad;
+    uint32_t dp_max;
+    uint32_t max_red_per_scen;   // most blocks of the split reduction any scenario has
     int32_t layer_mode, batch_mode;
 };
 

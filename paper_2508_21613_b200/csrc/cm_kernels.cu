@@ -204,9 +204,44 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
     }
 }
 
+// Both levels in one launch, for batches in which no scenario needs more than one block of the
+// split reduction (up to 1024 (strategy, split) pairs each): one CTA per scenario.
+__global__ void __launch_bounds__(256) cm_split_winner_kernel(Tables tb, BatchDev bd, uint64_t inf) {
+    __shared__ uint64_t rc[8], ri[8];
+    const uint32_t b = blockIdx.x;
+    const Scen sc = bd.scen[b];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
+    const uint64_t *best = bd.seg_best + sc.seg_base;
+    uint64_t best_c = inf, best_i = ~0ull;
+    if (sc.rep == b)
+        for (uint64_t item = threadIdx.x; item < tp.n_split_total; item += blockDim.x) {
+            const uint64_t T = item_step_time(tb, bd, tp, best, item, inf);
+            if (pair_less(T, item, best_c, best_i)) { best_c = T; best_i = item; }
+        }
+    for (int o = 16; o > 0; o >>= 1) {
+        uint64_t oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+        uint64_t oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { rc[threadIdx.x >> 5] = best_c; ri[threadIdx.x >> 5] = best_i; }
+    if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w)
+            if (pair_less(rc[w], ri[w], best_c, best_i)) { best_c = rc[w]; best_i = ri[w]; }
+        Winner w;
+        decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
+        bd.winner[b] = w;
+    }
+}
+
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st) {
     if (b.B <= 0) return cudaSuccess;
     const uint64_t inf = batch_inf_bits(b);
+    if (b.n_red_blocks <= (uint32_t)b.B && b.max_red_per_scen <= 1) {
+        cm_split_winner_kernel<<<b.B, 256, 0, st>>>(t, b, inf);
+        return cudaGetLastError();
+    }
     if (b.n_red_blocks) {
         cm_split_kernel<<<b.n_red_blocks, 256, 0, st>>>(t, b, inf);
         cudaError_t e = cudaGetLastError();
