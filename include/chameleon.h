@@ -334,7 +334,10 @@ int cm_int64_runs_in_fp64(const cm_ctx *ctx);
  * such a batch replays its launch sequence as a CUDA graph, captured on a library-owned stream
  * and launched on the context's stream; cm_last_stats then reports the whole device time but
  * not the per-phase times ([8], [11], [12] stay 0).  cm_set_latency_graphs(ctx, 0) keeps the
- * plain launches (default 1).  Results are identical either way. */
+ * plain launches (default 1).  Results are identical either way.  The first search for a
+ * survivor count builds its batch and the second captures its graph (1 to 2 ms each on the
+ * 32-device workload); a caller that wants the short path at failure time searches any failure
+ * set of each expected size twice beforehand. */
 cm_status cm_set_latency_graphs(cm_ctx *ctx, int on);
 
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
