@@ -351,6 +351,33 @@ def measure_shared(binding, torch, w, mode, local_rank, flush, steps=5):
         binding.cm_destroy(ctx)
 
 
+def measure_trace(binding, w, mode, local_rank, seed=7, hours=9.0, rate=0.10):
+    """The paper's simulated experiment in the library's model: devices fail at 10 % per hour for
+    9 hours; reroute-first, always-reconfigure and the full objective are replayed over the same
+    seeded trace (states the search windows cannot plan produce nothing)."""
+    from paper_2508_21613_b200 import trace as T, workloads as W
+    opts = w.options.with_cost_mode(mode)
+    n = w.profile.n_dp * w.profile.n_pp
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    try:
+        events = T.make_trace(n, rate, hours, seed)
+        objective = W.ObjectiveOptions(t_gap_ns=3600e9 / (rate * n))
+        base, _, _ = binding.cm_search_batch(ctx, [[]], opts, per_policy=True)
+        fault_free = float(base[0].cost_ns if mode else base[0].cost)     # nothing failed: rerouting = the base configuration
+        t0 = time.perf_counter()
+        r = T.replay(T.gpu_planner(binding, ctx, opts, objective), events, hours, fault_free)
+        dt = time.perf_counter() - t0
+        return {"devices": n, "failure_rate_per_device_hour": rate, "hours": hours, "seed": seed, "failures": r["events"],
+                "relative_work": {k: v["relative_work"] for k, v in r["rules"].items()},
+                "full_objective_vs_always_dynpar": r["full_objective_vs_always_dynpar"],
+                "full_objective_vs_reroute_first": r["full_objective_vs_reroute_first"],
+                "choices_of_full_objective": [t[2] for t in r["rules"]["full-objective"]["timeline"]],
+                "planning_ms_all_states": 1e3 * dt}
+    finally:
+        binding.cm_destroy(ctx)
+
+
 def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
     """Plan cache: every failure set of at most k devices searched ahead of time; lookups."""
     from paper_2508_21613_b200 import workloads as W
@@ -510,6 +537,7 @@ def main():
             line["shared_search"] = measure_shared(binding, torch, w, args.cost_mode, local_rank, flush)
         if not args.no_extra and world == 1 and args.scenarios == 0 and w.profile.n_dp * w.profile.n_pp <= 64:
             line["plan_cache"] = measure_cache(binding, w, args.cost_mode, local_rank)
+            line["failure_trace"] = measure_trace(binding, w, args.cost_mode, local_rank)
         if args.objective and "full_objective" not in line:
             line["full_objective"] = {w.name: measure_objective(binding, torch, w, args.cost_mode, args.steps,
                                                                 args.warmup, local_rank, flush)}
