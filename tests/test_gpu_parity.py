@@ -425,3 +425,29 @@ def test_per_failure_searches_reuse_resident_batches_and_match_the_batched_searc
             gpu.cm_search_batch(s.ctx, [[99]], t.options, latency=True)
     finally:
         s.close()
+
+
+def test_searches_on_a_caller_owned_stream(gpu, oracle_factory):
+    """cm_create takes the caller's CUDA stream: batched, per-failure (resident batch + graph
+    replay) and full-objective searches enqueue there and give the usual results."""
+    import torch
+    w = W.paper_scale(4, 4)
+    o = oracle_factory(w.profile, w.options)
+    stream = torch.cuda.Stream()
+    ctx = gpu.cm_create(0, stream.cuda_stream)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        scen = [w.scenarios[i] for i in (1, 2, 3, 40, 41, 42, 530, 531)]
+        a, _, _ = gpu.cm_search_batch(ctx, scen, w.options)
+        for rep in range(3):
+            b, _, _ = gpu.cm_search_batch(ctx, scen, w.options, latency=True)
+            assert [p.key() for p in gpu.plans_from_array(a)] == [p.key() for p in gpu.plans_from_array(b)]
+        best, trans, _, _, _ = gpu.cm_search_objective(ctx, scen, w.options, W.ObjectiveOptions(topk=3, sync_rounds=1))
+        for i in (0, 5):
+            want, _ = o.search(scen[i])
+            assert_same_plan(gpu.plans_from_array(a)[i], want, 0, f"stream {scen[i]}")
+            wo, wt = o.search_objective(scen[i], W.ObjectiveOptions(topk=3, sync_rounds=1))
+            assert gpu.plans_from_array(best)[i].key() == wo.key() and trans[i].objective == wt.objective
+        stream.synchronize()
+    finally:
+        gpu.cm_destroy(ctx)
