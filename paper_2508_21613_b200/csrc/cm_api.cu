@@ -644,7 +644,7 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
             ++launches;
             uint64_t stage_mask = 0;
             for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
-            CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &launches));
+            CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &ctx->side, &launches));
         }
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
     }
@@ -1263,7 +1263,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
         ++obj_launches;
         uint64_t stage_mask = 0;
         for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
-        CM_CUDA(ctx, launch_tiebreak_wide(tb, sd, stage_mask, st, &obj_launches));
+        CM_CUDA(ctx, launch_tiebreak_wide(tb, sd, stage_mask, st, &ctx->side, &obj_launches));
     }
     CM_CUDA(ctx, cudaEventRecord(ctx->ev_obj[2], st));
     CM_CUDA(ctx, launch_plan_matching(tb, bd, od, st));

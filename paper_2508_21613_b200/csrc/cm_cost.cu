@@ -28,16 +28,33 @@ static cudaError_t launch_class(const Tables &t, const BatchDev &b, const Launch
 }
 
 // stage_mask: bit S set = some template segment of the batch has S stages (17 <= S <= 48)
-cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st, int *launches) {
+cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st,
+                                 const SideStreams *side, int *launches) {
     if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
-    for (int S = kRegStagesMax + 1; S <= kWideStagesMax; ++S) {
-        if (!((stage_mask >> S) & 1ull)) continue;
-        cudaError_t e = native_i64(b) ? launch_tiebreak_deep<long long>(t, b, S, st)
-                                                  : launch_tiebreak_deep<double>(t, b, S, st);
+    int n_launch = 0;
+    for (int S = kRegStagesMax + 1; S <= kWideStagesMax; ++S) n_launch += (int)((stage_mask >> S) & 1ull);
+    // one kernel per depth, each over its own pipelines' slots: side by side like the search pass
+    const int n_side = (side && n_launch > 1) ? side->n : 0;
+    if (n_side) {
+        cudaError_t e = cudaEventRecord(side->fork, st);
+        for (int k = 0; k < n_side && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(side->stream[k], side->fork, 0);
         if (e != cudaSuccess) return e;
-        if (launches) ++*launches;
     }
-    return cudaSuccess;
+    cudaError_t err = cudaSuccess;
+    int slot = 0;
+    for (int S = kRegStagesMax + 1; S <= kWideStagesMax && err == cudaSuccess; ++S) {
+        if (!((stage_mask >> S) & 1ull)) continue;
+        cudaStream_t s = (n_side && slot % (n_side + 1)) ? side->stream[slot % (n_side + 1) - 1] : st;
+        ++slot;
+        err = native_i64(b) ? launch_tiebreak_deep<long long>(t, b, S, s) : launch_tiebreak_deep<double>(t, b, S, s);
+        if (err == cudaSuccess && launches) ++*launches;
+    }
+    for (int k = 0; k < n_side; ++k) {
+        cudaError_t e = cudaEventRecord(side->join[k], side->stream[k]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join[k], 0);
+        if (err == cudaSuccess) err = e;
+    }
+    return err;
 }
 
 // A 2-D grid may overshoot the class's chunk count; surplus CTAs find the last bucket,

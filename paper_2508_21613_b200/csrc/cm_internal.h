@@ -222,7 +222,8 @@ cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchCl
                               cudaStream_t st, const SideStreams *side, int *launches);
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);
 cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st);
-cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st, int *launches);
+cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st,
+                                 const SideStreams *side, int *launches);
 cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st);
 // single_policy < 0: candidates of the dynamic-parallelism segments; otherwise the one
 // candidate of that policy (its cost must already be in pol_cost of scenario 0)
