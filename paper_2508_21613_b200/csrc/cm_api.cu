@@ -870,7 +870,7 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
         c->pol_stream = nullptr;
     }
     ok = ok && cudaEventCreateWithFlags(&c->side.fork, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < 3 && ok; ++i) {
+    for (int i = 0; i < kSideStreams && ok; ++i) {
         ok = cudaStreamCreateWithFlags(&c->side.stream[i], cudaStreamNonBlocking) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->side.join[i], cudaEventDisableTiming) == cudaSuccess;
         if (ok) c->side.n = i + 1;
@@ -899,7 +899,7 @@ cm_status cm_destroy(cm_ctx *c) {
     if (c->pol_stream) { cudaStreamSynchronize(c->pol_stream); cudaStreamDestroy(c->pol_stream); }
     if (c->pol_fork) cudaEventDestroy(c->pol_fork);
     if (c->pol_join) cudaEventDestroy(c->pol_join);
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < kSideStreams; ++i) {
         if (c->side.stream[i]) { cudaStreamSynchronize(c->side.stream[i]); cudaStreamDestroy(c->side.stream[i]); }
         if (c->side.join[i]) cudaEventDestroy(c->side.join[i]);
     }

@@ -34,7 +34,7 @@ cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t st
     int n_launch = 0;
     for (int S = kRegStagesMax + 1; S <= kWideStagesMax; ++S) n_launch += (int)((stage_mask >> S) & 1ull);
     // one kernel per depth, each over its own pipelines' slots: side by side like the search pass
-    const int n_side = (side && n_launch > 1) ? side->n : 0;
+    const int n_side = (side && n_launch > 1) ? (side->n < n_launch - 1 ? side->n : n_launch - 1) : 0;
     if (n_side) {
         cudaError_t e = cudaEventRecord(side->fork, st);
         for (int k = 0; k < n_side && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(side->stream[k], side->fork, 0);
@@ -77,7 +77,7 @@ cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchCl
     int n_launch = 0;
     for (int i = first; i < n_classes; ++i) n_launch += classes[i].n_chunks ? 1 : 0;
     // classes only share the per-segment minima they atomically lower: run them side by side
-    const int n_side = (side && n_launch > 1) ? side->n : 0;
+    const int n_side = (side && n_launch > 1) ? (side->n < n_launch - 1 ? side->n : n_launch - 1) : 0;
     if (n_side) {
         cudaError_t e = cudaEventRecord(side->fork, st);
         for (int k = 0; k < n_side && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(side->stream[k], side->fork, 0);

@@ -213,9 +213,10 @@ inline unsigned tiebreak_grid_y(uint64_t nx, uint32_t max_tiles) {
 
 // side streams (may be NULL / 0): launch classes are independent of one another, so they are
 // spread over the caller's stream and the side streams and joined again before returning
+constexpr int kSideStreams = 7;
 struct SideStreams {
-    cudaStream_t stream[3];
-    cudaEvent_t fork, join[3];
+    cudaStream_t stream[kSideStreams];
+    cudaEvent_t fork, join[kSideStreams];
     int n;
 };
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
