@@ -418,6 +418,10 @@ def roofline_of(stats_sum, dev_seconds, arith, sm_max, peak_kind):
         "frac": achieved / peak_cells if peak_cells else None,
         "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {sm_max:.0f} MHz ({peak_kind} max clock) / "
                      f"{slots:.0f} scheduler cycles per recurrence cell (2 adds + 1 max of 64-bit values)",
+        # a stricter denominator for context: only the FP64 pipe's occupancy counted (3 FP64
+        # instructions of 2 cycles per cell, selects free) -- no kernel can reach it, the probe
+        # cell itself stays at 0.67-0.71 of it
+        "frac_of_fp64_pipe_only": (achieved / (N_SM * 4 * 32 * sm_max * 1e6 / 6.0)) if arith == 0 else None,
         "cells_per_launch": stats_sum["cells"] / launches,
         "ms_per_launch": 1e3 * cost_s / launches,
         "share_of_step": cost_s / dev_seconds if dev_seconds else None,
