@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libchameleon.so")
 SOURCES = ["cm_cost_deep_f64.cu", "cm_cost_deep_i64.cu", "cm_cost_shallow_f64.cu", "cm_cost_shallow_i64.cu",
-           "cm_kernels.cu", "cm_api.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu", "cm_restore.cu", "cm_cache.cu"]
+           "cm_kernels.cu", "cm_api.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu", "cm_cost_solo.cu", "cm_restore.cu", "cm_cache.cu"]
 HEADERS = ["cm_internal.h", "cm_device.cuh", "cm_plan_eval.cuh", "cm_cost_impl.cuh"]
 
 NVCC_FLAGS = [

@@ -250,8 +250,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket_tseg.clear();
     struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; };
     std::vector<Pre> pre;
-    auto kind_of = [](int S, int m, uint64_t n_seg) {
+    auto kind_of = [](int S, int m, uint64_t n_seg, uint64_t count) {
         if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_GENERIC;
+        if (count == 1) return (int)CM_CLASS_SOLO;
         if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
         return (int)CM_CLASS_GENERIC;
     };
@@ -273,19 +274,20 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 const uint64_t n_seg = (uint64_t)(j - i) * tp.n_scen;
                 if (n_seg >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "too many segments in one bucket");
                 Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(j - i), g.S, g.m,
-                      g.K ? g.K + 1 : 1, (uint32_t)n_seg, kind_of(g.S, g.m, n_seg)};
+                      g.K ? g.K + 1 : 1, (uint32_t)n_seg, kind_of(g.S, g.m, n_seg, g.K ? g.K + 1 : 1)};
                 for (size_t k = i; k < j; ++k) bt.bucket_tseg.push_back(idx[k]);
                 pre.push_back(q);
             }
             i = j;
         }
     }
-    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_GENERIC; ++kind) {
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_SOLO; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
-        LaunchClass generic{CM_CLASS_GENERIC, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
+        const bool pooled_kind = kind == CM_CLASS_GENERIC || kind == CM_CLASS_SOLO;   // every depth in one class
+        LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
             LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
-            LaunchClass &c = kind == CM_CLASS_GENERIC ? generic : cls;
+            LaunchClass &c = pooled_kind ? pooled : cls;
             if (kind == CM_CLASS_WIDE_UNI) {
                 // a warp of the transposed kernel takes several consecutive items once the class
                 // is large enough to fill the GPU anyway
@@ -310,15 +312,17 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
                     const uint64_t per_cta = (uint64_t)(kChunk / 32) * c.uni_items;
                     c.n_chunks += (items + per_cta - 1) / per_cta;
+                } else if (kind == CM_CLASS_SOLO) {
+                    c.n_chunks += ((uint64_t)bk.n_seg + kChunk / 32 - 1) / (kChunk / 32);   // a warp per segment
                 } else {
                     c.n_chunks += (bk.count * bk.n_seg + kChunk - 1) / kChunk;
                 }
                 bt.bucket.push_back(bk);
                 c.bucket_end = (uint32_t)bt.bucket.size();
             }
-            if (kind != CM_CLASS_GENERIC && cls.n_chunks) { bt.classes.push_back(cls); kind_chunks += cls.n_chunks; }
+            if (!pooled_kind && cls.n_chunks) { bt.classes.push_back(cls); kind_chunks += cls.n_chunks; }
         }
-        if (kind == CM_CLASS_GENERIC && generic.n_chunks) bt.classes.push_back(generic);
+        if (pooled_kind && pooled.n_chunks) bt.classes.push_back(pooled);
     }
     for (const LaunchClass &c : bt.classes)
         if (c.n_chunks >= (1ull << 44)) return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");

@@ -480,7 +480,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_w
         __syncthreads();
         const uint64_t count = g.K ? g.K + 1 : 1;
         const uint64_t first = tile * kChunk;
-        if (first >= count || found_so_far < first) break;              // uniform: later tiles cannot win either
+        if (first >= count || found_so_far <= first) break;              // uniform: later tiles cannot win either
         const uint64_t kappa = first + threadIdx.x;
         uint64_t hit = ~0ull;
         if (kappa < count) {

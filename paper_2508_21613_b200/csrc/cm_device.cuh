@@ -369,6 +369,15 @@ __device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, const 
     else pl.cost = __longlong_as_double((long long)bits);
 }
 
+// Start values of the tie-break pass for one winner record: "not found yet" for every
+// pipeline, except that a segment whose only candidate is the min-max partition has nothing
+// to search -- that candidate is feasible and within the step time, or the pair would not have
+// won -- so its rank is known at once and the tie-break kernels leave it alone.
+__device__ __forceinline__ void init_kappa_sel(const BatchDev &bd, const Winner &w, uint64_t *slot /* [kMaxP] */) {
+    for (int p = 0; p < kMaxP; ++p)
+        slot[p] = (p < (int)w.dp && w.cost_bits < batch_inf_bits(bd) && bd.tseg[w.seg[p]].K == 0) ? 0ull : ~0ull;
+}
+
 // ----------------------------------------------------------------------------------
 // The pipeline-time recurrence of ONE pipeline spread over a warp: PER consecutive stages
 // per lane (S <= 32 * PER), walked in lock step over time slots.  With unit durations the
@@ -422,6 +431,24 @@ __device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B
         }
     }
     return __shfl_sync(0xffffffffu, clock[0], 0);
+}
+
+// Bare time of one pipeline (no synchronisation term), its stages spread over the warp.
+template <typename T, int PER>
+__device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *cuts, int S, int m, uint64_t tier, int lane) {
+    T F[PER], B[PER], xt[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        const int i = lane * PER + k;
+        F[k] = (T)0; B[k] = (T)0; xt[k] = (T)0;
+        if (i < S) {
+            const int lo = cuts[i], hi = cuts[i + 1];
+            F[k] = sp.PF[hi] - sp.PF[lo];
+            B[k] = sp.PB[hi] - sp.PB[lo];
+            if (i < S - 1) xt[k] = sp.XT[(tier >> i) & 1ull][hi - 1];
+        }
+    }
+    return sim_lockstep_n<T, PER>(S, m, F, B, xt);
 }
 
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {

@@ -100,7 +100,10 @@ struct Bucket {
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
-enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_GENERIC = 3 };
+enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_GENERIC = 3, CM_CLASS_SOLO = 4 };
+// CM_CLASS_SOLO: segments deeper than kRegStagesMax whose only candidate is the min-max partition.
+// One plan is one dependent chain (2*S*m cells, ~100 us in a single thread); a warp walks it in
+// lock step instead, stages over the lanes, four segments per CTA, every depth in one launch.
 constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
 constexpr int kUniMinSegments = 16; // fewer segments in a bucket: not worth transposing
 constexpr int kAnyMaxChunks = 4096; // shallow classes smaller than this together: one launch for all depths

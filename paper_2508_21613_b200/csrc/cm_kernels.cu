@@ -195,12 +195,12 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
         uint64_t oi = __shfl_xor_sync(0xffffffffu, best_i, o);
         if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
     }
-    if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
     if (threadIdx.x == 0) {
         Winner w;
         if (sc.rep != b) { best_c = inf; best_i = ~0ull; }   // shares another scenario's search: nothing to tie-break here
         decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
+        init_kappa_sel(bd, w, bd.kappa_sel + (size_t)b * kMaxP);
     }
 }
 
@@ -224,7 +224,6 @@ __global__ void __launch_bounds__(256) cm_split_winner_kernel(Tables tb, BatchDe
         if (pair_less(oc, oi, best_c, best_i)) { best_c = oc; best_i = oi; }
     }
     if ((threadIdx.x & 31) == 0) { rc[threadIdx.x >> 5] = best_c; ri[threadIdx.x >> 5] = best_i; }
-    if (threadIdx.x < kMaxP) bd.kappa_sel[b * kMaxP + threadIdx.x] = ~0ull;
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < 8; ++w)
@@ -232,6 +231,7 @@ __global__ void __launch_bounds__(256) cm_split_winner_kernel(Tables tb, BatchDe
         Winner w;
         decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
+        init_kappa_sel(bd, w, bd.kappa_sel + (size_t)b * kMaxP);
     }
 }
 
@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         __syncthreads();
         const uint64_t count = g.K ? g.K + 1 : 1;
         const uint64_t first = tile * kTile;
-        if (first >= count || found_so_far < first) break;          // uniform: later tiles cannot win either
+        if (first >= count || found_so_far <= first) break;          // uniform: later tiles cannot win either
         const uint64_t kappa = first + threadIdx.x;
         uint64_t hit = ~0ull;
         if (kappa < count) {

@@ -64,8 +64,8 @@ __global__ void __launch_bounds__(256) cm_shortlist_kernel(Tables tb, BatchDev b
             decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
             od.short_win[slot] = w;
             od.short_bytes[slot] = -1;
+            init_kappa_sel(bd, w, od.short_kappa + slot * kMaxP);
         }
-        if (threadIdx.x < kMaxP) od.short_kappa[slot * kMaxP + threadIdx.x] = ~0ull;
         __syncthreads();
         if (last_c >= inf) exhausted = true;   // uniform: nothing is left for later rounds either
     }
@@ -355,24 +355,6 @@ struct RoundsWork {
     uint8_t cuts[kMaxP][kMaxS + 4];
     uint8_t colour[kMaxL];
 };
-
-// Bare time of one pipeline (no synchronisation term), its stages spread over the warp.
-template <typename T, int PER>
-__device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *cuts, int S, int m, uint64_t tier, int lane) {
-    T F[PER], B[PER], xt[PER];
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        const int i = lane * PER + k;
-        F[k] = (T)0; B[k] = (T)0; xt[k] = (T)0;
-        if (i < S) {
-            const int lo = cuts[i], hi = cuts[i + 1];
-            F[k] = sp.PF[hi] - sp.PF[lo];
-            B[k] = sp.PB[hi] - sp.PB[lo];
-            if (i < S - 1) xt[k] = sp.XT[(tier >> i) & 1ull][hi - 1];
-        }
-    }
-    return sim_lockstep_n<T, PER>(S, m, F, B, xt);
-}
 
 template <typename T>
 __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables tb, BatchDev bd, ObjDev od) {
