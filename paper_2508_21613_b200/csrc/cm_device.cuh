@@ -373,9 +373,8 @@ __device__ __forceinline__ void plan_set_cost(cm_plan &pl, uint64_t bits, const 
 // pipeline, except that a segment whose only candidate is the min-max partition has nothing
 // to search -- that candidate is feasible and within the step time, or the pair would not have
 // won -- so its rank is known at once and the tie-break kernels leave it alone.
-__device__ __forceinline__ void init_kappa_sel(const BatchDev &bd, const Winner &w, uint64_t *slot /* [kMaxP] */) {
-    for (int p = 0; p < kMaxP; ++p)
-        slot[p] = (p < (int)w.dp && w.cost_bits < batch_inf_bits(bd) && bd.tseg[w.seg[p]].K == 0) ? 0ull : ~0ull;
+__device__ __forceinline__ void init_kappa_sel(const BatchDev &bd, const Winner &w, uint64_t *slot /* [kMaxP] */, int p) {
+    slot[p] = (p < (int)w.dp && w.cost_bits < batch_inf_bits(bd) && bd.tseg[w.seg[p]].K == 0) ? 0ull : ~0ull;
 }
 
 // ----------------------------------------------------------------------------------

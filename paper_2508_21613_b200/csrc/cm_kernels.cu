@@ -200,8 +200,9 @@ __global__ void __launch_bounds__(32) cm_winner_kernel(Tables tb, BatchDev bd, u
         if (sc.rep != b) { best_c = inf; best_i = ~0ull; }   // shares another scenario's search: nothing to tie-break here
         decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
-        init_kappa_sel(bd, w, bd.kappa_sel + (size_t)b * kMaxP);
     }
+    __syncthreads();   // the record is written: one thread per pipeline sets its start value
+    if (threadIdx.x < kMaxP) init_kappa_sel(bd, bd.winner[b], bd.kappa_sel + (size_t)b * kMaxP, (int)threadIdx.x);
 }
 
 // Both levels in one launch, for batches in which no scenario needs more than one block of the
@@ -231,8 +232,9 @@ __global__ void __launch_bounds__(256) cm_split_winner_kernel(Tables tb, BatchDe
         Winner w;
         decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
         bd.winner[b] = w;
-        init_kappa_sel(bd, w, bd.kappa_sel + (size_t)b * kMaxP);
     }
+    __syncthreads();   // the record is written: one thread per pipeline sets its start value
+    if (threadIdx.x < kMaxP) init_kappa_sel(bd, bd.winner[b], bd.kappa_sel + (size_t)b * kMaxP, (int)threadIdx.x);
 }
 
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st) {

@@ -64,8 +64,9 @@ __global__ void __launch_bounds__(256) cm_shortlist_kernel(Tables tb, BatchDev b
             decode_winner(tb, bd, tp, b, best_c, best_i, inf, w);
             od.short_win[slot] = w;
             od.short_bytes[slot] = -1;
-            init_kappa_sel(bd, w, od.short_kappa + slot * kMaxP);
         }
+        __syncthreads();   // last_c / last_i and the record are written
+        if (threadIdx.x < kMaxP) init_kappa_sel(bd, od.short_win[slot], od.short_kappa + slot * kMaxP, (int)threadIdx.x);
         __syncthreads();
         if (last_c >= inf) exhausted = true;   // uniform: nothing is left for later rounds either
     }
