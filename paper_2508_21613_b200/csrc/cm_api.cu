@@ -273,10 +273,24 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
             if (g.m >= 1) {   // m = 0 cannot be feasible: no work is scheduled
                 const uint64_t n_seg = (uint64_t)(j - i) * tp.n_scen;
                 if (n_seg >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "too many segments in one bucket");
-                Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(j - i), g.S, g.m,
-                      g.K ? g.K + 1 : 1, (uint32_t)n_seg, kind_of(g.S, g.m, n_seg, g.K ? g.K + 1 : 1)};
-                for (size_t k = i; k < j; ++k) bt.bucket_tseg.push_back(idx[k]);
-                pre.push_back(q);
+                const uint64_t count = g.K ? g.K + 1 : 1;
+                // The transposed kernel gives every 32 segments a warp per composition, full or
+                // not.  With one scenario the segments are few: what does not fill most of a
+                // last warp goes to the per-lane kernel, which wastes no lane.
+                size_t cut = j;
+                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, count) == CM_CLASS_WIDE_UNI) {
+                    const size_t rest = (j - i) % 32;
+                    if (rest > 0 && rest < (size_t)kUniMinSegments) cut = j - rest;
+                }
+                for (int part = 0; part < 2; ++part) {
+                    const size_t p0 = part ? cut : i, p1 = part ? j : cut;
+                    if (p1 <= p0) continue;
+                    const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
+                    Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
+                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, count)};
+                    for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
+                    pre.push_back(q);
+                }
             }
             i = j;
         }

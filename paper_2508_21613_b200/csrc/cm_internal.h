@@ -105,7 +105,8 @@ enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLAS
 // One plan is one dependent chain (2*S*m cells, ~100 us in a single thread); a warp walks it in
 // lock step instead, stages over the lanes, four segments per CTA, every depth in one launch.
 constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
-constexpr int kUniMinSegments = 16; // fewer segments in a bucket: not worth transposing
+constexpr int kUniMinSegments = 22; // fewer segments in a bucket (or left over after full warps of 32): the per-lane kernel
+                                    // is faster than a transposed warp that is two-thirds empty
 constexpr int kAnyMaxChunks = 4096; // shallow classes smaller than this together: one launch for all depths
 struct LaunchClass {
     int kind, stages;
