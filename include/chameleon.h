@@ -262,7 +262,7 @@ cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *space, uint64_
 typedef struct {
     int32_t topk;              /* 1 .. CM_MAX_SHORTLIST                                   */
     int32_t sync_rounds;       /* 0: step time as the search computes it; 1: asymmetric
-                                  synchronisation rounds (below)                           */
+                                  synchronisation rounds (above)                           */
     double t_gap_ns;           /* time between two faults (fp64 mode), finite, > 0          */
     double t_restart_ns;       /* restart overhead of a reconstruction (fp64 mode), >= 0     */
     int64_t t_gap_ns_i;        /* the same, integer nanoseconds (int64 mode)                */
@@ -293,8 +293,8 @@ typedef struct {
  * transition.  shortlist (HOST [B * topk], may be NULL) receives the shortlisted plans in
  * rank order, shortlist_bytes (HOST [B * topk], may be NULL) their matched bytes,
  * shortlist_rounds (HOST [B * topk], may be NULL) their communication rounds (0 unless
- * sync_rounds = 1); unused slots have feasible = 0, bytes = -1, rounds = 0.  Several matchings of one plan can be optimal:
- * assign[] is one of them, xfer_bytes is unique.
+ * sync_rounds = 1); unused slots have feasible = 0, bytes = -1, rounds = 0.  Several
+ * matchings of one plan can be optimal: assign[] is one of them, xfer_bytes is unique.
  * Errors: CM_EINVAL (bad options; more than CM_MAX_MATCH devices in the profile's grid),
  * CM_ENOPROFILE, CM_EOVERFLOW, CM_ENOMEM, CM_ECUDA.  A scenario without any feasible plan
  * has best[b].feasible = 0 and is not an error of the batch.  Synchronises the stream. */
