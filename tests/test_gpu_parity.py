@@ -451,3 +451,35 @@ def test_searches_on_a_caller_owned_stream(gpu, oracle_factory):
         stream.synchronize()
     finally:
         gpu.cm_destroy(ctx)
+
+
+@pytest.mark.parametrize("seed", [100, 101])
+def test_deep_pipelines_across_every_switch(gpu, oracle_factory, seed):
+    """Pipelines of 18..64 stages (one-plan segments walked by a warp, per-lane and transposed
+    kernels, the local-memory fallback) under every combination of cost mode, sharing, forced
+    integer kernels, batched and per-failure (resident batch + graph) search."""
+    import itertools
+    w = W.deep_pipeline(seed)
+    base = w.options
+    for mode, (cap, lm) in itertools.product((0, 1), ((40, W.LAYERS_REMAINDER), (5000, W.LAYERS_REMAINDER),
+                                                      (1 << 62, W.LAYERS_MINMAX))):
+        opts = W.SearchOptions(base.dp_lo, base.dp_hi, base.pp_lo, base.pp_hi, lm, base.batch_mode, cap, mode)
+        o = oracle_factory(w.profile, opts)
+        want = [o.search(f) for f in w.scenarios]
+        for share, native, latency in itertools.product((False, True), (False, True), (False, True)):
+            if native and mode == 0:
+                continue
+            s = Session(gpu, w.profile)
+            try:
+                gpu.cm_set_sharing(s.ctx, share)
+                gpu.cm_set_int64_arithmetic(s.ctx, native)
+                for _ in range(3 if latency else 1):
+                    best, pol, _ = gpu.cm_search_batch(s.ctx, w.scenarios, opts, per_policy=True, latency=latency)
+                plans, per = gpu.plans_from_array(best), gpu.plans_from_array(pol)
+                for b, failed in enumerate(w.scenarios):
+                    what = f"{w.name} {failed} mode={mode} cap={cap} share={share} native={native} latency={latency}"
+                    assert_same_plan(plans[b], want[b][0], mode, what)
+                    for q in range(3):
+                        assert_same_plan(per[3 * b + q], want[b][1][q] if want[b][1][q].feasible else None, mode, what)
+            finally:
+                s.close()
