@@ -483,3 +483,46 @@ def test_deep_pipelines_across_every_switch(gpu, oracle_factory, seed):
                         assert_same_plan(per[3 * b + q], want[b][1][q] if want[b][1][q].feasible else None, mode, what)
             finally:
                 s.close()
+
+
+def test_handworked_readings_rerouting_redundant_memory_minmax_ties(gpu, oracle_factory):
+    """The hand-worked cases that fix the readings taken where the paper prints no formula
+    (``tests/golden/*_handworked.txt``): the library must give the fixtures' own numbers, not
+    merely agree with the oracle."""
+    import reading_cases as R
+    for mode in (0, 1):
+        for prof, failed, expected in R.reroute_cases():
+            s = Session(gpu, prof)
+            try:
+                space, n = gpu.cm_enumerate(s.ctx, W.POLICY_REROUTE, failed, R.options(mode))
+                got = gpu.cm_select(s.ctx, [space])
+                assert n == 1 and got.feasible and _plan_cost(got, mode) == expected
+                want = oracle_factory(prof, R.options(mode)).search_policy(failed, W.POLICY_REROUTE)
+                assert_same_plan(got, want, mode, "rerouting, non-uniform stages")
+                gpu.cm_space_free(space)
+            finally:
+                s.close()
+        for prof, failed, feasible in R.redundant_cases():
+            s = Session(gpu, prof)
+            try:
+                space, _ = gpu.cm_enumerate(s.ctx, W.POLICY_REDUNDANT, failed, R.options(mode))
+                got = gpu.cm_select(s.ctx, [space])
+                assert (got is not None and bool(got.feasible)) == feasible
+                want = oracle_factory(prof, R.options(mode)).search_policy(failed, W.POLICY_REDUNDANT)
+                assert_same_plan(got, want, mode, "redundant computation, memory binding")
+                gpu.cm_space_free(space)
+            finally:
+                s.close()
+        for prof, S, bottleneck, cuts in R.minmax_tie_cases():
+            s = Session(gpu, prof)
+            try:
+                opts = R.minmax_only_options(S, mode)
+                space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [], opts)
+                got = gpu.cm_select(s.ctx, [space])
+                assert n == 1 and got.feasible
+                assert gpu.cm_decode_plan(s.ctx, space, got) == [cuts]
+                want = oracle_factory(prof, opts).search_policy([], W.POLICY_DYNPAR)
+                assert_same_plan(got, want, mode, "min-max tie")
+                gpu.cm_space_free(space)
+            finally:
+                s.close()
