@@ -4,8 +4,9 @@ plan-search latency per failure on B200.
 A step is one pass of the whole hot path (descriptor tables -> min-max partitions ->
 rerouting / redundant-computation plans -> cost kernel over every pipeline-plan ->
 split reduction -> tie-break pass -> policy pick -> plans on the host) over one batch
-of synthetic failure scenarios.  Default workload: the paper-scale configuration
-(32 devices DP4 x PP8, L=32, 2576 failure sets of 1-4 devices, every policy).
+of synthetic failure scenarios.  Default workload: the failure-scenario sweep, the largest
+configuration that fits one GPU (256 devices DP8 x PP32, L=96, 1024 failure sets of 1-16
+devices, every policy); the other configurations are timed as context under "workloads".
 
   python bench.py --gpus 1 --steps K --warmup W            # this library
   python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
@@ -29,11 +30,23 @@ METRIC = "candidate_plans_evaluated_per_sec"
 UNIT = "plans/s"
 N_SM = 148
 SM_MAX_MHZ_FALLBACK = 1965.0
-# issue cycles per recurrence cell (2 adds + 1 max of 64-bit values) on sm_100a, where an
-# FP64 instruction holds a scheduler for 2 cycles (16 FP64 lanes per scheduler) and the
-# 64-bit integer max costs 4 half-rate integer instructions:
-#   fp64:  2 DADD (4) + DSETP (2) + 2 SEL (2) = 8       int64: measured 12.3 by a probe kernel
-ISSUE_SLOTS_PER_CELL = {0: 8.0, 1: 12.0}
+# The search pass is issue bound (no algorithmic HBM traffic, no contraction).  Its bound is
+#   cells/s <= N_SM x 4 schedulers x 32 lanes x f_clk / I_cell
+# with I_cell = executed thread-instructions per recurrence cell of the kernel class that
+# dominates the workload, taken from the ncu capture summarised in the named file under
+# profiles/ (instruction counters of one launch / its cells); `issue_active` is that capture's
+# issue-slot utilisation.  f_clk is the median SM clock sampled while the timed region ran.
+# class: "regs" = cm_cost_regs_kernel (pipelines of <= 16 stages), "wide" = the deep-pipeline
+# kernel (17 .. 64 stages); arithmetic 0 = fp64 (also the exact integer-valued mode), 1 = int64.
+KERNEL_PROFILES = {
+    ("regs", 0): {"i_cell": 5.79, "issue_active": 0.647, "fp64_pipe_active": 0.649,
+                  "profile": "profiles/cm_cost_regs_kernel_paper-scale-512.md"},
+    ("regs", 1): {"i_cell": 8.64, "issue_active": 0.630, "fp64_pipe_active": 0.0,
+                  "profile": "profiles/cm_cost_regs_kernel_int64_paper-scale-512.md"},
+    ("wide", 0): {"i_cell": 7.32, "issue_active": 0.586, "fp64_pipe_active": 0.530,
+                  "profile": "profiles/cm_cost_wide_kernel_175b-like-8.md"},
+}
+FP64_INSTR_PER_CELL = 3.0          # 2 DADD + 1 DSETP; an FP64 warp instruction occupies its pipe for 2 cycles
 TRAFFIC_BYTES_PER_CTA = 645888.0 / 55800.0   # dram__bytes_read+write of one ncu-captured launch / its CTAs
 
 
@@ -134,22 +147,38 @@ def gather_rows(values, world: int, device: str):
     return [g.cpu().tolist() for g in gathered]
 
 
-def oracle_sample(w, mode: int, budget_s: float, max_scenarios: int):
-    """Time the CPU oracle, as it stands, on the first scenarios of the workload until the
-    budget is used.  -> (plans, seconds, scenarios)."""
-    from oracle.oracle import Oracle
-    opts = w.options.with_cost_mode(mode)
-    orc = Oracle(w.profile, opts)
-    plans, t_total, n = 0, 0.0, 0
-    for failed in w.scenarios[:max_scenarios]:
-        t0 = time.perf_counter()
-        orc.search(failed)
-        t_total += time.perf_counter() - t0
-        plans += orc.count(failed)[0] + 2
-        n += 1
-        if t_total >= budget_s:
-            break
-    return plans, t_total, n
+ORACLE_SAMPLE = 65536   # candidates the oracle evaluates per sampled scenario
+
+
+def oracle_sample(orc, w, k: int, n_cand_sample: int = ORACLE_SAMPLE):
+    """A bounded sample of the workload for the CPU oracle, as it stands, single thread:
+    scenario k's rerouting and redundant-computation plans plus `n_cand_sample` of its
+    dynamic-parallelism candidates drawn uniformly (seeded) from its whole candidate space.
+    A full oracle search of one sweep scenario takes 10-30 s, too long for a bench step; the
+    sample keeps the workload's mix of pipeline shapes.  -> (plans evaluated, seconds)."""
+    import numpy as np
+    from paper_2508_21613_b200 import workloads as W
+    failed = w.scenarios[k % len(w.scenarios)]
+    t0 = time.perf_counter()
+    n = orc.count(failed)[0]
+    plans = 0
+    if n > 0:
+        if n <= n_cand_sample:
+            orc.evaluate(failed)
+            plans += n
+        else:
+            rng = W.SplitMix64(0x0A11CE + k)
+            idx = np.sort(np.asarray([rng.below(n) for _ in range(n_cand_sample)], dtype=np.uint64))
+            orc.evaluate(failed, idx=idx)
+            plans += n_cand_sample
+    orc.search_policy(failed, 0)
+    orc.search_policy(failed, 1)
+    return plans + 2, time.perf_counter() - t0
+
+
+def oracle_describe(w, n_scen: int) -> str:
+    return (f"{n_scen} failure scenario(s) of '{w.name}': the rerouting and the redundant-computation plan and a seeded "
+            f"uniform sample of {ORACLE_SAMPLE} dynamic-parallelism pipeline-plans each, single thread")
 
 
 def run_reference(args):
@@ -157,31 +186,34 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2508_21613_b200 import workloads as W
+    from oracle.oracle import Oracle
     w = W.ALL_WORKLOADS[args.workload]()
+    orc = Oracle(w.profile, w.options.with_cost_mode(args.cost_mode))
     per_step = max(1, args.ref_scenarios)
-    for _ in range(args.warmup):
-        oracle_sample(w, args.cost_mode, 1e9, min(2, per_step))
+    for k in range(args.warmup):
+        oracle_sample(orc, w, len(w.scenarios) - 1 - k)
     plans, seconds = 0, 0.0
     for k in range(args.steps):
-        sub = W.Workload(w.name, w.profile, w.options, w.scenarios[k * per_step:(k + 1) * per_step] or w.scenarios[:per_step])
-        p, s, _ = oracle_sample(sub, args.cost_mode, 1e9, per_step)
-        plans += p
-        seconds += s
+        for j in range(per_step):
+            p, s = oracle_sample(orc, w, k * per_step + j)
+            plans += p
+            seconds += s
     value = plans / seconds
-    sample = f"{per_step} failure scenarios of '{w.name}' per step, single thread, all three policies"
+    sample = oracle_describe(w, per_step) + " per step"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * seconds / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": ("f64 (integer-valued, exact)" if m["arith"] == 0 else "i64") if args.cost_mode else "f64",
+            "dtype": "i64" if args.cost_mode else "f64",
             "data": "synthetic",
-            "config": {"workload": w.name, "scenarios_per_step": per_step, "cost_mode": args.cost_mode},
+            "config": {"workload": w.name, "scenarios_per_step": per_step,
+                       "cost_mode": "int64ns" if args.cost_mode else "fp64"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
 def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, latency_scenarios, sample_clocks=True,
-            native_i64=False):
+            native_i64=False, cold_latency=True):
     """One workload on this rank: device-resident arm, end-to-end arm, per-failure latency."""
     import numpy as np
     opts = w.options.with_cost_mode(mode)
@@ -242,10 +274,41 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
         lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
         out["latency_us"] = {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
                              "max": float(lat[-1]), "scenarios": int(lat_pack.B),
-                             "what": "one failure set, all policies, descriptor build to plan on host"}
+                             "what": "one failure set, all policies, descriptor build to plan on host; third pass over "
+                                     "the scenarios: the batch of that survivor count is resident and its launch "
+                                     "sequence replays as a CUDA graph"}
     finally:
         binding.cm_destroy(ctx)
+    if cold_latency:
+        out["latency_us"]["cold"] = measure_cold_latency(binding, w, opts, local_rank, native_i64)
     return out
+
+
+def measure_cold_latency(binding, w, opts, local_rank, native_i64=False, max_sizes=16):
+    """A failure is a first occurrence: the latency of the FIRST search of a survivor count on a
+    context that has searched nothing yet (profile loaded; no resident batch, no captured graph,
+    min-max partitions not computed).  One fresh context and one scenario per failure-set size of
+    the workload; the process itself is warm (kernels were loaded by the legs before)."""
+    import numpy as np
+    by_size = {}
+    for sc in w.scenarios:
+        by_size.setdefault(len(sc), sc)
+    lat = []
+    for size in sorted(by_size)[:max_sizes]:
+        ctx = binding.cm_create(local_rank)
+        try:
+            binding.cm_load_profile(ctx, w.profile)
+            if native_i64:
+                binding.cm_set_int64_arithmetic(ctx, True)
+            pack = binding.PackedScenarios([by_size[size]])
+            pack.search(ctx, opts, latency=True)
+            lat.append(float(pack.latency[0]))
+        finally:
+            binding.cm_destroy(ctx)
+    lat = np.sort(np.asarray(lat))
+    return {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)), "max": float(lat[-1]),
+            "scenarios": int(len(lat)),
+            "what": "first search of a failure-set size on a fresh context (one per size), descriptor build to plan on host"}
 
 
 def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush):
@@ -406,42 +469,54 @@ def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
     return out
 
 
-def roofline_of(stats_sum, dev_seconds, arith, sm_max, peak_kind):
-    slots = ISSUE_SLOTS_PER_CELL[arith]
-    peak_cells = N_SM * 4 * 32 * sm_max * 1e6 / slots
+def kernel_class(w) -> str:
+    """Search-pass kernel that carries a workload: pipelines of the search window deeper than
+    16 stages run the deep-pipeline kernel, the others the register-resident one."""
+    return "wide" if w.options.pp_hi > 16 and w.profile.n_pp > 16 else "regs"
+
+
+def roofline_of(stats_sum, dev_seconds, arith, kclass, clocks, sm_max, peak_kind):
+    prof = KERNEL_PROFILES.get((kclass, arith)) or KERNEL_PROFILES[(kclass, 0)]
+    f_mhz = float((clocks or {}).get("sm_mhz") or sm_max)
+    lanes_per_s = N_SM * 4 * 32 * f_mhz * 1e6
+    peak_cells = lanes_per_s / prof["i_cell"]
     cost_s = stats_sum["cost_kernel_ns"] * 1e-9
     achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
     launches = max(1, stats_sum["cost_kernel_launches"])
     return {
-        "bound": "alu", "kernel": "search pass: cm_cost_regs_kernel / cm_cost_wide_kernel / cm_cost_generic_kernel",
+        "bound": "alu", "kernel": {"regs": "cm_cost_regs_kernel", "wide": "cm_cost_wide_kernel"}[kclass] + " (search pass)",
         "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell/s",
         "frac": achieved / peak_cells if peak_cells else None,
-        "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {sm_max:.0f} MHz ({peak_kind} max clock) / "
-                     f"{slots:.0f} scheduler cycles per recurrence cell (2 adds + 1 max of 64-bit values)",
-        # a stricter denominator for context: only the FP64 pipe's occupancy counted (3 FP64
-        # instructions of 2 cycles per cell, selects free) -- no kernel can reach it, the probe
-        # cell itself stays at 0.67-0.71 of it
-        "frac_of_fp64_pipe_only": (achieved / (N_SM * 4 * 32 * sm_max * 1e6 / 6.0)) if arith == 0 else None,
+        "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {f_mhz:.0f} MHz (median SM clock sampled during the timed region; "
+                     f"{peak_kind} max {sm_max:.0f}) / I_cell",
+        "i_cell": prof["i_cell"],
+        "i_cell_source": f"executed thread-instructions per recurrence cell, ncu capture in {prof['profile']}",
+        "issue_active_profiled": prof["issue_active"],
+        # against the FP64 pipe alone: 3 FP64 instructions per cell, each holding the pipe of a
+        # scheduler (16 lanes) for 2 cycles
+        "frac_of_fp64_pipe": (achieved / (lanes_per_s / (2.0 * FP64_INSTR_PER_CELL))) if arith == 0 else None,
+        "fp64_pipe_active_profiled": prof["fp64_pipe_active"],
         "cells_per_launch": stats_sum["cells"] / launches,
         "ms_per_launch": 1e3 * cost_s / launches,
         "share_of_step": cost_s / dev_seconds if dev_seconds else None,
-        # DRAM bytes of one search-pass launch from an ncu capture of the 512-scenario case
-        # (0.65 MB for 55 800 CTAs of the 12-stage kernel), scaled by CTAs; the kernel reads only
-        # the small descriptor tables, so this is context, not a bound
-        "traffic": TRAFFIC_BYTES_PER_CTA * stats_sum["plans"] / max(1, stats_sum["cost_kernel_launches"]) / 128.0,
+        # the search pass reads only the small descriptor tables: ~0 algorithmic bytes.  Not
+        # measured in this run: DRAM bytes of one ncu-captured launch (0.65 MB for 55 800 CTAs of
+        # the 12-stage kernel) scaled by this run's CTAs per launch.
+        "traffic": TRAFFIC_BYTES_PER_CTA * stats_sum["plans"] / launches / 128.0,
+        "traffic_source": "scaled by CTAs from the ncu capture in profiles/cm_cost_regs_kernel_paper-scale-512.md",
     }
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="paper-scale")
+    ap.add_argument("--workload", default="sweep")
     ap.add_argument("--cost-mode", type=int, default=0, choices=[0, 1])
-    ap.add_argument("--ref-scenarios", type=int, default=16, help="oracle scenarios per step (--impl reference)")
-    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--ref-scenarios", type=int, default=1, help="sampled oracle scenarios per step (--impl reference)")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--latency-scenarios", type=int, default=4096, help="scenarios searched one by one for latency")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads / cost mode summary")
@@ -496,6 +571,9 @@ def main():
             "dtype": ("f64 (integer-valued, exact)" if m["arith"] == 0 else "i64") if args.cost_mode else "f64",
             "data": "synthetic",
             "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": m["plans_per_step"],
+                       # plans whose recurrence ran / plans the memory estimator rejected before it
+                       "plans_simulated_per_step": m["stats"]["plans_simulated"] // args.steps + 2 * len(w.scenarios),
+                       "plans_memory_rejected": (m["stats"]["plans"] - m["stats"]["plans_simulated"]) // args.steps,
                        "policies": 3, "cost_mode": "int64ns" if args.cost_mode else "fp64",
                        "l2": "flushed between timed iterations (256 MB write)",
                        "parallelism": "replicas, scenarios independent" if world > 1 else "1 gpu"},
@@ -505,43 +583,53 @@ def main():
             "latency_us": m["latency_us"],
             "gpu_launches": int(m["stats"]["launches"]),
             "clocks": m["clocks"],
-            "roofline": roofline_of(m["stats"], m["dev_seconds"], m["arith"], sm_max, peak_kind),
+            "roofline": roofline_of(m["stats"], m["dev_seconds"], m["arith"], kernel_class(w), m["clocks"], sm_max, peak_kind),
         }
         if not args.no_cpu_baseline:
-            p, s, n = oracle_sample(w, args.cost_mode, args.cpu_budget, len(w.scenarios))
-            line["cpu_baseline"] = {"value": p / s, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": f"first {n} failure scenarios of '{w.name}', all three policies, "
-                                              f"{s:.1f} s single-threaded",
-                                    "latency_us_per_failure": 1e6 * s / n}
+            from oracle.oracle import Oracle
+            orc = Oracle(w.profile, w.options.with_cost_mode(args.cost_mode))
+            p_sum, s_sum, n = 0, 0.0, 0
+            while s_sum < args.cpu_budget and n < len(w.scenarios):
+                p, s = oracle_sample(orc, w, n)
+                p_sum, s_sum, n = p_sum + p, s_sum + s, n + 1
+            line["cpu_baseline"] = {"value": p_sum / s_sum, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": oracle_describe(w, n) + f", {s_sum:.1f} s"}
         if not args.no_extra and world == 1 and args.scenarios == 0:
             # the other configurations (and the other cost mode), two timed steps each: context
             # for the headline line above, same measurement code
             from paper_2508_21613_b200 import workloads as W
             extra = {}
             todo = [(args.workload, 1 - args.cost_mode)]
-            todo += [(name, args.cost_mode) for name in ("tiny", "70b-like", "175b-like", "sweep") if name != args.workload]
+            todo += [(name, args.cost_mode) for name in ("tiny", "paper-scale", "70b-like", "175b-like", "sweep") if name != args.workload]
+            n_extra = 5
             for name, mode in todo:
                 ew = W.ALL_WORKLOADS[name]()
-                em = measure(binding, torch, ew, mode, 2, 3, local_rank, barrier, flush, args.latency_scenarios,
-                             sample_clocks=False)
-                r = roofline_of(em["stats"], em["dev_seconds"], em["arith"], sm_max, peak_kind)
+                em = measure(binding, torch, ew, mode, n_extra, 3, local_rank, barrier, flush, args.latency_scenarios)
+                r = roofline_of(em["stats"], em["dev_seconds"], em["arith"], kernel_class(ew), em["clocks"], sm_max, peak_kind)
                 extra[f"{name}/{'int64ns' if mode else 'fp64'}"] = {
-                    "scenarios": len(ew.scenarios), "plans_per_step": em["plans_per_step"],
-                    "plans_per_s": em["plans_per_step"] * 2 / em["dev_seconds"],
-                    "ms_per_step": 1e3 * em["dev_seconds"] / 2, "e2e_ms_per_step": 1e3 * em["e2e_seconds"] / 2,
+                    "scenarios": len(ew.scenarios), "steps": n_extra, "plans_per_step": em["plans_per_step"],
+                    "plans_memory_rejected": (em["stats"]["plans"] - em["stats"]["plans_simulated"]) // n_extra,
+                    "plans_per_s": em["plans_per_step"] * n_extra / em["dev_seconds"],
+                    "ms_per_step": 1e3 * em["dev_seconds"] / n_extra, "e2e_ms_per_step": 1e3 * em["e2e_seconds"] / n_extra,
                     "latency_us_p50": em["latency_us"]["p50"], "latency_us_p99": em["latency_us"]["p99"],
+                    "latency_us_cold_p50": em["latency_us"]["cold"]["p50"], "latency_us_cold_p99": em["latency_us"]["cold"]["p99"],
                     "latency_scenarios": em["latency_us"]["scenarios"],
-                    "search_pass_gcell_s": r["achieved"], "search_pass_frac": r["frac"]}
+                    "search_pass_kernel": r["kernel"], "search_pass_gcell_s": r["achieved"],
+                    "search_pass_frac": r["frac"], "search_pass_frac_of_fp64_pipe": r["frac_of_fp64_pipe"],
+                    "clocks_sm_mhz": (em["clocks"] or {}).get("sm_mhz")}
             line["workloads"] = extra
             # widening beyond the plan search: transition time in the objective
             line["full_objective"] = {
                 name: measure_objective(binding, torch, W.ALL_WORKLOADS[name](), args.cost_mode, 3, 3, local_rank, flush)
-                for name in dict.fromkeys((args.workload, "175b-like", "sweep"))}
+                for name in dict.fromkeys((args.workload, "paper-scale", "175b-like"))}
         if not args.no_extra and world == 1 and args.scenarios == 0:
             line["shared_search"] = measure_shared(binding, torch, w, args.cost_mode, local_rank, flush)
-        if not args.no_extra and world == 1 and args.scenarios == 0 and w.profile.n_dp * w.profile.n_pp <= 64:
-            line["plan_cache"] = measure_cache(binding, w, args.cost_mode, local_rank)
-            line["failure_trace"] = measure_trace(binding, w, args.cost_mode, local_rank)
+        if not args.no_extra and world == 1 and args.scenarios == 0:
+            # plan cache and failure-trace replay at the scale of the paper's cluster (32 devices)
+            from paper_2508_21613_b200 import workloads as W
+            small = w if w.profile.n_dp * w.profile.n_pp <= 64 else W.paper_scale(0, 0)
+            line["plan_cache"] = dict(measure_cache(binding, small, args.cost_mode, local_rank), workload=small.name)
+            line["failure_trace"] = dict(measure_trace(binding, small, args.cost_mode, local_rank), workload=small.name)
         if args.objective and "full_objective" not in line:
             line["full_objective"] = {w.name: measure_objective(binding, torch, w, args.cost_mode, args.steps,
                                                                 args.warmup, local_rank, flush)}

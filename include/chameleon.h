@@ -303,6 +303,17 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist,
                               int64_t *shortlist_bytes, int32_t *shortlist_rounds);
 
+/* Transition time the full objective charges a reconstruction that moves xfer_bytes of model
+ * state (Section "Estimator", state-transition overhead = restart + weight transfer):
+ * fp64 mode t_restart_ns + bytes / bw_xfer (one IEEE operation each), int64 mode
+ * t_restart_ns_i + floor(bytes / bw_xfer) -- the very routine the objective kernel applies, so a
+ * caller can price the shortlisted plans that were not chosen from the shortlist_bytes of
+ * cm_search_objective without restating the rule.  All pointers HOST; n values; either output
+ * may be NULL; an entry of -1 (empty shortlist slot) gives -1.  No device work.
+ * CM_EINVAL on NULL options, negative n or a non-positive bandwidth. */
+cm_status cm_transition_time(const cm_objective_opts *objective, int32_t n, const int64_t *xfer_bytes,
+                             double *t_trans_ns, int64_t *t_trans_ns_i);
+
 /* The host-side descriptor builder alone, for one failure set and the dynamic-parallelism
  * policy (Algorithm 1, get_parallel_strategy; Section "Planner", batch and layer
  * distribution): no CUDA call is made, so it also runs on a machine without a GPU.
@@ -393,7 +404,7 @@ cm_status cm_cache_lookup(const cm_cache *cache, const uint32_t *failed_ids, int
 cm_status cm_cache_free(cm_cache *cache);
 
 /* Work counters of the last cm_select / cm_search_batch / cm_batch_search on this
- * context (HOST out[16]):
+ * context (HOST out[24]):
  *  [0] pipeline-plans evaluated by the search pass   [1] recurrence cells simulated by it
  *      (2 * stages * micro-batches per memory-feasible plan, counted on the device)
  *  [2] pipeline-plans re-evaluated by the tie-break pass   [3] kernels launched
@@ -402,8 +413,11 @@ cm_status cm_cache_free(cm_cache *cache);
  *  [8] device time of the search-pass cost kernel(s) alone, ns   [9] bytes copied host->device
  *  [10] bytes copied device->host   [11] device time of the tie-break kernel(s), ns
  *  [12] launches of the search-pass cost kernel   [13] host time building descriptor tables, ns
- *  [14] host time enqueueing the launch sequence, ns   [15] host time waiting for the stream, ns. */
-cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]);
+ *  [14] host time enqueueing the launch sequence, ns   [15] host time waiting for the stream, ns
+ *  [16] pipeline-plans of [0] whose recurrence ran, i.e. that passed the memory estimator
+ *       (Section "Estimator", memory estimator); [0] - [16] were rejected by it
+ *  [17..23] reserved, 0. */
+cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[24]);
 
 const char *cm_strerror(cm_status status);
 const char *cm_last_error(const cm_ctx *ctx);

@@ -31,8 +31,8 @@ EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_eva
            "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
            "cm_objective_stats", "cm_transfer_matching", "cm_cache_build", "cm_cache_lookup", "cm_cache_free",
            "cm_set_sharing", "cm_set_int64_arithmetic", "cm_host_describe", "cm_set_latency_graphs",
-           "cm_int64_runs_in_fp64", "cm_strerror", "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:24]
+           "cm_transition_time", "cm_int64_runs_in_fp64", "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:25]
 NOALLOC_MAX_CANDIDATES = 524288
 MAX_SHORTLIST, MAX_MATCH = 16, 256
 
@@ -157,6 +157,8 @@ def load_library() -> C.CDLL:
     lib.cm_set_latency_graphs.argtypes = [vp, C.c_int]
     lib.cm_host_describe.argtypes = [C.POINTER(cm_profile), C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_enum_opts), u64p]
     lib.cm_set_int64_arithmetic.argtypes = [vp, C.c_int]
+    lib.cm_transition_time.argtypes = [C.POINTER(cm_objective_opts), C.c_int32, C.POINTER(C.c_int64),
+                                       C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.cm_int64_runs_in_fp64.argtypes = [vp]
     lib.cm_int64_runs_in_fp64.restype = C.c_int
     for name in _STATUS_CALLS:
@@ -326,6 +328,19 @@ def cm_search_objective(ctx, scenarios: Sequence[Sequence[int]], opts, objective
     return packed.search_objective(ctx, opts, objective, shortlist)
 
 
+def cm_transition_time(objective, xfer_bytes) -> Tuple[np.ndarray, np.ndarray]:
+    """Transition times of reconstructions that move ``xfer_bytes`` (any shape, int64; -1 = empty
+    slot) -> (float64 ns for the fp64 mode, int64 ns for the integer mode), same shape."""
+    b = np.ascontiguousarray(xfer_bytes, dtype=np.int64)
+    t = np.zeros(b.shape, dtype=np.float64)
+    ti = np.zeros(b.shape, dtype=np.int64)
+    q = _objective(objective)
+    _check(None, load_library().cm_transition_time(C.byref(q), b.size, b.ctypes.data_as(C.POINTER(C.c_int64)),
+                                                   t.ctypes.data_as(C.POINTER(C.c_double)),
+                                                   ti.ctypes.data_as(C.POINTER(C.c_int64))))
+    return t, ti
+
+
 def cm_objective_stats(ctx) -> dict:
     out = (C.c_uint64 * 8)()
     _check(ctx, load_library().cm_objective_stats(ctx, out))
@@ -408,11 +423,11 @@ def cm_batch_free(batch) -> None:
 
 
 def cm_last_stats(ctx) -> dict:
-    out = (C.c_uint64 * 16)()
+    out = (C.c_uint64 * 24)()
     _check(ctx, load_library().cm_last_stats(ctx, out))
     keys = ["plans", "cells", "tiebreak_plans", "launches", "device_ns", "segments", "strategies", "splits",
             "cost_kernel_ns", "h2d_bytes", "d2h_bytes", "tiebreak_kernel_ns", "cost_kernel_launches",
-            "host_build_ns", "host_enqueue_ns", "host_wait_ns"]
+            "host_build_ns", "host_enqueue_ns", "host_wait_ns", "plans_simulated"]
     return dict(zip(keys, [int(v) for v in out]))
 
 

@@ -114,12 +114,18 @@ struct Batch {
     uint32_t max_tiles_per_seg = 0, dp_max = 0;
     int B = 0;
     bool intval = false;                   // integer mode evaluated in double arithmetic (fixed when the batch is built)
+    uint64_t profile_gen = 0;              // generation of the profile the tables describe (see cm_ctx::profile_gen)
 };
 
 struct cm_ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
     bool has_profile = false;
+    // Bumped by every cm_load_profile.  Descriptor tables (a cm_space, a cm_batch) are stamped with
+    // the generation they were built under: their segment shapes, min-max keys and candidate
+    // counts describe that profile's L and G, so they are refused once another profile is loaded.
+    uint64_t profile_gen = 0;
+    DevBuf<unsigned char> d_scratch;  // small per-call device scratch (cm_select, cm_transfer_matching): grown, never shrunk
     DevProfile hp{};                  // host copy: scalars, raw inputs, base cuts
     DevProfile *d_prof = nullptr;
     // The integer-nanosecond mode normally runs in double arithmetic: its inputs are integers,
@@ -165,7 +171,7 @@ struct cm_ctx {
     cudaStream_t pol_stream = nullptr;
     cudaEvent_t pol_fork = nullptr, pol_join = nullptr;
     SideStreams side{};               // library-owned streams for independent launch classes
-    uint64_t stats[16] = {0};
+    uint64_t stats[24] = {0};
     std::string err;
 };
 
@@ -188,6 +194,23 @@ cm_status fail(cm_ctx *c, cm_status s, const std::string &msg) {
     if (c) c->err = msg;
     return s;
 }
+
+// Tables built under an earlier profile describe another L and G: refuse them.
+bool stale(const cm_ctx *c, const Batch &bt) { return bt.profile_gen != c->profile_gen; }
+const char *const kStaleMsg = "space or batch was built for an earlier profile: enumerate / prepare it again after cm_load_profile";
+
+// No exception may cross the C ABI (the host side uses std::vector / std::string / std::map).
+cm_status api_caught(cm_ctx *c, cm_status s) noexcept {
+    if (c) {
+        try { c->err = s == CM_ENOMEM ? "host memory exhausted" : "internal error (unexpected exception)"; } catch (...) {}
+    }
+    return s;
+}
+#define CM_API_BEGIN try {
+#define CM_API_END(ctx)                                                           \
+    }                                                                             \
+    catch (const std::bad_alloc &) { return api_caught((ctx), CM_ENOMEM); }       \
+    catch (...) { return api_caught((ctx), CM_EINVAL); }
 
 #define CM_CUDA(ctx, expr)                                                                       \
     do {                                                                                         \
@@ -439,6 +462,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.scen.clear(); bt.tmpl.clear(); bt.strat.clear(); bt.tseg.clear(); bt.failed.clear(); bt.red_scen.clear();
     bt.keys.clear(); bt.tmpl_scen.clear(); bt.cross.clear();
     bt.opts = o;
+    bt.profile_gen = ctx->profile_gen;
     bt.intval = o.cost == CM_COST_INT64NS && ctx->exact53 && !ctx->force_native_i64;
     bt.policy_mask = policy_mask;
     bt.n_cand = bt.n_tiles = bt.n_split = bt.n_rows = 0;
@@ -731,6 +755,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far, cm_ctx::Single 
     ctx->stats[0] += (bt.policy_mask & (1u << CM_DYNPAR)) ? bt.n_cand : 0;
     ctx->stats[1] += counters_host[0];
     ctx->stats[2] += counters_host[1];
+    ctx->stats[16] += counters_host[2];
     ctx->stats[3] += (uint64_t)launches;
     ctx->stats[4] += (uint64_t)((double)ms * 1e6);
     ctx->stats[5] += bt.n_rows;
@@ -836,6 +861,7 @@ int cm_internal_grid_devices(const cm_ctx *ctx) { return ctx && ctx->has_profile
 cm_status cm_internal_space_view(cm_ctx *ctx, const cm_space *space, SpaceView *out) {
     if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
     Batch &bt = const_cast<Batch &>(space->batch);
+    if (stale(ctx, bt)) return fail(ctx, CM_EINVAL, kStaleMsg);
     out->tb = tables(ctx, bt);
     out->bd = dev_view(ctx, bt);
     out->n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
@@ -893,6 +919,7 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
              cudaEventCreateWithFlags(&c->side.join[i], cudaEventDisableTiming) == cudaSuccess;
         if (ok) c->side.n = i + 1;
     }
+    ok = ok && c->d_scratch.reserve(sizeof(cm_plan *) * 64 + sizeof(cm_plan));   // what cm_select needs
     if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess ||
         cudaMalloc((void **)&c->d_prof53, sizeof(DevProfile)) != cudaSuccess) {
         if (c->d_prof) cudaFree(c->d_prof);
@@ -1006,9 +1033,11 @@ static cm_status load_profile_host(cm_ctx *ctx, const cm_profile *p) {
 
 cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
     CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // nothing may still read the old profile
     ctx->has_profile = false;
+    ++ctx->profile_gen;                                  // spaces and batches of the old profile are refused from here on
     ctx->single.clear();                                 // prepared one-scenario batches describe the old profile
     cm_status s = load_profile_host(ctx, p);
     if (s != CM_OK) return s;
@@ -1032,12 +1061,14 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // ctx->hp / binom may change on the next load
     ctx->has_profile = true;
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 // The descriptor builder alone, for one failure set, without a GPU (no CUDA call is made).
 cm_status cm_host_describe(const cm_profile *p, const uint32_t *failed_ids, int32_t n_failed,
                            const cm_enum_opts *opts, uint64_t out[8]) {
     if (!p || !opts || !out || n_failed < 0 || (n_failed > 0 && !failed_ids)) return CM_EINVAL;
+    CM_API_BEGIN
     cm_ctx ctx;   // plain host object: nothing here touches the device
     cm_status s = load_profile_host(&ctx, p);
     if (s == CM_OK) s = check_opts(&ctx, opts);
@@ -1058,11 +1089,13 @@ cm_status cm_host_describe(const cm_profile *p, const uint32_t *failed_ids, int3
     out[6] = bt.bucket.size();
     out[7] = crossings;
     return CM_OK;
+    CM_API_END(nullptr)
 }
 
 cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids, int32_t n_failed,
                        const cm_enum_opts *opts, cm_space **out, uint64_t *n_candidates) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (!out) return fail(ctx, CM_EINVAL, "out is NULL");
     if (policy < CM_REROUTE || policy > CM_DYNPAR) return fail(ctx, CM_EINVAL, "bad policy");
@@ -1074,7 +1107,7 @@ cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids
     cm_status s = check_opts(ctx, &o);
     if (s != CM_OK) return s;
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
-    cm_space *sp = new (std::nothrow) cm_space();
+    std::unique_ptr<cm_space> sp(new (std::nothrow) cm_space());   // released on every error path, a thrown one included
     if (!sp) return fail(ctx, CM_ENOMEM, "host memory");
     sp->ctx = ctx;
     sp->policy = policy;
@@ -1091,12 +1124,12 @@ cm_status cm_enumerate(cm_ctx *ctx, cm_policy policy, const uint32_t *failed_ids
     if (s != CM_OK) {
         cudaStreamSynchronize(ctx->stream);
         forget_keys(ctx, sp->batch);
-        delete sp;
         return s;
     }
-    *out = sp;
     if (n_candidates) *n_candidates = policy == CM_DYNPAR ? sp->batch.n_cand : 1;
+    *out = sp.release();
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_space_free(cm_space *sp) {
@@ -1110,23 +1143,29 @@ cm_status cm_space_free(cm_space *sp) {
 cm_status cm_evaluate(cm_ctx *ctx, const cm_space *space, uint64_t first, uint64_t count,
                       const uint64_t *idx_dev, double *cost_dev, int64_t *cost_ns_dev, uint8_t *feasible_dev) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!space || space->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
-    if (count > (1ull << 40)) return fail(ctx, CM_EINVAL, "count too large");
+    // one thread per candidate, 128 per block, the block count a 31-bit grid dimension
+    if (count > 0x7fffffffull * 128ull) return fail(ctx, CM_EINVAL, "count too large: at most (2^31 - 1) * 128 candidates per call");
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
     Batch &bt = const_cast<Batch &>(space->batch);
+    if (stale(ctx, bt)) return fail(ctx, CM_EINVAL, kStaleMsg);
     const uint64_t n_cand = space->policy == CM_DYNPAR ? bt.n_cand : 1;
     if (!idx_dev && (first > n_cand || count > n_cand - first)) return fail(ctx, CM_EINVAL, "candidate range out of bounds");
     CM_CUDA(ctx, launch_evaluate(tables(ctx, bt), dev_view(ctx, bt), n_cand,
                                  space->policy == CM_DYNPAR ? -1 : space->policy, first, count, idx_dev,
                                  cost_dev, cost_ns_dev, feasible_dev, ctx->stream));
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_select(cm_ctx *ctx, cm_space *const *spaces, int32_t n_spaces, cm_plan *best) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!spaces || n_spaces < 1 || n_spaces > 64 || !best) return fail(ctx, CM_EINVAL, "bad arguments");
     for (int i = 0; i < n_spaces; ++i) {
         if (!spaces[i] || spaces[i]->ctx != ctx) return fail(ctx, CM_EINVAL, "space does not belong to this context");
+        if (stale(ctx, spaces[i]->batch)) return fail(ctx, CM_EINVAL, kStaleMsg);
         if (spaces[i]->batch.opts.cost != spaces[0]->batch.opts.cost) return fail(ctx, CM_EINVAL, "spaces mix cost modes");
     }
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
@@ -1138,29 +1177,30 @@ cm_status cm_select(cm_ctx *ctx, cm_space *const *spaces, int32_t n_spaces, cm_p
         if (s != CM_OK) return s;
         ptrs[i] = spaces[i]->batch.d_plans.p + spaces[i]->policy;
     }
-    // best over the spaces, on the device as well
-    const cm_plan **d_ptrs = nullptr;
-    cm_plan *d_out = nullptr;
-    CM_CUDA(ctx, cudaMalloc((void **)&d_ptrs, sizeof(cm_plan *) * n_spaces + sizeof(cm_plan)));
-    d_out = (cm_plan *)(d_ptrs + n_spaces);
+    // best over the spaces, on the device as well (scratch of the context: 64 pointers and a plan
+    // were reserved by cm_create, so this call allocates nothing)
+    if (!ctx->d_scratch.reserve(sizeof(cm_plan *) * 64 + sizeof(cm_plan))) return fail(ctx, CM_ENOMEM, "device memory");
+    const cm_plan **d_ptrs = reinterpret_cast<const cm_plan **>(ctx->d_scratch.p);
+    cm_plan *d_out = reinterpret_cast<cm_plan *>(ctx->d_scratch.p + sizeof(cm_plan *) * 64);
     cm_plan result;
     cudaError_t e = cudaMemcpyAsync(d_ptrs, ptrs.data(), sizeof(cm_plan *) * n_spaces, cudaMemcpyHostToDevice, ctx->stream);
     if (e == cudaSuccess) e = launch_pick(d_ptrs, n_spaces, d_out, mode, ctx->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(&result, d_out, sizeof(cm_plan), cudaMemcpyDeviceToHost, ctx->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
-    cudaFree(d_ptrs);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
     ctx->stats[3] += 1;
     scrub(result);
     *best = result;
     if (!result.feasible) return fail(ctx, CM_ENOFEASIBLE, "no feasible plan in the given spaces");
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
                           const cm_enum_opts *opts, cm_plan *best_per_scenario, cm_plan *best_per_policy,
                           float *latency_us) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (B < 0 || !offsets || !best_per_scenario || (offsets[B] > 0 && !failed_ids)) return fail(ctx, CM_EINVAL, "bad arguments");
     cm_status s = check_opts(ctx, opts);
@@ -1211,6 +1251,7 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         latency_us[b] = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
     }
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
@@ -1218,6 +1259,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
                               cm_plan *best, cm_transition *trans, cm_plan *shortlist, int64_t *shortlist_bytes,
                               int32_t *shortlist_rounds) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (B < 0 || !offsets || !best || !trans || !objective || (offsets[B] > 0 && !failed_ids))
         return fail(ctx, CM_EINVAL, "bad arguments");
@@ -1334,6 +1376,7 @@ cm_status cm_search_objective(cm_ctx *ctx, const uint32_t *failed_ids, const int
     }
     ctx->obj_stats[4] = solved;
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_set_int64_arithmetic(cm_ctx *ctx, int native) {
@@ -1358,6 +1401,17 @@ cm_status cm_set_sharing(cm_ctx *ctx, int on) {
     return CM_OK;
 }
 
+cm_status cm_transition_time(const cm_objective_opts *objective, int32_t n, const int64_t *xfer_bytes,
+                             double *t_trans_ns, int64_t *t_trans_ns_i) {
+    if (!objective || n < 0 || (n > 0 && !xfer_bytes) || objective->bw_xfer_Bpns <= 0) return CM_EINVAL;
+    for (int i = 0; i < n; ++i) {
+        const bool used = xfer_bytes[i] >= 0;   // -1 marks an empty shortlist slot
+        if (t_trans_ns) t_trans_ns[i] = used ? transition_time_f64(objective->t_restart_ns, xfer_bytes[i], objective->bw_xfer_Bpns) : -1.0;
+        if (t_trans_ns_i) t_trans_ns_i[i] = used ? transition_time_i64(objective->t_restart_ns_i, xfer_bytes[i], objective->bw_xfer_Bpns) : -1;
+    }
+    return CM_OK;
+}
+
 cm_status cm_objective_stats(const cm_ctx *ctx, uint64_t out[8]) {
     if (!ctx || !out) return CM_EINVAL;
     memcpy(out, ctx->obj_stats, sizeof(ctx->obj_stats));
@@ -1368,6 +1422,7 @@ cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *s
                                const uint8_t *old_hi, const uint8_t *new_lo, const uint8_t *new_hi,
                                int64_t *total, uint16_t *assign) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (n_problems < 0 || (n_problems > 0 && (!sizes || !old_lo || !old_hi || !new_lo || !new_hi || !total)))
         return fail(ctx, CM_EINVAL, "bad arguments");
@@ -1385,8 +1440,10 @@ cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *s
     const size_t off_sizes = 0, off_rng = ((size_t)n_problems * sizeof(int32_t) + 15) & ~(size_t)15;
     const size_t off_total = (off_rng + 4 * rows + 15) & ~(size_t)15, off_assign = off_total + (size_t)n_problems * sizeof(int64_t);
     const size_t bytes = off_assign + rows * sizeof(uint16_t);
-    unsigned char *d = nullptr;
-    CM_CUDA(ctx, cudaMalloc((void **)&d, bytes));
+    // scratch of the context: allocated when a call needs more than any call before it, kept afterwards
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // growing frees the old block: nothing may still use it
+    if (!ctx->d_scratch.reserve(bytes)) return fail(ctx, CM_ENOMEM, "device memory");
+    unsigned char *d = ctx->d_scratch.p;
     cudaStream_t st = ctx->stream;
     cudaError_t e = cudaMemcpyAsync(d + off_sizes, sizes, (size_t)n_problems * sizeof(int32_t), cudaMemcpyHostToDevice, st);
     const uint8_t *src[4] = {old_lo, old_hi, new_lo, new_hi};
@@ -1399,22 +1456,23 @@ cm_status cm_transfer_matching(cm_ctx *ctx, int32_t n_problems, const int32_t *s
     if (e == cudaSuccess) e = cudaMemcpyAsync(total, d + off_total, (size_t)n_problems * sizeof(int64_t), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && assign) e = cudaMemcpyAsync(assign, d + off_assign, rows * sizeof(uint16_t), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    cudaFree(d);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
     for (int q = 0; q < n_problems; ++q)
         if (total[q] < 0) return fail(ctx, CM_ECUDA, "matching iteration did not terminate");
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_batch_prepare(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t *offsets, int32_t B,
                            const cm_enum_opts *opts, cm_batch **out, uint64_t *n_candidates) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!ctx->has_profile) return fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (B < 0 || !offsets || !out || (offsets[B] > 0 && !failed_ids)) return fail(ctx, CM_EINVAL, "bad arguments");
     cm_status s = check_opts(ctx, opts);
     if (s != CM_OK) return s;
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
-    cm_batch *bp = new (std::nothrow) cm_batch();
+    std::unique_ptr<cm_batch> bp(new (std::nothrow) cm_batch());
     if (!bp) return fail(ctx, CM_ENOMEM, "host memory");
     bp->ctx = ctx;
     memset(ctx->stats, 0, sizeof(ctx->stats));
@@ -1424,17 +1482,19 @@ cm_status cm_batch_prepare(cm_ctx *ctx, const uint32_t *failed_ids, const int32_
     if (s != CM_OK) {
         cudaStreamSynchronize(ctx->stream);
         forget_keys(ctx, bp->batch);
-        delete bp;
         return s;
     }
-    *out = bp;
     if (n_candidates) *n_candidates = bp->batch.n_cand;
+    *out = bp.release();
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_batch_search(cm_ctx *ctx, cm_batch *bp, cm_plan *best_per_scenario, cm_plan *best_per_policy) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!bp || bp->ctx != ctx || !best_per_scenario) return fail(ctx, CM_EINVAL, "bad arguments");
+    if (stale(ctx, bp->batch)) return fail(ctx, CM_EINVAL, kStaleMsg);
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
     memset(ctx->stats, 0, sizeof(ctx->stats));
     Batch &bt = bp->batch;
@@ -1452,6 +1512,7 @@ cm_status cm_batch_search(cm_ctx *ctx, cm_batch *bp, cm_plan *best_per_scenario,
         best_per_scenario[b] = pl;
     }
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_batch_free(cm_batch *bp) {
@@ -1462,7 +1523,7 @@ cm_status cm_batch_free(cm_batch *bp) {
     return CM_OK;
 }
 
-cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]) {
+cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[24]) {
     if (!ctx || !out) return CM_EINVAL;
     memcpy(out, ctx->stats, sizeof(ctx->stats));
     return CM_OK;
@@ -1470,7 +1531,9 @@ cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[16]) {
 
 cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan, int32_t *cuts_out) {
     if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
     if (!space || space->ctx != ctx || !plan || !cuts_out) return fail(ctx, CM_EINVAL, "bad arguments");
+    if (stale(ctx, space->batch)) return fail(ctx, CM_EINVAL, kStaleMsg);
     if (plan->policy != space->policy) return fail(ctx, CM_EINVAL, "plan was not found in this space");
     const DevProfile &hp = ctx->hp;
     CM_CUDA(ctx, cudaSetDevice(ctx->device));
@@ -1540,6 +1603,7 @@ cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan
     }
     memcpy(cuts_out, cuts.data(), cuts.size() * sizeof(int32_t));
     return CM_OK;
+    CM_API_END(ctx)
 }
 
 }  // extern "C"

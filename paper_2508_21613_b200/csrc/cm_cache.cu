@@ -8,6 +8,7 @@
 // those sets, a few thousand at a time; this file only enumerates and indexes them and uses
 // the library's public entry points.
 #include <algorithm>
+#include <memory>
 #include <new>
 #include <vector>
 
@@ -55,8 +56,11 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
     if (n_devices < 1) return cm_internal_fail(ctx, CM_ENOPROFILE, "cm_load_profile first");
     if (max_failures < 0 || max_failures > 16 || max_failures > n_devices)
         return cm_internal_fail(ctx, CM_EINVAL, "max_failures must be 0 .. min(16, devices)");
-    cm_cache *c = new (std::nothrow) cm_cache();
-    if (!c) return CM_ENOMEM;
+    // the tables and the plan array below can be large (up to 2^20 sets x 4 plans): an allocation
+    // failure must come back as a status, not unwind through the C ABI
+    try {
+    std::unique_ptr<cm_cache> c(new (std::nothrow) cm_cache());
+    if (!c) return cm_internal_fail(ctx, CM_ENOMEM, "host memory");
     c->ctx = ctx;
     c->n_devices = n_devices;
     c->max_failures = max_failures;
@@ -76,10 +80,8 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
     c->offset.assign(K + 2, 0);
     for (int s = 0; s <= K; ++s) {
         const uint64_t cnt = c->choose(n_devices, s);
-        if (cnt > kMaxEntries || c->offset[s] + cnt > kMaxEntries) {
-            delete c;
+        if (cnt > kMaxEntries || c->offset[s] + cnt > kMaxEntries)
             return cm_internal_fail(ctx, CM_EOVERFLOW, "more than 2^20 failure sets");
-        }
         c->offset[s + 1] = c->offset[s] + cnt;
     }
     const uint64_t total = c->offset[K + 1];
@@ -89,7 +91,10 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
     std::vector<cm_plan> best(kBatch), pol((size_t)kBatch * 3);
     // failure sets that leave the same number of survivors with the same node boundaries have
     // the same dynamic-parallelism search: let the batches share it
-    const int sharing_before = cm_internal_set_sharing(ctx, 1);
+    struct Sharing {   // restored on every way out
+        cm_ctx *ctx; int before;
+        ~Sharing() { cm_internal_set_sharing(ctx, before); }
+    } sharing{ctx, cm_internal_set_sharing(ctx, 1)};
     for (int s = 0; s <= K; ++s) {
         const uint64_t cnt = c->choose(n_devices, s);
         for (uint64_t first = 0; first < cnt; first += kBatch) {
@@ -101,7 +106,7 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
                 offsets[b + 1] = (b + 1) * s;
             }
             cm_status st = cm_search_batch(ctx, ids.data(), offsets.data(), B, opts, best.data(), pol.data(), nullptr);
-            if (st != CM_OK) { cm_internal_set_sharing(ctx, sharing_before); delete c; return st; }
+            if (st != CM_OK) return st;
             for (int b = 0; b < B; ++b) {
                 cm_plan *dst = c->plans.data() + (size_t)(c->offset[s] + first + b) * 4;
                 for (int q = 0; q < 3; ++q) dst[q] = pol[(size_t)b * 3 + q];
@@ -109,10 +114,14 @@ cm_status cm_cache_build(cm_ctx *ctx, int32_t max_failures, const cm_enum_opts *
             }
         }
     }
-    cm_internal_set_sharing(ctx, sharing_before);
-    *out = c;
     if (n_scenarios) *n_scenarios = total;
+    *out = c.release();
     return CM_OK;
+    } catch (const std::bad_alloc &) {
+        return CM_ENOMEM;
+    } catch (...) {
+        return CM_EINVAL;
+    }
 }
 
 cm_status cm_cache_lookup(const cm_cache *c, const uint32_t *failed_ids, int32_t n_failed, cm_plan *best,

@@ -22,10 +22,11 @@
 //   cm_cost_generic_kernel<T>       any S <= CM_MAX_STAGES: per-stage state in local memory.
 #pragma once
 
+#include <atomic>
+
 #include "cm_plan_eval.cuh"
 
 namespace cm {
-
 
 // Bucket that owns a chunk: the last bucket of the class whose first chunk is not above it.
 __device__ __forceinline__ uint32_t find_bucket(const Bucket *bk, uint32_t b0, uint32_t b1, uint64_t chunk) {
@@ -78,15 +79,26 @@ __device__ __forceinline__ void segmented_min_commit(uint64_t *seg_best, uint32_
     if (last && row != 0xffffffffu && bits < inf) atomicMin((unsigned long long *)&seg_best[row], (unsigned long long)bits);
 }
 
-__device__ __forceinline__ void count_cells(unsigned long long *counter, unsigned long long my_cells,
+// Work counters of the search pass: recurrence cells simulated and plans whose recurrence ran
+// (the memory-feasible ones).  A thread reports both in one word -- cells in the low 40 bits,
+// plans above -- so that one shuffle reduction serves both; counters[0] takes the cells,
+// counters[2] the plans.
+constexpr int kWorkPlanShift = 40;
+__device__ __forceinline__ unsigned long long one_plan(unsigned long long cells) { return cells + (1ull << kWorkPlanShift); }
+__device__ __forceinline__ void add_work(unsigned long long *counters, unsigned long long packed) {
+    if (!packed) return;
+    atomicAdd(&counters[0], packed & ((1ull << kWorkPlanShift) - 1ull));
+    atomicAdd(&counters[2], packed >> kWorkPlanShift);
+}
+__device__ __forceinline__ void count_cells(unsigned long long *counters, unsigned long long my_work,
                                             unsigned long long *smem /* [kChunk/32] */) {
-    for (int o = 16; o > 0; o >>= 1) my_cells += __shfl_xor_sync(0xffffffffu, my_cells, o);
-    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = my_cells;
+    for (int o = 16; o > 0; o >>= 1) my_work += __shfl_xor_sync(0xffffffffu, my_work, o);
+    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = my_work;
     __syncthreads();
     if (threadIdx.x == 0) {
         unsigned long long c = 0;
         for (int w = 0; w < kChunk / 32; ++w) c += smem[w];
-        if (c) atomicAdd(counter, c);
+        add_work(counters, c);
     }
 }
 
@@ -114,7 +126,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
         T cost;
         if (plan_cost_regs<T, S>(sp, tb, bd.layer_mode, g, kappa, cost)) {
             bits = Num<T>::bits(cost);
-            my_cells = 2ull * S * g.m;
+            my_cells = one_plan(2ull * S * g.m);
         }
     }
     segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
@@ -143,7 +155,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, Bat
         T cost;
         if (plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost)) {
             bits = Num<T>::bits(cost);
-            my_cells = 2ull * g.S * g.m;
+            my_cells = one_plan(2ull * g.S * g.m);
         }
     }
     segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
@@ -255,7 +267,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
                         if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
                     }
                     const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, active));
-                    if (lane == 0) cells_w[warp] += 2ull * S * m * n_active;
+                    if (lane == 0) cells_w[warp] += one_plan(2ull * S * m) * n_active;
                     __syncwarp();   // the next item overwrites the stage times and cuts
                 }
             }
@@ -263,7 +275,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
             if (tid == 0) {
                 unsigned long long c = 0;
                 for (int w = 0; w < kChunk / 32; ++w) c += cells_w[w];
-                if (c) atomicAdd(&bd.counters[0], c);
+                add_work(bd.counters, c);
             }
             return;
         } else {
@@ -322,7 +334,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
                     if (active) {
                         const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval));
                         if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
-                        my_cells = 2ull * S * m;
+                        my_cells = one_plan(2ull * S * m);
                     }
                 }
             }
@@ -341,7 +353,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
             T cost;
             if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost)) {
                 bits = Num<T>::bits(cost);
-                my_cells = 2ull * S * m;
+                my_cells = one_plan(2ull * S * m);
             }
         }
         segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
@@ -369,7 +381,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, Batc
         T cost;
         if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
             bits = Num<T>::bits(cost);
-            my_cells = 2ull * g.S * g.m;
+            my_cells = one_plan(2ull * g.S * g.m);
         }
     }
     segmented_min_commit(bd.seg_best, row, bits, inf_bits<T>());
@@ -391,13 +403,16 @@ static cudaError_t launch_regs(const Tables &t, const BatchDev &b, const LaunchC
 template <typename T, int S, bool UNI>
 static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
     constexpr size_t smem = wide_smem_bytes<S, UNI, T>();
-    static bool configured[16] = {false};   // per device; the attribute sticks to the function
+    // One bit per device: the attribute sticks to the function on that device.  Setting it is
+    // idempotent, so two host threads (distinct contexts) that both find the bit clear both set
+    // it; the bit itself is atomic.
+    static std::atomic<uint64_t> configured{0};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev < 16 && !configured[dev]) {
+    if (dev >= 64 || !((configured.load(std::memory_order_acquire) >> dev) & 1ull)) {
         cudaError_t e = cudaFuncSetAttribute(cm_cost_wide_kernel<T, S, UNI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
     }
     cm_cost_wide_kernel<T, S, UNI><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin, (int)c.uni_items);
     return cudaGetLastError();
@@ -504,13 +519,13 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_w
 template <typename T, int S>
 static cudaError_t launch_tiebreak_wide_one(const Tables &t, const BatchDev &b, cudaStream_t st) {
     constexpr size_t smem = wide_smem_bytes<S, false, T>();
-    static bool configured[16] = {false};
+    static std::atomic<uint64_t> configured{0};   // as in launch_wide_one
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev < 16 && !configured[dev]) {
+    if (dev >= 64 || !((configured.load(std::memory_order_acquire) >> dev) & 1ull)) {
         cudaError_t e = cudaFuncSetAttribute(cm_tiebreak_wide_kernel<T, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
     }
     const uint64_t nx = (uint64_t)b.B * b.dp_max;
     if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;

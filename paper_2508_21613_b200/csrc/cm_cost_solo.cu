@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_solo_kernel(Tables tb, BatchDe
             if (lane == 0) {
                 const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval));
                 if (bits < bd.seg_best[g.row]) atomicMin((unsigned long long *)&bd.seg_best[g.row], (unsigned long long)bits);
-                my_cells = 2ull * S * m;
+                my_cells = one_plan(2ull * S * m);
             }
         }
     }

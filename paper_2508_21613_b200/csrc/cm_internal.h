@@ -195,6 +195,16 @@ struct ObjDev {
     cm_transition *trans;     // [B]
 };
 
+// Transition time of a reconstruction that moves `bytes` of model state (Section "Estimator",
+// state-transition overhead: restart + weight transfer; the search itself overlaps training).
+// One routine for the objective kernel and for cm_transition_time on the host.
+__host__ __device__ inline double transition_time_f64(double t_restart, long long bytes, long long bw) {
+    return t_restart + (double)bytes / (double)bw;
+}
+__host__ __device__ inline long long transition_time_i64(long long t_restart, long long bytes, long long bw) {
+    return t_restart + bytes / bw;
+}
+
 // Integer-nanosecond mode runs the long long instantiations unless the batch evaluates it in
 // double arithmetic on integer-valued inputs (BatchDev::intval).
 inline bool native_i64(const BatchDev &b) { return b.mode == CM_COST_INT64NS && !b.intval; }

@@ -130,6 +130,7 @@ extern "C" cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *spa
                                                 double *best_cost_dev, int64_t *best_cost_ns_dev,
                                                 uint64_t *best_index_dev) {
     if (!ctx) return CM_EINVAL;
+    try {   // the error paths below build std::string messages
     SpaceView v;
     cm_status s = cm_internal_space_view(ctx, space, &v);
     if (s != CM_OK) return s;
@@ -153,4 +154,7 @@ extern "C" cm_status cm_evaluate_argmin_noalloc(cm_ctx *ctx, const cm_space *spa
     e = cudaGetLastError();
     if (e != cudaSuccess) return cm_internal_fail(ctx, CM_ECUDA, cudaGetErrorString(e));
     return CM_OK;
+    } catch (...) {
+        return CM_ENOMEM;
+    }
 }

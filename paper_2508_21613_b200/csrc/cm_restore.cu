@@ -509,11 +509,11 @@ __global__ void __launch_bounds__(32) cm_objective_kernel(Tables tb, BatchDev bd
             double tt = 0.0;
             long long tti = 0;
             if (mode == CM_COST_INT64NS) {
-                tti = od.t_restart_i + bytes / od.bw_xfer;
+                tti = transition_time_i64(od.t_restart_i, bytes, od.bw_xfer);
                 j.ni = od.t_gap_i - tti;
                 j.di = batch_cost_ns(bd, step);
             } else {
-                tt = od.t_restart + (double)bytes / (double)od.bw_xfer;
+                tt = transition_time_f64(od.t_restart, bytes, od.bw_xfer);
                 j.nd = od.t_gap - tt;
                 j.dd = __longlong_as_double((long long)step);
             }

@@ -114,14 +114,14 @@ def gpu_planner(binding, ctx, opts, objective):
         mode = opts.cost_mode
         cost = lambda p: float(p.cost_ns if mode else p.cost)
         out = []
-        k = objective.topk
+        # the library prices the least-step-time reconfiguration (shortlist rank 0) itself
+        t_f64, t_i64 = binding.cm_transition_time(objective, sb[:, 0])
         for b in range(len(sets)):
             per = [pol[3 * b + q] for q in range(3)]
             step = tuple(cost(p) if p.feasible else None for p in per)
             dyn_trans = 0.0
             if sb[b, 0] >= 0:
-                t_xfer = (int(sb[b, 0]) // objective.bw_xfer_Bpns) if mode else float(int(sb[b, 0])) / float(objective.bw_xfer_Bpns)
-                dyn_trans = float(objective.t_restart_ns) + t_xfer
+                dyn_trans = float(t_i64[b] if mode else t_f64[b])
             tr = trans[b]
             chosen = None
             if tr.feasible:

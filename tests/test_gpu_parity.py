@@ -526,3 +526,37 @@ def test_handworked_readings_rerouting_redundant_memory_minmax_ties(gpu, oracle_
                 gpu.cm_space_free(space)
             finally:
                 s.close()
+
+
+def test_spaces_and_batches_of_an_earlier_profile_are_refused(gpu):
+    """A space or prepared batch describes the L, G and min-max partitions of the profile it was
+    built under; after cm_load_profile replaces that profile every call that takes it must fail
+    with CM_EINVAL instead of evaluating old descriptors against new tables."""
+    import torch
+    big, small = W.paper_scale(0, 0), W.tiny()
+    s = Session(gpu, big.profile)
+    try:
+        space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [3], big.options)
+        packed = gpu.PackedScenarios([[3], [4, 9]])
+        batch, _ = packed.prepare(s.ctx, big.options)
+        plan = gpu.cm_select(s.ctx, [space])
+        assert plan.feasible
+        gpu.cm_load_profile(s.ctx, small.profile)          # fewer layers, fewer micro-batches
+        cost = torch.zeros(16, dtype=torch.float64, device="cuda")
+        calls = [lambda: gpu.cm_evaluate(s.ctx, space, 0, 16, None, cost, None, None),
+                 lambda: gpu.cm_select(s.ctx, [space]),
+                 lambda: gpu.cm_decode_plan(s.ctx, space, plan),
+                 lambda: gpu.cm_evaluate_argmin_noalloc(s.ctx, space, 0, 16, cost, None, None),
+                 lambda: packed.search_prepared(s.ctx, batch)]
+        for call in calls:
+            with pytest.raises(gpu.ChameleonError) as e:
+                call()
+            assert e.value.status == gpu.CM_EINVAL and "earlier profile" in str(e.value)
+        gpu.cm_space_free(space)
+        gpu.cm_batch_free(batch)
+        # the context itself is fine: a space enumerated under the new profile works
+        space, n = gpu.cm_enumerate(s.ctx, W.POLICY_DYNPAR, [1], small.options)
+        assert gpu.cm_select(s.ctx, [space]).feasible
+        gpu.cm_space_free(space)
+    finally:
+        s.close()

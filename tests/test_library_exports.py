@@ -28,6 +28,25 @@ def test_every_declared_entry_point_is_exported(lib_path):
     assert set(binding.EXPORTS) == declared
 
 
+def test_binding_constants_match_the_header():
+    from paper_2508_21613_b200 import binding
+    header = open(os.path.join(ROOT, "include", "chameleon.h")).read()
+    defines = {k: int(v) for k, v in re.findall(r"#define\s+(CM_[A-Z_]+)\s+(\d+)", header)}
+    assert binding.NOALLOC_MAX_CANDIDATES == defines["CM_NOALLOC_MAX_CANDIDATES"]
+    assert (binding.MAX_PIPES, binding.MAX_STAGES, binding.MAX_LAYERS) == (
+        defines["CM_MAX_PIPES"], defines["CM_MAX_STAGES"], defines["CM_MAX_LAYERS"])
+    assert (binding.MAX_SHORTLIST, binding.MAX_MATCH) == (defines["CM_MAX_SHORTLIST"], defines["CM_MAX_MATCH"])
+
+
+def test_transition_time_needs_no_device(lib_path):
+    """cm_transition_time is host arithmetic: restart + bytes / bandwidth, floored in integer mode."""
+    from paper_2508_21613_b200 import binding, workloads as W
+    obj = W.ObjectiveOptions(t_restart_ns=5e9, bw_xfer_Bpns=25)
+    t, ti = binding.cm_transition_time(obj, [0, 1000, 1012, -1])
+    assert list(t) == [5e9, 5e9 + 40.0, 5e9 + 1012 / 25, -1.0]
+    assert list(ti) == [5 * 10**9, 5 * 10**9 + 40, 5 * 10**9 + 40, -1]
+
+
 def test_struct_layouts_match_the_header():
     from paper_2508_21613_b200 import binding
     assert ctypes.sizeof(binding.cm_plan) == 8 + 8 + 8 + 8 + 8 + 32 + 32 + 128
