@@ -7,20 +7,43 @@ namespace cm {
 template <typename T> cudaError_t launch_shallow_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 template <typename T> cudaError_t launch_shallow_any(const Tables &, const BatchDev &, uint32_t, uint32_t, uint64_t, cudaStream_t);
 template <typename T> cudaError_t launch_generic_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
-template <typename T> cudaError_t launch_deep_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
-template <typename T> cudaError_t launch_tiebreak_deep(const Tables &, const BatchDev &, int, cudaStream_t);
+template <typename T, int LO, int HI> cudaError_t launch_deep_range(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
+template <typename T, int LO, int HI> cudaError_t launch_tiebreak_range(const Tables &, const BatchDev &, int, cudaStream_t);
 template <typename T> cudaError_t launch_solo_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 
 #define CM_EXTERN(T)                                                                                                   \
     extern template cudaError_t launch_shallow_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
     extern template cudaError_t launch_shallow_any<T>(const Tables &, const BatchDev &, uint32_t, uint32_t, uint64_t, cudaStream_t); \
     extern template cudaError_t launch_generic_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
-    extern template cudaError_t launch_deep_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);    \
-    extern template cudaError_t launch_tiebreak_deep<T>(const Tables &, const BatchDev &, int, cudaStream_t);  \
     extern template cudaError_t launch_solo_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 CM_EXTERN(double)
 CM_EXTERN(long long)
 #undef CM_EXTERN
+
+// the deep-pipeline kernels: one translation unit per cost type and range of stage counts
+#define CM_DEEP_RANGE(LO, HI)                                                                                                     \
+    extern template cudaError_t launch_deep_range<double, LO, HI>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
+    extern template cudaError_t launch_deep_range<long long, LO, HI>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
+    extern template cudaError_t launch_tiebreak_range<double, LO, HI>(const Tables &, const BatchDev &, int, cudaStream_t);         \
+    extern template cudaError_t launch_tiebreak_range<long long, LO, HI>(const Tables &, const BatchDev &, int, cudaStream_t);
+CM_DEEP_RANGES(CM_DEEP_RANGE)
+#undef CM_DEEP_RANGE
+
+template <typename T>
+static cudaError_t launch_deep_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+#define CM_DEEP_RANGE(LO, HI) if (c.stages >= LO && c.stages <= HI) return launch_deep_range<T, LO, HI>(t, b, c, st);
+    CM_DEEP_RANGES(CM_DEEP_RANGE)
+#undef CM_DEEP_RANGE
+    return cudaErrorInvalidValue;
+}
+
+template <typename T>
+static cudaError_t launch_tiebreak_deep(const Tables &t, const BatchDev &b, int S, cudaStream_t st) {
+#define CM_DEEP_RANGE(LO, HI) if (S >= LO && S <= HI) return launch_tiebreak_range<T, LO, HI>(t, b, S, st);
+    CM_DEEP_RANGES(CM_DEEP_RANGE)
+#undef CM_DEEP_RANGE
+    return cudaSuccess;
+}
 
 template <typename T>
 static cudaError_t launch_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {

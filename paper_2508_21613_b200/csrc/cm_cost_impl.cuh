@@ -179,6 +179,47 @@ template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
                : sizeof(FB<T>) * S * kChunk + sizeof(T) * S * kChunk;
 }
 
+// Transposed kernel, per warp item: the layer composition kappa of an (S, m) bucket is the same
+// in all 32 segments the warp evaluates, so its cuts, stage times and memory check are worked
+// out once per warp -- every lane walks the cuts (lane 0 keeps them in `cuts`), then the stages
+// are shared out over the lanes for the sums and the check.  Returns, warp-uniform, whether
+// the composition is feasible; g_max = largest gradient bytes of a stage (in every lane).
+template <typename T, int S>
+__device__ __forceinline__ bool uni_composition(const SProf<T> &sp, const Tables &tb, int layer_mode, int m, uint64_t kappa,
+                                                uint64_t K, FB<T> *fb, uint8_t *cuts, uint32_t lane, long long &g_max) {
+    CutWalker cw;
+    bool ok = make_walker(cw, tb, layer_mode, sp.L, S, kappa, K, tb.mm_slot(S, m));
+    if (ok) {
+        int lo = 0;
+        for (int i = 0; i < S; ++i) {
+            const int hi = cw.next();
+            ok = ok && hi > lo;
+            if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+            lo = hi;
+        }
+        if (lane == 0) cuts[0] = 0;
+    }
+    __syncwarp();
+    g_max = 0;
+    if (ok) {
+        for (int i = lane; i < S; i += 32) {
+            const int lo = cuts[i], hi = cuts[i + 1];
+            ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+            FB<T> d;
+            d.f = sp.PF[hi] - sp.PF[lo];
+            d.b = sp.PB[hi] - sp.PB[lo];
+            fb[i] = d;
+            const long long gb = sp.PP[hi] - sp.PP[lo];
+            g_max = gb > g_max ? gb : g_max;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+            g_max = og > g_max ? og : g_max;
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
 template <typename T, int S, bool UNI>
 __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset, int uni_items) {
     __shared__ SProf<T> sp;
@@ -188,157 +229,67 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
     stage_profile(sp, tb.prof);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
-    const int m = bk.m, L = sp.L;
+    const int m = bk.m;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     unsigned long long my_cells = 0;
 
     if (UNI) {
-        if (S <= CM_UNI_BATCH_STAGES) {
-            // warp item = (kappa, group of 32 segments), group minor; a warp takes uni_items
-            // consecutive items, so that the CTA's fixed cost (staging the profile) is spread over
-            // more work and a composition shared by consecutive groups is unranked, summed and
-            // checked against memory only once.  Everything an item needs from the previous one
-            // lives in shared memory: nothing but the loop counter stays in registers across the
-            // recurrence, whose per-stage state needs nearly all of them.
-            __shared__ Bucket bks;
-            __shared__ unsigned long long st_kappa[kChunk / 32];
-            __shared__ long long st_gmax[kChunk / 32];
-            __shared__ int st_ok[kChunk / 32];
-            if (tid == 0) bks = bk;
-            if (lane == 0) { st_kappa[warp] = ~0ull; st_ok[warp] = 0; st_gmax[warp] = 0; cells_w[warp] = 0; }
-            __syncthreads();
-            for (int r = 0; r < uni_items; ++r) {
-                FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
-                T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
-                uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
-                const uint64_t item = ((chunk - bks.chunk_first) * (kChunk / 32) + warp) * (uint64_t)uni_items + r;
-                const uint32_t n_groups = (bks.n_seg + 31) / 32;
-                const uint64_t kappa = item / n_groups;
-                if (kappa >= bks.count || m < 1) break;            // warp-uniform; items ascend
-                const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
-                const bool active = seg_local < bks.n_seg;
-                const SegView g = bucket_segment(bd, bks, active ? seg_local : 0);
-                if (kappa != st_kappa[warp]) {
-                    // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
-                    CutWalker cw;
-                    bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
-                    if (ok) {
-                        int lo = 0;
-                        for (int i = 0; i < S; ++i) {
-                            const int hi = cw.next();
-                            ok = ok && hi > lo;
-                            if (lane == 0) cuts[i + 1] = (uint8_t)hi;
-                            lo = hi;
-                        }
-                        if (lane == 0) cuts[0] = 0;
-                    }
-                    __syncwarp();
-                    long long g_max = 0;
-                    if (ok) {
-                        // stage sums and the memory check, one stage per lane
-                        for (int i = lane; i < S; i += 32) {
-                            const int lo = cuts[i], hi = cuts[i + 1];
-                            ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-                            FB<T> d;
-                            d.f = sp.PF[hi] - sp.PF[lo];
-                            d.b = sp.PB[hi] - sp.PB[lo];
-                            fb[i] = d;
-                            const long long gb = sp.PP[hi] - sp.PP[lo];
-                            g_max = gb > g_max ? gb : g_max;
-                        }
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
-                            g_max = og > g_max ? og : g_max;
-                        }
-                    }
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (lane == 0) { st_kappa[warp] = kappa; st_ok[warp] = ok ? 1 : 0; st_gmax[warp] = g_max; }
-                    __syncwarp();
-                }
-                if (st_ok[warp]) {
-                    // transfer times of this lane's segment (its own link tiers)
-                    for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(g.tier >> i) & 1ull][cuts[i + 1] - 1];
-                    const uint32_t row = g.row;
-                    const int n_sync = g.n_sync;
-                    __syncwarp();
-                    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-                    if (active) {
-                        const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], n_sync, sp.bw_sync, sp.intval));
-                        if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
-                    }
-                    const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, active));
-                    if (lane == 0) cells_w[warp] += one_plan(2ull * S * m) * n_active;
-                    __syncwarp();   // the next item overwrites the stage times and cuts
-                }
-            }
-            __syncthreads();
-            if (tid == 0) {
-                unsigned long long c = 0;
-                for (int w = 0; w < kChunk / 32; ++w) c += cells_w[w];
-                add_work(bd.counters, c);
-            }
-            return;
-        } else {
-            FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
-            T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
-            uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (S + 1);
-            // warp item = (kappa, group of 32 segments), group minor
-            const uint64_t item = (chunk - bk.chunk_first) * (kChunk / 32) + warp;
-            const uint32_t n_groups = (bk.n_seg + 31) / 32;
+        // warp item = (kappa, group of 32 segments), group minor.  Up to CM_UNI_BATCH_STAGES a warp
+        // takes uni_items consecutive items, so that the CTA's fixed cost (staging the profile) is
+        // spread over more work and a composition shared by consecutive groups is set up only
+        // once; everything an item needs from the previous one lives in shared memory -- nothing
+        // but the loop counter stays in registers across the recurrence, whose per-stage state
+        // needs nearly all of them.  Deeper pipelines keep one item per warp.
+        constexpr bool kBatch = S <= CM_UNI_BATCH_STAGES;
+        __shared__ Bucket bks;
+        __shared__ unsigned long long st_kappa[kChunk / 32];
+        __shared__ long long st_gmax[kChunk / 32];
+        __shared__ int st_ok[kChunk / 32];
+        if (tid == 0) bks = bk;
+        if (lane == 0) { st_kappa[warp] = ~0ull; st_ok[warp] = 0; st_gmax[warp] = 0; cells_w[warp] = 0; }
+        __syncthreads();
+        FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+        T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+        uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (((S + 1) + 7) / 8 * 8);
+        const int n_items = kBatch ? uni_items : 1;
+        for (int r = 0; r < n_items; ++r) {
+            const uint64_t item = ((chunk - bks.chunk_first) * (kChunk / 32) + warp) * (uint64_t)n_items + r;
+            const uint32_t n_groups = (bks.n_seg + 31) / 32;
             const uint64_t kappa = item / n_groups;
+            if (kappa >= bks.count || m < 1) break;            // warp-uniform; items ascend
             const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
-            if (kappa < bk.count && m >= 1) {           // warp-uniform
-                const bool active = seg_local < bk.n_seg;
-                const SegView g = bucket_segment(bd, bk, active ? seg_local : 0);
+            const bool active = seg_local < bks.n_seg;
+            const SegView g = bucket_segment(bd, bks, active ? seg_local : 0);
+            if (kappa != st_kappa[warp]) {
+                long long g_max;
+                const bool ok = uni_composition<T, S>(sp, tb, bd.layer_mode, m, kappa, g.K, fb, cuts, lane, g_max);
+                if (lane == 0) { st_kappa[warp] = kappa; st_ok[warp] = ok ? 1 : 0; st_gmax[warp] = g_max; }
+                __syncwarp();
+            }
+            if (st_ok[warp]) {
+                // transfer times of this lane's segment (its own link tiers)
+                for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(g.tier >> i) & 1ull][cuts[i + 1] - 1];
                 const uint32_t row = g.row;
-                const uint64_t tier = g.tier;
                 const int n_sync = g.n_sync;
-                // cuts are a function of (S, m, kappa) only: every lane walks them, lane 0 keeps them
-                CutWalker cw;
-                bool ok = make_walker(cw, tb, bd.layer_mode, L, S, kappa, g.K, tb.mm_slot(S, m));
-                if (ok) {
-                    int lo = 0;
-                    for (int i = 0; i < S; ++i) {
-                        const int hi = cw.next();
-                        ok = ok && hi > lo;
-                        if (lane == 0) cuts[i + 1] = (uint8_t)hi;
-                        lo = hi;
-                    }
-                    if (lane == 0) cuts[0] = 0;
-                }
                 __syncwarp();
-                long long g_max = 0;
-                if (ok) {
-                    // stage sums and the memory check, one stage per lane
-                    for (int i = lane; i < S; i += 32) {
-                        const int lo = cuts[i], hi = cuts[i + 1];
-                        ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
-                        FB<T> d;
-                        d.f = sp.PF[hi] - sp.PF[lo];
-                        d.b = sp.PB[hi] - sp.PB[lo];
-                        fb[i] = d;
-                        const long long gb = sp.PP[hi] - sp.PP[lo];
-                        g_max = gb > g_max ? gb : g_max;
-                    }
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
-                        g_max = og > g_max ? og : g_max;
-                    }
-                    // transfer times of this lane's segment (its own link tiers)
-                    for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(tier >> i) & 1ull][cuts[i + 1] - 1];
+                const SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk> src{smem_addr(fb), smem_addr(xcol)};
+                const T t = sim_rounds<T, S>(m, src);
+                if (active) {
+                    const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], n_sync, sp.bw_sync, sp.intval));
+                    if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
                 }
-                ok = __all_sync(0xffffffffu, ok);
-                __syncwarp();
-                if (ok) {
-                    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fb + i); }, [&](int i) { return lds_t<T>(xcol + i * kChunk); });
-                    if (active) {
-                        const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval));
-                        if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
-                        my_cells = one_plan(2ull * S * m);
-                    }
-                }
+                const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, active));
+                if (lane == 0) cells_w[warp] += one_plan(2ull * S * m) * n_active;
+                __syncwarp();   // the next item overwrites the stage times and cuts
             }
         }
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long c = 0;
+            for (int w = 0; w < kChunk / 32; ++w) c += cells_w[w];
+            add_work(bd.counters, c);
+        }
+        return;
     } else {
         FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + tid;                               // [i * kChunk]
         T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + tid;           // [i * kChunk]
@@ -452,17 +403,18 @@ cudaError_t launch_generic_class(const Tables &t, const BatchDev &b, const Launc
     return cudaGetLastError();
 }
 
-template <typename T>
-cudaError_t launch_deep_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    switch (c.stages) {
-#define CM_CASE(S) case S: return launch_wide<T, S>(t, b, c, st);
-        CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
-        CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
-        CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
-        CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
-#undef CM_CASE
-    default: return cudaErrorInvalidValue;
-    }
+// Deep pipelines are instantiated per stage count; the stage counts LO .. HI of one cost type
+// form one translation unit (cm_cost_deep.cu, compiled once per range), so that the kernel
+// instantiations compile side by side.
+template <typename T, int S, int HI>
+static cudaError_t deep_dispatch(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    if (c.stages == S) return launch_wide<T, S>(t, b, c, st);
+    if constexpr (S < HI) return deep_dispatch<T, S + 1, HI>(t, b, c, st);
+    else return cudaErrorInvalidValue;
+}
+template <typename T, int LO, int HI>
+cudaError_t launch_deep_range(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    return deep_dispatch<T, LO, HI>(t, b, c, st);
 }
 
 // ----------------------------------------------------------------------------------
@@ -534,17 +486,15 @@ static cudaError_t launch_tiebreak_wide_one(const Tables &t, const BatchDev &b, 
     return cudaGetLastError();
 }
 
-template <typename T>
-cudaError_t launch_tiebreak_deep(const Tables &t, const BatchDev &b, int S, cudaStream_t st) {
-    switch (S) {
-#define CM_CASE(S) case S: return launch_tiebreak_wide_one<T, S>(t, b, st);
-        CM_CASE(17) CM_CASE(18) CM_CASE(19) CM_CASE(20) CM_CASE(21) CM_CASE(22) CM_CASE(23) CM_CASE(24)
-        CM_CASE(25) CM_CASE(26) CM_CASE(27) CM_CASE(28) CM_CASE(29) CM_CASE(30) CM_CASE(31) CM_CASE(32)
-        CM_CASE(33) CM_CASE(34) CM_CASE(35) CM_CASE(36) CM_CASE(37) CM_CASE(38) CM_CASE(39) CM_CASE(40)
-        CM_CASE(41) CM_CASE(42) CM_CASE(43) CM_CASE(44) CM_CASE(45) CM_CASE(46) CM_CASE(47) CM_CASE(48)
-#undef CM_CASE
-    default: return cudaSuccess;
-    }
+template <typename T, int S, int HI>
+static cudaError_t tiebreak_dispatch(const Tables &t, const BatchDev &b, int stages, cudaStream_t st) {
+    if (stages == S) return launch_tiebreak_wide_one<T, S>(t, b, st);
+    if constexpr (S < HI) return tiebreak_dispatch<T, S + 1, HI>(t, b, stages, st);
+    else return cudaSuccess;
+}
+template <typename T, int LO, int HI>
+cudaError_t launch_tiebreak_range(const Tables &t, const BatchDev &b, int S, cudaStream_t st) {
+    return tiebreak_dispatch<T, LO, HI>(t, b, S, st);
 }
 
 }  // namespace cm

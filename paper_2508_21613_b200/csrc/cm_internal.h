@@ -105,6 +105,9 @@ enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLAS
 // One plan is one dependent chain (2*S*m cells, ~100 us in a single thread); a warp walks it in
 // lock step instead, stages over the lanes, four segments per CTA, every depth in one launch.
 constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
+// Stage counts of the deep-pipeline kernels, cut into ranges that compile as separate
+// translation units (the build script passes the same pairs to cm_cost_deep.cu).
+#define CM_DEEP_RANGES(X) X(17, 28) X(29, 34) X(35, 41) X(42, 48)
 constexpr int kUniMinSegments = 22; // fewer segments in a bucket (or left over after full warps of 32): the per-lane kernel
                                     // is faster than a transposed warp that is two-thirds empty
 constexpr int kAnyMaxChunks = 4096; // shallow classes smaller than this together: one launch for all depths

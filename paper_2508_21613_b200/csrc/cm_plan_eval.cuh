@@ -71,90 +71,181 @@ __device__ __forceinline__ bool make_walker(CutWalker &w, const Tables &tb, int 
 // Per stage this is exactly the 1F1B order -- min(S-1-i, m) forwards, forward/backward
 // pairs, the remaining backwards -- for every m >= 1, and every dependency is either one
 // round or one stage old, so two values per stage are all the state there is.
-// Rounds S-1 .. m-1 have every stage fully active and carry no predicate at all; the
-// ramp-up and ramp-down rounds skip inactive stages with warp-uniform branches.
-//
-// stage(i) returns the stage's forward and backward time, xt(i) the transfer time of the
-// boundary above stage i; both are called with compile-time i only.
+// Rounds S-1 .. m-1 have every stage fully active and carry no predicate at all.
 // ----------------------------------------------------------------------------------
 template <typename T> struct alignas(16) FB { T f, b; };
 
-// Shared-memory loads the compiler must issue where they stand: the stage times are loop
-// invariants, and hoisting ~100 of them into registers would push the per-stage state out.
-template <typename T>
-__device__ __forceinline__ FB<T> lds_fb(const FB<T> *p) {
-    unsigned long long a, b;
-    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"((unsigned)__cvta_generic_to_shared(p)));
-    FB<T> d;
-    d.f = Num<T>::from_bits(a);
-    d.b = Num<T>::from_bits(b);
-    return d;
-}
-template <typename T>
-__device__ __forceinline__ T lds_t(const T *p) {
-    unsigned long long a;
-    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(a) : "r"((unsigned)__cvta_generic_to_shared(p)));
-    return Num<T>::from_bits(a);
-}
+// Where the recurrence finds its stage times.  Both sources are addressed with compile-time
+// stage indices only, so a register source stays in registers and a shared-memory source is
+// read with "base register + immediate" addresses: no address arithmetic per load.
+//
+// SmemStages: stage i's (f, b) pair at byte offset i * FB_STRIDE from `fb`, the transfer time
+// of the boundary above it at i * XT_STRIDE from `xt` (32-bit shared-window addresses).  The
+// loads are written where they are needed; the assembler keeps as many of these loop
+// invariants in registers as the per-stage state leaves room for and reloads the rest
+// (measured: 0.6-0.7 shared loads per cell where one per cell is written).
+template <typename T, int FB_STRIDE, int XT_STRIDE> struct SmemStages {
+    unsigned fb, xt;
+    template <int I> __device__ __forceinline__ FB<T> stage() const {
+        unsigned long long a, b;
+        asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];" : "=l"(a), "=l"(b) : "r"(fb), "n"(I * FB_STRIDE));
+        FB<T> d;
+        d.f = Num<T>::from_bits(a);
+        d.b = Num<T>::from_bits(b);
+        return d;
+    }
+    template <int I> __device__ __forceinline__ T f() const {
+        unsigned long long a;
+        asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(a) : "r"(fb), "n"(I * FB_STRIDE));
+        return Num<T>::from_bits(a);
+    }
+    template <int I> __device__ __forceinline__ T b() const {
+        unsigned long long a;
+        asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(a) : "r"(fb), "n"(I * FB_STRIDE + 8));
+        return Num<T>::from_bits(a);
+    }
+    template <int I> __device__ __forceinline__ T x() const {
+        unsigned long long a;
+        asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(a) : "r"(xt), "n"(I * XT_STRIDE));
+        return Num<T>::from_bits(a);
+    }
+};
+template <typename P> __device__ __forceinline__ unsigned smem_addr(const P *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
-template <typename T, int S, typename StageFn, typename XtFn>
-__device__ __forceinline__ T sim_rounds(int m, StageFn stage, XtFn xt) {
+// RegStages: the stage times of a shallow pipeline, held by the caller in registers.
+template <typename T, int S> struct RegStages {
+    const FB<T> (&st)[S];
+    const T (&xt)[S];
+    template <int I> __device__ __forceinline__ FB<T> stage() const { return st[I]; }
+    template <int I> __device__ __forceinline__ T f() const { return st[I].f; }
+    template <int I> __device__ __forceinline__ T b() const { return st[I].b; }
+    template <int I> __device__ __forceinline__ T x() const { return xt[I]; }
+};
+
+// State and cells of one pipeline of S stages (S compile-time): clock = end of the stage's
+// latest computation, pend = end of the forward the stage has not consumed yet (transfer
+// included).  Every method takes its stage as a template argument.
+template <typename T, int S, typename Src> struct Rounds {
     T clock[S], pend[S];
+    const Src &src;
+    __device__ __forceinline__ explicit Rounds(const Src &s) : src(s) {
 #pragma unroll
-    for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
-    // ramp-up: forwards only
-    for (int t = 0; t < S - 1; ++t) {
-#pragma unroll
-        for (int i = S - 2; i >= 0; --i) {
-            if (i <= t && t < i + m) {
-                const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-                const T fend = fstart + stage(i).f;
-                clock[i] = fend;
-                pend[i + 1] = fend + xt(i);
-            }
+        for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
+    }
+    // forward of stage I: fed by the forward stage I-1 ran one round earlier
+    template <int I> __device__ __forceinline__ void fwd() {
+        const T fstart = I > 0 ? tmax(clock[I], pend[I]) : clock[I];
+        const T fend = fstart + src.template f<I>();
+        clock[I] = fend;
+        if constexpr (I < S - 1) pend[I + 1] = fend + src.template x<I>();
+    }
+    // backward of stage I: fed by the backward stage I+1 ran just before in the same round
+    // (chain_b), at the last stage by its own forward, which is what clock holds there
+    template <int I> __device__ __forceinline__ void bwd(T &chain_b) {
+        const T c = clock[I];
+        T bstart = c;
+        if constexpr (I < S - 1) bstart = tmax(c, chain_b + src.template x<I>());
+        const T bend = bstart + src.template b<I>();
+        clock[I] = bend;
+        chain_b = bend;
+    }
+    // forward then backward of stage I (a steady round)
+    template <int I> __device__ __forceinline__ void both(T &chain_b) {
+        const FB<T> d = src.template stage<I>();
+        const T fstart = I > 0 ? tmax(clock[I], pend[I]) : clock[I];
+        const T fend = fstart + d.f;
+        T bstart = fend;
+        if constexpr (I < S - 1) {
+            const T x = src.template x<I>();
+            pend[I + 1] = fend + x;
+            bstart = tmax(fend, chain_b + x);
+        }
+        const T bend = bstart + d.b;
+        clock[I] = bend;
+        chain_b = bend;
+    }
+    // stages I, I-1, .., 0
+    template <int I> __device__ __forceinline__ void fwd_down() { fwd<I>(); if constexpr (I > 0) fwd_down<I - 1>(); }
+    template <int I> __device__ __forceinline__ void bwd_down(T &chain_b) { bwd<I>(chain_b); if constexpr (I > 0) bwd_down<I - 1>(chain_b); }
+    template <int I> __device__ __forceinline__ void both_down(T &chain_b) { both<I>(chain_b); if constexpr (I > 0) both_down<I - 1>(chain_b); }
+    // forwards of stages I, I-1, .., last (last >= 1, warp-uniform)
+    template <int I> __device__ __forceinline__ void fwd_down_to(int last) {
+        fwd<I>();
+        if constexpr (I > 1) { if (I != last) fwd_down_to<I - 1>(last); }
+    }
+    // stages I .. 0, each only if `active(i)`: the general ramp rounds
+    template <int I, typename Pred> __device__ __forceinline__ void fwd_down_if(Pred active) {
+        if (active(I)) fwd<I>();
+        if constexpr (I > 0) fwd_down_if<I - 1>(active);
+    }
+    template <int I, typename Pred> __device__ __forceinline__ void fwd_if_bwd_down(Pred active, T &chain_b) {
+        if (active(I)) fwd<I>();
+        bwd<I>(chain_b);
+        if constexpr (I > 0) fwd_if_bwd_down<I - 1>(active, chain_b);
+    }
+    // forwards of stages `top`, top-1, .., 0 with top chosen at run time (top <= S-2): a jump
+    // into the unrolled sequence, so that a ramp-up round costs its active stages and nothing more
+    __device__ __forceinline__ void fwd_down_from(int top) {
+        switch (top) {
+#define CM_RAMP(K) case K: if constexpr (K <= S - 2) fwd<(K <= S - 2 ? K : 0)>(); [[fallthrough]];
+            CM_RAMP(62) CM_RAMP(61) CM_RAMP(60) CM_RAMP(59) CM_RAMP(58) CM_RAMP(57) CM_RAMP(56) CM_RAMP(55)
+            CM_RAMP(54) CM_RAMP(53) CM_RAMP(52) CM_RAMP(51) CM_RAMP(50) CM_RAMP(49) CM_RAMP(48) CM_RAMP(47)
+            CM_RAMP(46) CM_RAMP(45) CM_RAMP(44) CM_RAMP(43) CM_RAMP(42) CM_RAMP(41) CM_RAMP(40) CM_RAMP(39)
+            CM_RAMP(38) CM_RAMP(37) CM_RAMP(36) CM_RAMP(35) CM_RAMP(34) CM_RAMP(33) CM_RAMP(32) CM_RAMP(31)
+            CM_RAMP(30) CM_RAMP(29) CM_RAMP(28) CM_RAMP(27) CM_RAMP(26) CM_RAMP(25) CM_RAMP(24) CM_RAMP(23)
+            CM_RAMP(22) CM_RAMP(21) CM_RAMP(20) CM_RAMP(19) CM_RAMP(18) CM_RAMP(17) CM_RAMP(16) CM_RAMP(15)
+            CM_RAMP(14) CM_RAMP(13) CM_RAMP(12) CM_RAMP(11) CM_RAMP(10) CM_RAMP(9) CM_RAMP(8) CM_RAMP(7)
+            CM_RAMP(6) CM_RAMP(5) CM_RAMP(4) CM_RAMP(3) CM_RAMP(2) CM_RAMP(1) CM_RAMP(0)
+#undef CM_RAMP
+        default: break;
         }
     }
-    // steady rounds: every stage does one forward and one backward
-    // four rounds per trip: the backward chain of one round overlaps the forwards of the
-    // next ones in the instruction stream, which hides its fixed latencies
+};
+
+// ----------------------------------------------------------------------------------
+// The recurrence in "rounds" (see above), any m >= 1.
+//   ramp-up    rounds 0 .. S-2        forwards only: stages max(0, t-m+1) .. t
+//   steady     rounds S-1 .. m-1      every stage one forward and one backward, no predicate
+//   ramp-down  rounds max(m,S-1) .. S-2+m   every stage a backward, stages above t-m a forward first
+// With m >= S-1 (every stage gets its full warm-up: the common case) the ramp rounds touch
+// exactly their active stages: ramp-up jumps into the unrolled forward sequence at stage t,
+// ramp-down runs the forwards from the last stage down to stage t-m+1 and then all
+// backwards (within a round the forwards depend only on the round before, so they may all
+// precede the backwards).  With fewer micro-batches the ramp rounds test every stage.
+// ----------------------------------------------------------------------------------
+template <typename T, int S, typename Src>
+__device__ __forceinline__ T sim_rounds(int m, const Src &src) {
+    Rounds<T, S, Src> r(src);
+    if constexpr (S == 1) {
+        for (int t = 0; t < m; ++t) { T chain_b = (T)0; r.template both<0>(chain_b); }
+        return r.clock[0];
+    } else {
+        if (m >= S - 1) {
+            for (int t = 0; t < S - 1; ++t) r.fwd_down_from(t);
+        } else {
+            for (int t = 0; t < S - 1; ++t) r.template fwd_down_if<S - 2>([&](int i) { return i <= t && t < i + m; });
+        }
+        // four rounds per trip: the backward chain of one round overlaps the forwards of the
+        // next ones in the instruction stream, which hides its fixed latencies
 #pragma unroll 4
-    for (int t = S - 1; t < m; ++t) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            const FB<T> d = stage(i);
-            const T x = i < S - 1 ? xt(i) : (T)0;
-            const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
-            const T fend = fstart + d.f;
-            if (i < S - 1) pend[i + 1] = fend + x;
-            const T dep = i < S - 1 ? chain_b + x : fend;
-            const T bstart = tmax(fend, dep);
-            const T bend = bstart + d.b;
-            clock[i] = bend;
-            chain_b = bend;
+        for (int t = S - 1; t < m; ++t) {
+            T chain_b = (T)0;
+            r.template both_down<S - 1>(chain_b);
         }
-    }
-    // ramp-down: every stage still has a backward, the upper ones a forward too
-    for (int t = (m > S - 1 ? m : S - 1); t < S - 1 + m; ++t) {
-        T chain_b = (T)0;
-#pragma unroll
-        for (int i = S - 1; i >= 0; --i) {
-            const FB<T> d = stage(i);
-            const T x = i < S - 1 ? xt(i) : (T)0;
-            T c = clock[i];
-            if (t < i + m) {
-                const T fstart = i > 0 ? tmax(c, pend[i]) : c;
-                c = fstart + d.f;
-                if (i < S - 1) pend[i + 1] = c + x;
+        if (m >= S - 1) {
+            for (int q = 0; q < S - 1; ++q) {      // round m + q: forwards of stages S-1 .. q+1
+                r.template fwd_down_to<S - 1>(q + 1);
+                T chain_b = (T)0;
+                r.template bwd_down<S - 1>(chain_b);
             }
-            const T dep = i < S - 1 ? chain_b + x : c;
-            const T bstart = tmax(c, dep);
-            const T bend = bstart + d.b;
-            clock[i] = bend;
-            chain_b = bend;
+        } else {
+            for (int t = S - 1; t < S - 1 + m; ++t) {
+                T chain_b = (T)0;
+                r.template fwd_if_bwd_down<S - 1>([&](int i) { return t < i + m; }, chain_b);
+            }
         }
+        return r.clock[0];
     }
-    return clock[0];
 }
 
 // ----------------------------------------------------------------------------------
@@ -275,8 +366,8 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
         lo = hi;
     }
     if (!ok) return false;
-    const T t = sim_rounds<T, S>(m, [&](int i) { return lds_fb<T>(fcol + i * kChunk); },
-                                 [&](int i) { return lds_t<T>(xcol + i * kChunk); });
+    const SmemStages<T, (int)sizeof(FB<T>) * kChunk, (int)sizeof(T) * kChunk> src{smem_addr(fcol), smem_addr(xcol)};
+    const T t = sim_rounds<T, S>(m, src);
     cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
     return true;
 }
