@@ -351,6 +351,19 @@ int cm_int64_runs_in_fp64(const cm_ctx *ctx);
  * set of each expected size twice beforehand. */
 cm_status cm_set_latency_graphs(cm_ctx *ctx, int on);
 
+/* Memory screen (on by default).  Whether a layer composition fits in memory depends on the
+ * stage count, the micro-batches in flight and the composition itself -- not on which devices
+ * failed, the link tiers or the cost mode (Section "Estimator", memory estimator).  The context
+ * therefore lists, once per profile and (layer mode, stages, micro-batches), the memory-feasible
+ * compositions in ascending order, and the search and tie-break passes walk those lists instead
+ * of all enumerated compositions (segments of more than 2^20 compositions are walked in full).
+ * The first search that meets a new (stages, micro-batches) pair builds its list: one small copy
+ * each way, one kernel and a stream synchronisation.  Results are identical either way; candidate
+ * indices, cm_evaluate and cm_decode_plan are unaffected; cm_last_stats [0] still counts every
+ * enumerated pipeline-plan and [16] those whose recurrence ran.  cm_set_memory_screen(ctx, 0)
+ * makes batches and spaces built afterwards test every composition inside the search pass. */
+cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
+
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
  * with node boundaries at the same places among them have identical dynamic-parallelism
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set

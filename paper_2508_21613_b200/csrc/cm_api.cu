@@ -115,6 +115,7 @@ struct Batch {
     int B = 0;
     bool intval = false;                   // integer mode evaluated in double arithmetic (fixed when the batch is built)
     uint64_t profile_gen = 0;              // generation of the profile the tables describe (see cm_ctx::profile_gen)
+    bool mm_launched = false;              // the min-max partitions of `keys` were already enqueued (with the feasible lists)
 };
 
 struct cm_ctx {
@@ -143,6 +144,15 @@ struct cm_ctx {
     uint8_t *d_mm[2] = {nullptr, nullptr};   // min-max cuts per cost mode
     std::vector<uint8_t> mm_done[2];
     int mm_stride_m = 0;
+    // Memory-feasible layer compositions per (layer mode, stages, micro-batches), listed once per
+    // profile (cm_feasible_kernel) into one device pool that only grows; key = S << 16 | m.
+    struct FeasEntry { uint32_t first, count; uint64_t K; };
+    std::map<uint32_t, FeasEntry> feas[3];
+    DevBuf<uint32_t> d_feas;
+    size_t feas_used = 0;
+    PinnedVec<unsigned char> feas_stage;      // keys, K, offsets out; counts back
+    DevBuf<unsigned char> d_feas_stage;
+    bool screen = true;               // walk only the listed feasible compositions (cm_set_memory_screen)
     Batch batch;                      // reused by cm_search_batch
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_obj[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // phases of the objective pass
@@ -271,11 +281,11 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket.clear();
     bt.classes.clear();
     bt.bucket_tseg.clear();
-    struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; };
+    struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
     std::vector<Pre> pre;
-    auto kind_of = [](int S, int m, uint64_t n_seg, uint64_t count) {
+    auto kind_of = [](int S, int m, uint64_t n_seg, uint64_t K) {
         if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_GENERIC;
-        if (count == 1) return (int)CM_CLASS_SOLO;
+        if (K == 0) return (int)CM_CLASS_SOLO;   // the min-max partition is the only candidate there is
         if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
         return (int)CM_CLASS_GENERIC;
     };
@@ -296,12 +306,14 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
             if (g.m >= 1) {   // m = 0 cannot be feasible: no work is scheduled
                 const uint64_t n_seg = (uint64_t)(j - i) * tp.n_scen;
                 if (n_seg >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "too many segments in one bucket");
-                const uint64_t count = g.K ? g.K + 1 : 1;
+                // candidates the search pass walks per segment: the listed feasible ones, or all
+                const uint64_t count = g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1);
+                if (count == 0) { i = j; continue; }   // nothing fits in memory: the segments stay infeasible
                 // The transposed kernel gives every 32 segments a warp per composition, full or
                 // not.  With one scenario the segments are few: what does not fill most of a
                 // last warp goes to the per-lane kernel, which wastes no lane.
                 size_t cut = j;
-                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, count) == CM_CLASS_WIDE_UNI) {
+                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, g.K) == CM_CLASS_WIDE_UNI) {
                     const size_t rest = (j - i) % 32;
                     if (rest > 0 && rest < (size_t)kUniMinSegments) cut = j - rest;
                 }
@@ -310,7 +322,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     if (p1 <= p0) continue;
                     const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
                     Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
-                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, count)};
+                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, g.K), g.feas_first};
                     for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
                     pre.push_back(q);
                 }
@@ -345,6 +357,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 bk.n_seg = q.n_seg;
                 bk.S = q.S;
                 bk.m = q.m;
+                bk.feas_first = q.feas_first;
                 if (kind == CM_CLASS_WIDE_UNI) {
                     const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
                     const uint64_t per_cta = (uint64_t)(kChunk / 32) * c.uni_items;
@@ -426,6 +439,8 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
                 g.n_sync = (uint16_t)dp;
                 g.off = (uint16_t)off;
                 g.K = K;
+                g.feas_first = kNoFeasList;
+                g.feas_count = 0;
                 g.cand_first = cand;
                 const uint64_t count = K ? K + 1 : 1;
                 const uint64_t tiles = (count + kTile - 1) / kTile;
@@ -451,6 +466,95 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
     tp.n_red = split_first ? (uint32_t)std::min<uint64_t>((split_first + 1023) / 1024, 64) : 0;
     *out = (uint32_t)bt.tmpl.size();
     bt.tmpl.push_back(tp);
+    return CM_OK;
+}
+
+Tables tables(const cm_ctx *ctx, const Batch &bt);
+
+// Grow the feasible-composition pool to hold `want` entries, keeping its contents.  The pool's
+// address changes, and captured launch sequences carry the old one: they are dropped and
+// captured again at their next use.
+cm_status grow_feas_pool(cm_ctx *ctx, size_t want) {
+    if (want <= ctx->d_feas.cap) return CM_OK;
+    size_t nc = std::max<size_t>(want, std::max<size_t>(ctx->d_feas.cap * 2, 1u << 20));
+    uint32_t *q = nullptr;
+    CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (cudaMalloc((void **)&q, nc * sizeof(uint32_t)) != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ENOMEM, "device memory"); }
+    if (ctx->feas_used) {
+        cudaError_t e = cudaMemcpyAsync(q, ctx->d_feas.p, ctx->feas_used * sizeof(uint32_t), cudaMemcpyDeviceToDevice, ctx->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+        if (e != cudaSuccess) { cudaFree(q); cudaGetLastError(); return fail(ctx, CM_ECUDA, cudaGetErrorString(e)); }
+    }
+    if (ctx->d_feas.p) cudaFree(ctx->d_feas.p);
+    ctx->d_feas.p = q;
+    ctx->d_feas.cap = nc;
+    for (auto &e : ctx->single)
+        if (e->exec) { cudaGraphExecDestroy(e->exec); e->exec = nullptr; }
+    return CM_OK;
+}
+
+// Point every template segment at the list of its memory-feasible candidates, building the
+// lists this context has not built yet (Section "Estimator", memory estimator: feasibility is
+// a function of stages, micro-batches and composition only).  New lists cost one small copy
+// each way, the min-max partitions they end with, one kernel and a synchronisation -- once
+// per (layer mode, stages, micro-batches) and profile.
+cm_status ensure_feasible_lists(cm_ctx *ctx, Batch &bt) {
+    const int lm = bt.opts.lm;
+    if (lm == CM_LAYERS_MINMAX) return CM_OK;
+    std::map<uint32_t, cm_ctx::FeasEntry> &known = ctx->feas[lm];
+    std::vector<uint32_t> new_keys;
+    std::vector<uint64_t> new_K;
+    std::vector<uint32_t> new_first;
+    size_t used = ctx->feas_used;
+    for (const TSeg &g : bt.tseg) {
+        if (g.K == 0 || g.K > kFeasMaxK || g.m < 1) continue;
+        const uint32_t key = ((uint32_t)g.S << 16) | g.m;
+        if (known.count(key)) continue;
+        if (used + g.K + 1 >= 0xfffffff0ull) break;   // pool offsets are 32-bit: later keys stay unscreened
+        known[key] = cm_ctx::FeasEntry{(uint32_t)used, kNoFeasList, g.K};   // count filled in below
+        new_keys.push_back(key);
+        new_K.push_back(g.K);
+        new_first.push_back((uint32_t)used);
+        used += g.K + 1;
+    }
+    if (!new_keys.empty()) {
+        auto undo = [&]() { for (uint32_t k : new_keys) known.erase(k); };
+        cm_status s = grow_feas_pool(ctx, used);
+        if (s != CM_OK) { undo(); return s; }
+        const size_t n = new_keys.size(), n_mm = bt.keys.size();
+        // staging layout: K (8n) | keys (4n) | first (4n) | min-max keys (4 n_mm) | counts (4n, device -> host)
+        const size_t off_key = 8 * n, off_first = off_key + 4 * n, off_mm = off_first + 4 * n, off_cnt = off_mm + 4 * n_mm;
+        const size_t bytes = off_cnt + 4 * n;
+        if (!ctx->feas_stage.resize(bytes) || !ctx->d_feas_stage.reserve(bytes)) { undo(); return fail(ctx, CM_ENOMEM, "memory"); }
+        unsigned char *h = ctx->feas_stage.p, *d = ctx->d_feas_stage.p;
+        memcpy(h, new_K.data(), 8 * n);
+        memcpy(h + off_key, new_keys.data(), 4 * n);
+        memcpy(h + off_first, new_first.data(), 4 * n);
+        if (n_mm) memcpy(h + off_mm, bt.keys.data(), 4 * n_mm);
+        const Tables tb = tables(ctx, bt);
+        cudaError_t e = cudaMemcpyAsync(d, h, off_cnt, cudaMemcpyHostToDevice, ctx->stream);
+        if (e == cudaSuccess && n_mm)
+            e = launch_minmax(tb, (const uint32_t *)(d + off_mm), (int)n_mm, bt.intval ? CM_COST_FP64 : bt.opts.cost, ctx->stream);
+        if (e == cudaSuccess)
+            e = launch_feasible(tb, lm, (const uint32_t *)(d + off_key), (const uint64_t *)d, (const uint32_t *)(d + off_first),
+                                (int)n, ctx->d_feas.p, (uint32_t *)(d + off_cnt), ctx->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(h + off_cnt, d + off_cnt, 4 * n, cudaMemcpyDeviceToHost, ctx->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+        if (e != cudaSuccess) { cudaGetLastError(); undo(); return fail(ctx, CM_ECUDA, std::string("feasible-composition lists: ") + cudaGetErrorString(e)); }
+        bt.mm_launched = n_mm > 0;
+        const uint32_t *cnt = (const uint32_t *)(h + off_cnt);
+        for (size_t q = 0; q < n; ++q) known[new_keys[q]].count = cnt[q];
+        ctx->feas_used = used;
+        ctx->stats[9] += off_cnt;
+        ctx->stats[10] += 4 * n;
+    }
+    for (TSeg &g : bt.tseg) {
+        if (g.K == 0 || g.K > kFeasMaxK || g.m < 1) continue;
+        auto it = known.find(((uint32_t)g.S << 16) | g.m);
+        if (it == known.end() || it->second.count == kNoFeasList) continue;
+        g.feas_first = it->second.first;
+        g.feas_count = it->second.count;
+    }
     return CM_OK;
 }
 
@@ -569,6 +673,11 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     }
     bt.n_rows = rows;
     bt.n_tiles = bt.max_tiles_per_seg ? 1 : 0;   // only "is there anything to tie-break" matters
+    bt.mm_launched = false;
+    if (ctx->d_prof && ctx->screen) {   // (a context without a device only describes: cm_host_describe)
+        cm_status s = ensure_feasible_lists(ctx, bt);
+        if (s != CM_OK) return s;
+    }
     return build_buckets(ctx, bt);
 }
 
@@ -590,6 +699,7 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.failed = (const uint32_t *)(a + bt.off_failed); v.cross = (const uint64_t *)(a + bt.off_cross);
     v.tmpl_scen = (const uint32_t *)(a + bt.off_tmpl_scen); v.bucket = (const Bucket *)(a + bt.off_bucket);
     v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
+    v.feas = ctx->d_feas.p;
     v.seg_best = bt.d_seg_best.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
@@ -601,7 +711,6 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.max_red_per_scen = 0;
     for (const Tmpl &tp : bt.tmpl) v.max_red_per_scen = std::max(v.max_red_per_scen, tp.n_scen ? tp.n_red : 0u);
     v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
-    (void)ctx;
     return v;
 }
 
@@ -644,7 +753,7 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
          bt.d_kappa_sel.reserve(B * kMaxP) && bt.d_pol_cost.reserve(B * 2) &&
          bt.d_rc_stages.reserve(B * kMaxP) && bt.d_plans.reserve(B * 4 + 1);   // + room for the counters
     if (!ok) return fail(ctx, CM_ENOMEM, "device memory");
-    if (bt.keys.size()) {
+    if (bt.keys.size() && !bt.mm_launched) {
         CM_CUDA(ctx, launch_minmax(tables(ctx, bt), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
                                    (int)bt.keys.size(), bt.intval ? CM_COST_FP64 : bt.opts.cost, ctx->stream));
         if (launches) ++*launches;
@@ -1039,6 +1148,8 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     ctx->has_profile = false;
     ++ctx->profile_gen;                                  // spaces and batches of the old profile are refused from here on
     ctx->single.clear();                                 // prepared one-scenario batches describe the old profile
+    for (auto &f : ctx->feas) f.clear();                 // so do the feasible-composition lists
+    ctx->feas_used = 0;
     cm_status s = load_profile_host(ctx, p);
     if (s != CM_OK) return s;
     DevProfile &h = ctx->hp;
@@ -1392,6 +1503,12 @@ int cm_int64_runs_in_fp64(const cm_ctx *ctx) {
 cm_status cm_set_latency_graphs(cm_ctx *ctx, int on) {
     if (!ctx) return CM_EINVAL;
     ctx->use_graphs = on != 0;
+    return CM_OK;
+}
+
+cm_status cm_set_memory_screen(cm_ctx *ctx, int on) {
+    if (!ctx) return CM_EINVAL;
+    ctx->screen = on != 0;
     return CM_OK;
 }
 

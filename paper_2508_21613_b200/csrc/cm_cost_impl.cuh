@@ -117,6 +117,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
     uint64_t seg_local, kappa;
     plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
     uint32_t row = 0xffffffffu;
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
@@ -146,6 +147,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, Bat
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
     uint64_t seg_local, kappa;
     plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
     uint32_t row = 0xffffffffu;
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
@@ -255,9 +257,10 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
         for (int r = 0; r < n_items; ++r) {
             const uint64_t item = ((chunk - bks.chunk_first) * (kChunk / 32) + warp) * (uint64_t)n_items + r;
             const uint32_t n_groups = (bks.n_seg + 31) / 32;
-            const uint64_t kappa = item / n_groups;
-            if (kappa >= bks.count || m < 1) break;            // warp-uniform; items ascend
-            const uint32_t seg_local = (uint32_t)(item - kappa * n_groups) * 32 + lane;
+            const uint64_t pos = item / n_groups;              // position in the bucket's walk
+            if (pos >= bks.count || m < 1) break;              // warp-uniform; items ascend
+            const uint64_t kappa = walk_kappa(bd.feas, bks.feas_first, pos);
+            const uint32_t seg_local = (uint32_t)(item - pos * n_groups) * 32 + lane;
             const bool active = seg_local < bks.n_seg;
             const SegView g = bucket_segment(bd, bks, active ? seg_local : 0);
             if (kappa != st_kappa[warp]) {
@@ -296,6 +299,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
         const uint64_t base = (chunk - bk.chunk_first) * kChunk;
         uint64_t seg_local, kappa;
         plan_of_thread(base, bk.count, tid, seg_local, kappa);
+        if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
         uint32_t row = 0xffffffffu;
         uint64_t bits = inf_bits<T>();
         if (seg_local < bk.n_seg && m >= 1) {
@@ -323,6 +327,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, Batc
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
     uint64_t seg_local, kappa;
     plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
     uint32_t row = 0xffffffffu;
     uint64_t bits = inf_bits<T>();
     unsigned long long my_cells = 0;
@@ -445,12 +450,13 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_w
             found_so_far = *(volatile uint64_t *)slot;
         }
         __syncthreads();
-        const uint64_t count = g.K ? g.K + 1 : 1;
+        const uint64_t count = walk_count(g);
         const uint64_t first = tile * kChunk;
-        if (first >= count || found_so_far <= first) break;              // uniform: later tiles cannot win either
-        const uint64_t kappa = first + threadIdx.x;
+        // uniform: later tiles hold higher compositions than one already found
+        if (first >= count || found_so_far <= walk_kappa(bd.feas, g.feas_first, first)) break;
         uint64_t hit = ~0ull;
-        if (kappa < count) {
+        if (first + threadIdx.x < count) {
+            const uint64_t kappa = walk_kappa(bd.feas, g.feas_first, first + threadIdx.x);
             T cost;
             if (plan_cost_wide_lane<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, cost) &&
                 Num<T>::bits(cost) <= w.cost_bits)

@@ -243,8 +243,18 @@ __device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, i
 struct SegView {
     uint64_t tier, K;
     uint32_t row;          // row of seg_best
+    uint32_t feas_first, feas_count;
     int S, m, n_sync;
 };
+
+// Candidates a pass walks in a segment, and the layer composition behind position idx of
+// that walk: the listed memory-feasible ones in ascending order, or all of them.
+__device__ __forceinline__ uint64_t walk_count(const SegView &g) {
+    return g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1);
+}
+__device__ __forceinline__ uint64_t walk_kappa(const uint32_t *feas, uint32_t feas_first, uint64_t idx) {
+    return feas_first != kNoFeasList ? (uint64_t)feas[feas_first + idx] : idx;
+}
 
 __device__ __forceinline__ uint64_t cut_bits(const uint64_t *words, int off, int n /* <= 63 */) {
     const int w = off >> 6, sh = off & 63;
@@ -261,6 +271,8 @@ __device__ __forceinline__ SegView seg_view(const BatchDev &bd, uint32_t scen_id
     v.m = g.m;
     v.n_sync = g.n_sync;
     v.K = g.K;
+    v.feas_first = g.feas_first;
+    v.feas_count = g.feas_count;
     v.row = sc.seg_base + (tseg_row - bd.tmpl[sc.tmpl].tseg_first);
     v.tier = cut_bits(bd.cross + sc.cross_first, g.off, g.S - 1);
     return v;

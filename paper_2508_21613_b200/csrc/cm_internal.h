@@ -45,12 +45,20 @@ struct DevProfile {
 // One template segment = (strategy, pipeline, micro-batch count): its candidates are the
 // layer compositions kappa = 0..K-1 followed by the min-max partition, or the min-max
 // partition alone (K = 0).
-struct TSeg {              // 24 bytes
+struct TSeg {              // 32 bytes
     uint64_t cand_first;   // index of its first candidate within one scenario's space
     uint64_t K;            // enumerated compositions
     uint16_t S, m, n_sync; // stages, micro-batches, data-parallel peers of the strategy
     uint16_t off;          // survivor index of the pipeline's first stage
+    uint32_t feas_first;   // its memory-feasible candidates, ascending, as a range of the feasible-
+    uint32_t feas_count;   //   composition pool (kNoFeasList: none was built, all K+1 are walked)
 };
+// Whether a layer composition fits in memory depends on (stages, micro-batches, composition)
+// only -- not on the failure scenario, the link tiers or the cost mode (Section "Estimator",
+// memory estimator).  So the feasible compositions of every (S, m) are listed once per profile
+// and the search pass and the tie-break pass walk that list instead of all K + 1 candidates.
+constexpr uint32_t kNoFeasList = 0xffffffffu;
+constexpr uint64_t kFeasMaxK = 1ull << 20;   // larger segments are walked unscreened
 
 // One parallel strategy of a template.
 struct Strat {
@@ -94,7 +102,7 @@ struct Bucket {
     uint32_t n_tseg;
     uint32_t tmpl, n_seg;  // n_seg = n_tseg * scenarios of the template
     uint16_t S, m;
-    uint32_t pad;
+    uint32_t feas_first;   // count = length of this list if there is one (kNoFeasList: count = K+1 or 1)
 };
 
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
@@ -148,6 +156,7 @@ struct BatchDev {
     const uint32_t *tmpl_scen;    // scenario ids grouped by template
     const Bucket *bucket;         // search-pass work layout
     const uint32_t *bucket_tseg;  // template segment rows grouped by bucket
+    const uint32_t *feas;         // feasible-composition pool of the context
     uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
     const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
     Partial *partial;       // [n_red_blocks]
@@ -215,6 +224,10 @@ inline bool native_i64(const BatchDev &b) { return b.mode == CM_COST_INT64NS && 
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
+// feasible compositions of n_keys (S << 16 | m) keys: list of key q written at pool + first[q]
+// (room for K[q] + 1 entries), its length to count[q]
+cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *keys_dev, const uint64_t *K_dev,
+                            const uint32_t *first_dev, int n_keys, uint32_t *pool, uint32_t *count_dev, cudaStream_t st);
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st);
 // Tiles of a segment that the tie-break kernels take side by side (grid.y); the rest is
 // walked serially inside the CTA.  A single scenario gets every tile its own CTA (lowest

@@ -2,6 +2,7 @@
 //
 //   cm_prefix_kernel      per-layer prefix sums and per-boundary transfer times
 //   cm_minmax_kernel      min-max contiguous layer partition per (stages, micro-batches)
+//   cm_feasible_kernel    memory-feasible layer compositions per (stages, micro-batches), listed once
 //   (data rerouting / redundant computation: cm_policy.cu)
 //   (the search pass over every pipeline-plan lives in cm_cost.cu)
 //   cm_split_kernel       (cost, index) argmin over (strategy, micro-batch split) per scenario
@@ -128,6 +129,73 @@ cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys,
     if (n_keys <= 0) return cudaSuccess;
     if (mode == CM_COST_INT64NS) cm_minmax_kernel<long long><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
     else cm_minmax_kernel<double><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// Memory-feasible layer compositions of an (S, m) key, in ascending order (Section
+// "Estimator", memory estimator: a stage's peak depends on its layers, its position and the
+// micro-batches in flight -- not on the failure scenario, so this is done once per key and
+// profile).  One CTA per key walks kappa = 0 .. K-1 in chunks of its size and compacts the
+// feasible ranks in order (ballot + prefix over the warps); the min-max partition, candidate
+// K, closes the list if a memory-feasible partition exists.
+// ----------------------------------------------------------------------------------
+constexpr int kFeasThreads = 1024;
+__global__ void __launch_bounds__(kFeasThreads) cm_feasible_kernel(Tables tb, int layer_mode, const uint32_t *keys,
+                                                                   const uint64_t *Ks, const uint32_t *first,
+                                                                   uint32_t *pool, uint32_t *count_out) {
+    __shared__ long long PA[kMaxL + 1], PS[kMaxL + 1];
+    __shared__ uint32_t warp_cnt[kFeasThreads / 32];
+    __shared__ uint32_t running;
+    const DevProfile *p = tb.prof;
+    const int L = p->L;
+    const uint32_t key = keys[blockIdx.x];
+    const int S = (int)(key >> 16), m = (int)(key & 0xffffu);
+    const uint64_t K = Ks[blockIdx.x];
+    uint32_t *out = pool + first[blockIdx.x];
+    const long long cap = p->cap;
+    for (int l = threadIdx.x; l <= L; l += blockDim.x) { PA[l] = p->PA[l]; PS[l] = p->PS[l]; }
+    if (threadIdx.x == 0) running = 0;
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint64_t base = 0; base < K; base += kFeasThreads) {
+        const uint64_t kappa = base + threadIdx.x;
+        bool ok = kappa < K;
+        if (ok) {
+            CutWalker cw;
+            make_walker(cw, tb, layer_mode, L, S, kappa, K, 0);
+            int lo = 0;
+            for (int i = 0; i < S && ok; ++i) {
+                const int hi = cw.next();
+                ok = hi > lo && stage_fits(PS[hi] - PS[lo], PA[hi] - PA[lo], i, S, m, cap);
+                lo = hi;
+            }
+        }
+        const uint32_t vote = __ballot_sync(0xffffffffu, ok);
+        if (lane == 0) warp_cnt[warp] = __popc(vote);
+        __syncthreads();
+        uint32_t before = running, total = 0;
+        for (uint32_t w = 0; w < kFeasThreads / 32; ++w) {
+            const uint32_t c = warp_cnt[w];
+            if (w < warp) before += c;
+            total += c;
+        }
+        if (ok) out[before + __popc(vote & ((1u << lane) - 1u))] = (uint32_t)kappa;
+        __syncthreads();
+        if (threadIdx.x == 0) running += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint32_t n = running;
+        if (tb.mm_cuts[(size_t)tb.mm_slot(S, m) * (kMaxS + 1)] == 0) out[n++] = (uint32_t)K;
+        count_out[blockIdx.x] = n;
+    }
+}
+
+cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *keys_dev, const uint64_t *K_dev,
+                            const uint32_t *first_dev, int n_keys, uint32_t *pool, uint32_t *count_dev, cudaStream_t st) {
+    if (n_keys <= 0) return cudaSuccess;
+    cm_feasible_kernel<<<n_keys, kFeasThreads, 0, st>>>(t, layer_mode, keys_dev, K_dev, first_dev, pool, count_dev);
     return cudaGetLastError();
 }
 
@@ -285,12 +353,13 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
             found_so_far = *(volatile uint64_t *)slot;
         }
         __syncthreads();
-        const uint64_t count = g.K ? g.K + 1 : 1;
+        const uint64_t count = walk_count(g);
         const uint64_t first = tile * kTile;
-        if (first >= count || found_so_far <= first) break;          // uniform: later tiles cannot win either
-        const uint64_t kappa = first + threadIdx.x;
+        // uniform: later tiles hold higher compositions than one already found
+        if (first >= count || found_so_far <= walk_kappa(bd.feas, g.feas_first, first)) break;
         uint64_t hit = ~0ull;
-        if (kappa < count) {
+        if (first + threadIdx.x < count) {
+            const uint64_t kappa = walk_kappa(bd.feas, g.feas_first, first + threadIdx.x);
             T cost;
             // shallow pipelines take the register-resident evaluation, the rest the generic one
             const bool ok = (g.S <= kRegStagesMax && g.m >= g.S - 1)

@@ -560,3 +560,37 @@ def test_spaces_and_batches_of_an_earlier_profile_are_refused(gpu):
         gpu.cm_space_free(space)
     finally:
         s.close()
+
+
+def test_memory_screen_changes_the_work_not_the_result(gpu, oracle_factory):
+    """With the screen on (default) the passes walk the listed memory-feasible compositions;
+    with it off they test every composition.  Plans, costs and the count of plans whose
+    recurrence ran must be identical; the oracle pins the plans themselves."""
+    for w, scen in ((W.tiny(mem_bound=True), None), (W.llama70b_like(), 6), (W.random_small(1, tight_memory=True), None)):
+        scenarios = w.scenarios if scen is None else w.scenarios[:scen]
+        for mode in (0, 1):
+            opts = w.options.with_cost_mode(mode)
+            results = []
+            for screen in (True, False):
+                s = Session(gpu, w.profile)
+                try:
+                    gpu.cm_set_memory_screen(s.ctx, screen)
+                    best, per, _ = gpu.cm_search_batch(s.ctx, scenarios, opts, per_policy=True)
+                    st = gpu.cm_last_stats(s.ctx)
+                    results.append((gpu.plans_from_array(best), gpu.plans_from_array(per), st["plans"], st["plans_simulated"]))
+                    # one at a time as well (resident batches, graph replay on the second pass)
+                    for _ in range(2):
+                        one = gpu.PackedScenarios(scenarios[:3])
+                        one.search(s.ctx, opts, latency=True)
+                        for b in range(3):
+                            assert_same_plan(gpu.plans_from_array(one.best)[b], results[-1][0][b], mode, "one by one")
+                finally:
+                    s.close()
+            on, off = results
+            assert on[2] == off[2] and on[3] == off[3] and on[3] <= on[2]
+            for a, b in zip(on[0] + on[1], off[0] + off[1]):
+                assert a.key() == b.key() and a.cost == b.cost and a.cost_ns == b.cost_ns
+            if w.name != "70b-like":
+                o = oracle_factory(w.profile, opts)
+                for b, failed in enumerate(scenarios):
+                    assert_same_plan(on[0][b], o.search(failed)[0], mode, f"{w.name} {failed}")
