@@ -24,6 +24,7 @@ MAX_PIPES = 16
 MAX_STAGES = 64
 
 REROUTE, REDUNDANT, DYNPAR = 0, 1, 2
+SCHED_1F1B, SCHED_GPIPE = 0, 1
 
 
 def build(force: bool = False) -> str:
@@ -60,7 +61,8 @@ class _Profile(C.Structure):
 
 class _Opts(C.Structure):
     _fields_ = [("dp_lo", C.c_int32), ("dp_hi", C.c_int32), ("pp_lo", C.c_int32), ("pp_hi", C.c_int32),
-                ("layer_mode", C.c_int32), ("batch_mode", C.c_int32), ("kappa_cap", C.c_uint64)]
+                ("layer_mode", C.c_int32), ("batch_mode", C.c_int32), ("kappa_cap", C.c_uint64),
+                ("schedule", C.c_int32)]
 
 
 class _Plan(C.Structure):
@@ -170,7 +172,8 @@ class Oracle:
     # -- helpers -------------------------------------------------------------
     def _opts(self, options=None) -> Tuple[_Opts, str]:
         o = options or self.options
-        return (_Opts(o.dp_lo, o.dp_hi, o.pp_lo, o.pp_hi, o.layer_mode, o.batch_mode, o.kappa_cap),
+        return (_Opts(o.dp_lo, o.dp_hi, o.pp_lo, o.pp_hi, o.layer_mode, o.batch_mode, o.kappa_cap,
+                      int(getattr(o, "schedule", 0))),
                 "_i64" if o.cost_mode == 1 else "_f64")
 
     @staticmethod
@@ -223,15 +226,15 @@ class Oracle:
         return [int(x) for x in out]
 
     # -- model -----------------------------------------------------------------
-    def pipe_time(self, F, B, xt, m: int, cost_mode: int = 0) -> float:
+    def pipe_time(self, F, B, xt, m: int, cost_mode: int = 0, schedule: int = 0) -> float:
         S = len(F)
         f = (C.c_double * S)(*F)
         b = (C.c_double * S)(*B)
         x = (C.c_double * S)(*(list(xt) + [0.0] * (S - len(xt))))
         sfx = "_i64" if cost_mode == 1 else "_f64"
-        return self._fn("orc_pipe_time", sfx)(S, m, f, b, x)
+        return self._fn("orc_pipe_time", sfx)(S, m, f, b, x, schedule)
 
-    def pipe(self, cuts: Sequence[int], m: int, devs: Sequence[int], n_sync: int, cost_mode: int = 0):
+    def pipe(self, cuts: Sequence[int], m: int, devs: Sequence[int], n_sync: int, cost_mode: int = 0, schedule: int = 0):
         """-> (feasible, cost as float, cost_ns, peak memory per stage)."""
         S = len(cuts) - 1
         c = np.ascontiguousarray(cuts, dtype=np.int32)
@@ -241,14 +244,14 @@ class Oracle:
         peak = np.zeros(S, dtype=np.int64)
         sfx = "_i64" if cost_mode == 1 else "_f64"
         ok = self._fn("orc_pipe", sfx)(C.byref(self._cp), S, _ptr(c, C.c_int32), m, _ptr(d, C.c_int32),
-                                       n_sync, C.byref(cost), C.byref(cost_ns), _ptr(peak, C.c_int64))
+                                       n_sync, C.byref(cost), C.byref(cost_ns), _ptr(peak, C.c_int64), schedule)
         return bool(ok), cost.value, cost_ns.value, [int(x) for x in peak]
 
-    def minmax(self, S: int, m: int, cost_mode: int = 0):
+    def minmax(self, S: int, m: int, cost_mode: int = 0, schedule: int = 0):
         cuts = np.zeros(S + 1, dtype=np.int32)
         val = C.c_double()
         sfx = "_i64" if cost_mode == 1 else "_f64"
-        ok = self._fn("orc_minmax", sfx)(C.byref(self._cp), S, m, _ptr(cuts, C.c_int32), C.byref(val))
+        ok = self._fn("orc_minmax", sfx)(C.byref(self._cp), S, m, _ptr(cuts, C.c_int32), C.byref(val), schedule)
         return bool(ok), [int(x) for x in cuts], val.value
 
     # -- search ----------------------------------------------------------------

@@ -24,6 +24,10 @@
 enum { ORC_REROUTE = 0, ORC_REDUNDANT = 1, ORC_DYNPAR = 2 };
 enum { ORC_LAYERS_FULL = 0, ORC_LAYERS_REMAINDER = 1, ORC_LAYERS_MINMAX = 2 };
 enum { ORC_BATCH_FULL = 0, ORC_BATCH_REMAINDER = 1 };
+/* Order of the computations on every stage: the dependency map f_2 of the transition equation
+ * (Section "Estimator").  1F1B = non-interleaved one-forward-one-backward; GPIPE = all forwards
+ * of the iteration, then all backwards. */
+enum { ORC_SCHED_1F1B = 0, ORC_SCHED_GPIPE = 1 };
 
 typedef struct {
     int32_t L, n_dp, n_pp, n_micro;
@@ -40,6 +44,7 @@ typedef struct {
     int32_t dp_lo, dp_hi, pp_lo, pp_hi;
     int32_t layer_mode, batch_mode;
     uint64_t kappa_cap;
+    int32_t schedule;   /* ORC_SCHED_* */
 } orc_opts;
 
 typedef struct {

@@ -37,14 +37,16 @@ static num_t nmax(num_t a, num_t b) { return a > b ? a : b; }
 typedef struct {
     const orc_profile *p;
     int L;
+    int schedule;      /* ORC_SCHED_*: order of the computations on every stage */
     num_t PF[ORC_MAX_LAYERS + 1], PB[ORC_MAX_LAYERS + 1];   /* time prefix sums  */
     int64_t PA[ORC_MAX_LAYERS + 1], PP[ORC_MAX_LAYERS + 1], PO[ORC_MAX_LAYERS + 1];
 } model;
 
 /* Prefix sums, accumulated left to right (PF[0]=0, PF[l+1]=PF[l]+f[l]). */
-static void model_init(model *M, const orc_profile *p) {
+static void model_init(model *M, const orc_profile *p, int schedule) {
     M->p = p;
     M->L = p->L;
+    M->schedule = schedule;
     M->PF[0] = 0; M->PB[0] = 0; M->PA[0] = 0; M->PP[0] = 0; M->PO[0] = 0;
     for (int l = 0; l < p->L; l++) {
 #if ORC_INT
@@ -87,11 +89,14 @@ static stage_t stage_of(const model *M, int lo, int hi) {
  * N_l (m_p + m_o + m_g) with m_g = m_p, plus (N_pp - i) micro-batches of activations
  * in flight, stage index from 0).  Per-layer bytes are summed over the stage instead
  * of using per-layer averages; the in-flight count is capped by the number of
- * micro-batches the pipeline runs (only matters when m < S).
+ * micro-batches the pipeline runs (only matters when m < S).  The (N_pp - i) count is
+ * that of the 1F1B order; under the all-forward-all-backward order (every stage runs its
+ * m forwards before its first backward) all m micro-batches are in flight at the peak.
  */
-static int64_t stage_peak_memory(const stage_t *s, int i, int S, int m) {
+static int64_t stage_peak_memory(const stage_t *s, int i, int S, int m, int schedule) {
     int inflight = S - i;
     if (m < inflight) inflight = m;
+    if (schedule == ORC_SCHED_GPIPE) inflight = m;
     return s->stat + (int64_t)inflight * s->A;
 }
 
@@ -103,15 +108,18 @@ static int64_t stage_peak_memory(const stage_t *s, int i, int S, int m) {
  * of the same stage and the computation it depends on in the neighbouring stage have
  * ended; a forward depends on the same micro-batch's forward one stage earlier, a
  * backward on the same micro-batch's backward one stage later (on its own forward at
- * the last stage).  The order of computations per stage is the non-interleaved 1F1B
- * order: w = min(S-1-i, m) warm-up forwards, then forward/backward pairs, then the
- * remaining backwards.  A transfer time xt[i] is paid on the boundary between stages
- * i and i+1 in both directions.
+ * the last stage).  The order of computations per stage -- the paper's f_2, "profiled
+ * from the actual execution order" -- is one of
+ *   ORC_SCHED_1F1B   non-interleaved 1F1B: w = min(S-1-i, m) warm-up forwards, then
+ *                    forward/backward pairs, then the remaining backwards;
+ *   ORC_SCHED_GPIPE  all forwards F_0..F_{m-1}, then all backwards B_0..B_{m-1}.
+ * A transfer time xt[i] is paid on the boundary between stages i and i+1 in both
+ * directions.
  *
  * Plain event simulation: sweep the stages and let each advance through its list while
  * the dependency of its next computation is known.
  */
-static num_t pipe_time(int S, int m, const num_t *F, const num_t *B, const num_t *xt) {
+static num_t pipe_time(int S, int m, const num_t *F, const num_t *B, const num_t *xt, int schedule) {
     const int n_ops = 2 * m;
     char *kind = (char *)malloc((size_t)S * n_ops);            /* 0 forward, 1 backward */
     int *mb = (int *)malloc(sizeof(int) * (size_t)S * n_ops);
@@ -125,6 +133,7 @@ static num_t pipe_time(int S, int m, const num_t *F, const num_t *B, const num_t
     for (int i = 0; i < S; i++) {
         int w = S - 1 - i;
         if (w > m) w = m;
+        if (schedule == ORC_SCHED_GPIPE) w = m;   /* every forward is a "warm-up" forward */
         int n = 0;
         for (int j = 0; j < w; j++) { kind[i * n_ops + n] = 0; mb[i * n_ops + n] = j; n++; }
         for (int k = 0; k < m - w; k++) {
@@ -225,13 +234,13 @@ static void pipe_eval(const model *M, int S, const stage_t *st, int m, const int
     *feasible = 0;
     if (m < 1) return;
     for (int i = 0; i < S; i++)
-        if (stage_peak_memory(&st[i], i, S, m) > M->p->mem_capacity_bytes) return;
+        if (stage_peak_memory(&st[i], i, S, m, M->schedule) > M->p->mem_capacity_bytes) return;
     for (int i = 0; i < S; i++) {
         F[i] = st[i].F;
         B[i] = st[i].B;
         xt[i] = (i < S - 1) ? transfer_time(st[i].X, link_bw(M->p, devs[i], devs[i + 1])) : 0;
     }
-    num_t t_pipe = pipe_time(S, m, F, B, xt);
+    num_t t_pipe = pipe_time(S, m, F, B, xt, M->schedule);
     num_t t_sync = 0;
     for (int i = 0; i < S; i++) t_sync = nmax(t_sync, sync_time(M->p, st[i].G, n_sync[i]));
     *cost = t_pipe + t_sync;
@@ -275,7 +284,7 @@ static int minmax_partition(const model *M, int S, int m, int32_t *cuts, num_t *
             num_t best = NUM_INF;
             for (int k = k_lo; k <= k_hi; k++) {
                 stage_t st = stage_of(M, k, l);
-                if (stage_peak_memory(&st, s - 1, S, m) > M->p->mem_capacity_bytes) continue;
+                if (stage_peak_memory(&st, s - 1, S, m, M->schedule) > M->p->mem_capacity_bytes) continue;
                 num_t W = st.F + st.B;
                 num_t prev = (s == 1) ? 0 : D[k][s - 1];
                 if (prev == NUM_INF) continue;
@@ -293,7 +302,7 @@ static int minmax_partition(const model *M, int S, int m, int32_t *cuts, num_t *
         int found = -1;
         for (int k = s - 1; k <= l - 1; k++) {
             stage_t st = stage_of(M, k, l);
-            if (stage_peak_memory(&st, s - 1, S, m) > M->p->mem_capacity_bytes) continue;
+            if (stage_peak_memory(&st, s - 1, S, m, M->schedule) > M->p->mem_capacity_bytes) continue;
             if (D[k][s - 1] == NUM_INF) continue;
             if (nmax(D[k][s - 1], st.F + st.B) == D[l][s]) { found = k; break; }
         }
@@ -475,7 +484,7 @@ static int micro_range(const space *sp, int si, int p, int *m_lo, int *m_hi) {
 static int space_build(space *sp, const orc_profile *prof, const orc_opts *o,
                        const uint32_t *failed, int n_failed) {
     memset(sp, 0, sizeof(*sp));
-    model_init(&sp->M, prof);
+    model_init(&sp->M, prof, o->schedule);
     sp->o = *o;
     int N = prof->n_dp * prof->n_pp;
     sp->G = prof->n_dp * prof->n_micro;
@@ -723,18 +732,18 @@ static num_t get_cost(const orc_plan *pl) {
 }
 
 /* Pipeline time of explicit stage times (tests pin this against the closed form). */
-double NAME(orc_pipe_time)(int S, int m, const double *F, const double *B, const double *xt) {
+double NAME(orc_pipe_time)(int S, int m, const double *F, const double *B, const double *xt, int schedule) {
     num_t f[ORC_MAX_STAGES], b[ORC_MAX_STAGES], x[ORC_MAX_STAGES];
     for (int i = 0; i < S; i++) { f[i] = (num_t)F[i]; b[i] = (num_t)B[i]; x[i] = (num_t)xt[i]; }
-    return (double)pipe_time(S, m, f, b, x);
+    return (double)pipe_time(S, m, f, b, x, schedule);
 }
 
 /* One pipeline from layer cuts on explicit devices; cost as double (exact for the
  * integer build below 2^53). Returns feasibility; peak memory per stage optional. */
 int NAME(orc_pipe)(const orc_profile *prof, int S, const int32_t *cuts, int m, const int32_t *devs,
-                   int n_sync, double *cost, int64_t *cost_ns, int64_t *peak_mem /* [S] or NULL */) {
+                   int n_sync, double *cost, int64_t *cost_ns, int64_t *peak_mem /* [S] or NULL */, int schedule) {
     model M;
-    model_init(&M, prof);
+    model_init(&M, prof, schedule);
     num_t c; int ok;
     int d[ORC_MAX_STAGES];
     for (int i = 0; i < S; i++) d[i] = devs[i];
@@ -742,16 +751,16 @@ int NAME(orc_pipe)(const orc_profile *prof, int S, const int32_t *cuts, int m, c
     if (peak_mem)
         for (int i = 0; i < S; i++) {
             stage_t st = stage_of(&M, cuts[i], cuts[i + 1]);
-            peak_mem[i] = stage_peak_memory(&st, i, S, m);
+            peak_mem[i] = stage_peak_memory(&st, i, S, m, schedule);
         }
     if (cost) *cost = ok ? (double)c : INFINITY;
     if (cost_ns) *cost_ns = ok ? (int64_t)c : INT64_MAX;
     return ok;
 }
 
-int NAME(orc_minmax)(const orc_profile *prof, int S, int m, int32_t *cuts, double *value) {
+int NAME(orc_minmax)(const orc_profile *prof, int S, int m, int32_t *cuts, double *value, int schedule) {
     model M;
-    model_init(&M, prof);
+    model_init(&M, prof, schedule);
     num_t v;
     int ok = minmax_partition(&M, S, m, cuts, &v);
     if (value) *value = ok ? (double)v : INFINITY;
@@ -823,7 +832,7 @@ void NAME(orc_search_policy)(const orc_profile *prof, const orc_opts *o, const u
         return;
     }
     model M;
-    model_init(&M, prof);
+    model_init(&M, prof, o ? o->schedule : ORC_SCHED_1F1B);
     num_t c; int ok;
     out->n_pipes = (uint32_t)prof->n_dp;
     for (int k = 0; k < prof->n_dp; k++) { out->stages[k] = (uint16_t)prof->n_pp; out->micro[k] = (uint16_t)prof->n_micro; }

@@ -28,6 +28,7 @@ POLICY_REROUTE, POLICY_REDUNDANT, POLICY_DYNPAR = 0, 1, 2
 COST_FP64, COST_INT64NS = 0, 1
 LAYERS_FULL, LAYERS_REMAINDER, LAYERS_MINMAX = 0, 1, 2
 BATCH_FULL, BATCH_REMAINDER = 0, 1
+SCHED_1F1B, SCHED_GPIPE = 0, 1
 
 
 class SplitMix64:
@@ -104,10 +105,15 @@ class SearchOptions:
     batch_mode: int
     kappa_cap: int
     cost_mode: int = COST_FP64
+    schedule: int = SCHED_1F1B
 
     def with_cost_mode(self, mode: int) -> "SearchOptions":
         return SearchOptions(self.dp_lo, self.dp_hi, self.pp_lo, self.pp_hi,
-                             self.layer_mode, self.batch_mode, self.kappa_cap, mode)
+                             self.layer_mode, self.batch_mode, self.kappa_cap, mode, self.schedule)
+
+    def with_schedule(self, schedule: int) -> "SearchOptions":
+        return SearchOptions(self.dp_lo, self.dp_hi, self.pp_lo, self.pp_hi,
+                             self.layer_mode, self.batch_mode, self.kappa_cap, self.cost_mode, schedule)
 
 
 @dataclass
