@@ -98,6 +98,15 @@ typedef struct {
     int64_t bw_intra_Bpns, bw_inter_Bpns;
 } cm_profile;
 
+/* Order of the computations on every stage: the dependency map f_2 of the start/end transition
+ * equation (Section "Estimator": "f_1(i), f_2(j) ... can be profiled from the actual execution
+ * order").  1F1B = non-interleaved one-forward-one-backward (min(S-1-i, m) warm-up forwards,
+ * forward/backward pairs, the remaining backwards; min(S-i, m) micro-batches of activations in
+ * flight at stage i, the paper's memory estimator).  GPIPE = all m forwards of the iteration,
+ * then all m backwards; all m micro-batches are in flight at every stage.  The order applies
+ * to every policy: rerouting and redundant computation are timed under it as well. */
+typedef enum { CM_SCHED_1F1B = 0, CM_SCHED_GPIPE = 1 } cm_schedule;
+
 /* Search window (Algorithm 1 inputs R_dp, R_pp) and enumeration modes.  A pipeline whose
  * enumerated layer compositions outnumber kappa_cap contributes only its min-max
  * partition. */
@@ -107,6 +116,7 @@ typedef struct {
     cm_batch_mode bm;
     uint64_t kappa_cap;
     cm_cost_mode cost;
+    cm_schedule sched;
 } cm_enum_opts;
 
 /* An execution plan (Definition 1: policy, parallel configuration, data distribution,

@@ -56,7 +56,8 @@ class cm_profile(C.Structure):
 
 class cm_enum_opts(C.Structure):
     _fields_ = [("dp_lo", C.c_int32), ("dp_hi", C.c_int32), ("pp_lo", C.c_int32), ("pp_hi", C.c_int32),
-                ("lm", C.c_int32), ("bm", C.c_int32), ("kappa_cap", C.c_uint64), ("cost", C.c_int32)]
+                ("lm", C.c_int32), ("bm", C.c_int32), ("kappa_cap", C.c_uint64), ("cost", C.c_int32),
+                ("sched", C.c_int32)]
 
 
 class cm_plan(C.Structure):
@@ -183,7 +184,8 @@ def _check(ctx, status: int, allow: Sequence[int] = ()):
 def _opts(o) -> cm_enum_opts:
     if isinstance(o, cm_enum_opts):
         return o
-    return cm_enum_opts(o.dp_lo, o.dp_hi, o.pp_lo, o.pp_hi, o.layer_mode, o.batch_mode, o.kappa_cap, o.cost_mode)
+    return cm_enum_opts(o.dp_lo, o.dp_hi, o.pp_lo, o.pp_hi, o.layer_mode, o.batch_mode, o.kappa_cap, o.cost_mode,
+                        int(getattr(o, "schedule", 0)))
 
 
 # ------------------------------------------------------------------ C-ABI level calls

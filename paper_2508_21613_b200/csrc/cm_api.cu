@@ -141,13 +141,17 @@ struct cm_ctx {
     std::vector<uint64_t> binom;      // [rows][kBinomCols+1]
     int binom_rows = 0;
     uint64_t *d_binom = nullptr;
-    uint8_t *d_mm[2] = {nullptr, nullptr};   // min-max cuts per cost mode
-    std::vector<uint8_t> mm_done[2];
+    // min-max cuts per (cost mode, execution order): the partition depends on the arithmetic of
+    // the stage times and, through the memory check, on the micro-batches in flight
+    static constexpr int kMmTables = 4;
+    static int mm_index(const cm_enum_opts &o) { return (int)o.cost * 2 + (int)o.sched; }
+    uint8_t *d_mm[kMmTables] = {nullptr, nullptr, nullptr, nullptr};
+    std::vector<uint8_t> mm_done[kMmTables];
     int mm_stride_m = 0;
     // Memory-feasible layer compositions per (layer mode, stages, micro-batches), listed once per
     // profile (cm_feasible_kernel) into one device pool that only grows; key = S << 16 | m.
     struct FeasEntry { uint32_t first, count; uint64_t K; };
-    std::map<uint32_t, FeasEntry> feas[3];
+    std::map<uint32_t, FeasEntry> feas[6];   // [layer mode * 2 + execution order]
     DevBuf<uint32_t> d_feas;
     size_t feas_used = 0;
     PinnedVec<unsigned char> feas_stage;      // keys, K, offsets out; counts back
@@ -270,6 +274,7 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
     if (o->lm < CM_LAYERS_FULL || o->lm > CM_LAYERS_MINMAX) return fail(ctx, CM_EINVAL, "bad layer mode");
     if (o->bm < CM_BATCH_FULL || o->bm > CM_BATCH_REMAINDER) return fail(ctx, CM_EINVAL, "bad batch mode");
     if (o->cost < CM_COST_FP64 || o->cost > CM_COST_INT64NS) return fail(ctx, CM_EINVAL, "bad cost mode");
+    if (o->sched < CM_SCHED_1F1B || o->sched > CM_SCHED_GPIPE) return fail(ctx, CM_EINVAL, "bad execution order");
     return CM_OK;
 }
 
@@ -388,7 +393,7 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
     const int L = hp.L, G = hp.G;
     const int dp_lo = std::max(1, (int)o.dp_lo), dp_hi = std::min((int)o.dp_hi, CM_MAX_PIPES);
     const int pp_lo = std::max(1, (int)o.pp_lo), pp_hi = std::min(std::min((int)o.pp_hi, L), CM_MAX_STAGES);
-    std::vector<uint8_t> &mm_done = ctx->mm_done[o.cost];
+    std::vector<uint8_t> &mm_done = ctx->mm_done[cm_ctx::mm_index(o)];
     Tmpl tp{};
     tp.strat_first = (uint32_t)bt.strat.size();
     tp.tseg_first = (uint32_t)bt.tseg.size();
@@ -501,7 +506,7 @@ cm_status grow_feas_pool(cm_ctx *ctx, size_t want) {
 cm_status ensure_feasible_lists(cm_ctx *ctx, Batch &bt) {
     const int lm = bt.opts.lm;
     if (lm == CM_LAYERS_MINMAX) return CM_OK;
-    std::map<uint32_t, cm_ctx::FeasEntry> &known = ctx->feas[lm];
+    std::map<uint32_t, cm_ctx::FeasEntry> &known = ctx->feas[lm * 2 + (int)bt.opts.sched];
     std::vector<uint32_t> new_keys;
     std::vector<uint64_t> new_K;
     std::vector<uint32_t> new_first;
@@ -717,7 +722,8 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
 Tables tables(const cm_ctx *ctx, const Batch &bt) {
     Tables t{};
     t.prof = bt.intval ? ctx->d_prof53 : ctx->d_prof; t.binom = ctx->d_binom; t.binom_rows = ctx->binom_rows;
-    t.mm_cuts = ctx->d_mm[bt.opts.cost]; t.mm_stride_m = ctx->mm_stride_m;
+    t.mm_cuts = ctx->d_mm[cm_ctx::mm_index(bt.opts)]; t.mm_stride_m = ctx->mm_stride_m;
+    t.sched = (int32_t)bt.opts.sched;
     return t;
 }
 
@@ -876,7 +882,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far, cm_ctx::Single 
 // Keys of min-max partitions that were scheduled but never computed must be asked for
 // again by the next batch.
 void forget_keys(cm_ctx *ctx, Batch &bt) {
-    std::vector<uint8_t> &done = ctx->mm_done[bt.opts.cost];
+    std::vector<uint8_t> &done = ctx->mm_done[cm_ctx::mm_index(bt.opts)];
     for (size_t i = 0; i < bt.keys.size(); ++i) {
         const uint32_t S = bt.keys[i] >> 16, m = bt.keys[i] & 0xffffu;
         done[(size_t)(S - 1) * ctx->mm_stride_m + m] = 0;
@@ -1061,7 +1067,7 @@ cm_status cm_destroy(cm_ctx *c) {
     if (c->d_prof) cudaFree(c->d_prof);
     if (c->d_prof53) cudaFree(c->d_prof53);
     if (c->d_binom) cudaFree(c->d_binom);
-    for (int i = 0; i < 2; ++i)
+    for (int i = 0; i < cm_ctx::kMmTables; ++i)
         if (c->d_mm[i]) cudaFree(c->d_mm[i]);
     delete c;
     return CM_OK;
@@ -1136,7 +1142,7 @@ static cm_status load_profile_host(cm_ctx *ctx, const cm_profile *p) {
     // min-max partition table, one row per (stages, micro-batches), per cost mode
     ctx->mm_stride_m = h.G + 2;
     const size_t slots = (size_t)CM_MAX_STAGES * ctx->mm_stride_m;
-    for (int i = 0; i < 2; ++i) ctx->mm_done[i].assign(slots, 0);
+    for (int i = 0; i < cm_ctx::kMmTables; ++i) ctx->mm_done[i].assign(slots, 0);
     return CM_OK;
 }
 
@@ -1164,7 +1170,7 @@ cm_status cm_load_profile(cm_ctx *ctx, const cm_profile *p) {
     CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_binom, ctx->binom.size() * sizeof(uint64_t)));
     CM_CUDA(ctx, cudaMemcpyAsync(ctx->d_binom, ctx->binom.data(), ctx->binom.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
     const size_t slots = (size_t)CM_MAX_STAGES * ctx->mm_stride_m;
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < cm_ctx::kMmTables; ++i) {
         if (ctx->d_mm[i]) { cudaFree(ctx->d_mm[i]); ctx->d_mm[i] = nullptr; }
         CM_CUDA(ctx, cudaMalloc((void **)&ctx->d_mm[i], slots * (kMaxS + 1)));
         CM_CUDA(ctx, cudaMemsetAsync(ctx->d_mm[i], 0xFF, slots * (kMaxS + 1), ctx->stream));
@@ -1710,7 +1716,7 @@ cm_status cm_decode_plan(cm_ctx *ctx, const cm_space *space, const cm_plan *plan
                 }
             } else {
                 uint8_t row[kMaxS + 1];
-                CM_CUDA(ctx, cudaMemcpyAsync(row, ctx->d_mm[bt.opts.cost] + ((size_t)(S - 1) * ctx->mm_stride_m + g.m) * (kMaxS + 1), kMaxS + 1,
+                CM_CUDA(ctx, cudaMemcpyAsync(row, ctx->d_mm[cm_ctx::mm_index(bt.opts)] + ((size_t)(S - 1) * ctx->mm_stride_m + g.m) * (kMaxS + 1), kMaxS + 1,
                                              cudaMemcpyDeviceToHost, ctx->stream));
                 CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
                 if (row[0] != 0) return fail(ctx, CM_EINVAL, "min-max partition of this pipeline is infeasible");

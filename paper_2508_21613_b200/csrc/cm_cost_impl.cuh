@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, Bat
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     const uint64_t chunk = (uint64_t)blockIdx.x;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
@@ -206,7 +206,7 @@ __device__ __forceinline__ bool uni_composition(const SProf<T> &sp, const Tables
     if (ok) {
         for (int i = lane; i < S; i += 32) {
             const int lo = cuts[i], hi = cuts[i + 1];
-            ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+            ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
             FB<T> d;
             d.f = sp.PF[hi] - sp.PF[lo];
             d.b = sp.PB[hi] - sp.PB[lo];
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
     __shared__ unsigned long long cells_w[kChunk / 32];
     extern __shared__ __align__(16) unsigned char dyn[];
     const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
     const int m = bk.m;
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
                 const int n_sync = g.n_sync;
                 __syncwarp();
                 const SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk> src{smem_addr(fb), smem_addr(xcol)};
-                const T t = sim_rounds<T, S>(m, src);
+                const T t = sim_stages<T, S>(sp.sched, m, src);
                 if (active) {
                     const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], n_sync, sp.bw_sync, sp.intval));
                     if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
@@ -321,7 +321,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, Batc
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
     const uint64_t base = (chunk - bk.chunk_first) * kChunk;
@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_w
     const Winner &w = bd.winner[b];
     if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;            // uniform over the CTA
     if (bd.tseg[w.seg[p]].S != S) return;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + threadIdx.x;
     T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + threadIdx.x;
     uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];

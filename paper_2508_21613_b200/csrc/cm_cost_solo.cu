@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_solo_kernel(Tables tb, BatchDe
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_solo_kernel(Tables tb, BatchDe
         if (ok)
             for (int i = lane; i < S; i += 32) {
                 const int lo = cuts[i], hi = cuts[i + 1];
-                ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+                ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
                 const long long gb = sp.PP[hi] - sp.PP[lo];
                 g_max = gb > g_max ? gb : g_max;
             }

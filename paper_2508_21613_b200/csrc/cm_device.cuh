@@ -76,11 +76,12 @@ template <typename T> struct SProf {
     T XT[2][kMaxL];
     long long cap, bw_sync;
     int L, n_dp, n_pp, n_micro;
-    int intval, pad;
+    int intval, sched;   // sched: order of the computations on a stage (cm_schedule), an option carried along
 };
 
 template <typename T>
-__device__ __forceinline__ void stage_profile(SProf<T> &s, const DevProfile *p) {
+__device__ __forceinline__ void stage_profile(SProf<T> &s, const Tables &tb) {
+    const DevProfile *p = tb.prof;
     const int L = p->L;
     for (int l = threadIdx.x; l <= L; l += blockDim.x) {
         s.PF[l] = Num<T>::PF(p)[l];
@@ -101,6 +102,7 @@ __device__ __forceinline__ void stage_profile(SProf<T> &s, const DevProfile *p) 
         s.n_pp = p->n_pp;
         s.n_micro = p->n_micro;
         s.intval = p->intval;
+        s.sched = tb.sched;
     }
 }
 
@@ -162,9 +164,33 @@ __device__ __forceinline__ void layer_cuts(const uint64_t *tab, int layer_mode, 
 // it has not consumed yet, transfer included).  xt[i] is the transfer time of the
 // boundary between stages i and i+1.
 // ----------------------------------------------------------------------------------
+// Under the all-forward-all-backward order (sched = CM_SCHED_GPIPE) the forwards run
+// micro-batch by micro-batch up the stages, then the backwards micro-batch by micro-batch
+// down the stages; the only state is the per-stage clock.
 template <typename T>
-__device__ __forceinline__ T sim_pipe(int S, int m, const T *F, const T *B, const T *xt, T *clock, T *pend) {
+__device__ __forceinline__ T sim_pipe(int S, int m, const T *F, const T *B, const T *xt, T *clock, T *pend, int sched) {
     for (int i = 0; i < S; ++i) clock[i] = (T)0;
+    if (sched == CM_SCHED_GPIPE) {
+        for (int j = 0; j < m; ++j) {
+            T chain = (T)0;
+            for (int i = 0; i < S; ++i) {
+                const T start = i > 0 ? tmax(clock[i], chain) : clock[i];
+                const T end = start + F[i];
+                clock[i] = end;
+                chain = end + xt[i];
+            }
+        }
+        for (int j = 0; j < m; ++j) {
+            T chain_b = (T)0;
+            for (int i = S - 1; i >= 0; --i) {
+                const T start = i < S - 1 ? tmax(clock[i], chain_b + xt[i]) : clock[i];
+                const T end = start + B[i];
+                clock[i] = end;
+                chain_b = end;
+            }
+        }
+        return clock[0];
+    }
     const int n_rows = m < S - 1 ? m : S - 1;
     for (int j = 0; j < n_rows; ++j) {
         T chain = (T)0;
@@ -201,10 +227,11 @@ __device__ __forceinline__ T sim_pipe(int S, int m, const T *F, const T *B, cons
 }
 
 // Peak memory of a stage at position i of S with m micro-batches (Section "Estimator",
-// memory estimator): static bytes + min(S - i, m) in-flight activations.
-__device__ __forceinline__ bool stage_fits(long long stat, long long act, int i, int S, int m, long long cap) {
+// memory estimator): static bytes + min(S - i, m) in-flight activations under 1F1B, all m of
+// them under the all-forward-all-backward order.
+__device__ __forceinline__ bool stage_fits(long long stat, long long act, int i, int S, int m, long long cap, int sched) {
     int inflight = S - i;
-    if (m < inflight) inflight = m;
+    if (m < inflight || sched == CM_SCHED_GPIPE) inflight = m;
     return stat + (long long)inflight * act <= cap;
 }
 
@@ -217,7 +244,7 @@ __device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, i
     for (int i = 0; i < S; ++i) {
         const int lo = cuts[i], hi = cuts[i + 1];
         if (hi <= lo) return false;
-        if (!stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap)) return false;
+        if (!stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched)) return false;
     }
     T F[kMaxS], B[kMaxS], xt[kMaxS], clock[kMaxS], pend[kMaxS];
     long long g_max = 0;
@@ -229,7 +256,7 @@ __device__ __forceinline__ bool pipe_cost_from_cuts(const SProf<T> &sp, int S, i
         long long g = sp.PP[hi] - sp.PP[lo];
         g_max = g > g_max ? g : g_max;
     }
-    T t = sim_pipe<T>(S, m, F, B, xt, clock, pend);
+    T t = sim_pipe<T>(S, m, F, B, xt, clock, pend, sp.sched);
     // the sync time is monotone in the gradient bytes, so max over stages = sync of the max
     cost = t + Num<T>::sync(g_max, n_sync, sp.bw_sync, sp.intval);
     return true;
@@ -399,13 +426,15 @@ __device__ __forceinline__ void init_kappa_sel(const BatchDev &bd, const Winner 
 // of a slot are gathered from the neighbours' state before any stage of the slot updates.
 // F, B, xt: the lane's own stages.  Returns the pipeline time in every lane.
 // ----------------------------------------------------------------------------------
+// Under the all-forward-all-backward order forward (i,j) sits at slot i+j and backward (i,j)
+// at slot (S+m-1) + (S-1-i) + j.
 template <typename T, int PER>
-__device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B, const T *xt) {
+__device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B, const T *xt, int sched) {
     const int lane = threadIdx.x & 31;
     T clock[PER], last_f[PER], last_b[PER];
 #pragma unroll
     for (int k = 0; k < PER; ++k) { clock[k] = (T)0; last_f[k] = (T)0; last_b[k] = (T)0; }
-    const int n_slots = 2 * (S + m) - 2;
+    const int n_slots = sched == CM_SCHED_GPIPE ? 2 * (S + m - 1) : 2 * (S + m) - 2;
     for (int s = 0; s < n_slots; ++s) {
         T f_in[PER], b_in[PER];
         const T up = __shfl_up_sync(0xffffffffu, last_f[PER - 1], 1);
@@ -421,14 +450,20 @@ __device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B
             if (i >= S) continue;
             bool is_f = false, is_b = false;
             const int d = s - i;
-            if (s <= S - 1) {
+            if (sched == CM_SCHED_GPIPE) {
                 is_f = d >= 0 && d < m;
-            } else if ((d & 1) == 0) {
-                const int j = d >> 1;
-                is_f = j > S - 1 - i && j < m;
+                const int e = s - (S + m - 1) - (S - 1 - i);
+                is_b = e >= 0 && e < m;
+            } else {
+                if (s <= S - 1) {
+                    is_f = d >= 0 && d < m;
+                } else if ((d & 1) == 0) {
+                    const int j = d >> 1;
+                    is_f = j > S - 1 - i && j < m;
+                }
+                const int e = s - (2 * S - 1 - i);
+                if (e >= 0 && (e & 1) == 0) is_b = (e >> 1) < m;
             }
-            const int e = s - (2 * S - 1 - i);
-            if (e >= 0 && (e & 1) == 0) is_b = (e >> 1) < m;
             if (is_f) {
                 const T start = i > 0 ? tmax(clock[k], f_in[k]) : clock[k];
                 clock[k] = start + F[k];
@@ -459,7 +494,7 @@ __device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *c
             if (i < S - 1) xt[k] = sp.XT[(tier >> i) & 1ull][hi - 1];
         }
     }
-    return sim_lockstep_n<T, PER>(S, m, F, B, xt);
+    return sim_lockstep_n<T, PER>(S, m, F, B, xt, sp.sched);
 }
 
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {

@@ -184,6 +184,7 @@ struct Tables {
     int32_t binom_rows;
     uint8_t *mm_cuts;           // [slots][kMaxS+1], min-max partitions; mm_cuts[slot][0]=255: infeasible
     int32_t mm_stride_m;        // slot = (S-1)*mm_stride_m + m
+    int32_t sched;              // cm_schedule of the batch / space these tables serve
     __host__ __device__ uint32_t mm_slot(int S, int m) const { return (uint32_t)((S - 1) * mm_stride_m + m); }
 };
 
@@ -223,7 +224,7 @@ inline bool native_i64(const BatchDev &b) { return b.mode == CM_COST_INT64NS && 
 
 // launchers (cm_kernels.cu); all enqueue on the stream and return the launch error
 cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st);
-cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);
+cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st);   // order: t.sched
 // feasible compositions of n_keys (S << 16 | m) keys: list of key q written at pool + first[q]
 // (room for K[q] + 1 entries), its length to count[q]
 cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *keys_dev, const uint64_t *K_dev,

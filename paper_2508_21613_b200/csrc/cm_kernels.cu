@@ -84,12 +84,12 @@ __global__ void __launch_bounds__(256) cm_minmax_kernel(Tables tb, const uint32_
             T best = INF;
             int best_k = 0;
             if (s == 1) {
-                if (lane == 0 && stage_fits(PS[l] - PS[0], PA[l] - PA[0], 0, S, m, cap))
+                if (lane == 0 && stage_fits(PS[l] - PS[0], PA[l] - PA[0], 0, S, m, cap, tb.sched))
                     best = (PF[l] - PF[0]) + (PB[l] - PB[0]);
             } else {
                 for (int k = s - 1 + lane; k <= l - 1; k += 32) {
                     if (prev[k] == INF) continue;
-                    if (!stage_fits(PS[l] - PS[k], PA[l] - PA[k], s - 1, S, m, cap)) continue;
+                    if (!stage_fits(PS[l] - PS[k], PA[l] - PA[k], s - 1, S, m, cap, tb.sched)) continue;
                     T w = (PF[l] - PF[k]) + (PB[l] - PB[k]);
                     T v = tmax(prev[k], w);
                     if (v < best) { best = v; best_k = k; }
@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(kFeasThreads) cm_feasible_kernel(Tables tb, in
             int lo = 0;
             for (int i = 0; i < S && ok; ++i) {
                 const int hi = cw.next();
-                ok = hi > lo && stage_fits(PS[hi] - PS[lo], PA[hi] - PA[lo], i, S, m, cap);
+                ok = hi > lo && stage_fits(PS[hi] - PS[lo], PA[hi] - PA[lo], i, S, m, cap, tb.sched);
                 lo = hi;
             }
         }
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
     __shared__ uint64_t red[kTile / 32];
     __shared__ SegView g;
     __shared__ uint64_t found_so_far;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     // grid.x runs over (scenario, pipeline), grid.y over tiles: CTAs are dispatched x-fastest,
     // so every segment's first tile is evaluated before anybody's second one and most later
     // tiles find their answer already there.
@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(128) cm_evaluate_kernel(Tables tb, BatchDev bd
                                                           const uint64_t *idx, uint64_t n_cand, double *cost,
                                                           int64_t *cost_ns, uint8_t *feas) {
     __shared__ SProf<T> sp;
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     __syncthreads();
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count) return;

@@ -41,7 +41,7 @@ cm_evaluate_argmin_kernel(Tables tb, BatchDev bd, uint64_t first, uint64_t count
     __shared__ bool is_last;
     unsigned long long *part_cost = scratch, *part_idx = scratch + kNoAllocMaxBlocks;
     unsigned int *arrived = reinterpret_cast<unsigned int *>(scratch + 2 * kNoAllocMaxBlocks);
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     __syncthreads();
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint64_t c = inf_bits<T>(), idx = ~0ull;

@@ -164,6 +164,17 @@ template <typename T, int S, typename Src> struct Rounds {
         clock[I] = bend;
         chain_b = bend;
     }
+    // forward of stage I fed through `chain` by the forward stage I-1 ran just before (the
+    // all-forward-all-backward order walks a micro-batch up the stages); stages I .. S-1
+    template <int I> __device__ __forceinline__ void fwd_up(T &chain) {
+        const T fstart = I > 0 ? tmax(clock[I], chain) : clock[I];
+        const T fend = fstart + src.template f<I>();
+        clock[I] = fend;
+        if constexpr (I < S - 1) {
+            chain = fend + src.template x<I>();
+            fwd_up<I + 1>(chain);
+        }
+    }
     // stages I, I-1, .., 0
     template <int I> __device__ __forceinline__ void fwd_down() { fwd<I>(); if constexpr (I > 0) fwd_down<I - 1>(); }
     template <int I> __device__ __forceinline__ void bwd_down(T &chain_b) { bwd<I>(chain_b); if constexpr (I > 0) bwd_down<I - 1>(chain_b); }
@@ -248,6 +259,30 @@ __device__ __forceinline__ T sim_rounds(int m, const Src &src) {
     }
 }
 
+// The all-forward-all-backward order (CM_SCHED_GPIPE): every micro-batch's forward runs up the
+// stages, then every micro-batch's backward runs down; the per-stage clock is all the state.
+template <typename T, int S, typename Src>
+__device__ __forceinline__ T sim_afab(int m, const Src &src) {
+    Rounds<T, S, Src> r(src);
+#pragma unroll 4
+    for (int j = 0; j < m; ++j) {
+        T chain = (T)0;
+        r.template fwd_up<0>(chain);
+    }
+#pragma unroll 4
+    for (int j = 0; j < m; ++j) {
+        T chain_b = (T)0;
+        r.template bwd_down<S - 1>(chain_b);
+    }
+    return r.clock[0];
+}
+
+// Pipeline time of S stages under the order `sched`, stage times from `src`.
+template <typename T, int S, typename Src>
+__device__ __forceinline__ T sim_stages(int sched, int m, const Src &src) {
+    return sched == CM_SCHED_GPIPE ? sim_afab<T, S>(m, src) : sim_rounds<T, S>(m, src);
+}
+
 // ----------------------------------------------------------------------------------
 // The same recurrence for shallow pipelines (S <= 16) with m >= S-1, where every stage
 // has its full warm-up: warm-up and cool-down are unrolled triangles without a single
@@ -326,7 +361,7 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
 #pragma unroll
     for (int i = 0; i < S; ++i) {
         const int hi = ok ? cw.next() : lo + 1;
-        ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+        ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
         st[i].f = sp.PF[hi] - sp.PF[lo];
         st[i].b = sp.PB[hi] - sp.PB[lo];
         xts[i] = i < S - 1 ? sp.XT[(g.tier >> i) & 1ull][hi - 1] : (T)0;
@@ -335,7 +370,14 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
         lo = hi;
     }
     if (!ok) return false;
-    cost = sim_regs<T, S>(m, st, xts) + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
+    T t;
+    if (sp.sched == CM_SCHED_GPIPE) {
+        const RegStages<T, S> src{st, xts};
+        t = sim_afab<T, S>(m, src);
+    } else {
+        t = sim_regs<T, S>(m, st, xts);
+    }
+    cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
     return true;
 }
 
@@ -355,7 +397,7 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
     int lo = 0;
     for (int i = 0; i < S && ok; ++i) {
         const int hi = cw.next();
-        ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap);
+        ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
         FB<T> d;
         d.f = sp.PF[hi] - sp.PF[lo];
         d.b = sp.PB[hi] - sp.PB[lo];
@@ -367,7 +409,7 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
     }
     if (!ok) return false;
     const SmemStages<T, (int)sizeof(FB<T>) * kChunk, (int)sizeof(T) * kChunk> src{smem_addr(fcol), smem_addr(xcol)};
-    const T t = sim_rounds<T, S>(m, src);
+    const T t = sim_stages<T, S>(sp.sched, m, src);
     cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
     return true;
 }

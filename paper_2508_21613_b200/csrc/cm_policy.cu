@@ -18,52 +18,7 @@
 
 namespace cm {
 
-// ----------------------------------------------------------------------------------
-// The recurrence with one stage per lane (S <= 32), in lock step over time slots.
-//
-// With unit durations the 1F1B schedule puts forward (i,j) at slot i+j while
-// j <= S-1-i and at slot i+2j afterwards, and backward (i,j) at slot 2S-1-i+2j.  Using
-// those slots as the evaluation order for arbitrary durations is a valid topological
-// order for every m >= 1: a stage runs at most one computation per slot, in its 1F1B
-// order, and what it depends on ran in an earlier slot and is still the neighbour's
-// latest result of that kind (the neighbour's next one comes in the same slot at the
-// earliest, and all lanes read before any lane writes).  So each lane keeps its clock,
-// its latest forward end (transfer added) and its latest backward end, and a slot costs
-// two shuffles and one cell.  Returns the pipeline time (the first stage's clock).
-// ----------------------------------------------------------------------------------
-template <typename T>
-__device__ __forceinline__ T sim_lockstep(int S, int m, T F, T B, T xt) {
-    const int i = threadIdx.x & 31;
-    T clock = (T)0, last_f = (T)0, last_b = (T)0;
-    const int n_slots = 2 * (S + m) - 2;
-    for (int s = 0; s < n_slots; ++s) {
-        const T f_in = __shfl_up_sync(0xffffffffu, last_f, 1);
-        const T b_in = __shfl_down_sync(0xffffffffu, last_b, 1);
-        if (i < S) {
-            bool is_f = false, is_b = false;
-            const int d = s - i;
-            if (s <= S - 1) {
-                is_f = d >= 0 && d < m;
-            } else if ((d & 1) == 0) {
-                const int j = d >> 1;
-                is_f = j > S - 1 - i && j < m;
-            }
-            const int e = s - (2 * S - 1 - i);
-            if (e >= 0 && (e & 1) == 0) is_b = (e >> 1) < m;
-            if (is_f) {
-                const T start = i > 0 ? tmax(clock, f_in) : clock;
-                clock = start + F;
-                last_f = clock + xt;
-            } else if (is_b) {
-                const T dep = i < S - 1 ? b_in + xt : clock;   // last stage: its own forward just ended
-                const T start = tmax(clock, dep);
-                clock = start + B;
-                last_b = clock;
-            }
-        }
-    }
-    return __shfl_sync(0xffffffffu, clock, 0);
-}
+// (the lock-step recurrence with one stage per lane is sim_lockstep_n<T, 1> of cm_device.cuh)
 
 template <typename T> __device__ __forceinline__ T warp_max(T v) {
     for (int o = 16; o > 0; o >>= 1) {
@@ -80,7 +35,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
     __shared__ uint64_t rc_bits[kMaxP];
     __shared__ uint16_t rc_S[kMaxP];
     const DevProfile *p = tb.prof;
-    stage_profile(sp, p);
+    stage_profile(sp, tb);
     for (int i = threadIdx.x; i <= p->n_pp; i += blockDim.x) base_cuts[i] = p->base_cuts[i];
     __syncthreads();
     const int b = blockIdx.x;
@@ -104,7 +59,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 T F = (T)0, B = (T)0, xt = (T)0, extra_i = (T)0, sync_i = (T)0;
                 if (i < S0) {
                     const int lo = base_cuts[i], hi = base_cuts[i + 1];
-                    ok = ok && fcnt < n_dp && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap);
+                    ok = ok && fcnt < n_dp && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap, sp.sched);
                     F = sp.PF[hi] - sp.PF[lo];
                     B = sp.PB[hi] - sp.PB[lo];
                     const int tier = (i / dpn == (i + 1) / dpn) ? 0 : 1;   // pipeline 0 sits on devices 0 .. S0-1
@@ -114,7 +69,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
-                    const T base = sim_lockstep<T>(S0, m, F, B, xt);
+                    const T base = sim_lockstep_n<T, 1>(S0, m, &F, &B, &xt, sp.sched);
                     const T t_sync = warp_max<T>(sync_i);
                     T extra = (T)0;   // summed in stage order, affected stages only
                     for (int s = 0; s < S0; ++s) {
@@ -132,7 +87,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 for (int i = 0; i < S0; ++i) ok = ok && fcnt[i] < n_dp;
                 for (int i = 0; i < S0 && ok; ++i) {
                     const int lo = base_cuts[i], hi = base_cuts[i + 1];
-                    ok = stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap);
+                    ok = stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S0, m, sp.cap, sp.sched);
                 }
                 if (ok) {
                     T extra = (T)0, t_sync = (T)0;
@@ -145,7 +100,7 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                         if (fcnt[i] > 0) extra = extra + Num<T>::reroute_extra(m * fcnt[i], Fs[i] + Bs[i], n_dp - fcnt[i], sp.intval);
                         t_sync = tmax(t_sync, Num<T>::sync(sp.PP[hi] - sp.PP[lo], n_dp - fcnt[i], sp.bw_sync, sp.intval));
                     }
-                    const T base = sim_pipe<T>(S0, m, Fs, Bs, xts, clk, pnd);
+                    const T base = sim_pipe<T>(S0, m, Fs, Bs, xts, clk, pnd, sp.sched);
                     out = Num<T>::bits((base + extra) + t_sync);
                 }
             }
@@ -198,11 +153,11 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                     act = act + act2;
                     xt = sp.XT[(dev / dpn == dev2 / dpn) ? 0 : 1][hi - 1];
                 }
-                fits = stage_fits(stat, act, j, S, m, sp.cap);
+                fits = stage_fits(stat, act, j, S, m, sp.cap, sp.sched);
             }
             ok = __all_sync(0xffffffffu, fits);
             if (ok) {
-                const T t = sim_lockstep<T>(S, m, f, bw, xt);
+                const T t = sim_lockstep_n<T, 1>(S, m, &f, &bw, &xt, sp.sched);
                 const long long g_max = warp_max<long long>(g);
                 bits = Num<T>::bits(t + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
             }
@@ -236,11 +191,11 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 }
                 Fs[i] = f;
                 Bs[i] = bw;
-                fits = stage_fits(stat, act, i, n, m, sp.cap);
+                fits = stage_fits(stat, act, i, n, m, sp.cap, sp.sched);
                 const long long gb = sp.PP[hi] - sp.PP[lo];
                 g_max = gb > g_max ? gb : g_max;
             }
-            if (fits) bits = Num<T>::bits(sim_pipe<T>(n, m, Fs, Bs, xts, clk, pnd) + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
+            if (fits) bits = Num<T>::bits(sim_pipe<T>(n, m, Fs, Bs, xts, clk, pnd, sp.sched) + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
         }
         if (wide) bits = __shfl_sync(0xffffffffu, bits, 0);
         if (lane == 0 && k < kMaxP) { rc_bits[k] = bits; rc_S[k] = (uint16_t)S; }

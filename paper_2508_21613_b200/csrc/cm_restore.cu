@@ -361,7 +361,7 @@ template <typename T>
 __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables tb, BatchDev bd, ObjDev od) {
     __shared__ SProf<T> sp;
     __shared__ RoundsWork work[kMatchWarps];
-    stage_profile(sp, tb.prof);
+    stage_profile(sp, tb);
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const size_t slot = (size_t)blockIdx.x * kMatchWarps + warp;

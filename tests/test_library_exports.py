@@ -53,6 +53,7 @@ def test_struct_layouts_match_the_header():
     assert binding.cm_plan.kappa.offset == 104
     assert ctypes.sizeof(binding.cm_enum_opts) == 40
     assert binding.cm_enum_opts.kappa_cap.offset == 24
+    assert binding.cm_enum_opts.cost.offset == 32 and binding.cm_enum_opts.sched.offset == 36
     assert ctypes.sizeof(binding.cm_profile) == 16 + 9 * 8 + 8 + 8 + 16
 
 
