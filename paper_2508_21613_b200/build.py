@@ -13,7 +13,7 @@ SOURCES = ["cm_cost_shallow_f64.cu", "cm_cost_shallow_i64.cu",
            "cm_kernels.cu", "cm_api.cu", "cm_policy.cu", "cm_noalloc.cu", "cm_cost.cu", "cm_cost_solo.cu", "cm_restore.cu", "cm_cache.cu"]
 # cm_cost_deep.cu is compiled once per cost type and range of stage counts (the ranges of
 # CM_DEEP_RANGES in cm_internal.h): (object suffix, extra flags)
-DEEP_RANGES = [(17, 28), (29, 34), (35, 41), (42, 48)]
+DEEP_RANGES = [(17, 28), (29, 34), (35, 41), (42, 48), (49, 56), (57, 64)]
 DEEP_UNITS = [(f"{tag}_{lo}_{hi}", [f"-DCM_DEEP_T={ctype}", f"-DCM_DEEP_LO={lo}", f"-DCM_DEEP_HI={hi}"])
               for lo, hi in DEEP_RANGES for tag, ctype in (("f64", "double"), ("i64", "long long"))]
 HEADERS = ["cm_internal.h", "cm_device.cuh", "cm_plan_eval.cuh", "cm_cost_impl.cuh"]

@@ -281,7 +281,7 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
 // Work layout of the search pass: the template segments of every template are grouped by
 // (stages, micro-batches) into buckets (a bucket's segments are its template segments
 // times the template's scenarios), buckets grouped into launch classes: one per
-// (kernel kind, stage count), the generic kernel takes the rest in one class.
+// (kernel kind, stage count); the short-pipeline and the one-plan kinds pool every depth in one class.
 cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket.clear();
     bt.classes.clear();
@@ -289,10 +289,10 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
     std::vector<Pre> pre;
     auto kind_of = [](int S, int m, uint64_t n_seg, uint64_t K) {
-        if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_GENERIC;
+        if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_SHORT;
         if (K == 0) return (int)CM_CLASS_SOLO;   // the min-max partition is the only candidate there is
         if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
-        return (int)CM_CLASS_GENERIC;
+        return (int)CM_CLASS_WIDE_UNI;           // deeper than kWideStagesMax: the transposed layout only
     };
     std::vector<uint32_t> idx;
     for (size_t t = 0; t < bt.tmpl.size(); ++t) {
@@ -337,7 +337,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     }
     for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_SOLO; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
-        const bool pooled_kind = kind == CM_CLASS_GENERIC || kind == CM_CLASS_SOLO;   // every depth in one class
+        const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO;   // every depth in one class
         LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
             LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};

@@ -11,7 +11,7 @@
 //       registers: stage forward/backward/transfer times, per-stage clock and pending
 //       forward; every loop over stages is unrolled, so a cell costs its two adds and one
 //       max and nothing else.
-//   cm_cost_wide_kernel<T, S, UNI>  S = 17..48.  Clock and pending forward stay in
+//   cm_cost_wide_kernel<T, S, UNI>  S = 17..64.  Up to 48 stages clock and pending forward stay in
 //       registers (4 S of them), the stage times move to shared memory.
 //       UNI = true ("transposed"): the 32 lanes of a warp take the SAME layer composition
 //       in 32 DIFFERENT segments of the bucket (they differ in link tiers and sync
@@ -19,7 +19,9 @@
 //       stage and round -- and memory feasibility is decided once per warp.
 //       UNI = false: one plan per lane as in the register kernel, stage times in a
 //       per-lane shared-memory column; for buckets with too few segments to transpose.
-//   cm_cost_generic_kernel<T>       any S <= CM_MAX_STAGES: per-stage state in local memory.
+//       S = 49..64 (transposed only): the pending forwards move to a per-lane shared-memory
+//       column as well; one CTA per SM.
+//   cm_cost_short_kernel<T>         S <= 16 with m < S-1: the rounds form, all in registers.
 #pragma once
 
 #include <atomic>
@@ -176,10 +178,14 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_any_kernel(Tables tb, Bat
 // deeper pipelines keep one item per warp -- their items are long enough to hide the CTA's
 // fixed cost, and their recurrence leaves no register for anything carried across it.
 #define CM_UNI_BATCH_STAGES kUniBatchStagesMax
+// Beyond kWideStagesMax stages the pending forwards move to a second per-lane column behind the
+// cuts (transposed layout only: a per-lane column of stage times as well would not fit).
 template <int S, bool UNI, typename T> constexpr size_t wide_smem_bytes() {
-    return UNI ? sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8)
+    return UNI ? sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8) +
+                     (S > kWideStagesMax ? sizeof(T) * S * kChunk : 0)
                : sizeof(FB<T>) * S * kChunk + sizeof(T) * S * kChunk;
 }
+template <int S> constexpr int wide_ctas_per_sm() { return S <= CM_WIDE3 ? 3 : (S <= kWideStagesMax ? 2 : 1); }
 
 // Transposed kernel, per warp item: the layer composition kappa of an (S, m) bucket is the same
 // in all 32 segments the warp evaluates, so its cuts, stage times and memory check are worked
@@ -223,7 +229,8 @@ __device__ __forceinline__ bool uni_composition(const SProf<T> &sp, const Tables
 }
 
 template <typename T, int S, bool UNI>
-__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset, int uni_items) {
+__global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_wide_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset, int uni_items) {
+    static_assert(UNI || S <= kWideStagesMax, "pipelines deeper than kWideStagesMax exist in the transposed layout only");
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -276,7 +283,15 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
                 const int n_sync = g.n_sync;
                 __syncwarp();
                 const SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk> src{smem_addr(fb), smem_addr(xcol)};
-                const T t = sim_stages<T, S>(sp.sched, m, src);
+                T t;
+                if constexpr (S <= kWideStagesMax) {
+                    t = sim_stages<T, S>(sp.sched, m, src);
+                } else {
+                    // 8-byte aligned column behind the four cut rows
+                    T *pcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + 4 * (((S + 1) + 7) / 8 * 8)) + tid;
+                    using ColPend = SmemPend<T, (int)sizeof(T) * kChunk>;
+                    t = sim_stages<T, S, SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk>, ColPend>(sp.sched, m, src, ColPend{smem_addr(pcol)});
+                }
                 if (active) {
                     const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], n_sync, sp.bw_sync, sp.intval));
                     if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
@@ -316,8 +331,10 @@ __global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_cost_wide_
     count_cells(&bd.counters[0], my_cells, cells_w);
 }
 
+// Shallow pipelines (<= 16 stages) with fewer micro-batches than warm-up slots (m < S-1): the
+// rounds form of the recurrence, state and stage times in registers, every such depth in one launch.
 template <typename T>
-__global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
+__global__ void __launch_bounds__(kChunk) cm_cost_short_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
     __shared__ SProf<T> sp;
     __shared__ unsigned long long cells_w[kChunk / 32];
     const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
@@ -335,7 +352,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_generic_kernel(Tables tb, Batc
         const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
         row = g.row;
         T cost;
-        if (segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost)) {
+        if (plan_cost_regs_any<T, true>(sp, tb, bd.layer_mode, g, kappa, cost)) {
             bits = Num<T>::bits(cost);
             my_cells = one_plan(2ull * g.S * g.m);
         }
@@ -376,7 +393,8 @@ static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const Lau
 
 template <typename T, int S>
 static cudaError_t launch_wide(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : launch_wide_one<T, S, false>(t, b, c, st);
+    if constexpr (S > kWideStagesMax) return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : cudaErrorInvalidValue;
+    else return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : launch_wide_one<T, S, false>(t, b, c, st);
 }
 
 
@@ -403,8 +421,8 @@ cudaError_t launch_shallow_any(const Tables &t, const BatchDev &b, uint32_t b0, 
 }
 
 template <typename T>
-cudaError_t launch_generic_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    cm_cost_generic_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+cudaError_t launch_short_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    cm_cost_short_kernel<T><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
     return cudaGetLastError();
 }
 
@@ -429,7 +447,7 @@ cudaError_t launch_deep_range(const Tables &t, const BatchDev &b, const LaunchCl
 // stage count; CTAs whose winner segment has another depth leave at once.
 // ----------------------------------------------------------------------------------
 template <typename T, int S>
-__global__ void __launch_bounds__(kChunk, (S <= CM_WIDE3) ? 3 : 2) cm_tiebreak_wide_kernel(Tables tb, BatchDev bd) {
+__global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_tiebreak_wide_kernel(Tables tb, BatchDev bd) {
     __shared__ SProf<T> sp;
     __shared__ uint64_t red[kChunk / 32];
     __shared__ SegView g;
@@ -494,7 +512,9 @@ static cudaError_t launch_tiebreak_wide_one(const Tables &t, const BatchDev &b, 
 
 template <typename T, int S, int HI>
 static cudaError_t tiebreak_dispatch(const Tables &t, const BatchDev &b, int stages, cudaStream_t st) {
-    if (stages == S) return launch_tiebreak_wide_one<T, S>(t, b, st);
+    if constexpr (S <= kWideStagesMax) {   // deeper winners are completed by the generic tie-break kernel
+        if (stages == S) return launch_tiebreak_wide_one<T, S>(t, b, st);
+    }
     if constexpr (S < HI) return tiebreak_dispatch<T, S + 1, HI>(t, b, stages, st);
     else return cudaSuccess;
 }

@@ -108,14 +108,15 @@ struct Bucket {
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
-enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_GENERIC = 3, CM_CLASS_SOLO = 4 };
+enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_SHORT = 3, CM_CLASS_SOLO = 4 };
+// CM_CLASS_SHORT: pipelines of at most kRegStagesMax stages with fewer micro-batches than warm-up slots (m < S-1).
 // CM_CLASS_SOLO: segments deeper than kRegStagesMax whose only candidate is the min-max partition.
 // One plan is one dependent chain (2*S*m cells, ~100 us in a single thread); a warp walks it in
 // lock step instead, stages over the lanes, four segments per CTA, every depth in one launch.
-constexpr int kWideStagesMax = 48;  // deepest pipeline with clock/pending state in registers
+constexpr int kWideStagesMax = 48;  // deepest pipeline with clock AND pending state in registers (deeper: pending forwards in shared memory)
 // Stage counts of the deep-pipeline kernels, cut into ranges that compile as separate
 // translation units (the build script passes the same pairs to cm_cost_deep.cu).
-#define CM_DEEP_RANGES(X) X(17, 28) X(29, 34) X(35, 41) X(42, 48)
+#define CM_DEEP_RANGES(X) X(17, 28) X(29, 34) X(35, 41) X(42, 48) X(49, 56) X(57, 64)
 constexpr int kUniMinSegments = 22; // fewer segments in a bucket (or left over after full warps of 32): the per-lane kernel
                                     // is faster than a transposed warp that is two-thirds empty
 constexpr int kAnyMaxChunks = 4096; // shallow classes smaller than this together: one launch for all depths

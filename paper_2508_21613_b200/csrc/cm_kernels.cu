@@ -361,10 +361,12 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
         if (first + threadIdx.x < count) {
             const uint64_t kappa = walk_kappa(bd.feas, g.feas_first, first + threadIdx.x);
             T cost;
-            // shallow pipelines take the register-resident evaluation, the rest the generic one
-            const bool ok = (g.S <= kRegStagesMax && g.m >= g.S - 1)
-                                ? plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost)
-                                : segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost);
+            // shallow pipelines take the register-resident evaluations, pipelines deeper than
+            // kWideStagesMax the local-memory one (the depths between: cm_tiebreak_wide_kernel)
+            bool ok;
+            if (g.S > kRegStagesMax) ok = segment_candidate_cost<T>(sp, tb, g, bd.layer_mode, kappa, cost);
+            else if (g.m >= g.S - 1) ok = plan_cost_regs_any<T>(sp, tb, bd.layer_mode, g, kappa, cost);
+            else ok = plan_cost_regs_any<T, true>(sp, tb, bd.layer_mode, g, kappa, cost);
             if (ok && Num<T>::bits(cost) <= w.cost_bits) hit = kappa;
         }
         hit = warp_min_u64(hit);

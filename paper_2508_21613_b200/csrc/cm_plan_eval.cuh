@@ -122,22 +122,45 @@ template <typename T, int S> struct RegStages {
     template <int I> __device__ __forceinline__ T x() const { return xt[I]; }
 };
 
+// Where a pipeline's pending forwards live (one value per stage, written by the stage below,
+// read one round later): in registers up to kWideStagesMax stages, beyond that in a per-lane
+// shared-memory column (element i at byte offset i * STRIDE), because clock and pend of 64
+// stages do not fit the register file of a thread.  Entries are written before they are read.
+template <typename T, int S> struct RegPend {
+    T v[S];
+    template <int I> __device__ __forceinline__ T get() const { return v[I]; }
+    template <int I> __device__ __forceinline__ void set(T x) { v[I] = x; }
+};
+template <typename T, int STRIDE> struct SmemPend {
+    unsigned base;
+    template <int I> __device__ __forceinline__ T get() const {
+        unsigned long long a;
+        asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(a) : "r"(base), "n"(I * STRIDE) : "memory");
+        return Num<T>::from_bits(a);
+    }
+    template <int I> __device__ __forceinline__ void set(T x) const {
+        asm volatile("st.shared.b64 [%0+%1], %2;" : : "r"(base), "n"(I * STRIDE), "l"(Num<T>::bits(x)) : "memory");
+    }
+};
+
 // State and cells of one pipeline of S stages (S compile-time): clock = end of the stage's
 // latest computation, pend = end of the forward the stage has not consumed yet (transfer
 // included).  Every method takes its stage as a template argument.
-template <typename T, int S, typename Src> struct Rounds {
-    T clock[S], pend[S];
+template <typename T, int S, typename Src, typename Pend = RegPend<T, S>> struct Rounds {
+    T clock[S];
+    Pend pend;
     const Src &src;
-    __device__ __forceinline__ explicit Rounds(const Src &s) : src(s) {
+    __device__ __forceinline__ explicit Rounds(const Src &s, Pend p = Pend()) : pend(p), src(s) {
 #pragma unroll
-        for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
+        for (int i = 0; i < S; ++i) clock[i] = (T)0;
     }
     // forward of stage I: fed by the forward stage I-1 ran one round earlier
     template <int I> __device__ __forceinline__ void fwd() {
-        const T fstart = I > 0 ? tmax(clock[I], pend[I]) : clock[I];
+        T fstart = clock[I];
+        if constexpr (I > 0) fstart = tmax(fstart, pend.template get<I>());
         const T fend = fstart + src.template f<I>();
         clock[I] = fend;
-        if constexpr (I < S - 1) pend[I + 1] = fend + src.template x<I>();
+        if constexpr (I < S - 1) pend.template set<I + 1>(fend + src.template x<I>());
     }
     // backward of stage I: fed by the backward stage I+1 ran just before in the same round
     // (chain_b), at the last stage by its own forward, which is what clock holds there
@@ -152,12 +175,13 @@ template <typename T, int S, typename Src> struct Rounds {
     // forward then backward of stage I (a steady round)
     template <int I> __device__ __forceinline__ void both(T &chain_b) {
         const FB<T> d = src.template stage<I>();
-        const T fstart = I > 0 ? tmax(clock[I], pend[I]) : clock[I];
+        T fstart = clock[I];
+        if constexpr (I > 0) fstart = tmax(fstart, pend.template get<I>());
         const T fend = fstart + d.f;
         T bstart = fend;
         if constexpr (I < S - 1) {
             const T x = src.template x<I>();
-            pend[I + 1] = fend + x;
+            pend.template set<I + 1>(fend + x);
             bstart = tmax(fend, chain_b + x);
         }
         const T bend = bstart + d.b;
@@ -224,9 +248,9 @@ template <typename T, int S, typename Src> struct Rounds {
 // backwards (within a round the forwards depend only on the round before, so they may all
 // precede the backwards).  With fewer micro-batches the ramp rounds test every stage.
 // ----------------------------------------------------------------------------------
-template <typename T, int S, typename Src>
-__device__ __forceinline__ T sim_rounds(int m, const Src &src) {
-    Rounds<T, S, Src> r(src);
+template <typename T, int S, typename Src, typename Pend = RegPend<T, S>>
+__device__ __forceinline__ T sim_rounds(int m, const Src &src, Pend pend = Pend()) {
+    Rounds<T, S, Src, Pend> r(src, pend);
     if constexpr (S == 1) {
         for (int t = 0; t < m; ++t) { T chain_b = (T)0; r.template both<0>(chain_b); }
         return r.clock[0];
@@ -278,9 +302,9 @@ __device__ __forceinline__ T sim_afab(int m, const Src &src) {
 }
 
 // Pipeline time of S stages under the order `sched`, stage times from `src`.
-template <typename T, int S, typename Src>
-__device__ __forceinline__ T sim_stages(int sched, int m, const Src &src) {
-    return sched == CM_SCHED_GPIPE ? sim_afab<T, S>(m, src) : sim_rounds<T, S>(m, src);
+template <typename T, int S, typename Src, typename Pend = RegPend<T, S>>
+__device__ __forceinline__ T sim_stages(int sched, int m, const Src &src, Pend pend = Pend()) {
+    return sched == CM_SCHED_GPIPE ? sim_afab<T, S>(m, src) : sim_rounds<T, S, Src, Pend>(m, src, pend);
 }
 
 // ----------------------------------------------------------------------------------
@@ -348,7 +372,9 @@ __device__ __forceinline__ T sim_regs(int m, const FB<T> (&st)[S], const T (&xt)
 // Cost of pipeline-plan kappa of a segment with S <= kRegStagesMax stages and m >= S-1
 // micro-batches, everything in registers.  Returns false if the plan is infeasible.
 // ----------------------------------------------------------------------------------
-template <typename T, int S>
+// ANY_M = true lifts the condition on m: the rounds form of the recurrence (any m >= 1) instead
+// of the unrolled triangles -- for the few segments with fewer micro-batches than warm-up slots.
+template <typename T, int S, bool ANY_M = false>
 __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables &tb, int layer_mode,
                                                const SegView &g, uint64_t kappa, T &cost) {
     const int m = g.m;
@@ -371,7 +397,11 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
     }
     if (!ok) return false;
     T t;
-    if (sp.sched == CM_SCHED_GPIPE) {
+    if constexpr (ANY_M) {
+        if (m < 1) return false;
+        const RegStages<T, S> src{st, xts};
+        t = sim_stages<T, S>(sp.sched, m, src);
+    } else if (sp.sched == CM_SCHED_GPIPE) {
         const RegStages<T, S> src{st, xts};
         t = sim_afab<T, S>(m, src);
     } else {
@@ -415,12 +445,13 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
 }
 
 // The same with S chosen at run time (one kernel for every shallow depth; used where the
-// work is too small to be worth one launch per depth).  Caller guarantees 1 <= S <= 16, m >= S-1.
-template <typename T>
+// work is too small to be worth one launch per depth).  Caller guarantees 1 <= S <= 16, and
+// m >= S-1 unless ANY_M.
+template <typename T, bool ANY_M = false>
 __device__ __forceinline__ bool plan_cost_regs_any(const SProf<T> &sp, const Tables &tb, int layer_mode,
                                                    const SegView &g, uint64_t kappa, T &cost) {
     switch (g.S) {
-#define CM_CASE(S) case S: return plan_cost_regs<T, S>(sp, tb, layer_mode, g, kappa, cost);
+#define CM_CASE(S) case S: return plan_cost_regs<T, S, ANY_M>(sp, tb, layer_mode, g, kappa, cost);
         CM_CASE(1) CM_CASE(2) CM_CASE(3) CM_CASE(4) CM_CASE(5) CM_CASE(6) CM_CASE(7) CM_CASE(8)
         CM_CASE(9) CM_CASE(10) CM_CASE(11) CM_CASE(12) CM_CASE(13) CM_CASE(14) CM_CASE(15) CM_CASE(16)
 #undef CM_CASE
