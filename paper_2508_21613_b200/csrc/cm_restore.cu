@@ -80,21 +80,36 @@ cudaError_t launch_shortlist(const Tables &t, const BatchDev &b, const ObjDev &o
 }
 
 // ----------------------------------------------------------------------------------
-// Minimum-cost perfect matching, one warp per problem (Kuhn-Munkres in its potentials /
-// shortest-augmenting-path form).  Rows = devices with their old layer range, columns =
-// positions with their new range.  Rows enter one at a time; for the new row an
-// alternating tree is grown column by column over the reduced costs
-// cost(i,j) - u[i] - v[j], potentials are shifted so that tree edges stay tight, and the
-// matching is flipped along the path to the first free column.  Every loop is bounded by
-// the problem size: the tree gains a column per step and a free column always exists.
+// Minimum-cost perfect matching, one warp per problem.  Rows = devices with their old layer
+// range, columns = positions with their new range, Cost[i][j] = range_cost below.
+//
+// Devices that hold the same old range are interchangeable (the survivors of one old stage: up
+// to N_dp of them), so the rows are first folded into CLASSES with a capacity, and the problem
+// is solved as a transportation problem by successive shortest augmenting paths with
+// potentials (Kuhn-Munkres, columns entering one at a time): u per class, v per column, reduced
+// cost Cost - u - v >= 0.  For an entering column an alternating tree grows over classes;
+// scanning a tree column is ONE cost evaluation per lane (lane = class), a class whose slack
+// reaches zero joins the tree in the same pass as every other such class, and with it the
+// columns it currently serves; only when nothing is tight do the potentials move by the least
+// slack, which costs the warp-wide reduction.  The first class with spare capacity ends the
+// search and the matching is flipped along the path.  Every loop is bounded by the problem
+// size.  Lane `lane` owns classes c*32+lane, c < NC.
 // ----------------------------------------------------------------------------------
 constexpr int kMatchWarps = 4;
 
 struct MatchWork {
-    long long u[kMaxMatch];                       // row potentials
-    short match[kMaxMatch], prev[kMaxMatch];      // row of a column (-1 = free); previous column on the path
-    int row_col[kMaxMatch];                       // column of a row (-1 = free); claimed with atomicCAS
-    uint8_t olo[kMaxMatch], ohi[kMaxMatch], nlo[kMaxMatch], nhi[kMaxMatch];
+    long long v[kMaxMatch];                       // column potentials
+    long long tbase[kMaxMatch];                   // tree columns: potential shift already applied when they joined
+    int cnt[kMaxMatch];                           // class: columns it serves now
+    int head[kMaxMatch];                          // class: first column of its list (-1 = none)
+    short cap[kMaxMatch];                         // class: rows folded into it
+    short way[kMaxMatch];                         // class: tree column that gave its least slack
+    short next_col[kMaxMatch];                    // column: next column served by the same class
+    short tcol[kMaxMatch];                        // tree columns in the order they joined
+    short row_class[kMaxMatch];                   // row -> class
+    short match[kMaxMatch];                       // column -> class while solving; column -> row on return
+    uint8_t olo[kMaxMatch], ohi[kMaxMatch], nlo[kMaxMatch], nhi[kMaxMatch];   // inputs
+    uint8_t clo[kMaxMatch], chi[kMaxMatch];       // class ranges
 };
 
 __device__ __forceinline__ long long range_cost(const long long *PW, long long need, int a, int b, int x, int y) {
@@ -102,122 +117,208 @@ __device__ __forceinline__ long long range_cost(const long long *PW, long long n
     return need - (hi > lo ? PW[hi] - PW[lo] : 0ll);
 }
 
+// warp minimum of a non-negative 64-bit value: two hardware min-reductions
+__device__ __forceinline__ long long warp_min_nonneg(long long x) {
+    const uint32_t hi = (uint32_t)((unsigned long long)x >> 32), lo = (uint32_t)x;
+    const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+    const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+    return (long long)(((unsigned long long)mhi << 32) | mlo);
+}
+
 // Returns the total of the matching (same value in every lane), -1 if the iteration broke
-// down (cannot happen for n >= 1; guards the loops).  w.match[j] = row of column j.
-// Lane `lane` owns the columns c*32+lane, c < NC, and keeps their range, column potential
-// and slack in registers; rows are read from shared memory (same address in every lane).
+// down (cannot happen for n >= 1; guards the loops).  On return w.match[j] = row of column j.
 template <int NC>
 __device__ long long warp_match(MatchWork &w, const long long *PW, int n, int lane) {
     const long long INF = LLONG_MAX / 4;
-    long long v[NC], slack[NC], need[NC];
-    int nlo[NC], nhi[NC];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        const int j = c * 32 + lane;
-        nlo[c] = j < n ? (int)w.nlo[j] : 0;
-        nhi[c] = j < n ? (int)w.nhi[j] : 0;
-        need[c] = nhi[c] > nlo[c] ? PW[nhi[c]] - PW[nlo[c]] : 0ll;
-        v[c] = INF;
-        if (j < n) { w.u[j] = 0; w.match[j] = -1; w.row_col[j] = -1; }
+    // ---- fold equal rows into classes, numbered by their first row
+    for (int i = lane; i < n; i += 32) {
+        int first = i;
+        for (int k = 0; k < i; ++k)
+            if (w.olo[k] == w.olo[i] && w.ohi[k] == w.ohi[i]) { first = k; break; }
+        w.tcol[i] = (short)first;                 // scratch: first row of i's class
+        w.cap[i] = 0; w.cnt[i] = 0; w.head[i] = -1; w.match[i] = -1; w.next_col[i] = -1;
     }
     __syncwarp();
-    // Start from feasible potentials instead of zeros: v[j] = the cheapest row of column j
-    // (u = 0), then every column claims a free row that attains it, scanning rows upwards.
-    // Most positions find a device that already holds most of their layers, so few rows are
-    // left for the augmenting phase.
-    for (int i = 0; i < n; ++i) {
-        const int a = w.olo[i], b = w.ohi[i];
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            const long long cost = range_cost(PW, need[c], a, b, nlo[c], nhi[c]);
-            v[c] = cost < v[c] ? cost : v[c];
+    int R = 0;
+    for (int base = 0; base < n; base += 32) {
+        const int i = base + lane;
+        const bool is_first = i < n && w.tcol[i] == i;
+        const uint32_t mask = __ballot_sync(0xffffffffu, is_first);
+        if (is_first) {
+            const int r = R + __popc(mask & ((1u << lane) - 1u));
+            w.row_class[i] = (short)r;
+            w.clo[r] = w.olo[i];
+            w.chi[r] = w.ohi[i];
         }
+        R += __popc(mask);
     }
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        const int j = c * 32 + lane;
-        if (j >= n) continue;
-        for (int i = 0; i < n; ++i) {
-            if (range_cost(PW, need[c], w.olo[i], w.ohi[i], nlo[c], nhi[c]) != v[c]) continue;
-            if (atomicCAS(&w.row_col[i], -1, j) == -1) { w.match[j] = (short)i; break; }
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) {
+        const int r = w.row_class[w.tcol[i]];
+        if (w.tcol[i] != i) w.row_class[i] = (short)r;
+        atomicAdd(&w.cnt[r], 1);                  // counted in cnt, moved to cap below
+    }
+    __syncwarp();
+    for (int r = lane; r < R; r += 32) { w.cap[r] = (short)w.cnt[r]; w.cnt[r] = 0; }
+    __syncwarp();
+    // ---- start: v[j] = cheapest class of column j (u = 0), then every column claims a class that
+    // attains it and still has room, lowest class first.  Most positions find a device that
+    // already holds most of their layers, so few columns are left for the augmenting phase.
+    for (int j = lane; j < n; j += 32) {
+        const int x = w.nlo[j], y = w.nhi[j];
+        const long long need = y > x ? PW[y] - PW[x] : 0ll;
+        long long best = INF;
+        for (int r = 0; r < R; ++r) {
+            const long long c = range_cost(PW, need, w.clo[r], w.chi[r], x, y);
+            best = c < best ? c : best;
+        }
+        w.v[j] = best;
+        for (int r = 0; r < R; ++r) {
+            if (range_cost(PW, need, w.clo[r], w.chi[r], x, y) != best) continue;
+            if (atomicAdd(&w.cnt[r], 1) < (int)w.cap[r]) {
+                w.match[j] = (short)r;
+                w.next_col[j] = (short)atomicExch(&w.head[r], j);
+                break;
+            }
+            atomicSub(&w.cnt[r], 1);
         }
     }
     __syncwarp();
+    // ---- augmenting phase: class potentials and slacks in registers of the owning lane
+    long long u[NC], slack[NC], ubase[NC];
+    int clo[NC], chi[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int r = c * 32 + lane;
+        u[c] = 0;
+        clo[c] = r < R ? (int)w.clo[r] : 0;
+        chi[c] = r < R ? (int)w.chi[r] : 0;
+    }
     bool broken = false;
-    for (int r = 0; r < n && !broken; ++r) {
-        if (w.row_col[r] >= 0) continue;           // uniform: already matched by the start-up pass
+    for (int j0 = 0; j0 < n && !broken; ++j0) {
+        if (w.match[j0] >= 0) continue;             // uniform: served since the start or an earlier flip
+        uint32_t tree = 0;                          // bit c: class c*32+lane belongs to the tree
+        long long D = 0;                            // potential shift so far
+        int nt = 1, scanned = 0, found = -1;
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            slack[c] = INF;
-            if (c * 32 + lane < n) w.prev[c * 32 + lane] = (short)n;
-        }
-        uint32_t tree = 0;            // bit c: column c*32+lane belongs to the tree
-        int col = n, row = r;         // column n is the root and holds the new row
-        for (int step = 0; step <= n; ++step) {
-            const int a = w.olo[row], b = w.ohi[row];
-            const long long ur = w.u[row];
-            long long delta = INF;
-            int next = n;
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-                const int j = c * 32 + lane;
-                if (j >= n || ((tree >> c) & 1u)) continue;
-                const long long red = range_cost(PW, need[c], a, b, nlo[c], nhi[c]) - ur - v[c];
-                if (red < slack[c]) { slack[c] = red; w.prev[j] = (short)col; }
-                if (slack[c] < delta) { delta = slack[c]; next = j; }
-            }
-            // warp argmin of (slack, column), lowest column on ties: three hardware min-reductions
-            // (high word, low word among the lanes that hold the least high word, column among
-            // the lanes that hold the least slack); slacks are never negative
-            {
-                const uint32_t hi = (uint32_t)((unsigned long long)delta >> 32), lo = (uint32_t)delta;
-                const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-                const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-                const bool least = hi == mhi && lo == mlo;
-                next = (int)__reduce_min_sync(0xffffffffu, least ? (uint32_t)next : 0xffffffffu);
-                delta = (long long)(((unsigned long long)mhi << 32) | mlo);
-            }
-            if (next >= n) { broken = true; break; }
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-                const int j = c * 32 + lane;
-                if (j >= n) continue;
-                if ((tree >> c) & 1u) { w.u[w.match[j]] += delta; v[c] -= delta; }
-                else slack[c] -= delta;
-            }
-            if (lane == 0) w.u[r] += delta;
-            __syncwarp();
-            col = next;
-            if ((col & 31) == lane) tree |= 1u << (col >> 5);
-            row = w.match[col];
-            if (row < 0) break;
-        }
-        if (row >= 0) broken = true;   // step bound hit without reaching a free column
-        // every lane must have read match[col] above before lane 0 rewrites the matching:
-        // a lane that sees the flipped entry would take the free column for a matched one
+        for (int c = 0; c < NC; ++c) slack[c] = INF;
+        if (lane == 0) { w.tcol[0] = (short)j0; w.tbase[0] = 0; }
         __syncwarp();
-        if (!broken && lane == 0) {
-            int c = col;
-            for (int step = 0; step <= n && c != n; ++step) {
-                const int p = w.prev[c];
-                w.match[c] = p == n ? (short)r : w.match[p];
-                c = p;
+        for (int iter = 0; iter <= 2 * (n + R) + 4 && found < 0; ++iter) {
+            // 1. scan the tree columns that have not been scanned yet
+            for (; scanned < nt; ++scanned) {
+                const int j = w.tcol[scanned];
+                const int x = w.nlo[j], y = w.nhi[j];
+                const long long need = y > x ? PW[y] - PW[x] : 0ll;
+                const long long vj = w.v[j];
+#pragma unroll
+                for (int c = 0; c < NC; ++c) {
+                    const int r = c * 32 + lane;
+                    if (r >= R || ((tree >> c) & 1u)) continue;
+                    const long long red = range_cost(PW, need, clo[c], chi[c], x, y) - u[c] - vj;
+                    if (red < slack[c]) { slack[c] = red; w.way[r] = (short)j; }
+                }
+            }
+            // 2. classes at zero slack join the tree; one with room ends the search, a full one
+            // brings the columns it serves
+            bool any_tight = false;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int r = c * 32 + lane;
+                const bool tight = r < R && !((tree >> c) & 1u) && slack[c] == 0;
+                uint32_t mask = __ballot_sync(0xffffffffu, tight);
+                if (tight) { tree |= 1u << c; ubase[c] = D; }
+                any_tight = any_tight || mask != 0;
+                while (mask && found < 0) {
+                    const int rr = c * 32 + (__ffs((int)mask) - 1);
+                    mask &= mask - 1;
+                    if (w.cnt[rr] < (int)w.cap[rr]) { found = rr; break; }      // uniform
+                    int j = w.head[rr];
+                    for (int k = 0; k <= n && j >= 0; ++k) {
+                        if (nt >= kMaxMatch) { broken = true; break; }
+                        if (lane == 0) { w.tcol[nt] = (short)j; w.tbase[nt] = D; }
+                        ++nt;
+                        j = w.next_col[j];
+                    }
+                }
+            }
+            __syncwarp();
+            if (found >= 0 || broken) break;
+            if (any_tight) continue;
+            // 3. nothing tight: shift the potentials by the least slack outside the tree
+            long long delta = INF;
+#pragma unroll
+            for (int c = 0; c < NC; ++c)
+                if (c * 32 + lane < R && !((tree >> c) & 1u) && slack[c] < delta) delta = slack[c];
+            delta = warp_min_nonneg(delta);
+            if (delta >= INF) { broken = true; break; }   // every class is in the tree and full: cannot happen
+            D += delta;
+#pragma unroll
+            for (int c = 0; c < NC; ++c)
+                if (!((tree >> c) & 1u)) slack[c] -= delta;
+        }
+        if (found < 0) broken = true;
+        if (broken) break;
+        // potentials: tree columns rose, tree classes fell, each by the shift since it joined
+        for (int k = lane; k < nt; k += 32) w.v[w.tcol[k]] += D - w.tbase[k];
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+            if ((tree >> c) & 1u) u[c] -= D - ubase[c];
+        __syncwarp();
+        // flip along the path: class `found` takes the column that reached it, the class that
+        // served this column before takes the one that reached it, ... down to the new column
+        if (lane == 0) {
+            int r = found;
+            for (int step = 0; step <= n; ++step) {
+                const int j = w.way[r];
+                const int old = w.match[j];
+                if (old >= 0) {     // unlink j from the class that served it
+                    int q = w.head[old];
+                    if (q == j) w.head[old] = w.next_col[j];
+                    else
+                        for (int k = 0; k <= n && q >= 0; ++k) {
+                            const int nx = w.next_col[q];
+                            if (nx == j) { w.next_col[q] = w.next_col[j]; break; }
+                            q = nx;
+                        }
+                    --w.cnt[old];
+                }
+                w.match[j] = (short)r;
+                w.next_col[j] = (short)w.head[r];
+                w.head[r] = j;
+                ++w.cnt[r];
+                if (old < 0) break;
+                r = old;
             }
         }
         __syncwarp();
     }
     if (broken) return -1;
     long long total = 0;
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        const int j = c * 32 + lane;
-        if (j < n) { const int i = w.match[j]; total += range_cost(PW, need[c], w.olo[i], w.ohi[i], nlo[c], nhi[c]); }
+    for (int j = lane; j < n; j += 32) {
+        const int r = w.match[j], x = w.nlo[j], y = w.nhi[j];
+        total += range_cost(PW, y > x ? PW[y] - PW[x] : 0ll, w.clo[r], w.chi[r], x, y);
     }
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    __syncwarp();
+    // hand the rows of every class to the columns it serves (rows ascending, list order)
+    for (int r = lane; r < R; r += 32) {
+        int j = w.head[r];
+        for (int i = 0; i < n && j >= 0; ++i) {
+            if (w.row_class[i] != r) continue;
+            const int nx = w.next_col[j];
+            w.tcol[j] = (short)i;                 // scratch: row of column j
+            j = nx;
+        }
+    }
+    __syncwarp();
+    for (int j = lane; j < n; j += 32) w.match[j] = w.tcol[j];
+    __syncwarp();
     return total;
 }
 
 __device__ __forceinline__ long long warp_match_any(MatchWork &w, const long long *PW, int n, int lane) {
+    // the class count is known only inside; NC is chosen for the row count, which bounds it
     if (n <= 32) return warp_match<1>(w, PW, n, lane);
     if (n <= 64) return warp_match<2>(w, PW, n, lane);
     if (n <= 128) return warp_match<4>(w, PW, n, lane);
