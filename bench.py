@@ -39,15 +39,14 @@ SM_MAX_MHZ_FALLBACK = 1965.0
 # class: "regs" = cm_cost_regs_kernel (pipelines of <= 16 stages), "wide" = the deep-pipeline
 # kernel (17 .. 64 stages); arithmetic 0 = fp64 (also the exact integer-valued mode), 1 = int64.
 KERNEL_PROFILES = {
-    ("regs", 0): {"i_cell": 5.79, "issue_active": 0.647, "fp64_pipe_active": 0.649,
+    ("regs", 0): {"i_cell": 5.85, "issue_active": 0.650, "fp64_pipe_active": 0.646, "dram_bytes_per_cell": 660480 / 8.54e9,
                   "profile": "profiles/cm_cost_regs_kernel_paper-scale-512.md"},
-    ("regs", 1): {"i_cell": 8.64, "issue_active": 0.630, "fp64_pipe_active": 0.0,
+    ("regs", 1): {"i_cell": 8.64, "issue_active": 0.630, "fp64_pipe_active": 0.0, "dram_bytes_per_cell": 620000 / 8.53e9,
                   "profile": "profiles/cm_cost_regs_kernel_int64_paper-scale-512.md"},
-    ("wide", 0): {"i_cell": 7.32, "issue_active": 0.586, "fp64_pipe_active": 0.530,
+    ("wide", 0): {"i_cell": 6.14, "issue_active": 0.574, "fp64_pipe_active": 0.558, "dram_bytes_per_cell": 173056 / 6.199e9,
                   "profile": "profiles/cm_cost_wide_kernel_175b-like-8.md"},
 }
 FP64_INSTR_PER_CELL = 3.0          # 2 DADD + 1 DSETP; an FP64 warp instruction occupies its pipe for 2 cycles
-TRAFFIC_BYTES_PER_CTA = 645888.0 / 55800.0   # dram__bytes_read+write of one ncu-captured launch / its CTAs
 
 
 def measured_peaks():
@@ -500,10 +499,10 @@ def roofline_of(stats_sum, dev_seconds, arith, kclass, clocks, sm_max, peak_kind
         "ms_per_launch": 1e3 * cost_s / launches,
         "share_of_step": cost_s / dev_seconds if dev_seconds else None,
         # the search pass reads only the small descriptor tables: ~0 algorithmic bytes.  Not
-        # measured in this run: DRAM bytes of one ncu-captured launch (0.65 MB for 55 800 CTAs of
-        # the 12-stage kernel) scaled by this run's CTAs per launch.
-        "traffic": TRAFFIC_BYTES_PER_CTA * stats_sum["plans"] / launches / 128.0,
-        "traffic_source": "scaled by CTAs from the ncu capture in profiles/cm_cost_regs_kernel_paper-scale-512.md",
+        # measured in this run: dram__bytes_read + write of the ncu capture named above, per
+        # recurrence cell of that launch, times this run's cells per launch.
+        "traffic": prof["dram_bytes_per_cell"] * stats_sum["cells"] / launches,
+        "traffic_source": f"scaled by cells from the ncu capture in {prof['profile']} (not measured in this run)",
     }
 
 
