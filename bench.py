@@ -440,6 +440,35 @@ def measure_trace(binding, w, mode, local_rank, seed=7, hours=9.0, rate=0.10):
         binding.cm_destroy(ctx)
 
 
+def measure_stretch(binding, torch, mode, local_rank, picks=(20, 63), reps=3):
+    """Stretch case: 70b-like with no cap on the layer compositions per pipeline (up to
+    C(32,16) = 6e8 of them): whole searches of single failure sets, 5e9-1e10 pipeline-plans each."""
+    import copy
+    from paper_2508_21613_b200 import workloads as W
+    w = W.llama70b_like()
+    opts = copy.copy(w.options.with_cost_mode(mode))
+    opts.kappa_cap = 1 << 62
+    ctx = binding.cm_create(local_rank)
+    binding.cm_load_profile(ctx, w.profile)
+    out = {"workload": "70b-like, kappa_cap unbounded", "failure_sets": []}
+    try:
+        for k in picks:
+            pack = binding.PackedScenarios([w.scenarios[k]])
+            pack.search(ctx, opts)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                pack.search(ctx, opts)
+            dt = (time.perf_counter() - t0) / reps
+            st = binding.cm_last_stats(ctx)
+            out["failure_sets"].append({"scenario": k, "failed_devices": len(w.scenarios[k]), "pipeline_plans": st["plans"],
+                                        "plans_simulated": st["plans_simulated"], "e2e_ms": 1e3 * dt,
+                                        "plans_per_s": st["plans"] / dt})
+    finally:
+        binding.cm_destroy(ctx)
+    return out
+
+
 def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
     """Plan cache: every failure set of at most k devices searched ahead of time; lookups."""
     from paper_2508_21613_b200 import workloads as W
@@ -494,6 +523,9 @@ def roofline_of(stats_sum, dev_seconds, arith, kclass, clocks, sm_max, peak_kind
         # against the FP64 pipe alone: 3 FP64 instructions per cell, each holding the pipe of a
         # scheduler (16 lanes) for 2 cycles
         "frac_of_fp64_pipe": (achieved / (lanes_per_s / (2.0 * FP64_INSTR_PER_CELL))) if arith == 0 else None,
+        # an FP64 warp instruction holds the dispatch slot for two cycles, so issue-active cannot pass
+        # I_cell / (I_cell + 3): the bound of this instruction stream in cells is lanes / (I_cell + 3)
+        "frac_of_dispatch_bound": (achieved / (lanes_per_s / (prof["i_cell"] + FP64_INSTR_PER_CELL))) if arith == 0 else None,
         "fp64_pipe_active_profiled": prof["fp64_pipe_active"],
         "cells_per_launch": stats_sum["cells"] / launches,
         "ms_per_launch": 1e3 * cost_s / launches,
@@ -629,6 +661,7 @@ def main():
             small = w if w.profile.n_dp * w.profile.n_pp <= 64 else W.paper_scale(0, 0)
             line["plan_cache"] = dict(measure_cache(binding, small, args.cost_mode, local_rank), workload=small.name)
             line["failure_trace"] = dict(measure_trace(binding, small, args.cost_mode, local_rank), workload=small.name)
+            line["stretch_uncapped"] = measure_stretch(binding, torch, args.cost_mode, local_rank)
         if args.objective and "full_objective" not in line:
             line["full_objective"] = {w.name: measure_objective(binding, torch, w, args.cost_mode, args.steps,
                                                                 args.warmup, local_rank, flush)}
