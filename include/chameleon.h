@@ -439,7 +439,10 @@ cm_status cm_cache_free(cm_cache *cache);
  *  [14] host time enqueueing the launch sequence, ns   [15] host time waiting for the stream, ns
  *  [16] pipeline-plans of [0] whose recurrence ran, i.e. that passed the memory estimator
  *       (Section "Estimator", memory estimator); [0] - [16] were rejected by it
- *  [17..23] reserved, 0. */
+ *  [17] host time spent listing memory-feasible compositions (inside [13]; includes one stream
+ *       synchronisation when a new (stages, micro-batches) pair is met), ns
+ *  [18] host time packing and uploading the descriptor tables, buffer allocation included, ns
+ *  [19..23] reserved, 0. */
 cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[24]);
 
 const char *cm_strerror(cm_status status);

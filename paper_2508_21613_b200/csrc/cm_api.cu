@@ -680,7 +680,9 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.n_tiles = bt.max_tiles_per_seg ? 1 : 0;   // only "is there anything to tie-break" matters
     bt.mm_launched = false;
     if (ctx->d_prof && ctx->screen) {   // (a context without a device only describes: cm_host_describe)
+        const uint64_t t0 = now_ns();
         cm_status s = ensure_feasible_lists(ctx, bt);
+        ctx->stats[17] += now_ns() - t0;
         if (s != CM_OK) return s;
     }
     return build_buckets(ctx, bt);
@@ -736,6 +738,7 @@ Tables tables_plain(const cm_ctx *ctx) {   // for kernels that only read the byt
 
 // Copy the tables of a batch to the device (one copy) and run the min-max partitions it needs.
 cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
+    struct Timer { cm_ctx *c; uint64_t t0; ~Timer() { c->stats[18] += now_ns() - t0; } } timer{ctx, now_ns()};
     bool ok = true;
     bt.arena.clear();
     bt.off_scen = arena_put(bt.arena, bt.scen, ok);
@@ -1035,6 +1038,9 @@ cm_status cm_create(cm_ctx **out, int cuda_device, void *cuda_stream) {
         if (ok) c->side.n = i + 1;
     }
     ok = ok && c->d_scratch.reserve(sizeof(cm_plan *) * 64 + sizeof(cm_plan));   // what cm_select needs
+    // the feasible-composition pool and its staging are allocated here, not at the first search:
+    // a pinned allocation costs milliseconds, which a failure handler should not pay
+    ok = ok && c->d_feas.reserve(1u << 20) && c->feas_stage.reserve(1u << 16) && c->d_feas_stage.reserve(1u << 16);
     if (!ok || cudaMalloc((void **)&c->d_prof, sizeof(DevProfile)) != cudaSuccess ||
         cudaMalloc((void **)&c->d_prof53, sizeof(DevProfile)) != cudaSuccess) {
         if (c->d_prof) cudaFree(c->d_prof);
