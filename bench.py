@@ -440,9 +440,11 @@ def measure_trace(binding, w, mode, local_rank, seed=7, hours=9.0, rate=0.10):
         binding.cm_destroy(ctx)
 
 
-def measure_stretch(binding, torch, mode, local_rank, picks=(20, 63), reps=3):
+def measure_stretch(binding, torch, mode, local_rank, picks=(63,), reps=2):
     """Stretch case: 70b-like with no cap on the layer compositions per pipeline (up to
-    C(32,16) = 6e8 of them): whole searches of single failure sets, 5e9-1e10 pipeline-plans each."""
+    C(32,16) = 6e8 of them): the whole search of one failure set of 8 devices, 4.7e9 pipeline-plans
+    (sets that leave more survivors have up to 1.2e10 plans, most of them memory-feasible, and take
+    tens of seconds: too long for a default run)."""
     import copy
     from paper_2508_21613_b200 import workloads as W
     w = W.llama70b_like()
