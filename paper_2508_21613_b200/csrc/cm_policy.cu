@@ -162,38 +162,42 @@ __global__ void __launch_bounds__(32 * (kMaxP + 1)) cm_policy_kernel(Tables tb, 
                 bits = Num<T>::bits(t + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
             }
         } else if (ok && lane == 0) {
-            int cuts[kMaxS + 1], devs[kMaxS];
-            int n = 0;
-            cuts[0] = 0;
-            for (int i = 0; i < S0; ++i) {
-                if ((dead >> i) & 1ull) continue;
-                int hi = base_cuts[i + 1];
-                if (i + 1 < S0 && ((dead >> (i + 1)) & 1ull)) hi = base_cuts[i + 2];
-                devs[n] = k * S0 + i;
-                cuts[n + 1] = hi;
-                ++n;
-            }
+            // deeper than a warp: lane 0 walks the surviving stages in order, each read off the
+            // alive mask exactly as the lanes do above (stage j = j-th set bit; its range runs to
+            // the end of a failed stage right behind it; the stage behind it rides along)
+            uint64_t rest = alive;
             long long g_max = 0;
             bool fits = true;
-            for (int i = 0; i < n && fits; ++i) {
-                const int lo = cuts[i], hi = cuts[i + 1];
-                long long stat = sp.PS[hi] - sp.PS[lo], act = sp.PA[hi] - sp.PA[lo];
+            int n = 0;
+            int orig = __ffsll((long long)rest) - 1;
+            rest &= rest - 1;
+            int lo = base_cuts[orig];
+            int hi = base_cuts[orig + 1 + ((orig + 1 < S0 && ((dead >> (orig + 1)) & 1ull)) ? 1 : 0)];
+            while (fits) {
                 T f = sp.PF[hi] - sp.PF[lo], bw = sp.PB[hi] - sp.PB[lo];
-                if (i < n - 1) {
-                    const int hi2 = cuts[i + 2];
-                    f = f + (sp.PF[hi2] - sp.PF[hi]);
-                    bw = bw + (sp.PB[hi2] - sp.PB[hi]);
-                    stat = stat + (sp.PS[hi2] - sp.PS[hi]);
-                    act = act + (sp.PA[hi2] - sp.PA[hi]);
-                    xts[i] = sp.XT[(devs[i] / dpn == devs[i + 1] / dpn) ? 0 : 1][hi - 1];
-                } else {
-                    xts[i] = (T)0;
-                }
-                Fs[i] = f;
-                Bs[i] = bw;
-                fits = stage_fits(stat, act, i, n, m, sp.cap, sp.sched);
+                long long stat = sp.PS[hi] - sp.PS[lo], act = sp.PA[hi] - sp.PA[lo];
                 const long long gb = sp.PP[hi] - sp.PP[lo];
                 g_max = gb > g_max ? gb : g_max;
+                xts[n] = (T)0;
+                const bool last = rest == 0;
+                int orig2 = 0, lo2 = 0, hi2 = 0;
+                if (!last) {
+                    orig2 = __ffsll((long long)rest) - 1;
+                    rest &= rest - 1;
+                    lo2 = base_cuts[orig2];
+                    hi2 = base_cuts[orig2 + 1 + ((orig2 + 1 < S0 && ((dead >> (orig2 + 1)) & 1ull)) ? 1 : 0)];
+                    f = f + (sp.PF[hi2] - sp.PF[lo2]);
+                    bw = bw + (sp.PB[hi2] - sp.PB[lo2]);
+                    stat = stat + (sp.PS[hi2] - sp.PS[lo2]);
+                    act = act + (sp.PA[hi2] - sp.PA[lo2]);
+                    xts[n] = sp.XT[((k * S0 + orig) / dpn == (k * S0 + orig2) / dpn) ? 0 : 1][hi - 1];
+                }
+                Fs[n] = f;
+                Bs[n] = bw;
+                fits = stage_fits(stat, act, n, S, m, sp.cap, sp.sched);
+                ++n;
+                if (last) break;
+                orig = orig2; lo = lo2; hi = hi2;
             }
             if (fits) bits = Num<T>::bits(sim_pipe<T>(n, m, Fs, Bs, xts, clk, pnd, sp.sched) + Num<T>::sync(g_max, n_dp, sp.bw_sync, sp.intval));
         }
