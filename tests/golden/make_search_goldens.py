@@ -10,7 +10,10 @@ feasible, strategy, pipelines, split rank, stages, micro-batches, layer-composit
 and the cost bits -- everything the parity bar requires to be bit-exact.  The GPU tests
 recompute the fingerprint from the library's plan and compare.
 
-    python tests/golden/make_search_goldens.py [workload ...] [--procs N] [--objective]
+    python tests/golden/make_search_goldens.py [workload ...] [--procs N] [--objective] [--schedule gpipe]
+
+With --schedule gpipe the time model runs under the all-forward-all-backward order and the
+results go to search_<workload>_gpipe_<mode>.txt.
 
 With --objective the full-objective search (default ObjectiveOptions) is stored instead, in
 objective_<workload>_<mode>.txt:
@@ -62,12 +65,12 @@ def line_of(plan, mode: int) -> str:
 _state = {}
 
 
-def _init(name, mode):
+def _init(name, mode, schedule=0):
     from oracle.oracle import Oracle
     from paper_2508_21613_b200 import workloads as W
     w = W.ALL_WORKLOADS[name]()
     _state["w"] = w
-    _state["o"] = Oracle(w.profile, w.options.with_cost_mode(mode))
+    _state["o"] = Oracle(w.profile, w.options.with_cost_mode(mode).with_schedule(schedule))
     _state["mode"] = mode
 
 
@@ -101,8 +104,8 @@ def objective_path(name: str, mode: int) -> str:
     return os.path.join(HERE, f"objective_{name}_{'i64' if mode else 'f64'}.txt")
 
 
-def golden_path(name: str, mode: int) -> str:
-    return os.path.join(HERE, f"search_{name}_{'i64' if mode else 'f64'}.txt")
+def golden_path(name: str, mode: int, schedule: int = 0) -> str:
+    return os.path.join(HERE, f"search_{name}_{'gpipe_' if schedule else ''}{'i64' if mode else 'f64'}.txt")
 
 
 def main():
@@ -111,7 +114,11 @@ def main():
     ap.add_argument("--procs", type=int, default=os.cpu_count())
     ap.add_argument("--modes", type=int, nargs="*", default=[0, 1])
     ap.add_argument("--objective", action="store_true", help="store the full-objective search instead")
+    ap.add_argument("--schedule", choices=["1f1b", "gpipe"], default="1f1b")
     args = ap.parse_args()
+    schedule = 1 if args.schedule == "gpipe" else 0
+    if schedule and args.objective:
+        ap.error("the full-objective results are stored for the 1F1B order only")
     from oracle.oracle import build
     build()
     from paper_2508_21613_b200 import workloads as W
@@ -119,7 +126,7 @@ def main():
         n = len(W.ALL_WORKLOADS[name]().scenarios)
         for mode in args.modes:
             t0 = time.time()
-            with mp.Pool(args.procs, initializer=_init, initargs=(name, mode)) as pool:
+            with mp.Pool(args.procs, initializer=_init, initargs=(name, mode, schedule)) as pool:
                 lines = [None] * n
                 for b, line in pool.imap_unordered(_one_objective if args.objective else _one, range(n), chunksize=1):
                     lines[b] = line
@@ -131,8 +138,8 @@ def main():
                     f.write("\n".join(lines) + "\n")
                 print(f"{name} mode {mode} (objective): {n} scenarios in {time.time() - t0:.0f} s", flush=True)
                 continue
-            with open(golden_path(name, mode), "w") as f:
-                f.write(f"# {name}, cost mode {'int64 ns' if mode else 'fp64'}: best plan per failure scenario from the CPU "
+            with open(golden_path(name, mode, schedule), "w") as f:
+                f.write(f"# {name}, cost mode {'int64 ns' if mode else 'fp64'}{', all-forward-all-backward order' if schedule else ''}: best plan per failure scenario from the CPU "
                         f"oracle (tests/golden/make_search_goldens.py)\n# policy feasible cost fingerprint\n")
                 f.write("\n".join(lines) + "\n")
             print(f"{name} mode {mode}: {n} scenarios in {time.time() - t0:.0f} s", flush=True)

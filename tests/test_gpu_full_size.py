@@ -52,6 +52,26 @@ def test_every_scenario_matches_the_stored_oracle_result(gpu, name, mode):
         gpu.cm_destroy(ctx)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_every_paper_scale_scenario_under_the_second_order(gpu, mode):
+    """The same comparison with the time model under the all-forward-all-backward order
+    (tests/golden/search_paper-scale_gpipe_*.txt, `make_search_goldens.py paper-scale --schedule gpipe`)."""
+    w = W.paper_scale()
+    path = goldens.golden_path(w.name, mode, W.SCHED_GPIPE)
+    assert os.path.exists(path), f"{path} is missing"
+    want = [l.strip() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(want) == len(w.scenarios)
+    ctx = gpu.cm_create(0)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, w.options.with_cost_mode(mode).with_schedule(W.SCHED_GPIPE))
+        got = [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)]
+        wrong = [b for b in range(len(want)) if got[b] != want[b]]
+        assert not wrong, f"{len(wrong)} of {len(want)} scenarios differ, first: {wrong[0]}: got {got[wrong[0]]} want {want[wrong[0]]}"
+    finally:
+        gpu.cm_destroy(ctx)
+
+
 def _stored_objective(name, mode):
     path = goldens.objective_path(name, mode)
     assert os.path.exists(path), f"{path} is missing: run tests/golden/make_search_goldens.py {name} --objective"
