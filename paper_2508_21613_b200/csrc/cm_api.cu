@@ -800,11 +800,21 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
         launches += (bd.n_red_blocks && bd.max_red_per_scen > 1) ? 2 : 1;
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[4], st));
         if (bt.n_tiles) {
-            CM_CUDA(ctx, launch_cost_pass2(tb, bd, st));
+            bool deep = false;
+            for (const TSeg &g : bt.tseg) deep = deep || (g.S > kRegStagesMax && g.K > 0);
+            // few winners (a failure handled on its own): the lock-step kernel completes every deep
+            // pipeline in one launch; many: one plan per lane, a kernel per depth
+            const bool by_warp = deep && (uint64_t)bt.B * bt.dp_max <= kWarpTieMaxPairs;
+            CM_CUDA(ctx, launch_cost_pass2(tb, bd, st, by_warp));
             ++launches;
-            uint64_t stage_mask = 0;
-            for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
-            CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &ctx->side, &launches));
+            if (by_warp) {
+                CM_CUDA(ctx, launch_tiebreak_warp(tb, bd, st));
+                ++launches;
+            } else if (deep) {
+                uint64_t stage_mask = 0;
+                for (const TSeg &g : bt.tseg) stage_mask |= 1ull << (g.S & 63);
+                CM_CUDA(ctx, launch_tiebreak_wide(tb, bd, stage_mask, st, &ctx->side, &launches));
+            }
         }
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[5], st));
     }

@@ -254,7 +254,13 @@ struct SideStreams {
 cudaError_t launch_cost_pass1(const Tables &t, const BatchDev &b, const LaunchClass *classes, int n_classes,
                               cudaStream_t st, const SideStreams *side, int *launches);
 cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t st);
-cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st);
+// deep_elsewhere: winners' pipelines deeper than kRegStagesMax are completed by another kernel
+// (the per-depth ones, or the lock-step one below), this one leaves them alone
+cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st, bool deep_elsewhere_all = false);
+// Tie-break pass for few winners (one failure at a time): a warp per layer composition walks the
+// pipeline in lock step, every depth above kRegStagesMax in one launch.
+constexpr uint64_t kWarpTieMaxPairs = 64;   // (scenario, pipeline) pairs up to which the lock-step tie-break is used
+cudaError_t launch_tiebreak_warp(const Tables &t, const BatchDev &b, cudaStream_t st);
 cudaError_t launch_tiebreak_wide(const Tables &t, const BatchDev &b, uint64_t stage_mask, cudaStream_t st,
                                  const SideStreams *side, int *launches);
 cudaError_t launch_finalize(const Tables &t, const BatchDev &b, cudaStream_t st);

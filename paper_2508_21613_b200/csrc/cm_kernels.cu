@@ -328,7 +328,7 @@ cudaError_t launch_split_reduce(const Tables &t, const BatchDev &b, cudaStream_t
 // grid.y = tiles of a segment.  Tiles above an already found index return at once.
 // ----------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev bd) {
+__global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev bd, int deep_elsewhere_all) {
     __shared__ SProf<T> sp;
     __shared__ uint64_t red[kTile / 32];
     __shared__ SegView g;
@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
     if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;          // uniform over the CTA
     {
         const int S = bd.tseg[w.seg[p]].S;   // 17..48 stages: cm_tiebreak_wide_kernel's job
-        if (S > kRegStagesMax && S <= kWideStagesMax) return;
+        if (S > kRegStagesMax && (S <= kWideStagesMax || deep_elsewhere_all)) return;
     }
     for (uint64_t tile = blockIdx.y; tile < bd.max_tiles_per_seg; tile += gridDim.y) {
         uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
@@ -381,13 +381,101 @@ __global__ void __launch_bounds__(kTile) cm_tiebreak_kernel(Tables tb, BatchDev 
     }
 }
 
-cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st) {
+cudaError_t launch_cost_pass2(const Tables &t, const BatchDev &b, cudaStream_t st, bool deep_elsewhere_all) {
     if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
     const uint64_t nx = (uint64_t)b.B * b.dp_max;
     if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
     dim3 grid((unsigned)nx, tiebreak_grid_y(nx, b.max_tiles_per_seg), 1);
-    if (native_i64(b)) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b);
-    else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b);
+    if (native_i64(b)) cm_tiebreak_kernel<long long><<<grid, kTile, 0, st>>>(t, b, deep_elsewhere_all ? 1 : 0);
+    else cm_tiebreak_kernel<double><<<grid, kTile, 0, st>>>(t, b, deep_elsewhere_all ? 1 : 0);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
+// The same pass when there are only a few winners (a single failure being handled): with one
+// plan per lane the first tile alone is a dependent chain of 2*S*m cells in every thread (0.1-0.2
+// ms at 30+ stages), whatever the number of compositions that are really needed.  Here a WARP
+// takes one composition and walks the pipeline in lock step, stages over its lanes (two per lane
+// above 32 stages): 2(S+m) slots of a few dozen cycles.  grid.x = (scenario, pipeline), grid.y
+// strides over the walk in groups of four compositions (one per warp), lowest first; a warp
+// stops as soon as a composition at or below its own has been found.  Every depth above
+// kRegStagesMax in one launch.
+// ----------------------------------------------------------------------------------
+constexpr int kWarpTieWarps = 4;
+template <typename T>
+__global__ void __launch_bounds__(kWarpTieWarps * 32) cm_tiebreak_warp_kernel(Tables tb, BatchDev bd) {
+    __shared__ SProf<T> sp;
+    __shared__ uint8_t cuts_s[kWarpTieWarps][kMaxS + 8];
+    const uint32_t b = blockIdx.x / bd.dp_max, p = blockIdx.x % bd.dp_max;
+    const Winner &w = bd.winner[b];
+    if (w.cost_bits >= inf_bits<T>() || p >= w.dp) return;          // uniform over the CTA
+    const SegView g = seg_view(bd, w.scen, w.seg[p]);
+    if (g.S <= kRegStagesMax || g.K == 0) return;                   // shallow: cm_tiebreak_kernel; one candidate: known already
+    stage_profile(sp, tb);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int S = g.S, m = g.m;
+    uint8_t *cuts = cuts_s[warp];
+    uint64_t *slot = &bd.kappa_sel[b * kMaxP + p];
+    const uint64_t count = walk_count(g);
+    unsigned long long evaluated = 0;
+    for (uint64_t pos = (uint64_t)blockIdx.y * kWarpTieWarps + warp; pos < count; pos += (uint64_t)gridDim.y * kWarpTieWarps) {
+        const uint64_t kappa = walk_kappa(bd.feas, g.feas_first, pos);
+        uint64_t found = 0;
+        if (lane == 0) found = *(volatile uint64_t *)slot;
+        found = __shfl_sync(0xffffffffu, found, 0);
+        if (found <= kappa) break;                                  // later compositions of this warp are higher still
+        CutWalker cw;
+        bool ok = make_walker(cw, tb, bd.layer_mode, sp.L, S, kappa, g.K, tb.mm_slot(S, m));
+        if (ok) {
+            int lo = 0;
+            for (int i = 0; i < S; ++i) {
+                const int hi = cw.next();
+                ok = ok && hi > lo;
+                if (lane == 0) cuts[i + 1] = (uint8_t)hi;
+                lo = hi;
+            }
+            if (lane == 0) cuts[0] = 0;
+        }
+        __syncwarp();
+        long long g_max = 0;
+        if (ok)
+            for (int i = lane; i < S; i += 32) {
+                const int lo = cuts[i], hi = cuts[i + 1];
+                ok = ok && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
+                const long long gb = sp.PP[hi] - sp.PP[lo];
+                g_max = gb > g_max ? gb : g_max;
+            }
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            for (int o = 16; o > 0; o >>= 1) {
+                const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
+                g_max = og > g_max ? og : g_max;
+            }
+            const T t = S <= 32 ? warp_pipe_time<T, 1>(sp, cuts, S, m, g.tier, lane)
+                                : warp_pipe_time<T, 2>(sp, cuts, S, m, g.tier, lane);
+            const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval));
+            if (lane == 0 && bits <= w.cost_bits) atomicMin((unsigned long long *)slot, (unsigned long long)kappa);
+        }
+        ++evaluated;
+        __syncwarp();                                               // the next composition overwrites the cuts
+    }
+    if (lane == 0 && evaluated) atomicAdd(&bd.counters[1], evaluated);
+}
+
+cudaError_t launch_tiebreak_warp(const Tables &t, const BatchDev &b, cudaStream_t st) {
+    if (b.B <= 0 || b.max_tiles_per_seg == 0 || b.dp_max == 0) return cudaSuccess;
+    const uint64_t nx = (uint64_t)b.B * b.dp_max;
+    if (nx >= (1ull << 31)) return cudaErrorInvalidConfiguration;
+    // as many groups of four compositions side by side as fill the GPU a few times over
+    uint64_t y = (4096 + nx - 1) / nx;
+    const uint64_t groups = (uint64_t)b.max_tiles_per_seg * (kTile / kWarpTieWarps);
+    if (y > groups) y = groups;
+    if (y > 65535) y = 65535;
+    if (y < 1) y = 1;
+    dim3 grid((unsigned)nx, (unsigned)y, 1);
+    if (native_i64(b)) cm_tiebreak_warp_kernel<long long><<<grid, kWarpTieWarps * 32, 0, st>>>(t, b);
+    else cm_tiebreak_warp_kernel<double><<<grid, kWarpTieWarps * 32, 0, st>>>(t, b);
     return cudaGetLastError();
 }
 
