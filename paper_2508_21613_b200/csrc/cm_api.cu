@@ -288,9 +288,20 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket_tseg.clear();
     struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
     std::vector<Pre> pre;
-    auto kind_of = [](int S, int m, uint64_t n_seg, uint64_t K) {
+    // plans of the deep pipelines that have a choice of composition, over the whole batch
+    uint64_t deep_plans = 0;
+    for (const Tmpl &tp : bt.tmpl)
+        for (uint32_t i = 0; i < tp.n_tseg && tp.n_scen; ++i) {
+            const TSeg &g = bt.tseg[tp.tseg_first + i];
+            if (g.S > kRegStagesMax && g.K > 0 && g.m >= 1)
+                deep_plans += (g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : g.K + 1) * tp.n_scen;
+        }
+    const bool by_warp = deep_plans <= kWarpPlansMax;
+    auto kind_of = [by_warp](int S, int m, uint64_t n_seg, uint64_t K, uint64_t count) {
+        (void)count;
         if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_SHORT;
         if (K == 0) return (int)CM_CLASS_SOLO;   // the min-max partition is the only candidate there is
+        if (by_warp) return (int)CM_CLASS_WARP;
         if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
         return (int)CM_CLASS_WIDE_UNI;           // deeper than kWideStagesMax: the transposed layout only
     };
@@ -318,7 +329,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 // not.  With one scenario the segments are few: what does not fill most of a
                 // last warp goes to the per-lane kernel, which wastes no lane.
                 size_t cut = j;
-                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, g.K) == CM_CLASS_WIDE_UNI) {
+                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, g.K, count) == CM_CLASS_WIDE_UNI) {
                     const size_t rest = (j - i) % 32;
                     if (rest > 0 && rest < (size_t)kUniMinSegments) cut = j - rest;
                 }
@@ -327,7 +338,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     if (p1 <= p0) continue;
                     const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
                     Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
-                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, g.K), g.feas_first};
+                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, g.K, count), g.feas_first};
                     for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
                     pre.push_back(q);
                 }
@@ -335,9 +346,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
             i = j;
         }
     }
-    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_SOLO; ++kind) {
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WARP; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
-        const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO;   // every depth in one class
+        const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO || kind == CM_CLASS_WARP;   // every depth in one class
         LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
             LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
@@ -369,6 +380,8 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     c.n_chunks += (items + per_cta - 1) / per_cta;
                 } else if (kind == CM_CLASS_SOLO) {
                     c.n_chunks += ((uint64_t)bk.n_seg + kChunk / 32 - 1) / (kChunk / 32);   // a warp per segment
+                } else if (kind == CM_CLASS_WARP) {
+                    c.n_chunks += (bk.count * bk.n_seg + kChunk / 32 - 1) / (kChunk / 32);   // a warp per plan
                 } else {
                     c.n_chunks += (bk.count * bk.n_seg + kChunk - 1) / kChunk;
                 }

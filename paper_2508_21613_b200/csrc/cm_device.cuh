@@ -3,6 +3,8 @@
 // sums with the memory check, and the 1F1B start/end recurrence.
 #pragma once
 
+#include <type_traits>
+
 #include "cm_internal.h"
 
 namespace cm {
@@ -428,17 +430,30 @@ __device__ __forceinline__ void init_kappa_sel(const BatchDev &bd, const Winner 
 // ----------------------------------------------------------------------------------
 // Under the all-forward-all-backward order forward (i,j) sits at slot i+j and backward (i,j)
 // at slot (S+m-1) + (S-1-i) + j.
+// The loop is branch-free inside a slot -- lanes that run a forward, a backward or nothing take
+// the same instructions, so the stages of a lane and the two kinds of work interleave -- and
+// the slot tests are kept short, because one warp alone issues them: times are non-negative,
+// so "no dependency" (forward of stage 0, backward of the last stage) is a dependency on time 0
+// (a stage past the end never runs and keeps its zeros), and under 1F1B the parity of s - i
+// says which kind of work a steady-state slot can hold.
 template <typename T, int PER>
 __device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B, const T *xt, int sched) {
     const int lane = threadIdx.x & 31;
     T clock[PER], last_f[PER], last_b[PER];
+    int d[PER];          // slot - stage
+    unsigned mk[PER];    // micro-batches of the stage (0: past the end)
 #pragma unroll
-    for (int k = 0; k < PER; ++k) { clock[k] = (T)0; last_f[k] = (T)0; last_b[k] = (T)0; }
-    const int n_slots = sched == CM_SCHED_GPIPE ? 2 * (S + m - 1) : 2 * (S + m) - 2;
-    for (int s = 0; s < n_slots; ++s) {
+    for (int k = 0; k < PER; ++k) {
+        clock[k] = (T)0; last_f[k] = (T)0; last_b[k] = (T)0;
+        d[k] = -(lane * PER + k);
+        mk[k] = lane * PER + k < S ? (unsigned)m : 0u;
+    }
+    auto slot = [&](auto only_forward, auto pick) {
+        T up = __shfl_up_sync(0xffffffffu, last_f[PER - 1], 1);
+        T down = __shfl_down_sync(0xffffffffu, last_b[0], 1);
+        up = lane == 0 ? (T)0 : up;       // the end lanes get their own value back from the shuffle
+        down = lane == 31 ? (T)0 : down;
         T f_in[PER], b_in[PER];
-        const T up = __shfl_up_sync(0xffffffffu, last_f[PER - 1], 1);
-        const T down = __shfl_down_sync(0xffffffffu, last_b[0], 1);
 #pragma unroll
         for (int k = 0; k < PER; ++k) {
             f_in[k] = k == 0 ? up : last_f[k > 0 ? k - 1 : 0];
@@ -446,35 +461,52 @@ __device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B
         }
 #pragma unroll
         for (int k = 0; k < PER; ++k) {
-            const int i = lane * PER + k;
-            if (i >= S) continue;
-            bool is_f = false, is_b = false;
-            const int d = s - i;
-            if (sched == CM_SCHED_GPIPE) {
-                is_f = d >= 0 && d < m;
-                const int e = s - (S + m - 1) - (S - 1 - i);
-                is_b = e >= 0 && e < m;
+            bool is_f, is_b;
+            pick(k, is_f, is_b);
+            if constexpr (decltype(only_forward)::value) {
+                const T fin = tmax(clock[k], f_in[k]) + F[k];
+                clock[k] = is_f ? fin : clock[k];
+                last_f[k] = is_f ? fin + xt[k] : last_f[k];
             } else {
-                if (s <= S - 1) {
-                    is_f = d >= 0 && d < m;
-                } else if ((d & 1) == 0) {
-                    const int j = d >> 1;
-                    is_f = j > S - 1 - i && j < m;
-                }
-                const int e = s - (2 * S - 1 - i);
-                if (e >= 0 && (e & 1) == 0) is_b = (e >> 1) < m;
+                const T dep = is_f ? f_in[k] : b_in[k] + xt[k];
+                const T fin = tmax(clock[k], dep) + (is_f ? F[k] : B[k]);
+                clock[k] = (is_f || is_b) ? fin : clock[k];
+                last_f[k] = is_f ? fin + xt[k] : last_f[k];
+                last_b[k] = is_b ? fin : last_b[k];
             }
-            if (is_f) {
-                const T start = i > 0 ? tmax(clock[k], f_in[k]) : clock[k];
-                clock[k] = start + F[k];
-                last_f[k] = clock[k] + xt[k];
-            } else if (is_b) {
-                const T dep = i < S - 1 ? b_in[k] + xt[k] : clock[k];   // last stage: its own forward just ended
-                const T start = tmax(clock[k], dep);
-                clock[k] = start + B[k];
-                last_b[k] = clock[k];
-            }
+            ++d[k];
         }
+    };
+    using Yes = std::true_type;
+    using No = std::false_type;
+    if (sched == CM_SCHED_GPIPE) {
+        // forward (i,j) at slot i+j; backward (i,j) at slot (S+m-1) + (S-1-i) + j
+        for (int s = 0; s < S + m - 1; ++s)
+            slot(Yes{}, [&](int k, bool &is_f, bool &is_b) { is_f = (unsigned)d[k] < mk[k]; is_b = false; });
+        int e[PER];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) e[k] = -(S - 1 - (lane * PER + k));
+        for (int s = 0; s < S + m - 1; ++s)
+            slot(No{}, [&](int k, bool &is_f, bool &is_b) { is_f = false; is_b = (unsigned)e[k] < mk[k]; ++e[k]; });
+    } else {
+        // slots 0 .. S-1: warm-up forwards only (the first backward sits at slot S)
+        for (int s = 0; s < S; ++s)
+            slot(Yes{}, [&](int k, bool &is_f, bool &is_b) { is_f = (unsigned)d[k] < mk[k]; is_b = false; });
+        // afterwards forward j = (s-i)/2 when s-i is even and j > S-1-i; backward (s-i-(2S-1-2i))/2 when s-i is odd
+        int warm[PER], off[PER];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            warm[k] = S - 1 - (lane * PER + k);
+            off[k] = 2 * S - 1 - 2 * (lane * PER + k);
+        }
+        const int n_slots = 2 * (S + m) - 2;
+        for (int s = S; s < n_slots; ++s)
+            slot(No{}, [&](int k, bool &is_f, bool &is_b) {
+                const bool even = (d[k] & 1) == 0;
+                const int j = d[k] >> 1;
+                is_f = even && j > warm[k] && (unsigned)j < mk[k];
+                is_b = !even && ((unsigned)(d[k] - off[k]) >> 1) < mk[k];
+            });
     }
     return __shfl_sync(0xffffffffu, clock[0], 0);
 }

@@ -108,7 +108,11 @@ struct Bucket {
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
-enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_SHORT = 3, CM_CLASS_SOLO = 4 };
+enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_SHORT = 3, CM_CLASS_SOLO = 4, CM_CLASS_WARP = 5 };
+// CM_CLASS_WARP: the pipelines deeper than kRegStagesMax of a batch that has so few plans there (after the memory
+// screen) that a thread per plan would leave the GPU waiting on a handful of long dependent chains: a warp per plan
+// in lock step, every depth in one launch.
+constexpr uint64_t kWarpPlansMax = 4096;   // deep plans of a batch up to which they are evaluated a warp per plan
 // CM_CLASS_SHORT: pipelines of at most kRegStagesMax stages with fewer micro-batches than warm-up slots (m < S-1).
 // CM_CLASS_SOLO: segments deeper than kRegStagesMax whose only candidate is the min-max partition.
 // One plan is one dependent chain (2*S*m cells, ~100 us in a single thread); a warp walks it in
