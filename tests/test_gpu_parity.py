@@ -485,6 +485,32 @@ def test_deep_pipelines_across_every_switch(gpu, oracle_factory, seed):
                 s.close()
 
 
+@pytest.mark.parametrize("sched", [W.SCHED_1F1B, W.SCHED_GPIPE])
+def test_pipelines_of_62_to_64_stages(gpu, oracle_factory, sched):
+    """The deepest pipelines the library takes: 16, 17 and 18 failures leave one pipeline of
+    64, 63 and 62 stages (both stages of the last lane in use, one, none), batched and one
+    failure at a time (a warp per plan and per tie-break composition), both cost modes."""
+    w = W.deep_pipeline(7)
+    rng = W.SplitMix64(62_64)
+    scen = [sorted(rng.sample_distinct(80, k)) for k in (16, 17, 18)]
+    base = w.options
+    for cap in (40, 3000):
+        w.options = W.SearchOptions(1, 2, 18, 64, base.layer_mode, base.batch_mode, cap, schedule=sched)
+        full_parity(gpu, oracle_factory, w, scen, candidates=cap == 40)
+        for mode in (0, 1):
+            opts = w.options.with_cost_mode(mode)
+            o = oracle_factory(w.profile, opts)
+            s = Session(gpu, w.profile)
+            try:
+                for _ in range(3):
+                    best, _, _ = gpu.cm_search_batch(s.ctx, scen, opts, latency=True)
+                for b, failed in enumerate(scen):
+                    want = o.search(failed)[0]
+                    assert_same_plan(gpu.plans_from_array(best)[b], want, mode, f"{failed} cap {cap} mode {mode} one at a time")
+            finally:
+                s.close()
+
+
 def test_handworked_readings_rerouting_redundant_memory_minmax_ties(gpu, oracle_factory):
     """The hand-worked cases that fix the readings taken where the paper prints no formula
     (``tests/golden/*_handworked.txt``): the library must give the fixtures' own numbers, not
