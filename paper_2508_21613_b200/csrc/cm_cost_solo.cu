@@ -39,8 +39,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_solo_kernel(Tables tb, BatchDe
                 const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
                 g_max = og > g_max ? og : g_max;
             }
-            const T t = S <= 32 ? warp_pipe_time<T, 1>(sp, cuts, S, m, g.tier, lane)
-                                : warp_pipe_time<T, 2>(sp, cuts, S, m, g.tier, lane);
+            const T t = warp_pipe_time<T>(sp, cuts, S, m, g.tier, lane);
             if (lane == 0) {
                 const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval));
                 if (bits < bd.seg_best[g.row]) atomicMin((unsigned long long *)&bd.seg_best[g.row], (unsigned long long)bits);
@@ -106,8 +105,7 @@ __global__ void __launch_bounds__(kChunk) cm_cost_warp_kernel(Tables tb, BatchDe
                 const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
                 g_max = og > g_max ? og : g_max;
             }
-            const T t = S <= 32 ? warp_pipe_time<T, 1>(sp, cuts, S, m, g.tier, lane)
-                                : warp_pipe_time<T, 2>(sp, cuts, S, m, g.tier, lane);
+            const T t = warp_pipe_time<T>(sp, cuts, S, m, g.tier, lane);
             if (lane == 0) {
                 const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval));
                 if (bits < bd.seg_best[g.row]) atomicMin((unsigned long long *)&bd.seg_best[g.row], (unsigned long long)bits);

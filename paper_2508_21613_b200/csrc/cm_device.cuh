@@ -511,13 +511,73 @@ __device__ __forceinline__ T sim_lockstep_n(int S, int m, const T *F, const T *B
     return __shfl_sync(0xffffffffu, clock[0], 0);
 }
 
-// Bare time of one pipeline (no synchronisation term), its stages spread over the warp.
-template <typename T, int PER>
+// The 1F1B order with TWO consecutive stages per lane (stage 2l and 2l+1; S <= 64).  After the
+// warm-up slots a stage alternates forward and backward, even stages run their forwards in even
+// slots and odd stages in odd ones, so which kind of work each of a lane's two stages can do in
+// a slot is known at compile time once the loop takes an even and an odd slot per iteration:
+// no selects between forward and backward operands.  In the odd slot both inputs are the lane's
+// own (the forward of stage 2l feeds stage 2l+1, the backward of stage 2l+1 feeds stage 2l), so
+// only the even slot shuffles.  With h = slot / 2 and c = h + l + 1 - S the micro-batch tests are
+//   even slot: stage 2l   forward  j = h - l     runs iff 0 <= c - 1 < m - S + 2l
+//              stage 2l+1 backward j = c         runs iff 0 <= c < m
+//   odd slot:  stage 2l   backward j = c         runs iff 0 <= c < m
+//              stage 2l+1 forward  j = h - l     runs iff 0 <= c < m - S + 2l + 1
+// Same operations on the same operands as sim_lockstep_n: identical bits.
+template <typename T>
+__device__ __forceinline__ T sim_lockstep_pairs(int S, int m, const T *F, const T *B, const T *xt) {
+    const int lane = threadIdx.x & 31;
+    const bool valid0 = 2 * lane < S, valid1 = 2 * lane + 1 < S;
+    T clock0 = (T)0, clock1 = (T)0, last_f0 = (T)0, last_f1 = (T)0, last_b0 = (T)0, last_b1 = (T)0;
+    {   // slots 0 .. S-1: warm-up forwards only, forward (i,j) at slot i+j
+        int d0 = -2 * lane, d1 = -2 * lane - 1;
+        const unsigned m0 = valid0 ? (unsigned)m : 0u, m1 = valid1 ? (unsigned)m : 0u;
+        for (int s = 0; s < S; ++s) {
+            T up = __shfl_up_sync(0xffffffffu, last_f1, 1);
+            up = lane == 0 ? (T)0 : up;
+            const T fin0 = tmax(clock0, up) + F[0];
+            const T fin1 = tmax(clock1, last_f0) + F[1];
+            if ((unsigned)d0 < m0) { clock0 = fin0; last_f0 = fin0 + xt[0]; }
+            if ((unsigned)d1 < m1) { clock1 = fin1; last_f1 = fin1 + xt[1]; }
+            ++d0; ++d1;
+        }
+    }
+    const int f0 = m - S + 2 * lane;
+    const unsigned lim_f0 = valid0 && f0 > 0 ? (unsigned)f0 : 0u;
+    const unsigned lim_f1 = valid1 && f0 + 1 > 0 ? (unsigned)(f0 + 1) : 0u;
+    const unsigned lim_b0 = valid0 ? (unsigned)m : 0u, lim_b1 = valid1 ? (unsigned)m : 0u;
+    int h = S >> 1;
+    int c = h + lane + 1 - S;
+    auto odd_slot = [&]() {
+        const T fin0 = tmax(clock0, last_b1 + xt[0]) + B[0];
+        const T fin1 = tmax(clock1, last_f0) + F[1];
+        if ((unsigned)c < lim_b0) { clock0 = fin0; last_b0 = fin0; }
+        if ((unsigned)c < lim_f1) { clock1 = fin1; last_f1 = fin1 + xt[1]; }
+    };
+    if (S & 1) {   // slot S is odd
+        odd_slot();
+        ++h; ++c;
+    }
+    for (; h <= S + m - 2; ++h, ++c) {
+        T up = __shfl_up_sync(0xffffffffu, last_f1, 1);
+        T down = __shfl_down_sync(0xffffffffu, last_b0, 1);
+        up = lane == 0 ? (T)0 : up;       // the end lanes get their own value back from the shuffle
+        down = lane == 31 ? (T)0 : down;
+        const T fin0 = tmax(clock0, up) + F[0];
+        const T fin1 = tmax(clock1, down + xt[1]) + B[1];
+        if ((unsigned)(c - 1) < lim_f0) { clock0 = fin0; last_f0 = fin0 + xt[0]; }
+        if ((unsigned)c < lim_b1) { clock1 = fin1; last_b1 = fin1; }
+        odd_slot();
+    }
+    return __shfl_sync(0xffffffffu, clock0, 0);
+}
+
+// Bare time of one pipeline (no synchronisation term), its stages spread over the warp, two per lane.
+template <typename T>
 __device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *cuts, int S, int m, uint64_t tier, int lane) {
-    T F[PER], B[PER], xt[PER];
+    T F[2], B[2], xt[2];
 #pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        const int i = lane * PER + k;
+    for (int k = 0; k < 2; ++k) {
+        const int i = lane * 2 + k;
         F[k] = (T)0; B[k] = (T)0; xt[k] = (T)0;
         if (i < S) {
             const int lo = cuts[i], hi = cuts[i + 1];
@@ -526,7 +586,7 @@ __device__ __forceinline__ T warp_pipe_time(const SProf<T> &sp, const uint8_t *c
             if (i < S - 1) xt[k] = sp.XT[(tier >> i) & 1ull][hi - 1];
         }
     }
-    return sim_lockstep_n<T, PER>(S, m, F, B, xt, sp.sched);
+    return sp.sched == CM_SCHED_GPIPE ? sim_lockstep_n<T, 2>(S, m, F, B, xt, sp.sched) : sim_lockstep_pairs<T>(S, m, F, B, xt);
 }
 
 __device__ __forceinline__ uint64_t warp_min_u64(uint64_t v) {

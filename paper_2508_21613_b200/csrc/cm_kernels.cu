@@ -452,8 +452,7 @@ __global__ void __launch_bounds__(kWarpTieWarps * 32) cm_tiebreak_warp_kernel(Ta
                 const long long og = __shfl_xor_sync(0xffffffffu, g_max, o);
                 g_max = og > g_max ? og : g_max;
             }
-            const T t = S <= 32 ? warp_pipe_time<T, 1>(sp, cuts, S, m, g.tier, lane)
-                                : warp_pipe_time<T, 2>(sp, cuts, S, m, g.tier, lane);
+            const T t = warp_pipe_time<T>(sp, cuts, S, m, g.tier, lane);
             const uint64_t bits = Num<T>::bits(t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval));
             if (lane == 0 && bits <= w.cost_bits) atomicMin((unsigned long long *)slot, (unsigned long long)kappa);
         }

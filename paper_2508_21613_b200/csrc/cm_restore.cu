@@ -489,10 +489,7 @@ __global__ void __launch_bounds__(kMatchWarps * 32) cm_plan_rounds_kernel(Tables
     T t_pipe = (T)0;
     for (int q = 0; q < dp; ++q) {            // one pipeline after the other, each over the whole warp
         const SegView g = seg_view(bd, w.scen, w.seg[q]);
-        T t;
-        if (g.S <= 32) t = warp_pipe_time<T, 1>(sp, rw.cuts[q], g.S, g.m, g.tier, lane);
-        else t = warp_pipe_time<T, 2>(sp, rw.cuts[q], g.S, g.m, g.tier, lane);
-        t_pipe = tmax(t_pipe, t);
+        t_pipe = tmax(t_pipe, warp_pipe_time<T>(sp, rw.cuts[q], g.S, g.m, g.tier, lane));
     }
     int rounds = 0;
     for (int l = 0; l < L; ++l) {
