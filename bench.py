@@ -389,8 +389,10 @@ def measure_objective(binding, torch, w, mode, steps, warmup, local_rank, flush)
 
 def measure_shared(binding, torch, w, mode, local_rank, flush, steps=5):
     """The same batch with sharing on: failure sets that leave the same survivor count and node
-    boundaries have identical dynamic-parallelism searches and are searched once.  Not the
-    headline: `value` above evaluates every scenario's plans."""
+    boundaries have identical dynamic-parallelism searches and are searched once, and every
+    distinct segment (stages, micro-batches, peers, link tiers) of the batch is searched once for
+    all the scenarios and strategies it occurs in.  Not the headline: `value` above evaluates
+    every scenario's plans."""
     opts = w.options.with_cost_mode(mode)
     ctx = binding.cm_create(local_rank)
     binding.cm_load_profile(ctx, w.profile)
@@ -408,7 +410,9 @@ def measure_shared(binding, torch, w, mode, local_rank, flush, steps=5):
             wall += time.perf_counter() - t0
         st = binding.cm_last_stats(ctx)
         return {"scenarios": packed.B, "e2e_ms_per_step": 1e3 * wall / steps, "device_ms_per_step": 1e-6 * st["device_ns"],
-                "plans_evaluated_per_step": st["plans"], "scenarios_per_s": packed.B / (wall / steps)}
+                "plans_of_searched_scenarios_per_step": st["plans"], "plans_simulated_per_step": st["plans_simulated"],
+                "scenarios_per_s": packed.B / (wall / steps),
+                "host_ms_per_step": {"descriptors": 1e-6 * st["host_build_ns"], "upload_and_segment_keys": 1e-6 * st["host_upload_ns"]}}
     finally:
         binding.cm_destroy(ctx)
 

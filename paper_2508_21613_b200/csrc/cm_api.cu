@@ -116,6 +116,21 @@ struct Batch {
     bool intval = false;                   // integer mode evaluated in double arithmetic (fixed when the batch is built)
     uint64_t profile_gen = 0;              // generation of the profile the tables describe (see cm_ctx::profile_gen)
     bool mm_launched = false;              // the min-max partitions of `keys` were already enqueued (with the feasible lists)
+    // Segments shared between scenarios (sharing on, more than one scenario): classes = distinct
+    // (stages, micro-batches, peers), their table and list regions, the class of every template
+    // segment; the buckets are laid out in upload_batch, once the device has counted the distinct
+    // segments of every class.
+    bool useg = false;
+    struct USegInfo { uint16_t S, m, n_sync; uint64_t K; uint32_t feas_first, feas_count; uint64_t rows; };
+    std::vector<USegInfo> ucls_info;
+    std::vector<USegClass> ucls;
+    std::vector<uint32_t> tseg_cls;
+    size_t off_ucls = 0, off_tseg_cls = 0;
+    uint64_t utab_slots = 0, ulist_len = 0;
+    DevBuf<unsigned long long> d_utab;
+    DevBuf<uint32_t> d_urep, d_slot_of, d_ucount;
+    DevBuf<uint2> d_useg;
+    PinnedVec<uint32_t> ucount_host;
 };
 
 struct cm_ctx {
@@ -282,11 +297,24 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
 // (stages, micro-batches) into buckets (a bucket's segments are its template segments
 // times the template's scenarios), buckets grouped into launch classes: one per
 // (kernel kind, stage count); the short-pipeline and the one-plan kinds pool every depth in one class.
+struct PreBucket { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
+
+// Kernel kind of a bucket.  by_warp: the batch has so few deep plans that they go a warp per plan.
+int bucket_kind(bool by_warp, int S, int m, uint64_t n_seg, uint64_t K) {
+    if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_SHORT;
+    if (K == 0) return (int)CM_CLASS_SOLO;   // the min-max partition is the only candidate there is
+    if (by_warp) return (int)CM_CLASS_WARP;
+    if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
+    return (int)CM_CLASS_WIDE_UNI;           // deeper than kWideStagesMax: the transposed layout only
+}
+
+cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &pre);
+
 cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket.clear();
     bt.classes.clear();
     bt.bucket_tseg.clear();
-    struct Pre { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
+    using Pre = PreBucket;
     std::vector<Pre> pre;
     // plans of the deep pipelines that have a choice of composition, over the whole batch
     uint64_t deep_plans = 0;
@@ -297,14 +325,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 deep_plans += (g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : g.K + 1) * tp.n_scen;
         }
     const bool by_warp = deep_plans <= kWarpPlansMax;
-    auto kind_of = [by_warp](int S, int m, uint64_t n_seg, uint64_t K, uint64_t count) {
-        (void)count;
-        if (S <= kRegStagesMax) return m >= S - 1 ? (int)CM_CLASS_REGS : (int)CM_CLASS_SHORT;
-        if (K == 0) return (int)CM_CLASS_SOLO;   // the min-max partition is the only candidate there is
-        if (by_warp) return (int)CM_CLASS_WARP;
-        if (S <= kWideStagesMax) return n_seg >= (uint64_t)kUniMinSegments ? (int)CM_CLASS_WIDE_UNI : (int)CM_CLASS_WIDE_LANE;
-        return (int)CM_CLASS_WIDE_UNI;           // deeper than kWideStagesMax: the transposed layout only
-    };
+    auto kind_of = [by_warp](int S, int m, uint64_t n_seg, uint64_t K, uint64_t) { return bucket_kind(by_warp, S, m, n_seg, K); };
     std::vector<uint32_t> idx;
     for (size_t t = 0; t < bt.tmpl.size(); ++t) {
         const Tmpl &tp = bt.tmpl[t];
@@ -346,6 +367,12 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
             i = j;
         }
     }
+    return layout_buckets(ctx, bt, pre);
+}
+
+// Buckets and launch classes from the collected (template or shared-list) segment groups.
+cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &pre) {
+    using Pre = PreBucket;
     for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WARP; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
         const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO || kind == CM_CLASS_WARP;   // every depth in one class
@@ -395,6 +422,86 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     for (const LaunchClass &c : bt.classes)
         if (c.n_chunks >= (1ull << 44)) return fail(ctx, CM_EOVERFLOW, "candidate count does not fit the index type");
     return CM_OK;
+}
+
+// Segments shared between scenarios, host part 1: the classes (stages, micro-batches, peers) of
+// the template segments that are searched, with room for every row in the class's table (twice
+// the rows, a power of two) and list.  The bucket table gets two placeholder entries per class:
+// its real content follows once the device has counted the distinct segments.
+cm_status build_segment_classes(cm_ctx *ctx, Batch &bt) {
+    std::map<uint64_t, uint32_t> ids;
+    bt.tseg_cls.assign(bt.tseg.size(), kNoSegClass);
+    bt.ucls_info.clear();
+    bt.ucls.clear();
+    for (const Tmpl &tp : bt.tmpl) {
+        if (tp.n_scen == 0) continue;
+        for (uint32_t i = 0; i < tp.n_tseg; ++i) {
+            const TSeg &g = bt.tseg[tp.tseg_first + i];
+            if (g.m < 1) continue;                                                 // no work is scheduled: stays infeasible
+            if (g.feas_first != kNoFeasList && g.feas_count == 0) continue;       // nothing fits in memory
+            const uint64_t key = ((uint64_t)g.S << 32) | ((uint64_t)g.m << 16) | g.n_sync;
+            auto it = ids.find(key);
+            if (it == ids.end()) {
+                it = ids.emplace(key, (uint32_t)bt.ucls_info.size()).first;
+                bt.ucls_info.push_back(Batch::USegInfo{g.S, g.m, g.n_sync, g.K, g.feas_first, g.feas_count, 0});
+            }
+            bt.ucls_info[it->second].rows += tp.n_scen;
+            bt.tseg_cls[tp.tseg_first + i] = it->second;
+        }
+    }
+    uint64_t slots = 0, list = 0;
+    for (const Batch::USegInfo &u : bt.ucls_info) {
+        uint64_t cap = 64;
+        while (cap < 2 * u.rows) cap <<= 1;
+        bt.ucls.push_back(USegClass{(uint32_t)slots, (uint32_t)(cap - 1), (uint32_t)list, 0});
+        slots += cap;
+        list += u.rows;
+        if (slots >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "batch too large for the index type");
+    }
+    bt.utab_slots = slots;
+    bt.ulist_len = list;
+    bt.bucket.assign(std::max<size_t>(2 * bt.ucls_info.size(), 1), Bucket{});
+    bt.classes.clear();
+    bt.bucket_tseg.clear();
+    return CM_OK;
+}
+
+// Host part 2: one bucket per class over its list of distinct segments (counted on the device).
+// What does not fill most of a last transposed warp goes to the per-lane kernel.
+cm_status build_shared_buckets(cm_ctx *ctx, Batch &bt, const uint32_t *n_distinct) {
+    const size_t room = bt.bucket.size();
+    bt.bucket.clear();
+    bt.classes.clear();
+    std::vector<PreBucket> pre;
+    auto count_of = [](const Batch::USegInfo &u) {
+        return u.feas_first != kNoFeasList ? (uint64_t)u.feas_count : (u.K ? u.K + 1 : 1);
+    };
+    uint64_t deep_plans = 0;
+    for (size_t c = 0; c < bt.ucls_info.size(); ++c) {
+        const Batch::USegInfo &u = bt.ucls_info[c];
+        if (u.S > kRegStagesMax && u.K > 0) deep_plans += count_of(u) * n_distinct[c];
+    }
+    const bool by_warp = deep_plans <= kWarpPlansMax;
+    for (size_t c = 0; c < bt.ucls_info.size(); ++c) {
+        const Batch::USegInfo &u = bt.ucls_info[c];
+        const uint32_t n = n_distinct[c];
+        if (n == 0) continue;
+        if (n > u.rows) return fail(ctx, CM_ECUDA, "internal: more distinct segments than rows");
+        uint32_t cut = n;
+        if (bucket_kind(by_warp, u.S, u.m, n, u.K) == CM_CLASS_WIDE_UNI && u.S <= kWideStagesMax) {
+            const uint32_t rest = n % 32;
+            if (rest > 0 && rest < (uint32_t)kUniMinSegments) cut = n - rest;
+        }
+        for (int part = 0; part < 2; ++part) {
+            const uint32_t p0 = part ? cut : 0, p1 = part ? n : cut;
+            if (p1 <= p0) continue;
+            pre.push_back(PreBucket{kSharedBucket, bt.ucls[c].list_first + p0, 0, u.S, u.m, count_of(u), p1 - p0,
+                                    bucket_kind(by_warp, u.S, u.m, p1 - p0, u.K), u.feas_first});
+        }
+    }
+    cm_status s = layout_buckets(ctx, bt, pre);
+    if (s == CM_OK && bt.bucket.size() > room) return fail(ctx, CM_ECUDA, "internal: bucket table outgrew its room");
+    return s;
 }
 
 // The template of a survivor count (Algorithm 1, get_parallel_strategy, plus the batch
@@ -698,6 +805,12 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
         ctx->stats[17] += now_ns() - t0;
         if (s != CM_OK) return s;
     }
+    // With sharing on, a batch of several scenarios also shares SEGMENTS: the distinct (stages,
+    // micro-batches, peers, link tiers) are found on the device once the tables are there.
+    bt.useg = ctx->share && ctx->d_prof && B > 1 && (policy_mask & (1u << CM_DYNPAR)) && rows > 0;
+    if (bt.useg) return build_segment_classes(ctx, bt);
+    bt.ucls.clear();
+    bt.tseg_cls.clear();
     return build_buckets(ctx, bt);
 }
 
@@ -720,6 +833,7 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.tmpl_scen = (const uint32_t *)(a + bt.off_tmpl_scen); v.bucket = (const Bucket *)(a + bt.off_bucket);
     v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
     v.feas = ctx->d_feas.p;
+    v.useg = bt.d_useg.p;
     v.seg_best = bt.d_seg_best.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
@@ -732,6 +846,17 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     for (const Tmpl &tp : bt.tmpl) v.max_red_per_scen = std::max(v.max_red_per_scen, tp.n_scen ? tp.n_red : 0u);
     v.layer_mode = bt.opts.lm; v.batch_mode = bt.opts.bm;
     return v;
+}
+
+USegDev useg_view(const Batch &bt) {
+    USegDev u{};
+    u.cls = (const USegClass *)(bt.d_arena.p + bt.off_ucls);
+    u.tseg_cls = (const uint32_t *)(bt.d_arena.p + bt.off_tseg_cls);
+    u.tab = bt.d_utab.p; u.rep = bt.d_urep.p; u.slot_of = bt.d_slot_of.p; u.count = bt.d_ucount.p; u.list = bt.d_useg.p;
+    u.n_cls = (uint32_t)bt.ucls.size();
+    u.n_rep_scen = 0;
+    for (const Tmpl &tp : bt.tmpl) u.n_rep_scen += tp.n_scen;
+    return u;
 }
 
 Tables tables(const cm_ctx *ctx, const Batch &bt) {
@@ -764,6 +889,8 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     bt.off_tmpl_scen = arena_put(bt.arena, bt.tmpl_scen, ok);
     bt.off_bucket_tseg = arena_put(bt.arena, bt.bucket_tseg, ok);
     bt.off_cross = arena_put(bt.arena, bt.cross, ok);
+    bt.off_ucls = arena_put(bt.arena, bt.ucls, ok);
+    bt.off_tseg_cls = arena_put(bt.arena, bt.tseg_cls, ok);
     bt.off_bucket = arena_put(bt.arena, bt.bucket, ok);
     if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
     if (!bt.d_arena.reserve(bt.arena.size())) return fail(ctx, CM_ENOMEM, "device memory");
@@ -779,6 +906,33 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
         CM_CUDA(ctx, launch_minmax(tables(ctx, bt), (const uint32_t *)(bt.d_arena.p + bt.off_keys),
                                    (int)bt.keys.size(), bt.intval ? CM_COST_FP64 : bt.opts.cost, ctx->stream));
         if (launches) ++*launches;
+    }
+    if (bt.useg) {
+        // key every row, list the distinct segments, count them per class; the counts decide the
+        // work layout, so they come back (one small copy, one synchronisation) before the buckets
+        // are laid out and their table -- the last section of the arena -- is copied again
+        const size_t n_cls = bt.ucls.size();
+        ok = bt.d_utab.reserve(std::max<uint64_t>(bt.utab_slots, 1)) && bt.d_urep.reserve(std::max<uint64_t>(bt.utab_slots, 1)) &&
+             bt.d_slot_of.reserve(std::max<uint64_t>(bt.n_rows, 1)) && bt.d_ucount.reserve(n_cls + 1) &&
+             bt.d_useg.reserve(std::max<uint64_t>(bt.ulist_len, 1)) && bt.ucount_host.resize(n_cls + 1);
+        if (!ok) return fail(ctx, CM_ENOMEM, "memory");
+        CM_CUDA(ctx, cudaMemsetAsync(bt.d_utab.p, 0xFF, bt.utab_slots * sizeof(unsigned long long), ctx->stream));
+        CM_CUDA(ctx, cudaMemsetAsync(bt.d_urep.p, 0xFF, bt.utab_slots * sizeof(uint32_t), ctx->stream));
+        CM_CUDA(ctx, cudaMemsetAsync(bt.d_ucount.p, 0, (n_cls + 1) * sizeof(uint32_t), ctx->stream));
+        CM_CUDA(ctx, launch_useg_keys(dev_view(ctx, bt), useg_view(bt), ctx->stream));
+        if (launches) *launches += 2;
+        CM_CUDA(ctx, cudaMemcpyAsync(bt.ucount_host.p, bt.d_ucount.p, (n_cls + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream));
+        CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        ctx->stats[10] += (n_cls + 1) * sizeof(uint32_t);
+        if (bt.ucount_host[n_cls] != 0) return fail(ctx, CM_ECUDA, "internal: segment table full");
+        cm_status s = build_shared_buckets(ctx, bt, bt.ucount_host.p);
+        if (s != CM_OK) return s;
+        if (!bt.bucket.empty()) {
+            memcpy(bt.arena.p + bt.off_bucket, bt.bucket.data(), bt.bucket.size() * sizeof(Bucket));
+            CM_CUDA(ctx, cudaMemcpyAsync(bt.d_arena.p + bt.off_bucket, bt.arena.p + bt.off_bucket, bt.bucket.size() * sizeof(Bucket),
+                                         cudaMemcpyHostToDevice, ctx->stream));
+            ctx->stats[9] += bt.bucket.size() * sizeof(Bucket);
+        }
     }
     return CM_OK;
 }
@@ -808,6 +962,10 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[2], st));
         CM_CUDA(ctx, launch_cost_pass1(tb, bd, bt.classes.data(), (int)bt.classes.size(), st, &ctx->side, &cost_launches));
         launches += cost_launches;
+        if (bt.useg) {   // rows that share a segment take its representative's minimum
+            CM_CUDA(ctx, launch_useg_copy(bd, useg_view(bt), st));
+            ++launches;
+        }
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
         CM_CUDA(ctx, launch_split_reduce(tb, bd, st));
         launches += (bd.n_red_blocks && bd.max_red_per_scen > 1) ? 2 : 1;

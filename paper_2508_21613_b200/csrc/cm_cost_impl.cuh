@@ -61,6 +61,10 @@ __device__ __forceinline__ void plan_of_thread(uint64_t base, uint64_t count, ui
 // Segment number `seg_local` of a bucket = (template segment of the bucket, scenario of the
 // template), scenario minor.
 __device__ __forceinline__ SegView bucket_segment(const BatchDev &bd, const Bucket &bk, uint32_t seg_local) {
+    if (bk.tmpl == kSharedBucket) {   // a range of the list of distinct segments
+        const uint2 p = bd.useg[bk.list_first + seg_local];
+        return seg_view(bd, p.x, p.y);
+    }
     const Tmpl &tp = bd.tmpl[bk.tmpl];
     const uint32_t ti = seg_local / tp.n_scen, si = seg_local - ti * tp.n_scen;
     return seg_view(bd, bd.tmpl_scen[tp.scen_first + si], bd.bucket_tseg[bk.list_first + ti]);

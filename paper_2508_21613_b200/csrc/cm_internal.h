@@ -105,6 +105,31 @@ struct Bucket {
     uint32_t feas_first;   // count = length of this list if there is one (kNoFeasList: count = K+1 or 1)
 };
 
+// Segments shared between scenarios.  The least cost of a segment over its layer compositions
+// depends on its stages, micro-batches, data-parallel peers and the link tiers of its S-1
+// boundaries -- not on the scenario or the strategy it belongs to (Section "Estimator": a
+// pipeline's time is a function of its own stages and links).  With sharing on, the segments
+// of a batch are keyed by exactly that, every distinct key is searched once, and the other
+// rows copy the result.  A class = (S, m, peers); within a class the key is the tier word,
+// found in an open-addressing table; a bucket with tmpl == kSharedBucket walks a range of the
+// (scenario, template segment) list of the distinct segments of one class.
+constexpr uint32_t kSharedBucket = 0xffffffffu;
+constexpr uint32_t kNoSegClass = 0xffffffffu;   // template segment that is not searched (no micro-batches, nothing fits)
+struct USegClass {
+    uint32_t tab_first, tab_mask;   // its table: slots tab_first .. tab_first + tab_mask (a power of two of them)
+    uint32_t list_first, pad;       // its distinct segments: list entries list_first .. list_first + count - 1
+};
+struct USegDev {
+    const USegClass *cls;
+    const uint32_t *tseg_cls;       // class of every template segment (kNoSegClass: none)
+    unsigned long long *tab;        // tier words, all-ones = empty
+    uint32_t *rep;                  // per slot: lowest row with that key
+    uint32_t *slot_of;              // per row: its slot (kNoSegClass: none)
+    uint32_t *count;                // per class: distinct segments; count[n_cls]: probes that found no slot (never)
+    uint2 *list;                    // (scenario, template segment) of every distinct segment, by class
+    uint32_t n_cls, n_rep_scen;
+};
+
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
@@ -162,6 +187,7 @@ struct BatchDev {
     const Bucket *bucket;         // search-pass work layout
     const uint32_t *bucket_tseg;  // template segment rows grouped by bucket
     const uint32_t *feas;         // feasible-composition pool of the context
+    const uint2 *useg;            // distinct segments of a batch searched with sharing (buckets with tmpl == kSharedBucket)
     uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
     const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
     Partial *partial;       // [n_red_blocks]
@@ -235,6 +261,10 @@ cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys,
 cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *keys_dev, const uint64_t *K_dev,
                             const uint32_t *first_dev, int n_keys, uint32_t *pool, uint32_t *count_dev, cudaStream_t st);
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st);
+// segments shared between scenarios: key every row and list the distinct ones (tab, rep, count
+// cleared by the caller); after the search pass, give every other row its representative's result
+cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st);
+cudaError_t launch_useg_copy(const BatchDev &b, const USegDev &u, cudaStream_t st);
 // Tiles of a segment that the tie-break kernels take side by side (grid.y); the rest is
 // walked serially inside the CTA.  A single scenario gets every tile its own CTA (lowest
 // latency), a large batch about one CTA per (scenario, pipeline): most of those stop after

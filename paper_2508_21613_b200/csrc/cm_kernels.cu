@@ -200,6 +200,83 @@ cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *key
 }
 
 // ----------------------------------------------------------------------------------
+// Segments shared between scenarios (USegDev): one CTA per searched scenario, a thread per
+// template segment.  cm_useg_key_kernel finds or claims the slot of the row's tier word in its
+// class's table (linear probing, at most as many probes as the table has slots; a table holds
+// at least twice the rows of its class) and leaves the lowest row per slot as its
+// representative; cm_useg_list_kernel appends every representative to its class's list (the
+// order within a class is whatever the atomics give: results do not depend on it);
+// cm_useg_copy_kernel, after the search pass, gives every other row its representative's minimum.
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t mix64(uint64_t x) {
+    x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;
+    x ^= x >> 27; x *= 0x94d049bb133111ebull;
+    x ^= x >> 31;
+    return (uint32_t)x;
+}
+
+__global__ void __launch_bounds__(128) cm_useg_key_kernel(BatchDev bd, USegDev ud) {
+    const uint32_t scen_id = bd.tmpl_scen[blockIdx.x];
+    const Scen sc = bd.scen[scen_id];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
+    for (uint32_t i = threadIdx.x; i < tp.n_tseg; i += blockDim.x) {
+        const uint32_t trow = tp.tseg_first + i, row = sc.seg_base + i;
+        const uint32_t ci = ud.tseg_cls[trow];
+        uint32_t slot = kNoSegClass;
+        if (ci != kNoSegClass) {
+            const TSeg g = bd.tseg[trow];
+            const USegClass c = ud.cls[ci];
+            const unsigned long long tier = cut_bits(bd.cross + sc.cross_first, g.off, g.S - 1);   // < 2^63: never all-ones
+            uint32_t h = mix64(tier) & c.tab_mask;
+            for (uint32_t probe = 0; probe <= c.tab_mask; ++probe) {
+                const unsigned long long old = atomicCAS(&ud.tab[c.tab_first + h], ~0ull, tier);
+                if (old == ~0ull || old == tier) { slot = c.tab_first + h; break; }
+                h = (h + 1) & c.tab_mask;
+            }
+            if (slot == kNoSegClass) atomicAdd(&ud.count[ud.n_cls], 1u);
+            else atomicMin(&ud.rep[slot], row);
+        }
+        ud.slot_of[row] = slot;
+    }
+}
+
+__global__ void __launch_bounds__(128) cm_useg_list_kernel(BatchDev bd, USegDev ud) {
+    const uint32_t scen_id = bd.tmpl_scen[blockIdx.x];
+    const Scen sc = bd.scen[scen_id];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
+    for (uint32_t i = threadIdx.x; i < tp.n_tseg; i += blockDim.x) {
+        const uint32_t trow = tp.tseg_first + i, row = sc.seg_base + i;
+        const uint32_t slot = ud.slot_of[row];
+        if (slot == kNoSegClass || ud.rep[slot] != row) continue;
+        const uint32_t ci = ud.tseg_cls[trow];
+        const uint32_t pos = atomicAdd(&ud.count[ci], 1u);
+        ud.list[ud.cls[ci].list_first + pos] = make_uint2(scen_id, trow);
+    }
+}
+
+__global__ void __launch_bounds__(256) cm_useg_copy_kernel(BatchDev bd, USegDev ud) {
+    const uint32_t row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= bd.n_rows) return;
+    const uint32_t slot = ud.slot_of[row];
+    if (slot == kNoSegClass) return;
+    const uint32_t r = ud.rep[slot];
+    if (r != row) bd.seg_best[row] = bd.seg_best[r];   // representatives are only read here
+}
+
+cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st) {
+    if (u.n_rep_scen == 0) return cudaSuccess;
+    cm_useg_key_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u);
+    cm_useg_list_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_useg_copy(const BatchDev &b, const USegDev &u, cudaStream_t st) {
+    if (b.n_rows == 0) return cudaSuccess;
+    cm_useg_copy_kernel<<<(b.n_rows + 255) / 256, 256, 0, st>>>(b, u);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------
 // Locate the segment that owns a tile / a candidate: the last row whose first index is
 // not above the query (rows are sorted and every segment owns at least one).
 // ----------------------------------------------------------------------------------

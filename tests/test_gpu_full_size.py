@@ -52,8 +52,9 @@ def test_every_scenario_matches_the_stored_oracle_result(gpu, name, mode):
         gpu.cm_destroy(ctx)
 
 
+@pytest.mark.parametrize("share", [False, True])
 @pytest.mark.parametrize("mode", [0, 1])
-def test_every_paper_scale_scenario_under_the_second_order(gpu, mode):
+def test_every_paper_scale_scenario_under_the_second_order(gpu, mode, share):
     """The same comparison with the time model under the all-forward-all-backward order
     (tests/golden/search_paper-scale_gpipe_*.txt, `make_search_goldens.py paper-scale --schedule gpipe`)."""
     w = W.paper_scale()
@@ -64,6 +65,7 @@ def test_every_paper_scale_scenario_under_the_second_order(gpu, mode):
     ctx = gpu.cm_create(0)
     try:
         gpu.cm_load_profile(ctx, w.profile)
+        gpu.cm_set_sharing(ctx, share)
         best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, w.options.with_cost_mode(mode).with_schedule(W.SCHED_GPIPE))
         got = [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)]
         wrong = [b for b in range(len(want)) if got[b] != want[b]]
@@ -138,15 +140,16 @@ def test_full_objective_of_every_scenario_matches_the_stored_oracle_result(gpu, 
 
 
 @pytest.mark.parametrize("mode", [0, 1])
-@pytest.mark.parametrize("name", ["paper-scale", "175b-like"])
+@pytest.mark.parametrize("name", ["paper-scale", "70b-like", "175b-like", "sweep"])
 def test_shared_search_matches_the_stored_oracle_results(gpu, name, mode):
-    """With sharing on, scenarios whose dynamic-parallelism spaces coincide are searched once;
+    """With sharing on, scenarios whose dynamic-parallelism spaces coincide are searched once,
+    and so is every distinct segment (stages, micro-batches, peers, link tiers) of the batch;
     every scenario must still come out exactly as the oracle has it, in the plain search and
     in the full-objective search."""
     from types import SimpleNamespace
     w = W.ALL_WORKLOADS[name]()
     want = _stored(name, mode)
-    want_obj = _stored_objective(name, mode)
+    want_obj = _stored_objective(name, mode) if os.path.exists(goldens.objective_path(name, mode)) else None
     obj = W.ObjectiveOptions()
     k = obj.topk
     ctx = gpu.cm_create(0)
@@ -154,15 +157,20 @@ def test_shared_search_matches_the_stored_oracle_results(gpu, name, mode):
         gpu.cm_load_profile(ctx, w.profile)
         opts = w.options.with_cost_mode(mode)
         gpu.cm_search_batch(ctx, w.scenarios, opts)
-        plain_plans = gpu.cm_last_stats(ctx)["plans"]
+        plain_plans, plain_simulated = (gpu.cm_last_stats(ctx)[k_] for k_ in ("plans", "plans_simulated"))
         gpu.cm_set_sharing(ctx, True)
-        best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, opts)
-        shared_plans = gpu.cm_last_stats(ctx)["plans"]
-        got = [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)]
-        assert got == want
+        for _ in range(2):   # the distinct segments are listed in whatever order the atomics give: twice
+            best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, opts)
+            shared_plans, shared_simulated = (gpu.cm_last_stats(ctx)[k_] for k_ in ("plans", "plans_simulated"))
+            got = [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)]
+            assert got == want
         assert shared_plans <= plain_plans
         if name == "paper-scale":
             assert shared_plans * 20 < plain_plans        # 2576 failure sets fall into a few dozen classes
+        if name != "70b-like":                            # (there the memory screen leaves almost nothing to share)
+            assert shared_simulated * 30 < plain_simulated    # few distinct segments among the scenarios' pipelines
+        if want_obj is None:
+            return
         best, trans, sl, sb, _ = gpu.cm_search_objective(ctx, w.scenarios, opts, obj, shortlist=True)
         plans = gpu.plans_from_array(best)
         short = gpu.plans_from_array(sl)
