@@ -379,8 +379,14 @@ cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set
  * enters that policy's model.  With sharing on, cm_search_batch / cm_batch_prepare search
  * such scenarios once and copy the result; rerouting and redundant computation are always
- * evaluated per scenario.  Results are identical either way; cm_last_stats then counts only
- * the plans that were actually evaluated.  cm_cache_build always shares. */
+ * evaluated per scenario.  In a batch of more than one scenario the pipelines are shared as
+ * well: the least time of a pipeline over its layer compositions depends on its stages, its
+ * micro-batches, the data-parallel peers of its strategy and the link tiers of its stage
+ * boundaries only (Section "Estimator"), so the distinct such tuples of the batch are found on
+ * the device (one small device->host copy and one synchronisation of the context's stream per
+ * prepared batch) and each is searched once.  Results are identical either way; cm_last_stats
+ * [0] then counts only the plans of the scenarios that were searched and [16] only the plans
+ * whose recurrence ran.  cm_cache_build always shares. */
 cm_status cm_set_sharing(cm_ctx *ctx, int on);
 
 /* Device time and work of the objective pass of the last cm_search_objective (HOST out[8]):
