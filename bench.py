@@ -276,6 +276,16 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
                              "what": "one failure set, all policies, descriptor build to plan on host; third pass over "
                                      "the scenarios: the batch of that survivor count is resident and its launch "
                                      "sequence replays as a CUDA graph"}
+        # the same with sharing on: a failure set's duplicate pipelines (equal stages, micro-batches,
+        # peers and link tiers) are searched once where that saves enough to pay for launching the
+        # sequence directly instead of replaying the resident graph
+        binding.cm_set_sharing(ctx, True)
+        for _ in range(2):
+            lat_pack.search(ctx, opts, latency=True)
+        binding.cm_set_sharing(ctx, False)
+        lat = np.sort(lat_pack.latency[:lat_pack.B].astype(np.float64))
+        out["latency_us"]["shared_segments"] = {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
+                                                "max": float(lat[-1])}
     finally:
         binding.cm_destroy(ctx)
     if cold_latency:

@@ -131,6 +131,11 @@ struct Batch {
     DevBuf<uint32_t> d_urep, d_slot_of, d_ucount;
     DevBuf<uint2> d_useg;
     PinnedVec<uint32_t> ucount_host;
+    // A resident one-scenario batch searched with shared segments keeps its template buckets (the
+    // replayed graph uses them) and lays the shared ones out beside them, per search.
+    const Bucket *bucket_override = nullptr;
+    DevBuf<Bucket> d_alt_bucket;
+    PinnedVec<unsigned char> alt_stage;   // slot_of | rep | list | buckets, staged for the copies
 };
 
 struct cm_ctx {
@@ -428,7 +433,7 @@ cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &p
 // the template segments that are searched, with room for every row in the class's table (twice
 // the rows, a power of two) and list.  The bucket table gets two placeholder entries per class:
 // its real content follows once the device has counted the distinct segments.
-cm_status build_segment_classes(cm_ctx *ctx, Batch &bt) {
+void assign_segment_classes(Batch &bt) {
     std::map<uint64_t, uint32_t> ids;
     bt.tseg_cls.assign(bt.tseg.size(), kNoSegClass);
     bt.ucls_info.clear();
@@ -449,6 +454,10 @@ cm_status build_segment_classes(cm_ctx *ctx, Batch &bt) {
             bt.tseg_cls[tp.tseg_first + i] = it->second;
         }
     }
+}
+
+cm_status build_segment_classes(cm_ctx *ctx, Batch &bt) {
+    assign_segment_classes(bt);
     uint64_t slots = 0, list = 0;
     for (const Batch::USegInfo &u : bt.ucls_info) {
         uint64_t cap = 64;
@@ -830,7 +839,8 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.scen = (const Scen *)(a + bt.off_scen); v.tmpl = (const Tmpl *)(a + bt.off_tmpl);
     v.strat = (const Strat *)(a + bt.off_strat); v.tseg = (const TSeg *)(a + bt.off_tseg);
     v.failed = (const uint32_t *)(a + bt.off_failed); v.cross = (const uint64_t *)(a + bt.off_cross);
-    v.tmpl_scen = (const uint32_t *)(a + bt.off_tmpl_scen); v.bucket = (const Bucket *)(a + bt.off_bucket);
+    v.tmpl_scen = (const uint32_t *)(a + bt.off_tmpl_scen);
+    v.bucket = bt.bucket_override ? bt.bucket_override : (const Bucket *)(a + bt.off_bucket);
     v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
     v.feas = ctx->d_feas.p;
     v.useg = bt.d_useg.p;
@@ -1061,6 +1071,107 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far, cm_ctx::Single 
     ctx->stats[6] += bt.strat.size();
     ctx->stats[7] += bt.n_split;
     return CM_OK;
+}
+
+// One resident scenario searched with its duplicate segments removed (sharing on).  A single
+// failure set repeats pipelines too: strategies share stage counts, and a pipeline that starts a
+// whole number of nodes further on sees the same link tiers.  The few hundred template segments
+// are keyed on the host (class, tier word), sorted, and the distinct ones laid out as shared
+// buckets beside the template buckets; the sequence is launched directly (its grids change from
+// failure to failure, so the resident graph does not fit).  *done = false: too little would be
+// saved to pay for the direct launches -- the caller replays the graph as usual.
+constexpr uint64_t kShareSingleMinCells = 250000000ull;   // recurrence cells that sharing must save (~70 us of search pass)
+cm_status run_single_shared(cm_ctx *ctx, Batch &bt, int launches_so_far, bool *done) {
+    *done = false;
+    if (bt.B != 1 || !(bt.policy_mask & (1u << CM_DYNPAR)) || bt.scen.empty()) return CM_OK;
+    const Scen &sc = bt.scen[0];
+    const Tmpl &tp = bt.tmpl[sc.tmpl];
+    if (tp.n_tseg < 2) return CM_OK;
+    if (bt.tseg_cls.size() != bt.tseg.size()) assign_segment_classes(bt);   // once per resident batch
+    const size_t n_cls = bt.ucls_info.size();
+    struct Key { uint32_t cls; uint64_t tier; uint32_t row; };
+    std::vector<Key> keys;
+    keys.reserve(tp.n_tseg);
+    const uint64_t *words = bt.cross.data() + sc.cross_first;
+    for (uint32_t i = 0; i < tp.n_tseg; ++i) {
+        const uint32_t c = bt.tseg_cls[tp.tseg_first + i];
+        if (c == kNoSegClass) continue;
+        const TSeg &g = bt.tseg[tp.tseg_first + i];
+        const int w = g.off >> 6, sh = g.off & 63, n = g.S - 1;
+        uint64_t v = words[w] >> sh;
+        if (sh) v |= words[w + 1] << (64 - sh);
+        keys.push_back(Key{c, v & ((1ull << n) - 1ull), i});
+    }
+    std::sort(keys.begin(), keys.end(), [](const Key &a, const Key &b) {
+        return a.cls != b.cls ? a.cls < b.cls : a.tier != b.tier ? a.tier < b.tier : a.row < b.row;
+    });
+    auto cells_of = [&](uint32_t c) {
+        const Batch::USegInfo &u = bt.ucls_info[c];
+        const uint64_t count = u.feas_first != kNoFeasList ? (uint64_t)u.feas_count : (u.K ? u.K + 1 : 1);
+        return count * 2ull * u.S * u.m;
+    };
+    std::vector<uint32_t> counts(n_cls + 1, 0);
+    uint64_t all_cells = 0, distinct_cells = 0;
+    size_t n_distinct = 0;
+    for (size_t i = 0; i < keys.size(); ++i) {
+        const bool first = i == 0 || keys[i].cls != keys[i - 1].cls || keys[i].tier != keys[i - 1].tier;
+        all_cells += cells_of(keys[i].cls);
+        if (first) { distinct_cells += cells_of(keys[i].cls); ++counts[keys[i].cls]; ++n_distinct; }
+    }
+    if (all_cells - distinct_cells < kShareSingleMinCells) return CM_OK;
+
+    // staging: slot_of [rows] | rep [distinct] | list [distinct] | buckets [2 per class]
+    const size_t rows = bt.n_rows, max_buckets = std::max<size_t>(2 * n_cls, 1);
+    const size_t off_rep = 4 * rows, off_list = (off_rep + 4 * n_distinct + 7) & ~(size_t)7;
+    const size_t off_bk = (off_list + 8 * n_distinct + 15) & ~(size_t)15, bytes = off_bk + max_buckets * sizeof(Bucket);
+    bool ok = bt.alt_stage.resize(bytes) && bt.d_slot_of.reserve(std::max<size_t>(rows, 1)) && bt.d_urep.reserve(std::max<size_t>(n_distinct, 1)) &&
+              bt.d_useg.reserve(std::max<size_t>(n_distinct, 1)) && bt.d_alt_bucket.reserve(max_buckets);
+    if (!ok) return fail(ctx, CM_ENOMEM, "memory");
+    uint32_t *slot_of = (uint32_t *)bt.alt_stage.p, *rep = (uint32_t *)(bt.alt_stage.p + off_rep);
+    uint2 *list = (uint2 *)(bt.alt_stage.p + off_list);
+    std::fill(slot_of, slot_of + rows, kNoSegClass);
+    bt.ucls.assign(n_cls, USegClass{0, 0, 0, 0});
+    uint32_t first_of = 0;
+    for (size_t c = 0; c < n_cls; ++c) { bt.ucls[c].list_first = first_of; first_of += counts[c]; }
+    uint32_t u = 0;
+    for (size_t i = 0; i < keys.size(); ++i) {
+        const bool first = i == 0 || keys[i].cls != keys[i - 1].cls || keys[i].tier != keys[i - 1].tier;
+        if (first) {   // keys are sorted by class, so list positions follow the class regions
+            rep[u] = sc.seg_base + keys[i].row;
+            list[u] = make_uint2(0u, tp.tseg_first + keys[i].row);
+            ++u;
+        }
+        slot_of[sc.seg_base + keys[i].row] = u - 1;
+    }
+    std::vector<Bucket> keep_buckets;
+    std::vector<LaunchClass> keep_classes;
+    keep_buckets.swap(bt.bucket);
+    keep_classes.swap(bt.classes);
+    bt.bucket.assign(max_buckets, Bucket{});
+    cm_status s = build_shared_buckets(ctx, bt, counts.data());
+    cudaError_t e = cudaSuccess;
+    if (s == CM_OK) {
+        if (!bt.bucket.empty()) memcpy(bt.alt_stage.p + off_bk, bt.bucket.data(), bt.bucket.size() * sizeof(Bucket));
+        cudaStream_t st = ctx->stream;
+        e = cudaMemcpyAsync(bt.d_slot_of.p, slot_of, 4 * rows, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && n_distinct) e = cudaMemcpyAsync(bt.d_urep.p, rep, 4 * n_distinct, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && n_distinct) e = cudaMemcpyAsync(bt.d_useg.p, list, 8 * n_distinct, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && !bt.bucket.empty())
+            e = cudaMemcpyAsync(bt.d_alt_bucket.p, bt.alt_stage.p + off_bk, bt.bucket.size() * sizeof(Bucket), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) {
+            ctx->stats[9] += 4 * rows + 12 * n_distinct + bt.bucket.size() * sizeof(Bucket);
+            bt.bucket_override = bt.d_alt_bucket.p;
+            bt.useg = true;
+            s = run_batch(ctx, bt, launches_so_far, nullptr);
+            *done = s == CM_OK;
+        }
+    }
+    bt.useg = false;
+    bt.bucket_override = nullptr;
+    bt.bucket.swap(keep_buckets);
+    bt.classes.swap(keep_classes);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(ctx, CM_ECUDA, std::string("shared segments: ") + cudaGetErrorString(e)); }
+    return s;
 }
 
 // Keys of min-max partitions that were scheduled but never computed must be asked for
@@ -1542,7 +1653,14 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         cm_ctx::Single *entry = nullptr;
         if ((s = single_batch(ctx, failed_ids + offsets[b], offsets[b + 1] - offsets[b], *opts, mask, &sb, &launches, &entry)) != CM_OK) return s;
         ctx->stats[13] += now_ns() - h0;
-        if ((s = run_batch(ctx, *sb, launches, entry)) != CM_OK) return s;
+        bool done = false;
+        if (ctx->share && entry) {
+            const uint64_t h1 = now_ns();
+            s = run_single_shared(ctx, *sb, launches, &done);
+            if (!done) ctx->stats[13] += now_ns() - h1;   // (the keys were built and found not worth using)
+            if (s != CM_OK) return s;
+        }
+        if (!done && (s = run_batch(ctx, *sb, launches, entry)) != CM_OK) return s;
         for (int pol = 0; pol < 3; ++pol) {
             cm_plan pl = sb->plans_host[pol];
             scrub(pl);

@@ -74,25 +74,35 @@ def test_every_paper_scale_scenario_under_the_second_order(gpu, mode, share):
         gpu.cm_destroy(ctx)
 
 
+@pytest.mark.parametrize("share", [False, True])
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("name,picks", [("70b-like", range(64)), ("175b-like", range(0, 64, 3)), ("sweep", range(0, 256, 7))])
-def test_one_failure_at_a_time_matches_the_stored_oracle_result(gpu, name, picks, mode):
+def test_one_failure_at_a_time_matches_the_stored_oracle_result(gpu, name, picks, mode, share):
     """The per-failure path (cm_search_batch with a latency buffer handles one failure set at a time: its own launch classes --
     a warp per plan where the memory screen leaves few deep plans -- the lock-step tie-break
     pass and, from the second search of a survivor count on, the replayed launch graph), each
-    scenario searched three times in a row, against the same stored oracle results."""
+    scenario searched three times in a row, against the same stored oracle results.  With
+    sharing on, a failure set whose duplicate pipelines are worth removing is searched over its
+    distinct segments instead (keyed on the host, launched directly)."""
     w = W.ALL_WORKLOADS[name]()
     want = _stored(name, mode)
     opts = w.options.with_cost_mode(mode)
     ctx = gpu.cm_create(0)
     try:
         gpu.cm_load_profile(ctx, w.profile)
+        gpu.cm_set_sharing(ctx, share)
+        saved = 0
         for b in picks:
             for rep in range(3):
                 best, _, lat = gpu.cm_search_batch(ctx, [w.scenarios[b]], opts, latency=True)
                 assert lat[0] > 0
                 got = goldens.line_of(gpu.plans_from_array(best)[0], mode)
                 assert got == want[b], f"scenario {b} {w.scenarios[b]} (search {rep}): got {got} want {want[b]}"
+                st = gpu.cm_last_stats(ctx)
+                if rep == 2 and share and name != "70b-like":
+                    saved += st["plans"] > 3 * st["plans_simulated"]
+        if share and name != "70b-like":
+            assert saved > 0   # some failure sets of these jobs repeat most of their pipelines
     finally:
         gpu.cm_destroy(ctx)
 
