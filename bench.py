@@ -660,6 +660,8 @@ def main():
                     "ms_per_step": 1e3 * em["dev_seconds"] / n_extra, "e2e_ms_per_step": 1e3 * em["e2e_seconds"] / n_extra,
                     "latency_us_p50": em["latency_us"]["p50"], "latency_us_p99": em["latency_us"]["p99"],
                     "latency_us_cold_p50": em["latency_us"]["cold"]["p50"], "latency_us_cold_p99": em["latency_us"]["cold"]["p99"],
+                    "latency_us_shared_segments_p50": em["latency_us"]["shared_segments"]["p50"],
+                    "latency_us_shared_segments_p99": em["latency_us"]["shared_segments"]["p99"],
                     "latency_scenarios": em["latency_us"]["scenarios"],
                     "search_pass_kernel": r["kernel"], "search_pass_gcell_s": r["achieved"],
                     "search_pass_frac": r["frac"], "search_pass_frac_of_fp64_pipe": r["frac_of_fp64_pipe"],

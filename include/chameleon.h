@@ -384,7 +384,10 @@ cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
  * micro-batches, the data-parallel peers of its strategy and the link tiers of its stage
  * boundaries only (Section "Estimator"), so the distinct such tuples of the batch are found on
  * the device (one small device->host copy and one synchronisation of the context's stream per
- * prepared batch) and each is searched once.  Results are identical either way; cm_last_stats
+ * prepared batch) and each is searched once.  A single failure set searched through the latency
+ * path of cm_search_batch has its duplicate pipelines removed on the host when enough work is
+ * saved to pay for launching its sequence directly instead of replaying the resident graph.
+ * Results are identical either way; cm_last_stats
  * [0] then counts only the plans of the scenarios that were searched and [16] only the plans
  * whose recurrence ran.  cm_cache_build always shares. */
 cm_status cm_set_sharing(cm_ctx *ctx, int on);
