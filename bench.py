@@ -290,10 +290,12 @@ def measure(binding, torch, w, mode, steps, warmup, local_rank, barrier, flush, 
         binding.cm_destroy(ctx)
     if cold_latency:
         out["latency_us"]["cold"] = measure_cold_latency(binding, w, opts, local_rank, native_i64)
+        cold = measure_cold_latency(binding, w, opts, local_rank, native_i64, share=True)
+        out["latency_us"]["shared_segments"]["cold"] = {k: cold[k] for k in ("p50", "p99", "max", "scenarios")}
     return out
 
 
-def measure_cold_latency(binding, w, opts, local_rank, native_i64=False, max_sizes=16):
+def measure_cold_latency(binding, w, opts, local_rank, native_i64=False, max_sizes=16, share=False):
     """A failure is a first occurrence: the latency of the FIRST search of a survivor count on a
     context that has searched nothing yet (profile loaded; no resident batch, no captured graph,
     min-max partitions not computed).  One fresh context and one scenario per failure-set size of
@@ -309,6 +311,7 @@ def measure_cold_latency(binding, w, opts, local_rank, native_i64=False, max_siz
             binding.cm_load_profile(ctx, w.profile)
             if native_i64:
                 binding.cm_set_int64_arithmetic(ctx, True)
+            binding.cm_set_sharing(ctx, share)
             pack = binding.PackedScenarios([by_size[size]])
             pack.search(ctx, opts, latency=True)
             lat.append(float(pack.latency[0]))

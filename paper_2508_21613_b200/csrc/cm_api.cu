@@ -1654,7 +1654,7 @@ cm_status cm_search_batch(cm_ctx *ctx, const uint32_t *failed_ids, const int32_t
         if ((s = single_batch(ctx, failed_ids + offsets[b], offsets[b + 1] - offsets[b], *opts, mask, &sb, &launches, &entry)) != CM_OK) return s;
         ctx->stats[13] += now_ns() - h0;
         bool done = false;
-        if (ctx->share && entry) {
+        if (ctx->share) {
             const uint64_t h1 = now_ns();
             s = run_single_shared(ctx, *sb, launches, &done);
             if (!done) ctx->stats[13] += now_ns() - h1;   // (the keys were built and found not worth using)
