@@ -374,6 +374,17 @@ cm_status cm_set_latency_graphs(cm_ctx *ctx, int on);
  * makes batches and spaces built afterwards test every composition inside the search pass. */
 cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
 
+/* Micro-batch pairs (on by default).  A pipeline of a strategy appears with two micro-batch
+ * counts, m and m + 1 (the two shares the remainder rule leaves it; consecutive counts under the
+ * full split enumeration).  Under the 1F1B order the recurrences of the two coincide in every
+ * round before the ramp-down of the shorter one -- whether micro-batch m exists shows first in
+ * round m -- so for pipelines of 17 to 48 stages with m >= stages one thread evaluates both: the
+ * common rounds once, then the two tails.  Same operations on the same values: results are
+ * bit-identical; cm_last_stats [1] counts the recurrence cells that actually ran.
+ * cm_set_micro_batch_pairs(ctx, 0) makes batches and spaces built afterwards evaluate every
+ * segment on its own. */
+cm_status cm_set_micro_batch_pairs(cm_ctx *ctx, int on);
+
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
  * with node boundaries at the same places among them have identical dynamic-parallelism
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set

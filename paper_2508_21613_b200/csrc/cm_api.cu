@@ -122,6 +122,10 @@ struct Batch {
     // segments of every class.
     bool useg = false;
     struct USegInfo { uint16_t S, m, n_sync; uint64_t K; uint32_t feas_first, feas_count; uint64_t rows; };
+    // Role of every template segment in the search pass: on its own, head of a micro-batch pair
+    // (evaluated together with the next row), or that next row.
+    enum : uint8_t { kAlone = 0, kPairHead = 1, kPairPartner = 2 };
+    std::vector<uint8_t> role;
     std::vector<USegInfo> ucls_info;
     std::vector<USegClass> ucls;
     std::vector<uint32_t> tseg_cls;
@@ -177,6 +181,7 @@ struct cm_ctx {
     PinnedVec<unsigned char> feas_stage;      // keys, K, offsets out; counts back
     DevBuf<unsigned char> d_feas_stage;
     bool screen = true;               // walk only the listed feasible compositions (cm_set_memory_screen)
+    bool pairs = true;                // one recurrence for a pipeline's m and m+1 micro-batch variants (cm_set_micro_batch_pairs)
     Batch batch;                      // reused by cm_search_batch
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_obj[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // phases of the objective pass
@@ -302,7 +307,30 @@ cm_status check_opts(cm_ctx *ctx, const cm_enum_opts *o) {
 // (stages, micro-batches) into buckets (a bucket's segments are its template segments
 // times the template's scenarios), buckets grouped into launch classes: one per
 // (kernel kind, stage count); the short-pipeline and the one-plan kinds pool every depth in one class.
-struct PreBucket { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; };
+struct PreBucket { uint32_t tmpl, list_first, n_tseg; uint16_t S, m; uint64_t count; uint32_t n_seg; int kind; uint32_t feas_first; uint32_t pair; };
+
+// Micro-batch pairs (Bucket::pair): template segment t and t+1 are the same pipeline with m and
+// m+1 micro-batches (the two shares the remainder rule of Section "Planner" leaves a pipeline;
+// consecutive counts under the full split enumeration).  They pair up where one recurrence can
+// serve both and both walk the same compositions: 1F1B, a depth of the deep-pipeline kernels,
+// a choice of compositions, m >= S, equal feasible-list lengths.
+void mark_pairs(const cm_ctx *ctx, Batch &bt) {
+    bt.role.assign(bt.tseg.size(), Batch::kAlone);
+    if (!ctx->pairs || bt.opts.sched != CM_SCHED_1F1B) return;
+    for (const Tmpl &tp : bt.tmpl)
+        for (uint32_t i = 0; i + 1 < tp.n_tseg; ++i) {
+            const uint32_t t = tp.tseg_first + i;
+            if (bt.role[t] != Batch::kAlone) continue;
+            const TSeg &a = bt.tseg[t], &b = bt.tseg[t + 1];
+            const bool same_pipe = a.S == b.S && a.off == b.off && a.n_sync == b.n_sync && a.K == b.K && b.m == a.m + 1 &&
+                                   b.cand_first == a.cand_first + (a.K ? a.K + 1 : 1);
+            if (!same_pipe || a.S < kPairStagesMin || a.S > kPairStagesMax || a.K == 0 || a.m < a.S) continue;
+            if ((a.feas_first == kNoFeasList) != (b.feas_first == kNoFeasList) || a.feas_count != b.feas_count) continue;
+            if (a.feas_first != kNoFeasList && a.feas_count == 0) continue;
+            bt.role[t] = Batch::kPairHead;
+            bt.role[t + 1] = Batch::kPairPartner;
+        }
+}
 
 // Kernel kind of a bucket.  by_warp: the batch has so few deep plans that they go a warp per plan.
 int bucket_kind(bool by_warp, int S, int m, uint64_t n_seg, uint64_t K) {
@@ -321,6 +349,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     bt.bucket_tseg.clear();
     using Pre = PreBucket;
     std::vector<Pre> pre;
+    std::vector<uint8_t> role = bt.role;   // pairs too few for the transposed kernel are dissolved here, for this layout only
     // plans of the deep pipelines that have a choice of composition, over the whole batch
     uint64_t deep_plans = 0;
     for (const Tmpl &tp : bt.tmpl)
@@ -335,16 +364,35 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     for (size_t t = 0; t < bt.tmpl.size(); ++t) {
         const Tmpl &tp = bt.tmpl[t];
         if (tp.n_scen == 0 || tp.n_tseg == 0) continue;
-        idx.resize(tp.n_tseg);
-        for (uint32_t i = 0; i < tp.n_tseg; ++i) idx[i] = tp.tseg_first + i;
+        // micro-batch pairs go to the transposed kernel; a group of pair heads too small for it is
+        // evaluated as single segments instead
+        {
+            std::map<uint32_t, uint32_t> heads;   // (S << 16 | m) -> pair heads of the template
+            for (uint32_t i = 0; i < tp.n_tseg; ++i)
+                if (role[tp.tseg_first + i] == Batch::kPairHead) {
+                    const TSeg &g = bt.tseg[tp.tseg_first + i];
+                    ++heads[((uint32_t)g.S << 16) | g.m];
+                }
+            for (uint32_t i = 0; i < tp.n_tseg; ++i)
+                if (role[tp.tseg_first + i] == Batch::kPairHead) {
+                    const TSeg &g = bt.tseg[tp.tseg_first + i];
+                    const uint64_t n_pairs = (uint64_t)heads[((uint32_t)g.S << 16) | g.m] * tp.n_scen;
+                    if (bucket_kind(by_warp, g.S, g.m, n_pairs, g.K) != CM_CLASS_WIDE_UNI)
+                        role[tp.tseg_first + i] = role[tp.tseg_first + i + 1] = Batch::kAlone;
+                }
+        }
+        idx.clear();
+        for (uint32_t i = 0; i < tp.n_tseg; ++i)
+            if (role[tp.tseg_first + i] != Batch::kPairPartner) idx.push_back(tp.tseg_first + i);
         std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
             const TSeg &x = bt.tseg[a], &y = bt.tseg[b];
-            return x.S != y.S ? x.S < y.S : x.m < y.m;
+            return x.S != y.S ? x.S < y.S : x.m != y.m ? x.m < y.m : role[a] < role[b];
         });
         for (size_t i = 0; i < idx.size();) {
             size_t j = i;
             const TSeg &g = bt.tseg[idx[i]];
-            while (j < idx.size() && bt.tseg[idx[j]].S == g.S && bt.tseg[idx[j]].m == g.m) ++j;
+            const uint32_t pair = role[idx[i]] == Batch::kPairHead ? 1u : 0u;
+            while (j < idx.size() && bt.tseg[idx[j]].S == g.S && bt.tseg[idx[j]].m == g.m && role[idx[j]] == role[idx[i]]) ++j;
             if (g.m >= 1) {   // m = 0 cannot be feasible: no work is scheduled
                 const uint64_t n_seg = (uint64_t)(j - i) * tp.n_scen;
                 if (n_seg >= (1ull << 31)) return fail(ctx, CM_EOVERFLOW, "too many segments in one bucket");
@@ -355,7 +403,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 // not.  With one scenario the segments are few: what does not fill most of a
                 // last warp goes to the per-lane kernel, which wastes no lane.
                 size_t cut = j;
-                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, g.K, count) == CM_CLASS_WIDE_UNI) {
+                if (tp.n_scen == 1 && !pair && kind_of(g.S, g.m, n_seg, g.K, count) == CM_CLASS_WIDE_UNI) {
                     const size_t rest = (j - i) % 32;
                     if (rest > 0 && rest < (size_t)kUniMinSegments) cut = j - rest;
                 }
@@ -364,7 +412,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     if (p1 <= p0) continue;
                     const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
                     Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
-                          count, (uint32_t)ns, kind_of(g.S, g.m, ns, g.K, count), g.feas_first};
+                          count, (uint32_t)ns, pair ? (int)CM_CLASS_WIDE_PAIR : kind_of(g.S, g.m, ns, g.K, count), g.feas_first, pair};
                     for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
                     pre.push_back(q);
                 }
@@ -378,14 +426,15 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
 // Buckets and launch classes from the collected (template or shared-list) segment groups.
 cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &pre) {
     using Pre = PreBucket;
-    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WARP; ++kind) {
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WIDE_PAIR; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
         const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO || kind == CM_CLASS_WARP;   // every depth in one class
         LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
         for (int S = 1; S <= CM_MAX_STAGES; ++S) {
             LaunchClass cls{kind, S, kind_chunks, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};
             LaunchClass &c = pooled_kind ? pooled : cls;
-            if (kind == CM_CLASS_WIDE_UNI) {
+            const bool transposed = kind == CM_CLASS_WIDE_UNI || kind == CM_CLASS_WIDE_PAIR;
+            if (transposed) {
                 // a warp of the transposed kernel takes several consecutive items once the class
                 // is large enough to fill the GPU anyway
                 uint64_t items = 0;
@@ -406,7 +455,8 @@ cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &p
                 bk.S = q.S;
                 bk.m = q.m;
                 bk.feas_first = q.feas_first;
-                if (kind == CM_CLASS_WIDE_UNI) {
+                bk.pair = q.pair;
+                if (transposed) {
                     const uint64_t items = bk.count * ((bk.n_seg + 31) / 32);
                     const uint64_t per_cta = (uint64_t)(kChunk / 32) * c.uni_items;
                     c.n_chunks += (items + per_cta - 1) / per_cta;
@@ -433,6 +483,7 @@ cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &p
 // the template segments that are searched, with room for every row in the class's table (twice
 // the rows, a power of two) and list.  The bucket table gets two placeholder entries per class:
 // its real content follows once the device has counted the distinct segments.
+constexpr size_t kSharedBucketsPerClass = 2;   // transposed part and per-lane remainder
 void assign_segment_classes(Batch &bt) {
     std::map<uint64_t, uint32_t> ids;
     bt.tseg_cls.assign(bt.tseg.size(), kNoSegClass);
@@ -469,7 +520,7 @@ cm_status build_segment_classes(cm_ctx *ctx, Batch &bt) {
     }
     bt.utab_slots = slots;
     bt.ulist_len = list;
-    bt.bucket.assign(std::max<size_t>(2 * bt.ucls_info.size(), 1), Bucket{});
+    bt.bucket.assign(std::max<size_t>(kSharedBucketsPerClass * bt.ucls_info.size(), 1), Bucket{});
     bt.classes.clear();
     bt.bucket_tseg.clear();
     return CM_OK;
@@ -505,7 +556,7 @@ cm_status build_shared_buckets(cm_ctx *ctx, Batch &bt, const uint32_t *n_distinc
             const uint32_t p0 = part ? cut : 0, p1 = part ? n : cut;
             if (p1 <= p0) continue;
             pre.push_back(PreBucket{kSharedBucket, bt.ucls[c].list_first + p0, 0, u.S, u.m, count_of(u), p1 - p0,
-                                    bucket_kind(by_warp, u.S, u.m, p1 - p0, u.K), u.feas_first});
+                                    bucket_kind(by_warp, u.S, u.m, p1 - p0, u.K), u.feas_first, 0});
         }
     }
     cm_status s = layout_buckets(ctx, bt, pre);
@@ -816,6 +867,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     }
     // With sharing on, a batch of several scenarios also shares SEGMENTS: the distinct (stages,
     // micro-batches, peers, link tiers) are found on the device once the tables are there.
+    mark_pairs(ctx, bt);
     bt.useg = ctx->share && ctx->d_prof && B > 1 && (policy_mask & (1u << CM_DYNPAR)) && rows > 0;
     if (bt.useg) return build_segment_classes(ctx, bt);
     bt.ucls.clear();
@@ -1121,7 +1173,7 @@ cm_status run_single_shared(cm_ctx *ctx, Batch &bt, int launches_so_far, bool *d
     if (all_cells - distinct_cells < kShareSingleMinCells) return CM_OK;
 
     // staging: slot_of [rows] | rep [distinct] | list [distinct] | buckets [2 per class]
-    const size_t rows = bt.n_rows, max_buckets = std::max<size_t>(2 * n_cls, 1);
+    const size_t rows = bt.n_rows, max_buckets = std::max<size_t>(kSharedBucketsPerClass * n_cls, 1);
     const size_t off_rep = 4 * rows, off_list = (off_rep + 4 * n_distinct + 7) & ~(size_t)7;
     const size_t off_bk = (off_list + 8 * n_distinct + 15) & ~(size_t)15, bytes = off_bk + max_buckets * sizeof(Bucket);
     bool ok = bt.alt_stage.resize(bytes) && bt.d_slot_of.reserve(std::max<size_t>(rows, 1)) && bt.d_urep.reserve(std::max<size_t>(n_distinct, 1)) &&
@@ -1821,6 +1873,19 @@ cm_status cm_set_memory_screen(cm_ctx *ctx, int on) {
     if (!ctx) return CM_EINVAL;
     ctx->screen = on != 0;
     return CM_OK;
+}
+
+cm_status cm_set_micro_batch_pairs(cm_ctx *ctx, int on) {
+    if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
+    if ((on != 0) != ctx->pairs) {
+        // resident one-scenario batches were laid out under the other setting
+        if (ctx->stream) cudaStreamSynchronize(ctx->stream);
+        ctx->single.clear();
+    }
+    ctx->pairs = on != 0;
+    return CM_OK;
+    CM_API_END(ctx)
 }
 
 cm_status cm_set_sharing(cm_ctx *ctx, int on) {

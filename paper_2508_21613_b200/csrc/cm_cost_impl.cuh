@@ -91,6 +91,11 @@ __device__ __forceinline__ void segmented_min_commit(uint64_t *seg_best, uint32_
 // counters[2] the plans.
 constexpr int kWorkPlanShift = 40;
 __device__ __forceinline__ unsigned long long one_plan(unsigned long long cells) { return cells + (1ull << kWorkPlanShift); }
+// a pair (m and m + 1 micro-batches in one recurrence, sim_rounds_pair): the cells of the longer
+// recurrence plus the ramp-down of the shorter one (S-1 rounds of S backwards and S-1-q forwards)
+template <int S> __device__ __forceinline__ unsigned long long pair_plans(int m) {
+    return 2ull * S * (m + 1) + 3ull * S * (S - 1) / 2 + (2ull << kWorkPlanShift);
+}
 __device__ __forceinline__ void add_work(unsigned long long *counters, unsigned long long packed) {
     if (!packed) return;
     atomicAdd(&counters[0], packed & ((1ull << kWorkPlanShift) - 1ull));
@@ -335,6 +340,78 @@ __global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_wide_ke
     count_cells(&bd.counters[0], my_cells, cells_w);
 }
 
+// ----------------------------------------------------------------------------------
+// Micro-batch pairs, 17 <= S <= 48, transposed layout: every segment of the bucket stands for
+// itself (m micro-batches) and its next row (the same pipeline with m + 1); one recurrence
+// serves both (sim_rounds_pair).  Built only for 1F1B with m >= S, where the two walk the same
+// feasible compositions and have the same min-max partition (a stage holds S - i micro-batches
+// in flight either way), so the composition is set up once, with m.  What the two commits need
+// (row, peers) waits in the free last entry of the lane's transfer-time column, not in registers.
+// Dynamic shared memory as the transposed cm_cost_wide_kernel.
+// ----------------------------------------------------------------------------------
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_pair_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset, int uni_items) {
+    static_assert(S >= kPairStagesMin && S <= kPairStagesMax, "pairs exist for the register-resident deep kernels only");
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    __shared__ Bucket bks;
+    __shared__ unsigned long long st_kappa[kChunk / 32];
+    __shared__ long long st_gmax[kChunk / 32];
+    __shared__ int st_ok[kChunk / 32];
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    if (tid == 0) bks = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    if (lane == 0) { st_kappa[warp] = ~0ull; st_ok[warp] = 0; st_gmax[warp] = 0; cells_w[warp] = 0; }
+    __syncthreads();
+    constexpr bool kBatch = S <= CM_UNI_BATCH_STAGES;
+    FB<T> *fb = reinterpret_cast<FB<T> *>(dyn) + warp * S;
+    T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * 4 * S) + tid;           // [i * kChunk]
+    uint8_t *cuts = dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * S * kChunk + warp * (((S + 1) + 7) / 8 * 8);
+    unsigned long long *note = reinterpret_cast<unsigned long long *>(xcol + (S - 1) * kChunk);   // entry S-1 holds no transfer time
+    const int n_items = kBatch ? uni_items : 1;
+    for (int r = 0; r < n_items; ++r) {
+        const int m = bks.m;
+        const uint64_t item = ((chunk - bks.chunk_first) * (kChunk / 32) + warp) * (uint64_t)n_items + r;
+        const uint32_t n_groups = (bks.n_seg + 31) / 32;
+        const uint64_t pos = item / n_groups;
+        if (pos >= bks.count) break;                       // warp-uniform; items ascend
+        const uint64_t kappa = walk_kappa(bd.feas, bks.feas_first, pos);
+        const uint32_t seg_local = (uint32_t)(item - pos * n_groups) * 32 + lane;
+        const bool active = seg_local < bks.n_seg;
+        const SegView g = bucket_segment(bd, bks, active ? seg_local : 0);
+        if (kappa != st_kappa[warp]) {
+            long long g_max;
+            const bool ok = uni_composition<T, S>(sp, tb, bd.layer_mode, m, kappa, g.K, fb, cuts, lane, g_max);
+            if (lane == 0) { st_kappa[warp] = kappa; st_ok[warp] = ok ? 1 : 0; st_gmax[warp] = g_max; }
+            __syncwarp();
+        }
+        if (st_ok[warp]) {
+            for (int i = 0; i < S - 1; ++i) xcol[i * kChunk] = sp.XT[(g.tier >> i) & 1ull][cuts[i + 1] - 1];
+            *note = active ? ((unsigned long long)g.n_sync << 32) | g.row : ~0ull;
+            __syncwarp();
+            const SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk> src{smem_addr(fb), smem_addr(xcol)};
+            sim_rounds_pair<T, S>(m, src, [&](int v, T t) {
+                const unsigned long long nt = *note;
+                if (nt == ~0ull) return;
+                const uint32_t row = (uint32_t)nt + (uint32_t)v;
+                const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], (int)(nt >> 32), sp.bw_sync, sp.intval));
+                if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
+            });
+            const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, *note != ~0ull));
+            if (lane == 0) cells_w[warp] += pair_plans<S>(bks.m) * n_active;
+            __syncwarp();   // the next item overwrites the stage times and cuts
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long c = 0;
+        for (int w = 0; w < kChunk / 32; ++w) c += cells_w[w];
+        add_work(bd.counters, c);
+    }
+}
+
 // Shallow pipelines (<= 16 stages) with fewer micro-batches than warm-up slots (m < S-1): the
 // rounds form of the recurrence, state and stage times in registers, every such depth in one launch.
 template <typename T>
@@ -396,7 +473,26 @@ static cudaError_t launch_wide_one(const Tables &t, const BatchDev &b, const Lau
 }
 
 template <typename T, int S>
+static cudaError_t launch_pair_one(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, true, T>();
+    static std::atomic<uint64_t> configured{0};   // as in launch_wide_one
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 64 || !((configured.load(std::memory_order_acquire) >> dev) & 1ull)) {
+        cudaError_t e = cudaFuncSetAttribute(cm_cost_pair_kernel<T, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
+    }
+    cm_cost_pair_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin, (int)c.uni_items);
+    return cudaGetLastError();
+}
+
+template <typename T, int S>
 static cudaError_t launch_wide(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    if (c.kind == CM_CLASS_WIDE_PAIR) {
+        if constexpr (S >= kPairStagesMin && S <= kPairStagesMax) return launch_pair_one<T, S>(t, b, c, st);
+        else return cudaErrorInvalidValue;
+    }
     if constexpr (S > kWideStagesMax) return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : cudaErrorInvalidValue;
     else return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : launch_wide_one<T, S, false>(t, b, c, st);
 }

@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(128) cm_useg_key_kernel(BatchDev bd, USegDev u
                 if (old == ~0ull || old == tier) { slot = c.tab_first + h; break; }
                 h = (h + 1) & c.tab_mask;
             }
-            if (slot == kNoSegClass) atomicAdd(&ud.count[ud.n_cls], 1u);
+            if (slot == kNoSegClass) atomicAdd(&ud.count[ud.n_cls], 1u);   // (no free slot: cannot happen)
             else atomicMin(&ud.rep[slot], row);
         }
         ud.slot_of[row] = slot;

@@ -218,6 +218,15 @@ template <typename T, int S, typename Src, typename Pend = RegPend<T, S>> struct
         bwd<I>(chain_b);
         if constexpr (I > 0) fwd_if_bwd_down<I - 1>(active, chain_b);
     }
+    // park the state (clocks, and the pending forwards of stages 1 .. S-1) in memory / bring it back
+    template <int I> __device__ __forceinline__ void park(volatile T *mem) const {
+        mem[I] = clock[I];
+        if constexpr (I > 0) { mem[S + I] = pend.template get<I>(); park<I - 1>(mem); }
+    }
+    template <int I> __device__ __forceinline__ void unpark(const volatile T *mem) {
+        clock[I] = mem[I];
+        if constexpr (I > 0) { pend.template set<I>(mem[S + I]); unpark<I - 1>(mem); }
+    }
     // forwards of stages `top`, top-1, .., 0 with top chosen at run time (top <= S-2): a jump
     // into the unrolled sequence, so that a ramp-up round costs its active stages and nothing more
     __device__ __forceinline__ void fwd_down_from(int top) {
@@ -280,6 +289,43 @@ __device__ __forceinline__ T sim_rounds(int m, const Src &src, Pend pend = Pend(
             }
         }
         return r.clock[0];
+    }
+}
+
+// Pipeline times for m AND m+1 micro-batches from one recurrence (1F1B, m >= S-1, S >= 2).
+// Round t runs forward t-i and backward t-S+1: whether a micro-batch m exists shows first in
+// round m, so rounds 0 .. m-1 of the two recurrences are the same operations on the same values
+// and are run once.  The state (2S-1 values) is then parked in local memory, the ramp-down of
+// the m-recurrence runs, the state comes back, and one more steady round plus the ramp-down
+// finish the (m+1)-recurrence.  The two tails share their code (a loop of two trips); each
+// hands its pipeline time to emit(v, t), v = 0 for m and 1 for m+1, so that nothing has to
+// stay in registers across the second tail.
+template <typename T, int S, typename Src, typename Emit>
+__device__ __forceinline__ void sim_rounds_pair(int m, const Src &src, Emit emit) {
+    static_assert(S >= 2, "a one-stage pipeline has no ramp");
+    Rounds<T, S, Src, RegPend<T, S>> r(src);
+    for (int t = 0; t < S - 1; ++t) r.fwd_down_from(t);
+#pragma unroll 4
+    for (int t = S - 1; t < m; ++t) {
+        T chain_b = (T)0;
+        r.template both_down<S - 1>(chain_b);
+    }
+    T parked[2 * S];
+    volatile T *mem = parked;   // volatile: real local-memory stores and loads, not 2S more registers
+    r.template park<S - 1>(mem);
+#pragma unroll 1
+    for (int v = 0; v < 2; ++v) {
+        if (v) {
+            r.template unpark<S - 1>(mem);
+            T chain_b = (T)0;
+            r.template both_down<S - 1>(chain_b);
+        }
+        for (int q = 0; q < S - 1; ++q) {
+            r.template fwd_down_to<S - 1>(q + 1);
+            T chain_b = (T)0;
+            r.template bwd_down<S - 1>(chain_b);
+        }
+        emit(v, r.clock[0]);
     }
 }
 
