@@ -45,7 +45,11 @@ KERNEL_PROFILES = {
                   "profile": "profiles/cm_cost_regs_kernel_int64_paper-scale-512.md"},
     ("wide", 0): {"i_cell": 6.14, "issue_active": 0.574, "fp64_pipe_active": 0.558, "dram_bytes_per_cell": 173056 / 6.199e9,
                   "profile": "profiles/cm_cost_wide_kernel_175b-like-8.md"},
+    # the deep pipelines of a batch with micro-batch pairs on (the default): cm_cost_pair_kernel
+    ("pair", 0): {"i_cell": 6.57, "issue_active": 0.546, "fp64_pipe_active": 0.496, "dram_bytes_per_cell": 6529024 / 3.653e9,
+                  "profile": "profiles/cm_cost_pair_kernel_175b-like-8.md"},
 }
+KERNEL_NAMES = {"regs": "cm_cost_regs_kernel", "wide": "cm_cost_wide_kernel", "pair": "cm_cost_pair_kernel"}
 FP64_INSTR_PER_CELL = 3.0          # 2 DADD + 1 DSETP; an FP64 warp instruction occupies its pipe for 2 cycles
 
 
@@ -519,7 +523,13 @@ def measure_cache(binding, w, mode, local_rank, sizes=(2, 3, 4)):
 def kernel_class(w) -> str:
     """Search-pass kernel that carries a workload: pipelines of the search window deeper than
     16 stages run the deep-pipeline kernel, the others the register-resident one."""
-    return "wide" if w.options.pp_hi > 16 and w.profile.n_pp > 16 else "regs"
+    if not (w.options.pp_hi > 16 and w.profile.n_pp > 16):
+        return "regs"
+    # 1F1B, remainder split of the micro-batches, stage counts of 17-48 with at least as many
+    # micro-batches: the pipelines come as (m, m+1) pairs and the pair kernel carries the batch
+    paired = (getattr(w.options, "schedule", 0) == 0 and w.options.pp_hi <= 48 and
+              w.profile.n_micro * w.profile.n_dp // max(1, w.options.dp_hi) >= w.options.pp_hi)
+    return "pair" if paired else "wide"
 
 
 def roofline_of(stats_sum, dev_seconds, arith, kclass, clocks, sm_max, peak_kind):
@@ -531,7 +541,7 @@ def roofline_of(stats_sum, dev_seconds, arith, kclass, clocks, sm_max, peak_kind
     achieved = stats_sum["cells"] / cost_s if cost_s > 0 else 0.0
     launches = max(1, stats_sum["cost_kernel_launches"])
     return {
-        "bound": "alu", "kernel": {"regs": "cm_cost_regs_kernel", "wide": "cm_cost_wide_kernel"}[kclass] + " (search pass)",
+        "bound": "alu", "kernel": KERNEL_NAMES[kclass] + " (search pass)",
         "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell/s",
         "frac": achieved / peak_cells if peak_cells else None,
         "peak_kind": f"148 SM x 4 schedulers x 32 lanes x {f_mhz:.0f} MHz (median SM clock sampled during the timed region; "

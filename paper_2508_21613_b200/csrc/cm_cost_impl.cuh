@@ -392,11 +392,14 @@ __global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_pair_ke
             *note = active ? ((unsigned long long)g.n_sync << 32) | g.row : ~0ull;
             __syncwarp();
             const SmemStages<T, (int)sizeof(FB<T>), (int)sizeof(T) * kChunk> src{smem_addr(fb), smem_addr(xcol)};
-            sim_rounds_pair<T, S>(m, src, [&](int v, T t) {
-                const unsigned long long nt = *note;
+            // (the commit works from the thread index and shared memory alone: it keeps no register
+            // alive across the recurrence)
+            sim_rounds_pair<T, S>(m, src, [&bd](int v, T t) {
+                const unsigned long long nt =
+                    reinterpret_cast<const unsigned long long *>(dyn + sizeof(FB<T>) * 4 * S + sizeof(T) * (S - 1) * kChunk)[threadIdx.x];
                 if (nt == ~0ull) return;
                 const uint32_t row = (uint32_t)nt + (uint32_t)v;
-                const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[warp], (int)(nt >> 32), sp.bw_sync, sp.intval));
+                const uint64_t bits = Num<T>::bits(t + Num<T>::sync(st_gmax[threadIdx.x >> 5], (int)(nt >> 32), sp.bw_sync, sp.intval));
                 if (bits < bd.seg_best[row]) atomicMin((unsigned long long *)&bd.seg_best[row], (unsigned long long)bits);
             });
             const uint32_t n_active = __popc(__ballot_sync(0xffffffffu, *note != ~0ull));
