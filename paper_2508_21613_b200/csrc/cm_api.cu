@@ -138,6 +138,7 @@ struct Batch {
     // A resident one-scenario batch searched with shared segments keeps its template buckets (the
     // replayed graph uses them) and lays the shared ones out beside them, per search.
     const Bucket *bucket_override = nullptr;
+    uint64_t single_cells = 0;            // recurrence cells of the one scenario's search pass, every segment on its own
     DevBuf<Bucket> d_alt_bucket;
     PinnedVec<unsigned char> alt_stage;   // slot_of | rep | list | buckets, staged for the copies
 };
@@ -1139,7 +1140,16 @@ cm_status run_single_shared(cm_ctx *ctx, Batch &bt, int launches_so_far, bool *d
     const Scen &sc = bt.scen[0];
     const Tmpl &tp = bt.tmpl[sc.tmpl];
     if (tp.n_tseg < 2) return CM_OK;
-    if (bt.tseg_cls.size() != bt.tseg.size()) assign_segment_classes(bt);   // once per resident batch
+    if (bt.tseg_cls.size() != bt.tseg.size()) {   // once per resident batch
+        assign_segment_classes(bt);
+        bt.single_cells = 0;
+        for (uint32_t i = 0; i < tp.n_tseg; ++i) {
+            const TSeg &g = bt.tseg[tp.tseg_first + i];
+            if (bt.tseg_cls[tp.tseg_first + i] == kNoSegClass) continue;
+            bt.single_cells += (g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1)) * 2ull * g.S * g.m;
+        }
+    }
+    if (bt.single_cells < kShareSingleMinCells) return CM_OK;   // not even all of its cells would be worth it
     const size_t n_cls = bt.ucls_info.size();
     struct Key { uint32_t cls; uint64_t tier; uint32_t row; };
     std::vector<Key> keys;

@@ -195,6 +195,29 @@ def test_shared_search_matches_the_stored_oracle_results(gpu, name, mode):
         gpu.cm_destroy(ctx)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_micro_batch_pairs_change_the_work_not_the_result(gpu, mode):
+    """A pipeline's m and m+1 micro-batch variants evaluated in one recurrence (the default) and
+    each on its own: every 175b-like scenario equals the stored oracle result either way, and
+    the paired search runs fewer recurrence cells for the same plans."""
+    w = W.gpt175b_like()
+    want = _stored(w.name, mode)
+    ctx = gpu.cm_create(0)
+    try:
+        gpu.cm_load_profile(ctx, w.profile)
+        cells = {}
+        for pairs in (True, False):
+            gpu.cm_set_micro_batch_pairs(ctx, pairs)
+            best, _, _ = gpu.cm_search_batch(ctx, w.scenarios, w.options.with_cost_mode(mode))
+            st = gpu.cm_last_stats(ctx)
+            cells[pairs] = (st["cells"], st["plans_simulated"])
+            assert [goldens.line_of(p, mode) for p in gpu.plans_from_array(best)] == want
+        assert cells[True][1] == cells[False][1]            # the same plans ...
+        assert cells[True][0] * 3 < cells[False][0] * 2     # ... in under two thirds of the cells
+    finally:
+        gpu.cm_destroy(ctx)
+
+
 @pytest.mark.parametrize("name", ["paper-scale", "175b-like"])
 def test_forced_integer_kernels_match_the_stored_oracle_results(gpu, name):
     """The integer mode normally runs in double arithmetic (exact for these profiles); the
