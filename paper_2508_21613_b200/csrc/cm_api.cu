@@ -325,7 +325,8 @@ void mark_pairs(const cm_ctx *ctx, Batch &bt) {
             const TSeg &a = bt.tseg[t], &b = bt.tseg[t + 1];
             const bool same_pipe = a.S == b.S && a.off == b.off && a.n_sync == b.n_sync && a.K == b.K && b.m == a.m + 1 &&
                                    b.cand_first == a.cand_first + (a.K ? a.K + 1 : 1);
-            if (!same_pipe || a.S < kPairStagesMin || a.S > kPairStagesMax || a.K == 0 || a.m < a.S) continue;
+            if (!same_pipe || a.S > kPairStagesMax || a.m < a.S) continue;
+            if (a.S >= kPairStagesMin && a.K == 0) continue;   // (a deep one-plan segment is walked by a warp)
             if ((a.feas_first == kNoFeasList) != (b.feas_first == kNoFeasList) || a.feas_count != b.feas_count) continue;
             if (a.feas_first != kNoFeasList && a.feas_count == 0) continue;
             bt.role[t] = Batch::kPairHead;
@@ -378,7 +379,10 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 if (role[tp.tseg_first + i] == Batch::kPairHead) {
                     const TSeg &g = bt.tseg[tp.tseg_first + i];
                     const uint64_t n_pairs = (uint64_t)heads[((uint32_t)g.S << 16) | g.m] * tp.n_scen;
-                    if (bucket_kind(by_warp, g.S, g.m, n_pairs, g.K) != CM_CLASS_WIDE_UNI)
+                    const uint64_t count = g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1);
+                    const bool keep = g.S <= kRegStagesMax ? n_pairs * count >= kRegsPairMinPlans
+                                                           : bucket_kind(by_warp, g.S, g.m, n_pairs, g.K) == CM_CLASS_WIDE_UNI;
+                    if (!keep)
                         role[tp.tseg_first + i] = role[tp.tseg_first + i + 1] = Batch::kAlone;
                 }
         }
@@ -413,7 +417,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     if (p1 <= p0) continue;
                     const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
                     Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
-                          count, (uint32_t)ns, pair ? (int)CM_CLASS_WIDE_PAIR : kind_of(g.S, g.m, ns, g.K, count), g.feas_first, pair};
+                          count, (uint32_t)ns,
+                          pair ? (g.S <= kRegStagesMax ? (int)CM_CLASS_REGS_PAIR : (int)CM_CLASS_WIDE_PAIR) : kind_of(g.S, g.m, ns, g.K, count),
+                          g.feas_first, pair};
                     for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
                     pre.push_back(q);
                 }
@@ -427,7 +433,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
 // Buckets and launch classes from the collected (template or shared-list) segment groups.
 cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &pre) {
     using Pre = PreBucket;
-    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WIDE_PAIR; ++kind) {
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_REGS_PAIR; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
         const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO || kind == CM_CLASS_WARP;   // every depth in one class
         LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};

@@ -6,6 +6,7 @@ namespace cm {
 
 template <typename T> cudaError_t launch_shallow_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 template <typename T> cudaError_t launch_shallow_any(const Tables &, const BatchDev &, uint32_t, uint32_t, uint64_t, cudaStream_t);
+template <typename T> cudaError_t launch_shallow_pair_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 template <typename T> cudaError_t launch_short_class(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 template <typename T, int LO, int HI> cudaError_t launch_deep_range(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
 template <typename T, int LO, int HI> cudaError_t launch_tiebreak_range(const Tables &, const BatchDev &, int, cudaStream_t);
@@ -15,6 +16,7 @@ template <typename T> cudaError_t launch_warp_class(const Tables &, const BatchD
 #define CM_EXTERN(T)                                                                                                   \
     extern template cudaError_t launch_shallow_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
     extern template cudaError_t launch_shallow_any<T>(const Tables &, const BatchDev &, uint32_t, uint32_t, uint64_t, cudaStream_t); \
+    extern template cudaError_t launch_shallow_pair_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
     extern template cudaError_t launch_short_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
     extern template cudaError_t launch_solo_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t); \
     extern template cudaError_t launch_warp_class<T>(const Tables &, const BatchDev &, const LaunchClass &, cudaStream_t);
@@ -50,6 +52,7 @@ static cudaError_t launch_tiebreak_deep(const Tables &t, const BatchDev &b, int 
 template <typename T>
 static cudaError_t launch_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
     if (c.kind == CM_CLASS_REGS) return launch_shallow_class<T>(t, b, c, st);
+    if (c.kind == CM_CLASS_REGS_PAIR) return launch_shallow_pair_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_WIDE_UNI || c.kind == CM_CLASS_WIDE_LANE || c.kind == CM_CLASS_WIDE_PAIR) return launch_deep_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_SOLO) return launch_solo_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_WARP) return launch_warp_class<T>(t, b, c, st);

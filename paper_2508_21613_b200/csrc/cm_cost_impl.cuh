@@ -145,6 +145,39 @@ __global__ void __launch_bounds__(kChunk) cm_cost_regs_kernel(Tables tb, BatchDe
     count_cells(&bd.counters[0], my_cells, cells_w);
 }
 
+// The same over micro-batch pairs (Bucket::pair): a thread evaluates its plan for the segment
+// (m micro-batches) and for the next row (the same pipeline with m + 1) in one recurrence.
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk) cm_cost_regs_pair_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1,
+                                                                   uint64_t chunk_offset) {
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, threadIdx.x, seg_local, kappa);
+    if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits0 = inf_bits<T>(), bits1 = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T c0, c1;
+        if (plan_cost_regs_pair<T, S>(sp, tb, bd.layer_mode, g, kappa, c0, c1)) {
+            bits0 = Num<T>::bits(c0);
+            bits1 = Num<T>::bits(c1);
+            my_cells = pair_plans<S>(g.m);
+        }
+    }
+    segmented_min_commit(bd.seg_best, row, bits0, inf_bits<T>());
+    segmented_min_commit(bd.seg_best, row == 0xffffffffu ? row : row + 1, bits1, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
 // Every shallow depth in one launch: for batches so small that a launch per depth would
 // cost more than the work (a single failure scenario of a 32-device job is ~250 CTAs).
 template <typename T>
@@ -510,6 +543,23 @@ template <typename T>
 cudaError_t launch_shallow_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
     switch (c.stages) {
 #define CM_CASE(S) case S: return launch_regs<T, S>(t, b, c, st);
+        CM_CASE(1) CM_CASE(2) CM_CASE(3) CM_CASE(4) CM_CASE(5) CM_CASE(6) CM_CASE(7) CM_CASE(8)
+        CM_CASE(9) CM_CASE(10) CM_CASE(11) CM_CASE(12) CM_CASE(13) CM_CASE(14) CM_CASE(15) CM_CASE(16)
+#undef CM_CASE
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+template <typename T, int S>
+static cudaError_t launch_regs_pair(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    cm_cost_regs_pair_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, 0, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_shallow_pair_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    switch (c.stages) {
+#define CM_CASE(S) case S: return launch_regs_pair<T, S>(t, b, c, st);
         CM_CASE(1) CM_CASE(2) CM_CASE(3) CM_CASE(4) CM_CASE(5) CM_CASE(6) CM_CASE(7) CM_CASE(8)
         CM_CASE(9) CM_CASE(10) CM_CASE(11) CM_CASE(12) CM_CASE(13) CM_CASE(14) CM_CASE(15) CM_CASE(16)
 #undef CM_CASE

@@ -105,14 +105,14 @@ struct Bucket {
     uint32_t feas_first;   // count = length of this list if there is one (kNoFeasList: count = K+1 or 1)
     // 1: every segment of the bucket stands for TWO template segments, itself (m micro-batches) and
     // the next row (the same pipeline with m + 1): their recurrences share all rounds before the
-    // ramp-down, so one thread evaluates both (sim_rounds_pair).  Built only where the two have
+    // ramp-down, so one thread evaluates both (sim_rounds_pair, sim_regs_pair).  Built only where the two have
     // the same feasible compositions: 1F1B with m >= S, where a stage holds min(S - i, m) = S - i
     // micro-batches in flight either way (Section "Estimator", memory estimator), and only for
     // template buckets (with shared segments the distinct ones are searched singly: pairing
     // (m, m+1) and (m+1, m+2) heads would search the middle one twice).
     uint32_t pair, pad;
 };
-constexpr int kPairStagesMin = kRegStagesMax + 1, kPairStagesMax = 48;   // depths whose kernels evaluate pairs
+constexpr int kPairStagesMin = kRegStagesMax + 1, kPairStagesMax = 48;   // depths whose transposed kernel evaluates pairs (shallow ones: all)
 
 // Segments shared between scenarios.  The least cost of a segment over its layer compositions
 // depends on its stages, micro-batches, data-parallel peers and the link tiers of its S-1
@@ -143,8 +143,11 @@ struct USegDev {
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
 enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_SHORT = 3, CM_CLASS_SOLO = 4, CM_CLASS_WARP = 5,
-       CM_CLASS_WIDE_PAIR = 6 };
-// CM_CLASS_WIDE_PAIR: the transposed layout over micro-batch pairs (Bucket::pair), cm_cost_pair_kernel.
+       CM_CLASS_WIDE_PAIR = 6, CM_CLASS_REGS_PAIR = 7 };
+// CM_CLASS_WIDE_PAIR / CM_CLASS_REGS_PAIR: micro-batch pairs (Bucket::pair) in the transposed layout
+// (cm_cost_pair_kernel) and in the register-resident one (cm_cost_regs_pair_kernel).
+constexpr uint64_t kRegsPairMinPlans = 8192;   // shallow pairs are formed where a group has at least this many plans;
+                                               // smaller batches stay with the one launch for every shallow depth
 // CM_CLASS_WARP: the pipelines deeper than kRegStagesMax of a batch that has so few plans there (after the memory
 // screen) that a thread per plan would leave the GPU waiting on a handful of long dependent chains: a warp per plan
 // in lock step, every depth in one launch.

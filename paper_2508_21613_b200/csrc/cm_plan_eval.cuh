@@ -414,6 +414,76 @@ __device__ __forceinline__ T sim_regs(int m, const FB<T> (&st)[S], const T (&xt)
     return clock[0];
 }
 
+// sim_regs for m AND m+1 micro-batches (m >= S-1): warm-up and the m-S+1 steady rounds of the
+// two recurrences coincide (see sim_rounds_pair) and run once; the state is parked in local
+// memory, the cool-down of m runs and hands its time to emit(0, t); the state comes back, one
+// more steady round and the cool-down give emit(1, t) for m+1.  The tails are one loop of two trips.
+template <typename T, int S, typename Emit>
+__device__ __forceinline__ void sim_regs_pair(int m, const FB<T> (&st)[S], const T (&xt)[S], Emit emit) {
+    T clock[S], pend[S];
+#pragma unroll
+    for (int i = 0; i < S; ++i) { clock[i] = (T)0; pend[i] = (T)0; }
+#pragma unroll
+    for (int j = 0; j < S - 1; ++j) {
+        T chain = (T)0;
+#pragma unroll
+        for (int i = 0; i <= S - 2 - j; ++i) {
+            const T start = i > 0 ? tmax(clock[i], chain) : clock[i];
+            const T end = start + st[i].f;
+            clock[i] = end;
+            chain = end + xt[i];
+        }
+        pend[S - 1 - j] = chain;
+    }
+    auto steady = [&]() {
+        T chain_b = (T)0;
+#pragma unroll
+        for (int i = S - 1; i >= 0; --i) {
+            const T fstart = i > 0 ? tmax(clock[i], pend[i]) : clock[i];
+            const T fend = fstart + st[i].f;
+            if (i < S - 1) pend[i + 1] = fend + xt[i];
+            const T dep = i < S - 1 ? chain_b + xt[i] : fend;
+            const T bstart = tmax(fend, dep);
+            const T bend = bstart + st[i].b;
+            clock[i] = bend;
+            chain_b = bend;
+        }
+    };
+#pragma unroll 4
+    for (int k = 0; k <= m - S; ++k) steady();
+    T parked[2 * S];
+    volatile T *mem = parked;   // volatile: real local-memory stores and loads, not 2S more registers
+#pragma unroll
+    for (int i = 0; i < S; ++i) { mem[i] = clock[i]; if (i > 0) mem[S + i] = pend[i]; }
+#pragma unroll 1
+    for (int v = 0; v < 2; ++v) {
+        if (v) {
+#pragma unroll
+            for (int i = 0; i < S; ++i) { clock[i] = mem[i]; if (i > 0) pend[i] = mem[S + i]; }
+            steady();
+        }
+#pragma unroll
+        for (int r = 0; r < S - 1; ++r) {
+            T chain_b = (T)0;
+#pragma unroll
+            for (int i = S - 1; i >= 0; --i) {
+                T c = clock[i];
+                if (i > r) {
+                    const T fstart = i > 0 ? tmax(c, pend[i]) : c;
+                    c = fstart + st[i].f;
+                    if (i < S - 1) pend[i + 1] = c + xt[i];
+                }
+                const T dep = i < S - 1 ? chain_b + xt[i] : c;
+                const T bstart = tmax(c, dep);
+                const T bend = bstart + st[i].b;
+                clock[i] = bend;
+                chain_b = bend;
+            }
+        }
+        emit(v, clock[0]);
+    }
+}
+
 // ----------------------------------------------------------------------------------
 // Cost of pipeline-plan kappa of a segment with S <= kRegStagesMax stages and m >= S-1
 // micro-batches, everything in registers.  Returns false if the plan is infeasible.
@@ -454,6 +524,35 @@ __device__ __forceinline__ bool plan_cost_regs(const SProf<T> &sp, const Tables 
         t = sim_regs<T, S>(m, st, xts);
     }
     cost = t + Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
+    return true;
+}
+
+// The same for a micro-batch pair (Bucket::pair; 1F1B, m >= S): cost of the plan with m
+// micro-batches and with m + 1, one composition, one recurrence.
+template <typename T, int S>
+__device__ __forceinline__ bool plan_cost_regs_pair(const SProf<T> &sp, const Tables &tb, int layer_mode,
+                                                    const SegView &g, uint64_t kappa, T &cost_m, T &cost_m1) {
+    const int m = g.m;
+    CutWalker cw;
+    bool ok = make_walker(cw, tb, layer_mode, sp.L, S, kappa, g.K, tb.mm_slot(S, m));
+    FB<T> st[S];
+    T xts[S];
+    long long g_max = 0;
+    int lo = 0;
+#pragma unroll
+    for (int i = 0; i < S; ++i) {
+        const int hi = ok ? cw.next() : lo + 1;
+        ok = ok && hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
+        st[i].f = sp.PF[hi] - sp.PF[lo];
+        st[i].b = sp.PB[hi] - sp.PB[lo];
+        xts[i] = i < S - 1 ? sp.XT[(g.tier >> i) & 1ull][hi - 1] : (T)0;
+        const long long gb = sp.PP[hi] - sp.PP[lo];
+        g_max = gb > g_max ? gb : g_max;
+        lo = hi;
+    }
+    if (!ok) return false;
+    const T sync = Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
+    sim_regs_pair<T, S>(m, st, xts, [&](int v, T t) { if (v) cost_m1 = t + sync; else cost_m = t + sync; });
     return true;
 }
 
