@@ -45,11 +45,14 @@ KERNEL_PROFILES = {
                   "profile": "profiles/cm_cost_regs_kernel_int64_paper-scale-512.md"},
     ("wide", 0): {"i_cell": 6.14, "issue_active": 0.574, "fp64_pipe_active": 0.558, "dram_bytes_per_cell": 173056 / 6.199e9,
                   "profile": "profiles/cm_cost_wide_kernel_175b-like-8.md"},
+    ("regs_pair", 0): {"i_cell": 5.80, "issue_active": 0.628, "fp64_pipe_active": 0.631, "dram_bytes_per_cell": 957184 / 4.992e9,
+                       "profile": "profiles/cm_cost_regs_pair_kernel_paper-scale-512.md"},
     # the deep pipelines of a batch with micro-batch pairs on (the default): cm_cost_pair_kernel
     ("pair", 0): {"i_cell": 6.57, "issue_active": 0.546, "fp64_pipe_active": 0.496, "dram_bytes_per_cell": 6529024 / 3.653e9,
                   "profile": "profiles/cm_cost_pair_kernel_175b-like-8.md"},
 }
-KERNEL_NAMES = {"regs": "cm_cost_regs_kernel", "wide": "cm_cost_wide_kernel", "pair": "cm_cost_pair_kernel"}
+KERNEL_NAMES = {"regs": "cm_cost_regs_kernel", "regs_pair": "cm_cost_regs_pair_kernel", "wide": "cm_cost_wide_kernel",
+                "pair": "cm_cost_pair_kernel"}
 FP64_INSTR_PER_CELL = 3.0          # 2 DADD + 1 DSETP; an FP64 warp instruction occupies its pipe for 2 cycles
 
 
@@ -524,7 +527,9 @@ def kernel_class(w) -> str:
     """Search-pass kernel that carries a workload: pipelines of the search window deeper than
     16 stages run the deep-pipeline kernel, the others the register-resident one."""
     if not (w.options.pp_hi > 16 and w.profile.n_pp > 16):
-        return "regs"
+        # shallow pipelines pair up under the same conditions once a group of them holds enough plans
+        big = len(w.scenarios) >= 256 and getattr(w.options, "schedule", 0) == 0
+        return "regs_pair" if big and w.profile.n_micro * w.profile.n_dp // max(1, w.options.dp_hi) >= w.options.pp_hi else "regs"
     # 1F1B, remainder split of the micro-batches, stage counts of 17-48 with at least as many
     # micro-batches: the pipelines come as (m, m+1) pairs and the pair kernel carries the batch
     paired = (getattr(w.options, "schedule", 0) == 0 and w.options.pp_hi <= 48 and
