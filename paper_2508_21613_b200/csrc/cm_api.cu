@@ -380,8 +380,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     const TSeg &g = bt.tseg[tp.tseg_first + i];
                     const uint64_t n_pairs = (uint64_t)heads[((uint32_t)g.S << 16) | g.m] * tp.n_scen;
                     const uint64_t count = g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1);
+                    const int kind = bucket_kind(by_warp, g.S, g.m, n_pairs, g.K);
                     const bool keep = g.S <= kRegStagesMax ? n_pairs * count >= kRegsPairMinPlans
-                                                           : bucket_kind(by_warp, g.S, g.m, n_pairs, g.K) == CM_CLASS_WIDE_UNI;
+                                                           : kind == CM_CLASS_WIDE_UNI || kind == CM_CLASS_WIDE_LANE;
                     if (!keep)
                         role[tp.tseg_first + i] = role[tp.tseg_first + i + 1] = Batch::kAlone;
                 }
@@ -408,7 +409,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                 // not.  With one scenario the segments are few: what does not fill most of a
                 // last warp goes to the per-lane kernel, which wastes no lane.
                 size_t cut = j;
-                if (tp.n_scen == 1 && !pair && kind_of(g.S, g.m, n_seg, g.K, count) == CM_CLASS_WIDE_UNI) {
+                if (tp.n_scen == 1 && kind_of(g.S, g.m, n_seg, g.K, count) == CM_CLASS_WIDE_UNI) {
                     const size_t rest = (j - i) % 32;
                     if (rest > 0 && rest < (size_t)kUniMinSegments) cut = j - rest;
                 }
@@ -418,7 +419,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
                     const uint64_t ns = (uint64_t)(p1 - p0) * tp.n_scen;
                     Pre q{(uint32_t)t, (uint32_t)bt.bucket_tseg.size(), (uint32_t)(p1 - p0), g.S, g.m,
                           count, (uint32_t)ns,
-                          pair ? (g.S <= kRegStagesMax ? (int)CM_CLASS_REGS_PAIR : (int)CM_CLASS_WIDE_PAIR) : kind_of(g.S, g.m, ns, g.K, count),
+                          !pair ? kind_of(g.S, g.m, ns, g.K, count)
+                          : g.S <= kRegStagesMax ? (int)CM_CLASS_REGS_PAIR
+                          : kind_of(g.S, g.m, ns, g.K, count) == CM_CLASS_WIDE_UNI ? (int)CM_CLASS_WIDE_PAIR : (int)CM_CLASS_WIDE_LANE_PAIR,
                           g.feas_first, pair};
                     for (size_t k = p0; k < p1; ++k) bt.bucket_tseg.push_back(idx[k]);
                     pre.push_back(q);
@@ -433,7 +436,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
 // Buckets and launch classes from the collected (template or shared-list) segment groups.
 cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &pre) {
     using Pre = PreBucket;
-    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_REGS_PAIR; ++kind) {
+    for (int kind = CM_CLASS_REGS; kind <= CM_CLASS_WIDE_LANE_PAIR; ++kind) {
         uint64_t kind_chunks = 0;   // chunks are numbered through all classes of a kind
         const bool pooled_kind = kind == CM_CLASS_SHORT || kind == CM_CLASS_SOLO || kind == CM_CLASS_WARP;   // every depth in one class
         LaunchClass pooled{kind, 0, 0, (uint32_t)bt.bucket.size(), (uint32_t)bt.bucket.size(), 0, 1, 0};

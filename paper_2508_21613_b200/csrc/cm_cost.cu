@@ -53,7 +53,8 @@ template <typename T>
 static cudaError_t launch_class(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
     if (c.kind == CM_CLASS_REGS) return launch_shallow_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_REGS_PAIR) return launch_shallow_pair_class<T>(t, b, c, st);
-    if (c.kind == CM_CLASS_WIDE_UNI || c.kind == CM_CLASS_WIDE_LANE || c.kind == CM_CLASS_WIDE_PAIR) return launch_deep_class<T>(t, b, c, st);
+    if (c.kind == CM_CLASS_WIDE_UNI || c.kind == CM_CLASS_WIDE_LANE || c.kind == CM_CLASS_WIDE_PAIR ||
+        c.kind == CM_CLASS_WIDE_LANE_PAIR) return launch_deep_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_SOLO) return launch_solo_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_WARP) return launch_warp_class<T>(t, b, c, st);
     if (c.kind == CM_CLASS_SHORT) return launch_short_class<T>(t, b, c, st);

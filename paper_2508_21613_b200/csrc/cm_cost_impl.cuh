@@ -448,6 +448,44 @@ __global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_pair_ke
     }
 }
 
+// Micro-batch pairs in the per-lane layout (buckets with too few pairs for a transposed warp:
+// a failure handled on its own): one plan per lane, evaluated for the segment and for its next
+// row.  Dynamic shared memory as the per-lane cm_cost_wide_kernel.
+template <typename T, int S>
+__global__ void __launch_bounds__(kChunk, wide_ctas_per_sm<S>()) cm_cost_lane_pair_kernel(Tables tb, BatchDev bd, uint32_t b0, uint32_t b1, uint64_t chunk_offset) {
+    static_assert(S >= kPairStagesMin && S <= kPairStagesMax, "pairs exist for the register-resident deep kernels only");
+    __shared__ SProf<T> sp;
+    __shared__ unsigned long long cells_w[kChunk / 32];
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const uint64_t chunk = chunk_offset + (uint64_t)blockIdx.x + (uint64_t)blockIdx.y * gridDim.x;
+    stage_profile(sp, tb);
+    const Bucket bk = bd.bucket[find_bucket(bd.bucket, b0, b1, chunk)];
+    __syncthreads();
+    const uint32_t tid = threadIdx.x;
+    FB<T> *fcol = reinterpret_cast<FB<T> *>(dyn) + tid;                               // [i * kChunk]
+    T *xcol = reinterpret_cast<T *>(dyn + sizeof(FB<T>) * S * kChunk) + tid;           // [i * kChunk]
+    const uint64_t base = (chunk - bk.chunk_first) * kChunk;
+    uint64_t seg_local, kappa;
+    plan_of_thread(base, bk.count, tid, seg_local, kappa);
+    if (seg_local < bk.n_seg) kappa = walk_kappa(bd.feas, bk.feas_first, kappa);
+    uint32_t row = 0xffffffffu;
+    uint64_t bits0 = inf_bits<T>(), bits1 = inf_bits<T>();
+    unsigned long long my_cells = 0;
+    if (seg_local < bk.n_seg) {
+        const SegView g = bucket_segment(bd, bk, (uint32_t)seg_local);
+        row = g.row;
+        T c0, c1;
+        if (plan_cost_wide_lane_pair<T, S>(sp, tb, bd.layer_mode, g, kappa, fcol, xcol, c0, c1)) {
+            bits0 = Num<T>::bits(c0);
+            bits1 = Num<T>::bits(c1);
+            my_cells = pair_plans<S>(bk.m);
+        }
+    }
+    segmented_min_commit(bd.seg_best, row, bits0, inf_bits<T>());
+    segmented_min_commit(bd.seg_best, row == 0xffffffffu ? row : row + 1, bits1, inf_bits<T>());
+    count_cells(&bd.counters[0], my_cells, cells_w);
+}
+
 // Shallow pipelines (<= 16 stages) with fewer micro-batches than warm-up slots (m < S-1): the
 // rounds form of the recurrence, state and stage times in registers, every such depth in one launch.
 template <typename T>
@@ -524,9 +562,25 @@ static cudaError_t launch_pair_one(const Tables &t, const BatchDev &b, const Lau
 }
 
 template <typename T, int S>
+static cudaError_t launch_lane_pair_one(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
+    constexpr size_t smem = wide_smem_bytes<S, false, T>();
+    static std::atomic<uint64_t> configured{0};   // as in launch_wide_one
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 64 || !((configured.load(std::memory_order_acquire) >> dev) & 1ull)) {
+        cudaError_t e = cudaFuncSetAttribute(cm_cost_lane_pair_kernel<T, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
+    }
+    cm_cost_lane_pair_kernel<T, S><<<chunk_grid(c.n_chunks), kChunk, smem, st>>>(t, b, c.bucket_begin, c.bucket_end, c.chunk_begin);
+    return cudaGetLastError();
+}
+
+template <typename T, int S>
 static cudaError_t launch_wide(const Tables &t, const BatchDev &b, const LaunchClass &c, cudaStream_t st) {
-    if (c.kind == CM_CLASS_WIDE_PAIR) {
-        if constexpr (S >= kPairStagesMin && S <= kPairStagesMax) return launch_pair_one<T, S>(t, b, c, st);
+    if (c.kind == CM_CLASS_WIDE_PAIR || c.kind == CM_CLASS_WIDE_LANE_PAIR) {
+        if constexpr (S >= kPairStagesMin && S <= kPairStagesMax)
+            return c.kind == CM_CLASS_WIDE_PAIR ? launch_pair_one<T, S>(t, b, c, st) : launch_lane_pair_one<T, S>(t, b, c, st);
         else return cudaErrorInvalidValue;
     }
     if constexpr (S > kWideStagesMax) return c.kind == CM_CLASS_WIDE_UNI ? launch_wide_one<T, S, true>(t, b, c, st) : cudaErrorInvalidValue;

@@ -143,9 +143,10 @@ struct USegDev {
 // flattened plans (segment-in-bucket * count + kappa) into chunks of kChunk; the
 // transposed class cuts its (kappa, group of 32 segments) warp items into chunks of 4.
 enum { CM_CLASS_REGS = 0, CM_CLASS_WIDE_UNI = 1, CM_CLASS_WIDE_LANE = 2, CM_CLASS_SHORT = 3, CM_CLASS_SOLO = 4, CM_CLASS_WARP = 5,
-       CM_CLASS_WIDE_PAIR = 6, CM_CLASS_REGS_PAIR = 7 };
-// CM_CLASS_WIDE_PAIR / CM_CLASS_REGS_PAIR: micro-batch pairs (Bucket::pair) in the transposed layout
-// (cm_cost_pair_kernel) and in the register-resident one (cm_cost_regs_pair_kernel).
+       CM_CLASS_WIDE_PAIR = 6, CM_CLASS_REGS_PAIR = 7, CM_CLASS_WIDE_LANE_PAIR = 8 };
+// CM_CLASS_WIDE_PAIR / CM_CLASS_WIDE_LANE_PAIR / CM_CLASS_REGS_PAIR: micro-batch pairs (Bucket::pair) in the
+// transposed layout (cm_cost_pair_kernel), the per-lane layout (cm_cost_lane_pair_kernel) and the
+// register-resident one (cm_cost_regs_pair_kernel).
 constexpr uint64_t kRegsPairMinPlans = 8192;   // shallow pairs are formed where a group has at least this many plans;
                                                // smaller batches stay with the one launch for every shallow depth
 // CM_CLASS_WARP: the pipelines deeper than kRegStagesMax of a batch that has so few plans there (after the memory

@@ -589,6 +589,35 @@ __device__ __forceinline__ bool plan_cost_wide_lane(const SProf<T> &sp, const Ta
     return true;
 }
 
+// The same for a micro-batch pair (Bucket::pair; 1F1B, m >= S): the plan with m micro-batches
+// and with m + 1, one composition, one recurrence.
+template <typename T, int S>
+__device__ __forceinline__ bool plan_cost_wide_lane_pair(const SProf<T> &sp, const Tables &tb, int layer_mode, const SegView &g,
+                                                         uint64_t kappa, FB<T> *fcol, T *xcol, T &cost_m, T &cost_m1) {
+    const int m = g.m;
+    CutWalker cw;
+    bool ok = make_walker(cw, tb, layer_mode, sp.L, S, kappa, g.K, tb.mm_slot(S, m));
+    long long g_max = 0;
+    int lo = 0;
+    for (int i = 0; i < S && ok; ++i) {
+        const int hi = cw.next();
+        ok = hi > lo && stage_fits(sp.PS[hi] - sp.PS[lo], sp.PA[hi] - sp.PA[lo], i, S, m, sp.cap, sp.sched);
+        FB<T> d;
+        d.f = sp.PF[hi] - sp.PF[lo];
+        d.b = sp.PB[hi] - sp.PB[lo];
+        fcol[i * kChunk] = d;
+        xcol[i * kChunk] = i < S - 1 ? sp.XT[(g.tier >> i) & 1ull][hi - 1] : (T)0;
+        const long long gb = sp.PP[hi] - sp.PP[lo];
+        g_max = gb > g_max ? gb : g_max;
+        lo = hi;
+    }
+    if (!ok) return false;
+    const SmemStages<T, (int)sizeof(FB<T>) * kChunk, (int)sizeof(T) * kChunk> src{smem_addr(fcol), smem_addr(xcol)};
+    const T sync = Num<T>::sync(g_max, g.n_sync, sp.bw_sync, sp.intval);
+    sim_rounds_pair<T, S>(m, src, [&](int v, T t) { if (v) cost_m1 = t + sync; else cost_m = t + sync; });
+    return true;
+}
+
 // The same with S chosen at run time (one kernel for every shallow depth; used where the
 // work is too small to be worth one launch per depth).  Caller guarantees 1 <= S <= 16, and
 // m >= S-1 unless ANY_M.
