@@ -511,6 +511,36 @@ def test_pipelines_of_62_to_64_stages(gpu, oracle_factory, sched):
                 s.close()
 
 
+@pytest.mark.parametrize("layer_mode,batch_mode", [(W.LAYERS_FULL, W.BATCH_FULL), (W.LAYERS_FULL, W.BATCH_REMAINDER)])
+def test_micro_batch_pairs_on_shallow_pipelines_against_the_oracle(gpu, oracle_factory, layer_mode, batch_mode):
+    """Pairs of consecutive micro-batch counts in the register-resident kernels, under the full
+    enumeration of splits (every count from 1 up: pairs (m, m+1), (m+2, m+3), .. wherever
+    m >= stages) and under the remainder rule: a batch large enough for the shallow pair
+    kernel (every failure set of one or two of the twelve devices, a third of the triples), non-uniform stage
+    times, tight and loose memory; every scenario against the oracle, pairs on and off."""
+    import itertools
+    for tight in (False, True):
+        w = W.random_small(11 + tight, L=13, n_dp=3, n_pp=4, n_micro=7, tight_memory=tight)
+        scen = [list(c) for k in (1, 2) for c in itertools.combinations(range(12), k)]
+        scen += [list(c) for c in itertools.combinations(range(12), 3)][::3]
+        for mode in (0, 1):
+            opts = W.SearchOptions(1, 3, 2, 6, layer_mode, batch_mode, 1 << 62, mode)
+            o = oracle_factory(w.profile, opts)
+            want = [o.search(f)[0] for f in scen]
+            cells = {}
+            s = Session(gpu, w.profile)
+            try:
+                for pairs in (True, False):
+                    gpu.cm_set_micro_batch_pairs(s.ctx, pairs)
+                    best, _, _ = gpu.cm_search_batch(s.ctx, scen, opts)
+                    cells[pairs] = gpu.cm_last_stats(s.ctx)["cells"]
+                    for b, failed in enumerate(scen):
+                        assert_same_plan(gpu.plans_from_array(best)[b], want[b], mode, f"{failed} pairs={pairs} tight={tight}")
+            finally:
+                s.close()
+            assert cells[True] < cells[False]   # some groups were large enough to be paired
+
+
 def test_handworked_readings_rerouting_redundant_memory_minmax_ties(gpu, oracle_factory):
     """The hand-worked cases that fix the readings taken where the paper prints no formula
     (``tests/golden/*_handworked.txt``): the library must give the fixtures' own numbers, not
