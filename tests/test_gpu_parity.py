@@ -541,6 +541,36 @@ def test_micro_batch_pairs_on_shallow_pipelines_against_the_oracle(gpu, oracle_f
             assert cells[True] < cells[False]   # some groups were large enough to be paired
 
 
+def test_micro_batch_pairs_on_deep_pipelines_against_the_oracle(gpu, oracle_factory):
+    """The transposed pair kernel on strongly non-uniform stages: every single failure of the
+    deep, narrow job in one batch (80 scenarios of one survivor count, so groups of pair heads
+    fill transposed warps), pipelines of 18-61 stages, each scenario against the oracle with
+    pairs on and off; then three of them one at a time (the per-lane pair kernel)."""
+    w = W.deep_pipeline(3)
+    scen = [[d] for d in range(80)]
+    for mode in (0, 1):
+        opts = W.SearchOptions(1, 3, 18, 64, W.LAYERS_REMAINDER, W.BATCH_REMAINDER, 600, mode)
+        o = oracle_factory(w.profile, opts)
+        want = [o.search(f) for f in scen]
+        cells = {}
+        s = Session(gpu, w.profile)
+        try:
+            for pairs in (True, False):
+                gpu.cm_set_micro_batch_pairs(s.ctx, pairs)
+                best, per, _ = gpu.cm_search_batch(s.ctx, scen, opts, per_policy=True)
+                cells[pairs] = gpu.cm_last_stats(s.ctx)["cells"]
+                for b, failed in enumerate(scen):
+                    assert_same_plan(gpu.plans_from_array(best)[b], want[b][0], mode, f"{failed} pairs={pairs}")
+                    assert_same_plan(gpu.plans_from_array(per)[3 * b + 2], want[b][1][2], mode, f"{failed} dynpar pairs={pairs}")
+                for _ in range(2):
+                    best, _, _ = gpu.cm_search_batch(s.ctx, scen[:3], opts, latency=True)
+                    for b in range(3):
+                        assert_same_plan(gpu.plans_from_array(best)[b], want[b][0], mode, f"{scen[b]} alone pairs={pairs}")
+        finally:
+            s.close()
+        assert cells[True] * 10 < cells[False] * 9   # (many of these pipelines have fewer micro-batches than stages)
+
+
 def test_handworked_readings_rerouting_redundant_memory_minmax_ties(gpu, oracle_factory):
     """The hand-worked cases that fix the readings taken where the paper prints no formula
     (``tests/golden/*_handworked.txt``): the library must give the fixtures' own numbers, not
