@@ -366,8 +366,9 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     for (size_t t = 0; t < bt.tmpl.size(); ++t) {
         const Tmpl &tp = bt.tmpl[t];
         if (tp.n_scen == 0 || tp.n_tseg == 0) continue;
-        // micro-batch pairs go to the transposed kernel; a group of pair heads too small for it is
-        // evaluated as single segments instead
+        // which micro-batch pairs this layout keeps: deep ones where the group of pair heads goes to
+        // the transposed or the per-lane kernel (not where the batch's few deep plans go a warp per
+        // plan), shallow ones where the group holds enough plans to be worth a launch of its own
         {
             std::map<uint32_t, uint32_t> heads;   // (S << 16 | m) -> pair heads of the template
             for (uint32_t i = 0; i < tp.n_tseg; ++i)
