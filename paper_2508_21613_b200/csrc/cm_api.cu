@@ -121,15 +121,16 @@ struct Batch {
     // segment; the buckets are laid out in upload_batch, once the device has counted the distinct
     // segments of every class.
     bool useg = false;
-    struct USegInfo { uint16_t S, m, n_sync; uint64_t K; uint32_t feas_first, feas_count; uint64_t rows; };
+    struct USegInfo { uint16_t S, m, n_sync, pair; uint64_t K; uint32_t feas_first, feas_count; uint64_t rows; };
     // Role of every template segment in the search pass: on its own, head of a micro-batch pair
     // (evaluated together with the next row), or that next row.
     enum : uint8_t { kAlone = 0, kPairHead = 1, kPairPartner = 2 };
     std::vector<uint8_t> role;
     std::vector<USegInfo> ucls_info;
     std::vector<USegClass> ucls;
-    std::vector<uint32_t> tseg_cls;
-    size_t off_ucls = 0, off_tseg_cls = 0;
+    std::vector<uint32_t> tseg_cls, look_head, look_part;
+    uint32_t n_pair_cls = 0;
+    size_t off_ucls = 0, off_tseg_cls = 0, off_look_head = 0, off_look_part = 0;
     uint64_t utab_slots = 0, ulist_len = 0;
     DevBuf<unsigned long long> d_utab;
     DevBuf<uint32_t> d_urep, d_slot_of, d_ucount;
@@ -496,24 +497,64 @@ cm_status layout_buckets(cm_ctx *ctx, Batch &bt, const std::vector<PreBucket> &p
 // its real content follows once the device has counted the distinct segments.
 constexpr size_t kSharedBucketsPerClass = 2;   // transposed part and per-lane remainder
 void assign_segment_classes(Batch &bt) {
-    std::map<uint64_t, uint32_t> ids;
     bt.tseg_cls.assign(bt.tseg.size(), kNoSegClass);
+    bt.look_head.assign(bt.tseg.size(), kNoSegClass);
+    bt.look_part.assign(bt.tseg.size(), kNoSegClass);
     bt.ucls_info.clear();
     bt.ucls.clear();
+    auto searched = [](const TSeg &g) { return g.m >= 1 && !(g.feas_first != kNoFeasList && g.feas_count == 0); };
+    auto key_of = [](const TSeg &g, uint16_t m) { return ((uint64_t)g.S << 32) | ((uint64_t)m << 16) | g.n_sync; };
+    // pair classes first: the micro-batch counts at which pair heads occur, per (stages, peers),
+    // taken greedily from the lowest so that no two pair classes overlap
+    std::map<uint64_t, uint32_t> pair_ids, single_ids;
+    {
+        std::map<std::pair<uint32_t, uint16_t>, const TSeg *> by_group;   // ((S << 16 | peers), m)
+        for (const Tmpl &tp : bt.tmpl) {
+            if (tp.n_scen == 0) continue;
+            for (uint32_t i = 0; i < tp.n_tseg; ++i) {
+                const TSeg &g = bt.tseg[tp.tseg_first + i];
+                if (bt.role[tp.tseg_first + i] == Batch::kPairHead && searched(g))
+                    by_group.emplace(std::make_pair(((uint32_t)g.S << 16) | g.n_sync, g.m), &g);
+            }
+        }
+        uint32_t group = 0xffffffffu;
+        int last_start = -2;
+        for (const auto &e : by_group) {
+            if (e.first.first != group) { group = e.first.first; last_start = -2; }
+            const int m = e.first.second;
+            if (m == last_start + 1) continue;   // covered as the second count of the pair class before
+            last_start = m;
+            const TSeg &g = *e.second;
+            pair_ids.emplace(key_of(g, g.m), (uint32_t)bt.ucls_info.size());
+            bt.ucls_info.push_back(Batch::USegInfo{g.S, g.m, g.n_sync, 1, g.K, g.feas_first, g.feas_count, 0});
+        }
+    }
+    bt.n_pair_cls = (uint32_t)bt.ucls_info.size();
     for (const Tmpl &tp : bt.tmpl) {
         if (tp.n_scen == 0) continue;
         for (uint32_t i = 0; i < tp.n_tseg; ++i) {
-            const TSeg &g = bt.tseg[tp.tseg_first + i];
-            if (g.m < 1) continue;                                                 // no work is scheduled: stays infeasible
-            if (g.feas_first != kNoFeasList && g.feas_count == 0) continue;       // nothing fits in memory
-            const uint64_t key = ((uint64_t)g.S << 32) | ((uint64_t)g.m << 16) | g.n_sync;
-            auto it = ids.find(key);
-            if (it == ids.end()) {
-                it = ids.emplace(key, (uint32_t)bt.ucls_info.size()).first;
-                bt.ucls_info.push_back(Batch::USegInfo{g.S, g.m, g.n_sync, g.K, g.feas_first, g.feas_count, 0});
+            const uint32_t t = tp.tseg_first + i;
+            const TSeg &g = bt.tseg[t];
+            if (!searched(g) || bt.tseg_cls[t] == kPartnerSeg) continue;
+            auto own = pair_ids.find(key_of(g, g.m));
+            if (bt.role[t] == Batch::kPairHead && own != pair_ids.end()) {
+                bt.tseg_cls[t] = own->second;        // keyed as a pair head; the next row rides with it
+                bt.tseg_cls[t + 1] = kPartnerSeg;
+                bt.ucls_info[own->second].rows += tp.n_scen;
+                continue;
+            }
+            if (own != pair_ids.end()) bt.look_head[t] = own->second;
+            if (g.m >= 1) {
+                auto before = pair_ids.find(key_of(g, (uint16_t)(g.m - 1)));
+                if (before != pair_ids.end()) bt.look_part[t] = before->second;
+            }
+            auto it = single_ids.find(key_of(g, g.m));
+            if (it == single_ids.end()) {
+                it = single_ids.emplace(key_of(g, g.m), (uint32_t)bt.ucls_info.size()).first;
+                bt.ucls_info.push_back(Batch::USegInfo{g.S, g.m, g.n_sync, 0, g.K, g.feas_first, g.feas_count, 0});
             }
             bt.ucls_info[it->second].rows += tp.n_scen;
-            bt.tseg_cls[tp.tseg_first + i] = it->second;
+            bt.tseg_cls[t] = it->second;
         }
     }
 }
@@ -550,7 +591,7 @@ cm_status build_shared_buckets(cm_ctx *ctx, Batch &bt, const uint32_t *n_distinc
     uint64_t deep_plans = 0;
     for (size_t c = 0; c < bt.ucls_info.size(); ++c) {
         const Batch::USegInfo &u = bt.ucls_info[c];
-        if (u.S > kRegStagesMax && u.K > 0) deep_plans += count_of(u) * n_distinct[c];
+        if (u.S > kRegStagesMax && u.K > 0) deep_plans += count_of(u) * n_distinct[c] * (u.pair ? 2 : 1);
     }
     const bool by_warp = deep_plans <= kWarpPlansMax;
     for (size_t c = 0; c < bt.ucls_info.size(); ++c) {
@@ -566,8 +607,20 @@ cm_status build_shared_buckets(cm_ctx *ctx, Batch &bt, const uint32_t *n_distinc
         for (int part = 0; part < 2; ++part) {
             const uint32_t p0 = part ? cut : 0, p1 = part ? n : cut;
             if (p1 <= p0) continue;
-            pre.push_back(PreBucket{kSharedBucket, bt.ucls[c].list_first + p0, 0, u.S, u.m, count_of(u), p1 - p0,
-                                    bucket_kind(by_warp, u.S, u.m, p1 - p0, u.K), u.feas_first, 0});
+            const int kind = bucket_kind(by_warp, u.S, u.m, p1 - p0, u.K);
+            const uint32_t first = bt.ucls[c].list_first + p0;
+            if (!u.pair) {
+                pre.push_back(PreBucket{kSharedBucket, first, 0, u.S, u.m, count_of(u), p1 - p0, kind, u.feas_first, 0});
+            } else if (kind == CM_CLASS_REGS || kind == CM_CLASS_WIDE_UNI || kind == CM_CLASS_WIDE_LANE) {
+                const int pk = kind == CM_CLASS_REGS ? CM_CLASS_REGS_PAIR : kind == CM_CLASS_WIDE_UNI ? CM_CLASS_WIDE_PAIR : CM_CLASS_WIDE_LANE_PAIR;
+                pre.push_back(PreBucket{kSharedBucket, first, 0, u.S, u.m, count_of(u), p1 - p0, pk, u.feas_first, 1});
+            } else {
+                // a kernel without a pair form (the batch's few deep plans go a warp per plan): the
+                // heads as they are, and their next rows (m + 1, the same compositions) through the same list
+                pre.push_back(PreBucket{kSharedBucket, first, 0, u.S, u.m, count_of(u), p1 - p0, kind, u.feas_first, 0});
+                pre.push_back(PreBucket{kSharedBucket, first, 0, u.S, (uint16_t)(u.m + 1), count_of(u), p1 - p0,
+                                        bucket_kind(by_warp, u.S, u.m + 1, p1 - p0, u.K), u.feas_first, 2});
+            }
         }
     }
     cm_status s = layout_buckets(ctx, bt, pre);
@@ -883,6 +936,8 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     if (bt.useg) return build_segment_classes(ctx, bt);
     bt.ucls.clear();
     bt.tseg_cls.clear();
+    bt.look_head.clear();
+    bt.look_part.clear();
     return build_buckets(ctx, bt);
 }
 
@@ -925,6 +980,9 @@ USegDev useg_view(const Batch &bt) {
     USegDev u{};
     u.cls = (const USegClass *)(bt.d_arena.p + bt.off_ucls);
     u.tseg_cls = (const uint32_t *)(bt.d_arena.p + bt.off_tseg_cls);
+    u.look_head = (const uint32_t *)(bt.d_arena.p + bt.off_look_head);
+    u.look_part = (const uint32_t *)(bt.d_arena.p + bt.off_look_part);
+    u.n_pair_cls = bt.n_pair_cls;
     u.tab = bt.d_utab.p; u.rep = bt.d_urep.p; u.slot_of = bt.d_slot_of.p; u.count = bt.d_ucount.p; u.list = bt.d_useg.p;
     u.n_cls = (uint32_t)bt.ucls.size();
     u.n_rep_scen = 0;
@@ -964,6 +1022,8 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     bt.off_cross = arena_put(bt.arena, bt.cross, ok);
     bt.off_ucls = arena_put(bt.arena, bt.ucls, ok);
     bt.off_tseg_cls = arena_put(bt.arena, bt.tseg_cls, ok);
+    bt.off_look_head = arena_put(bt.arena, bt.look_head, ok);
+    bt.off_look_part = arena_put(bt.arena, bt.look_part, ok);
     bt.off_bucket = arena_put(bt.arena, bt.bucket, ok);
     if (!ok) return fail(ctx, CM_ENOMEM, "host memory");
     if (!bt.d_arena.reserve(bt.arena.size())) return fail(ctx, CM_ENOMEM, "device memory");
@@ -993,7 +1053,7 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
         CM_CUDA(ctx, cudaMemsetAsync(bt.d_urep.p, 0xFF, bt.utab_slots * sizeof(uint32_t), ctx->stream));
         CM_CUDA(ctx, cudaMemsetAsync(bt.d_ucount.p, 0, (n_cls + 1) * sizeof(uint32_t), ctx->stream));
         CM_CUDA(ctx, launch_useg_keys(dev_view(ctx, bt), useg_view(bt), ctx->stream));
-        if (launches) *launches += 2;
+        if (launches) *launches += 3;
         CM_CUDA(ctx, cudaMemcpyAsync(bt.ucount_host.p, bt.d_ucount.p, (n_cls + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream));
         CM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
         ctx->stats[10] += (n_cls + 1) * sizeof(uint32_t);
@@ -1161,36 +1221,69 @@ cm_status run_single_shared(cm_ctx *ctx, Batch &bt, int launches_so_far, bool *d
     }
     if (bt.single_cells < kShareSingleMinCells) return CM_OK;   // not even all of its cells would be worth it
     const size_t n_cls = bt.ucls_info.size();
-    struct Key { uint32_t cls; uint64_t tier; uint32_t row; };
-    std::vector<Key> keys;
-    keys.reserve(tp.n_tseg);
+    // The same keying as cm_useg_key_kernel, on the host: the heads of the pair classes first, then
+    // every other row, which joins a pair that holds its tier (as head: its own m; as second row:
+    // m - 1) before it is keyed among the single segments.  `joined`: slot_of value of such a row.
+    struct Key { uint32_t cls; uint64_t tier; uint32_t row; uint32_t joined; };
+    std::vector<Key> heads, others;
+    heads.reserve(tp.n_tseg);
+    others.reserve(tp.n_tseg);
     const uint64_t *words = bt.cross.data() + sc.cross_first;
+    auto single_cells_of = [&](const TSeg &g) {
+        return (g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : (g.K ? g.K + 1 : 1)) * 2ull * g.S * g.m;
+    };
+    uint64_t all_cells = 0, distinct_cells = 0;
     for (uint32_t i = 0; i < tp.n_tseg; ++i) {
         const uint32_t c = bt.tseg_cls[tp.tseg_first + i];
         if (c == kNoSegClass) continue;
         const TSeg &g = bt.tseg[tp.tseg_first + i];
+        all_cells += single_cells_of(g);
+        if (c == kPartnerSeg) continue;
         const int w = g.off >> 6, sh = g.off & 63, n = g.S - 1;
         uint64_t v = words[w] >> sh;
         if (sh) v |= words[w + 1] << (64 - sh);
-        keys.push_back(Key{c, v & ((1ull << n) - 1ull), i});
+        (c < bt.n_pair_cls ? heads : others).push_back(Key{c, v & ((1ull << n) - 1ull), i, kNoSegClass});
     }
-    std::sort(keys.begin(), keys.end(), [](const Key &a, const Key &b) {
+    auto by_key = [](const Key &a, const Key &b) {
         return a.cls != b.cls ? a.cls < b.cls : a.tier != b.tier ? a.tier < b.tier : a.row < b.row;
-    });
+    };
+    auto same_key = [](const Key &a, const Key &b) { return a.cls == b.cls && a.tier == b.tier; };
+    std::sort(heads.begin(), heads.end(), by_key);
+    std::vector<Key> pair_reps;   // distinct pair heads, sorted by (class, tier); index = their slot
+    for (size_t i = 0; i < heads.size(); ++i)
+        if (i == 0 || !same_key(heads[i], heads[i - 1])) pair_reps.push_back(heads[i]);
+    auto find_pair = [&](uint32_t cls, uint64_t tier) -> uint32_t {
+        if (cls == kNoSegClass) return kNoSegClass;
+        const Key probe{cls, tier, 0, 0};
+        auto it = std::lower_bound(pair_reps.begin(), pair_reps.end(), probe, [](const Key &a, const Key &b) {
+            return a.cls != b.cls ? a.cls < b.cls : a.tier < b.tier;
+        });
+        return it != pair_reps.end() && same_key(*it, probe) ? (uint32_t)(it - pair_reps.begin()) : kNoSegClass;
+    };
+    std::vector<Key> singles;
+    singles.reserve(others.size());
+    for (Key &k : others) {
+        const uint32_t t = tp.tseg_first + k.row;
+        uint32_t at = find_pair(bt.look_head[t], k.tier);
+        if (at == kNoSegClass) {
+            at = find_pair(bt.look_part[t], k.tier);
+            if (at != kNoSegClass) at |= kSecondRowFlag;
+        }
+        k.joined = at;
+        if (at == kNoSegClass) singles.push_back(k);
+    }
+    std::sort(singles.begin(), singles.end(), by_key);
     auto cells_of = [&](uint32_t c) {
         const Batch::USegInfo &u = bt.ucls_info[c];
         const uint64_t count = u.feas_first != kNoFeasList ? (uint64_t)u.feas_count : (u.K ? u.K + 1 : 1);
-        return count * 2ull * u.S * u.m;
+        return count * (u.pair ? 2ull * u.S * (u.m + 1) + 3ull * u.S * (u.S - 1) / 2 : 2ull * u.S * u.m);
     };
     std::vector<uint32_t> counts(n_cls + 1, 0);
-    uint64_t all_cells = 0, distinct_cells = 0;
-    size_t n_distinct = 0;
-    for (size_t i = 0; i < keys.size(); ++i) {
-        const bool first = i == 0 || keys[i].cls != keys[i - 1].cls || keys[i].tier != keys[i - 1].tier;
-        all_cells += cells_of(keys[i].cls);
-        if (first) { distinct_cells += cells_of(keys[i].cls); ++counts[keys[i].cls]; ++n_distinct; }
-    }
-    if (all_cells - distinct_cells < kShareSingleMinCells) return CM_OK;
+    size_t n_distinct = pair_reps.size();
+    for (const Key &k : pair_reps) { distinct_cells += cells_of(k.cls); ++counts[k.cls]; }
+    for (size_t i = 0; i < singles.size(); ++i)
+        if (i == 0 || !same_key(singles[i], singles[i - 1])) { distinct_cells += cells_of(singles[i].cls); ++counts[singles[i].cls]; ++n_distinct; }
+    if (all_cells < distinct_cells + kShareSingleMinCells) return CM_OK;
 
     // staging: slot_of [rows] | rep [distinct] | list [distinct] | buckets [2 per class]
     const size_t rows = bt.n_rows, max_buckets = std::max<size_t>(kSharedBucketsPerClass * n_cls, 1);
@@ -1205,15 +1298,27 @@ cm_status run_single_shared(cm_ctx *ctx, Batch &bt, int launches_so_far, bool *d
     bt.ucls.assign(n_cls, USegClass{0, 0, 0, 0});
     uint32_t first_of = 0;
     for (size_t c = 0; c < n_cls; ++c) { bt.ucls[c].list_first = first_of; first_of += counts[c]; }
+    // slots (= list positions): the distinct pair heads, then the distinct single segments; pair
+    // classes have the lower class numbers, so the positions follow the class regions
     uint32_t u = 0;
-    for (size_t i = 0; i < keys.size(); ++i) {
-        const bool first = i == 0 || keys[i].cls != keys[i - 1].cls || keys[i].tier != keys[i - 1].tier;
-        if (first) {   // keys are sorted by class, so list positions follow the class regions
-            rep[u] = sc.seg_base + keys[i].row;
-            list[u] = make_uint2(0u, tp.tseg_first + keys[i].row);
+    for (size_t i = 0; i < heads.size(); ++i) {
+        if (i == 0 || !same_key(heads[i], heads[i - 1])) {
+            rep[u] = sc.seg_base + heads[i].row;
+            list[u] = make_uint2(0u, tp.tseg_first + heads[i].row);
             ++u;
         }
-        slot_of[sc.seg_base + keys[i].row] = u - 1;
+        slot_of[sc.seg_base + heads[i].row] = u - 1;
+        slot_of[sc.seg_base + heads[i].row + 1] = kPartnerSeg;
+    }
+    for (const Key &k : others)
+        if (k.joined != kNoSegClass) slot_of[sc.seg_base + k.row] = k.joined;
+    for (size_t i = 0; i < singles.size(); ++i) {
+        if (i == 0 || !same_key(singles[i], singles[i - 1])) {
+            rep[u] = sc.seg_base + singles[i].row;
+            list[u] = make_uint2(0u, tp.tseg_first + singles[i].row);
+            ++u;
+        }
+        slot_of[sc.seg_base + singles[i].row] = u - 1;
     }
     std::vector<Bucket> keep_buckets;
     std::vector<LaunchClass> keep_classes;

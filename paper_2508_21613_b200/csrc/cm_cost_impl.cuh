@@ -63,7 +63,7 @@ __device__ __forceinline__ void plan_of_thread(uint64_t base, uint64_t count, ui
 __device__ __forceinline__ SegView bucket_segment(const BatchDev &bd, const Bucket &bk, uint32_t seg_local) {
     if (bk.tmpl == kSharedBucket) {   // a range of the list of distinct segments
         const uint2 p = bd.useg[bk.list_first + seg_local];
-        return seg_view(bd, p.x, p.y);
+        return seg_view(bd, p.x, p.y + (bk.pair == 2 ? 1u : 0u));   // pair == 2: the second rows of a list of pair heads
     }
     const Tmpl &tp = bd.tmpl[bk.tmpl];
     const uint32_t ti = seg_local / tp.n_scen, si = seg_local - ti * tp.n_scen;

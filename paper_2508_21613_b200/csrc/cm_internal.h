@@ -124,19 +124,30 @@ constexpr int kPairStagesMin = kRegStagesMax + 1, kPairStagesMax = 48;   // dept
 // (scenario, template segment) list of the distinct segments of one class.
 constexpr uint32_t kSharedBucket = 0xffffffffu;
 constexpr uint32_t kNoSegClass = 0xffffffffu;   // template segment that is not searched (no micro-batches, nothing fits)
+// Micro-batch pairs among shared segments.  Classes of pair heads are formed at non-overlapping
+// micro-batch counts (m, m+1), (m+2, m+3), .. of a (stages, peers) group; a head of such a class
+// is keyed in the class's table and searched together with its next row.  Every other row first
+// looks its tier up in the pair class that would hold it as a head (its own m) and in the one
+// that would hold it as a second row (m - 1); only if neither has it is it keyed in the class of
+// single segments of its m.  So every distinct (stages, m, peers, tiers) is searched once.
+constexpr uint32_t kPartnerSeg = 0xfffffffeu;   // second row of a keyed pair head: takes the row after its head's representative
+constexpr uint32_t kSecondRowFlag = 0x80000000u;   // in slot_of: the row after the slot's representative holds this row's result
 struct USegClass {
     uint32_t tab_first, tab_mask;   // its table: slots tab_first .. tab_first + tab_mask (a power of two of them)
     uint32_t list_first, pad;       // its distinct segments: list entries list_first .. list_first + count - 1
 };
 struct USegDev {
     const USegClass *cls;
-    const uint32_t *tseg_cls;       // class of every template segment (kNoSegClass: none)
+    const uint32_t *tseg_cls;       // class of every template segment (kNoSegClass: none; kPartnerSeg: rides with the row before)
+    const uint32_t *look_head;      // per template segment that is not a keyed pair head: the pair class of its own m, or kNoSegClass
+    const uint32_t *look_part;      //   and the pair class of m - 1
     unsigned long long *tab;        // tier words, all-ones = empty
     uint32_t *rep;                  // per slot: lowest row with that key
     uint32_t *slot_of;              // per row: its slot (kNoSegClass: none)
     uint32_t *count;                // per class: distinct segments; count[n_cls]: probes that found no slot (never)
     uint2 *list;                    // (scenario, template segment) of every distinct segment, by class
     uint32_t n_cls, n_rep_scen;
+    uint32_t n_pair_cls;            // classes 0 .. n_pair_cls-1 are the pair classes
 };
 
 // Buckets that one kernel instantiation handles.  Plan-major classes cut a bucket's
@@ -278,7 +289,7 @@ cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *key
 cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaStream_t st);
 // segments shared between scenarios: key every row and list the distinct ones (tab, rep, count
 // cleared by the caller); after the search pass, give every other row its representative's result
-cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st);
+cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st);   // three launches
 cudaError_t launch_useg_copy(const BatchDev &b, const USegDev &u, cudaStream_t st);
 // Tiles of a segment that the tie-break kernels take side by side (grid.y); the rest is
 // walked serially inside the CTA.  A single scenario gets every tile its own CTA (lowest

@@ -215,27 +215,53 @@ __device__ __forceinline__ uint32_t mix64(uint64_t x) {
     return (uint32_t)x;
 }
 
-__global__ void __launch_bounds__(128) cm_useg_key_kernel(BatchDev bd, USegDev ud) {
+// phase 0: the heads of the pair classes; phase 1 (a launch of its own, after phase 0 is complete):
+// every other row, which joins a pair it finds in the tables of phase 0 before it is keyed itself
+__device__ __forceinline__ uint32_t useg_find(const USegDev &ud, const USegClass &c, unsigned long long tier) {
+    uint32_t h = mix64(tier) & c.tab_mask;
+    for (uint32_t probe = 0; probe <= c.tab_mask; ++probe) {
+        const unsigned long long v = ud.tab[c.tab_first + h];
+        if (v == tier) return c.tab_first + h;
+        if (v == ~0ull) break;
+        h = (h + 1) & c.tab_mask;
+    }
+    return kNoSegClass;
+}
+
+__global__ void __launch_bounds__(128) cm_useg_key_kernel(BatchDev bd, USegDev ud, int phase) {
     const uint32_t scen_id = bd.tmpl_scen[blockIdx.x];
     const Scen sc = bd.scen[scen_id];
     const Tmpl tp = bd.tmpl[sc.tmpl];
     for (uint32_t i = threadIdx.x; i < tp.n_tseg; i += blockDim.x) {
         const uint32_t trow = tp.tseg_first + i, row = sc.seg_base + i;
         const uint32_t ci = ud.tseg_cls[trow];
-        uint32_t slot = kNoSegClass;
-        if (ci != kNoSegClass) {
-            const TSeg g = bd.tseg[trow];
-            const USegClass c = ud.cls[ci];
-            const unsigned long long tier = cut_bits(bd.cross + sc.cross_first, g.off, g.S - 1);   // < 2^63: never all-ones
-            uint32_t h = mix64(tier) & c.tab_mask;
-            for (uint32_t probe = 0; probe <= c.tab_mask; ++probe) {
-                const unsigned long long old = atomicCAS(&ud.tab[c.tab_first + h], ~0ull, tier);
-                if (old == ~0ull || old == tier) { slot = c.tab_first + h; break; }
-                h = (h + 1) & c.tab_mask;
-            }
-            if (slot == kNoSegClass) atomicAdd(&ud.count[ud.n_cls], 1u);   // (no free slot: cannot happen)
-            else atomicMin(&ud.rep[slot], row);
+        if (ci == kNoSegClass || ci == kPartnerSeg) {
+            if (phase == 0) ud.slot_of[row] = ci;
+            continue;
         }
+        if ((ci < ud.n_pair_cls) != (phase == 0)) continue;
+        const TSeg g = bd.tseg[trow];
+        const unsigned long long tier = cut_bits(bd.cross + sc.cross_first, g.off, g.S - 1);   // < 2^63: never all-ones
+        if (phase == 1) {
+            uint32_t found = kNoSegClass;
+            const uint32_t lh = ud.look_head[trow], lp = ud.look_part[trow];
+            if (lh != kNoSegClass) found = useg_find(ud, ud.cls[lh], tier);
+            if (found == kNoSegClass && lp != kNoSegClass) {
+                found = useg_find(ud, ud.cls[lp], tier);
+                if (found != kNoSegClass) found |= kSecondRowFlag;
+            }
+            if (found != kNoSegClass) { ud.slot_of[row] = found; continue; }
+        }
+        const USegClass c = ud.cls[ci];
+        uint32_t slot = kNoSegClass;
+        uint32_t h = mix64(tier) & c.tab_mask;
+        for (uint32_t probe = 0; probe <= c.tab_mask; ++probe) {
+            const unsigned long long old = atomicCAS(&ud.tab[c.tab_first + h], ~0ull, tier);
+            if (old == ~0ull || old == tier) { slot = c.tab_first + h; break; }
+            h = (h + 1) & c.tab_mask;
+        }
+        if (slot == kNoSegClass) atomicAdd(&ud.count[ud.n_cls], 1u);   // (no free slot: cannot happen)
+        else atomicMin(&ud.rep[slot], row);
         ud.slot_of[row] = slot;
     }
 }
@@ -247,8 +273,8 @@ __global__ void __launch_bounds__(128) cm_useg_list_kernel(BatchDev bd, USegDev 
     for (uint32_t i = threadIdx.x; i < tp.n_tseg; i += blockDim.x) {
         const uint32_t trow = tp.tseg_first + i, row = sc.seg_base + i;
         const uint32_t slot = ud.slot_of[row];
-        if (slot == kNoSegClass || ud.rep[slot] != row) continue;
-        const uint32_t ci = ud.tseg_cls[trow];
+        if (slot == kNoSegClass || slot == kPartnerSeg || (slot & kSecondRowFlag) || ud.rep[slot] != row) continue;
+        const uint32_t ci = ud.tseg_cls[trow];   // a representative was keyed in its own class
         const uint32_t pos = atomicAdd(&ud.count[ci], 1u);
         ud.list[ud.cls[ci].list_first + pos] = make_uint2(scen_id, trow);
     }
@@ -257,15 +283,24 @@ __global__ void __launch_bounds__(128) cm_useg_list_kernel(BatchDev bd, USegDev 
 __global__ void __launch_bounds__(256) cm_useg_copy_kernel(BatchDev bd, USegDev ud) {
     const uint32_t row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= bd.n_rows) return;
-    const uint32_t slot = ud.slot_of[row];
+    uint32_t slot = ud.slot_of[row];
     if (slot == kNoSegClass) return;
-    const uint32_t r = ud.rep[slot];
-    if (r != row) bd.seg_best[row] = bd.seg_best[r];   // representatives are only read here
+    uint32_t second = 0;
+    if (slot == kPartnerSeg) {   // second row of a keyed pair head
+        slot = ud.slot_of[row - 1];
+        second = 1;
+    } else if (slot & kSecondRowFlag) {
+        slot &= ~kSecondRowFlag;
+        second = 1;
+    }
+    const uint32_t r = ud.rep[slot] + second;
+    if (r != row) bd.seg_best[row] = bd.seg_best[r];   // representatives and their second rows are only read here
 }
 
 cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st) {
     if (u.n_rep_scen == 0) return cudaSuccess;
-    cm_useg_key_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u);
+    cm_useg_key_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u, 0);
+    cm_useg_key_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u, 1);
     cm_useg_list_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u);
     return cudaGetLastError();
 }
