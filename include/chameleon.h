@@ -395,7 +395,8 @@ cm_status cm_set_micro_batch_pairs(cm_ctx *ctx, int on);
  * micro-batches, the data-parallel peers of its strategy and the link tiers of its stage
  * boundaries only (Section "Estimator"), so the distinct such tuples of the batch are found on
  * the device (one small device->host copy and one synchronisation of the context's stream per
- * prepared batch) and each is searched once.  A single failure set searched through the latency
+ * prepared batch) and each is searched once (as one half of a micro-batch pair where two distinct
+ * pipelines differ only by one micro-batch).  A single failure set searched through the latency
  * path of cm_search_batch has its duplicate pipelines removed on the host when enough work is
  * saved to pay for launching its sequence directly instead of replaying the resident graph.
  * Results are identical either way; cm_last_stats
