@@ -385,6 +385,17 @@ cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
  * segment on its own. */
 cm_status cm_set_micro_batch_pairs(cm_ctx *ctx, int on);
 
+/* Pipeline reuse (on by default).  The strategies of one survivor count have pipelines in
+ * common: the stage tuples (30, 31, ..) and (30, 32, ..) both start with 30 stages over the first
+ * 30 survivors, with the same micro-batch counts and the same number of data-parallel peers.
+ * Such a pipeline has the same candidates with the same costs whatever strategy it is part of
+ * (Section "Estimator": a pipeline's time and memory are functions of its own stages, links and
+ * micro-batches), so its least cost is searched once per scenario and the other strategies take
+ * the result.  Results are identical; cm_last_stats [0] still counts every pipeline-plan of the
+ * search space, [16] those whose recurrence ran.  cm_set_pipeline_reuse(ctx, 0) makes batches and
+ * spaces built afterwards search every (strategy, pipeline) on its own. */
+cm_status cm_set_pipeline_reuse(cm_ctx *ctx, int on);
+
 /* Sharing (off by default): in a batch, failure sets that leave the same number of survivors
  * with node boundaries at the same places among them have identical dynamic-parallelism
  * searches -- survivors are placed in consecutive blocks and nothing else of the failure set

@@ -31,9 +31,9 @@ EXPORTS = ["cm_create", "cm_destroy", "cm_load_profile", "cm_enumerate", "cm_eva
            "cm_batch_free", "cm_evaluate_argmin_noalloc", "cm_last_stats", "cm_search_objective",
            "cm_objective_stats", "cm_transfer_matching", "cm_cache_build", "cm_cache_lookup", "cm_cache_free",
            "cm_set_sharing", "cm_set_int64_arithmetic", "cm_host_describe", "cm_set_latency_graphs",
-           "cm_transition_time", "cm_set_memory_screen", "cm_set_micro_batch_pairs", "cm_int64_runs_in_fp64", "cm_strerror",
-           "cm_last_error"]
-_STATUS_CALLS = EXPORTS[:27]
+           "cm_transition_time", "cm_set_memory_screen", "cm_set_micro_batch_pairs", "cm_set_pipeline_reuse", "cm_int64_runs_in_fp64",
+           "cm_strerror", "cm_last_error"]
+_STATUS_CALLS = EXPORTS[:28]
 NOALLOC_MAX_CANDIDATES = 524288
 MAX_SHORTLIST, MAX_MATCH = 16, 256
 
@@ -159,6 +159,7 @@ def load_library() -> C.CDLL:
     lib.cm_set_latency_graphs.argtypes = [vp, C.c_int]
     lib.cm_set_memory_screen.argtypes = [vp, C.c_int]
     lib.cm_set_micro_batch_pairs.argtypes = [vp, C.c_int]
+    lib.cm_set_pipeline_reuse.argtypes = [vp, C.c_int]
     lib.cm_host_describe.argtypes = [C.POINTER(cm_profile), C.POINTER(C.c_uint32), C.c_int32, C.POINTER(cm_enum_opts), u64p]
     lib.cm_set_int64_arithmetic.argtypes = [vp, C.c_int]
     lib.cm_transition_time.argtypes = [C.POINTER(cm_objective_opts), C.c_int32, C.POINTER(C.c_int64),
@@ -407,6 +408,11 @@ def cm_set_sharing(ctx, on: bool) -> None:
 def cm_set_micro_batch_pairs(ctx, on: bool) -> None:
     """One recurrence for a pipeline's m and m+1 micro-batch variants (on by default)."""
     _check(ctx, load_library().cm_set_micro_batch_pairs(ctx, int(bool(on))))
+
+
+def cm_set_pipeline_reuse(ctx, on: bool) -> None:
+    """Search a pipeline that several strategies of a survivor count have in common once (on by default)."""
+    _check(ctx, load_library().cm_set_pipeline_reuse(ctx, int(bool(on))))
 
 
 def cm_set_memory_screen(ctx, on: bool) -> None:

@@ -80,6 +80,9 @@ struct Batch {
     std::vector<Strat> strat;
     std::vector<TSeg> tseg;
     std::vector<uint32_t> failed, red_scen, keys, tmpl_scen, bucket_tseg;
+    std::vector<uint32_t> tseg_canon;      // first template segment with the same (stages, micro-batches, peers, offset): itself if none before
+    uint32_t n_dup = 0;                    // template segments that are not their own first occurrence
+    size_t off_canon = 0;
     std::vector<uint64_t> cross;
     std::vector<Bucket> bucket;
     std::vector<LaunchClass> classes;
@@ -183,6 +186,7 @@ struct cm_ctx {
     PinnedVec<unsigned char> feas_stage;      // keys, K, offsets out; counts back
     DevBuf<unsigned char> d_feas_stage;
     bool screen = true;               // walk only the listed feasible compositions (cm_set_memory_screen)
+    bool dedup = true;                // search a pipeline that several strategies of a survivor count share once (cm_set_pipeline_reuse)
     bool pairs = true;                // one recurrence for a pipeline's m and m+1 micro-batch variants (cm_set_micro_batch_pairs)
     Batch batch;                      // reused by cm_search_batch
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -323,6 +327,7 @@ void mark_pairs(const cm_ctx *ctx, Batch &bt) {
         for (uint32_t i = 0; i + 1 < tp.n_tseg; ++i) {
             const uint32_t t = tp.tseg_first + i;
             if (bt.role[t] != Batch::kAlone) continue;
+            if (bt.tseg_canon[t] != t || bt.tseg_canon[t + 1] != t + 1) continue;   // a duplicate is not searched at all
             const TSeg &a = bt.tseg[t], &b = bt.tseg[t + 1];
             const bool same_pipe = a.S == b.S && a.off == b.off && a.n_sync == b.n_sync && a.K == b.K && b.m == a.m + 1 &&
                                    b.cand_first == a.cand_first + (a.K ? a.K + 1 : 1);
@@ -358,6 +363,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
     for (const Tmpl &tp : bt.tmpl)
         for (uint32_t i = 0; i < tp.n_tseg && tp.n_scen; ++i) {
             const TSeg &g = bt.tseg[tp.tseg_first + i];
+            if (bt.tseg_canon[tp.tseg_first + i] != tp.tseg_first + i) continue;
             if (g.S > kRegStagesMax && g.K > 0 && g.m >= 1)
                 deep_plans += (g.feas_first != kNoFeasList ? (uint64_t)g.feas_count : g.K + 1) * tp.n_scen;
         }
@@ -391,7 +397,8 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
         }
         idx.clear();
         for (uint32_t i = 0; i < tp.n_tseg; ++i)
-            if (role[tp.tseg_first + i] != Batch::kPairPartner) idx.push_back(tp.tseg_first + i);
+            if (role[tp.tseg_first + i] != Batch::kPairPartner && bt.tseg_canon[tp.tseg_first + i] == tp.tseg_first + i)
+                idx.push_back(tp.tseg_first + i);
         std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
             const TSeg &x = bt.tseg[a], &y = bt.tseg[b];
             return x.S != y.S ? x.S < y.S : x.m != y.m ? x.m < y.m : role[a] < role[b];
@@ -502,7 +509,10 @@ void assign_segment_classes(Batch &bt) {
     bt.look_part.assign(bt.tseg.size(), kNoSegClass);
     bt.ucls_info.clear();
     bt.ucls.clear();
-    auto searched = [](const TSeg &g) { return g.m >= 1 && !(g.feas_first != kNoFeasList && g.feas_count == 0); };
+    auto searched = [&](const TSeg &g) {
+        const uint32_t t = (uint32_t)(&g - bt.tseg.data());
+        return bt.tseg_canon[t] == t && g.m >= 1 && !(g.feas_first != kNoFeasList && g.feas_count == 0);
+    };
     auto key_of = [](const TSeg &g, uint16_t m) { return ((uint64_t)g.S << 32) | ((uint64_t)m << 16) | g.n_sync; };
     // pair classes first: the micro-batch counts at which pair heads occur, per (stages, peers),
     // taken greedily from the lowest so that no two pair classes overlap
@@ -710,6 +720,19 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
     }
     tp.n_strat = (uint32_t)bt.strat.size() - tp.strat_first;
     tp.n_tseg = (uint32_t)bt.tseg.size() - tp.tseg_first;
+    // pipelines that strategies of this survivor count have in common: searched once (BatchDev::tseg_canon)
+    {
+        std::map<uint64_t, uint32_t> first_of;
+        bt.tseg_canon.resize(bt.tseg.size());
+        for (uint32_t i = 0; i < tp.n_tseg; ++i) {
+            const uint32_t t = tp.tseg_first + i;
+            const TSeg &g = bt.tseg[t];
+            const uint64_t key = ((uint64_t)g.S << 48) | ((uint64_t)g.m << 32) | ((uint64_t)g.n_sync << 16) | g.off;
+            const uint32_t c = ctx->dedup ? first_of.emplace(key, t).first->second : t;
+            bt.tseg_canon[t] = c;
+            if (c != t) ++bt.n_dup;
+        }
+    }
     tp.n_split_total = split_first;
     tp.n_cand = cand;
     tp.n_red = split_first ? (uint32_t)std::min<uint64_t>((split_first + 1023) / 1024, 64) : 0;
@@ -813,7 +836,8 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     const DevProfile &hp = ctx->hp;
     const int N = hp.n_dp * hp.n_pp;
     bt.scen.clear(); bt.tmpl.clear(); bt.strat.clear(); bt.tseg.clear(); bt.failed.clear(); bt.red_scen.clear();
-    bt.keys.clear(); bt.tmpl_scen.clear(); bt.cross.clear();
+    bt.keys.clear(); bt.tmpl_scen.clear(); bt.cross.clear(); bt.tseg_canon.clear();
+    bt.n_dup = 0;
     bt.opts = o;
     bt.profile_gen = ctx->profile_gen;
     bt.intval = o.cost == CM_COST_INT64NS && ctx->exact53 && !ctx->force_native_i64;
@@ -962,6 +986,9 @@ BatchDev dev_view(const cm_ctx *ctx, Batch &bt) {
     v.bucket_tseg = (const uint32_t *)(a + bt.off_bucket_tseg); v.red_scen = (const uint32_t *)(a + bt.off_red);
     v.feas = ctx->d_feas.p;
     v.useg = bt.d_useg.p;
+    v.tseg_canon = bt.n_dup ? (const uint32_t *)(a + bt.off_canon) : nullptr;
+    v.n_rep_scen = 0;
+    for (const Tmpl &tp : bt.tmpl) v.n_rep_scen += tp.n_scen;
     v.seg_best = bt.d_seg_best.p; v.partial = bt.d_partial.p;
     v.winner = bt.d_winner.p; v.kappa_sel = bt.d_kappa_sel.p; v.pol_cost = bt.d_pol_cost.p;
     v.rc_stages = bt.d_rc_stages.p; v.plans = bt.d_plans.p;
@@ -1020,6 +1047,7 @@ cm_status upload_batch(cm_ctx *ctx, Batch &bt, int *launches) {
     bt.off_tmpl_scen = arena_put(bt.arena, bt.tmpl_scen, ok);
     bt.off_bucket_tseg = arena_put(bt.arena, bt.bucket_tseg, ok);
     bt.off_cross = arena_put(bt.arena, bt.cross, ok);
+    bt.off_canon = arena_put(bt.arena, bt.tseg_canon, ok);
     bt.off_ucls = arena_put(bt.arena, bt.ucls, ok);
     bt.off_tseg_cls = arena_put(bt.arena, bt.tseg_cls, ok);
     bt.off_look_head = arena_put(bt.arena, bt.look_head, ok);
@@ -1097,6 +1125,10 @@ cm_status enqueue_search(cm_ctx *ctx, Batch &bt, cudaStream_t st, bool phase_eve
         launches += cost_launches;
         if (bt.useg) {   // rows that share a segment take its representative's minimum
             CM_CUDA(ctx, launch_useg_copy(bd, useg_view(bt), st));
+            ++launches;
+        }
+        if (bt.n_dup) {  // pipelines that strategies have in common were searched once
+            CM_CUDA(ctx, launch_dup_copy(bd, st));
             ++launches;
         }
         if (phase_events) CM_CUDA(ctx, cudaEventRecord(ctx->ev[3], st));
@@ -2009,6 +2041,19 @@ cm_status cm_set_micro_batch_pairs(cm_ctx *ctx, int on) {
         ctx->single.clear();
     }
     ctx->pairs = on != 0;
+    return CM_OK;
+    CM_API_END(ctx)
+}
+
+cm_status cm_set_pipeline_reuse(cm_ctx *ctx, int on) {
+    if (!ctx) return CM_EINVAL;
+    CM_API_BEGIN
+    if ((on != 0) != ctx->dedup) {
+        // resident one-scenario batches were laid out under the other setting
+        if (ctx->stream) cudaStreamSynchronize(ctx->stream);
+        ctx->single.clear();
+    }
+    ctx->dedup = on != 0;
     return CM_OK;
     CM_API_END(ctx)
 }

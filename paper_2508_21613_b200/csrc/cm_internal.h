@@ -214,6 +214,13 @@ struct BatchDev {
     const uint32_t *bucket_tseg;  // template segment rows grouped by bucket
     const uint32_t *feas;         // feasible-composition pool of the context
     const uint2 *useg;            // distinct segments of a batch searched with sharing (buckets with tmpl == kSharedBucket)
+    // Strategies of one survivor count repeat pipelines: the same stages over the same survivors with
+    // the same micro-batches and peers (the tuples (30,31,..) and (30,32,..) start with the same
+    // pipeline).  Such template segments have the same candidates with the same costs in every
+    // scenario, so only the first of them -- tseg_canon[t] == t -- is searched; the others take its
+    // per-segment minimum afterwards (cm_dup_copy_kernel).  NULL: the batch has no duplicates.
+    const uint32_t *tseg_canon;
+    uint32_t n_rep_scen;          // scenarios that own result rows (entries of tmpl_scen in use)
     uint64_t *seg_best;     // [n_seg] min cost over kappa, order-preserving bits
     const uint32_t *red_scen;  // [n_red_blocks] scenario of every block of the split reduction
     Partial *partial;       // [n_red_blocks]
@@ -291,6 +298,7 @@ cudaError_t launch_policies(const Tables &t, const BatchDev &b, int n_dp, cudaSt
 // cleared by the caller); after the search pass, give every other row its representative's result
 cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st);   // three launches
 cudaError_t launch_useg_copy(const BatchDev &b, const USegDev &u, cudaStream_t st);
+cudaError_t launch_dup_copy(const BatchDev &b, cudaStream_t st);   // duplicate template segments take their first occurrence's minimum
 // Tiles of a segment that the tie-break kernels take side by side (grid.y); the rest is
 // walked serially inside the CTA.  A single scenario gets every tile its own CTA (lowest
 // latency), a large batch about one CTA per (scenario, pipeline): most of those stop after

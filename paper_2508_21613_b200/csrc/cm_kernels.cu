@@ -297,6 +297,21 @@ __global__ void __launch_bounds__(256) cm_useg_copy_kernel(BatchDev bd, USegDev 
     if (r != row) bd.seg_best[row] = bd.seg_best[r];   // representatives and their second rows are only read here
 }
 
+__global__ void __launch_bounds__(128) cm_dup_copy_kernel(BatchDev bd) {
+    const Scen sc = bd.scen[bd.tmpl_scen[blockIdx.x]];
+    const Tmpl tp = bd.tmpl[sc.tmpl];
+    for (uint32_t i = threadIdx.x; i < tp.n_tseg; i += blockDim.x) {
+        const uint32_t c = bd.tseg_canon[tp.tseg_first + i];
+        if (c != tp.tseg_first + i) bd.seg_best[sc.seg_base + i] = bd.seg_best[sc.seg_base + (c - tp.tseg_first)];
+    }
+}
+
+cudaError_t launch_dup_copy(const BatchDev &b, cudaStream_t st) {
+    if (!b.tseg_canon || b.n_rep_scen == 0) return cudaSuccess;
+    cm_dup_copy_kernel<<<b.n_rep_scen, 128, 0, st>>>(b);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_useg_keys(const BatchDev &b, const USegDev &u, cudaStream_t st) {
     if (u.n_rep_scen == 0) return cudaSuccess;
     cm_useg_key_kernel<<<u.n_rep_scen, 128, 0, st>>>(b, u, 0);
