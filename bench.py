@@ -636,15 +636,22 @@ def main():
             "dtype": ("f64 (integer-valued, exact)" if m["arith"] == 0 else "i64") if args.cost_mode else "f64",
             "data": "synthetic",
             "config": {"workload": w.name, "scenarios": len(w.scenarios), "plans_per_step": m["plans_per_step"],
-                       # plans whose recurrence ran / plans the memory estimator rejected before it
+                       # plans_per_step counts every pipeline-plan of the search space, i.e. every
+                       # (strategy, pipeline, micro-batch count, layer composition), as the oracle
+                       # enumerates them.  Of these: plans_reused belong to pipelines that another
+                       # strategy of the same survivor count has as well and are not searched again;
+                       # plans_memory_rejected fail the memory estimator; plans_simulated ran the recurrence.
+                       "plans_reused_per_step": (m["stats"]["plans"] - m["stats"]["plans_own"]) // args.steps,
+                       "plans_memory_rejected": (m["stats"]["plans_own"] - m["stats"]["plans_simulated"]) // args.steps,
                        "plans_simulated_per_step": m["stats"]["plans_simulated"] // args.steps + 2 * len(w.scenarios),
-                       "plans_memory_rejected": (m["stats"]["plans"] - m["stats"]["plans_simulated"]) // args.steps,
                        "policies": 3, "cost_mode": "int64ns" if args.cost_mode else "fp64",
                        "l2": "flushed between timed iterations (256 MB write)",
                        "parallelism": "replicas, scenarios independent" if world > 1 else "1 gpu"},
             "e2e": {"value": total_plans / max_e2e, "unit": UNIT, "ms_per_step": 1e3 * max_e2e / args.steps,
                     "h2d_bytes_per_step": int(m["h2d"]), "d2h_bytes_per_step": int(m["d2h"]),
                     "timing": "wall clock around cm_search_batch (host descriptor build inside)"},
+            # the same rate counted on the pipeline-plans that are searched in their own right only
+            "value_without_reused_plans": (m["stats"]["plans_own"] + 2 * len(w.scenarios) * args.steps) * world / max_dev,
             "latency_us": m["latency_us"],
             "gpu_launches": int(m["stats"]["launches"]),
             "clocks": m["clocks"],
@@ -673,7 +680,8 @@ def main():
                 r = roofline_of(em["stats"], em["dev_seconds"], em["arith"], kernel_class(ew), em["clocks"], sm_max, peak_kind)
                 extra[f"{name}/{'int64ns' if mode else 'fp64'}"] = {
                     "scenarios": len(ew.scenarios), "steps": n_extra, "plans_per_step": em["plans_per_step"],
-                    "plans_memory_rejected": (em["stats"]["plans"] - em["stats"]["plans_simulated"]) // n_extra,
+                    "plans_reused_per_step": (em["stats"]["plans"] - em["stats"]["plans_own"]) // n_extra,
+                    "plans_memory_rejected": (em["stats"]["plans_own"] - em["stats"]["plans_simulated"]) // n_extra,
                     "plans_per_s": em["plans_per_step"] * n_extra / em["dev_seconds"],
                     "ms_per_step": 1e3 * em["dev_seconds"] / n_extra, "e2e_ms_per_step": 1e3 * em["e2e_seconds"] / n_extra,
                     "latency_us_p50": em["latency_us"]["p50"], "latency_us_p99": em["latency_us"]["p99"],

@@ -469,12 +469,16 @@ cm_status cm_cache_free(cm_cache *cache);
  *  [10] bytes copied device->host   [11] device time of the tie-break kernel(s), ns
  *  [12] launches of the search-pass cost kernel   [13] host time building descriptor tables, ns
  *  [14] host time enqueueing the launch sequence, ns   [15] host time waiting for the stream, ns
- *  [16] pipeline-plans of [0] whose recurrence ran, i.e. that passed the memory estimator
- *       (Section "Estimator", memory estimator); [0] - [16] were rejected by it
+ *  [16] pipeline-plans whose recurrence ran, i.e. that are searched in their own right ([19]) and
+ *       passed the memory estimator (Section "Estimator", memory estimator)
  *  [17] host time spent listing memory-feasible compositions (inside [13]; includes one stream
  *       synchronisation when a new (stages, micro-batches) pair is met), ns
  *  [18] host time packing and uploading the descriptor tables, buffer allocation included, ns
- *  [19..23] reserved, 0. */
+ *  [19] pipeline-plans of [0] that are searched in their own right: [0] - [19] belong to pipelines
+ *       that another strategy of the same survivor count has as well and take its result
+ *       (cm_set_pipeline_reuse); [19] - [16] were rejected by the memory estimator (with sharing
+ *       on, [16] also leaves out what other scenarios' segments already covered)
+ *  [20..23] reserved, 0. */
 cm_status cm_last_stats(const cm_ctx *ctx, uint64_t out[24]);
 
 const char *cm_strerror(cm_status status);

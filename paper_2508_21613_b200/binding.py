@@ -450,7 +450,7 @@ def cm_last_stats(ctx) -> dict:
     keys = ["plans", "cells", "tiebreak_plans", "launches", "device_ns", "segments", "strategies", "splits",
             "cost_kernel_ns", "h2d_bytes", "d2h_bytes", "tiebreak_kernel_ns", "cost_kernel_launches",
             "host_build_ns", "host_enqueue_ns", "host_wait_ns", "plans_simulated", "host_feasible_ns",
-            "host_upload_ns"]
+            "host_upload_ns", "plans_own"]
     return dict(zip(keys, [int(v) for v in out]))
 
 

@@ -113,6 +113,8 @@ struct Batch {
     cm_enum_opts opts{};
     uint32_t policy_mask = 0;
     uint64_t n_cand = 0, n_tiles = 0, n_split = 0;
+    uint64_t n_cand_own = 0;               // candidates of the template segments that are searched in their own right
+    std::vector<uint64_t> tmpl_cand_own;   // the same per template (one scenario)
     uint64_t n_rows = 0;                   // rows of seg_best over all scenarios
     uint32_t max_tiles_per_seg = 0, dp_max = 0;
     int B = 0;
@@ -723,6 +725,7 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
     // pipelines that strategies of this survivor count have in common: searched once (BatchDev::tseg_canon)
     {
         std::map<uint64_t, uint32_t> first_of;
+        uint64_t own = 0;
         bt.tseg_canon.resize(bt.tseg.size());
         for (uint32_t i = 0; i < tp.n_tseg; ++i) {
             const uint32_t t = tp.tseg_first + i;
@@ -731,7 +734,10 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
             const uint32_t c = ctx->dedup ? first_of.emplace(key, t).first->second : t;
             bt.tseg_canon[t] = c;
             if (c != t) ++bt.n_dup;
+            else own = sat_add(own, g.K ? g.K + 1 : 1);
         }
+        bt.tmpl_cand_own.resize(bt.tmpl.size() + 1, 0);
+        bt.tmpl_cand_own[bt.tmpl.size()] = own;
     }
     tp.n_split_total = split_first;
     tp.n_cand = cand;
@@ -843,6 +849,8 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
     bt.intval = o.cost == CM_COST_INT64NS && ctx->exact53 && !ctx->force_native_i64;
     bt.policy_mask = policy_mask;
     bt.n_cand = bt.n_tiles = bt.n_split = bt.n_rows = 0;
+    bt.n_cand_own = 0;
+    bt.tmpl_cand_own.assign(1, 0);   // template 0 has no strategies
     bt.max_tiles_per_seg = 0;
     bt.dp_max = 0;
     bt.B = B;
@@ -940,6 +948,7 @@ cm_status build_batch(cm_ctx *ctx, Batch &bt, const uint32_t *failed_ids, const 
         red += tp.n_red;
         for (uint32_t r = 0; r < tp.n_red; ++r) bt.red_scen.push_back((uint32_t)b);
         bt.n_cand = sat_add(bt.n_cand, tp.n_cand);
+        bt.n_cand_own = sat_add(bt.n_cand_own, bt.tmpl_cand_own[sc.tmpl]);
         bt.n_split = sat_add(bt.n_split, tp.n_split_total);
         if (rows >= (1ull << 31) || red >= (1ull << 31) || bt.n_cand >= (1ull << 62))
             return fail(ctx, CM_EOVERFLOW, "batch too large for the index type");
@@ -1217,6 +1226,7 @@ cm_status run_batch(cm_ctx *ctx, Batch &bt, int launches_so_far, cm_ctx::Single 
     ctx->stats[10] += back_bytes;
     const unsigned long long *counters_host = reinterpret_cast<const unsigned long long *>(bt.plans_host.p + (size_t)bt.B * 4);
     ctx->stats[0] += (bt.policy_mask & (1u << CM_DYNPAR)) ? bt.n_cand : 0;
+    ctx->stats[19] += (bt.policy_mask & (1u << CM_DYNPAR)) ? bt.n_cand_own : 0;
     ctx->stats[1] += counters_host[0];
     ctx->stats[2] += counters_host[1];
     ctx->stats[16] += counters_host[2];
