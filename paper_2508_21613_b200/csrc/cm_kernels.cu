@@ -55,8 +55,11 @@ cudaError_t launch_prefix(DevProfile *prof, cudaStream_t st) {
 // (value, k) with the lowest k on ties closes each cell.  Backtracking follows the
 // stored argmin, which is the smallest k that attains D[l][s].
 // ----------------------------------------------------------------------------------
+// a warp per layer of a DP column: 32 warps take the column of a 96-layer model in three sweeps
+// (the kernel sits on the path of the first search of a survivor count)
+constexpr int kMinmaxThreads = 1024;
 template <typename T>
-__global__ void __launch_bounds__(256) cm_minmax_kernel(Tables tb, const uint32_t *keys, int n_keys) {
+__global__ void __launch_bounds__(kMinmaxThreads) cm_minmax_kernel(Tables tb, const uint32_t *keys, int n_keys) {
     __shared__ T PF[kMaxL + 1], PB[kMaxL + 1];
     __shared__ long long PA[kMaxL + 1], PS[kMaxL + 1];
     __shared__ T D[2][kMaxL + 1];
@@ -127,8 +130,8 @@ __global__ void __launch_bounds__(256) cm_minmax_kernel(Tables tb, const uint32_
 
 cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys, int mode, cudaStream_t st) {
     if (n_keys <= 0) return cudaSuccess;
-    if (mode == CM_COST_INT64NS) cm_minmax_kernel<long long><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
-    else cm_minmax_kernel<double><<<n_keys, 256, 0, st>>>(t, keys_dev, n_keys);
+    if (mode == CM_COST_INT64NS) cm_minmax_kernel<long long><<<n_keys, kMinmaxThreads, 0, st>>>(t, keys_dev, n_keys);
+    else cm_minmax_kernel<double><<<n_keys, kMinmaxThreads, 0, st>>>(t, keys_dev, n_keys);
     return cudaGetLastError();
 }
 
