@@ -11,6 +11,9 @@
 //   cm_finalize_kernel    assembles the plans and picks the best policy
 //   cm_evaluate_kernel    per-candidate cost / feasibility for cm_evaluate
 //   cm_pick_kernel        best of several spaces for cm_select
+#include <algorithm>
+#include <atomic>
+
 #include "cm_plan_eval.cuh"
 
 namespace cm {
@@ -146,12 +149,18 @@ cudaError_t launch_minmax(const Tables &t, const uint32_t *keys_dev, int n_keys,
 constexpr int kFeasThreads = 1024;
 __global__ void __launch_bounds__(kFeasThreads) cm_feasible_kernel(Tables tb, int layer_mode, const uint32_t *keys,
                                                                    const uint64_t *Ks, const uint32_t *first,
-                                                                   uint32_t *pool, uint32_t *count_out) {
+                                                                   uint32_t *pool, uint32_t *count_out, int binom_rows_staged) {
     __shared__ long long PA[kMaxL + 1], PS[kMaxL + 1];
     __shared__ uint32_t warp_cnt[kFeasThreads / 32];
     __shared__ uint32_t running;
+    // the rows of the binomial table that unranking reads (n <= stages under the remainder rule,
+    // n < layers under the full enumeration), staged once: a rank is unranked through ~S dependent
+    // look-ups, and this kernel sits on the path of the first search of a survivor count
+    extern __shared__ uint64_t binom_s[];
     const DevProfile *p = tb.prof;
     const int L = p->L;
+    for (int q = threadIdx.x; q < binom_rows_staged * (kBinomCols + 1); q += blockDim.x) binom_s[q] = tb.binom[q];
+    tb.binom = binom_s;
     const uint32_t key = keys[blockIdx.x];
     const int S = (int)(key >> 16), m = (int)(key & 0xffffu);
     const uint64_t K = Ks[blockIdx.x];
@@ -198,7 +207,19 @@ __global__ void __launch_bounds__(kFeasThreads) cm_feasible_kernel(Tables tb, in
 cudaError_t launch_feasible(const Tables &t, int layer_mode, const uint32_t *keys_dev, const uint64_t *K_dev,
                             const uint32_t *first_dev, int n_keys, uint32_t *pool, uint32_t *count_dev, cudaStream_t st) {
     if (n_keys <= 0) return cudaSuccess;
-    cm_feasible_kernel<<<n_keys, kFeasThreads, 0, st>>>(t, layer_mode, keys_dev, K_dev, first_dev, pool, count_dev);
+    // rows 0 .. 64 (remainder rule: n <= CM_MAX_STAGES) or 0 .. 127 (full enumeration: n < CM_MAX_LAYERS)
+    const int rows = std::min(t.binom_rows, layer_mode == CM_LAYERS_REMAINDER ? kMaxS + 1 : kMaxL);
+    const size_t smem = (size_t)rows * (kBinomCols + 1) * sizeof(uint64_t);
+    static std::atomic<uint64_t> configured{0};   // one bit per device, as for the deep cost kernels
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 64 || !((configured.load(std::memory_order_acquire) >> dev) & 1ull)) {
+        cudaError_t e = cudaFuncSetAttribute(cm_feasible_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)((size_t)kMaxL * (kBinomCols + 1) * sizeof(uint64_t)));
+        if (e != cudaSuccess) return e;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
+    }
+    cm_feasible_kernel<<<n_keys, kFeasThreads, smem, st>>>(t, layer_mode, keys_dev, K_dev, first_dev, pool, count_dev, rows);
     return cudaGetLastError();
 }
 
