@@ -378,8 +378,9 @@ cm_status cm_set_memory_screen(cm_ctx *ctx, int on);
  * counts, m and m + 1 (the two shares the remainder rule leaves it; consecutive counts under the
  * full split enumeration).  Under the 1F1B order the recurrences of the two coincide in every
  * round before the ramp-down of the shorter one -- whether micro-batch m exists shows first in
- * round m -- so for pipelines of 17 to 48 stages with m >= stages one thread evaluates both: the
- * common rounds once, then the two tails.  Same operations on the same values: results are
+ * round m -- so for pipelines of up to 48 stages with m >= stages one thread evaluates both: the
+ * common rounds once, then the two tails (shallow pipelines, up to 16 stages, where a group of
+ * them holds enough plans to be worth a launch of its own).  Same operations on the same values: results are
  * bit-identical; cm_last_stats [1] counts the recurrence cells that actually ran.
  * cm_set_micro_batch_pairs(ctx, 0) makes batches and spaces built afterwards evaluate every
  * segment on its own. */
