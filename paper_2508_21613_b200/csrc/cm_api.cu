@@ -8,6 +8,7 @@
 #include <algorithm>
 #include <chrono>
 #include <map>
+#include <unordered_map>
 #include <memory>
 #include <cmath>
 #include <cstdio>
@@ -379,7 +380,7 @@ cm_status build_buckets(cm_ctx *ctx, Batch &bt) {
         // the transposed or the per-lane kernel (not where the batch's few deep plans go a warp per
         // plan), shallow ones where the group holds enough plans to be worth a launch of its own
         {
-            std::map<uint32_t, uint32_t> heads;   // (S << 16 | m) -> pair heads of the template
+            std::unordered_map<uint32_t, uint32_t> heads;   // (S << 16 | m) -> pair heads of the template
             for (uint32_t i = 0; i < tp.n_tseg; ++i)
                 if (role[tp.tseg_first + i] == Batch::kPairHead) {
                     const TSeg &g = bt.tseg[tp.tseg_first + i];
@@ -724,7 +725,8 @@ cm_status build_template(cm_ctx *ctx, Batch &bt, int n_surv, uint32_t *out) {
     tp.n_tseg = (uint32_t)bt.tseg.size() - tp.tseg_first;
     // pipelines that strategies of this survivor count have in common: searched once (BatchDev::tseg_canon)
     {
-        std::map<uint64_t, uint32_t> first_of;
+        std::unordered_map<uint64_t, uint32_t> first_of;
+        first_of.reserve(2 * (size_t)tp.n_tseg);
         uint64_t own = 0;
         bt.tseg_canon.resize(bt.tseg.size());
         for (uint32_t i = 0; i < tp.n_tseg; ++i) {
